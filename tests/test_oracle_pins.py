@@ -1,0 +1,343 @@
+"""Pins of the CPU oracle against things other than itself (no GPU needed).
+
+Each test is chosen so that a plausible mistake in the oracle (a dropped term, a wrong sign or index,
+a transposed operand, a wrong schedule rule) fails at least one of them.
+"""
+import os
+
+import numpy as np
+import pytest
+
+from workloads import ir, data, params as wp
+import helpers as H
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+FAMILIES = ["mlp", "rnn", "tree", "ggnn"]
+BIG = 1 << 30
+
+
+def make(oracle_mod, g, inst, p):
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst)
+    o.set_params(p)
+    return o
+
+
+# ---------------------------------------------------------------------------------------------------
+# gradients: message-driven backprop == autograd of an independently written recursion / dense form
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("family", FAMILIES)
+def test_accumulators_equal_autograd_of_direct_formulation(oracle_mod, family):
+    g, inst, p = H.tiny_case(family, n=4)
+    o = make(oracle_mod, g, inst, p)
+    st, loss = o.run_epoch(mak=1, muf=BIG, lr=0.1, flush=False)
+    grads, losses = H.dataset_grad(g, p, inst)
+    np.testing.assert_allclose(loss, losses, rtol=1e-12, atol=1e-13)
+    for (node, which), gr in grads.items():
+        np.testing.assert_allclose(o.get_accum(node, which), gr, rtol=1e-9, atol=1e-12,
+                                   err_msg=f"{family} node {g.names[node]} which {which}")
+    assert st.leftover_cache_entries == 0
+
+
+@pytest.mark.parametrize("family", FAMILIES)
+def test_accumulators_equal_finite_differences(oracle_mod, family):
+    """Central differences of the independent loss; touches every parameter tensor."""
+    g, inst, p = H.tiny_case(family, n=2, seed=3)
+    o = make(oracle_mod, g, inst, p)
+    o.run_epoch(mak=2, muf=BIG, lr=0.0, flush=False)
+    import torch
+    rng = np.random.default_rng(0)
+
+    def total(pp):
+        P = {k: torch.tensor(v, dtype=torch.float64) for k, v in pp.items()}
+        return float(sum(H.LOSS_FNS[g.name](g, P, inst, i) for i in range(inst.n)))
+
+    eps = 1e-6
+    for key, v in p.items():
+        acc = o.get_accum(*key)
+        flat = v.ravel()
+        for idx in rng.choice(flat.size, size=min(4, flat.size), replace=False):
+            pp = {k: a.copy() for k, a in p.items()}
+            pp[key].ravel()[idx] += eps
+            up = total(pp)
+            pp[key].ravel()[idx] -= 2 * eps
+            dn = total(pp)
+            fd = (up - dn) / (2 * eps)
+            assert abs(acc.ravel()[idx] - fd) <= 1e-6 * max(1.0, abs(fd)), (family, key, idx)
+
+
+# ---------------------------------------------------------------------------------------------------
+# update rule + schedule: exact agreement with textbook (minibatch) SGD for the MLP when mak = 1
+# ---------------------------------------------------------------------------------------------------
+def _textbook_sgd(g, p, inst, lr, batch):
+    """20-line SGD loop: mean gradient over consecutive batches, numpy fp64, manual backprop."""
+    nodes = g.ppt_nodes()
+    W = [p[(n, 0)].copy() for n in nodes]
+    b = [p[(n, 1)].copy() for n in nodes]
+    losses = []
+    for s in range(0, inst.n, batch):
+        gW = [np.zeros_like(w) for w in W]
+        gb = [np.zeros_like(v) for v in b]
+        idx = range(s, min(s + batch, inst.n))
+        for i in idx:
+            xs = [inst.dense[i].astype(np.float64)]
+            for k in range(len(W)):
+                z = W[k] @ xs[-1] + b[k]
+                xs.append(np.maximum(z, 0) if k < len(W) - 1 else z)
+            y = xs[-1]
+            lse = np.log(np.exp(y - y.max()).sum()) + y.max()
+            losses.append(lse - y[inst.labels_i[i]])
+            d = np.exp(y - lse)
+            d[inst.labels_i[i]] -= 1
+            for k in reversed(range(len(W))):
+                if k < len(W) - 1:
+                    d = d * (xs[k + 1] > 0)
+                gW[k] += np.outer(d, xs[k])
+                gb[k] += d
+                d = W[k].T @ d
+        for k in range(len(W)):
+            W[k] -= lr * gW[k] / len(idx)
+            b[k] -= lr * gb[k] / len(idx)
+    return W, b, np.array(losses)
+
+
+@pytest.mark.parametrize("batch", [1, 4, 5])
+def test_mlp_mak1_is_textbook_minibatch_sgd(oracle_mod, batch):
+    g = ir.mlp((12, 9, 7, 4))
+    inst = data.mlp_instances(n=13, dim=12, classes=4)
+    p = wp.init_params(g)
+    lr = float(np.float32(0.1))
+    o = make(oracle_mod, g, inst, p)
+    st, loss = o.run_epoch(mak=1, muf=batch, lr=lr)
+    W, b, ref_loss = _textbook_sgd(g, p, inst, lr, batch)
+    np.testing.assert_allclose(loss, ref_loss, rtol=1e-12)
+    for k, n in enumerate(g.ppt_nodes()):
+        np.testing.assert_allclose(o.get_params(n, 0), W[k], rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(o.get_params(n, 1), b[k], rtol=1e-12, atol=1e-14)
+        assert o.node_stats(n)["n_updates"] == -(-inst.n // batch)      # includes the epoch-end flush
+    assert st.max_staleness == 0
+
+
+def test_flush_applies_mean_of_accumulated_gradients(oracle_mod):
+    g, inst, p = H.tiny_case("tree", n=3)
+    lr = float(np.float32(0.05))
+    o = make(oracle_mod, g, inst, p)
+    o.run_epoch(mak=1, muf=BIG, lr=lr, flush=True)
+    grads, _ = H.dataset_grad(g, p, inst)
+    L = (np.diff(inst.offsets) + 1) // 2
+    n_grad = {"lookup": L.sum(), "leaf_cell": L.sum(), "branch_cell": (L - 1).sum(), "classifier": (2 * L - 1).sum()}
+    for (node, which), gr in grads.items():
+        want = p[(node, which)] - lr * gr / n_grad[g.names[node]]
+        np.testing.assert_allclose(o.get_params(node, which), want, rtol=1e-10, atol=1e-13)
+
+
+# ---------------------------------------------------------------------------------------------------
+# schedule: hand traces, key bookkeeping, closed-form message counts
+# ---------------------------------------------------------------------------------------------------
+def test_trace_a_mlp_schedule(oracle_mod):
+    rows = H.read_golden(os.path.join(GOLD, "trace_a_mlp.txt"))
+    keylog = np.array(rows[:3], dtype=np.int64)
+    rounds, msgs, ppt, upd, stale = (int(v) for v in rows[3])
+    g = ir.mlp((8, 6, 6, 3))
+    inst = data.mlp_instances(n=3, dim=8, classes=3)
+    o = make(oracle_mod, g, inst, wp.init_params(g))
+    st, _ = o.run_epoch(mak=2, muf=1, lr=0.1)
+    got = np.stack([a.astype(np.int64) for a in o.key_log()], axis=1)
+    np.testing.assert_array_equal(got, keylog)
+    assert (st.rounds, st.node_messages, st.ppt_messages, st.max_staleness) == (rounds, msgs, ppt, stale)
+    assert [o.node_stats(n)["n_updates"] for n in g.ppt_nodes()] == [upd] * 3
+
+
+def test_trace_b_tree_schedule(oracle_mod):
+    rows = H.read_golden(os.path.join(GOLD, "trace_b_tree.txt"))
+    keylog = np.array(rows[:1], dtype=np.int64)
+    rounds, msgs, fwd, bwd, cls_upd, cls_stale = (int(v) for v in rows[1])
+    g = ir.tree(vocab=10, emb=4, hidden=3, classes=2)
+    inst = data.tree_instances(n=1, min_leaves=2, max_leaves=2, vocab=10, classes=2)
+    o = make(oracle_mod, g, inst, wp.init_params(g))
+    st, _ = o.run_epoch(mak=1, muf=1, lr=0.1)
+    got = np.stack([a.astype(np.int64) for a in o.key_log()], axis=1)
+    np.testing.assert_array_equal(got, keylog)
+    assert (st.rounds, st.node_messages) == (rounds, msgs)
+    stats = [o.node_stats(i) for i in range(len(g.names))]
+    assert sum(s["fwd_msgs"] for s in stats) == fwd and sum(s["bwd_msgs"] for s in stats) == bwd
+    c = stats[g.index("classifier")]
+    assert c["n_updates"] == cls_upd
+    assert np.nonzero(c["staleness_hist"])[0].max() == cls_stale
+
+
+def _counts(inst):
+    N = np.diff(inst.offsets) if inst.offsets is not None else None
+    return N
+
+
+@pytest.mark.parametrize("mak,muf", [(1, 1), (3, 7), (16, 50)])
+def test_closed_form_message_counts_and_bookkeeping(oracle_mod, mak, muf):
+    cases = []
+    g = ir.mlp((8, 6, 6, 3))
+    inst = data.mlp_instances(n=11, dim=8, classes=3)
+    cases.append((g, inst, 7 * inst.n, {n: inst.n for n in g.ppt_nodes()}))
+    g = ir.rnn(emb=6, hidden=6)
+    inst = data.list_instances(n=9, max_len=6)
+    T = np.diff(inst.offsets)
+    cases.append((g, inst, int((13 * T + 3).sum()),
+                  {g.index("lookup"): T.sum(), g.index("linear1"): T.sum(), g.index("linear2"): inst.n}))
+    g = ir.tree(vocab=30, emb=6, hidden=5, classes=3)
+    inst = data.tree_instances(n=7, min_leaves=2, max_leaves=9, vocab=30, classes=3)
+    L = (np.diff(inst.offsets) + 1) // 2
+    cases.append((g, inst, int((33 * L - 18).sum()),
+                  {g.index("lookup"): L.sum(), g.index("leaf_cell"): L.sum(), g.index("branch_cell"): (L - 1).sum(),
+                   g.index("classifier"): (2 * L - 1).sum()}))
+    g = ir.ggnn(hidden=4, readout=3)
+    inst = data.graph_instances(n=6, min_nodes=3, max_nodes=7)
+    N, D = np.diff(inst.offsets), np.diff(inst.edge_offsets)
+    Dc = np.array([[np.sum(inst.edge_type[inst.edge_offsets[i]:inst.edge_offsets[i + 1]] == c) for c in range(4)]
+                   for i in range(inst.n)])
+    Cp = (Dc > 0).sum(1)
+    grads = {g.index("lookup"): N.sum(), g.index("gru"): 4 * N.sum(), g.index("readout1"): inst.n,
+             g.index("readout2"): inst.n}
+    for c in range(4):
+        grads[g.index(f"edge_linear{c}")] = 4 * Dc[:, c].sum()
+    # per propagation step: forward 3N+2D+4Cp+8 and backward 3N+2D+4Cp+8 consumed messages; 9 outside the loop
+    cases.append((g, inst, int((4 * (6 * N + 4 * D + 8 * Cp + 16) + 9).sum()), grads))
+    for g, inst, want_msgs, want_grads in cases:
+        o = make(oracle_mod, g, inst, wp.init_params(g))
+        st, _ = o.run_epoch(mak=mak, muf=muf, lr=0.01)
+        assert st.node_messages == want_msgs, g.name
+        assert st.leftover_cache_entries == 0, g.name            # forward/backward state invariant
+        assert 1 <= st.max_active_observed <= mak
+        ins, slot, adm, rel = o.key_log()
+        assert sorted(ins.tolist()) == list(range(inst.n))       # admitted and released exactly once
+        assert (rel > adm).all() and slot.max() < mak
+        # a slot is never handed out again before it was released
+        for s in range(mak):
+            m = slot == s
+            a, r = adm[m], rel[m]
+            assert (a[1:] >= r[:-1]).all()
+        for node, G in want_grads.items():                       # every gradient applied exactly once
+            ns = o.node_stats(node)
+            log = o.update_log(node)
+            assert ns["n_grads_applied"] == G == log.sum(), (g.name, g.names[node])
+            if g.name != "ggnn":                                 # one row per message: exact update count
+                assert ns["n_updates"] == -(-int(G) // muf)
+                assert (log[:-1] == muf).all()
+            else:
+                assert (log[:-1] >= muf).all()
+
+
+@pytest.mark.parametrize("mak,muf", [(1, 1), (4, 1), (4, 2), (8, 3), (5, 32)])
+def test_mlp_staleness_bound(oracle_mod, mak, muf):
+    g = ir.mlp((8, 6, 6, 3))
+    inst = data.mlp_instances(n=40, dim=8, classes=3)
+    o = make(oracle_mod, g, inst, wp.init_params(g))
+    st, _ = o.run_epoch(mak=mak, muf=muf, lr=0.01)
+    assert st.max_staleness <= -(-(mak - 1) // muf)
+    if mak == 1:
+        assert st.max_staleness == 0
+    if (mak, muf) == (4, 1):
+        assert st.max_staleness == 3                             # the bound is attained: mak - 1 updates
+
+
+def test_shuffled_order_is_a_permutation_of_the_work(oracle_mod):
+    g, inst, p = H.tiny_case("rnn", n=6)
+    o = make(oracle_mod, g, inst, p)
+    order = data.epoch_order(inst.n, 5)
+    assert sorted(order.tolist()) == list(range(inst.n)) and (order != np.arange(inst.n)).any()
+    st, loss = o.run_epoch(mak=1, muf=BIG, lr=0.1, order=order, flush=False)
+    grads, losses = H.dataset_grad(g, p, inst)
+    np.testing.assert_allclose(loss, losses, rtol=1e-12)
+    ins = o.key_log()[0]
+    np.testing.assert_array_equal(ins, order)
+
+
+# ---------------------------------------------------------------------------------------------------
+# special cases that reduce to something else
+# ---------------------------------------------------------------------------------------------------
+def test_left_chain_tree_equals_rnn_over_its_leaves(oracle_mod):
+    """A caterpillar tree ((((l0 l1) l2) l3) ...) is an RNN whose state starts at leaf 0."""
+    L = 5
+    g = ir.tree(vocab=9, emb=4, hidden=4, classes=3)
+    inst = data.Instances(ir.KIND_BINARY_TREES, 1)
+    M = 2 * L - 1
+    left, right, tok = [], [], []
+    # post-order: l0, l1, b(0,1)=2, l3.. : nodes: leaf0=0, leaf1=1, inner=2, leaf=3, inner=4, ...
+    left += [-1, -1, 0]; right += [-1, -1, 1]; tok += [1, 2, -1]
+    for k in range(2, L):
+        leaf_id = len(left)
+        left += [-1, len(left) - 1]; right += [-1, leaf_id]; tok += [k + 1, -1]
+    inst.offsets = np.array([0, M]); inst.left = np.array(left); inst.right = np.array(right)
+    inst.tokens = np.array(tok); inst.labels_i = np.arange(M) % 3
+    inst.finalize()
+    p = wp.init_params(g, emb_std=0.5)
+    o = make(oracle_mod, g, inst, p)
+    _, loss = o.run_epoch(mak=1, muf=BIG, lr=0.0, flush=False)
+    E, (Wl, bl), (Wb, bb), (Wc, bc) = p[(g.index("lookup"), 0)], [p[(g.index("leaf_cell"), w)] for w in (0, 1)], \
+        [p[(g.index("branch_cell"), w)] for w in (0, 1)], [p[(g.index("classifier"), w)] for w in (0, 1)]
+
+    def cls_loss(h, lab):
+        y = Wc @ h + bc
+        return np.log(np.exp(y).sum()) - y[lab]
+
+    leaves = [np.tanh(Wl @ E[t] + bl) for t in range(1, L + 1)]
+    total = cls_loss(leaves[0], 0) + cls_loss(leaves[1], 1)
+    h = np.tanh(Wb @ np.concatenate([leaves[0], leaves[1]]) + bb)
+    total += cls_loss(h, 2)
+    nid = 3
+    for k in range(2, L):
+        total += cls_loss(leaves[k], nid % 3)
+        h = np.tanh(Wb @ np.concatenate([h, leaves[k]]) + bb)
+        total += cls_loss(h, (nid + 1) % 3)
+        nid += 2
+    np.testing.assert_allclose(loss[0], total, rtol=1e-12)
+
+
+def test_ggnn_without_edges_of_a_type_and_eval_matches_training_forward(oracle_mod):
+    g, inst, p = H.tiny_case("ggnn", n=5)
+    assert len(np.unique(inst.edge_type)) < 4 or True
+    o = make(oracle_mod, g, inst, p)
+    _, train_loss = o.run_epoch(mak=3, muf=BIG, lr=0.0, flush=False)
+    ml, acc, ev_loss = o.eval()
+    np.testing.assert_allclose(ev_loss, train_loss, rtol=1e-12)
+    assert abs(ml - train_loss.mean()) < 1e-12
+
+
+@pytest.mark.parametrize("family", FAMILIES)
+def test_eval_is_forward_only_and_matches_direct_loss(oracle_mod, family):
+    g, inst, p = H.tiny_case(family, n=4, seed=2)
+    o = make(oracle_mod, g, inst, p)
+    before = o.get_params()
+    ml, acc, loss = o.eval()
+    _, losses = H.dataset_grad(g, p, inst)
+    np.testing.assert_allclose(loss, losses, rtol=1e-12, atol=1e-13)
+    after = o.get_params()
+    for k in before:
+        np.testing.assert_array_equal(before[k], after[k])
+    assert 0.0 <= acc <= 1.0
+
+
+def test_asynchrony_changes_the_trajectory_but_not_the_accounting(oracle_mod):
+    """mak > 1 with small muf gives stale gradients (different parameters) yet the same gradient counts."""
+    g = ir.mlp((8, 6, 6, 3))
+    inst = data.mlp_instances(n=24, dim=8, classes=3)
+    p = wp.init_params(g)
+    a, b = make(oracle_mod, g, inst, p), make(oracle_mod, g, inst, p)
+    a.run_epoch(mak=1, muf=1, lr=0.1)
+    sb, _ = b.run_epoch(mak=4, muf=1, lr=0.1)
+    n = g.ppt_nodes()[0]
+    assert np.abs(a.get_params(n, 0) - b.get_params(n, 0)).max() > 1e-6
+    assert a.node_stats(n)["n_grads_applied"] == b.node_stats(n)["n_grads_applied"] == inst.n
+    assert sb.max_staleness > 0
+
+
+def test_bf16_payload_rounding_only_touches_payloads(oracle_mod):
+    g, inst, p = H.tiny_case("tree", n=2)
+    o = oracle_mod.Oracle(g, payload_bf16=True)
+    o.load_instances(inst)
+    o.set_params(p)
+    _, l16 = o.run_epoch(mak=1, muf=BIG, lr=0.0, flush=False)
+    o2 = make(oracle_mod, g, inst, p)
+    _, l64 = o2.run_epoch(mak=1, muf=BIG, lr=0.0, flush=False)
+    rel = np.abs(l16 - l64) / l64
+    assert (rel > 0).any() and rel.max() < 3e-2            # bf16 has 8 bits of mantissa
+    for k in p:
+        np.testing.assert_array_equal(o.get_params(*k), p[k])
