@@ -1,0 +1,186 @@
+/* ampnet.h -- C ABI of the B200-native AMPNet training engine.
+ *
+ * The engine executes the hot path of asynchronous model-parallel (AMP) training of dynamic networks
+ * (AMPNet, arXiv 1705.09786): the message-driven execution of a static IR graph.  Forward and backward
+ * messages keyed by instance flow through parameterised nodes (Linear, GRU cell, embedding lookup) and
+ * control-flow nodes (Cond, Phi, Isu, Concat, Bcast, Group, Ungroup, Flatmap); every parameterised node
+ * accumulates gradients locally and applies an SGD update once min_update_frequency gradients have
+ * arrived (Sec. 3); max_active_keys bounds the instances in flight (Sec. 3).  On the device this is one
+ * persistent kernel whose CTAs own row tiles of the parameterised nodes (weights and fp32 accumulators in
+ * shared memory) and exchange messages through lock-free ring queues in device memory.
+ *
+ * Conventions.  Every call returns a status; nothing aborts the process or traps the GPU; every device-side
+ * wait is bounded and reports AMPNET_ETIMEOUT.  Input arrays are caller-owned HOST memory and are copied.
+ * Output arrays are caller-allocated HOST memory.  The handle owns all device memory, obtained through the
+ * allocator given at creation (cudaMalloc when none is given).  Matrices are row-major [out x in], fp32.
+ * Calls on one handle are not thread-safe.  All work is issued on the stream given at creation.
+ */
+#ifndef AMPNET_H
+#define AMPNET_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ampnet_graph ampnet_graph_t; /* opaque, owned by the library */
+
+typedef enum {
+  AMPNET_OK = 0,
+  AMPNET_EINVAL = 1,    /* malformed argument or IR description (see ampnet_last_error)            */
+  AMPNET_ENOMEM = 2,    /* device allocation failed                                                */
+  AMPNET_ECUDA = 3,     /* a CUDA runtime call failed                                              */
+  AMPNET_ETIMEOUT = 4,  /* a bounded device-side wait gave up; the GPU context stays usable        */
+  AMPNET_EOVERFLOW = 5, /* a queue / cache / key-space bound was exceeded; nothing blocked         */
+  AMPNET_ESTATE = 6     /* call order wrong (for example run before load)                          */
+} ampnet_status_t;
+
+/* ---- IR description (Sec. 4: a static graph of nodes and edges) ---------------------------------------- */
+
+/* node types */
+enum {
+  AMPNET_SOURCE = 0,      /* controller output: pumps one admitted instance (fn = AMPNET_SRC_*)          */
+  AMPNET_LINEAR = 1,      /* PPT: y = act(W x + b), row-wise for matrix payloads                         */
+  AMPNET_LOOKUP = 2,      /* PPT: embedding table, in_dim = vocabulary, out_dim = width                  */
+  AMPNET_GRUCELL = 3,     /* PPT: x = [a; h] (in_dim = 2H): z = s(Wz x + bz), r = s(Wr x + br),
+                             c = tanh(Wc [a; r*h] + bc), h' = (1 - z) * h + z * c                        */
+  AMPNET_LOSS_CE = 4,     /* softmax cross-entropy against an integer label; starts the backward pass    */
+  AMPNET_LOSS_MSE = 5,    /* (y - t)^2 against a float target                                            */
+  AMPNET_NPT_SUMROWS = 6, /* non-parameterised transform: sum of the rows of the payload                 */
+  AMPNET_COND = 7,        /* routes on the state (fn = AMPNET_COND_*)                                    */
+  AMPNET_PHI = 8,         /* join: records the origin keyed on the state, backpropagates to it           */
+  AMPNET_ISU = 9,         /* invertible state update (fn = AMPNET_ISU_*)                                 */
+  AMPNET_CONCAT = 10,     /* fn_arg ports of width in_dim -> one payload of width out_dim                */
+  AMPNET_SPLIT = 11,      /* inverse of CONCAT (declared; not executed by the device engine yet)         */
+  AMPNET_BCAST = 12,      /* same payload to fn_arg successors; backward = sum in successor order        */
+  AMPNET_GROUP = 13,      /* collect messages by state into one matrix payload (fn = AMPNET_GROUP_*)     */
+  AMPNET_UNGROUP = 14,    /* one message per row (fn = AMPNET_UNGROUP_*)                                 */
+  AMPNET_FLATMAP = 15,    /* one message per generated state, payload replicated (fn = AMPNET_FLATMAP_*) */
+  AMPNET_SINK = 16        /* answers a forward message with a zero gradient                              */
+};
+enum { AMPNET_ACT_NONE = 0, AMPNET_ACT_RELU = 1, AMPNET_ACT_TANH = 2, AMPNET_ACT_SIGMOID = 3 };
+/* state functions; the message state is (inst, seq, slot, it, u, port)                                     */
+enum { AMPNET_SRC_DENSE_ROW = 1, AMPNET_SRC_TOKENS = 2, AMPNET_SRC_ZERO_STATE = 3, AMPNET_SRC_TREE_LEAVES = 4,
+       AMPNET_SRC_GRAPH_NODES = 5 };
+enum { AMPNET_COND_SEQ_END = 1,   /* u < #tokens ? 0 : 1        */
+       AMPNET_COND_TREE_ROOT = 2, /* u is the root ? 0 : 1      */
+       AMPNET_COND_BY_U = 3,      /* successor = u              */
+       AMPNET_COND_IT_LT = 4 };   /* it < fn_arg ? 0 : 1        */
+enum { AMPNET_ISU_U_INC = 1, AMPNET_ISU_TREE_PARENT = 2, AMPNET_ISU_IT_INC = 3 };
+enum { AMPNET_CONCAT_BY_EDGE = 1, AMPNET_CONCAT_BY_STATE_PORT = 2 };
+enum { AMPNET_GROUP_EDGES_BY_TYPE = 1, AMPNET_GROUP_EDGES_BY_DST = 2, AMPNET_GROUP_ALL_NODES = 3 };
+enum { AMPNET_UNGROUP_NODES = 1, AMPNET_UNGROUP_TYPE_EDGES = 2 };
+enum { AMPNET_FLATMAP_OUT_EDGES = 1 };
+enum { AMPNET_LABEL_PER_INSTANCE = 1, AMPNET_LABEL_PER_TREE_NODE = 2 };
+enum { AMPNET_FLAG_SOURCE_ADJACENT = 1 }; /* PPT fed directly by a SOURCE: no input gradient, retire instead */
+
+typedef struct {
+  int32_t type, in_dim, out_dim, act;
+  int32_t fn, fn_arg;
+  int32_t muf_override; /* 0 = use the run configuration's min_update_frequency (per-node threshold)   */
+  int32_t flags;
+} ampnet_node_desc_t;
+typedef struct { int32_t src_node, src_port, dst_node, dst_port; } ampnet_edge_desc_t;
+typedef struct {
+  int32_t n_nodes, n_edges;
+  const ampnet_node_desc_t* nodes; /* host */
+  const ampnet_edge_desc_t* edges; /* host */
+  int32_t payload_dtype;           /* 0 = fp32 (the only one executed so far) */
+} ampnet_ir_desc_t;
+
+/* Device-memory allocator supplied by the caller (for example a PyTorch caching allocator).  `alloc` returns a
+ * device pointer aligned to 256 bytes or NULL; `free` releases it.  Both are called from the calling thread. */
+typedef void* (*ampnet_alloc_fn)(void* ctx, size_t bytes);
+typedef void (*ampnet_free_fn)(void* ctx, void* ptr);
+typedef struct { ampnet_alloc_fn alloc; ampnet_free_fn free; void* ctx; } ampnet_allocator_t;
+
+/* Sec. 4 "a model = an IR graph + a controller loop".  Validates the IR, places the parameterised nodes on
+ * CTAs, allocates and initialises the parameters (seeded).  `cuda_stream` is a cudaStream_t (NULL = default
+ * stream); `allocator` may be NULL.  On failure *out is NULL and the status says why.                         */
+ampnet_status_t ampnet_graph_create(const ampnet_ir_desc_t* ir, uint64_t init_seed, void* cuda_stream,
+                                    const ampnet_allocator_t* allocator, ampnet_graph_t** out);
+void ampnet_graph_destroy(ampnet_graph_t*);
+
+/* ---- instances (what the controller pumps, Sec. 4) ----------------------------------------------------- */
+enum { AMPNET_KIND_DENSE_ROWS = 0, AMPNET_KIND_SEQUENCES = 1, AMPNET_KIND_BINARY_TREES = 2,
+       AMPNET_KIND_TYPED_GRAPHS = 3 };
+typedef struct {
+  int32_t kind;
+  int64_t n_instances;
+  const int64_t* offsets;      /* n+1: tokens / tree nodes / graph nodes per instance (NULL for dense rows)   */
+  const int32_t* tokens;       /* token id / leaf token id (-1 at inner tree nodes) / graph node type id      */
+  const int32_t *left, *right; /* trees: local child ids, -1 at leaves; children precede parents             */
+  const int64_t* edge_offsets; /* graphs: n+1                                                                */
+  const int32_t *edge_src, *edge_dst, *edge_type; /* graphs: directed edges, local node ids                  */
+  const float* dense;          /* dense rows: n x dense_dim                                                  */
+  int32_t dense_dim;
+  const int32_t* labels_i;     /* class per instance, or per tree node (AMPNET_LABEL_PER_TREE_NODE)          */
+  const float* labels_f;       /* regression target per instance                                             */
+} ampnet_instances_t;
+
+/* Copies the instances to the device and encodes their structure into routing tables (parents and child
+ * slots of trees; out-edge, in-edge and per-type edge lists and ranks of graphs).  split: 0 train, 1 valid.  */
+ampnet_status_t ampnet_load_instances(ampnet_graph_t*, int32_t split, const ampnet_instances_t*);
+
+/* ---- training (Sec. 3) ---------------------------------------------------------------------------------- */
+typedef struct {
+  int32_t max_active_keys;      /* instances in flight                                                       */
+  int32_t min_update_frequency; /* gradients accumulated by a node before it updates                         */
+  float lr;                     /* SGD: theta -= lr * (accumulated gradient / number of gradients)           */
+  int32_t deterministic;        /* 1: canonical round schedule (reproducible; for checking), 0: asynchronous */
+  const int64_t* order;         /* host, instance order of the epoch; NULL = dataset order                   */
+  int64_t n_order;              /* number of instances to train on (ignored when order == NULL: all)         */
+  double timeout_s;             /* bound on the whole device run; 0 = default (120 s)                        */
+  int32_t max_batch_rows;       /* cap on payload rows a node processes as one micro-batch; 0 = automatic    */
+  int32_t n_ctas;               /* CTAs to use; 0 = one per SM                                               */
+} ampnet_run_cfg_t;
+
+typedef struct {
+  int64_t instances, node_messages, ppt_messages, rounds;
+  double seconds;   /* device time of the run (CUDA events)                                                  */
+  double mean_loss; /* mean per-instance loss of the epoch                                                   */
+  int32_t max_staleness;
+  int64_t max_active_observed;
+  uint64_t route_hash; /* order-independent fingerprint of all routed (node, direction, state) messages     */
+  int64_t micro_batches, micro_batch_rows; /* batches executed by all nodes and the payload rows in them    */
+} ampnet_epoch_stats_t;
+
+/* One pass over the training split: admission under max_active_keys, message-driven forward and backward
+ * execution, local updates, retirement; accumulators are flushed at the end.  per_instance_loss: host,
+ * n_instances floats (indexed by instance), may be NULL.                                                    */
+ampnet_status_t ampnet_run_epoch(ampnet_graph_t*, const ampnet_run_cfg_t*, ampnet_epoch_stats_t* out,
+                                 float* per_instance_loss);
+
+/* Forward-only messages over a split; nothing cached, no parameter touched.  accuracy: fraction of correct
+ * arg-max predictions over all loss evaluations (0 for MSE).                                                */
+ampnet_status_t ampnet_eval(ampnet_graph_t*, int32_t split, int32_t max_active_keys, double* mean_loss,
+                            double* accuracy, float* per_instance_loss);
+
+/* ---- parameters and statistics --------------------------------------------------------------------------- */
+/* which: LINEAR 0 = W, 1 = b; LOOKUP 0 = E; GRUCELL 0..2 = Wz, Wr, Wc, 3..5 = bz, br, bc.                    */
+ampnet_status_t ampnet_param_count(ampnet_graph_t*, int32_t node, int32_t which, int64_t* n);
+ampnet_status_t ampnet_get_params(ampnet_graph_t*, int32_t node, int32_t which, float* dst_host, int64_t n);
+ampnet_status_t ampnet_set_params(ampnet_graph_t*, int32_t node, int32_t which, const float* src_host, int64_t n);
+
+/* Statistics of the last run.  staleness_hist: 64 bins (updates between a gradient's forward and backward).  */
+ampnet_status_t ampnet_get_node_stats(ampnet_graph_t*, int32_t node, int64_t* n_updates, int64_t* n_grads_applied,
+                                      int64_t* staleness_hist, int64_t* fwd_msgs, int64_t* bwd_msgs);
+/* Gradient count of each update of a node, in order; returns the number of updates through *n.               */
+ampnet_status_t ampnet_get_update_log(ampnet_graph_t*, int32_t node, int32_t* n_per_update, int64_t cap, int64_t* n);
+/* Key bookkeeping of the last deterministic run: instance, slot, admission round, release round.             */
+ampnet_status_t ampnet_get_key_log(ampnet_graph_t*, int64_t* inst, int32_t* slot, int64_t* admit_round,
+                                   int64_t* release_round, int64_t cap, int64_t* n);
+/* Number of keyed cache entries (join counters, recorded origins) still set after the last run; the
+ * forward/backward state invariant of Sec. 4 makes this 0.                                                   */
+ampnet_status_t ampnet_leftover_cache_entries(ampnet_graph_t*, int64_t* n);
+/* Placement chosen for a parameterised node: number of row tiles (CTAs) and micro-batch row capacity.        */
+ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_tiles, int32_t* batch_rows);
+
+const char* ampnet_last_error(const ampnet_graph_t*); /* library-owned string */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AMPNET_H */

@@ -1,0 +1,986 @@
+// Host side of the AMPNet engine: the C ABI of include/ampnet.h.
+//   * IR builder checks and placement of the parameterised nodes on CTAs ("scheduler on the host"),
+//   * structure encoder: trees / graphs / lists -> routing tables in device memory,
+//   * key-space inference, allocation of queues and keyed caches, kernel launch, statistics.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/ampnet.h"
+#include "engine.cuh"
+
+using namespace amp;
+
+namespace {
+
+struct DeviceArena {           // one allocation carved into aligned pieces
+  char* base = nullptr;
+  size_t size = 0, used = 0;
+  template <class T> T* take(size_t n) {
+    used = (used + 255) & ~(size_t)255;
+    T* p = base ? reinterpret_cast<T*>(base + used) : nullptr;
+    used += n * sizeof(T);
+    return p;
+  }
+};
+
+struct HostDataset {
+  bool loaded = false;
+  int kind = -1, dense_dim = 0, NT = 1, labels_per_node = 0;
+  long long n = 0;
+  int maxT = 1, maxM = 1, maxN = 1, maxD = 1, maxDc = 1, maxIn = 1, maxOut = 1, maxL = 1;
+  long long total_pos = 0, total_edges = 0;
+  DevInst dev{};
+  std::vector<void*> allocs;
+};
+
+struct HostPPT {
+  int node = 0, kind = 0, in = 0, out = 0, nmat = 1;
+  float *W = nullptr, *b = nullptr;
+  size_t nW = 0, nb = 0;
+  int T = 1, R = 0, BM = 0, J = 0;
+  size_t smem_floats = 0;
+};
+
+}  // namespace
+
+struct ampnet_graph {
+  std::vector<ampnet_node_desc_t> nodes;
+  std::vector<ampnet_edge_desc_t> edges;
+  std::vector<DevNode> hnodes;        // topology filled at creation, storage at run time
+  std::vector<HostPPT> ppts;
+  std::vector<int> sources, losses;
+  bool has_it = false; int it_steps = 0;
+  ampnet_allocator_t alloc{};
+  cudaStream_t stream = nullptr;
+  int device = 0, n_sms = 0, max_smem = 0;
+  HostDataset data[2];
+  std::string err;
+  // run state
+  DeviceArena ctl, bulk;
+  void *ctl_mem = nullptr, *bulk_mem = nullptr;
+  size_t ctl_cap = 0, bulk_cap = 0;
+  std::vector<std::pair<size_t, size_t>> leftover_regions;   // (offset, bytes) inside ctl
+  std::vector<PPTStats*> d_stats;
+  std::vector<int*> d_update_log;
+  unsigned long long* d_node_msgs = nullptr;
+  KeyLog* d_keylog = nullptr;
+  long long n_keylog = 0;
+  int update_log_cap = 1 << 20;
+  std::vector<PPTStats> last_stats;
+  std::vector<unsigned long long> last_node_msgs;
+  bool have_run = false;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+};
+
+namespace {
+
+ampnet_status_t set_err(ampnet_graph* g, ampnet_status_t st, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (g) g->err = buf;
+  return st;
+}
+
+#define CUDA_TRY(g, call)                                                                                  \
+  do {                                                                                                     \
+    cudaError_t e_ = (call);                                                                               \
+    if (e_ != cudaSuccess) return set_err(g, AMPNET_ECUDA, "%s failed: %s", #call, cudaGetErrorString(e_)); \
+  } while (0)
+
+void* dev_alloc(ampnet_graph* g, size_t bytes) {
+  if (bytes == 0) bytes = 256;
+  if (g->alloc.alloc) return g->alloc.alloc(g->alloc.ctx, bytes);
+  void* p = nullptr;
+  if (cudaMalloc(&p, bytes) != cudaSuccess) return nullptr;
+  return p;
+}
+void dev_free(ampnet_graph* g, void* p) {
+  if (!p) return;
+  if (g->alloc.free) g->alloc.free(g->alloc.ctx, p);
+  else if (!g->alloc.alloc) cudaFree(p);
+}
+
+bool is_ppt_type(int t) { return t == LINEAR || t == LOOKUP || t == GRUCELL; }
+
+uint64_t splitmix(uint64_t& s) {
+  uint64_t z = (s += 0x9E3779B97F4A7C15ull);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+double uniform01(uint64_t& s) { return (double)(splitmix(s) >> 11) * (1.0 / 9007199254740992.0); }
+
+int j_bucket(int in) {
+  const int j = (in + 31) / 32;
+  const int b[] = {4, 7, 10, 16, 25, 32};
+  for (int v : b) if (j <= v) return v;
+  return -1;
+}
+
+template <class T>
+ampnet_status_t upload(ampnet_graph* g, HostDataset& D, const std::vector<T>& h, const T** out) {
+  void* p = dev_alloc(g, std::max<size_t>(h.size(), 1) * sizeof(T));
+  if (!p) return set_err(g, AMPNET_ENOMEM, "device allocation of %zu bytes failed", h.size() * sizeof(T));
+  D.allocs.push_back(p);
+  if (!h.empty()) CUDA_TRY(g, cudaMemcpyAsync(p, h.data(), h.size() * sizeof(T), cudaMemcpyHostToDevice, g->stream));
+  *out = reinterpret_cast<const T*>(p);
+  return AMPNET_OK;
+}
+template <class T>
+ampnet_status_t upload_raw(ampnet_graph* g, HostDataset& D, const T* h, size_t n, const T** out) {
+  void* p = dev_alloc(g, std::max<size_t>(n, 1) * sizeof(T));
+  if (!p) return set_err(g, AMPNET_ENOMEM, "device allocation of %zu bytes failed", n * sizeof(T));
+  D.allocs.push_back(p);
+  if (n) CUDA_TRY(g, cudaMemcpyAsync(p, h, n * sizeof(T), cudaMemcpyHostToDevice, g->stream));
+  *out = reinterpret_cast<const T*>(p);
+  return AMPNET_OK;
+}
+
+void free_dataset(ampnet_graph* g, HostDataset& D) {
+  for (void* p : D.allocs) dev_free(g, p);
+  D = HostDataset();
+}
+
+// ---- IR checks ---------------------------------------------------------------------------------------
+ampnet_status_t build_topology(ampnet_graph* g) {
+  const int n = (int)g->nodes.size();
+  g->hnodes.assign(n, DevNode{});
+  for (int i = 0; i < n; i++) {
+    const auto& d = g->nodes[i];
+    if (d.type < 0 || d.type >= N_NODE_TYPES) return set_err(g, AMPNET_EINVAL, "node %d: unknown type %d", i, d.type);
+    if (d.type == SPLIT) return set_err(g, AMPNET_EINVAL, "node %d: SPLIT is not executed by the device engine", i);
+    if (d.in_dim < 0 || d.out_dim < 0) return set_err(g, AMPNET_EINVAL, "node %d: negative dimension", i);
+    DevNode& h = g->hnodes[i];
+    h.type = d.type; h.in_dim = d.in_dim; h.out_dim = d.out_dim; h.act = d.act; h.fn = d.fn; h.fn_arg = d.fn_arg;
+    h.flags = d.flags; h.ppt = -1;
+    for (int k = 0; k < MAX_PORTS; k++) h.succ_node[k] = h.pred_node[k] = h.succ_port[k] = h.pred_port[k] = -1;
+    if (d.act < 0 || d.act > 3) return set_err(g, AMPNET_EINVAL, "node %d: unknown activation %d", i, d.act);
+  }
+  for (size_t k = 0; k < g->edges.size(); k++) {
+    const auto& e = g->edges[k];
+    if (e.src_node < 0 || e.src_node >= n || e.dst_node < 0 || e.dst_node >= n)
+      return set_err(g, AMPNET_EINVAL, "edge %zu: node index out of range", k);
+    if (e.src_port < 0 || e.src_port >= MAX_PORTS || e.dst_port < 0 || e.dst_port >= MAX_PORTS)
+      return set_err(g, AMPNET_EINVAL, "edge %zu: port out of range (max %d)", k, MAX_PORTS);
+    DevNode &s = g->hnodes[e.src_node], &d = g->hnodes[e.dst_node];
+    if (s.succ_node[e.src_port] >= 0) return set_err(g, AMPNET_EINVAL, "edge %zu: source port used twice", k);
+    if (d.pred_node[e.dst_port] >= 0) return set_err(g, AMPNET_EINVAL, "edge %zu: destination port used twice", k);
+    s.succ_node[e.src_port] = e.dst_node; s.succ_port[e.src_port] = e.dst_port;
+    d.pred_node[e.dst_port] = e.src_node; d.pred_port[e.dst_port] = e.src_port;
+    s.n_succ = std::max(s.n_succ, e.src_port + 1);
+    d.n_pred = std::max(d.n_pred, e.dst_port + 1);
+  }
+  for (int i = 0; i < n; i++) {
+    DevNode& h = g->hnodes[i];
+    for (int k = 0; k < h.n_succ; k++) if (h.succ_node[k] < 0) return set_err(g, AMPNET_EINVAL, "node %d: successor port %d unconnected", i, k);
+    for (int k = 0; k < h.n_pred; k++) if (h.pred_node[k] < 0) return set_err(g, AMPNET_EINVAL, "node %d: predecessor port %d unconnected", i, k);
+    auto need = [&](bool c, const char* what) { return c ? AMPNET_OK : set_err(g, AMPNET_EINVAL, "node %d: %s", i, what); };
+    ampnet_status_t st = AMPNET_OK;
+    switch (h.type) {
+      case SOURCE:
+        st = need(h.n_pred == 0 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 5, "SOURCE needs one successor and a valid fn");
+        if (st == AMPNET_OK) g->sources.push_back(i);
+        break;
+      case LINEAR:
+        st = need(h.n_pred == 1 && h.n_succ == 1 && h.in_dim > 0 && h.out_dim > 0, "LINEAR needs one predecessor, one successor, positive dims");
+        if (st == AMPNET_OK) {
+          const bool fed = g->hnodes[h.pred_node[0]].type == SOURCE;
+          st = need(fed == ((h.flags & 1) != 0), "FLAG_SOURCE_ADJACENT must be set exactly on PPT nodes fed by a SOURCE");
+        }
+        break;
+      case LOOKUP:
+        st = need(h.n_pred == 1 && h.n_succ == 1 && h.in_dim > 0 && h.out_dim > 0 && g->hnodes[h.pred_node[0]].type == SOURCE &&
+                  (h.flags & 1), "LOOKUP must be fed by a SOURCE and flagged source-adjacent");
+        break;
+      case GRUCELL:
+        st = need(h.n_pred == 1 && h.n_succ == 1 && h.out_dim > 0 && h.in_dim == 2 * h.out_dim && !(h.flags & 1), "GRUCELL needs in_dim == 2*out_dim");
+        break;
+      case LOSS_CE: case LOSS_MSE:
+        st = need(h.n_pred == 1 && h.n_succ == 0 && h.in_dim > 0 && (h.type == LOSS_CE || h.in_dim == 1), "LOSS needs one predecessor and no successor");
+        if (st == AMPNET_OK) g->losses.push_back(i);
+        break;
+      case SINK: st = need(h.n_pred == 1 && h.n_succ == 0, "SINK needs one predecessor and no successor"); break;
+      case COND: st = need(h.n_pred == 1 && h.n_succ >= 1 && h.fn >= 1 && h.fn <= 4, "COND needs one predecessor and a valid fn"); break;
+      case PHI: st = need(h.n_pred >= 1 && h.n_succ == 1, "PHI needs predecessors and one successor"); break;
+      case ISU:
+        st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 3, "ISU needs a valid fn");
+        break;
+      case CONCAT:
+        st = need(h.n_succ == 1 && h.fn_arg >= 1 && h.fn_arg <= MAX_PORTS && h.out_dim == h.fn_arg * h.in_dim &&
+                  ((h.fn == 1 && h.n_pred == h.fn_arg) || (h.fn == 2 && h.n_pred == 1)), "CONCAT ports / widths inconsistent");
+        break;
+      case BCAST: st = need(h.n_pred == 1 && h.fn_arg >= 1 && h.n_succ == h.fn_arg, "BCAST needs fn_arg successors"); break;
+      case GROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 3, "GROUP needs a valid fn"); break;
+      case UNGROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 2, "UNGROUP needs a valid fn"); break;
+      case FLATMAP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn == 1, "FLATMAP needs a valid fn"); break;
+      case NPT_SUMROWS: st = need(h.n_pred == 1 && h.n_succ == 1, "NPT_SUMROWS needs one predecessor and one successor"); break;
+    }
+    if (st != AMPNET_OK) return st;
+    if (h.type == ISU && h.fn == 3) g->has_it = true;
+    if (h.type == COND && h.fn == 4) g->it_steps = std::max(g->it_steps, h.fn_arg);
+  }
+  if (g->sources.empty() || g->sources.size() > 4) return set_err(g, AMPNET_EINVAL, "the graph needs 1..4 SOURCE nodes");
+  if (g->losses.empty() || g->losses.size() > 4) return set_err(g, AMPNET_EINVAL, "the graph needs 1..4 LOSS nodes");
+  // widths along the edges
+  auto out_width = [&](const DevNode& h) {
+    if (h.type == LINEAR || h.type == LOOKUP || h.type == GRUCELL || h.type == CONCAT) return h.out_dim;
+    if (h.type == SOURCE) return (h.fn == 1 || h.fn == 3) ? h.out_dim : 0;
+    return h.in_dim;
+  };
+  for (size_t k = 0; k < g->edges.size(); k++) {
+    const DevNode &s = g->hnodes[g->edges[k].src_node], &d = g->hnodes[g->edges[k].dst_node];
+    const int w = out_width(s);
+    if (d.type == LOOKUP || w == 0) continue;
+    if (d.type == SINK) continue;
+    if (w != d.in_dim) return set_err(g, AMPNET_EINVAL, "edge %zu: width %d does not match the destination's in_dim %d", k, w, d.in_dim);
+  }
+  // every cycle must pass through a PHI: the graph without PHI nodes is acyclic
+  std::vector<int> indeg(n, 0);
+  for (const auto& e : g->edges) if (g->hnodes[e.src_node].type != PHI && g->hnodes[e.dst_node].type != PHI) indeg[e.dst_node]++;
+  std::vector<int> q;
+  int seen = 0, n_non_phi = 0;
+  for (int i = 0; i < n; i++) if (g->hnodes[i].type != PHI) { n_non_phi++; if (!indeg[i]) q.push_back(i); }
+  while (!q.empty()) {
+    int u = q.back(); q.pop_back(); seen++;
+    for (int k = 0; k < g->hnodes[u].n_succ; k++) {
+      int v = g->hnodes[u].succ_node[k];
+      if (g->hnodes[v].type == PHI) continue;
+      if (--indeg[v] == 0) q.push_back(v);
+    }
+  }
+  if (seen != n_non_phi) return set_err(g, AMPNET_EINVAL, "the IR graph has a cycle that does not pass through a PHI node");
+  return AMPNET_OK;
+}
+
+ampnet_status_t create_params(ampnet_graph* g, uint64_t seed) {
+  uint64_t s = seed * 0x9E3779B97F4A7C15ull + 12345;
+  for (int i = 0; i < (int)g->hnodes.size(); i++) {
+    DevNode& h = g->hnodes[i];
+    if (!is_ppt_type(h.type)) continue;
+    HostPPT P;
+    P.node = i; P.kind = h.type; P.in = h.in_dim; P.out = h.out_dim; P.nmat = h.type == GRUCELL ? 3 : 1;
+    if (h.type != LOOKUP && j_bucket(h.in_dim) < 0) return set_err(g, AMPNET_EINVAL, "node %d: in_dim %d above 1024 is not supported", i, h.in_dim);
+    P.nW = (size_t)P.nmat * P.in * P.out;
+    P.nb = h.type == LOOKUP ? 0 : (size_t)P.nmat * P.out;
+    std::vector<float> w(P.nW), b(P.nb, 0.f);
+    if (h.type == LOOKUP) {
+      for (size_t k = 0; k + 1 < w.size() + 1; k += 2) {      // Box-Muller, N(0, 0.1)
+        double u1 = std::max(uniform01(s), 1e-300), u2 = uniform01(s);
+        double r = std::sqrt(-2.0 * std::log(u1)) * 0.1;
+        w[k] = (float)(r * std::cos(6.283185307179586 * u2));
+        if (k + 1 < w.size()) w[k + 1] = (float)(r * std::sin(6.283185307179586 * u2));
+      }
+    } else {
+      const double lim = std::sqrt(6.0 / (P.in + P.out));
+      for (auto& v : w) v = (float)((2.0 * uniform01(s) - 1.0) * lim);
+    }
+    P.W = (float*)dev_alloc(g, P.nW * sizeof(float));
+    P.b = (float*)dev_alloc(g, std::max<size_t>(P.nb, 1) * sizeof(float));
+    if (!P.W || !P.b) return set_err(g, AMPNET_ENOMEM, "parameter allocation failed");
+    CUDA_TRY(g, cudaMemcpy(P.W, w.data(), P.nW * sizeof(float), cudaMemcpyHostToDevice));
+    if (P.nb) CUDA_TRY(g, cudaMemcpy(P.b, b.data(), P.nb * sizeof(float), cudaMemcpyHostToDevice));
+    h.ppt = (int)g->ppts.size();
+    g->ppts.push_back(P);
+  }
+  if (g->ppts.empty()) return set_err(g, AMPNET_EINVAL, "the graph has no parameterised node");
+  return AMPNET_OK;
+}
+
+// ---- key-space inference: bounds of the position u and of the payload rows at every node ---------------
+struct Dom { int U, rows; };
+
+void infer_domains(ampnet_graph* g, const HostDataset& D) {
+  const int n = (int)g->hnodes.size();
+  std::vector<Dom> in(n, Dom{1, 1}), out(n, Dom{1, 1});
+  for (int pass = 0; pass < 4 * n + 8; pass++) {
+    bool changed = false;
+    for (int i = 0; i < n; i++) {
+      DevNode& h = g->hnodes[i];
+      Dom a{1, 1};
+      for (int k = 0; k < h.n_pred; k++) { const Dom& p = out[h.pred_node[k]]; a.U = std::max(a.U, p.U); a.rows = std::max(a.rows, p.rows); }
+      Dom o = a;
+      switch (h.type) {
+        case SOURCE:
+          if (h.fn == 2) o = Dom{D.maxT + 1, 1};
+          else if (h.fn == 4) o = Dom{D.maxM, 1};
+          else if (h.fn == 5) o = Dom{1, D.maxN};
+          else o = Dom{1, 1};
+          break;
+        case FLATMAP: o = Dom{D.maxD, 1}; break;
+        case GROUP:
+          if (h.fn == 1) o = Dom{D.NT, D.maxDc};
+          else if (h.fn == 2) o = Dom{D.maxN, D.maxIn};
+          else o = Dom{1, D.maxN};
+          break;
+        case UNGROUP: o = h.fn == 2 ? Dom{D.maxD, 1} : Dom{D.maxN, 1}; break;
+        case NPT_SUMROWS: o = Dom{a.U, 1}; break;
+        default: break;
+      }
+      if (o.U != out[i].U || o.rows != out[i].rows || a.U != in[i].U || a.rows != in[i].rows) changed = true;
+      in[i] = a; out[i] = o;
+    }
+    if (!changed) break;
+  }
+  for (int i = 0; i < n; i++) {
+    g->hnodes[i].U_in = in[i].U; g->hnodes[i].rows_in = in[i].rows;
+    g->hnodes[i].U_out = out[i].U; g->hnodes[i].rows_out = out[i].rows;
+  }
+}
+
+unsigned pow2_at_least(unsigned long long v) {
+  unsigned p = 64;
+  while (p < v && p < (1u << 30)) p <<= 1;
+  return p;
+}
+
+size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
+  if (P.kind == LOOKUP) return 64;
+  return (size_t)P.nmat * (2 * (size_t)R * P.in + 2 * R) + (size_t)BM * P.in + 2 * (size_t)P.nmat * BM * R + 64;
+}
+
+// Placement: row tiles per PPT node.  Enough tiles that a tile's weights + accumulators + staging fit in
+// shared memory, then the remaining CTAs in proportion to the nodes' multiply-add volume.
+ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles) {
+  const size_t budget = ((size_t)g->max_smem - 12 * 1024) / sizeof(float);
+  int max_tiles = 16;
+  if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, atoi(e));
+  double total_w = 0;
+  for (auto& P : g->ppts) if (P.kind != LOOKUP) total_w += (double)P.nmat * P.in * P.out;
+  const int avail = std::max(1, n_ctas - 1 - (int)g->ppts.size());
+  int used = 1;
+  for (auto& P : g->ppts) {
+    const DevNode& h = g->hnodes[P.node];
+    const int rows_max = h.rows_in;
+    int BM = rows_max <= 32 ? 32 : 64;
+    if (max_batch_rows > 0) BM = std::max(rows_max, std::min(BM, max_batch_rows));
+    if (rows_max > 64) return set_err(g, AMPNET_EINVAL, "node %d: %d payload rows per message exceed the supported 64", P.node, rows_max);
+    P.J = P.kind == LOOKUP ? 4 : j_bucket(P.in);
+    if (P.kind == LOOKUP) { P.T = 1; P.R = 0; P.BM = BM; P.smem_floats = tile_smem_floats(P, 0, BM); used += 1; continue; }
+    int T = 1 + (int)std::floor((double)P.nmat * P.in * P.out / total_w * avail);
+    T = std::max(1, std::min({T, max_tiles, std::max(1, P.out / 4)}));
+    for (;;) {
+      int R = (P.out + T - 1) / T;
+      int bm = BM;
+      while (tile_smem_floats(P, R, bm) > budget && bm > std::max(rows_max, 4)) bm = std::max(std::max(rows_max, 4), bm / 2);
+      if (tile_smem_floats(P, R, bm) <= budget) { P.R = R; P.BM = bm; P.T = (P.out + R - 1) / R; break; }
+      if (R == 1) return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory even at one row per tile", P.node);
+      T = std::min(P.out, T + 1);
+    }
+    P.smem_floats = tile_smem_floats(P, P.R, P.BM);
+    used += P.T;
+  }
+  if (used > n_ctas) return set_err(g, AMPNET_EINVAL, "placement needs %d CTAs but only %d are available", used, n_ctas);
+  roles.clear();
+  roles.push_back(Role{-1, 0});
+  for (int p = 0; p < (int)g->ppts.size(); p++)
+    for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t});
+  return AMPNET_OK;
+}
+
+// ---- run ---------------------------------------------------------------------------------------------------
+struct RunPlan {
+  std::vector<DevNode> nodes;
+  std::vector<DevPPT> ppts;
+  std::vector<Role> roles;
+  Ctx ctx{};
+  size_t smem_bytes = 0;
+};
+
+ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval, const ampnet_run_cfg_t* cfg,
+                         long long n_order, bool dry, RunPlan& R) {
+  HostDataset& D = g->data[split];
+  infer_domains(g, D);
+  const int IT = g->has_it ? g->it_steps + 1 : 1;
+  int n_ctas = cfg && cfg->n_ctas > 0 ? std::min(cfg->n_ctas, g->n_sms) : g->n_sms;
+  ampnet_status_t st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles);
+  if (st != AMPNET_OK) return st;
+  n_ctas = (int)R.roles.size();
+  DeviceArena &C = g->ctl, &B = g->bulk;
+  C.used = B.used = 0;
+  if (dry) { C.base = B.base = nullptr; } else { C.base = (char*)g->ctl_mem; B.base = (char*)g->bulk_mem; }
+  g->leftover_regions.clear();
+  auto track = [&](void* p, size_t bytes) { if (!dry) g->leftover_regions.push_back({(size_t)((char*)p - C.base), bytes}); };
+  R.nodes = g->hnodes;
+  R.ppts.assign(g->ppts.size(), DevPPT{});
+  g->d_stats.assign(g->ppts.size(), nullptr);
+  g->d_update_log.assign(g->ppts.size(), nullptr);
+  size_t max_smem_floats = 64;
+  int cta = 1;
+  for (size_t p = 0; p < g->ppts.size(); p++) {
+    const HostPPT& H = g->ppts[p];
+    const DevNode& h = g->hnodes[H.node];
+    DevPPT& P = R.ppts[p];
+    P.node = H.node; P.kind = H.kind; P.in_dim = H.in; P.out_dim = H.out; P.act = h.act; P.flags = h.flags;
+    P.muf_override = g->nodes[H.node].muf_override;
+    P.T = H.T; P.cta0 = cta; cta += H.T; P.R = H.R; P.BM = H.BM; P.J = H.J;
+    P.U = h.U_in; P.rows_max = h.rows_in;
+    P.W = H.W; P.b = H.b;
+    const size_t keys = (size_t)mak * IT * P.U;
+    const bool source_fed = g->hnodes[h.pred_node[0]].type == SOURCE;
+    if (!source_fed) P.xcache = B.take<float>(keys * P.rows_max * P.in_dim);
+    if (H.kind != LOOKUP) P.ycache = B.take<float>(keys * P.rows_max * P.out_dim);
+    P.gbuf = B.take<float>(keys * P.rows_max * P.out_dim);
+    if (H.kind == GRUCELL) {
+      P.zc = B.take<float>(keys * P.rows_max * P.out_dim);
+      P.rc = B.take<float>(keys * P.rows_max * P.out_dim);
+      P.cc = B.take<float>(keys * P.rows_max * P.out_dim);
+      P.part2 = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
+    }
+    P.vcache = B.take<int>(keys);
+    const unsigned cap = pow2_at_least(2ull * keys);
+    if (cap > (1u << 20)) return set_err(g, AMPNET_EINVAL, "node %d: queue capacity %u above the supported 2^20 (lower max_active_keys)", H.node, cap);
+    for (int d = 0; d < 2; d++) {
+      P.ring[d].e = B.take<Hdr>(cap);
+      P.ring[d].seq = C.take<unsigned>(cap);
+      P.ring[d].tail = C.take<unsigned>(1);
+      P.ring[d].mask = cap - 1;
+    }
+    P.sched = B.take<unsigned>(2 * (size_t)cap); P.sched_mask = 2 * cap - 1;
+    P.batches = B.take<BatchDesc>(2 * (size_t)cap); P.batch_mask = 2 * cap - 1;
+    P.batch_pub = C.take<unsigned>(1);
+    P.sortbuf = B.take<unsigned long long>(cap);
+    if (P.T > 1 && H.kind != LOOKUP) P.dxpart = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
+    P.stage = B.take<float>((size_t)P.BM * std::max(P.in_dim, P.out_dim));
+    P.nbar = C.take<unsigned>(1);
+    P.stats = C.take<PPTStats>(1);
+    P.update_log = B.take<int>(g->update_log_cap); P.update_log_cap = g->update_log_cap;
+    if (H.kind == LOOKUP) {
+      P.A = C.take<float>(H.nW);
+      P.touched_flag = C.take<int>(H.in);
+      P.touched_list = C.take<int>(H.in);
+      P.touched_n = C.take<int>(1);
+    }
+    P.smem_floats = (int)H.smem_floats;
+    max_smem_floats = std::max(max_smem_floats, H.smem_floats);
+    g->d_stats[p] = P.stats; g->d_update_log[p] = P.update_log;
+  }
+  for (size_t i = 0; i < R.nodes.size(); i++) {
+    DevNode& n = R.nodes[i];
+    const size_t kin = (size_t)mak * IT * n.U_in, kout = (size_t)mak * IT * n.U_out;
+    switch (n.type) {
+      case CONCAT: {
+        n.jstride = (long long)n.rows_in * n.out_dim;
+        n.jcnt = C.take<int>(kout); track(n.jcnt, kout * sizeof(int));
+        const DevNode& s = R.nodes[n.succ_node[0]];
+        if (is_ppt_type(s.type) && R.ppts[s.ppt].xcache && s.U_in == n.U_out && s.rows_in == n.rows_in) { n.jbuf = R.ppts[s.ppt].xcache; n.jalias = 1; }
+        else n.jbuf = B.take<float>(kout * n.jstride);
+      } break;
+      case GROUP:
+        n.jstride = (long long)n.rows_out * n.in_dim;
+        n.jbuf = B.take<float>(kout * n.jstride);
+        n.jcnt = C.take<int>(kout); track(n.jcnt, kout * sizeof(int));
+        break;
+      case UNGROUP:
+        n.jstride = (long long)n.rows_in * n.in_dim;
+        n.jbuf = B.take<float>(kin * n.jstride);
+        n.jcnt = C.take<int>(kin); track(n.jcnt, kin * sizeof(int));
+        break;
+      case FLATMAP:
+        n.jstride = (long long)(D.maxOut + 1) * n.in_dim;
+        n.jbuf = B.take<float>(kin * n.jstride);
+        n.jcnt = C.take<int>(kin); track(n.jcnt, kin * sizeof(int));
+        break;
+      case BCAST:
+        n.jstride = (long long)(n.fn_arg + 1) * n.rows_in * n.in_dim;
+        n.jbuf = B.take<float>(kin * n.jstride);
+        n.jcnt = C.take<int>(kin); track(n.jcnt, kin * sizeof(int));
+        break;
+      case NPT_SUMROWS:
+        n.jstride = n.in_dim;
+        n.jbuf = B.take<float>(kin * n.jstride);
+        n.rowcnt = C.take<int>(kin); track(n.rowcnt, kin * sizeof(int));
+        break;
+      case LOSS_CE: case LOSS_MSE:
+        n.jstride = n.in_dim;
+        n.jbuf = B.take<float>(kin * n.jstride);
+        n.lossval = B.take<float>(kin);
+        n.predok = B.take<int>(kin);
+        break;
+      case PHI:
+        n.origin = C.take<unsigned char>(kin); track(n.origin, kin);
+        break;
+      default: break;
+    }
+  }
+  Ctx& X = R.ctx;
+  X.n_nodes = (int)R.nodes.size(); X.n_ppts = (int)R.ppts.size(); X.n_ctas = n_ctas;
+  X.nodes = B.take<DevNode>(R.nodes.size());
+  X.ppts = B.take<DevPPT>(R.ppts.size());
+  X.roles = B.take<Role>(R.roles.size());
+  X.inst = D.dev;
+  X.g = C.take<Globals>(1);
+  X.node_msgs = C.take<unsigned long long>(R.nodes.size() * 2);
+  g->d_node_msgs = X.node_msgs;
+  X.n_sources = (int)g->sources.size();
+  for (size_t k = 0; k < g->sources.size(); k++) X.src_nodes[k] = g->sources[k];
+  X.n_loss = (int)g->losses.size();
+  for (size_t k = 0; k < g->losses.size(); k++) X.loss_nodes[k] = g->losses[k];
+  X.slot_inst = B.take<int>(mak);
+  X.outstanding = C.take<int>(mak);
+  X.slot_log = C.take<int>(mak);
+  X.keylog = det ? B.take<KeyLog>((size_t)std::max<long long>(n_order, 1)) : nullptr;
+  g->d_keylog = X.keylog;
+  const unsigned rcap = pow2_at_least(2ull * mak * (unsigned long long)std::max({D.maxT + 1, D.maxL, D.maxM + 1, 2}));
+  X.retire_e = B.take<unsigned>(rcap);
+  X.retire_seq = C.take<unsigned>(rcap);
+  X.retire_mask = rcap - 1;
+  X.order = nullptr; X.n_order = n_order;
+  X.loss_out = B.take<float>((size_t)std::max<long long>(D.n, 1));
+  X.mak = mak; X.muf = cfg ? cfg->min_update_frequency : 1; X.det = det; X.eval = eval; X.IT = IT;
+  X.lr = cfg ? cfg->lr : 0.f;
+  double to = cfg && cfg->timeout_s > 0 ? cfg->timeout_s : 120.0;
+  X.timeout_ns = (unsigned long long)(to * 1e9);
+  R.smem_bytes = max_smem_floats * sizeof(float);
+  return AMPNET_OK;
+}
+
+ampnet_status_t ensure_arenas(ampnet_graph* g, size_t ctl_need, size_t bulk_need) {
+  ctl_need += 4096; bulk_need += 4096;
+  if (ctl_need > g->ctl_cap) {
+    dev_free(g, g->ctl_mem);
+    g->ctl_mem = dev_alloc(g, ctl_need);
+    g->ctl_cap = g->ctl_mem ? ctl_need : 0;
+    if (!g->ctl_mem) return set_err(g, AMPNET_ENOMEM, "device allocation of %zu bytes (queues, counters) failed", ctl_need);
+  }
+  if (bulk_need > g->bulk_cap) {
+    dev_free(g, g->bulk_mem);
+    g->bulk_mem = dev_alloc(g, bulk_need);
+    g->bulk_cap = g->bulk_mem ? bulk_need : 0;
+    if (!g->bulk_mem) return set_err(g, AMPNET_ENOMEM, "device allocation of %zu bytes (keyed caches) failed", bulk_need);
+  }
+  return AMPNET_OK;
+}
+
+ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, const ampnet_run_cfg_t* cfg,
+                        ampnet_epoch_stats_t* out, float* per_instance_loss, double* accuracy) {
+  HostDataset& D = g->data[split];
+  if (!D.loaded) return set_err(g, AMPNET_ESTATE, "no instances loaded for split %d", split);
+  if (mak < 1) return set_err(g, AMPNET_EINVAL, "max_active_keys must be >= 1");
+  if (!eval && cfg->min_update_frequency < 1) return set_err(g, AMPNET_EINVAL, "min_update_frequency must be >= 1");
+  long long n_order = D.n;
+  const long long* order = nullptr;
+  if (cfg && cfg->order) {
+    order = reinterpret_cast<const long long*>(cfg->order); n_order = cfg->n_order;
+    if (n_order < 0) return set_err(g, AMPNET_EINVAL, "n_order must be >= 0");
+    for (long long i = 0; i < n_order; i++)
+      if (order[i] < 0 || order[i] >= D.n) return set_err(g, AMPNET_EINVAL, "order[%lld] = %lld is not an instance", i, (long long)order[i]);
+  }
+  if (det && n_order >= (1ll << 24)) return set_err(g, AMPNET_EINVAL, "the deterministic schedule supports fewer than 2^24 instances per epoch");
+  CUDA_TRY(g, cudaSetDevice(g->device));
+  RunPlan R;
+  ampnet_status_t st = plan_run(g, split, mak, det, eval, cfg, n_order, true, R);
+  if (st != AMPNET_OK) return st;
+  const size_t order_bytes = order ? (size_t)n_order * sizeof(long long) : 0;
+  st = ensure_arenas(g, g->ctl.used, g->bulk.used + order_bytes + 512);
+  if (st != AMPNET_OK) return st;
+  st = plan_run(g, split, mak, det, eval, cfg, n_order, false, R);
+  if (st != AMPNET_OK) return st;
+  if (order) {
+    long long* d_order = g->bulk.take<long long>((size_t)n_order);
+    CUDA_TRY(g, cudaMemcpyAsync(d_order, order, order_bytes, cudaMemcpyHostToDevice, g->stream));
+    R.ctx.order = d_order;
+  }
+  if ((size_t)R.smem_bytes > (size_t)g->max_smem) return set_err(g, AMPNET_EINVAL, "tile needs %zu bytes of shared memory", R.smem_bytes);
+  CUDA_TRY(g, cudaMemsetAsync(g->ctl_mem, 0, g->ctl.used, g->stream));
+  CUDA_TRY(g, cudaMemsetAsync(R.ctx.slot_inst, 0xFF, (size_t)mak * sizeof(int), g->stream));
+  CUDA_TRY(g, cudaMemsetAsync(R.ctx.loss_out, 0, (size_t)std::max<long long>(D.n, 1) * sizeof(float), g->stream));
+  CUDA_TRY(g, cudaMemcpyAsync(R.ctx.nodes, R.nodes.data(), R.nodes.size() * sizeof(DevNode), cudaMemcpyHostToDevice, g->stream));
+  CUDA_TRY(g, cudaMemcpyAsync(R.ctx.ppts, R.ppts.data(), R.ppts.size() * sizeof(DevPPT), cudaMemcpyHostToDevice, g->stream));
+  CUDA_TRY(g, cudaMemcpyAsync(R.ctx.roles, R.roles.data(), R.roles.size() * sizeof(Role), cudaMemcpyHostToDevice, g->stream));
+  CUDA_TRY(g, cudaFuncSetAttribute(ampnet_engine, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)R.smem_bytes));
+  int per_sm = 0;
+  CUDA_TRY(g, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ampnet_engine, THREADS, R.smem_bytes));
+  if (per_sm < 1 || (long long)per_sm * g->n_sms < R.ctx.n_ctas)
+    return set_err(g, AMPNET_EINVAL, "%d CTAs cannot be co-resident (%d per SM)", R.ctx.n_ctas, per_sm);
+  void* args[] = {&R.ctx};
+  CUDA_TRY(g, cudaEventRecord(g->ev0, g->stream));
+  CUDA_TRY(g, cudaLaunchCooperativeKernel((void*)ampnet_engine, dim3(R.ctx.n_ctas), dim3(THREADS), args, R.smem_bytes, g->stream));
+  CUDA_TRY(g, cudaEventRecord(g->ev1, g->stream));
+  Globals G;
+  CUDA_TRY(g, cudaMemcpyAsync(&G, R.ctx.g, sizeof G, cudaMemcpyDeviceToHost, g->stream));
+  g->last_stats.assign(g->ppts.size(), PPTStats{});
+  for (size_t p = 0; p < g->ppts.size(); p++)
+    CUDA_TRY(g, cudaMemcpyAsync(&g->last_stats[p], g->d_stats[p], sizeof(PPTStats), cudaMemcpyDeviceToHost, g->stream));
+  g->last_node_msgs.assign(R.nodes.size() * 2, 0);
+  CUDA_TRY(g, cudaMemcpyAsync(g->last_node_msgs.data(), g->d_node_msgs, g->last_node_msgs.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost, g->stream));
+  if (per_instance_loss)
+    CUDA_TRY(g, cudaMemcpyAsync(per_instance_loss, R.ctx.loss_out, (size_t)D.n * sizeof(float), cudaMemcpyDeviceToHost, g->stream));
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  g->have_run = true;
+  g->n_keylog = det ? G.n_keylog : 0;
+  float ms = 0;
+  CUDA_TRY(g, cudaEventElapsedTime(&ms, g->ev0, g->ev1));
+  if (out) {
+    std::memset(out, 0, sizeof *out);
+    out->instances = n_order; out->node_messages = (int64_t)G.node_messages; out->rounds = (int64_t)G.rounds;
+    out->seconds = ms * 1e-3; out->mean_loss = n_order ? G.total_loss / (double)n_order : 0.0;
+    out->max_active_observed = G.max_active; out->route_hash = G.route_hash;
+    for (auto& s : g->last_stats) {
+      out->ppt_messages += (int64_t)s.msgs; out->max_staleness = std::max(out->max_staleness, s.max_staleness);
+      out->micro_batches += (int64_t)s.batches; out->micro_batch_rows += (int64_t)s.batch_rows;
+    }
+  }
+  if (accuracy) *accuracy = G.n_pred ? (double)G.correct / (double)G.n_pred : 0.0;
+  if (G.status == ST_TIMEOUT) return set_err(g, AMPNET_ETIMEOUT, "a bounded device wait gave up (node %d, detail %d)", G.err_node, G.err_detail);
+  if (G.status == ST_OVERFLOW) return set_err(g, AMPNET_EOVERFLOW, "a queue / cache / key-space bound was exceeded (node %d, detail %d)", G.err_node, G.err_detail);
+  if (G.status != 0) return set_err(g, AMPNET_ECUDA, "device status %d", G.status);
+  return AMPNET_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------------------
+// C ABI
+// ---------------------------------------------------------------------------------------------------------
+extern "C" {
+
+ampnet_status_t ampnet_graph_create(const ampnet_ir_desc_t* ir, uint64_t init_seed, void* cuda_stream,
+                                    const ampnet_allocator_t* allocator, ampnet_graph_t** out) {
+  if (!out) return AMPNET_EINVAL;
+  *out = nullptr;
+  if (!ir || !ir->nodes || ir->n_nodes < 1 || ir->n_edges < 0 || (ir->n_edges > 0 && !ir->edges)) return AMPNET_EINVAL;
+  if (ir->payload_dtype != 0) return AMPNET_EINVAL;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return AMPNET_ECUDA;
+  ampnet_graph* g = new ampnet_graph();
+  g->nodes.assign(ir->nodes, ir->nodes + ir->n_nodes);
+  if (ir->n_edges) g->edges.assign(ir->edges, ir->edges + ir->n_edges);
+  if (allocator) g->alloc = *allocator;
+  g->stream = (cudaStream_t)cuda_stream;
+  ampnet_status_t st = AMPNET_OK;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&g->device) != cudaSuccess || cudaGetDeviceProperties(&prop, g->device) != cudaSuccess) st = AMPNET_ECUDA;
+  if (st == AMPNET_OK) {
+    g->n_sms = prop.multiProcessorCount;
+    g->max_smem = (int)prop.sharedMemPerBlockOptin;
+    if (!prop.cooperativeLaunch) st = set_err(g, AMPNET_ECUDA, "the device does not support cooperative launch");
+  }
+  if (st == AMPNET_OK) st = build_topology(g);
+  if (st == AMPNET_OK) st = create_params(g, init_seed);
+  if (st == AMPNET_OK && (cudaEventCreate(&g->ev0) != cudaSuccess || cudaEventCreate(&g->ev1) != cudaSuccess)) st = AMPNET_ECUDA;
+  if (st != AMPNET_OK) {
+    // keep the message readable through a static buffer: the handle is not returned
+    static thread_local std::string last;
+    last = g->err;
+    ampnet_graph_destroy(g);
+    return st;
+  }
+  *out = g;
+  return AMPNET_OK;
+}
+
+void ampnet_graph_destroy(ampnet_graph_t* g) {
+  if (!g) return;
+  cudaStreamSynchronize(g->stream);
+  for (auto& P : g->ppts) { dev_free(g, P.W); dev_free(g, P.b); }
+  free_dataset(g, g->data[0]);
+  free_dataset(g, g->data[1]);
+  dev_free(g, g->ctl_mem);
+  dev_free(g, g->bulk_mem);
+  if (g->ev0) cudaEventDestroy(g->ev0);
+  if (g->ev1) cudaEventDestroy(g->ev1);
+  delete g;
+}
+
+const char* ampnet_last_error(const ampnet_graph_t* g) { return g ? g->err.c_str() : "invalid handle"; }
+
+ampnet_status_t ampnet_load_instances(ampnet_graph_t* g, int32_t split, const ampnet_instances_t* in) {
+  if (!g) return AMPNET_EINVAL;
+  if (split < 0 || split > 1 || !in) return set_err(g, AMPNET_EINVAL, "bad split or NULL instances");
+  if (in->n_instances < 0 || in->kind < 0 || in->kind > 3) return set_err(g, AMPNET_EINVAL, "bad kind or instance count");
+  CUDA_TRY(g, cudaSetDevice(g->device));
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  free_dataset(g, g->data[split]);
+  HostDataset& D = g->data[split];
+  const long long n = in->n_instances;
+  D.kind = in->kind; D.n = n;
+  // which inputs does the graph need
+  int vocab = 0; bool per_node_labels = false, need_int_labels = false, need_float_labels = false;
+  for (auto& h : g->hnodes) {
+    if (h.type == LOOKUP) vocab = vocab ? std::min(vocab, h.in_dim) : h.in_dim;
+    if (h.type == LOSS_CE) { need_int_labels = true; if (h.fn == 2) per_node_labels = true; }
+    if (h.type == LOSS_MSE) need_float_labels = true;
+  }
+  for (int s : g->sources) {
+    const int fn = g->hnodes[s].fn;
+    const int want = fn == 1 ? 0 : fn == 2 ? 1 : fn == 4 ? 2 : fn == 5 ? 3 : -1;
+    if (want >= 0 && want != in->kind) return set_err(g, AMPNET_EINVAL, "instance kind %d does not match the graph's source (fn %d)", in->kind, fn);
+    if (fn == 1 && g->hnodes[s].out_dim != in->dense_dim) return set_err(g, AMPNET_EINVAL, "dense_dim %d does not match the source width %d", in->dense_dim, g->hnodes[s].out_dim);
+  }
+  if (need_int_labels && !in->labels_i) return set_err(g, AMPNET_EINVAL, "labels_i is required by the loss");
+  if (need_float_labels && !in->labels_f) return set_err(g, AMPNET_EINVAL, "labels_f is required by the loss");
+  D.labels_per_node = per_node_labels ? 1 : 0;
+  DevInst& V = D.dev;
+  V = DevInst{};
+  V.kind = in->kind; V.n = n; V.labels_per_node = D.labels_per_node;
+  ampnet_status_t st;
+  long long total = 0;
+  if (in->kind == AMPNET_KIND_DENSE_ROWS) {
+    if (!in->dense || in->dense_dim < 1) return set_err(g, AMPNET_EINVAL, "dense rows need dense and dense_dim");
+    D.dense_dim = V.dense_dim = in->dense_dim;
+    if ((st = upload_raw(g, D, in->dense, (size_t)n * in->dense_dim, &V.dense)) != AMPNET_OK) return st;
+  } else {
+    if (!in->offsets || !in->tokens) return set_err(g, AMPNET_EINVAL, "offsets and tokens are required");
+    if (in->offsets[0] != 0) return set_err(g, AMPNET_EINVAL, "offsets[0] must be 0");
+    for (long long i = 0; i < n; i++) {
+      const long long len = in->offsets[i + 1] - in->offsets[i];
+      if (len < 1) return set_err(g, AMPNET_EINVAL, "instance %lld is empty", i);
+      if (len > 16000) return set_err(g, AMPNET_EINVAL, "instance %lld has %lld positions (max 16000)", i, len);
+    }
+    total = in->offsets[n];
+    D.total_pos = total;
+    if ((st = upload_raw(g, D, in->offsets, (size_t)n + 1, reinterpret_cast<const int64_t**>(&V.offsets))) != AMPNET_OK) return st;
+    if ((st = upload_raw(g, D, in->tokens, (size_t)total, &V.tokens)) != AMPNET_OK) return st;
+  }
+  if (in->kind == AMPNET_KIND_SEQUENCES) {
+    for (long long i = 0; i < n; i++) D.maxT = std::max<int>(D.maxT, (int)(in->offsets[i + 1] - in->offsets[i]));
+    for (long long k = 0; k < total; k++)
+      if (in->tokens[k] < 0 || (vocab && in->tokens[k] >= vocab)) return set_err(g, AMPNET_EINVAL, "token %lld = %d outside the vocabulary", k, in->tokens[k]);
+  } else if (in->kind == AMPNET_KIND_BINARY_TREES) {
+    if (!in->left || !in->right) return set_err(g, AMPNET_EINVAL, "trees need left and right");
+    std::vector<int> parent((size_t)total, -1), cslot((size_t)total, 0), root((size_t)n, -1), leaf_ids;
+    std::vector<long long> leaf_off((size_t)n + 1, 0);
+    for (long long i = 0; i < n; i++) {
+      const long long o = in->offsets[i];
+      const int m = (int)(in->offsets[i + 1] - o);
+      D.maxM = std::max(D.maxM, m);
+      int nl = 0;
+      for (int u = 0; u < m; u++) {
+        const int l = in->left[o + u], r = in->right[o + u];
+        if ((l < 0) != (r < 0)) return set_err(g, AMPNET_EINVAL, "tree %lld node %d has exactly one child", i, u);
+        if (l >= 0) {
+          if (l >= u || r >= u || l == r) return set_err(g, AMPNET_EINVAL, "tree %lld node %d: children must precede their parent", i, u);
+          if (parent[o + l] >= 0 || parent[o + r] >= 0) return set_err(g, AMPNET_EINVAL, "tree %lld: node with two parents", i);
+          parent[o + l] = u; cslot[o + l] = 0; parent[o + r] = u; cslot[o + r] = 1;
+        } else {
+          const int t = in->tokens[o + u];
+          if (t < 0 || (vocab && t >= vocab)) return set_err(g, AMPNET_EINVAL, "tree %lld leaf %d: token %d outside the vocabulary", i, u, t);
+          leaf_ids.push_back(u); nl++;
+        }
+      }
+      int nroot = 0;
+      for (int u = 0; u < m; u++) if (parent[o + u] < 0) { root[i] = u; nroot++; }
+      if (nroot != 1) return set_err(g, AMPNET_EINVAL, "tree %lld has %d roots", i, nroot);
+      leaf_off[i + 1] = leaf_off[i] + nl;
+      D.maxL = std::max(D.maxL, nl);
+    }
+    if ((st = upload_raw(g, D, in->left, (size_t)total, &V.left)) != AMPNET_OK) return st;
+    if ((st = upload_raw(g, D, in->right, (size_t)total, &V.right)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, parent, &V.parent)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, cslot, &V.child_slot)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, root, &V.root)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, leaf_off, &V.leaf_off)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, leaf_ids, &V.leaf_ids)) != AMPNET_OK) return st;
+  } else if (in->kind == AMPNET_KIND_TYPED_GRAPHS) {
+    if (!in->edge_offsets || !in->edge_src || !in->edge_dst || !in->edge_type) return set_err(g, AMPNET_EINVAL, "graphs need the edge arrays");
+    const long long E = in->edge_offsets[n];
+    D.total_edges = E;
+    int NT = 1;
+    for (long long e = 0; e < E; e++) {
+      if (in->edge_type[e] < 0 || in->edge_type[e] >= MAX_PORTS) return set_err(g, AMPNET_EINVAL, "edge %lld: type %d out of range", e, in->edge_type[e]);
+      NT = std::max(NT, in->edge_type[e] + 1);
+    }
+    for (auto& h : g->hnodes) if (h.type == COND && h.fn == 3) NT = std::max(NT, h.n_succ);
+    D.NT = V.NT = NT;
+    std::vector<long long> out_off((size_t)total + 1, 0), in_off((size_t)total + 1, 0), type_off((size_t)n * NT + 1, 0);
+    std::vector<int> out_list((size_t)E), in_list((size_t)E), type_list((size_t)E), rank_out((size_t)E), rank_in((size_t)E), rank_type((size_t)E);
+    for (long long i = 0; i < n; i++) {
+      const long long o = in->offsets[i], eo = in->edge_offsets[i];
+      const int N = (int)(in->offsets[i + 1] - o), ne = (int)(in->edge_offsets[i + 1] - eo);
+      if (ne < 0) return set_err(g, AMPNET_EINVAL, "graph %lld: negative edge count", i);
+      D.maxN = std::max(D.maxN, N); D.maxD = std::max(D.maxD, ne);
+      std::vector<int> od(N, 0), id(N, 0), td(NT, 0);
+      for (int e = 0; e < ne; e++) {
+        const int s = in->edge_src[eo + e], d = in->edge_dst[eo + e];
+        if (s < 0 || s >= N || d < 0 || d >= N) return set_err(g, AMPNET_EINVAL, "graph %lld edge %d: endpoint out of range", i, e);
+        rank_out[eo + e] = od[s]++; rank_in[eo + e] = id[d]++; rank_type[eo + e] = td[in->edge_type[eo + e]]++;
+      }
+      for (int v = 0; v < N; v++) {
+        if (od[v] == 0 || id[v] == 0) return set_err(g, AMPNET_EINVAL, "graph %lld: node %d has no incoming or no outgoing edge", i, v);
+        out_off[o + v + 1] = out_off[o + v] + od[v]; in_off[o + v + 1] = in_off[o + v] + id[v];
+        D.maxOut = std::max(D.maxOut, od[v]); D.maxIn = std::max(D.maxIn, id[v]);
+        const int t = in->tokens[o + v];
+        if (t < 0 || (vocab && t >= vocab)) return set_err(g, AMPNET_EINVAL, "graph %lld node %d: type %d outside the vocabulary", i, v, t);
+      }
+      for (int c = 0; c < NT; c++) { type_off[i * NT + c + 1] = type_off[i * NT + c] + td[c]; D.maxDc = std::max(D.maxDc, td[c]); }
+      for (int e = 0; e < ne; e++) {
+        const int s = in->edge_src[eo + e], d = in->edge_dst[eo + e], c = in->edge_type[eo + e];
+        out_list[out_off[o + s] + rank_out[eo + e]] = e;
+        in_list[in_off[o + d] + rank_in[eo + e]] = e;
+        type_list[type_off[i * NT + c] + rank_type[eo + e]] = e;
+      }
+    }
+    if ((st = upload_raw(g, D, in->edge_offsets, (size_t)n + 1, reinterpret_cast<const int64_t**>(&V.edge_off))) != AMPNET_OK) return st;
+    if ((st = upload_raw(g, D, in->edge_src, (size_t)E, &V.esrc)) != AMPNET_OK) return st;
+    if ((st = upload_raw(g, D, in->edge_dst, (size_t)E, &V.edst)) != AMPNET_OK) return st;
+    if ((st = upload_raw(g, D, in->edge_type, (size_t)E, &V.etype)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, rank_out, &V.rank_out)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, rank_in, &V.rank_in)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, rank_type, &V.rank_type)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, out_off, &V.out_off)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, in_off, &V.in_off)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, type_off, &V.type_off)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, out_list, &V.out_list)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, in_list, &V.in_list)) != AMPNET_OK) return st;
+    if ((st = upload(g, D, type_list, &V.type_list)) != AMPNET_OK) return st;
+  }
+  if (in->labels_i) {
+    const size_t nl = per_node_labels ? (size_t)total : (size_t)n;
+    int classes = 0;
+    for (int l : g->losses) if (g->hnodes[l].type == LOSS_CE) classes = g->hnodes[l].in_dim;
+    for (size_t k = 0; k < nl && classes; k++)
+      if (in->labels_i[k] < 0 || in->labels_i[k] >= classes) return set_err(g, AMPNET_EINVAL, "label %zu = %d outside 0..%d", k, in->labels_i[k], classes - 1);
+    if ((st = upload_raw(g, D, in->labels_i, nl, &V.labels_i)) != AMPNET_OK) return st;
+  }
+  if (in->labels_f) if ((st = upload_raw(g, D, in->labels_f, (size_t)n, &V.labels_f)) != AMPNET_OK) return st;
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  D.loaded = true;
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_run_epoch(ampnet_graph_t* g, const ampnet_run_cfg_t* cfg, ampnet_epoch_stats_t* out,
+                                 float* per_instance_loss) {
+  if (!g) return AMPNET_EINVAL;
+  if (!cfg) return set_err(g, AMPNET_EINVAL, "NULL run configuration");
+  return execute(g, 0, cfg->max_active_keys, cfg->deterministic ? 1 : 0, 0, cfg, out, per_instance_loss, nullptr);
+}
+
+ampnet_status_t ampnet_eval(ampnet_graph_t* g, int32_t split, int32_t max_active_keys, double* mean_loss,
+                            double* accuracy, float* per_instance_loss) {
+  if (!g) return AMPNET_EINVAL;
+  if (split < 0 || split > 1) return set_err(g, AMPNET_EINVAL, "bad split");
+  ampnet_run_cfg_t cfg{};
+  cfg.max_active_keys = max_active_keys > 0 ? max_active_keys : 64;
+  cfg.min_update_frequency = 1;
+  ampnet_epoch_stats_t st{};
+  ampnet_status_t rc = execute(g, split, cfg.max_active_keys, 0, 1, &cfg, &st, per_instance_loss, accuracy);
+  if (mean_loss) *mean_loss = st.mean_loss;
+  return rc;
+}
+
+static HostPPT* find_ppt(ampnet_graph_t* g, int node) {
+  if (!g || node < 0 || node >= (int)g->hnodes.size() || g->hnodes[node].ppt < 0) return nullptr;
+  return &g->ppts[g->hnodes[node].ppt];
+}
+static bool param_slice(const HostPPT& P, int which, float** base, size_t* n) {
+  if (P.kind == LINEAR) {
+    if (which == 0) { *base = P.W; *n = P.nW; return true; }
+    if (which == 1) { *base = P.b; *n = P.nb; return true; }
+  } else if (P.kind == LOOKUP) {
+    if (which == 0) { *base = P.W; *n = P.nW; return true; }
+  } else if (P.kind == GRUCELL) {
+    const size_t m = (size_t)P.in * P.out;
+    if (which >= 0 && which < 3) { *base = P.W + which * m; *n = m; return true; }
+    if (which >= 3 && which < 6) { *base = P.b + (which - 3) * P.out; *n = P.out; return true; }
+  }
+  return false;
+}
+
+ampnet_status_t ampnet_param_count(ampnet_graph_t* g, int32_t node, int32_t which, int64_t* n) {
+  HostPPT* P = find_ppt(g, node);
+  float* b; size_t c;
+  if (!P || !n || !param_slice(*P, which, &b, &c)) return g ? set_err(g, AMPNET_EINVAL, "no parameter (%d, %d)", node, which) : AMPNET_EINVAL;
+  *n = (int64_t)c;
+  return AMPNET_OK;
+}
+ampnet_status_t ampnet_get_params(ampnet_graph_t* g, int32_t node, int32_t which, float* dst, int64_t n) {
+  HostPPT* P = find_ppt(g, node);
+  float* b; size_t c;
+  if (!P || !dst || !param_slice(*P, which, &b, &c) || (int64_t)c != n) return g ? set_err(g, AMPNET_EINVAL, "bad parameter request (%d, %d, %lld)", node, which, (long long)n) : AMPNET_EINVAL;
+  CUDA_TRY(g, cudaMemcpyAsync(dst, b, c * sizeof(float), cudaMemcpyDeviceToHost, g->stream));
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  return AMPNET_OK;
+}
+ampnet_status_t ampnet_set_params(ampnet_graph_t* g, int32_t node, int32_t which, const float* src, int64_t n) {
+  HostPPT* P = find_ppt(g, node);
+  float* b; size_t c;
+  if (!P || !src || !param_slice(*P, which, &b, &c) || (int64_t)c != n) return g ? set_err(g, AMPNET_EINVAL, "bad parameter request (%d, %d, %lld)", node, which, (long long)n) : AMPNET_EINVAL;
+  CUDA_TRY(g, cudaMemcpyAsync(b, src, c * sizeof(float), cudaMemcpyHostToDevice, g->stream));
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_get_node_stats(ampnet_graph_t* g, int32_t node, int64_t* n_updates, int64_t* n_grads_applied,
+                                      int64_t* staleness_hist, int64_t* fwd_msgs, int64_t* bwd_msgs) {
+  if (!g) return AMPNET_EINVAL;
+  if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
+  if (node < 0 || node >= (int)g->hnodes.size()) return set_err(g, AMPNET_EINVAL, "bad node");
+  if (fwd_msgs) *fwd_msgs = (int64_t)g->last_node_msgs[node * 2];
+  if (bwd_msgs) *bwd_msgs = (int64_t)g->last_node_msgs[node * 2 + 1];
+  const int p = g->hnodes[node].ppt;
+  if (n_updates) *n_updates = p >= 0 ? (int64_t)g->last_stats[p].n_updates : 0;
+  if (n_grads_applied) *n_grads_applied = p >= 0 ? (int64_t)g->last_stats[p].n_grads_applied : 0;
+  if (staleness_hist) for (int k = 0; k < 64; k++) staleness_hist[k] = p >= 0 ? (int64_t)g->last_stats[p].stale_hist[k] : 0;
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_get_update_log(ampnet_graph_t* g, int32_t node, int32_t* n_per_update, int64_t cap, int64_t* n) {
+  if (!g) return AMPNET_EINVAL;
+  if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
+  if (node < 0 || node >= (int)g->hnodes.size() || g->hnodes[node].ppt < 0) return set_err(g, AMPNET_EINVAL, "not a parameterised node");
+  const int p = g->hnodes[node].ppt;
+  const int64_t have = std::min<int64_t>(g->last_stats[p].log_n, g->update_log_cap);
+  if (n) *n = g->last_stats[p].log_n;
+  const int64_t c = std::min(have, cap);
+  if (c > 0 && n_per_update) {
+    CUDA_TRY(g, cudaMemcpyAsync(n_per_update, g->d_update_log[p], (size_t)c * sizeof(int), cudaMemcpyDeviceToHost, g->stream));
+    CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  }
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_get_key_log(ampnet_graph_t* g, int64_t* inst, int32_t* slot, int64_t* admit_round,
+                                   int64_t* release_round, int64_t cap, int64_t* n) {
+  if (!g) return AMPNET_EINVAL;
+  if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
+  if (n) *n = g->n_keylog;
+  const int64_t c = std::min<int64_t>(g->n_keylog, cap);
+  if (c > 0) {
+    std::vector<KeyLog> h((size_t)c);
+    CUDA_TRY(g, cudaMemcpyAsync(h.data(), g->d_keylog, (size_t)c * sizeof(KeyLog), cudaMemcpyDeviceToHost, g->stream));
+    CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+    for (int64_t i = 0; i < c; i++) {
+      if (inst) inst[i] = h[i].inst;
+      if (slot) slot[i] = h[i].slot;
+      if (admit_round) admit_round[i] = h[i].admit;
+      if (release_round) release_round[i] = h[i].release;
+    }
+  }
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_leftover_cache_entries(ampnet_graph_t* g, int64_t* n) {
+  if (!g || !n) return AMPNET_EINVAL;
+  if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
+  int64_t cnt = 0;
+  std::vector<unsigned char> h;
+  for (auto& r : g->leftover_regions) {
+    h.resize(r.second);
+    CUDA_TRY(g, cudaMemcpyAsync(h.data(), (char*)g->ctl_mem + r.first, r.second, cudaMemcpyDeviceToHost, g->stream));
+    CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+    for (unsigned char c : h) cnt += c != 0;
+  }
+  *n = cnt;
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_get_placement(ampnet_graph_t* g, int32_t node, int32_t* n_tiles, int32_t* batch_rows) {
+  HostPPT* P = find_ppt(g, node);
+  if (!P) return g ? set_err(g, AMPNET_EINVAL, "not a parameterised node") : AMPNET_EINVAL;
+  if (n_tiles) *n_tiles = P->T;
+  if (batch_rows) *batch_rows = P->BM;
+  return AMPNET_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,1209 @@
+// Persistent message-driven training kernel (device code).
+//
+// One CTA per role: CTA 0 is the controller (admission under max_active_keys, retirement, Sec. 3 / Sec. 4
+// "controller loop"); every other CTA owns one row tile of one parameterised (PPT) node and keeps that
+// tile's weights and fp32 gradient accumulators in shared memory for the whole epoch.  Messages are headers
+// in per-node ring queues; their payloads live in caches keyed by (key slot, iteration, position), which
+// double as the activation caches of Sec. 4.  The parameter-free nodes (Cond, Phi, Isu, Concat, Bcast,
+// Group, Ungroup, Flatmap, row sum, Loss, Sink) are executed by the warp that emits a message: it walks
+// the IR graph until the message lands in the input cache and queue of the next PPT node.
+#pragma once
+#include <cuda_runtime.h>
+#include "engine_types.h"
+
+namespace amp {
+
+// ------------------------------------------------------------------------------------------------
+// memory-model helpers, bounded waits
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned ld_acq(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_rel(unsigned* p, unsigned v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void fail(const Ctx& C, int code, int node, int detail) {
+  if (atomicCAS(&C.g->status, 0, code) == 0) { C.g->err_node = node; C.g->err_detail = detail; }
+  __threadfence();
+  st_rel(&C.g->abort_flag, 1u);
+}
+__device__ __forceinline__ bool aborted(const Ctx& C) { return ld_acq(&C.g->abort_flag) != 0; }
+
+// Every wait in the kernel goes through this: it gives up when another CTA has raised the abort word or
+// when the run's time budget is spent (status AMPNET_ETIMEOUT), so no wait can hang the GPU.
+template <class Cond>
+__device__ __forceinline__ bool spin_until(const Ctx& C, unsigned long long t0, Cond cond) {
+  unsigned it = 0;
+  while (!cond()) {
+    if ((++it & 31u) == 0) {
+      if (aborted(C)) return false;
+      if (gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, -1, 0); return false; }
+    }
+    __nanosleep(it < 64 ? 20 : 100);
+  }
+  return true;
+}
+
+// Barrier among `n` CTAs on a monotone counter; gen is the caller's local generation.  Returns false on abort.
+__device__ __forceinline__ bool cta_barrier(const Ctx& C, unsigned long long t0, unsigned* ctr, unsigned n,
+                                            unsigned& gen, int* s_ok) {
+  __syncthreads();
+  gen++;
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(ctr, 1u);
+    unsigned target = gen * n;
+    bool ok = spin_until(C, t0, [&] { return ld_acq(ctr) >= target; });
+    __threadfence();
+    *s_ok = ok ? 1 : 0;
+  }
+  __syncthreads();
+  return *s_ok != 0;
+}
+
+__device__ __forceinline__ long long key_of(const Ctx& C, int node, int slot, int it, int u, int U) {
+  if ((unsigned)slot >= (unsigned)C.mak || (unsigned)it >= (unsigned)C.IT || (unsigned)u >= (unsigned)U) {
+    fail(C, ST_OVERFLOW, node, u);
+    return -1;
+  }
+  return ((long long)slot * C.IT + it) * U + u;
+}
+
+__device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
+  x += 0x9E3779B97F4A7C15ull;
+  x = (x ^ (x >> 30)) * 0xBF58476D1CE4E5B9ull;
+  x = (x ^ (x >> 27)) * 0x94D049BB133111EBull;
+  return x ^ (x >> 31);
+}
+
+// ------------------------------------------------------------------------------------------------
+// walking warp: executes the parameter-free nodes between two PPT nodes
+// ------------------------------------------------------------------------------------------------
+struct Frame {
+  int node, aport, dir, iter;
+  int inst, seq, slot, it, u, port, rows, flags;
+  int dim, ld;
+  const float* p;       // payload rows (device memory); nullptr = zeros
+};
+
+struct WalkAcc { unsigned long long msgs, hash; };
+
+__device__ __forceinline__ void warp_copy(float* dst, int dld, const float* src, int sld, int rows, int dim,
+                                          int lane) {
+  for (int r = 0; r < rows; r++)
+    for (int i = lane; i < dim; i += 32) dst[(size_t)r * dld + i] = src ? __ldcg(src + (size_t)r * sld + i) : 0.f;
+}
+
+__device__ __forceinline__ void ring_push(Ring& r, const Frame& f) {   // one lane, after the payload is fenced
+  unsigned t = atomicAdd(r.tail, 1u);
+  unsigned s = t & r.mask;
+  int4* d = reinterpret_cast<int4*>(&r.e[s]);
+  d[0] = make_int4(f.inst, f.seq, f.slot, f.it);
+  d[1] = make_int4(f.u, f.port, f.rows, f.flags);
+  st_rel(&r.seq[s], t + 1u);
+}
+
+__device__ __forceinline__ void retire_push(const Ctx& C, int slot) {
+  unsigned t = atomicAdd(&C.g->retire_tail, 1u);
+  unsigned s = t & C.retire_mask;
+  C.retire_e[s] = (unsigned)slot;
+  st_rel(&C.retire_seq[s], t + 1u);
+}
+
+// Join on a keyed counter: every arriving warp has written its part; the one that completes the count
+// continues.  Returns true for the completing arrival (and resets the counter for the key's next use).
+__device__ __forceinline__ bool join_arrive(int* cnt, int expected, int lane) {
+  __threadfence();
+  __syncwarp();
+  int last = 0;
+  if (lane == 0) {
+    int old = atomicAdd(cnt, 1);
+    last = (old + 1 == expected);
+    if (last) { *cnt = 0; }
+  }
+  last = __shfl_sync(0xffffffffu, last, 0);
+  if (last) __threadfence();
+  return last != 0;
+}
+
+__device__ __forceinline__ void to_succ(Frame& f, const DevNode& n, int k) {
+  f.node = n.succ_node[k]; f.aport = n.succ_port[k]; f.dir = FWD; f.iter = 0;
+}
+__device__ __forceinline__ void to_pred(Frame& f, const DevNode& n, int j) {
+  f.node = n.pred_node[j]; f.aport = n.pred_port[j]; f.dir = BWD; f.iter = 0;
+}
+
+__device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
+  const int lane = threadIdx.x & 31;
+  const DevInst& I = C.inst;
+  int sp = 0;
+  bool have = true;
+  while (have) {
+    if (f.node < 0) { fail(C, ST_OVERFLOW, -2, 0); return; }
+    const DevNode& n = C.nodes[f.node];
+    bool cont = false;                       // true: f was rewritten and continues
+    if (n.type == SOURCE) {                  // a source message came home to the controller
+      if (f.dir == BWD && lane == 0) retire_push(C, f.slot);
+    } else {
+      if (f.iter == 0) {
+        acc.msgs++;
+        unsigned long long a = (unsigned long long)f.node | ((unsigned long long)f.dir << 16) |
+                               ((unsigned long long)(f.aport & 0xff) << 20) | ((unsigned long long)(f.port & 0xff) << 28);
+        unsigned long long b = ((unsigned long long)(unsigned)f.inst << 32) | ((unsigned long long)(f.it & 0xff) << 24) |
+                               (unsigned long long)(f.u & 0xffffff);
+        acc.hash += mix64(mix64(a) ^ (b * 0x9E3779B97F4A7C15ull));
+        if (lane == 0) atomicAdd(&C.node_msgs[f.node * 2 + f.dir], 1ull);
+      }
+      const long long ibase = I.offsets ? I.offsets[f.inst] : 0;     // first position of the instance
+      switch (n.type) {
+        case LINEAR: case LOOKUP: case GRUCELL: {
+          DevPPT& P = C.ppts[n.ppt];
+          long long key = key_of(C, f.node, f.slot, f.it, f.u, P.U);
+          if (key < 0) return;
+          if (f.rows > P.rows_max) { fail(C, ST_OVERFLOW, f.node, f.rows); return; }
+          if (f.dir == FWD) {
+            if (P.xcache) {
+              float* dst = P.xcache + key * (long long)P.rows_max * P.in_dim;
+              if (f.p != dst) warp_copy(dst, P.in_dim, f.p, f.ld, f.rows, P.in_dim, lane);
+            }
+          } else if (n.type != LOOKUP || f.dim > 0) {
+            warp_copy(P.gbuf + key * (long long)P.rows_max * P.out_dim, P.out_dim, f.p, f.ld, f.rows, P.out_dim, lane);
+          }
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) ring_push(P.ring[f.dir], f);
+        } break;
+        case LOSS_CE: case LOSS_MSE: {
+          long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
+          if (key < 0) return;
+          float* g = n.jbuf + key * n.jstride;
+          if (n.type == LOSS_CE) {
+            int label = I.labels_i[I.labels_per_node ? ibase + f.u : f.inst];
+            float mx = -3.4e38f; int arg = 0x7fffffff;
+            for (int j = lane; j < n.in_dim; j += 32) { float v = __ldcg(f.p + j); if (v > mx) { mx = v; arg = j; } }
+            for (int o = 16; o; o >>= 1) {
+              float om = __shfl_xor_sync(0xffffffffu, mx, o); int oa = __shfl_xor_sync(0xffffffffu, arg, o);
+              if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+            }
+            float s = 0.f;
+            for (int j = lane; j < n.in_dim; j += 32) s += expf(__ldcg(f.p + j) - mx);
+            for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+            float lse = mx + logf(s);
+            for (int j = lane; j < n.in_dim; j += 32) g[j] = expf(__ldcg(f.p + j) - lse) - (j == label ? 1.f : 0.f);
+            if (lane == 0) { n.lossval[key] = lse - __ldcg(f.p + label); n.predok[key] = (arg == label) ? 1 : 0; }
+          } else {
+            if (lane == 0) {
+              float d = __ldcg(f.p) - I.labels_f[f.inst];
+              n.lossval[key] = d * d; g[0] = 2.f * d; n.predok[key] = 0;
+            }
+          }
+          if (f.flags & HDR_EVAL) { __threadfence(); __syncwarp(); if (lane == 0) retire_push(C, f.slot); }
+          else { __syncwarp(); f.p = g; f.dim = n.in_dim; f.ld = n.in_dim; to_pred(f, n, 0); cont = true; }
+        } break;
+        case SINK:
+          if (f.flags & HDR_EVAL) { if (lane == 0) retire_push(C, f.slot); }
+          else { f.p = nullptr; to_pred(f, n, 0); cont = true; }
+          break;
+        case COND:
+          if (f.dir == FWD) {
+            int k = 0;
+            switch (n.fn) {
+              case 1: k = f.u < (int)(I.offsets[f.inst + 1] - ibase) ? 0 : 1; break;
+              case 2: k = f.u == I.root[f.inst] ? 0 : 1; break;
+              case 3: k = f.u; break;
+              case 4: k = f.it < n.fn_arg ? 0 : 1; break;
+            }
+            if ((unsigned)k >= (unsigned)n.n_succ) { fail(C, ST_OVERFLOW, f.node, k); return; }
+            to_succ(f, n, k);
+          } else to_pred(f, n, 0);
+          cont = true;
+          break;
+        case PHI: {
+          long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
+          if (key < 0) return;
+          if (f.dir == FWD) {
+            if (lane == 0 && !(f.flags & HDR_EVAL)) n.origin[key] = (unsigned char)(f.aport + 1);
+            to_succ(f, n, 0);
+          } else {
+            int j = (int)*(volatile unsigned char*)&n.origin[key] - 1;
+            if (j < 0 || j >= n.n_pred) { fail(C, ST_OVERFLOW, f.node, j); return; }
+            __syncwarp();
+            if (lane == 0) n.origin[key] = 0;
+            to_pred(f, n, j);
+          }
+          cont = true;
+        } break;
+        case ISU:
+          if (f.dir == FWD) {
+            if (n.fn == 1) f.u += 1;
+            else if (n.fn == 2) { f.port = I.child_slot[ibase + f.u]; f.u = I.parent[ibase + f.u]; }
+            else f.it += 1;
+            to_succ(f, n, 0);
+          } else {
+            if (n.fn == 1) f.u -= 1;
+            else if (n.fn == 2) { f.u = f.port == 0 ? I.left[ibase + f.u] : I.right[ibase + f.u]; f.port = 0; }
+            else f.it -= 1;
+            to_pred(f, n, 0);
+          }
+          cont = true;
+          break;
+        case BCAST:
+          if (f.dir == FWD) {
+            int k = f.iter;
+            if (k + 1 < n.fn_arg) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                    Frame c = f; c.iter = k + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            to_succ(f, n, k);
+            cont = true;
+          } else {
+            long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
+            if (key < 0) return;
+            float* base = n.jbuf + key * n.jstride;
+            const int blk = n.rows_in * n.in_dim;
+            warp_copy(base + (size_t)f.aport * blk, n.in_dim, f.p, f.ld, f.rows, n.in_dim, lane);
+            if (join_arrive(&n.jcnt[key], n.fn_arg, lane)) {
+              float* sum = base + (size_t)n.fn_arg * blk;
+              for (int i = lane; i < f.rows * n.in_dim; i += 32) {
+                float s = 0.f;
+                for (int k = 0; k < n.fn_arg; k++) s += __ldcg(base + (size_t)k * blk + i);   // successor order
+                sum[i] = s;
+              }
+              __syncwarp();
+              f.p = sum; f.ld = n.in_dim; f.dim = n.in_dim;
+              to_pred(f, n, 0);
+              cont = true;
+            }
+          }
+          break;
+        case CONCAT:
+          if (f.dir == FWD) {
+            int port = n.fn == 2 ? f.port : f.aport;
+            long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_out);
+            if (key < 0) return;
+            if ((unsigned)port >= (unsigned)n.fn_arg || f.rows > n.rows_in) { fail(C, ST_OVERFLOW, f.node, port); return; }
+            float* base = n.jbuf + key * n.jstride;
+            warp_copy(base + port * n.in_dim, n.out_dim, f.p, f.ld, f.rows, n.in_dim, lane);
+            if (join_arrive(&n.jcnt[key], n.fn_arg, lane)) {
+              f.p = base; f.dim = n.out_dim; f.ld = n.out_dim; f.port = 0;
+              to_succ(f, n, 0);
+              cont = true;
+            }
+          } else {
+            int k = f.iter;
+            if (k + 1 < n.fn_arg) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                    Frame c = f; c.iter = k + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            f.p = f.p ? f.p + k * n.in_dim : nullptr; f.dim = n.in_dim;
+            if (n.fn == 2) { f.port = k; to_pred(f, n, 0); } else to_pred(f, n, k);
+            cont = true;
+          }
+          break;
+        case GROUP:
+          if (f.dir == FWD) {
+            int gkey = 0, member = 0, count = 1;
+            const long long ebase = I.edge_off ? I.edge_off[f.inst] : 0;
+            if (n.fn == 1) { int c = I.etype[ebase + f.u]; gkey = c; member = I.rank_type[ebase + f.u];
+                             const long long* to = I.type_off + (long long)f.inst * I.NT + c; count = (int)(to[1] - to[0]); }
+            else if (n.fn == 2) { int v = I.edst[ebase + f.u]; gkey = v; member = I.rank_in[ebase + f.u];
+                                  count = (int)(I.in_off[ibase + v + 1] - I.in_off[ibase + v]); }
+            else { gkey = 0; member = f.u; count = (int)(I.offsets[f.inst + 1] - ibase); }
+            long long key = key_of(C, f.node, f.slot, f.it, gkey, n.U_out);
+            if (key < 0) return;
+            if (member >= n.rows_out || count > n.rows_out) { fail(C, ST_OVERFLOW, f.node, member); return; }
+            float* base = n.jbuf + key * n.jstride;
+            warp_copy(base + (size_t)member * n.in_dim, n.in_dim, f.p, f.ld, 1, n.in_dim, lane);
+            if (join_arrive(&n.jcnt[key], count, lane)) {
+              f.u = gkey; f.rows = count; f.p = base; f.ld = n.in_dim; f.dim = n.in_dim;
+              to_succ(f, n, 0);
+              cont = true;
+            }
+          } else {
+            int i = f.iter;
+            if (i + 1 < f.rows) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                  Frame c = f; c.iter = i + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            const long long ebase = I.edge_off ? I.edge_off[f.inst] : 0;
+            int mu;
+            if (n.fn == 1) mu = I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i];
+            else if (n.fn == 2) mu = I.in_list[I.in_off[ibase + f.u] + i];
+            else mu = i;
+            (void)ebase;
+            f.p = f.p ? f.p + (size_t)i * f.ld : nullptr; f.rows = 1; f.u = mu;
+            to_pred(f, n, 0);
+            cont = true;
+          }
+          break;
+        case UNGROUP:
+          if (f.dir == FWD) {
+            int i = f.iter;
+            if (i + 1 < f.rows) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                  Frame c = f; c.iter = i + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            int mu = n.fn == 2 ? I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i] : i;
+            f.p = f.p ? f.p + (size_t)i * f.ld : nullptr; f.rows = 1; f.u = mu;
+            to_succ(f, n, 0);
+            cont = true;
+          } else {
+            int gkey, row, expected;
+            if (n.fn == 2) { const long long ebase = I.edge_off[f.inst]; gkey = I.etype[ebase + f.u]; row = I.rank_type[ebase + f.u];
+                             const long long* to = I.type_off + (long long)f.inst * I.NT + gkey; expected = (int)(to[1] - to[0]); }
+            else { gkey = 0; row = f.u; expected = (int)(I.offsets[f.inst + 1] - ibase); }
+            long long key = key_of(C, f.node, f.slot, f.it, gkey, n.U_in);
+            if (key < 0) return;
+            if (row >= n.rows_in) { fail(C, ST_OVERFLOW, f.node, row); return; }
+            float* base = n.jbuf + key * n.jstride;
+            warp_copy(base + (size_t)row * n.in_dim, n.in_dim, f.p, f.ld, 1, n.in_dim, lane);
+            if (join_arrive(&n.jcnt[key], expected, lane)) {
+              f.u = gkey; f.rows = expected; f.p = base; f.ld = n.in_dim; f.dim = n.in_dim;
+              to_pred(f, n, 0);
+              cont = true;
+            }
+          }
+          break;
+        case FLATMAP: {
+          if (f.dir == FWD) {
+            const long long* oo = I.out_off + ibase + f.u;
+            int deg = (int)(oo[1] - oo[0]);
+            int i = f.iter;
+            if (deg > 0) {
+              if (i + 1 < deg) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                 Frame c = f; c.iter = i + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+              f.u = I.out_list[oo[0] + i];
+              to_succ(f, n, 0);
+              cont = true;
+            }
+          } else {
+            const long long ebase = I.edge_off[f.inst];
+            int v = I.esrc[ebase + f.u], member = I.rank_out[ebase + f.u];
+            int deg = (int)(I.out_off[ibase + v + 1] - I.out_off[ibase + v]);
+            long long key = key_of(C, f.node, f.slot, f.it, v, n.U_in);
+            if (key < 0) return;
+            const int maxdeg = (int)(n.jstride / n.in_dim) - 1;
+            if (member >= maxdeg || deg > maxdeg) { fail(C, ST_OVERFLOW, f.node, member); return; }
+            float* base = n.jbuf + key * n.jstride;
+            warp_copy(base + (size_t)member * n.in_dim, n.in_dim, f.p, f.ld, 1, n.in_dim, lane);
+            if (join_arrive(&n.jcnt[key], deg, lane)) {
+              float* sum = base + (size_t)maxdeg * n.in_dim;
+              for (int i = lane; i < n.in_dim; i += 32) {
+                float s = 0.f;
+                for (int k = 0; k < deg; k++) s += __ldcg(base + (size_t)k * n.in_dim + i);     // edge order
+                sum[i] = s;
+              }
+              __syncwarp();
+              f.u = v; f.rows = 1; f.p = sum; f.ld = n.in_dim; f.dim = n.in_dim;
+              to_pred(f, n, 0);
+              cont = true;
+            }
+          }
+        } break;
+        case NPT_SUMROWS: {
+          long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
+          if (key < 0) return;
+          if (f.dir == FWD) {
+            float* out = n.jbuf + key * n.jstride;
+            for (int i = lane; i < n.in_dim; i += 32) {
+              float s = 0.f;
+              for (int r = 0; r < f.rows; r++) s += f.p ? __ldcg(f.p + (size_t)r * f.ld + i) : 0.f;   // row order
+              out[i] = s;
+            }
+            if (lane == 0 && !(f.flags & HDR_EVAL)) n.rowcnt[key] = f.rows;
+            __syncwarp();
+            f.rows = 1; f.p = out; f.ld = n.in_dim; f.dim = n.in_dim;
+            to_succ(f, n, 0);
+          } else {
+            int rows = *(volatile int*)&n.rowcnt[key];
+            __syncwarp();
+            if (lane == 0) n.rowcnt[key] = 0;
+            f.rows = rows; f.ld = 0;         // the same gradient row for every summed row
+            to_pred(f, n, 0);
+          }
+          cont = true;
+        } break;
+        default:
+          fail(C, ST_OVERFLOW, f.node, n.type);
+          return;
+      }
+    }
+    if (!cont) {
+      if (sp > 0) { __syncwarp(); f = stack[--sp]; __syncwarp(); }
+      else have = false;
+    }
+  }
+}
+
+__device__ __forceinline__ void flush_acc(const Ctx& C, WalkAcc& a, int lane) {
+  if (lane == 0 && a.msgs) {
+    atomicAdd(&C.g->node_messages, a.msgs);
+    atomicAdd(&C.g->route_hash, a.hash);
+  }
+  a.msgs = 0; a.hash = 0;
+}
+
+// ------------------------------------------------------------------------------------------------
+// tile arithmetic: lanes stride over the input dimension (column i = lane + 32 j)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ float act_fwd(int a, float v) {
+  switch (a) {
+    case 1: return v > 0.f ? v : 0.f;
+    case 2: return tanhf(v);
+    case 3: return 1.f / (1.f + expf(-v));
+    default: return v;
+  }
+}
+__device__ __forceinline__ float act_grad(int a, float y) {
+  switch (a) {
+    case 1: return y > 0.f ? 1.f : 0.f;
+    case 2: return 1.f - y * y;
+    case 3: return y * (1.f - y);
+    default: return 1.f;
+  }
+}
+
+// out[b][r] = sum_i X[b][i] * W[r][i]  for b < nb, r < R.  4 batch rows x 4 weight rows per warp pass; the 16
+// lane-partial sums are reduced across the warp with a halving butterfly (16 shuffles instead of 80).
+template <int J>
+__device__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const float* __restrict__ Ws, int ldw, int R,
+                         int in_dim, float* __restrict__ out, int ldo) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nbg = (nb + 3) >> 2, nrg = (R + 3) >> 2;
+  for (int unit = warp; unit < nbg * nrg; unit += WARPS) {
+    const int b0 = (unit / nrg) * 4, r0 = (unit % nrg) * 4;
+    float acc[16];
+#pragma unroll
+    for (int k = 0; k < 16; k++) acc[k] = 0.f;
+#pragma unroll
+    for (int j = 0; j < J; j++) {
+      const int i = lane + 32 * j;
+      if (i < in_dim) {
+        float x[4], w[4];
+#pragma unroll
+        for (int m = 0; m < 4; m++) x[m] = (b0 + m < nb) ? Xs[(b0 + m) * ldx + i] : 0.f;
+#pragma unroll
+        for (int q = 0; q < 4; q++) w[q] = (r0 + q < R) ? Ws[(r0 + q) * ldw + i] : 0.f;
+#pragma unroll
+        for (int m = 0; m < 4; m++)
+#pragma unroll
+          for (int q = 0; q < 4; q++) acc[m * 4 + q] = fmaf(x[m], w[q], acc[m * 4 + q]);
+      }
+    }
+    // halving butterfly: after the step with offset o, a lane keeps the half of its values selected by bit o
+#pragma unroll
+    for (int h = 8, o = 16; h >= 1; h >>= 1, o >>= 1) {
+      const bool up = (lane & o) != 0;
+#pragma unroll
+      for (int k = 0; k < h; k++) {
+        float send = up ? acc[k] : acc[k + h];
+        float keep = up ? acc[k + h] : acc[k];
+        acc[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+      }
+    }
+    float v = acc[0] + __shfl_xor_sync(0xffffffffu, acc[0], 1);
+    // lane bits (16,8,4,2) selected value index k = 8*b16 + 4*b8 + 2*b4 + b2
+    const int k = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
+    const int m = k >> 2, q = k & 3;
+    if ((lane & 1) == 0 && b0 + m < nb && r0 + q < R) out[(b0 + m) * ldo + r0 + q] = v;
+  }
+}
+
+// dx[b][i] = sum_r D[b][r] * W[r][i], written to dst (device memory, ld = in_dim).
+template <int J>
+__device__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Ws, int ldw, int R,
+                        int in_dim, float* __restrict__ dst) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int b0 = warp * 4; b0 < nb; b0 += WARPS * 4) {
+    float acc[4][J];
+#pragma unroll
+    for (int m = 0; m < 4; m++)
+#pragma unroll
+      for (int j = 0; j < J; j++) acc[m][j] = 0.f;
+    for (int r = 0; r < R; r++) {
+      float d[4];
+#pragma unroll
+      for (int m = 0; m < 4; m++) d[m] = (b0 + m < nb) ? Ds[(b0 + m) * ldd + r] : 0.f;
+#pragma unroll
+      for (int j = 0; j < J; j++) {
+        const int i = lane + 32 * j;
+        const float w = i < in_dim ? Ws[r * ldw + i] : 0.f;
+#pragma unroll
+        for (int m = 0; m < 4; m++) acc[m][j] = fmaf(d[m], w, acc[m][j]);
+      }
+    }
+#pragma unroll
+    for (int m = 0; m < 4; m++)
+      if (b0 + m < nb)
+#pragma unroll
+        for (int j = 0; j < J; j++) {
+          const int i = lane + 32 * j;
+          if (i < in_dim) dst[(size_t)(b0 + m) * in_dim + i] = acc[m][j];
+        }
+  }
+}
+
+// A[r][i] += sum_b D[b][r] * X[b][i];  work unit = 4 weight rows x 4 column chunks.
+__device__ void tile_accum(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Xs, int ldx,
+                           float* __restrict__ As, int lda, int R, int in_dim) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int nj = (in_dim + 31) >> 5, ncg = (nj + 3) >> 2, nrg = (R + 3) >> 2;
+  for (int unit = warp; unit < nrg * ncg; unit += WARPS) {
+    const int r0 = (unit / ncg) * 4, j0 = (unit % ncg) * 4;
+    float a[4][4];
+#pragma unroll
+    for (int q = 0; q < 4; q++)
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const int i = lane + 32 * (j0 + j);
+        a[q][j] = (r0 + q < R && i < in_dim) ? As[(r0 + q) * lda + i] : 0.f;
+      }
+    for (int b = 0; b < nb; b++) {
+      float d[4], x[4];
+#pragma unroll
+      for (int q = 0; q < 4; q++) d[q] = (r0 + q < R) ? Ds[b * ldd + r0 + q] : 0.f;
+#pragma unroll
+      for (int j = 0; j < 4; j++) { const int i = lane + 32 * (j0 + j); x[j] = i < in_dim ? Xs[b * ldx + i] : 0.f; }
+#pragma unroll
+      for (int q = 0; q < 4; q++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) a[q][j] = fmaf(d[q], x[j], a[q][j]);
+    }
+#pragma unroll
+    for (int q = 0; q < 4; q++)
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const int i = lane + 32 * (j0 + j);
+        if (r0 + q < R && i < in_dim) As[(r0 + q) * lda + i] = a[q][j];
+      }
+  }
+}
+
+#define AMP_DISPATCH_J(Jv, CALL)                                  \
+  switch (Jv) {                                                   \
+    case 4: { constexpr int J = 4; CALL; } break;                 \
+    case 7: { constexpr int J = 7; CALL; } break;                 \
+    case 10: { constexpr int J = 10; CALL; } break;               \
+    case 16: { constexpr int J = 16; CALL; } break;               \
+    case 25: { constexpr int J = 25; CALL; } break;               \
+    default: { constexpr int J = 32; CALL; } break;               \
+  }
+
+// ------------------------------------------------------------------------------------------------
+// PPT tile: batch bookkeeping in shared memory
+// ------------------------------------------------------------------------------------------------
+struct LeaderState { unsigned head[2], sched_w, batch_w; int n_acc, version; };
+
+struct TileShared {
+  BatchDesc desc;
+  Hdr hdr[MAX_BATCH_MSGS];
+  long long key[MAX_BATCH_MSGS];
+  int rowoff[MAX_BATCH_MSGS + 1];
+  int rowmsg[64];
+  LeaderState ls;
+  int ok;
+  unsigned tail_snapshot;
+  unsigned long long stale_hist[64];
+  int max_stale;
+  Frame stack[WARPS][WALK_STACK];
+};
+
+__device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) {
+  return P.muf_override > 0 ? P.muf_override : C.muf;
+}
+
+// Warp 0 of the leader tile: take up to 32 candidate messages (ring slot per lane, in processing order), cut
+// the batch at the row capacity and at the message that triggers an update (Sec. 3), publish it.
+// Returns the number of messages taken.
+__device__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, unsigned slot, int ncand) {
+  const int lane = threadIdx.x & 31;
+  Ring& R = P.ring[dir];
+  Hdr h = {0, 0, 0, 0, 0, 0, 0, 0};
+  if (lane < ncand) {
+    const int4* e = reinterpret_cast<const int4*>(&R.e[slot]);
+    int4 a = __ldcg(e), b = __ldcg(e + 1);
+    h.inst = a.x; h.seq = a.y; h.slot = a.z; h.it = a.w; h.u = b.x; h.port = b.y; h.rows = b.z; h.flags = b.w;
+  }
+  const int rows = lane < ncand ? (h.rows > 0 ? h.rows : 1) : 0;
+  int cum = rows;
+  for (int o = 1; o < 32; o <<= 1) { int v = __shfl_up_sync(0xffffffffu, cum, o); if (lane >= o) cum += v; }
+  const bool ok = lane < ncand && cum <= P.BM;
+  unsigned okm = __ballot_sync(0xffffffffu, ok);
+  int take = __ffs(~okm) - 1;
+  if (take < 0) take = 32;
+  if (take == 0) { fail(C, ST_OVERFLOW, P.node, rows); return 0; }     // a single message larger than a batch
+  bool upd = false;
+  const bool eval = (h.flags & HDR_EVAL) != 0;
+  const int eval0 = __shfl_sync(0xffffffffu, (int)eval, 0);
+  if (dir == BWD && !eval0) {
+    const int muf = node_muf(C, P);
+    unsigned tm = __ballot_sync(0xffffffffu, ok && lane < take && (S.ls.n_acc + cum >= muf));
+    if (tm) { take = __ffs(tm); upd = true; }
+  }
+  const int total = __shfl_sync(0xffffffffu, cum, take - 1);
+  if (lane < take) {
+    P.sched[(S.ls.sched_w + lane) & P.sched_mask] = slot;
+    if (!eval0) {
+      long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      if (key >= 0) {
+        if (dir == FWD) P.vcache[key] = S.ls.version;
+        else {
+          int s = S.ls.version - P.vcache[key];
+          if (s < 0) s = 0;
+          atomicAdd(&S.stale_hist[s > 63 ? 63 : s], 1ull);
+          atomicMax(&S.max_stale, s);
+        }
+      }
+    }
+  }
+  __syncwarp();
+  if (lane == 0) {
+    BatchDesc d;
+    d.sched_start = S.ls.sched_w; d.count = take; d.dir = dir; d.flags = upd ? BATCH_UPDATE : 0;
+    d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.pad0 = d.pad1 = 0;
+    P.batches[S.ls.batch_w & P.batch_mask] = d;
+    __threadfence();
+    st_rel(P.batch_pub, S.ls.batch_w + 1u);
+    S.ls.batch_w++;
+    S.ls.sched_w += take;
+    PPTStats& st = *P.stats;
+    st.msgs += take; st.batches++; st.batch_rows += total;
+    if (upd) {
+      if (st.log_n < P.update_log_cap) P.update_log[st.log_n] = d.n_upd;
+      st.log_n++; st.n_updates++; st.n_grads_applied += d.n_upd;
+      S.ls.n_acc = 0; S.ls.version++;
+    } else if (dir == BWD && !eval0) S.ls.n_acc += total;
+  }
+  __syncwarp();
+  return take;
+}
+
+__device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags) {   // one thread
+  BatchDesc d;
+  d.sched_start = S.ls.sched_w; d.count = 0; d.dir = BWD; d.flags = flags; d.n_upd = 0; d.nrows = 0; d.pad0 = d.pad1 = 0;
+  if ((flags & BATCH_TERMINATE) && S.ls.n_acc > 0 && !C.eval) {      // epoch-end flush of the leftover gradients
+    d.flags |= BATCH_UPDATE; d.n_upd = S.ls.n_acc;
+    PPTStats& st = *P.stats;
+    if (st.log_n < P.update_log_cap) P.update_log[st.log_n] = d.n_upd;
+    st.log_n++; st.n_updates++; st.n_grads_applied += d.n_upd;
+    S.ls.n_acc = 0; S.ls.version++;
+  }
+  P.batches[S.ls.batch_w & P.batch_mask] = d;
+  __threadfence();
+  st_rel(P.batch_pub, S.ls.batch_w + 1u);
+  S.ls.batch_w++;
+}
+
+// Asynchronous mode, warp 0 of the leader: whatever is pending, backward first (App. A).
+__device__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
+  const int lane = threadIdx.x & 31;
+  for (int dir = BWD; dir >= FWD; dir--) {
+    Ring& R = P.ring[dir];
+    const unsigned t = S.ls.head[dir] + lane;
+    const unsigned slot = t & R.mask;
+    const bool ready = ld_acq(&R.seq[slot]) == t + 1u;
+    const unsigned m = __ballot_sync(0xffffffffu, ready);
+    int n = __ffs(~m) - 1;
+    if (n < 0) n = 32;
+    if (n == 0) continue;
+    int take = form_batch(C, P, S, dir, slot, n);
+    if (lane == 0) S.ls.head[dir] += take;
+    __syncwarp();
+    return true;
+  }
+  if (ld_acq(&C.g->done)) {
+    if (lane == 0) publish_marker(C, P, S, BATCH_TERMINATE);
+    __syncwarp();
+    return true;
+  }
+  return false;
+}
+
+// Deterministic mode, whole leader CTA: this round's inbox = tickets [head, tail) of each ring, sorted by
+// (admission seq, it, u, port), backward ring first; cut into batches; then the end-of-round marker.
+__device__ void leader_schedule_round(const Ctx& C, DevPPT& P, TileShared& S, unsigned long long t0) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (ld_acq(&C.g->done)) {
+    if (tid == 0) publish_marker(C, P, S, BATCH_TERMINATE);
+    __syncthreads();
+    return;
+  }
+  for (int dir = BWD; dir >= FWD; dir--) {
+    Ring& R = P.ring[dir];
+    if (tid == 0) S.tail_snapshot = ld_acq(R.tail);
+    __syncthreads();
+    const unsigned head = S.ls.head[dir];
+    const unsigned n = S.tail_snapshot - head;
+    if (n == 0) { __syncthreads(); continue; }
+    if (n > R.mask + 1u) { if (tid == 0) fail(C, ST_OVERFLOW, P.node, (int)n); __syncthreads(); return; }
+    unsigned np2 = 1;
+    while (np2 < n) np2 <<= 1;
+    for (unsigned i = tid; i < np2; i += THREADS) {
+      unsigned long long k = ~0ull;
+      if (i < n) {
+        const unsigned slot = (head + i) & R.mask;
+        spin_until(C, t0, [&] { return ld_acq(&R.seq[slot]) == head + i + 1u; });
+        const int4* e = reinterpret_cast<const int4*>(&R.e[slot]);
+        int4 a = __ldcg(e), b = __ldcg(e + 1);
+        k = ((unsigned long long)(a.y & 0xffffff) << 40) | ((unsigned long long)(a.w & 0xf) << 36) |
+            ((unsigned long long)(b.x & 0x3fff) << 22) | ((unsigned long long)(b.y & 0x3) << 20) | (unsigned long long)i;
+      }
+      P.sortbuf[i] = k;
+    }
+    __syncthreads();
+    for (unsigned k2 = 2; k2 <= np2; k2 <<= 1)
+      for (unsigned j = k2 >> 1; j > 0; j >>= 1) {
+        for (unsigned i = tid; i < np2; i += THREADS) {
+          unsigned ixj = i ^ j;
+          if (ixj > i) {
+            unsigned long long a = P.sortbuf[i], b = P.sortbuf[ixj];
+            bool asc = (i & k2) == 0;
+            if ((a > b) == asc) { P.sortbuf[i] = b; P.sortbuf[ixj] = a; }
+          }
+        }
+        __syncthreads();
+      }
+    if (warp == 0) {
+      unsigned pos = 0;
+      while (pos < n) {
+        int nc = (int)min(32u, n - pos);
+        unsigned slot = 0;
+        if (lane < nc) slot = (head + (unsigned)(P.sortbuf[pos + lane] & 0xfffffull)) & R.mask;
+        int take = form_batch(C, P, S, dir, slot, nc);
+        if (take <= 0) break;
+        pos += take;
+      }
+      if (lane == 0) S.ls.head[dir] = head + n;
+    }
+    __syncthreads();
+  }
+  if (tid == 0) publish_marker(C, P, S, BATCH_END_ROUND);
+  __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------------
+// PPT tile main loop
+// ------------------------------------------------------------------------------------------------
+struct TileMem {           // carve-up of the dynamic shared memory of a tile (floats)
+  float *Ws, *As, *bs, *Abs, *Xs, *Ds, *Ys;
+};
+
+__device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, const Hdr& h, long long key) {
+  if (P.xcache) return P.xcache + key * (long long)P.rows_max * P.in_dim;
+  return C.inst.dense + (long long)h.inst * C.inst.dense_dim;         // fed directly by a dense-row source
+}
+
+__device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileShared& S,
+                         const unsigned long long t0) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const DevNode& N = C.nodes[P.node];
+  const int in = P.in_dim, out = P.out_dim;
+  const int r_begin = tile * P.R;
+  const int R = P.kind == LOOKUP ? 0 : max(0, min(P.R, out - r_begin));
+  const int nmat = P.kind == GRUCELL ? 3 : 1;
+  TileMem M;
+  {
+    float* p = smem;
+    M.Ws = p; p += (size_t)nmat * P.R * in;
+    M.As = p; p += (size_t)nmat * P.R * in;
+    M.bs = p; p += nmat * P.R;
+    M.Abs = p; p += nmat * P.R;
+    M.Xs = p; p += (size_t)P.BM * in;
+    M.Ds = p; p += (size_t)nmat * P.BM * P.R;
+    M.Ys = p; p += (size_t)nmat * P.BM * P.R;
+  }
+  if (P.kind != LOOKUP) {
+    for (int m = 0; m < nmat; m++) {
+      for (int i = tid; i < R * in; i += THREADS) {
+        M.Ws[m * P.R * in + i] = P.W[(size_t)m * out * in + (size_t)r_begin * in + i];
+        M.As[m * P.R * in + i] = 0.f;
+      }
+      for (int i = tid; i < R; i += THREADS) { M.bs[m * P.R + i] = P.b[m * out + r_begin + i]; M.Abs[m * P.R + i] = 0.f; }
+    }
+  }
+  if (tid == 0) { S.ls.head[0] = S.ls.head[1] = 0; S.ls.sched_w = S.ls.batch_w = 0; S.ls.n_acc = 0; S.ls.version = 0; S.max_stale = 0; }
+  if (tid < 64) S.stale_hist[tid] = 0;
+  __syncthreads();
+
+  unsigned my_batch = 0, grid_gen = 0, node_gen = 0;
+  WalkAcc acc = {0, 0};
+  bool running = true;
+  while (running) {
+    if (C.det) {
+      if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;     // barrier A
+      if (tile == 0) leader_schedule_round(C, P, S, t0);
+    }
+    bool round_open = true;
+    while (round_open) {
+      // ---- obtain the next batch ------------------------------------------------------------
+      if (tid == 0) S.ok = 1;
+      __syncthreads();
+      if (tile == 0) {
+        if (warp == 0) {
+          unsigned it = 0;
+          while (S.ls.batch_w == my_batch) {
+            if (C.det) { if (lane == 0) { fail(C, ST_OVERFLOW, P.node, -7); S.ok = 0; } break; }
+            if (leader_try_schedule(C, P, S)) break;
+            if ((++it & 15u) == 0) {
+              if (aborted(C)) { if (lane == 0) S.ok = 0; break; }
+              if (gtime() - t0 > C.timeout_ns) { if (lane == 0) { fail(C, ST_TIMEOUT, P.node, 1); S.ok = 0; } break; }
+            }
+            __nanosleep(it < 16 ? 20 : 200);
+          }
+          __syncwarp();
+        }
+      } else if (tid == 0) {
+        if (!spin_until(C, t0, [&] { return ld_acq(P.batch_pub) > my_batch; })) S.ok = 0;
+      }
+      __syncthreads();
+      if (!S.ok || aborted(C)) { running = false; break; }
+      if (tid == 0) S.desc = P.batches[my_batch & P.batch_mask];
+      __syncthreads();
+      const BatchDesc d = S.desc;
+      my_batch++;
+      const int count = d.count, dir = d.dir;
+      // ---- headers, keys, row offsets ----------------------------------------------------------
+      if (tid < count) {
+        const unsigned slot = P.sched[(d.sched_start + tid) & P.sched_mask];
+        const int4* e = reinterpret_cast<const int4*>(&P.ring[dir].e[slot]);
+        int4 a = __ldcg(e), b = __ldcg(e + 1);
+        Hdr h; h.inst = a.x; h.seq = a.y; h.slot = a.z; h.it = a.w; h.u = b.x; h.port = b.y; h.rows = b.z; h.flags = b.w;
+        if (h.rows <= 0) h.rows = 1;
+        S.hdr[tid] = h;
+        S.key[tid] = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      }
+      __syncthreads();
+      if (tid == 0) {
+        int o = 0;
+        for (int i = 0; i < count; i++) {
+          S.rowoff[i] = o;
+          for (int r = 0; r < S.hdr[i].rows && o + r < 64; r++) S.rowmsg[o + r] = i;
+          o += S.hdr[i].rows;
+        }
+        S.rowoff[count] = o;
+        for (int i = 0; i < count; i++) if (S.key[i] < 0) S.ok = 0;
+        if (o > P.BM) { fail(C, ST_OVERFLOW, P.node, o); S.ok = 0; }
+      }
+      __syncthreads();
+      if (!S.ok) { running = false; break; }
+      const int nb = S.rowoff[count];
+      const bool eval = count > 0 && (S.hdr[0].flags & HDR_EVAL);
+
+      if (count > 0 && P.kind == LINEAR) {
+        // stage the cached inputs of the batch
+        for (int idx = tid; idx < nb * in; idx += THREADS) {
+          const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
+          M.Xs[idx] = __ldcg(msg_x(C, P, S.hdr[m], S.key[m]) + (size_t)(b - S.rowoff[m]) * in + c);
+        }
+        if (dir == FWD) {
+          __syncthreads();
+          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.Xs, in, nb, M.Ws, in, R, in, M.Ys, P.R)));
+          __syncthreads();
+          for (int idx = tid; idx < nb * R; idx += THREADS) {
+            const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
+            const float y = act_fwd(P.act, M.Ys[b * P.R + r] + M.bs[r]);
+            P.ycache[(S.key[m] * P.rows_max + (b - S.rowoff[m])) * out + r_begin + r] = y;
+          }
+        } else {
+          for (int idx = tid; idx < nb * R; idx += THREADS) {
+            const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
+            const size_t o = (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * out + r_begin + r;
+            M.Ds[b * P.R + r] = __ldcg(P.gbuf + o) * act_grad(P.act, __ldcg(P.ycache + o));
+          }
+          __syncthreads();
+          if (!(P.flags & 1)) {
+            float* dst = P.T > 1 ? P.dxpart + ((size_t)(my_batch & 1) * P.T + tile) * P.BM * in : P.stage;
+            AMP_DISPATCH_J(P.J, (tile_dW<J>(M.Ds, P.R, nb, M.Ws, in, R, in, dst)));
+          }
+          tile_accum(M.Ds, P.R, nb, M.Xs, in, M.As, in, R, in);
+          for (int r = tid; r < R; r += THREADS) {
+            float s = M.Abs[r];
+            for (int b = 0; b < nb; b++) s += M.Ds[b * P.R + r];
+            M.Abs[r] = s;
+          }
+        }
+      } else if (count > 0 && P.kind == LOOKUP) {
+        const DevInst& I = C.inst;
+        if (dir == FWD) {
+          for (int idx = tid; idx < nb * out; idx += THREADS) {
+            const int b = idx / out, c = idx - b * out, m = S.rowmsg[b];
+            const Hdr& h = S.hdr[m];
+            const int pos = I.kind == 3 ? (b - S.rowoff[m]) : h.u;
+            const int id = I.tokens[I.offsets[h.inst] + pos];
+            P.stage[idx] = ((unsigned)id < (unsigned)in) ? P.W[(size_t)id * out + c] : 0.f;
+          }
+        } else {
+          for (int c = tid; c < out; c += THREADS)
+            for (int b = 0; b < nb; b++) {
+              const int m = S.rowmsg[b];
+              const Hdr& h = S.hdr[m];
+              const int pos = I.kind == 3 ? (b - S.rowoff[m]) : h.u;
+              const int id = I.tokens[I.offsets[h.inst] + pos];
+              if ((unsigned)id >= (unsigned)in) continue;
+              const float g = __ldcg(P.gbuf + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * out + c);
+              P.A[(size_t)id * out + c] += g;
+              if (c == 0 && !P.touched_flag[id]) { P.touched_flag[id] = 1; P.touched_list[(*P.touched_n)++] = id; }
+            }
+        }
+      }
+      __syncthreads();
+      // ---- local update (Sec. 3): theta -= lr * A / n, accumulator cleared --------------------------
+      if (d.flags & BATCH_UPDATE) {
+        const float scale = C.lr / (float)d.n_upd;
+        if (P.kind == LOOKUP) {
+          __threadfence_block();
+          const int nt = *P.touched_n;
+          for (int idx = tid; idx < nt * out; idx += THREADS) {
+            const int id = P.touched_list[idx / out], c = idx % out;
+            const size_t o = (size_t)id * out + c;
+            P.W[o] = fmaf(-scale, P.A[o], P.W[o]);
+            P.A[o] = 0.f;
+          }
+          __syncthreads();
+          for (int k = tid; k < nt; k += THREADS) P.touched_flag[P.touched_list[k]] = 0;
+          __syncthreads();
+          if (tid == 0) *P.touched_n = 0;
+        } else {
+          for (int m = 0; m < nmat; m++) {
+            for (int i = tid; i < R * in; i += THREADS) {
+              const int o = m * P.R * in + i;
+              M.Ws[o] = fmaf(-scale, M.As[o], M.Ws[o]);
+              M.As[o] = 0.f;
+            }
+            for (int i = tid; i < R; i += THREADS) {
+              const int o = m * P.R + i;
+              M.bs[o] = fmaf(-scale, M.Abs[o], M.bs[o]);
+              M.Abs[o] = 0.f;
+            }
+          }
+        }
+        __syncthreads();
+      }
+      // ---- all tiles of the node done with the batch, then emit ------------------------------------
+      if (count > 0) {
+        __threadfence();
+        if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
+        else __syncthreads();
+        int mine = 0;
+        for (int i = 0; i < count; i++) {
+          if (i % P.T != tile) continue;
+          if ((mine++ % WARPS) != warp) continue;
+          const Hdr& h = S.hdr[i];
+          Frame f;
+          f.iter = 0; f.inst = h.inst; f.seq = h.seq; f.slot = h.slot; f.it = h.it; f.u = h.u; f.port = h.port;
+          f.rows = h.rows; f.flags = h.flags;
+          if (dir == FWD) {
+            f.node = N.succ_node[0]; f.aport = N.succ_port[0]; f.dir = FWD; f.dim = out; f.ld = out;
+            f.p = P.kind == LOOKUP ? P.stage + (size_t)S.rowoff[i] * out
+                                   : P.ycache + (size_t)S.key[i] * P.rows_max * out;
+          } else {
+            f.node = N.pred_node[0]; f.aport = N.pred_port[0]; f.dir = BWD; f.dim = in; f.ld = in;
+            if (P.kind == LOOKUP || (P.flags & 1)) { f.p = nullptr; f.dim = 0; f.rows = 1; }
+            else {
+              float* dx = P.stage + (size_t)S.rowoff[i] * in;
+              if (P.T > 1) {                                  // reduce the tiles' partial input gradients, tile order
+                const float* part = P.dxpart + (size_t)(my_batch & 1) * P.T * P.BM * in + (size_t)S.rowoff[i] * in;
+                for (int k = lane; k < h.rows * in; k += 32) {
+                  float s = 0.f;
+                  for (int t = 0; t < P.T; t++) s += __ldcg(part + (size_t)t * P.BM * in + k);
+                  dx[k] = s;
+                }
+                __syncwarp();
+              }
+              f.p = dx;
+            }
+          }
+          walk(C, f, S.stack[warp], acc);
+        }
+        flush_acc(C, acc, lane);
+        __syncthreads();
+      }
+      if (d.flags & BATCH_TERMINATE) { running = false; round_open = false; }
+      if (d.flags & BATCH_END_ROUND) round_open = false;
+      (void)eval;
+    }
+    if (!running) break;
+    if (C.det) { if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break; }   // barrier B
+  }
+  // ---- epilogue: parameters back to device memory, statistics ---------------------------------------
+  __syncthreads();
+  if (P.kind != LOOKUP)
+    for (int m = 0; m < nmat; m++) {
+      for (int i = tid; i < R * in; i += THREADS) P.W[(size_t)m * out * in + (size_t)r_begin * in + i] = M.Ws[m * P.R * in + i];
+      for (int i = tid; i < R; i += THREADS) P.b[m * out + r_begin + i] = M.bs[m * P.R + i];
+    }
+  if (tile == 0) {
+    if (tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
+    if (tid == 0) P.stats->max_staleness = S.max_stale;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// controller CTA: admission under max_active_keys, source messages, retirement (Sec. 3, Sec. 4)
+// ------------------------------------------------------------------------------------------------
+struct CtrlShared {
+  int ok;
+  long long next, retired;
+  int active;
+  unsigned retire_head;
+  int admit_slot, admit_inst, admit_seq, n_src_msgs;
+  int src_count[4], src_base[5];
+  Frame stack[WARPS][WALK_STACK];
+};
+
+__device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long long t0) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const DevInst& I = C.inst;
+  if (tid == 0) { S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; }
+  __syncthreads();
+  unsigned grid_gen = 0;
+  WalkAcc acc = {0, 0};
+  long long round = 0;
+  unsigned idle = 0;
+  for (;; round++) {
+    // ---- retirements ------------------------------------------------------------------------------
+    if (warp == 0) {
+      for (;;) {
+        const unsigned h = S.retire_head;
+        const unsigned s = h & C.retire_mask;
+        if (ld_acq(&C.retire_seq[s]) != h + 1u) break;
+        const int slot = (int)__ldcg(&C.retire_e[s]);
+        __syncwarp();
+        int left = 0;
+        if (lane == 0) { S.retire_head = h + 1u; left = --C.outstanding[slot]; }
+        left = __shfl_sync(0xffffffffu, left, 0);
+        if (left == 0) {
+          // instance finished: sum its loss cells in key order, free the slot
+          const int inst = C.slot_inst[slot];
+          double tot = 0.0; int okc = 0, np = 0;
+          for (int li = 0; li < C.n_loss; li++) {
+            const DevNode& L = C.nodes[C.loss_nodes[li]];
+            const long long k0 = (long long)slot * C.IT * L.U_in, k1 = k0 + (long long)C.IT * L.U_in;
+            double dpart = 0.0;   // lane partial over a strided subset, then a fixed-order warp sum
+            for (long long k = k0 + lane; k < k1; k += 32) {
+              const int pk = __ldcg(&L.predok[k]);
+              if (pk >= 0) { dpart += (double)__ldcg(&L.lossval[k]); okc += pk; np += 1; }
+            }
+            for (int o = 16; o; o >>= 1) dpart += __shfl_xor_sync(0xffffffffu, dpart, o);
+            tot += dpart;
+          }
+          for (int o = 16; o; o >>= 1) { okc += __shfl_xor_sync(0xffffffffu, okc, o); np += __shfl_xor_sync(0xffffffffu, np, o); }
+          if (lane == 0) {
+            C.loss_out[inst] = (float)tot;
+            C.g->total_loss += tot; C.g->correct += okc; C.g->n_pred += np;
+            C.slot_inst[slot] = -1;
+            S.active--; S.retired++;
+            if (C.det && C.keylog) C.keylog[C.slot_log[slot]].release = round;
+          }
+          __syncwarp();
+        }
+      }
+    }
+    __syncthreads();
+    // ---- admission ----------------------------------------------------------------------------------
+    for (;;) {
+      if (tid == 0) {
+        S.admit_slot = -1;
+        if (S.active < C.mak && S.next < C.n_order) {
+          int slot = 0;
+          while (slot < C.mak && C.slot_inst[slot] >= 0) slot++;          // lowest free slot
+          const int inst = (int)(C.order ? C.order[S.next] : S.next);
+          S.admit_slot = slot; S.admit_inst = inst; S.admit_seq = (int)S.next;
+          C.slot_inst[slot] = inst;
+          S.active++;
+          if (S.active > C.g->max_active) C.g->max_active = S.active;
+          int total = 0;
+          for (int s = 0; s < C.n_sources; s++) {
+            const DevNode& sn = C.nodes[C.src_nodes[s]];
+            int cnt = 1;
+            if (sn.fn == 2) cnt = (int)(I.offsets[inst + 1] - I.offsets[inst]);
+            else if (sn.fn == 4) cnt = (int)(I.leaf_off[inst + 1] - I.leaf_off[inst]);
+            S.src_base[s] = total; S.src_count[s] = cnt; total += cnt;
+          }
+          S.src_base[C.n_sources] = total;
+          S.n_src_msgs = total;
+          if (C.eval) {      // forward only: the instance is finished when every Loss / Sink has been reached
+            int exp = 1;
+            if (I.kind == 2) exp = (int)(I.offsets[inst + 1] - I.offsets[inst]) + 1;
+            C.outstanding[slot] = exp;
+          } else C.outstanding[slot] = total;
+          if (C.det && C.keylog) {
+            const long long li = C.g->n_keylog++;
+            C.slot_log[slot] = (int)li;
+            KeyLog kl; kl.inst = inst; kl.slot = slot; kl.pad = 0; kl.admit = round; kl.release = -1;
+            C.keylog[li] = kl;
+          }
+          S.next++;
+        }
+      }
+      __syncthreads();
+      const int slot = S.admit_slot;
+      if (slot < 0) break;
+      // clear the slot's loss cells (predok = -1 marks "no loss evaluated at this key")
+      for (int li = 0; li < C.n_loss; li++) {
+        const DevNode& L = C.nodes[C.loss_nodes[li]];
+        const long long k0 = (long long)slot * C.IT * L.U_in, cnt = (long long)C.IT * L.U_in;
+        for (long long k = tid; k < cnt; k += THREADS) { L.lossval[k0 + k] = 0.f; L.predok[k0 + k] = -1; }
+      }
+      __threadfence();
+      __syncthreads();
+      // pump the source messages (Sec. 4: tokens / leaves / graph nodes, initial hidden state, dense row)
+      const int inst = S.admit_inst;
+      for (int mi = warp; mi < S.n_src_msgs; mi += WARPS) {
+        int s = 0;
+        while (mi >= S.src_base[s + 1]) s++;
+        const int k = mi - S.src_base[s];
+        const DevNode& sn = C.nodes[C.src_nodes[s]];
+        Frame f;
+        f.node = sn.succ_node[0]; f.aport = sn.succ_port[0]; f.dir = FWD; f.iter = 0;
+        f.inst = inst; f.seq = S.admit_seq; f.slot = slot; f.it = 0; f.u = 0; f.port = 0; f.rows = 1;
+        f.flags = C.eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr;
+        switch (sn.fn) {
+          case 1: f.p = I.dense + (long long)inst * I.dense_dim; f.dim = I.dense_dim; f.ld = I.dense_dim; break;
+          case 2: f.u = k; break;
+          case 3: f.dim = sn.out_dim; f.ld = sn.out_dim; break;
+          case 4: f.u = I.leaf_ids[I.leaf_off[inst] + k]; break;
+          case 5: f.rows = (int)(I.offsets[inst + 1] - I.offsets[inst]); break;
+        }
+        walk(C, f, S.stack[warp], acc);
+      }
+      flush_acc(C, acc, lane);
+      __syncthreads();
+    }
+    // ---- termination / pacing -------------------------------------------------------------------------
+    const bool finished = S.retired == C.n_order;
+    if (finished && tid == 0) { C.g->rounds = (unsigned long long)(round + 1); __threadfence(); st_rel(&C.g->done, 1u); }
+    if (C.det) {
+      if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;   // barrier A
+      if (finished) break;
+      if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;   // barrier B
+    } else {
+      if (finished) break;
+      if (tid == 0) {
+        S.ok = 1;
+        if ((++idle & 15u) == 0) {
+          if (aborted(C)) S.ok = 0;
+          else if (gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, -1, 2); S.ok = 0; }
+        }
+        // wait for the next retire notice instead of spinning through the whole loop
+        const unsigned h = S.retire_head;
+        unsigned spins = 0;
+        while (ld_acq(&C.retire_seq[h & C.retire_mask]) != h + 1u && spins < 64) { __nanosleep(50); spins++; }
+      }
+      __syncthreads();
+      if (!S.ok) break;
+    }
+  }
+}
+
+union SharedUnion { TileShared t; CtrlShared c; };
+
+__global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constant__ Ctx C) {
+  extern __shared__ __align__(16) float dyn_smem[];
+  __shared__ SharedUnion SU;
+  const unsigned long long t0 = gtime();
+  const Role role = C.roles[blockIdx.x];
+  if (role.ppt < 0) controller_main(C, SU.c, t0);
+  else ppt_main(C, C.ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
+}
+
+}  // namespace amp

@@ -1,0 +1,136 @@
+// Device-side data structures of the AMPNet engine (shared by the host library and the kernel).
+#pragma once
+#include <stdint.h>
+
+namespace amp {
+
+constexpr int MAX_PORTS = 8;
+constexpr int THREADS = 256;          // threads per CTA
+constexpr int WARPS = THREADS / 32;
+constexpr int MAX_BATCH_MSGS = 32;    // messages per micro-batch (one warp schedules them)
+constexpr int WALK_STACK = 12;        // continuation frames per walking warp
+
+enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, CONCAT, SPLIT,
+                BCAST, GROUP, UNGROUP, FLATMAP, SINK, N_NODE_TYPES };
+enum { FWD = 0, BWD = 1 };
+enum { HDR_EVAL = 1 };
+enum { BATCH_UPDATE = 1, BATCH_END_ROUND = 2, BATCH_TERMINATE = 4 };
+enum { ST_OK = 0, ST_TIMEOUT = 4, ST_OVERFLOW = 5 };
+
+// Message header: the state of Sec. 4 (instance id, position, iteration, ...) plus the payload row count.
+struct __align__(16) Hdr { int inst, seq, slot, it, u, port, rows, flags; };
+
+struct Ring {            // multi-producer ring of headers; payloads live in the keyed caches
+  Hdr* e;
+  unsigned* seq;         // per slot: ticket + 1 once published
+  unsigned* tail;        // next ticket
+  unsigned mask;
+};
+
+struct __align__(16) BatchDesc { unsigned sched_start; int count, dir, flags, n_upd, nrows, pad0, pad1; };
+
+struct PPTStats {
+  unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
+  unsigned long long stale_hist[64];
+  int max_staleness, log_n;
+};
+
+struct DevNode {
+  int type, in_dim, out_dim, act, fn, fn_arg, flags, ppt;
+  int n_succ, n_pred;
+  int succ_node[MAX_PORTS], succ_port[MAX_PORTS];
+  int pred_node[MAX_PORTS], pred_port[MAX_PORTS];
+  int U_in, U_out, rows_in, rows_out;   // bounds of the position u and of the payload rows, before / after
+  // keyed storage; its meaning depends on the node type
+  float* jbuf;            // join / result buffer, jstride floats per key
+  long long jstride;
+  int* jcnt;              // arrival counter per key
+  unsigned char* origin;  // PHI: recorded predecessor per key
+  int* rowcnt;            // NPT_SUMROWS: cached row count per key
+  float* lossval;         // LOSS: loss per key
+  int* predok;            // LOSS_CE: 1 if the arg-max equals the label
+  int jalias;             // CONCAT: jbuf is the input cache of the succeeding PPT node
+  int pad;
+};
+
+struct DevPPT {
+  int node, kind, in_dim, out_dim, act, flags, muf_override, pad0;
+  int T, cta0, R, BM;                 // row tiles, first CTA, rows per tile, batch row capacity
+  int U, rows_max, J, pad1;           // key space, max rows per message, ceil(in_dim / 32) bucket
+  float *W, *b;                       // LINEAR: W[out][in], b[out]; LOOKUP: W = E[V][d]; GRUCELL: W[3][H][2H], b[3][H]
+  float* A;                           // LOOKUP: accumulator [V][d] in device memory
+  int *touched_flag, *touched_list, *touched_n;
+  float *xcache, *ycache, *gbuf;      // [key][rows_max][in | out | out]
+  float *zc, *rc, *cc;                // GRUCELL caches [key][rows_max][H]
+  int* vcache;                        // version at forward time, per key
+  Ring ring[2];
+  unsigned* sched; unsigned sched_mask;
+  BatchDesc* batches; unsigned batch_mask; unsigned* batch_pub;
+  unsigned long long* sortbuf;
+  float* dxpart;                      // [2][T][BM][in_dim] partial input gradients of the row tiles
+  float* stage;                       // [BM][max(in_dim, out_dim)] reduced input gradients / gathered rows
+  float* part2;                       // GRUCELL scratch
+  unsigned* nbar;                     // barrier counter of the node's tiles
+  PPTStats* stats;
+  int* update_log; int update_log_cap;
+  int smem_floats;
+};
+
+struct DevInst {                      // instances + routing tables produced by the structure encoder
+  int kind, dense_dim, NT, labels_per_node;
+  long long n;
+  const long long* offsets;
+  const int* tokens;
+  const int *left, *right, *parent, *child_slot;
+  const int* root;                    // per instance
+  const long long* leaf_off; const int* leaf_ids;
+  const long long* edge_off;
+  const int *esrc, *edst, *etype, *rank_out, *rank_in, *rank_type;
+  const long long *out_off, *in_off, *type_off;   // per global node (+1) / per (instance, type) (+1)
+  const int *out_list, *in_list, *type_list;      // local edge ids
+  const float* dense;
+  const int* labels_i;
+  const float* labels_f;
+};
+
+struct KeyLog { long long inst; int slot; int pad; long long admit, release; };
+
+struct Globals {                      // mutable run state in device memory (zeroed before every run)
+  unsigned grid_bar;
+  unsigned abort_flag;
+  int status;
+  unsigned done;
+  unsigned long long node_messages, route_hash;
+  unsigned long long rounds;
+  long long max_active;
+  unsigned long long correct, n_pred;
+  double total_loss;
+  long long n_keylog;
+  unsigned retire_tail;
+  int err_node, err_detail;
+};
+
+struct Role { int ppt, tile; };
+
+struct Ctx {
+  DevNode* nodes; int n_nodes;
+  DevPPT* ppts; int n_ppts;
+  Role* roles; int n_ctas;
+  DevInst inst;
+  Globals* g;
+  unsigned long long* node_msgs;       // [n_nodes][2]
+  // controller
+  int n_sources; int src_nodes[4];
+  int n_loss; int loss_nodes[4];
+  int* slot_inst; int* outstanding; int* slot_log;
+  KeyLog* keylog;
+  unsigned* retire_e; unsigned* retire_seq; unsigned retire_mask;
+  const long long* order; long long n_order;
+  float* loss_out;
+  // configuration
+  int mak, muf, det, eval, IT;
+  float lr;
+  unsigned long long timeout_ns;
+};
+
+}  // namespace amp
