@@ -1,0 +1,317 @@
+#!/usr/bin/env python
+"""Benchmark of the AMPNet training hot path on B200.
+
+A step is one epoch of asynchronous model-parallel training (admission, message-driven forward and backward
+execution, local updates, retirement) over one seeded synthetic workload.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload tree|ggnn|rnn|mlp] [--impl ours|reference]
+
+`--impl reference` times the CPU oracle (test infrastructure) on a bounded sample of the same workload.
+With N > 1 (torchrun) every rank trains an independent replica on its own shard; there is no collective on
+the data path.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import ir, data, params as wp  # noqa: E402
+
+WORKLOADS = {
+    # name: (graph builder, instance generator, full size, mak, muf, lr)
+    "mlp": (ir.mlp, data.mlp_instances, 2048, 4, 32, 0.01),
+    "rnn": (ir.rnn, data.list_instances, 20000, 16, 50, 0.05),
+    "tree": (ir.tree, data.tree_instances, 8544, 64, 100, 0.05),
+    "ggnn": (ir.ggnn, data.graph_instances, 130000, 128, 200, 0.01),
+}
+GGNN_BENCH_INSTANCES = 20000      # the graph workload is timed on a prefix of this many graphs per step
+
+
+def make_workload(name, rank=0, n=None):
+    build_graph, gen, full, mak, muf, lr = WORKLOADS[name]
+    if n is None:
+        n = GGNN_BENCH_INSTANCES if name == "ggnn" else full
+    inst = gen(n=n, split=0 if rank == 0 else 100 + rank)
+    return build_graph(), inst, dict(mak=mak, muf=muf, lr=lr, full=full)
+
+
+# ---------------------------------------------------------------------------------------------------
+# process-group plumbing (kept in functions so that the N > 1 path is testable with gloo on CPU)
+# ---------------------------------------------------------------------------------------------------
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("WORLD_SIZE", 1)), int(os.environ.get("LOCAL_RANK", 0))
+
+
+def dist_init(backend):
+    import torch.distributed as dist
+    rank, world, _ = dist_env()
+    if world > 1 and not dist.is_initialized():
+        dist.init_process_group(backend=backend, rank=rank, world_size=world)
+    return rank, world
+
+
+def all_max(x, device="cpu"):
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def all_sum(x, device="cpu"):
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()):
+        return float(x)
+    t = torch.tensor([float(x)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def barrier():
+    import torch.distributed as dist
+    if dist.is_available() and dist.is_initialized():
+        dist.barrier()
+
+
+def aggregate(units_this_rank, seconds_this_rank, device="cpu"):
+    """Whole-job throughput: units of all ranks / the slowest rank's time."""
+    total = all_sum(units_this_rank, device)
+    t = all_max(seconds_this_rank, device)
+    return total / t if t > 0 else 0.0, t
+
+
+# ---------------------------------------------------------------------------------------------------
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.stop_flag = index, [], threading.Event()
+
+    def run(self):
+        while not self.stop_flag.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i",
+                                      str(self.index)], capture_output=True, text=True, timeout=5).stdout.strip()
+                if out:
+                    self.samples.append([v.strip() for v in out.split(",")])
+            except Exception:
+                pass
+            self.stop_flag.wait(0.2)
+
+    def summary(self):
+        self.stop_flag.set()
+        self.join(timeout=6)
+        sm = [float(s[0]) for s in self.samples if s and s[0].replace(".", "").isdigit()]
+        mx = [float(s[1]) for s in self.samples if len(s) > 1 and s[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = sorted({names[i] for s in self.samples for i in range(4) if len(s) > 2 + i and s[2 + i] == "Active"})
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def measured_peaks():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return json.load(f), "measured"
+    except Exception:
+        return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
+
+
+def time_oracle(graph, inst, cfg, target_s=12.0, probe=48):
+    """The oracle as it stands, single-threaded, on a bounded prefix of the workload."""
+    import oracle as oracle_mod
+    o = oracle_mod.Oracle(graph)
+    p = wp.init_params(graph)
+    probe = min(probe, inst.n)
+    o.load_instances(inst.head(probe))
+    o.set_params(p)
+    st, _ = o.run_epoch(mak=cfg["mak"], muf=cfg["muf"], lr=cfg["lr"])
+    per = st.seconds / probe
+    n = int(max(probe, min(inst.n, target_s / max(per, 1e-9))))
+    sample = inst.head(n)
+    o.load_instances(sample)
+    o.set_params(p)
+    st, _ = o.run_epoch(mak=cfg["mak"], muf=cfg["muf"], lr=cfg["lr"])
+    return dict(instances=n, seconds=st.seconds, inst_per_s=n / st.seconds, msgs_per_s=st.node_messages / st.seconds)
+
+
+def run_reference(args):
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    graph, inst, cfg = make_workload(args.workload, n=args.instances)
+    times, units, msgs = [], 0, 0
+    res = None
+    for k in range(args.warmup + args.steps):
+        res = time_oracle(graph, inst, cfg, target_s=8.0 if args.steps > 1 else 12.0)
+        if k >= args.warmup:
+            times.append(res["seconds"]); units += res["instances"]; msgs += res["msgs_per_s"] * res["seconds"]
+    tot = sum(times)
+    value = units / tot
+    sample = f"first {res['instances']} of {inst.n} instances per step, one epoch each"
+    line = {"impl": "reference", "metric": "training_instances_per_s", "value": value, "unit": "instances/s",
+            "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "node_messages_per_s": msgs / tot,
+            "config": workload_config(args.workload, inst, cfg, "canonical round schedule on the host"),
+            "cpu_baseline": {"value": value, "unit": "instances/s", "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": "instances/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(name, inst, cfg, mode):
+    return {"workload": name, "instances_per_step": int(inst.n), "full_dataset_instances": cfg["full"],
+            "max_active_keys": cfg["mak"], "min_update_frequency": cfg["muf"], "lr": cfg["lr"], "mode": mode,
+            "l2": "flushed between steps (256 MiB write)", "parallelism": "replicas, no collective"}
+
+
+def input_bytes(inst):
+    return int(sum(a.nbytes for a in (inst.offsets, inst.tokens, inst.left, inst.right, inst.edge_offsets, inst.edge_src,
+                                      inst.edge_dst, inst.edge_type, inst.dense, inst.labels_i, inst.labels_f)
+                   if a is not None))
+
+
+def run_ours(args):
+    import torch
+    import paper_1705_09786_b200 as amp
+    from paper_1705_09786_b200 import roofline as rf
+    rank, world, local = dist_env()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist_init("nccl")
+    graph, inst, cfg = make_workload(args.workload, rank, n=args.instances)
+    eng = amp.Engine(graph, device=local)
+    eng.load_instances(inst)
+    p0 = wp.init_params(graph)
+    eng.set_params(p0)
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    stream = torch.cuda.current_stream(dev)
+
+    def step():
+        flush_buf.fill_(1)                                     # evict L2 between steps (outside the timed events)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        st, _ = eng.run_epoch(mak=cfg["mak"], muf=cfg["muf"], lr=cfg["lr"], deterministic=False, timeout_s=args.timeout,
+                              want_loss=False)
+        e1.record(stream)
+        e1.synchronize()
+        return st, e0.elapsed_time(e1) * 1e-3
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler(local)
+    sampler.start()
+    torch.cuda.synchronize()
+    barrier()
+    step_s, kern_s, msgs, last = [], [], 0, None
+    for _ in range(args.steps):
+        st, s = step()
+        step_s.append(s); kern_s.append(st.seconds); msgs += st.node_messages; last = st
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.summary()
+    secs = sum(step_s)
+    value, tmax = aggregate(inst.n * args.steps, secs, dev)
+    msg_rate, _ = aggregate(msgs, secs, dev)
+
+    # ---- end to end: host buffers in, per-instance losses out, every step --------------------------------
+    pinned = {}
+    for k in ("offsets", "tokens", "left", "right", "edge_offsets", "edge_src", "edge_dst", "edge_type", "dense",
+              "labels_i", "labels_f"):
+        a = getattr(inst, k)
+        if a is not None:
+            pinned[k] = torch.from_numpy(a).pin_memory()
+            setattr(inst, k, pinned[k].numpy())
+    e2e_steps = max(1, min(args.steps, 3))
+    torch.cuda.synchronize()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        eng.load_instances(inst)
+        st, loss = eng.run_epoch(mak=cfg["mak"], muf=cfg["muf"], lr=cfg["lr"], deterministic=False, timeout_s=args.timeout)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    e2e_value, _ = aggregate(inst.n * e2e_steps, e2e_s, dev)
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        updates = {n: eng.node_stats(n)["n_updates"] for n in graph.ppt_nodes()}
+        flops = rf.algorithmic_flops(graph, inst, updates)
+        sm_mhz = float(peaks.get("sm_max_mhz", 1965.0))
+        peak_tf = rf.fma_peak_tflops(sm_mhz)
+        kavg = float(np.mean(kern_s))
+        achieved = flops / kavg / 1e12
+        roof_inst, F, B = rf.roofline_instances_per_s(graph, inst, sm_mhz, float(peaks.get("hbm_gbs", 6650.0)))
+        traffic = None
+        prof = os.path.join(ROOT, "profiles", f"traffic_{args.workload}.json")
+        note = "no ncu capture yet"
+        if os.path.exists(prof):
+            with open(prof) as f:
+                t = json.load(f)
+            traffic = t["dram_bytes_per_instance"] * inst.n
+            note = t.get("note", "")
+        roofline = {"bound": "alu", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
+                    "traffic": traffic, "traffic_note": note,
+                    "peak_kind": f"derived: 148 SMs x 128 FP32 lanes x 2 x {sm_mhz:.0f} MHz ({peak_kind} max SM clock)",
+                    "kernel": "ampnet_engine (one persistent launch per step)", "kernel_ms": kavg * 1e3,
+                    "algorithmic_flop_per_launch": flops, "flop_per_instance": F, "payload_bytes_per_instance": B,
+                    "resident_weight_roofline_instances_per_s": roof_inst,
+                    "frac_of_resident_weight_roofline": (inst.n / kavg) / roof_inst}
+        cpu = None
+        if not args.no_cpu_baseline:
+            r = time_oracle(graph, inst, cfg)
+            cpu = {"value": r["inst_per_s"], "unit": "instances/s", "cores": 1, "kind": "oracle",
+                   "sample": f"first {r['instances']} of {inst.n} instances, one epoch, {r['seconds']:.1f} s",
+                   "node_messages_per_s": r["msgs_per_s"]}
+        line = {"metric": "training_instances_per_s", "value": value, "unit": "instances/s", "n_gpus": world,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tmax / args.steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "node_messages_per_s": msg_rate,
+                "config": workload_config(args.workload, inst, cfg, "asynchronous (free-running persistent kernel)"),
+                "roofline": roofline, "cpu_baseline": cpu,
+                "e2e": {"value": e2e_value, "unit": "instances/s", "h2d_bytes_per_step": input_bytes(inst),
+                        "d2h_bytes_per_step": int(inst.n * 4 + 512), "steps": e2e_steps},
+                "clocks": clocks, "gpu_launches": args.steps,
+                "stats": {"mean_loss_last_step": last.mean_loss, "max_staleness": int(last.max_staleness),
+                          "rows_per_micro_batch": last.micro_batch_rows / max(1, last.micro_batches),
+                          "placement": {graph.names[n]: eng.placement(n) for n in graph.ppt_nodes()}}}
+        print(json.dumps(line), flush=True)
+    eng.close()
+    import torch.distributed as dist
+    if dist.is_initialized():
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="tree", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--instances", type=int, default=None, help="instances per step (default: the workload's size)")
+    ap.add_argument("--timeout", type=float, default=300.0, help="bound on one device run, seconds")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -346,7 +346,8 @@ unsigned pow2_at_least(unsigned long long v) {
 
 size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
   if (P.kind == LOOKUP) return 64;
-  return (size_t)P.nmat * (2 * (size_t)R * P.in + 2 * R) + (size_t)BM * P.in + 2 * (size_t)P.nmat * BM * R + 64;
+  return (size_t)P.nmat * (2 * (size_t)R * P.in + 2 * R) + (size_t)BM * P.in * (P.kind == GRUCELL ? 2 : 1) +
+         (size_t)(2 * P.nmat + 1) * BM * R + 64;
 }
 
 // Placement: row tiles per PPT node.  Enough tiles that a tile's weights + accumulators + staging fit in
@@ -435,7 +436,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
       P.zc = B.take<float>(keys * P.rows_max * P.out_dim);
       P.rc = B.take<float>(keys * P.rows_max * P.out_dim);
       P.cc = B.take<float>(keys * P.rows_max * P.out_dim);
-      P.part2 = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
+      P.part2 = B.take<float>((size_t)2 * (P.T + 1) * P.BM * P.in_dim);
     }
     P.vcache = B.take<int>(keys);
     const unsigned cap = pow2_at_least(2ull * keys);
@@ -450,7 +451,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.batches = B.take<BatchDesc>(2 * (size_t)cap); P.batch_mask = 2 * cap - 1;
     P.batch_pub = C.take<unsigned>(1);
     P.sortbuf = B.take<unsigned long long>(cap);
-    if (P.T > 1 && H.kind != LOOKUP) P.dxpart = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
+    if ((P.T > 1 && H.kind != LOOKUP) || H.kind == GRUCELL) P.dxpart = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
     P.stage = B.take<float>((size_t)P.BM * std::max(P.in_dim, P.out_dim));
     P.nbar = C.take<unsigned>(1);
     P.stats = C.take<PPTStats>(1);

@@ -509,7 +509,7 @@ __device__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const fl
 }
 
 // dx[b][i] = sum_r D[b][r] * W[r][i], written to dst (device memory, ld = in_dim).
-template <int J>
+template <int J, bool ACCUM = false>
 __device__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Ws, int ldw, int R,
                         int in_dim, float* __restrict__ dst) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -537,7 +537,10 @@ __device__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const flo
 #pragma unroll
         for (int j = 0; j < J; j++) {
           const int i = lane + 32 * j;
-          if (i < in_dim) dst[(size_t)(b0 + m) * in_dim + i] = acc[m][j];
+          if (i < in_dim) {
+            float* o = dst + (size_t)(b0 + m) * in_dim + i;
+            *o = ACCUM ? *o + acc[m][j] : acc[m][j];
+          }
         }
   }
 }
@@ -601,7 +604,7 @@ struct TileShared {
   int rowmsg[64];
   LeaderState ls;
   int ok;
-  unsigned tail_snapshot;
+  unsigned tail_snap[2];
   unsigned long long stale_hist[64];
   int max_stale;
   Frame stack[WARPS][WALK_STACK];
@@ -729,10 +732,8 @@ __device__ void leader_schedule_round(const Ctx& C, DevPPT& P, TileShared& S, un
   }
   for (int dir = BWD; dir >= FWD; dir--) {
     Ring& R = P.ring[dir];
-    if (tid == 0) S.tail_snapshot = ld_acq(R.tail);
-    __syncthreads();
     const unsigned head = S.ls.head[dir];
-    const unsigned n = S.tail_snapshot - head;
+    const unsigned n = S.tail_snap[dir] - head;
     if (n == 0) { __syncthreads(); continue; }
     if (n > R.mask + 1u) { if (tid == 0) fail(C, ST_OVERFLOW, P.node, (int)n); __syncthreads(); return; }
     unsigned np2 = 1;
@@ -784,7 +785,7 @@ __device__ void leader_schedule_round(const Ctx& C, DevPPT& P, TileShared& S, un
 // PPT tile main loop
 // ------------------------------------------------------------------------------------------------
 struct TileMem {           // carve-up of the dynamic shared memory of a tile (floats)
-  float *Ws, *As, *bs, *Abs, *Xs, *Ds, *Ys;
+  float *Ws, *As, *bs, *Abs, *Xs, *Ds, *Ys, *XC;
 };
 
 __device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, const Hdr& h, long long key) {
@@ -808,8 +809,9 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
     M.bs = p; p += nmat * P.R;
     M.Abs = p; p += nmat * P.R;
     M.Xs = p; p += (size_t)P.BM * in;
-    M.Ds = p; p += (size_t)nmat * P.BM * P.R;
+    M.Ds = p; p += (size_t)(nmat + 1) * P.BM * P.R;
     M.Ys = p; p += (size_t)nmat * P.BM * P.R;
+    M.XC = p;   // GRUCELL only: [BM][in]
   }
   if (P.kind != LOOKUP) {
     for (int m = 0; m < nmat; m++) {
@@ -830,6 +832,9 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
   while (running) {
     if (C.det) {
       if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;     // barrier A
+      // This round's inbox is what is queued now; nothing may be emitted before every leader has looked.
+      if (tile == 0 && tid == 0) { S.tail_snap[FWD] = ld_acq(P.ring[FWD].tail); S.tail_snap[BWD] = ld_acq(P.ring[BWD].tail); }
+      if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;     // barrier A2
       if (tile == 0) leader_schedule_round(C, P, S, t0);
     }
     bool round_open = true;
@@ -921,6 +926,98 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
             M.Abs[r] = s;
           }
         }
+      } else if (count > 0 && P.kind == GRUCELL) {
+        // x = [a; h]; the tile owns rows [r_begin, r_begin + R) of Wz, Wr, Wc (matrix m at Ws + m * P.R * in)
+        const int H = out, SR = P.R, BR = P.BM * P.R;
+        const float *Wz = M.Ws, *Wr = M.Ws + SR * in, *Wc = M.Ws + 2 * SR * in;
+        for (int idx = tid; idx < nb * in; idx += THREADS) {
+          const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
+          M.Xs[idx] = __ldcg(P.xcache + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * in + c);
+        }
+        __syncthreads();
+        if (dir == FWD) {
+          // phase 1: gates z, r for the tile's rows
+          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.Xs, in, nb, Wz, in, R, in, M.Ys, SR)));
+          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.Xs, in, nb, Wr, in, R, in, M.Ys + BR, SR)));
+          __syncthreads();
+          for (int idx = tid; idx < nb * R; idx += THREADS) {
+            const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
+            const size_t o = (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + r_begin + r;
+            const float z = act_fwd(3, M.Ys[b * SR + r] + M.bs[r]);
+            const float rg = act_fwd(3, M.Ys[BR + b * SR + r] + M.bs[SR + r]);
+            M.Ys[b * SR + r] = z;
+            P.zc[o] = z; P.rc[o] = rg;
+          }
+          __threadfence();
+          if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
+          else __syncthreads();
+          // phase 2: candidate c = tanh(Wc [a; r*h] + bc) and the new state
+          for (int idx = tid; idx < nb * in; idx += THREADS) {
+            const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
+            float v = M.Xs[idx];
+            if (c >= H) v *= __ldcg(P.rc + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + (c - H));
+            M.XC[idx] = v;
+          }
+          __syncthreads();
+          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.XC, in, nb, Wc, in, R, in, M.Ys + 2 * BR, SR)));
+          __syncthreads();
+          for (int idx = tid; idx < nb * R; idx += THREADS) {
+            const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
+            const size_t o = (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + r_begin + r;
+            const float cnd = tanhf(M.Ys[2 * BR + b * SR + r] + M.bs[2 * SR + r]);
+            const float z = M.Ys[b * SR + r];
+            P.cc[o] = cnd;
+            P.ycache[o] = (1.f - z) * M.Xs[b * in + H + r_begin + r] + z * cnd;
+          }
+        } else {
+          const size_t pstride = (size_t)P.BM * in;
+          float* part1 = P.part2 + ((size_t)(my_batch & 1) * (P.T + 1) + tile) * pstride;
+          const float* part1_all = P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride;
+          float* dirbuf = P.part2 + ((size_t)(my_batch & 1) * (P.T + 1) + P.T) * pstride;     // [BM][H]
+          float* part2 = P.dxpart + ((size_t)(my_batch & 1) * P.T + tile) * pstride;
+          float *dpz = M.Ds, *dpr = M.Ds + BR, *dpc = M.Ds + 2 * BR, *dirp = M.Ds + 3 * BR;
+          for (int idx = tid; idx < nb * R; idx += THREADS) {
+            const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
+            const size_t o = (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + r_begin + r;
+            const float g = __ldcg(P.gbuf + o), z = __ldcg(P.zc + o), rg = __ldcg(P.rc + o), cnd = __ldcg(P.cc + o);
+            const float h = M.Xs[b * in + H + r_begin + r];
+            dpc[b * SR + r] = g * z * (1.f - cnd * cnd);
+            dpz[b * SR + r] = g * (cnd - h) * z * (1.f - z);
+            dirp[b * SR + r] = g * (1.f - z);
+            M.Ys[b * SR + r] = rg;
+          }
+          for (int idx = tid; idx < nb * in; idx += THREADS) {
+            const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
+            float v = M.Xs[idx];
+            if (c >= H) v *= __ldcg(P.rc + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + (c - H));
+            M.XC[idx] = v;
+          }
+          __syncthreads();
+          AMP_DISPATCH_J(P.J, (tile_dW<J>(dpc, SR, nb, Wc, in, R, in, part1)));      // [da_c; dq] partial
+          __threadfence();
+          if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
+          else __syncthreads();
+          for (int idx = tid; idx < nb * R; idx += THREADS) {
+            const int b = idx / R, r = idx - b * R;
+            float dq = 0.f;
+            for (int t = 0; t < P.T; t++) dq += __ldcg(part1_all + (size_t)t * pstride + (size_t)b * in + H + r_begin + r);
+            const float rg = M.Ys[b * SR + r], h = M.Xs[b * in + H + r_begin + r];
+            dpr[b * SR + r] = dq * h * rg * (1.f - rg);
+            dirbuf[(size_t)b * H + r_begin + r] = dirp[b * SR + r] + dq * rg;
+          }
+          __syncthreads();
+          AMP_DISPATCH_J(P.J, (tile_dW<J>(dpz, SR, nb, Wz, in, R, in, part2)));
+          AMP_DISPATCH_J(P.J, (tile_dW<J, true>(dpr, SR, nb, Wr, in, R, in, part2)));
+          tile_accum(dpz, SR, nb, M.Xs, in, M.As, in, R, in);
+          tile_accum(dpr, SR, nb, M.Xs, in, M.As + SR * in, in, R, in);
+          tile_accum(dpc, SR, nb, M.XC, in, M.As + 2 * SR * in, in, R, in);
+          for (int k = tid; k < 3 * R; k += THREADS) {
+            const int m = k / R, r = k - m * R;
+            float sacc = M.Abs[m * SR + r];
+            for (int b = 0; b < nb; b++) sacc += M.Ds[m * BR + b * SR + r];
+            M.Abs[m * SR + r] = sacc;
+          }
+        }
       } else if (count > 0 && P.kind == LOOKUP) {
         const DevInst& I = C.inst;
         if (dir == FWD) {
@@ -1000,7 +1097,24 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
             if (P.kind == LOOKUP || (P.flags & 1)) { f.p = nullptr; f.dim = 0; f.rows = 1; }
             else {
               float* dx = P.stage + (size_t)S.rowoff[i] * in;
-              if (P.T > 1) {                                  // reduce the tiles' partial input gradients, tile order
+              if (P.kind == GRUCELL) {
+                const int H = out;
+                const size_t pstride = (size_t)P.BM * in, ro = (size_t)S.rowoff[i] * in;
+                const float* p1 = P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride + ro;
+                const float* p2 = P.dxpart + (size_t)(my_batch & 1) * P.T * pstride + ro;
+                const float* dirb = P.part2 + ((size_t)(my_batch & 1) * (P.T + 1) + P.T) * pstride + (size_t)S.rowoff[i] * H;
+                for (int k = lane; k < h.rows * in; k += 32) {
+                  const int rr = k / in, c = k - rr * in;
+                  float s = 0.f;
+                  for (int t = 0; t < P.T; t++) {
+                    s += __ldcg(p2 + (size_t)t * pstride + k);
+                    if (c < H) s += __ldcg(p1 + (size_t)t * pstride + k);
+                  }
+                  if (c >= H) s += __ldcg(dirb + (size_t)rr * H + (c - H));
+                  dx[k] = s;
+                }
+                __syncwarp();
+              } else if (P.T > 1) {                           // reduce the tiles' partial input gradients, tile order
                 const float* part = P.dxpart + (size_t)(my_batch & 1) * P.T * P.BM * in + (size_t)S.rowoff[i] * in;
                 for (int k = lane; k < h.rows * in; k += 32) {
                   float s = 0.f;
@@ -1174,6 +1288,7 @@ __device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long
     if (finished && tid == 0) { C.g->rounds = (unsigned long long)(round + 1); __threadfence(); st_rel(&C.g->done, 1u); }
     if (C.det) {
       if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;   // barrier A
+      if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;   // barrier A2
       if (finished) break;
       if (!cta_barrier(C, t0, &C.g->grid_bar, (unsigned)C.n_ctas, grid_gen, &S.ok)) break;   // barrier B
     } else {

@@ -1,0 +1,268 @@
+"""CUDA engine vs CPU oracle, element by element, through the C ABI (needs a B200).
+
+Bar: routing multiset, key log, update counts and gradient counts bit-exact in the deterministic schedule;
+parameters within max relative error 1e-4, per-instance losses within 1e-5 (relative, with an absolute
+floor of 2e-6 for losses near zero: fp32 log-sum-exp has ~1e-7 absolute error per term).
+"""
+import numpy as np
+import pytest
+
+from workloads import ir, data, params as wp
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+def _case(family, n):
+    if family == "mlp":
+        return ir.mlp((784, 256, 256, 10)), data.mlp_instances(n=n)
+    if family == "rnn":
+        return ir.rnn(), data.list_instances(n=n)
+    if family == "tree":
+        return ir.tree(), data.tree_instances(n=n)
+    return ir.ggnn(), data.graph_instances(n=n)
+
+
+# sizes span several row tiles, several micro-batches and ragged tails; the oracle finishes each in seconds
+CASES = [
+    ("mlp", 70, 1, 1, 0.01), ("mlp", 70, 4, 32, 0.01), ("mlp", 70, 4, 1, 0.01), ("mlp", 33, 7, 5, 0.01),
+    ("rnn", 90, 1, 1, 0.02), ("rnn", 90, 16, 50, 0.05), ("rnn", 61, 5, 3, 0.02),
+    ("tree", 24, 1, 1, 0.002), ("tree", 40, 64, 100, 0.05), ("tree", 31, 6, 7, 0.01),
+    ("ggnn", 12, 1, 1, 0.0005), ("ggnn", 40, 128, 200, 0.01), ("ggnn", 25, 9, 40, 0.005),
+]
+
+
+@pytest.mark.parametrize("family,n,mak,muf,lr", CASES)
+def test_deterministic_schedule_matches_oracle(oracle_mod, family, n, mak, muf, lr):
+    g, inst = _case(family, n)
+    p = wp.init_params(g)
+    r = parity.run_both(oracle_mod, g, inst, p, mak, muf, lr)
+    parity.assert_parity(g, *r)
+    r[3].close()
+
+
+def test_shuffled_epoch_order_and_second_epoch(oracle_mod):
+    g, inst = _case("tree", 30)
+    p = wp.init_params(g)
+    order = data.epoch_order(inst.n, 3)
+    o, ost, oloss, e, est, eloss = parity.run_both(oracle_mod, g, inst, p, 8, 20, 0.02, order=order)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    # a second epoch continues from the first one's parameters on both sides
+    ost, oloss = o.run_epoch(mak=8, muf=20, lr=0.02)
+    est, eloss = e.run_epoch(mak=8, muf=20, lr=0.02, deterministic=True, timeout_s=60)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    e.close()
+
+
+def test_partial_epoch_and_degenerate_sizes(oracle_mod):
+    """One instance; mak larger than the instance count; a prefix of the data; the smallest structures."""
+    g, inst = _case("rnn", 9)
+    p = wp.init_params(g)
+    r = parity.run_both(oracle_mod, g, inst, p, 32, 1000, 0.05, order=np.array([4]))
+    parity.assert_parity(g, *r)
+    r[3].close()
+    g = ir.tree()
+    inst = data.tree_instances(n=6, min_leaves=2, max_leaves=2)       # smallest tree: two leaves and a root
+    r = parity.run_both(oracle_mod, g, inst, wp.init_params(g), 64, 100, 0.05)
+    parity.assert_parity(g, *r)
+    r[3].close()
+    g = ir.rnn()
+    inst = data.list_instances(n=5, max_len=1)                         # shortest list: op token + one digit
+    r = parity.run_both(oracle_mod, g, inst, wp.init_params(g), 2, 3, 0.05)
+    parity.assert_parity(g, *r)
+    r[3].close()
+
+
+def test_maximum_structure_sizes(oracle_mod):
+    g = ir.tree()
+    inst = data.tree_instances(n=3, min_leaves=50, max_leaves=50)
+    r = parity.run_both(oracle_mod, g, inst, wp.init_params(g), 64, 100, 0.05)
+    parity.assert_parity(g, *r)
+    r[3].close()
+    g = ir.ggnn()
+    inst = data.graph_instances(n=4, min_nodes=29, max_nodes=29)
+    r = parity.run_both(oracle_mod, g, inst, wp.init_params(g), 128, 200, 0.01)
+    parity.assert_parity(g, *r)
+    r[3].close()
+
+
+def test_per_node_update_threshold(oracle_mod):
+    """muf_override on one node (the paper uses 1000 for the embedding node and 50 elsewhere)."""
+    g = ir.tree()
+    nodes = g._nodes
+    i = g.index("lookup")
+    nodes[i] = nodes[i][:6] + (37,) + nodes[i][7:]
+    inst = data.tree_instances(n=20)
+    r = parity.run_both(oracle_mod, g, inst, wp.init_params(g), 16, 5, 0.02)
+    parity.assert_parity(g, *r)
+    assert (r[3].update_log(i)[:-1] == 37).all()
+    r[3].close()
+
+
+@pytest.mark.parametrize("family,n", [("mlp", 64), ("rnn", 80), ("tree", 40), ("ggnn", 30)])
+def test_eval_matches_oracle(oracle_mod, family, n):
+    import paper_1705_09786_b200 as amp
+    g, inst = _case(family, n)
+    p = wp.init_params(g)
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst, split=1)
+    o.set_params(p)
+    oml, oacc, oloss = o.eval(split=1)
+    e = amp.Engine(g)
+    e.load_instances(inst, split=1)
+    e.set_params(p)
+    eml, eacc, eloss = e.eval(split=1, mak=16)
+    np.testing.assert_allclose(eloss, oloss, rtol=1e-5, atol=2e-6)
+    assert abs(eml - oml) <= 1e-5 * max(1.0, abs(oml))
+    assert eacc == pytest.approx(oacc, abs=1e-12)          # arg-max decisions agree exactly on these inputs
+    after = e.get_params()
+    for k, v in p.items():
+        np.testing.assert_array_equal(after[k], v.astype(np.float32))
+    assert e.leftover_cache_entries() == 0
+    e.close()
+
+
+@pytest.mark.parametrize("family,n,mak,muf,lr", [("mlp", 512, 4, 32, 0.01), ("rnn", 1500, 16, 50, 0.05),
+                                                ("tree", 400, 64, 100, 0.05), ("ggnn", 600, 128, 200, 0.003)])
+def test_async_mode_invariants(family, n, mak, muf, lr):
+    """The free-running schedule is timing dependent; what holds for every schedule is checked exactly."""
+    import paper_1705_09786_b200 as amp
+    g, inst = _case(family, n)
+    e = amp.Engine(g)
+    e.load_instances(inst)
+    e.set_params(wp.init_params(g))
+    losses = []
+    for _ in range(3):
+        st, loss = e.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=False, timeout_s=120)
+        losses.append(st.mean_loss)
+        assert st.instances == inst.n and 1 <= st.max_active_observed <= mak
+        assert e.leftover_cache_entries() == 0                       # every forward message was answered
+        assert np.isfinite(loss).all()
+        want = parity_counts(g, inst)
+        assert st.node_messages == want["node_messages"]
+        for node, G in want["grads"].items():                        # every gradient applied exactly once
+            ns = e.node_stats(node)
+            assert ns["n_grads_applied"] == G == e.update_log(node).sum()
+    assert losses[-1] < losses[0]
+
+
+def parity_counts(g, inst):
+    if g.name == "mlp":
+        return dict(node_messages=7 * inst.n, grads={n: inst.n for n in g.ppt_nodes()})
+    if g.name == "rnn":
+        T = np.diff(inst.offsets)
+        return dict(node_messages=int((13 * T + 3).sum()),
+                    grads={g.index("lookup"): T.sum(), g.index("linear1"): T.sum(), g.index("linear2"): inst.n})
+    if g.name == "tree":
+        L = (np.diff(inst.offsets) + 1) // 2
+        return dict(node_messages=int((33 * L - 18).sum()),
+                    grads={g.index("lookup"): L.sum(), g.index("leaf_cell"): L.sum(),
+                           g.index("branch_cell"): (L - 1).sum(), g.index("classifier"): (2 * L - 1).sum()})
+    N, D = np.diff(inst.offsets), np.diff(inst.edge_offsets)
+    gid = np.repeat(np.arange(inst.n), D)
+    Dc = np.zeros((inst.n, 4), np.int64)
+    np.add.at(Dc, (gid, inst.edge_type), 1)
+    Cp = (Dc > 0).sum(1)
+    grads = {g.index("lookup"): N.sum(), g.index("gru"): 4 * N.sum(), g.index("readout1"): inst.n,
+             g.index("readout2"): inst.n}
+    for c in range(4):
+        grads[g.index(f"edge_linear{c}")] = 4 * Dc[:, c].sum()
+    return dict(node_messages=int((4 * (6 * N + 4 * D + 8 * Cp + 16) + 9).sum()), grads=grads)
+
+
+def test_async_convergence_matches_synchronous_oracle(oracle_mod):
+    """Asynchronous training (mak = 16) reaches the synchronous oracle's accuracy within 1 point in the same
+    number of epochs on the list-reduction task."""
+    import paper_1705_09786_b200 as amp
+    g = ir.rnn()
+    train, valid = data.list_instances(n=3000), data.list_instances(n=1000, split=1)
+    p = wp.init_params(g)
+    o = oracle_mod.Oracle(g)
+    o.load_instances(train)
+    o.load_instances(valid, split=1)
+    o.set_params(p)
+    e = amp.Engine(g)
+    e.load_instances(train)
+    e.load_instances(valid, split=1)
+    e.set_params(p)
+    epochs = 6
+    for _ in range(epochs):
+        o.run_epoch(mak=1, muf=50, lr=0.05)
+        e.run_epoch(mak=16, muf=50, lr=0.05, deterministic=False, timeout_s=120)
+    _, oacc, _ = o.eval(split=1)
+    assert oacc > 0.3                                   # the task is being learnt (chance is 0.1)
+    best = e.eval(split=1)[1]
+    for _ in range(2):                                  # "a similar number of epochs": at most two more
+        if best >= oacc - 0.01:
+            break
+        e.run_epoch(mak=16, muf=50, lr=0.05, deterministic=False, timeout_s=120)
+        best = max(best, e.eval(split=1)[1])
+    assert best >= oacc - 0.01                          # within one accuracy point
+    e.close()
+
+
+# ---------------------------------------------------------------------------------------------------
+# failure paths: every one returns a status, none faults or hangs the device
+# ---------------------------------------------------------------------------------------------------
+def test_error_statuses_and_recovery():
+    import paper_1705_09786_b200 as amp
+    g, inst = _case("tree", 200)
+    e = amp.Engine(g)
+    with pytest.raises(amp.AmpnetError) as ei:                       # run before load
+        e.run_epoch(mak=4, muf=10, lr=0.01)
+    assert ei.value.status == 6
+    e.load_instances(inst)
+    e.set_params(wp.init_params(g))
+    with pytest.raises(amp.AmpnetError) as ei:                       # the run's time budget is 20 microseconds
+        e.run_epoch(mak=64, muf=100, lr=0.05, timeout_s=2e-5)
+    assert ei.value.status == 4
+    # the context is still usable and a normal run completes
+    e.set_params(wp.init_params(g))
+    st, loss = e.run_epoch(mak=64, muf=100, lr=0.05, timeout_s=60)
+    assert st.instances == inst.n and np.isfinite(loss).all()
+    with pytest.raises(amp.AmpnetError) as ei:
+        e.run_epoch(mak=0, muf=100, lr=0.05)
+    assert ei.value.status == 1
+    with pytest.raises(amp.AmpnetError) as ei:
+        e.run_epoch(mak=4, muf=100, lr=0.05, order=np.array([0, 999999]))
+    assert ei.value.status == 1
+    e.close()
+
+
+def test_malformed_ir_and_instances_are_rejected():
+    import paper_1705_09786_b200 as amp
+    g = ir.mlp((8, 4, 3))
+    g._edges[1] = (1, 0, 2, 3)                                       # predecessor ports 0..2 left unconnected
+    with pytest.raises(amp.AmpnetError) as ei:
+        amp.Engine(g)
+    assert ei.value.status == 1
+    g = ir.IRGraph("cycle")                                          # a loop that does not pass through a Phi
+    s = g.node("src", ir.SOURCE, out_dim=4, fn=ir.SRC_DENSE_ROW)
+    a = g.node("a", ir.LINEAR, 4, 4, flags=ir.FLAG_SOURCE_ADJACENT)
+    c = g.node("cat", ir.CONCAT, 4, 8, fn=ir.CONCAT_BY_EDGE, fn_arg=2)
+    b = g.node("b", ir.LINEAR, 8, 4)
+    bc = g.node("bc", ir.BCAST, 4, 4, fn_arg=2)
+    l = g.node("loss", ir.LOSS_CE, 4, 0, fn=ir.LABEL_PER_INSTANCE)
+    g.edge(s, a); g.edge(a, c, 0, 0); g.edge(c, b); g.edge(b, bc); g.edge(bc, l, 0, 0); g.edge(bc, c, 1, 1)
+    with pytest.raises(amp.AmpnetError):
+        amp.Engine(g)
+    g = ir.ggnn()
+    e = amp.Engine(g)
+    inst = data.graph_instances(n=3)
+    inst.edge_src = inst.edge_src.copy(); inst.edge_dst = inst.edge_dst.copy()
+    v = int(inst.offsets[1] - inst.offsets[0]) - 1                   # make the last node of graph 0 isolated
+    o0, o1 = int(inst.edge_offsets[0]), int(inst.edge_offsets[1])
+    inst.edge_src[o0:o1][inst.edge_src[o0:o1] == v] = 0
+    inst.edge_dst[o0:o1][inst.edge_dst[o0:o1] == v] = 1
+    with pytest.raises(amp.AmpnetError) as ei:
+        e.load_instances(inst)
+    assert ei.value.status == 1
+    bad = data.tree_instances(n=2)
+    with pytest.raises(amp.AmpnetError):                             # trees into a graph network
+        e.load_instances(bad)
+    e.close()
+    g = ir.tree(vocab=100)
+    e = amp.Engine(g)
+    with pytest.raises(amp.AmpnetError):                             # leaf tokens beyond the embedding table
+        e.load_instances(data.tree_instances(n=5, vocab=20000))
+    e.close()
