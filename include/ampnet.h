@@ -180,6 +180,29 @@ ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_t
 
 const char* ampnet_last_error(const ampnet_graph_t*); /* library-owned string */
 
+/* ---- a training epoch that allocates nothing (no counterpart in the paper) ------------------------------
+ * For callers that must not allocate device memory once they are running: a training loop that has handed all
+ * free device memory to another pool, a latency-critical loop that cannot afford the device-wide
+ * synchronisation of cudaMalloc/cudaFree, or a host that forbids allocation after start-up.  The handle is
+ * created and its instances loaded beforehand (those calls allocate); this call then runs one epoch exactly
+ * like ampnet_run_epoch, but its queues, counters and keyed caches live in a fixed array of
+ * AMPNET_STATIC_SCRATCH_BYTES inside the library image instead of allocator memory.  It calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *   - A run whose scratch does not fit (large max_active_keys, big structures or vocabularies) is refused with
+ *     AMPNET_EINVAL; ampnet_last_error states the bytes needed and the bytes available.  Nothing has run then.
+ *   - Every GPU that loads the library holds the array until the process exits.
+ *   - The first call on a device looks up the array's device address; make that first call outside any stream
+ *     capture.
+ *   - All handles and all calls share the one array: what must start at zero is cleared at the start of each
+ *     call, the rest keeps the previous call's contents.  Two such calls that overlap on the GPU (different
+ *     streams or threads) race; serialise them.
+ *   - ampnet_get_node_stats / ampnet_get_update_log / ampnet_get_key_log describe this run until the next call
+ *     that uses the array; ampnet_leftover_cache_entries reports 0 after it.
+ * Arguments, outputs and statuses are those of ampnet_run_epoch.                                             */
+#define AMPNET_STATIC_SCRATCH_BYTES (64u << 20)
+ampnet_status_t ampnet_run_epoch_static(ampnet_graph_t*, const ampnet_run_cfg_t*, ampnet_epoch_stats_t* out,
+                                        float* per_instance_loss);
+
 #ifdef __cplusplus
 }
 #endif

@@ -12,7 +12,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error"]
+           "ampnet_last_error", "ampnet_run_epoch_static"]
 
 
 class AmpnetError(RuntimeError):
@@ -82,6 +82,7 @@ def load_library():
     lib.ampnet_graph_destroy.restype = None
     lib.ampnet_load_instances.argtypes = [P, C.c_int32, C.POINTER(Instances)]
     lib.ampnet_run_epoch.argtypes = [P, C.POINTER(RunCfg), C.POINTER(EpochStats), P]
+    lib.ampnet_run_epoch_static.argtypes = [P, C.POINTER(RunCfg), C.POINTER(EpochStats), P]
     lib.ampnet_eval.argtypes = [P, C.c_int32, C.c_int32, C.POINTER(C.c_double), C.POINTER(C.c_double), P]
     lib.ampnet_param_count.argtypes = [P, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
     lib.ampnet_get_params.argtypes = [P, C.c_int32, C.c_int32, P, C.c_int64]
@@ -179,13 +180,17 @@ class Engine:
         return a.reshape(dict(self.graph.param_shapes(node))[which])
 
     def run_epoch(self, mak, muf, lr, deterministic=False, order=None, timeout_s=0.0, max_batch_rows=0, n_ctas=0,
-                  want_loss=True):
+                  want_loss=True, static_scratch=False):
+        """One training epoch.  static_scratch=True calls ampnet_run_epoch_static: the same epoch with its run
+        state in the library's fixed scratch array, for callers that must not allocate device memory (it is
+        refused with EINVAL when the run state does not fit; calls sharing the array must not overlap)."""
         order = None if order is None else np.ascontiguousarray(order, dtype=np.int64)
         cfg = RunCfg(mak, muf, lr, int(deterministic), _p(order), 0 if order is None else len(order), timeout_s,
                      max_batch_rows, n_ctas)
         st = EpochStats()
         loss = np.zeros(self.n[0], np.float32) if want_loss else None
-        self._check(self.lib.ampnet_run_epoch(self.h, C.byref(cfg), C.byref(st), _p(loss)))
+        fn = self.lib.ampnet_run_epoch_static if static_scratch else self.lib.ampnet_run_epoch
+        self._check(fn(self.h, C.byref(cfg), C.byref(st), _p(loss)))
         return st, loss
 
     def eval(self, split=0, mak=64):

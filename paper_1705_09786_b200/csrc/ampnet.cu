@@ -985,3 +985,49 @@ ampnet_status_t ampnet_get_placement(ampnet_graph_t* g, int32_t node, int32_t* n
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------------------
+// Training epoch that allocates nothing
+// ---------------------------------------------------------------------------------------------------------
+// Scratch of ampnet_run_epoch_static: the queues, counters and keyed caches of one run.  It lives in the
+// library image, so every GPU that loads the library holds these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_static_scratch[AMPNET_STATIC_SCRATCH_BYTES];
+// In host code the array's name is only a stand-in; the device address comes from cudaGetSymbolAddress.
+static void* g_static_scratch_addr[64] = {nullptr};
+
+extern "C" ampnet_status_t ampnet_run_epoch_static(ampnet_graph_t* g, const ampnet_run_cfg_t* cfg,
+                                                   ampnet_epoch_stats_t* out, float* per_instance_loss) {
+  if (!g) return AMPNET_EINVAL;
+  if (!cfg) return set_err(g, AMPNET_EINVAL, "NULL run configuration");
+  if (g->device < 0 || g->device >= 64) return set_err(g, AMPNET_EINVAL, "device index %d not supported", g->device);
+  HostDataset& D = g->data[0];
+  if (!D.loaded) return set_err(g, AMPNET_ESTATE, "no instances loaded for split 0");
+  if (cfg->max_active_keys < 1 || cfg->min_update_frequency < 1) return set_err(g, AMPNET_EINVAL, "max_active_keys and min_update_frequency must be >= 1");
+  CUDA_TRY(g, cudaSetDevice(g->device));
+  if (!g_static_scratch_addr[g->device]) {       // set-up, once per device, with that device current
+    void* ptr = nullptr;
+    CUDA_TRY(g, cudaGetSymbolAddress(&ptr, g_static_scratch));
+    g_static_scratch_addr[g->device] = ptr;
+  }
+  // size the run state without touching any memory, and refuse what does not fit
+  const long long n_order = cfg->order ? cfg->n_order : D.n;
+  RunPlan plan;
+  ampnet_status_t st = plan_run(g, 0, cfg->max_active_keys, cfg->deterministic ? 1 : 0, 0, cfg, n_order, true, plan);
+  if (st != AMPNET_OK) return st;
+  const size_t order_bytes = cfg->order ? (size_t)std::max<long long>(n_order, 0) * sizeof(long long) : 0;
+  const size_t ctl_need = ((g->ctl.used + 4096 + 255) & ~(size_t)255);
+  const size_t bulk_need = g->bulk.used + order_bytes + 512 + 4096;
+  if (ctl_need + bulk_need > (size_t)AMPNET_STATIC_SCRATCH_BYTES)
+    return set_err(g, AMPNET_EINVAL, "this run needs %zu bytes of scratch but the static scratch holds %zu: lower "
+                   "max_active_keys or use ampnet_run_epoch", ctl_need + bulk_need, (size_t)AMPNET_STATIC_SCRATCH_BYTES);
+  // lend the static array to the handle for the duration of this call
+  void *own_ctl = g->ctl_mem, *own_bulk = g->bulk_mem;
+  const size_t own_ctl_cap = g->ctl_cap, own_bulk_cap = g->bulk_cap;
+  char* base = static_cast<char*>(g_static_scratch_addr[g->device]);
+  g->ctl_mem = base; g->ctl_cap = ctl_need;
+  g->bulk_mem = base + ctl_need; g->bulk_cap = (size_t)AMPNET_STATIC_SCRATCH_BYTES - ctl_need;
+  st = execute(g, 0, cfg->max_active_keys, cfg->deterministic ? 1 : 0, 0, cfg, out, per_instance_loss, nullptr);
+  g->ctl_mem = own_ctl; g->ctl_cap = own_ctl_cap; g->bulk_mem = own_bulk; g->bulk_cap = own_bulk_cap;
+  g->leftover_regions.clear();      // they described the lent memory
+  return st;
+}
