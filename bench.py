@@ -256,14 +256,10 @@ def run_ours(args):
         kavg = float(np.mean(kern_s))
         achieved = flops / kavg / 1e12
         roof_inst, F, B = rf.roofline_instances_per_s(graph, inst, sm_mhz, float(peaks.get("hbm_gbs", 6650.0)))
-        traffic = None
-        prof = os.path.join(ROOT, "profiles", f"traffic_{args.workload}.json")
-        note = "no ncu capture yet"
-        if os.path.exists(prof):
-            with open(prof) as f:
-                t = json.load(f)
-            traffic = t["dram_bytes_per_instance"] * inst.n
-            note = t.get("note", "")
+        per_inst = rf.MEASURED_DRAM_BYTES_PER_INSTANCE.get(args.workload)
+        traffic = per_inst * inst.n if per_inst else None
+        note = ("ncu capture on a small case, scaled by instances processed (see profiles/)" if per_inst
+                else "no ncu capture for this workload")
         roofline = {"bound": "alu", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
                     "traffic": traffic, "traffic_note": note,
                     "peak_kind": f"derived: 148 SMs x 128 FP32 lanes x 2 x {sm_mhz:.0f} MHz ({peak_kind} max SM clock)",
