@@ -178,6 +178,11 @@ ampnet_status_t ampnet_leftover_cache_entries(ampnet_graph_t*, int64_t* n);
 /* Placement chosen for a parameterised node: number of row tiles (CTAs) and micro-batch row capacity.        */
 ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_tiles, int32_t* batch_rows);
 
+/* Where the leader tile of a node spent its SM cycles in the last run: [0] waiting for messages, [1] fetching a
+ * batch descriptor, [2] loading headers, [3] staging + arithmetic, [4] local updates, [5] barrier among the node's
+ * tiles, [6] emission (walking the parameter-free nodes), [7] loop overhead.  batches: micro-batches executed.   */
+ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles8, int64_t* batches);
+
 const char* ampnet_last_error(const ampnet_graph_t*); /* library-owned string */
 
 /* ---- a training epoch that allocates nothing (no counterpart in the paper) ------------------------------

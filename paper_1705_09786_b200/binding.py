@@ -12,7 +12,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error", "ampnet_run_epoch_static"]
+           "ampnet_last_error", "ampnet_run_epoch_static", "ampnet_get_phase_cycles"]
 
 
 class AmpnetError(RuntimeError):
@@ -92,6 +92,7 @@ def load_library():
     lib.ampnet_get_key_log.argtypes = [P, P, P, P, P, C.c_int64, C.POINTER(C.c_int64)]
     lib.ampnet_leftover_cache_entries.argtypes = [P, C.POINTER(C.c_int64)]
     lib.ampnet_get_placement.argtypes = [P, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
+    lib.ampnet_get_phase_cycles.argtypes = [P, C.c_int32, P, C.POINTER(C.c_int64)]
     lib.ampnet_last_error.argtypes = [P]
     lib.ampnet_last_error.restype = C.c_char_p
     _LIB = lib
@@ -227,6 +228,12 @@ class Engine:
         n = C.c_int64()
         self._check(self.lib.ampnet_leftover_cache_entries(self.h, C.byref(n)))
         return n.value
+
+    def phase_cycles(self, node):
+        a = np.zeros(8, np.uint64)
+        b = C.c_int64()
+        self._check(self.lib.ampnet_get_phase_cycles(self.h, node, _p(a), C.byref(b)))
+        return a, b.value
 
     def placement(self, node):
         t, b = C.c_int32(), C.c_int32()

@@ -355,7 +355,7 @@ size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
 ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles) {
   const size_t budget = ((size_t)g->max_smem - 12 * 1024) / sizeof(float);
   int max_tiles = 16;
-  if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, atoi(e));
+  if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, std::min(MAX_TILES, atoi(e)));
   double total_w = 0;
   for (auto& P : g->ppts) if (P.kind != LOOKUP) total_w += (double)P.nmat * P.in * P.out;
   const int avail = std::max(1, n_ctas - 1 - (int)g->ppts.size());
@@ -973,6 +973,16 @@ ampnet_status_t ampnet_leftover_cache_entries(ampnet_graph_t* g, int64_t* n) {
     for (unsigned char c : h) cnt += c != 0;
   }
   *n = cnt;
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t* g, int32_t node, uint64_t* cycles8, int64_t* batches) {
+  if (!g) return AMPNET_EINVAL;
+  if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
+  if (node < 0 || node >= (int)g->hnodes.size() || g->hnodes[node].ppt < 0) return set_err(g, AMPNET_EINVAL, "not a parameterised node");
+  const PPTStats& s = g->last_stats[g->hnodes[node].ppt];
+  if (cycles8) for (int k = 0; k < 8; k++) cycles8[k] = s.phase_cycles[k];
+  if (batches) *batches = (int64_t)s.batches;
   return AMPNET_OK;
 }
 

@@ -90,18 +90,44 @@ struct Frame {
   int node, aport, dir, iter;
   int inst, seq, slot, it, u, port, rows, flags;
   int dim, ld;
+  int nsum, sstride;    // payload element (r, i) = sum over j < nsum of p[j * sstride + r * ld + i]
   const float* p;       // payload rows (device memory); nullptr = zeros
+};
+
+// Frames offered by a walking warp to the other warps of its CTA (continuations of forks).
+constexpr int POOL = 64;
+struct WalkPool {
+  Frame f[POOL];
+  unsigned ready[POOL];      // ticket + 1 while the slot holds a frame, 0 when free
+  unsigned head, tail;
+  int outstanding;           // frames queued or being walked
 };
 
 struct WalkAcc { unsigned long long msgs, hash; };
 
-__device__ __forceinline__ void warp_copy(float* dst, int dld, const float* src, int sld, int rows, int dim,
-                                          int lane) {
-  for (int r = 0; r < rows; r++)
-    for (int i = lane; i < dim; i += 32) dst[(size_t)r * dld + i] = src ? __ldcg(src + (size_t)r * sld + i) : 0.f;
+__device__ __forceinline__ float ld_payload(const float* p, int nsum, int sstride, size_t off) {
+  float s = __ldcg(p + off);
+  for (int j = 1; j < nsum; j++) s += __ldcg(p + (size_t)j * sstride + off);     // addend order
+  return s;
+}
+// Copy payload rows into a cache; a lazy sum is evaluated on the way.  Four elements per lane in flight.
+__device__ __forceinline__ void warp_copy(float* dst, int dld, const Frame& f, int rows, int dim, int lane) {
+  const float* src = f.p;
+  for (int r = 0; r < rows; r++) {
+    float* d = dst + (size_t)r * dld;
+    if (!src) { for (int i = lane; i < dim; i += 32) d[i] = 0.f; continue; }
+    const size_t ro = (size_t)r * f.ld;
+    for (int i0 = lane; i0 < dim; i0 += 128) {
+      float v[4];
+#pragma unroll
+      for (int k = 0; k < 4; k++) { const int i = i0 + 32 * k; v[k] = i < dim ? ld_payload(src, f.nsum, f.sstride, ro + i) : 0.f; }
+#pragma unroll
+      for (int k = 0; k < 4; k++) { const int i = i0 + 32 * k; if (i < dim) d[i] = v[k]; }
+    }
+  }
 }
 
-__device__ __forceinline__ void ring_push(Ring& r, const Frame& f) {   // one lane, after the payload is fenced
+__device__ __forceinline__ void ring_push(Ring& r, const Frame& f) {   // one lane; the release store orders the payload
   unsigned t = atomicAdd(r.tail, 1u);
   unsigned s = t & r.mask;
   int4* d = reinterpret_cast<int4*>(&r.e[s]);
@@ -119,18 +145,47 @@ __device__ __forceinline__ void retire_push(const Ctx& C, int slot) {
 
 // Join on a keyed counter: every arriving warp has written its part; the one that completes the count
 // continues.  Returns true for the completing arrival (and resets the counter for the key's next use).
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
 __device__ __forceinline__ bool join_arrive(int* cnt, int expected, int lane) {
-  __threadfence();
-  __syncwarp();
+  __syncwarp();                       // the lanes' writes of this part are ordered before lane 0's release
   int last = 0;
   if (lane == 0) {
-    int old = atomicAdd(cnt, 1);
+    int old = atom_add_acq_rel(cnt, 1);
     last = (old + 1 == expected);
     if (last) { *cnt = 0; }
   }
   last = __shfl_sync(0xffffffffu, last, 0);
-  if (last) __threadfence();
   return last != 0;
+}
+
+// ---- CTA-wide pool of frames: a warp that forks offers the rest of the fork to idle warps --------------
+__device__ __forceinline__ bool pool_offer(WalkPool* Q, const Frame& c, int lane) {
+  if (!Q) return false;
+  int ok = 0;
+  if (lane == 0) {
+    unsigned t = *(volatile unsigned*)&Q->tail;
+    for (;;) {
+      const unsigned h = *(volatile unsigned*)&Q->head;
+      if (t - h >= (unsigned)POOL) break;
+      const unsigned old = atomicCAS(&Q->tail, t, t + 1u);
+      if (old == t) { ok = 1; break; }
+      t = old;
+    }
+    if (ok) {
+      const unsigned idx = t % POOL;
+      atomicAdd(&Q->outstanding, 1);
+      int spins = 0;
+      while (*(volatile unsigned*)&Q->ready[idx] != 0u && ++spins < (1 << 20)) {}
+      Q->f[idx] = c;
+      __threadfence_block();
+      *(volatile unsigned*)&Q->ready[idx] = t + 1u;
+    }
+  }
+  return __shfl_sync(0xffffffffu, ok, 0) != 0;
 }
 
 __device__ __forceinline__ void to_succ(Frame& f, const DevNode& n, int k) {
@@ -140,7 +195,7 @@ __device__ __forceinline__ void to_pred(Frame& f, const DevNode& n, int j) {
   f.node = n.pred_node[j]; f.aport = n.pred_port[j]; f.dir = BWD; f.iter = 0;
 }
 
-__device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
+__device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool* Q) {
   const int lane = threadIdx.x & 31;
   const DevInst& I = C.inst;
   int sp = 0;
@@ -171,12 +226,11 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
           if (f.dir == FWD) {
             if (P.xcache) {
               float* dst = P.xcache + key * (long long)P.rows_max * P.in_dim;
-              if (f.p != dst) warp_copy(dst, P.in_dim, f.p, f.ld, f.rows, P.in_dim, lane);
+              if (f.p != dst) warp_copy(dst, P.in_dim, f, f.rows, P.in_dim, lane);
             }
           } else if (n.type != LOOKUP || f.dim > 0) {
-            warp_copy(P.gbuf + key * (long long)P.rows_max * P.out_dim, P.out_dim, f.p, f.ld, f.rows, P.out_dim, lane);
+            warp_copy(P.gbuf + key * (long long)P.rows_max * P.out_dim, P.out_dim, f, f.rows, P.out_dim, lane);
           }
-          __threadfence();
           __syncwarp();
           if (lane == 0) ring_push(P.ring[f.dir], f);
         } break;
@@ -187,29 +241,29 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
           if (n.type == LOSS_CE) {
             int label = I.labels_i[I.labels_per_node ? ibase + f.u : f.inst];
             float mx = -3.4e38f; int arg = 0x7fffffff;
-            for (int j = lane; j < n.in_dim; j += 32) { float v = __ldcg(f.p + j); if (v > mx) { mx = v; arg = j; } }
+            for (int j = lane; j < n.in_dim; j += 32) { float v = ld_payload(f.p, f.nsum, f.sstride, j); if (v > mx) { mx = v; arg = j; } }
             for (int o = 16; o; o >>= 1) {
               float om = __shfl_xor_sync(0xffffffffu, mx, o); int oa = __shfl_xor_sync(0xffffffffu, arg, o);
               if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
             }
             float s = 0.f;
-            for (int j = lane; j < n.in_dim; j += 32) s += expf(__ldcg(f.p + j) - mx);
+            for (int j = lane; j < n.in_dim; j += 32) s += expf(ld_payload(f.p, f.nsum, f.sstride, j) - mx);
             for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             float lse = mx + logf(s);
-            for (int j = lane; j < n.in_dim; j += 32) g[j] = expf(__ldcg(f.p + j) - lse) - (j == label ? 1.f : 0.f);
-            if (lane == 0) { n.lossval[key] = lse - __ldcg(f.p + label); n.predok[key] = (arg == label) ? 1 : 0; }
+            for (int j = lane; j < n.in_dim; j += 32) g[j] = expf(ld_payload(f.p, f.nsum, f.sstride, j) - lse) - (j == label ? 1.f : 0.f);
+            if (lane == 0) { n.lossval[key] = lse - ld_payload(f.p, f.nsum, f.sstride, label); n.predok[key] = (arg == label) ? 1 : 0; }
           } else {
             if (lane == 0) {
-              float d = __ldcg(f.p) - I.labels_f[f.inst];
+              float d = ld_payload(f.p, f.nsum, f.sstride, 0) - I.labels_f[f.inst];
               n.lossval[key] = d * d; g[0] = 2.f * d; n.predok[key] = 0;
             }
           }
-          if (f.flags & HDR_EVAL) { __threadfence(); __syncwarp(); if (lane == 0) retire_push(C, f.slot); }
-          else { __syncwarp(); f.p = g; f.dim = n.in_dim; f.ld = n.in_dim; to_pred(f, n, 0); cont = true; }
+          if (f.flags & HDR_EVAL) { __syncwarp(); if (lane == 0) retire_push(C, f.slot); }
+          else { __syncwarp(); f.p = g; f.nsum = 1; f.dim = n.in_dim; f.ld = n.in_dim; to_pred(f, n, 0); cont = true; }
         } break;
         case SINK:
           if (f.flags & HDR_EVAL) { if (lane == 0) retire_push(C, f.slot); }
-          else { f.p = nullptr; to_pred(f, n, 0); cont = true; }
+          else { f.p = nullptr; f.nsum = 1; to_pred(f, n, 0); cont = true; }
           break;
         case COND:
           if (f.dir == FWD) {
@@ -257,8 +311,9 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
         case BCAST:
           if (f.dir == FWD) {
             int k = f.iter;
-            if (k + 1 < n.fn_arg) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
-                                    Frame c = f; c.iter = k + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            if (k + 1 < n.fn_arg) { Frame c = f; c.iter = k + 1;
+              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                             if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             to_succ(f, n, k);
             cont = true;
           } else {
@@ -266,16 +321,10 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
             if (key < 0) return;
             float* base = n.jbuf + key * n.jstride;
             const int blk = n.rows_in * n.in_dim;
-            warp_copy(base + (size_t)f.aport * blk, n.in_dim, f.p, f.ld, f.rows, n.in_dim, lane);
+            warp_copy(base + (size_t)f.aport * blk, n.in_dim, f, f.rows, n.in_dim, lane);
             if (join_arrive(&n.jcnt[key], n.fn_arg, lane)) {
-              float* sum = base + (size_t)n.fn_arg * blk;
-              for (int i = lane; i < f.rows * n.in_dim; i += 32) {
-                float s = 0.f;
-                for (int k = 0; k < n.fn_arg; k++) s += __ldcg(base + (size_t)k * blk + i);   // successor order
-                sum[i] = s;
-              }
-              __syncwarp();
-              f.p = sum; f.ld = n.in_dim; f.dim = n.in_dim;
+              f.p = base; f.nsum = n.fn_arg; f.sstride = blk;      // summed in successor order by whoever reads it
+              f.ld = n.in_dim; f.dim = n.in_dim;
               to_pred(f, n, 0);
               cont = true;
             }
@@ -288,16 +337,17 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
             if (key < 0) return;
             if ((unsigned)port >= (unsigned)n.fn_arg || f.rows > n.rows_in) { fail(C, ST_OVERFLOW, f.node, port); return; }
             float* base = n.jbuf + key * n.jstride;
-            warp_copy(base + port * n.in_dim, n.out_dim, f.p, f.ld, f.rows, n.in_dim, lane);
+            warp_copy(base + port * n.in_dim, n.out_dim, f, f.rows, n.in_dim, lane);
             if (join_arrive(&n.jcnt[key], n.fn_arg, lane)) {
-              f.p = base; f.dim = n.out_dim; f.ld = n.out_dim; f.port = 0;
+              f.p = base; f.nsum = 1; f.dim = n.out_dim; f.ld = n.out_dim; f.port = 0;
               to_succ(f, n, 0);
               cont = true;
             }
           } else {
             int k = f.iter;
-            if (k + 1 < n.fn_arg) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
-                                    Frame c = f; c.iter = k + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            if (k + 1 < n.fn_arg) { Frame c = f; c.iter = k + 1;
+              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                             if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             f.p = f.p ? f.p + k * n.in_dim : nullptr; f.dim = n.in_dim;
             if (n.fn == 2) { f.port = k; to_pred(f, n, 0); } else to_pred(f, n, k);
             cont = true;
@@ -316,16 +366,17 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
             if (key < 0) return;
             if (member >= n.rows_out || count > n.rows_out) { fail(C, ST_OVERFLOW, f.node, member); return; }
             float* base = n.jbuf + key * n.jstride;
-            warp_copy(base + (size_t)member * n.in_dim, n.in_dim, f.p, f.ld, 1, n.in_dim, lane);
+            warp_copy(base + (size_t)member * n.in_dim, n.in_dim, f, 1, n.in_dim, lane);
             if (join_arrive(&n.jcnt[key], count, lane)) {
-              f.u = gkey; f.rows = count; f.p = base; f.ld = n.in_dim; f.dim = n.in_dim;
+              f.u = gkey; f.rows = count; f.p = base; f.nsum = 1; f.ld = n.in_dim; f.dim = n.in_dim;
               to_succ(f, n, 0);
               cont = true;
             }
           } else {
             int i = f.iter;
-            if (i + 1 < f.rows) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
-                                  Frame c = f; c.iter = i + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            if (i + 1 < f.rows) { Frame c = f; c.iter = i + 1;
+              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                             if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             const long long ebase = I.edge_off ? I.edge_off[f.inst] : 0;
             int mu;
             if (n.fn == 1) mu = I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i];
@@ -340,8 +391,9 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
         case UNGROUP:
           if (f.dir == FWD) {
             int i = f.iter;
-            if (i + 1 < f.rows) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
-                                  Frame c = f; c.iter = i + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            if (i + 1 < f.rows) { Frame c = f; c.iter = i + 1;
+              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                             if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             int mu = n.fn == 2 ? I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i] : i;
             f.p = f.p ? f.p + (size_t)i * f.ld : nullptr; f.rows = 1; f.u = mu;
             to_succ(f, n, 0);
@@ -355,9 +407,9 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
             if (key < 0) return;
             if (row >= n.rows_in) { fail(C, ST_OVERFLOW, f.node, row); return; }
             float* base = n.jbuf + key * n.jstride;
-            warp_copy(base + (size_t)row * n.in_dim, n.in_dim, f.p, f.ld, 1, n.in_dim, lane);
+            warp_copy(base + (size_t)row * n.in_dim, n.in_dim, f, 1, n.in_dim, lane);
             if (join_arrive(&n.jcnt[key], expected, lane)) {
-              f.u = gkey; f.rows = expected; f.p = base; f.ld = n.in_dim; f.dim = n.in_dim;
+              f.u = gkey; f.rows = expected; f.p = base; f.nsum = 1; f.ld = n.in_dim; f.dim = n.in_dim;
               to_pred(f, n, 0);
               cont = true;
             }
@@ -369,8 +421,9 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
             int deg = (int)(oo[1] - oo[0]);
             int i = f.iter;
             if (deg > 0) {
-              if (i + 1 < deg) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
-                                 Frame c = f; c.iter = i + 1; if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+              if (i + 1 < deg) { Frame c = f; c.iter = i + 1;
+              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                             if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
               f.u = I.out_list[oo[0] + i];
               to_succ(f, n, 0);
               cont = true;
@@ -384,16 +437,10 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
             const int maxdeg = (int)(n.jstride / n.in_dim) - 1;
             if (member >= maxdeg || deg > maxdeg) { fail(C, ST_OVERFLOW, f.node, member); return; }
             float* base = n.jbuf + key * n.jstride;
-            warp_copy(base + (size_t)member * n.in_dim, n.in_dim, f.p, f.ld, 1, n.in_dim, lane);
+            warp_copy(base + (size_t)member * n.in_dim, n.in_dim, f, 1, n.in_dim, lane);
             if (join_arrive(&n.jcnt[key], deg, lane)) {
-              float* sum = base + (size_t)maxdeg * n.in_dim;
-              for (int i = lane; i < n.in_dim; i += 32) {
-                float s = 0.f;
-                for (int k = 0; k < deg; k++) s += __ldcg(base + (size_t)k * n.in_dim + i);     // edge order
-                sum[i] = s;
-              }
-              __syncwarp();
-              f.u = v; f.rows = 1; f.p = sum; f.ld = n.in_dim; f.dim = n.in_dim;
+              f.u = v; f.rows = 1; f.p = base; f.nsum = deg; f.sstride = n.in_dim;   // summed in edge order when read
+              f.ld = n.in_dim; f.dim = n.in_dim;
               to_pred(f, n, 0);
               cont = true;
             }
@@ -406,12 +453,12 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc) {
             float* out = n.jbuf + key * n.jstride;
             for (int i = lane; i < n.in_dim; i += 32) {
               float s = 0.f;
-              for (int r = 0; r < f.rows; r++) s += f.p ? __ldcg(f.p + (size_t)r * f.ld + i) : 0.f;   // row order
+              for (int r = 0; r < f.rows; r++) s += f.p ? ld_payload(f.p, f.nsum, f.sstride, (size_t)r * f.ld + i) : 0.f;   // row order
               out[i] = s;
             }
             if (lane == 0 && !(f.flags & HDR_EVAL)) n.rowcnt[key] = f.rows;
             __syncwarp();
-            f.rows = 1; f.p = out; f.ld = n.in_dim; f.dim = n.in_dim;
+            f.rows = 1; f.p = out; f.nsum = 1; f.ld = n.in_dim; f.dim = n.in_dim;
             to_succ(f, n, 0);
           } else {
             int rows = *(volatile int*)&n.rowcnt[key];
@@ -440,6 +487,44 @@ __device__ __forceinline__ void flush_acc(const Ctx& C, WalkAcc& a, int lane) {
     atomicAdd(&C.g->route_hash, a.hash);
   }
   a.msgs = 0; a.hash = 0;
+}
+
+// A warp that has walked its own frames helps with what the others offered, until nothing is outstanding.
+__device__ void pool_steal(const Ctx& C, WalkPool* Q, Frame* stack, WalkAcc& acc) {
+  const int lane = threadIdx.x & 31;
+  unsigned idle = 0;
+  for (;;) {
+    int got = 0;
+    unsigned h = 0;
+    if (lane == 0) {
+      h = *(volatile unsigned*)&Q->head;
+      unsigned t = *(volatile unsigned*)&Q->tail;
+      while (h != t) {
+        const unsigned old = atomicCAS(&Q->head, h, h + 1u);
+        if (old == h) { got = 1; break; }
+        h = old;
+        t = *(volatile unsigned*)&Q->tail;
+      }
+    }
+    got = __shfl_sync(0xffffffffu, got, 0);
+    if (got) {
+      h = __shfl_sync(0xffffffffu, h, 0);
+      const unsigned idx = h % POOL;
+      if (lane == 0) { int spins = 0; while (*(volatile unsigned*)&Q->ready[idx] != h + 1u && ++spins < (1 << 20)) {} }
+      __syncwarp();
+      Frame f = Q->f[idx];
+      __syncwarp();
+      if (lane == 0) *(volatile unsigned*)&Q->ready[idx] = 0u;
+      walk(C, f, stack, acc, Q);
+      __syncwarp();
+      if (lane == 0) atomicSub(&Q->outstanding, 1);
+      idle = 0;
+    } else {
+      if (*(volatile int*)&Q->outstanding <= 0) break;
+      if ((++idle & 1023u) == 0 && aborted(C)) break;
+      __nanosleep(20);
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -594,7 +679,11 @@ __device__ void tile_accum(const float* __restrict__ Ds, int ldd, int nb, const 
 // ------------------------------------------------------------------------------------------------
 // PPT tile: batch bookkeeping in shared memory
 // ------------------------------------------------------------------------------------------------
-struct LeaderState { unsigned head[2], sched_w, batch_w; int n_acc, version; };
+struct LeaderState {
+  unsigned head[2], sched_w, batch_w;
+  int n_acc, version, log_n;
+  unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
+};
 
 struct TileShared {
   BatchDesc desc;
@@ -602,12 +691,15 @@ struct TileShared {
   long long key[MAX_BATCH_MSGS];
   int rowoff[MAX_BATCH_MSGS + 1];
   int rowmsg[64];
+  const float* rowptr[64];
   LeaderState ls;
   int ok;
   unsigned tail_snap[2];
   unsigned long long stale_hist[64];
   int max_stale;
+  unsigned long long phase[8];
   Frame stack[WARPS][WALK_STACK];
+  WalkPool pool;
 };
 
 __device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) {
@@ -668,7 +760,7 @@ __device__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, unsig
     st_rel(P.batch_pub, S.ls.batch_w + 1u);
     S.ls.batch_w++;
     S.ls.sched_w += take;
-    PPTStats& st = *P.stats;
+    LeaderState& st = S.ls;
     st.msgs += take; st.batches++; st.batch_rows += total;
     if (upd) {
       if (st.log_n < P.update_log_cap) P.update_log[st.log_n] = d.n_upd;
@@ -685,7 +777,7 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
   d.sched_start = S.ls.sched_w; d.count = 0; d.dir = BWD; d.flags = flags; d.n_upd = 0; d.nrows = 0; d.pad0 = d.pad1 = 0;
   if ((flags & BATCH_TERMINATE) && S.ls.n_acc > 0 && !C.eval) {      // epoch-end flush of the leftover gradients
     d.flags |= BATCH_UPDATE; d.n_upd = S.ls.n_acc;
-    PPTStats& st = *P.stats;
+    LeaderState& st = S.ls;
     if (st.log_n < P.update_log_cap) P.update_log[st.log_n] = d.n_upd;
     st.log_n++; st.n_updates++; st.n_grads_applied += d.n_upd;
     S.ls.n_acc = 0; S.ls.version++;
@@ -699,16 +791,19 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
 // Asynchronous mode, warp 0 of the leader: whatever is pending, backward first (App. A).
 __device__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
   const int lane = threadIdx.x & 31;
-  for (int dir = BWD; dir >= FWD; dir--) {
-    Ring& R = P.ring[dir];
+  unsigned slot[2], mready[2];
+#pragma unroll
+  for (int dir = 0; dir < 2; dir++) {            // both rings are polled before either result is needed
     const unsigned t = S.ls.head[dir] + lane;
-    const unsigned slot = t & R.mask;
-    const bool ready = ld_acq(&R.seq[slot]) == t + 1u;
-    const unsigned m = __ballot_sync(0xffffffffu, ready);
+    slot[dir] = t & P.ring[dir].mask;
+    mready[dir] = (ld_acq(&P.ring[dir].seq[slot[dir]]) == t + 1u) ? 1u : 0u;
+  }
+  for (int dir = BWD; dir >= FWD; dir--) {
+    const unsigned m = __ballot_sync(0xffffffffu, mready[dir] != 0);
     int n = __ffs(~m) - 1;
     if (n < 0) n = 32;
     if (n == 0) continue;
-    int take = form_batch(C, P, S, dir, slot, n);
+    int take = form_batch(C, P, S, dir, slot[dir], n);
     if (lane == 0) S.ls.head[dir] += take;
     __syncwarp();
     return true;
@@ -784,6 +879,41 @@ __device__ void leader_schedule_round(const Ctx& C, DevPPT& P, TileShared& S, un
 // ------------------------------------------------------------------------------------------------
 // PPT tile main loop
 // ------------------------------------------------------------------------------------------------
+// Copy the cached input rows of a batch into shared memory with several loads in flight per thread.
+// rowptr[b] points at row b's `width` floats in device memory; V = 4, 2 or 1 floats per load.
+template <int V>
+__device__ __forceinline__ void stage_rows_v(float* __restrict__ Xs, const float* const* rowptr, int nb, int width) {
+  const int wv = width / V, total = nb * wv;
+  for (int base = threadIdx.x; base < total; base += THREADS * 4) {
+    float v[4][V];
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int idx = base + k * THREADS;
+      if (idx < total) {
+        const int b = idx / wv, c = idx - b * wv;
+        const float* src = rowptr[b] + c * V;
+        if (V == 4) { float4 t = __ldcg(reinterpret_cast<const float4*>(src)); v[k][0] = t.x; v[k][1] = t.y; v[k][2 % V] = t.z; v[k][3 % V] = t.w; }
+        else if (V == 2) { float2 t = __ldcg(reinterpret_cast<const float2*>(src)); v[k][0] = t.x; v[k][1 % V] = t.y; }
+        else v[k][0] = __ldcg(src);
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int idx = base + k * THREADS;
+      if (idx < total) {
+        const int b = idx / wv, c = idx - b * wv;
+#pragma unroll
+        for (int q = 0; q < V; q++) Xs[b * width + c * V + q] = v[k][q];
+      }
+    }
+  }
+}
+__device__ __forceinline__ void stage_rows(float* Xs, const float* const* rowptr, int nb, int width, int align_floats) {
+  if ((width & 3) == 0 && (align_floats & 3) == 0) stage_rows_v<4>(Xs, rowptr, nb, width);
+  else if ((width & 1) == 0 && (align_floats & 1) == 0) stage_rows_v<2>(Xs, rowptr, nb, width);
+  else stage_rows_v<1>(Xs, rowptr, nb, width);
+}
+
 struct TileMem {           // carve-up of the dynamic shared memory of a tile (floats)
   float *Ws, *As, *bs, *Abs, *Xs, *Ds, *Ys, *XC;
 };
@@ -822,9 +952,17 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
       for (int i = tid; i < R; i += THREADS) { M.bs[m * P.R + i] = P.b[m * out + r_begin + i]; M.Abs[m * P.R + i] = 0.f; }
     }
   }
-  if (tid == 0) { S.ls.head[0] = S.ls.head[1] = 0; S.ls.sched_w = S.ls.batch_w = 0; S.ls.n_acc = 0; S.ls.version = 0; S.max_stale = 0; }
+  if (tid == 0) {
+    S.ls.head[0] = S.ls.head[1] = 0; S.ls.sched_w = S.ls.batch_w = 0; S.ls.n_acc = 0; S.ls.version = 0; S.max_stale = 0;
+    S.ls.log_n = 0; S.ls.n_updates = S.ls.n_grads_applied = S.ls.msgs = S.ls.batches = S.ls.batch_rows = 0;
+  }
   if (tid < 64) S.stale_hist[tid] = 0;
+  if (tid < 8) S.phase[tid] = 0;
+  if (tid < POOL) S.pool.ready[tid] = 0;
+  if (tid == 0) { S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
   __syncthreads();
+#define AMP_PHASE(k) do { if (tid == 0) { long long now_ = clock64(); S.phase[k] += (unsigned long long)(now_ - tph); tph = now_; } } while (0)
+  long long tph = clock64();
 
   unsigned my_batch = 0, grid_gen = 0, node_gen = 0;
   WalkAcc acc = {0, 0};
@@ -840,6 +978,7 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
     bool round_open = true;
     while (round_open) {
       // ---- obtain the next batch ------------------------------------------------------------
+      AMP_PHASE(7);
       if (tid == 0) S.ok = 1;
       __syncthreads();
       if (tile == 0) {
@@ -865,6 +1004,7 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
       __syncthreads();
       const BatchDesc d = S.desc;
       my_batch++;
+      AMP_PHASE(d.count > 0 ? 1 : 0);
       const int count = d.count, dir = d.dir;
       // ---- headers, keys, row offsets ----------------------------------------------------------
       if (tid < count) {
@@ -891,14 +1031,17 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
       __syncthreads();
       if (!S.ok) { running = false; break; }
       const int nb = S.rowoff[count];
+      if (tid < nb && P.kind != LOOKUP) {
+        const int m = S.rowmsg[tid];
+        S.rowptr[tid] = msg_x(C, P, S.hdr[m], S.key[m]) + (size_t)(tid - S.rowoff[m]) * in;
+      }
+      __syncthreads();
       const bool eval = count > 0 && (S.hdr[0].flags & HDR_EVAL);
+      AMP_PHASE(2);
 
       if (count > 0 && P.kind == LINEAR) {
         // stage the cached inputs of the batch
-        for (int idx = tid; idx < nb * in; idx += THREADS) {
-          const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
-          M.Xs[idx] = __ldcg(msg_x(C, P, S.hdr[m], S.key[m]) + (size_t)(b - S.rowoff[m]) * in + c);
-        }
+        stage_rows(M.Xs, S.rowptr, nb, in, P.xcache ? in : C.inst.dense_dim);
         if (dir == FWD) {
           __syncthreads();
           AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.Xs, in, nb, M.Ws, in, R, in, M.Ys, P.R)));
@@ -930,10 +1073,7 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
         // x = [a; h]; the tile owns rows [r_begin, r_begin + R) of Wz, Wr, Wc (matrix m at Ws + m * P.R * in)
         const int H = out, SR = P.R, BR = P.BM * P.R;
         const float *Wz = M.Ws, *Wr = M.Ws + SR * in, *Wc = M.Ws + 2 * SR * in;
-        for (int idx = tid; idx < nb * in; idx += THREADS) {
-          const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
-          M.Xs[idx] = __ldcg(P.xcache + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * in + c);
-        }
+        stage_rows(M.Xs, S.rowptr, nb, in, in);
         __syncthreads();
         if (dir == FWD) {
           // phase 1: gates z, r for the tile's rows
@@ -1043,6 +1183,7 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
         }
       }
       __syncthreads();
+      AMP_PHASE(3);
       // ---- local update (Sec. 3): theta -= lr * A / n, accumulator cleared --------------------------
       if (d.flags & BATCH_UPDATE) {
         const float scale = C.lr / (float)d.n_upd;
@@ -1075,11 +1216,43 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
         }
         __syncthreads();
       }
+      AMP_PHASE(4);
       // ---- all tiles of the node done with the batch, then emit ------------------------------------
       if (count > 0) {
         __threadfence();
         if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
         else __syncthreads();
+        AMP_PHASE(5);
+        if (dir == BWD && P.kind != LOOKUP && !(P.flags & 1) && (P.T > 1 || P.kind == GRUCELL)) {
+          // Sum the tiles' partial input gradients (tile order) for the messages this tile emits; every thread keeps
+          // all T loads of an element in flight.
+          const size_t pstride = (size_t)P.BM * in;
+          const float* pa = P.dxpart + (size_t)(my_batch & 1) * P.T * pstride;
+          const float* pb = P.kind == GRUCELL ? P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride : nullptr;
+          const float* dirb = pb ? pb + (size_t)P.T * pstride : nullptr;
+          const int H = out;
+          for (int i = tile; i < count; i += P.T) {
+            const int ro = S.rowoff[i], ne = S.hdr[i].rows * in;
+            for (int k = tid; k < ne; k += THREADS) {
+              const size_t e = (size_t)ro * in + k;
+              const int c = k % in;
+              float v[MAX_TILES], w[MAX_TILES];
+#pragma unroll
+              for (int t = 0; t < MAX_TILES; t++) {
+                v[t] = t < P.T ? __ldcg(pa + (size_t)t * pstride + e) : 0.f;
+                w[t] = (pb && c < H && t < P.T) ? __ldcg(pb + (size_t)t * pstride + e) : 0.f;
+              }
+              float sum = 0.f;
+#pragma unroll
+              for (int t = 0; t < MAX_TILES; t++) { sum += v[t]; sum += w[t]; }
+              if (pb && c >= H) sum += __ldcg(dirb + (size_t)(ro + k / in) * H + (c - H));
+              P.stage[e] = sum;
+            }
+          }
+          __syncthreads();
+        }
+        if (tid == 0) S.pool.outstanding = tile < count ? (count - tile + P.T - 1) / P.T : 0;   // this tile's messages
+        __syncthreads();
         int mine = 0;
         for (int i = 0; i < count; i++) {
           if (i % P.T != tile) continue;
@@ -1087,7 +1260,7 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
           const Hdr& h = S.hdr[i];
           Frame f;
           f.iter = 0; f.inst = h.inst; f.seq = h.seq; f.slot = h.slot; f.it = h.it; f.u = h.u; f.port = h.port;
-          f.rows = h.rows; f.flags = h.flags;
+          f.rows = h.rows; f.flags = h.flags; f.nsum = 1; f.sstride = 0;
           if (dir == FWD) {
             f.node = N.succ_node[0]; f.aport = N.succ_port[0]; f.dir = FWD; f.dim = out; f.ld = out;
             f.p = P.kind == LOOKUP ? P.stage + (size_t)S.rowoff[i] * out
@@ -1097,39 +1270,17 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
             if (P.kind == LOOKUP || (P.flags & 1)) { f.p = nullptr; f.dim = 0; f.rows = 1; }
             else {
               float* dx = P.stage + (size_t)S.rowoff[i] * in;
-              if (P.kind == GRUCELL) {
-                const int H = out;
-                const size_t pstride = (size_t)P.BM * in, ro = (size_t)S.rowoff[i] * in;
-                const float* p1 = P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride + ro;
-                const float* p2 = P.dxpart + (size_t)(my_batch & 1) * P.T * pstride + ro;
-                const float* dirb = P.part2 + ((size_t)(my_batch & 1) * (P.T + 1) + P.T) * pstride + (size_t)S.rowoff[i] * H;
-                for (int k = lane; k < h.rows * in; k += 32) {
-                  const int rr = k / in, c = k - rr * in;
-                  float s = 0.f;
-                  for (int t = 0; t < P.T; t++) {
-                    s += __ldcg(p2 + (size_t)t * pstride + k);
-                    if (c < H) s += __ldcg(p1 + (size_t)t * pstride + k);
-                  }
-                  if (c >= H) s += __ldcg(dirb + (size_t)rr * H + (c - H));
-                  dx[k] = s;
-                }
-                __syncwarp();
-              } else if (P.T > 1) {                           // reduce the tiles' partial input gradients, tile order
-                const float* part = P.dxpart + (size_t)(my_batch & 1) * P.T * P.BM * in + (size_t)S.rowoff[i] * in;
-                for (int k = lane; k < h.rows * in; k += 32) {
-                  float s = 0.f;
-                  for (int t = 0; t < P.T; t++) s += __ldcg(part + (size_t)t * P.BM * in + k);
-                  dx[k] = s;
-                }
-                __syncwarp();
-              }
               f.p = dx;
             }
           }
-          walk(C, f, S.stack[warp], acc);
+          walk(C, f, S.stack[warp], acc, &S.pool);
+          __syncwarp();
+          if (lane == 0) atomicSub(&S.pool.outstanding, 1);
         }
+        pool_steal(C, &S.pool, S.stack[warp], acc);
         flush_acc(C, acc, lane);
         __syncthreads();
+        AMP_PHASE(6);
       }
       if (d.flags & BATCH_TERMINATE) { running = false; round_open = false; }
       if (d.flags & BATCH_END_ROUND) round_open = false;
@@ -1147,7 +1298,12 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
     }
   if (tile == 0) {
     if (tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
-    if (tid == 0) P.stats->max_staleness = S.max_stale;
+    if (tid == 0) {
+      PPTStats& st = *P.stats;
+      st.max_staleness = S.max_stale; st.log_n = S.ls.log_n; st.n_updates = S.ls.n_updates;
+      st.n_grads_applied = S.ls.n_grads_applied; st.msgs = S.ls.msgs; st.batches = S.ls.batches; st.batch_rows = S.ls.batch_rows;
+    }
+    if (tid < 8) P.stats->phase_cycles[tid] = S.phase[tid];
   }
 }
 
@@ -1162,12 +1318,14 @@ struct CtrlShared {
   int admit_slot, admit_inst, admit_seq, n_src_msgs;
   int src_count[4], src_base[5];
   Frame stack[WARPS][WALK_STACK];
+  WalkPool pool;
 };
 
 __device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const DevInst& I = C.inst;
-  if (tid == 0) { S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; }
+  if (tid == 0) { S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
+  if (tid < POOL) S.pool.ready[tid] = 0;
   __syncthreads();
   unsigned grid_gen = 0;
   WalkAcc acc = {0, 0};
@@ -1262,6 +1420,8 @@ __device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long
       __syncthreads();
       // pump the source messages (Sec. 4: tokens / leaves / graph nodes, initial hidden state, dense row)
       const int inst = S.admit_inst;
+      if (tid == 0) S.pool.outstanding = S.n_src_msgs;
+      __syncthreads();
       for (int mi = warp; mi < S.n_src_msgs; mi += WARPS) {
         int s = 0;
         while (mi >= S.src_base[s + 1]) s++;
@@ -1270,7 +1430,7 @@ __device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long
         Frame f;
         f.node = sn.succ_node[0]; f.aport = sn.succ_port[0]; f.dir = FWD; f.iter = 0;
         f.inst = inst; f.seq = S.admit_seq; f.slot = slot; f.it = 0; f.u = 0; f.port = 0; f.rows = 1;
-        f.flags = C.eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr;
+        f.flags = C.eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr; f.nsum = 1; f.sstride = 0;
         switch (sn.fn) {
           case 1: f.p = I.dense + (long long)inst * I.dense_dim; f.dim = I.dense_dim; f.ld = I.dense_dim; break;
           case 2: f.u = k; break;
@@ -1278,8 +1438,11 @@ __device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long
           case 4: f.u = I.leaf_ids[I.leaf_off[inst] + k]; break;
           case 5: f.rows = (int)(I.offsets[inst + 1] - I.offsets[inst]); break;
         }
-        walk(C, f, S.stack[warp], acc);
+        walk(C, f, S.stack[warp], acc, &S.pool);
+        __syncwarp();
+        if (lane == 0) atomicSub(&S.pool.outstanding, 1);
       }
+      pool_steal(C, &S.pool, S.stack[warp], acc);
       flush_acc(C, acc, lane);
       __syncthreads();
     }

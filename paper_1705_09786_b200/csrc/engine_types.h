@@ -8,6 +8,7 @@ constexpr int MAX_PORTS = 8;
 constexpr int THREADS = 256;          // threads per CTA
 constexpr int WARPS = THREADS / 32;
 constexpr int MAX_BATCH_MSGS = 32;    // messages per micro-batch (one warp schedules them)
+constexpr int MAX_TILES = 16;        // row tiles per PPT node
 constexpr int WALK_STACK = 12;        // continuation frames per walking warp
 
 enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, CONCAT, SPLIT,
@@ -33,6 +34,7 @@ struct PPTStats {
   unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
   unsigned long long stale_hist[64];
   int max_staleness, log_n;
+  unsigned long long phase_cycles[8];   // leader tile: idle, fetch, headers, compute, update, barrier, emit
 };
 
 struct DevNode {
