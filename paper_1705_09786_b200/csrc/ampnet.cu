@@ -368,8 +368,10 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
     if (rows_max > 64) return set_err(g, AMPNET_EINVAL, "node %d: %d payload rows per message exceed the supported 64", P.node, rows_max);
     P.J = P.kind == LOOKUP ? 4 : j_bucket(P.in);
     if (P.kind == LOOKUP) { P.T = 1; P.R = 0; P.BM = BM; P.smem_floats = tile_smem_floats(P, 0, BM); used += 1; continue; }
-    int T = 1 + (int)std::floor((double)P.nmat * P.in * P.out / total_w * avail);
-    T = std::max(1, std::min({T, max_tiles, std::max(1, P.out / 4)}));
+    // small nodes (a classifier) still emit one message per gradient: give them tiles for the emission work
+    const double share = std::max((double)P.nmat * P.in * P.out / total_w, 0.1);
+    int T = 1 + (int)std::floor(share * avail);
+    T = std::max(1, std::min({T, max_tiles, P.out <= 16 ? P.out : std::max(1, P.out / 4)}));
     for (;;) {
       int R = (P.out + T - 1) / T;
       int bm = BM;
@@ -450,6 +452,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.sched = B.take<unsigned>(2 * (size_t)cap); P.sched_mask = 2 * cap - 1;
     P.batches = B.take<BatchDesc>(2 * (size_t)cap); P.batch_mask = 2 * cap - 1;
     P.batch_pub = C.take<unsigned>(1);
+    P.bhdr = B.take<Hdr>((size_t)BATCH_BLOCKS * MAX_BATCH_MSGS);
     P.sortbuf = B.take<unsigned long long>(cap);
     if ((P.T > 1 && H.kind != LOOKUP) || H.kind == GRUCELL) P.dxpart = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
     P.stage = B.take<float>((size_t)P.BM * std::max(P.in_dim, P.out_dim));
@@ -478,8 +481,8 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
         else n.jbuf = B.take<float>(kout * n.jstride);
       } break;
       case GROUP:
+        n.jld = n.in_dim;
         n.jstride = (long long)n.rows_out * n.in_dim;
-        n.jbuf = B.take<float>(kout * n.jstride);
         n.jcnt = C.take<int>(kout); track(n.jcnt, kout * sizeof(int));
         break;
       case UNGROUP:
@@ -514,6 +517,16 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
       default: break;
     }
   }
+  // GROUP buffers come second: a Group that feeds an edge-wise Concat assembles its rows inside the Concat's buffer
+  for (size_t i = 0; i < R.nodes.size(); i++) {
+    DevNode& n = R.nodes[i];
+    if (n.type != GROUP) continue;
+    const size_t kout = (size_t)mak * IT * n.U_out;
+    const DevNode& s = R.nodes[n.succ_node[0]];
+    if (s.type == CONCAT && s.fn == 1 && s.U_out == n.U_out && s.rows_in == n.rows_out && s.in_dim == n.in_dim && s.jbuf) {
+      n.jbuf = s.jbuf + (size_t)n.succ_port[0] * s.in_dim; n.jld = s.out_dim; n.jstride = s.jstride; n.jalias = 1;
+    } else n.jbuf = B.take<float>(kout * n.jstride);
+  }
   Ctx& X = R.ctx;
   X.n_nodes = (int)R.nodes.size(); X.n_ppts = (int)R.ppts.size(); X.n_ctas = n_ctas;
   X.nodes = B.take<DevNode>(R.nodes.size());
@@ -538,6 +551,8 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   X.retire_mask = rcap - 1;
   X.order = nullptr; X.n_order = n_order;
   X.loss_out = B.take<float>((size_t)std::max<long long>(D.n, 1));
+  X.wide = 0;
+  for (auto& hn : g->hnodes) if (hn.type == UNGROUP || hn.type == GROUP) X.wide = 1;
   X.mak = mak; X.muf = cfg ? cfg->min_update_frequency : 1; X.det = det; X.eval = eval; X.IT = IT;
   X.lr = cfg ? cfg->lr : 0.f;
   double to = cfg && cfg->timeout_s > 0 ? cfg->timeout_s : 120.0;
@@ -578,8 +593,10 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
       if (order[i] < 0 || order[i] >= D.n) return set_err(g, AMPNET_EINVAL, "order[%lld] = %lld is not an instance", i, (long long)order[i]);
   }
   if (det && n_order >= (1ll << 24)) return set_err(g, AMPNET_EINVAL, "the deterministic schedule supports fewer than 2^24 instances per epoch");
+  const bool dbg = getenv("AMPNET_DEBUG") != nullptr;
   CUDA_TRY(g, cudaSetDevice(g->device));
   RunPlan R;
+  if (dbg) fprintf(stderr, "[ampnet] planning\n");
   ampnet_status_t st = plan_run(g, split, mak, det, eval, cfg, n_order, true, R);
   if (st != AMPNET_OK) return st;
   const size_t order_bytes = order ? (size_t)n_order * sizeof(long long) : 0;
@@ -604,6 +621,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   CUDA_TRY(g, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ampnet_engine, THREADS, R.smem_bytes));
   if (per_sm < 1 || (long long)per_sm * g->n_sms < R.ctx.n_ctas)
     return set_err(g, AMPNET_EINVAL, "%d CTAs cannot be co-resident (%d per SM)", R.ctx.n_ctas, per_sm);
+  if (dbg) fprintf(stderr, "[ampnet] launching %d CTAs, %zu B smem, ctl %zu B, bulk %zu B\n", R.ctx.n_ctas, R.smem_bytes, g->ctl.used, g->bulk.used);
   void* args[] = {&R.ctx};
   CUDA_TRY(g, cudaEventRecord(g->ev0, g->stream));
   CUDA_TRY(g, cudaLaunchCooperativeKernel((void*)ampnet_engine, dim3(R.ctx.n_ctas), dim3(THREADS), args, R.smem_bytes, g->stream));
@@ -617,7 +635,9 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   CUDA_TRY(g, cudaMemcpyAsync(g->last_node_msgs.data(), g->d_node_msgs, g->last_node_msgs.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost, g->stream));
   if (per_instance_loss)
     CUDA_TRY(g, cudaMemcpyAsync(per_instance_loss, R.ctx.loss_out, (size_t)D.n * sizeof(float), cudaMemcpyDeviceToHost, g->stream));
+  if (dbg) fprintf(stderr, "[ampnet] launched, waiting\n");
   CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  if (dbg) fprintf(stderr, "[ampnet] done\n");
   g->have_run = true;
   g->n_keylog = det ? G.n_keylog : 0;
   float ms = 0;

@@ -35,6 +35,14 @@ __device__ __forceinline__ void fail(const Ctx& C, int code, int node, int detai
   st_rel(&C.g->abort_flag, 1u);
 }
 __device__ __forceinline__ bool aborted(const Ctx& C) { return ld_acq(&C.g->abort_flag) != 0; }
+// Warp-uniform reads: one lane reads, all lanes take its value, so that a value changing under the warp can never
+// send lanes of one warp down different paths around a warp-synchronous primitive.
+__device__ __forceinline__ unsigned warp_uniform(unsigned v) { return __shfl_sync(0xffffffffu, v, 0); }
+__device__ __forceinline__ bool aborted_warp(const Ctx& C) {
+  unsigned v = 0;
+  if ((threadIdx.x & 31) == 0) v = *(volatile unsigned*)&C.g->abort_flag;
+  return warp_uniform(v) != 0;
+}
 
 // Every wait in the kernel goes through this: it gives up when another CTA has raised the abort word or
 // when the run's time budget is spent (status AMPNET_ETIMEOUT), so no wait can hang the GPU.
@@ -91,6 +99,8 @@ struct Frame {
   int inst, seq, slot, it, u, port, rows, flags;
   int dim, ld;
   int nsum, sstride;    // payload element (r, i) = sum over j < nsum of p[j * sstride + r * ld + i]
+  int part, nparts;     // nparts > 1: the rows of the first row-wise fork are shared among nparts CTAs; this walker takes
+                        // rows j = part (mod nparts); until that fork only part 0 has side effects (the others are shadows)
   const float* p;       // payload rows (device memory); nullptr = zeros
 };
 
@@ -110,21 +120,53 @@ __device__ __forceinline__ float ld_payload(const float* p, int nsum, int sstrid
   for (int j = 1; j < nsum; j++) s += __ldcg(p + (size_t)j * sstride + off);     // addend order
   return s;
 }
-// Copy payload rows into a cache; a lazy sum is evaluated on the way.  Four elements per lane in flight.
-__device__ __forceinline__ void warp_copy(float* dst, int dld, const Frame& f, int rows, int dim, int lane) {
+// Copy payload rows into a cache; a lazy sum is evaluated on the way.  The rows are flattened so that every lane keeps
+// four (vector) loads in flight whatever the row length.
+template <int V>
+__device__ __forceinline__ void warp_copy_v(float* dst, int dld, const Frame& f, int rows, int dim, int lane) {
   const float* src = f.p;
-  for (int r = 0; r < rows; r++) {
-    float* d = dst + (size_t)r * dld;
-    if (!src) { for (int i = lane; i < dim; i += 32) d[i] = 0.f; continue; }
-    const size_t ro = (size_t)r * f.ld;
-    for (int i0 = lane; i0 < dim; i0 += 128) {
-      float v[4];
+  const int wv = dim / V, total = rows * wv;
+  for (int base = lane; base < total; base += 128) {
+    float v[4][V];
 #pragma unroll
-      for (int k = 0; k < 4; k++) { const int i = i0 + 32 * k; v[k] = i < dim ? ld_payload(src, f.nsum, f.sstride, ro + i) : 0.f; }
+    for (int k = 0; k < 4; k++) {
+      const int idx = base + 32 * k;
+      if (idx < total) {
+        const int r = idx / wv, c = idx - r * wv;
+        const size_t off = (size_t)r * f.ld + (size_t)c * V;
 #pragma unroll
-      for (int k = 0; k < 4; k++) { const int i = i0 + 32 * k; if (i < dim) d[i] = v[k]; }
+        for (int q = 0; q < V; q++) v[k][q] = 0.f;
+        for (int j = 0; j < f.nsum; j++) {                       // addend order
+          const float* a = src + (size_t)j * f.sstride + off;
+          if (V == 4) { const float4 t = __ldcg(reinterpret_cast<const float4*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; v[k][2 % V] += t.z; v[k][3 % V] += t.w; }
+          else if (V == 2) { const float2 t = __ldcg(reinterpret_cast<const float2*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; }
+          else v[k][0] += __ldcg(a);
+        }
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+      const int idx = base + 32 * k;
+      if (idx < total) {
+        const int r = idx / wv, c = idx - r * wv;
+        float* d = dst + (size_t)r * dld + (size_t)c * V;
+        if (V == 4) *reinterpret_cast<float4*>(d) = make_float4(v[k][0], v[k][1 % V], v[k][2 % V], v[k][3 % V]);
+        else if (V == 2) *reinterpret_cast<float2*>(d) = make_float2(v[k][0], v[k][1 % V]);
+        else d[0] = v[k][0];
+      }
     }
   }
+}
+__device__ __noinline__ void warp_copy(float* dst, int dld, const Frame& f, int rows, int dim, int lane) {
+  if (!f.p) {
+    for (int r = 0; r < rows; r++) for (int i = lane; i < dim; i += 32) dst[(size_t)r * dld + i] = 0.f;
+    return;
+  }
+  const unsigned long long al = (unsigned long long)dst | (unsigned long long)f.p;
+  const int geo = dim | dld | (rows > 1 ? f.ld : 0) | (f.nsum > 1 ? f.sstride : 0);
+  if (((geo & 3) == 0) && ((al & 15) == 0)) warp_copy_v<4>(dst, dld, f, rows, dim, lane);
+  else if (((geo & 1) == 0) && ((al & 7) == 0)) warp_copy_v<2>(dst, dld, f, rows, dim, lane);
+  else warp_copy_v<1>(dst, dld, f, rows, dim, lane);
 }
 
 __device__ __forceinline__ void ring_push(Ring& r, const Frame& f) {   // one lane; the release store orders the payload
@@ -195,19 +237,34 @@ __device__ __forceinline__ void to_pred(Frame& f, const DevNode& n, int j) {
   f.node = n.pred_node[j]; f.aport = n.pred_port[j]; f.dir = BWD; f.iter = 0;
 }
 
-__device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool* Q) {
+__device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool* Q) {
   const int lane = threadIdx.x & 31;
   const DevInst& I = C.inst;
   int sp = 0;
   bool have = true;
+  int steps = 0;
   while (have) {
     if (f.node < 0) { fail(C, ST_OVERFLOW, -2, 0); return; }
+    // self-checks: no endless walk, no absurd fork width, stop early once the run is being aborted
+    if (++steps > (1 << 20) || (unsigned)f.nsum > 64u || (unsigned)f.rows > 4096u || (unsigned)f.nparts > 64u) {
+      fail(C, ST_OVERFLOW, -3, f.node * 100000 + (f.rows & 0xffff));
+      return;
+    }
+    if ((steps & 7) == 0 && aborted_warp(C)) return;
     const DevNode& n = C.nodes[f.node];
     bool cont = false;                       // true: f was rewritten and continues
-    if (n.type == SOURCE) {                  // a source message came home to the controller
+    const bool shadow = f.nparts > 1 && f.part > 0;
+    const bool dies_as_shadow = shadow && (n.type == LINEAR || n.type == LOOKUP || n.type == GRUCELL || n.type == LOSS_CE ||
+                                           n.type == LOSS_MSE || n.type == SINK || n.type == SOURCE || n.type == NPT_SUMROWS ||
+                                           (n.type == BCAST && f.dir == BWD) || (n.type == CONCAT && f.dir == FWD) ||
+                                           (n.type == GROUP && f.dir == FWD) || (n.type == UNGROUP && f.dir == BWD) ||
+                                           (n.type == FLATMAP && f.dir == BWD));
+    if (dies_as_shadow) {
+      // a shadow reached a node with side effects before any row-wise fork: the real walker handles it
+    } else if (n.type == SOURCE) {           // a source message came home to the controller
       if (f.dir == BWD && lane == 0) retire_push(C, f.slot);
     } else {
-      if (f.iter == 0) {
+      if (f.iter == 0 && !shadow) {
         acc.msgs++;
         unsigned long long a = (unsigned long long)f.node | ((unsigned long long)f.dir << 16) |
                                ((unsigned long long)(f.aport & 0xff) << 20) | ((unsigned long long)(f.port & 0xff) << 28);
@@ -283,16 +340,20 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool
           long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
           if (key < 0) return;
           if (f.dir == FWD) {
-            if (lane == 0 && !(f.flags & HDR_EVAL)) n.origin[key] = (unsigned char)(f.aport + 1);
+            if (lane == 0 && !(f.flags & HDR_EVAL) && !shadow) n.origin[key] = (unsigned char)(f.aport + 1);
             to_succ(f, n, 0);
+            cont = true;
           } else {
             int j = (int)*(volatile unsigned char*)&n.origin[key] - 1;
-            if (j < 0 || j >= n.n_pred) { fail(C, ST_OVERFLOW, f.node, j); return; }
-            __syncwarp();
-            if (lane == 0) n.origin[key] = 0;
-            to_pred(f, n, j);
+            if (shadow) { if (j >= 0 && j < n.n_pred) { to_pred(f, n, j); cont = true; } }   // the real walker may have cleared it
+            else {
+              if (j < 0 || j >= n.n_pred) { fail(C, ST_OVERFLOW, f.node, j); return; }
+              __syncwarp();
+              if (lane == 0) n.origin[key] = 0;
+              to_pred(f, n, j);
+              cont = true;
+            }
           }
-          cont = true;
         } break;
         case ISU:
           if (f.dir == FWD) {
@@ -337,7 +398,7 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool
             if (key < 0) return;
             if ((unsigned)port >= (unsigned)n.fn_arg || f.rows > n.rows_in) { fail(C, ST_OVERFLOW, f.node, port); return; }
             float* base = n.jbuf + key * n.jstride;
-            warp_copy(base + port * n.in_dim, n.out_dim, f, f.rows, n.in_dim, lane);
+            if (f.p != base + port * n.in_dim || f.nsum != 1) warp_copy(base + port * n.in_dim, n.out_dim, f, f.rows, n.in_dim, lane);
             if (join_arrive(&n.jcnt[key], n.fn_arg, lane)) {
               f.p = base; f.nsum = 1; f.dim = n.out_dim; f.ld = n.out_dim; f.port = 0;
               to_succ(f, n, 0);
@@ -366,17 +427,19 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool
             if (key < 0) return;
             if (member >= n.rows_out || count > n.rows_out) { fail(C, ST_OVERFLOW, f.node, member); return; }
             float* base = n.jbuf + key * n.jstride;
-            warp_copy(base + (size_t)member * n.in_dim, n.in_dim, f, 1, n.in_dim, lane);
+            warp_copy(base + (size_t)member * n.jld, n.jld, f, 1, n.in_dim, lane);
             if (join_arrive(&n.jcnt[key], count, lane)) {
-              f.u = gkey; f.rows = count; f.p = base; f.nsum = 1; f.ld = n.in_dim; f.dim = n.in_dim;
+              f.u = gkey; f.rows = count; f.p = base; f.nsum = 1; f.ld = n.jld; f.dim = n.in_dim;
               to_succ(f, n, 0);
               cont = true;
             }
           } else {
-            int i = f.iter;
-            if (i + 1 < f.rows) { Frame c = f; c.iter = i + 1;
+            const int i = f.iter * f.nparts + f.part;       // this walker's share of the rows
+            if (i >= f.rows) break;
+            if (i + f.nparts < f.rows) { Frame c = f; c.iter = f.iter + 1;
               if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
+            f.nparts = 1; f.part = 0;
             const long long ebase = I.edge_off ? I.edge_off[f.inst] : 0;
             int mu;
             if (n.fn == 1) mu = I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i];
@@ -390,10 +453,12 @@ __device__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool
           break;
         case UNGROUP:
           if (f.dir == FWD) {
-            int i = f.iter;
-            if (i + 1 < f.rows) { Frame c = f; c.iter = i + 1;
+            const int i = f.iter * f.nparts + f.part;       // this walker's share of the rows
+            if (i >= f.rows) break;
+            if (i + f.nparts < f.rows) { Frame c = f; c.iter = f.iter + 1;
               if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
+            f.nparts = 1; f.part = 0;
             int mu = n.fn == 2 ? I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i] : i;
             f.p = f.p ? f.p + (size_t)i * f.ld : nullptr; f.rows = 1; f.u = mu;
             to_succ(f, n, 0);
@@ -490,7 +555,7 @@ __device__ __forceinline__ void flush_acc(const Ctx& C, WalkAcc& a, int lane) {
 }
 
 // A warp that has walked its own frames helps with what the others offered, until nothing is outstanding.
-__device__ void pool_steal(const Ctx& C, WalkPool* Q, Frame* stack, WalkAcc& acc) {
+__device__ __noinline__ void pool_steal(const Ctx& C, WalkPool* Q, Frame* stack, WalkAcc& acc) {
   const int lane = threadIdx.x & 31;
   unsigned idle = 0;
   for (;;) {
@@ -509,6 +574,11 @@ __device__ void pool_steal(const Ctx& C, WalkPool* Q, Frame* stack, WalkAcc& acc
     got = __shfl_sync(0xffffffffu, got, 0);
     if (got) {
       h = __shfl_sync(0xffffffffu, h, 0);
+      if (aborted_warp(C)) {                                // the run is being aborted: drain without walking
+        __syncwarp();
+        if (lane == 0) { *(volatile unsigned*)&Q->ready[h % POOL] = 0u; atomicSub(&Q->outstanding, 1); }
+        continue;
+      }
       const unsigned idx = h % POOL;
       if (lane == 0) { int spins = 0; while (*(volatile unsigned*)&Q->ready[idx] != h + 1u && ++spins < (1 << 20)) {} }
       __syncwarp();
@@ -520,8 +590,13 @@ __device__ void pool_steal(const Ctx& C, WalkPool* Q, Frame* stack, WalkAcc& acc
       if (lane == 0) atomicSub(&Q->outstanding, 1);
       idle = 0;
     } else {
-      if (*(volatile int*)&Q->outstanding <= 0) break;
-      if ((++idle & 1023u) == 0 && aborted(C)) break;
+      int left = 0;
+      if (lane == 0) left = *(volatile int*)&Q->outstanding;
+      if ((int)warp_uniform((unsigned)left) <= 0) break;
+      if ((++idle & 1023u) == 0) {
+        if (aborted_warp(C)) break;
+        if (idle > (1u << 26)) { fail(C, ST_TIMEOUT, -4, 0); break; }
+      }
       __nanosleep(20);
     }
   }
@@ -550,7 +625,7 @@ __device__ __forceinline__ float act_grad(int a, float y) {
 // out[b][r] = sum_i X[b][i] * W[r][i]  for b < nb, r < R.  4 batch rows x 4 weight rows per warp pass; the 16
 // lane-partial sums are reduced across the warp with a halving butterfly (16 shuffles instead of 80).
 template <int J>
-__device__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const float* __restrict__ Ws, int ldw, int R,
+__device__ __noinline__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const float* __restrict__ Ws, int ldw, int R,
                          int in_dim, float* __restrict__ out, int ldo) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nbg = (nb + 3) >> 2, nrg = (R + 3) >> 2;
@@ -595,7 +670,7 @@ __device__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const fl
 
 // dx[b][i] = sum_r D[b][r] * W[r][i], written to dst (device memory, ld = in_dim).
 template <int J, bool ACCUM = false>
-__device__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Ws, int ldw, int R,
+__device__ __noinline__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Ws, int ldw, int R,
                         int in_dim, float* __restrict__ dst) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int b0 = warp * 4; b0 < nb; b0 += WARPS * 4) {
@@ -631,7 +706,7 @@ __device__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const flo
 }
 
 // A[r][i] += sum_b D[b][r] * X[b][i];  work unit = 4 weight rows x 4 column chunks.
-__device__ void tile_accum(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Xs, int ldx,
+__device__ __noinline__ void tile_accum(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Xs, int ldx,
                            float* __restrict__ As, int lda, int R, int in_dim) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int nj = (in_dim + 31) >> 5, ncg = (nj + 3) >> 2, nrg = (R + 3) >> 2;
@@ -709,7 +784,7 @@ __device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) {
 // Warp 0 of the leader tile: take up to 32 candidate messages (ring slot per lane, in processing order), cut
 // the batch at the row capacity and at the message that triggers an update (Sec. 3), publish it.
 // Returns the number of messages taken.
-__device__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, unsigned slot, int ncand) {
+__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, unsigned slot, int ncand) {
   const int lane = threadIdx.x & 31;
   Ring& R = P.ring[dir];
   Hdr h = {0, 0, 0, 0, 0, 0, 0, 0};
@@ -737,6 +812,11 @@ __device__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, unsig
   const int total = __shfl_sync(0xffffffffu, cum, take - 1);
   if (lane < take) {
     P.sched[(S.ls.sched_w + lane) & P.sched_mask] = slot;
+    if (!C.det) {
+      int4* b = reinterpret_cast<int4*>(&P.bhdr[(S.ls.batch_w & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + lane]);
+      b[0] = make_int4(h.inst, h.seq, h.slot, h.it);
+      b[1] = make_int4(h.u, h.port, h.rows, h.flags);
+    }
     if (!eval0) {
       long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
       if (key >= 0) {
@@ -789,7 +869,7 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
 }
 
 // Asynchronous mode, warp 0 of the leader: whatever is pending, backward first (App. A).
-__device__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
+__device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
   const int lane = threadIdx.x & 31;
   unsigned slot[2], mready[2];
 #pragma unroll
@@ -808,7 +888,9 @@ __device__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
     __syncwarp();
     return true;
   }
-  if (ld_acq(&C.g->done)) {
+  unsigned fin = 0;
+  if (lane == 0) fin = ld_acq(&C.g->done);
+  if (warp_uniform(fin)) {
     if (lane == 0) publish_marker(C, P, S, BATCH_TERMINATE);
     __syncwarp();
     return true;
@@ -818,7 +900,7 @@ __device__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
 
 // Deterministic mode, whole leader CTA: this round's inbox = tickets [head, tail) of each ring, sorted by
 // (admission seq, it, u, port), backward ring first; cut into batches; then the end-of-round marker.
-__device__ void leader_schedule_round(const Ctx& C, DevPPT& P, TileShared& S, unsigned long long t0) {
+__device__ __noinline__ void leader_schedule_round(const Ctx& C, DevPPT& P, TileShared& S, unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (ld_acq(&C.g->done)) {
     if (tid == 0) publish_marker(C, P, S, BATCH_TERMINATE);
@@ -908,7 +990,7 @@ __device__ __forceinline__ void stage_rows_v(float* __restrict__ Xs, const float
     }
   }
 }
-__device__ __forceinline__ void stage_rows(float* Xs, const float* const* rowptr, int nb, int width, int align_floats) {
+__device__ __noinline__ void stage_rows(float* Xs, const float* const* rowptr, int nb, int width, int align_floats) {
   if ((width & 3) == 0 && (align_floats & 3) == 0) stage_rows_v<4>(Xs, rowptr, nb, width);
   else if ((width & 1) == 0 && (align_floats & 1) == 0) stage_rows_v<2>(Xs, rowptr, nb, width);
   else stage_rows_v<1>(Xs, rowptr, nb, width);
@@ -923,7 +1005,7 @@ __device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, con
   return C.inst.dense + (long long)h.inst * C.inst.dense_dim;         // fed directly by a dense-row source
 }
 
-__device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileShared& S,
+__device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileShared& S,
                          const unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const DevNode& N = C.nodes[P.node];
@@ -984,12 +1066,17 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
       if (tile == 0) {
         if (warp == 0) {
           unsigned it = 0;
-          while (S.ls.batch_w == my_batch) {
+          for (;;) {
+            unsigned bw = 0;
+            if (lane == 0) bw = S.ls.batch_w;
+            if (warp_uniform(bw) != my_batch) break;
             if (C.det) { if (lane == 0) { fail(C, ST_OVERFLOW, P.node, -7); S.ok = 0; } break; }
             if (leader_try_schedule(C, P, S)) break;
             if ((++it & 15u) == 0) {
-              if (aborted(C)) { if (lane == 0) S.ok = 0; break; }
-              if (gtime() - t0 > C.timeout_ns) { if (lane == 0) { fail(C, ST_TIMEOUT, P.node, 1); S.ok = 0; } break; }
+              if (aborted_warp(C)) { if (lane == 0) S.ok = 0; break; }
+              unsigned late = 0;
+              if (lane == 0) late = gtime() - t0 > C.timeout_ns;
+              if (warp_uniform(late)) { if (lane == 0) { fail(C, ST_TIMEOUT, P.node, 1); S.ok = 0; } break; }
             }
             __nanosleep(it < 16 ? 20 : 200);
           }
@@ -1008,8 +1095,9 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
       const int count = d.count, dir = d.dir;
       // ---- headers, keys, row offsets ----------------------------------------------------------
       if (tid < count) {
-        const unsigned slot = P.sched[(d.sched_start + tid) & P.sched_mask];
-        const int4* e = reinterpret_cast<const int4*>(&P.ring[dir].e[slot]);
+        const unsigned slot = C.det ? P.sched[(d.sched_start + tid) & P.sched_mask] : 0u;
+        const int4* e = C.det ? reinterpret_cast<const int4*>(&P.ring[dir].e[slot])
+                              : reinterpret_cast<const int4*>(&P.bhdr[((my_batch - 1u) & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + tid]);
         int4 a = __ldcg(e), b = __ldcg(e + 1);
         Hdr h; h.inst = a.x; h.seq = a.y; h.slot = a.z; h.it = a.w; h.u = b.x; h.port = b.y; h.rows = b.z; h.flags = b.w;
         if (h.rows <= 0) h.rows = 1;
@@ -1223,19 +1311,28 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
         if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
         else __syncthreads();
         AMP_PHASE(5);
+        if (tile == 0 && warp == 0 && !C.det) {                         // look ahead: form the next batch now
+          unsigned bw = 0;
+          if (lane == 0) bw = S.ls.batch_w;
+          if (warp_uniform(bw) == my_batch) leader_try_schedule(C, P, S);
+        }
+        const bool split = C.wide && P.T > 1;          // share row-wise forks among the node's tiles
         if (dir == BWD && P.kind != LOOKUP && !(P.flags & 1) && (P.T > 1 || P.kind == GRUCELL)) {
-          // Sum the tiles' partial input gradients (tile order) for the messages this tile emits; every thread keeps
+          // Sum the tiles' partial input gradients (tile order) for the rows this tile emits; every thread keeps
           // all T loads of an element in flight.
           const size_t pstride = (size_t)P.BM * in;
           const float* pa = P.dxpart + (size_t)(my_batch & 1) * P.T * pstride;
           const float* pb = P.kind == GRUCELL ? P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride : nullptr;
           const float* dirb = pb ? pb + (size_t)P.T * pstride : nullptr;
           const int H = out;
-          for (int i = tile; i < count; i += P.T) {
+          for (int i = split ? 0 : tile; i < count; i += split ? 1 : P.T) {
+            const int part = (tile - i % P.T + P.T) % P.T;
             const int ro = S.rowoff[i], ne = S.hdr[i].rows * in;
             for (int k = tid; k < ne; k += THREADS) {
+              const int row = k / in;
+              if (part != 0 && row % P.T != part) continue;
               const size_t e = (size_t)ro * in + k;
-              const int c = k % in;
+              const int c = k - row * in;
               float v[MAX_TILES], w[MAX_TILES];
 #pragma unroll
               for (int t = 0; t < MAX_TILES; t++) {
@@ -1245,22 +1342,24 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
               float sum = 0.f;
 #pragma unroll
               for (int t = 0; t < MAX_TILES; t++) { sum += v[t]; sum += w[t]; }
-              if (pb && c >= H) sum += __ldcg(dirb + (size_t)(ro + k / in) * H + (c - H));
+              if (pb && c >= H) sum += __ldcg(dirb + (size_t)(ro + row) * H + (c - H));
               P.stage[e] = sum;
             }
           }
           __syncthreads();
         }
-        if (tid == 0) S.pool.outstanding = tile < count ? (count - tile + P.T - 1) / P.T : 0;   // this tile's messages
+        if (tid == 0) S.pool.outstanding = split ? count : (tile < count ? (count - tile + P.T - 1) / P.T : 0);
         __syncthreads();
         int mine = 0;
         for (int i = 0; i < count; i++) {
-          if (i % P.T != tile) continue;
+          const int part = (tile - i % P.T + P.T) % P.T;
+          if (!split && part != 0) continue;
           if ((mine++ % WARPS) != warp) continue;
           const Hdr& h = S.hdr[i];
           Frame f;
           f.iter = 0; f.inst = h.inst; f.seq = h.seq; f.slot = h.slot; f.it = h.it; f.u = h.u; f.port = h.port;
           f.rows = h.rows; f.flags = h.flags; f.nsum = 1; f.sstride = 0;
+          f.part = split ? part : 0; f.nparts = split ? P.T : 1;
           if (dir == FWD) {
             f.node = N.succ_node[0]; f.aport = N.succ_port[0]; f.dir = FWD; f.dim = out; f.ld = out;
             f.p = P.kind == LOOKUP ? P.stage + (size_t)S.rowoff[i] * out
@@ -1268,10 +1367,7 @@ __device__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, T
           } else {
             f.node = N.pred_node[0]; f.aport = N.pred_port[0]; f.dir = BWD; f.dim = in; f.ld = in;
             if (P.kind == LOOKUP || (P.flags & 1)) { f.p = nullptr; f.dim = 0; f.rows = 1; }
-            else {
-              float* dx = P.stage + (size_t)S.rowoff[i] * in;
-              f.p = dx;
-            }
+            else f.p = P.stage + (size_t)S.rowoff[i] * in;
           }
           walk(C, f, S.stack[warp], acc, &S.pool);
           __syncwarp();
@@ -1321,7 +1417,7 @@ struct CtrlShared {
   WalkPool pool;
 };
 
-__device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long long t0) {
+__device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const DevInst& I = C.inst;
   if (tid == 0) { S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
@@ -1335,9 +1431,11 @@ __device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long
     // ---- retirements ------------------------------------------------------------------------------
     if (warp == 0) {
       for (;;) {
-        const unsigned h = S.retire_head;
+        unsigned h = 0, ready = 0;
+        if (lane == 0) { h = S.retire_head; ready = ld_acq(&C.retire_seq[h & C.retire_mask]) == h + 1u; }
+        h = warp_uniform(h);
+        if (!warp_uniform(ready)) break;
         const unsigned s = h & C.retire_mask;
-        if (ld_acq(&C.retire_seq[s]) != h + 1u) break;
         const int slot = (int)__ldcg(&C.retire_e[s]);
         __syncwarp();
         int left = 0;
@@ -1430,7 +1528,7 @@ __device__ void controller_main(const Ctx& C, CtrlShared& S, const unsigned long
         Frame f;
         f.node = sn.succ_node[0]; f.aport = sn.succ_port[0]; f.dir = FWD; f.iter = 0;
         f.inst = inst; f.seq = S.admit_seq; f.slot = slot; f.it = 0; f.u = 0; f.port = 0; f.rows = 1;
-        f.flags = C.eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr; f.nsum = 1; f.sstride = 0;
+        f.flags = C.eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr; f.nsum = 1; f.sstride = 0; f.part = 0; f.nparts = 1;
         switch (sn.fn) {
           case 1: f.p = I.dense + (long long)inst * I.dense_dim; f.dim = I.dense_dim; f.ld = I.dense_dim; break;
           case 2: f.u = k; break;

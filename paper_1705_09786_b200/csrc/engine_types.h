@@ -8,6 +8,7 @@ constexpr int MAX_PORTS = 8;
 constexpr int THREADS = 256;          // threads per CTA
 constexpr int WARPS = THREADS / 32;
 constexpr int MAX_BATCH_MSGS = 32;    // messages per micro-batch (one warp schedules them)
+constexpr int BATCH_BLOCKS = 8;      // header blocks travelling with batch descriptors (asynchronous mode)
 constexpr int MAX_TILES = 16;        // row tiles per PPT node
 constexpr int WALK_STACK = 12;        // continuation frames per walking warp
 
@@ -51,8 +52,9 @@ struct DevNode {
   int* rowcnt;            // NPT_SUMROWS: cached row count per key
   float* lossval;         // LOSS: loss per key
   int* predok;            // LOSS_CE: 1 if the arg-max equals the label
-  int jalias;             // CONCAT: jbuf is the input cache of the succeeding PPT node
-  int pad;
+  int jalias;             // CONCAT: jbuf is the input cache of the succeeding PPT node; GROUP: jbuf lies inside the
+                          // buffer of the succeeding CONCAT
+  int jld;                // GROUP: row stride of the assembled rows
 };
 
 struct DevPPT {
@@ -68,6 +70,7 @@ struct DevPPT {
   Ring ring[2];
   unsigned* sched; unsigned sched_mask;
   BatchDesc* batches; unsigned batch_mask; unsigned* batch_pub;
+  Hdr* bhdr;                          // [BATCH_BLOCKS][MAX_BATCH_MSGS] headers of the most recent batches
   unsigned long long* sortbuf;
   float* dxpart;                      // [2][T][BM][in_dim] partial input gradients of the row tiles
   float* stage;                       // [BM][max(in_dim, out_dim)] reduced input gradients / gathered rows
@@ -131,6 +134,7 @@ struct Ctx {
   float* loss_out;
   // configuration
   int mak, muf, det, eval, IT;
+  int wide;                           // the graph has row-wise forks (Ungroup / Group)
   float lr;
   unsigned long long timeout_ns;
 };
