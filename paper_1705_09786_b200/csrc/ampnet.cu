@@ -294,6 +294,8 @@ ampnet_status_t create_params(ampnet_graph* g, uint64_t seed) {
     g->ppts.push_back(P);
   }
   if (g->ppts.empty()) return set_err(g, AMPNET_EINVAL, "the graph has no parameterised node");
+  if ((int)g->hnodes.size() > MAX_SMEM_NODES || (int)g->ppts.size() > MAX_SMEM_PPTS)
+    return set_err(g, AMPNET_EINVAL, "the IR graph is too large: at most %d nodes and %d parameterised nodes", MAX_SMEM_NODES, MAX_SMEM_PPTS);
   return AMPNET_OK;
 }
 
@@ -353,7 +355,10 @@ size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
 // Placement: row tiles per PPT node.  Enough tiles that a tile's weights + accumulators + staging fit in
 // shared memory, then the remaining CTAs in proportion to the nodes' multiply-add volume.
 ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles) {
-  const size_t budget = ((size_t)g->max_smem - 12 * 1024) / sizeof(float);
+  cudaFuncAttributes fa{};
+  size_t static_smem = 40 * 1024;
+  if (cudaFuncGetAttributes(&fa, ampnet_engine) == cudaSuccess) static_smem = fa.sharedSizeBytes;
+  const size_t budget = ((size_t)g->max_smem - static_smem - 1024) / sizeof(float);
   int max_tiles = 16;
   if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, std::min(MAX_TILES, atoi(e)));
   double total_w = 0;
@@ -553,6 +558,9 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   X.loss_out = B.take<float>((size_t)std::max<long long>(D.n, 1));
   X.wide = 0;
   for (auto& hn : g->hnodes) if (hn.type == UNGROUP || hn.type == GROUP) X.wide = 1;
+  X.tune = 0;
+  if (const char* e = getenv("AMPNET_TUNE")) X.tune = atoi(e);
+  if (X.tune & 1) X.wide = 0;
   X.mak = mak; X.muf = cfg ? cfg->min_update_frequency : 1; X.det = det; X.eval = eval; X.IT = IT;
   X.lr = cfg ? cfg->lr : 0.f;
   double to = cfg && cfg->timeout_s > 0 ? cfg->timeout_s : 120.0;
@@ -639,6 +647,11 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   CUDA_TRY(g, cudaStreamSynchronize(g->stream));
   if (dbg) fprintf(stderr, "[ampnet] done\n");
   g->have_run = true;
+  if (getenv("AMPNET_TUNE") && (atoi(getenv("AMPNET_TUNE")) & 8)) {
+    static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK"};
+    for (int t = 0; t < N_NODE_TYPES * 2; t++)
+      if (G.walk_steps[t]) fprintf(stderr, "[walk] %-8s %s steps %10llu cycles/step %8.0f\n", names[t / 2], t & 1 ? "BWD" : "FWD", G.walk_steps[t], (double)G.walk_cycles[t] / G.walk_steps[t]);
+  }
   g->n_keylog = det ? G.n_keylog : 0;
   float ms = 0;
   CUDA_TRY(g, cudaEventElapsedTime(&ms, g->ev0, g->ev1));

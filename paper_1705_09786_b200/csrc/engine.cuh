@@ -54,7 +54,7 @@ __device__ __forceinline__ bool spin_until(const Ctx& C, unsigned long long t0, 
       if (aborted(C)) return false;
       if (gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, -1, 0); return false; }
     }
-    __nanosleep(it < 64 ? 20 : 100);
+    if (it > 32) __nanosleep(it < 256 ? 20 : 100);
   }
   return true;
 }
@@ -91,6 +91,10 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
   return x ^ (x >> 31);
 }
 
+// Per-CTA copies of the node and PPT tables (read on every step of a walk): shared memory instead of device memory.
+__shared__ DevNode g_nodes[MAX_SMEM_NODES];
+__shared__ DevPPT g_ppts[MAX_SMEM_PPTS];
+
 // ------------------------------------------------------------------------------------------------
 // walking warp: executes the parameter-free nodes between two PPT nodes
 // ------------------------------------------------------------------------------------------------
@@ -123,8 +127,7 @@ __device__ __forceinline__ float ld_payload(const float* p, int nsum, int sstrid
 // Copy payload rows into a cache; a lazy sum is evaluated on the way.  The rows are flattened so that every lane keeps
 // four (vector) loads in flight whatever the row length.
 template <int V>
-__device__ __forceinline__ void warp_copy_v(float* dst, int dld, const Frame& f, int rows, int dim, int lane) {
-  const float* src = f.p;
+__device__ __forceinline__ void warp_copy_v(float* dst, int dld, const float* src, int sld, int nsum, int sstride, int rows, int dim, int lane) {
   const int wv = dim / V, total = rows * wv;
   for (int base = lane; base < total; base += 128) {
     float v[4][V];
@@ -133,11 +136,11 @@ __device__ __forceinline__ void warp_copy_v(float* dst, int dld, const Frame& f,
       const int idx = base + 32 * k;
       if (idx < total) {
         const int r = idx / wv, c = idx - r * wv;
-        const size_t off = (size_t)r * f.ld + (size_t)c * V;
+        const size_t off = (size_t)r * sld + (size_t)c * V;
 #pragma unroll
         for (int q = 0; q < V; q++) v[k][q] = 0.f;
-        for (int j = 0; j < f.nsum; j++) {                       // addend order
-          const float* a = src + (size_t)j * f.sstride + off;
+        for (int j = 0; j < nsum; j++) {                       // addend order
+          const float* a = src + (size_t)j * sstride + off;
           if (V == 4) { const float4 t = __ldcg(reinterpret_cast<const float4*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; v[k][2 % V] += t.z; v[k][3 % V] += t.w; }
           else if (V == 2) { const float2 t = __ldcg(reinterpret_cast<const float2*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; }
           else v[k][0] += __ldcg(a);
@@ -157,17 +160,20 @@ __device__ __forceinline__ void warp_copy_v(float* dst, int dld, const Frame& f,
     }
   }
 }
-__device__ __noinline__ void warp_copy(float* dst, int dld, const Frame& f, int rows, int dim, int lane) {
-  if (!f.p) {
+__device__ __noinline__ void warp_copy_p(float* dst, int dld, const float* src, int sld, int nsum, int sstride, int rows, int dim,
+                                          int lane) {
+  if (!src) {
     for (int r = 0; r < rows; r++) for (int i = lane; i < dim; i += 32) dst[(size_t)r * dld + i] = 0.f;
     return;
   }
-  const unsigned long long al = (unsigned long long)dst | (unsigned long long)f.p;
-  const int geo = dim | dld | (rows > 1 ? f.ld : 0) | (f.nsum > 1 ? f.sstride : 0);
-  if (((geo & 3) == 0) && ((al & 15) == 0)) warp_copy_v<4>(dst, dld, f, rows, dim, lane);
-  else if (((geo & 1) == 0) && ((al & 7) == 0)) warp_copy_v<2>(dst, dld, f, rows, dim, lane);
-  else warp_copy_v<1>(dst, dld, f, rows, dim, lane);
+  const unsigned long long al = (unsigned long long)dst | (unsigned long long)src;
+  const int geo = dim | dld | (rows > 1 ? sld : 0) | (nsum > 1 ? sstride : 0);
+  if (((geo & 3) == 0) && ((al & 15) == 0)) warp_copy_v<4>(dst, dld, src, sld, nsum, sstride, rows, dim, lane);
+  else if (((geo & 1) == 0) && ((al & 7) == 0)) warp_copy_v<2>(dst, dld, src, sld, nsum, sstride, rows, dim, lane);
+  else warp_copy_v<1>(dst, dld, src, sld, nsum, sstride, rows, dim, lane);
 }
+
+#define warp_copy(dst, dld, f, rows, dim, lane) warp_copy_p((dst), (dld), (f).p, (f).ld, (f).nsum, (f).sstride, (rows), (dim), (lane))
 
 __device__ __forceinline__ void ring_push(Ring& r, const Frame& f) {   // one lane; the release store orders the payload
   unsigned t = atomicAdd(r.tail, 1u);
@@ -237,6 +243,8 @@ __device__ __forceinline__ void to_pred(Frame& f, const DevNode& n, int j) {
   f.node = n.pred_node[j]; f.aport = n.pred_port[j]; f.dir = BWD; f.iter = 0;
 }
 
+// first position (token / tree node / graph node) of an instance
+#define IBASE(inst) (I.offsets ? I.offsets[(inst)] : 0)
 __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool* Q) {
   const int lane = threadIdx.x & 31;
   const DevInst& I = C.inst;
@@ -250,11 +258,13 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
       fail(C, ST_OVERFLOW, -3, f.node * 100000 + (f.rows & 0xffff));
       return;
     }
-    if ((steps & 7) == 0 && aborted_warp(C)) return;
-    const DevNode& n = C.nodes[f.node];
+    if ((steps & 63) == 0 && aborted_warp(C)) return;
+    const DevNode& n = g_nodes[f.node];
+    const long long tstep = (C.tune & 8) ? clock64() : 0;
+    const int ptype = n.type * 2 + f.dir;
     bool cont = false;                       // true: f was rewritten and continues
     const bool shadow = f.nparts > 1 && f.part > 0;
-    const bool dies_as_shadow = shadow && (n.type == LINEAR || n.type == LOOKUP || n.type == GRUCELL || n.type == LOSS_CE ||
+    const bool dies_as_shadow = shadow && !(n.type == COND || n.type == PHI || n.type == ISU) && (n.type == LINEAR || n.type == LOOKUP || n.type == GRUCELL || n.type == LOSS_CE ||
                                            n.type == LOSS_MSE || n.type == SINK || n.type == SOURCE || n.type == NPT_SUMROWS ||
                                            (n.type == BCAST && f.dir == BWD) || (n.type == CONCAT && f.dir == FWD) ||
                                            (n.type == GROUP && f.dir == FWD) || (n.type == UNGROUP && f.dir == BWD) ||
@@ -264,19 +274,18 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
     } else if (n.type == SOURCE) {           // a source message came home to the controller
       if (f.dir == BWD && lane == 0) retire_push(C, f.slot);
     } else {
-      if (f.iter == 0 && !shadow) {
-        acc.msgs++;
+      if (f.iter == 0 && !shadow) acc.msgs++;
+      if (f.iter == 0 && !shadow && (C.det || (C.tune & 16))) {
         unsigned long long a = (unsigned long long)f.node | ((unsigned long long)f.dir << 16) |
                                ((unsigned long long)(f.aport & 0xff) << 20) | ((unsigned long long)(f.port & 0xff) << 28);
         unsigned long long b = ((unsigned long long)(unsigned)f.inst << 32) | ((unsigned long long)(f.it & 0xff) << 24) |
                                (unsigned long long)(f.u & 0xffffff);
         acc.hash += mix64(mix64(a) ^ (b * 0x9E3779B97F4A7C15ull));
-        if (lane == 0) atomicAdd(&C.node_msgs[f.node * 2 + f.dir], 1ull);
+        if (lane == 0 && !(C.tune & 4)) atomicAdd(&C.node_msgs[f.node * 2 + f.dir], 1ull);
       }
-      const long long ibase = I.offsets ? I.offsets[f.inst] : 0;     // first position of the instance
       switch (n.type) {
         case LINEAR: case LOOKUP: case GRUCELL: {
-          DevPPT& P = C.ppts[n.ppt];
+          DevPPT& P = g_ppts[n.ppt];
           long long key = key_of(C, f.node, f.slot, f.it, f.u, P.U);
           if (key < 0) return;
           if (f.rows > P.rows_max) { fail(C, ST_OVERFLOW, f.node, f.rows); return; }
@@ -296,7 +305,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (key < 0) return;
           float* g = n.jbuf + key * n.jstride;
           if (n.type == LOSS_CE) {
-            int label = I.labels_i[I.labels_per_node ? ibase + f.u : f.inst];
+            int label = I.labels_i[I.labels_per_node ? IBASE(f.inst) + f.u : f.inst];
             float mx = -3.4e38f; int arg = 0x7fffffff;
             for (int j = lane; j < n.in_dim; j += 32) { float v = ld_payload(f.p, f.nsum, f.sstride, j); if (v > mx) { mx = v; arg = j; } }
             for (int o = 16; o; o >>= 1) {
@@ -326,7 +335,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (f.dir == FWD) {
             int k = 0;
             switch (n.fn) {
-              case 1: k = f.u < (int)(I.offsets[f.inst + 1] - ibase) ? 0 : 1; break;
+              case 1: k = f.u < (int)(I.offsets[f.inst + 1] - IBASE(f.inst)) ? 0 : 1; break;
               case 2: k = f.u == I.root[f.inst] ? 0 : 1; break;
               case 3: k = f.u; break;
               case 4: k = f.it < n.fn_arg ? 0 : 1; break;
@@ -358,12 +367,12 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
         case ISU:
           if (f.dir == FWD) {
             if (n.fn == 1) f.u += 1;
-            else if (n.fn == 2) { f.port = I.child_slot[ibase + f.u]; f.u = I.parent[ibase + f.u]; }
+            else if (n.fn == 2) { f.port = I.child_slot[IBASE(f.inst) + f.u]; f.u = I.parent[IBASE(f.inst) + f.u]; }
             else f.it += 1;
             to_succ(f, n, 0);
           } else {
             if (n.fn == 1) f.u -= 1;
-            else if (n.fn == 2) { f.u = f.port == 0 ? I.left[ibase + f.u] : I.right[ibase + f.u]; f.port = 0; }
+            else if (n.fn == 2) { f.u = f.port == 0 ? I.left[IBASE(f.inst) + f.u] : I.right[IBASE(f.inst) + f.u]; f.port = 0; }
             else f.it -= 1;
             to_pred(f, n, 0);
           }
@@ -421,8 +430,8 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             if (n.fn == 1) { int c = I.etype[ebase + f.u]; gkey = c; member = I.rank_type[ebase + f.u];
                              const long long* to = I.type_off + (long long)f.inst * I.NT + c; count = (int)(to[1] - to[0]); }
             else if (n.fn == 2) { int v = I.edst[ebase + f.u]; gkey = v; member = I.rank_in[ebase + f.u];
-                                  count = (int)(I.in_off[ibase + v + 1] - I.in_off[ibase + v]); }
-            else { gkey = 0; member = f.u; count = (int)(I.offsets[f.inst + 1] - ibase); }
+                                  count = (int)(I.in_off[IBASE(f.inst) + v + 1] - I.in_off[IBASE(f.inst) + v]); }
+            else { gkey = 0; member = f.u; count = (int)(I.offsets[f.inst + 1] - IBASE(f.inst)); }
             long long key = key_of(C, f.node, f.slot, f.it, gkey, n.U_out);
             if (key < 0) return;
             if (member >= n.rows_out || count > n.rows_out) { fail(C, ST_OVERFLOW, f.node, member); return; }
@@ -443,7 +452,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             const long long ebase = I.edge_off ? I.edge_off[f.inst] : 0;
             int mu;
             if (n.fn == 1) mu = I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i];
-            else if (n.fn == 2) mu = I.in_list[I.in_off[ibase + f.u] + i];
+            else if (n.fn == 2) mu = I.in_list[I.in_off[IBASE(f.inst) + f.u] + i];
             else mu = i;
             (void)ebase;
             f.p = f.p ? f.p + (size_t)i * f.ld : nullptr; f.rows = 1; f.u = mu;
@@ -467,7 +476,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             int gkey, row, expected;
             if (n.fn == 2) { const long long ebase = I.edge_off[f.inst]; gkey = I.etype[ebase + f.u]; row = I.rank_type[ebase + f.u];
                              const long long* to = I.type_off + (long long)f.inst * I.NT + gkey; expected = (int)(to[1] - to[0]); }
-            else { gkey = 0; row = f.u; expected = (int)(I.offsets[f.inst + 1] - ibase); }
+            else { gkey = 0; row = f.u; expected = (int)(I.offsets[f.inst + 1] - IBASE(f.inst)); }
             long long key = key_of(C, f.node, f.slot, f.it, gkey, n.U_in);
             if (key < 0) return;
             if (row >= n.rows_in) { fail(C, ST_OVERFLOW, f.node, row); return; }
@@ -482,7 +491,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           break;
         case FLATMAP: {
           if (f.dir == FWD) {
-            const long long* oo = I.out_off + ibase + f.u;
+            const long long* oo = I.out_off + IBASE(f.inst) + f.u;
             int deg = (int)(oo[1] - oo[0]);
             int i = f.iter;
             if (deg > 0) {
@@ -496,7 +505,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           } else {
             const long long ebase = I.edge_off[f.inst];
             int v = I.esrc[ebase + f.u], member = I.rank_out[ebase + f.u];
-            int deg = (int)(I.out_off[ibase + v + 1] - I.out_off[ibase + v]);
+            int deg = (int)(I.out_off[IBASE(f.inst) + v + 1] - I.out_off[IBASE(f.inst) + v]);
             long long key = key_of(C, f.node, f.slot, f.it, v, n.U_in);
             if (key < 0) return;
             const int maxdeg = (int)(n.jstride / n.in_dim) - 1;
@@ -539,6 +548,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           return;
       }
     }
+    if ((C.tune & 8) && lane == 0) { atomicAdd(&C.g->walk_cycles[ptype], (unsigned long long)(clock64() - tstep)); atomicAdd(&C.g->walk_steps[ptype], 1ull); }
     if (!cont) {
       if (sp > 0) { __syncwarp(); f = stack[--sp]; __syncwarp(); }
       else have = false;
@@ -574,11 +584,6 @@ __device__ __noinline__ void pool_steal(const Ctx& C, WalkPool* Q, Frame* stack,
     got = __shfl_sync(0xffffffffu, got, 0);
     if (got) {
       h = __shfl_sync(0xffffffffu, h, 0);
-      if (aborted_warp(C)) {                                // the run is being aborted: drain without walking
-        __syncwarp();
-        if (lane == 0) { *(volatile unsigned*)&Q->ready[h % POOL] = 0u; atomicSub(&Q->outstanding, 1); }
-        continue;
-      }
       const unsigned idx = h % POOL;
       if (lane == 0) { int spins = 0; while (*(volatile unsigned*)&Q->ready[idx] != h + 1u && ++spins < (1 << 20)) {} }
       __syncwarp();
@@ -1008,7 +1013,7 @@ __device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, con
 __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileShared& S,
                          const unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const DevNode& N = C.nodes[P.node];
+  const DevNode& N = g_nodes[P.node];
   const int in = P.in_dim, out = P.out_dim;
   const int r_begin = tile * P.R;
   const int R = P.kind == LOOKUP ? 0 : max(0, min(P.R, out - r_begin));
@@ -1087,43 +1092,54 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       }
       __syncthreads();
       if (!S.ok || aborted(C)) { running = false; break; }
-      if (tid == 0) S.desc = P.batches[my_batch & P.batch_mask];
+      // ---- descriptor, headers, keys, row offsets, row pointers: one warp, one block barrier --------------
+      if (warp == 0) {
+        const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]);
+        const int4 d0 = __ldcg(dp), d1 = __ldcg(dp + 1);          // same address in every lane
+        int4 ha = make_int4(0, 0, 0, 0), hb = make_int4(0, 0, 0, 0);
+        if (!C.det) {                                             // headers travel with the descriptor: load both at once
+          const int4* e = reinterpret_cast<const int4*>(&P.bhdr[(my_batch & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + lane]);
+          ha = __ldcg(e); hb = __ldcg(e + 1);
+        }
+        const int cnt = d0.y, ddir = d0.z;
+        if (C.det && lane < cnt) {
+          const unsigned slot = P.sched[((unsigned)d0.x + lane) & P.sched_mask];
+          const int4* e = reinterpret_cast<const int4*>(&P.ring[ddir].e[slot]);
+          ha = __ldcg(e); hb = __ldcg(e + 1);
+        }
+        Hdr h; h.inst = ha.x; h.seq = ha.y; h.slot = ha.z; h.it = ha.w; h.u = hb.x; h.port = hb.y; h.rows = hb.z; h.flags = hb.w;
+        if (h.rows <= 0) h.rows = 1;
+        const int rows = lane < cnt ? h.rows : 0;
+        int cum = rows;
+        for (int o = 1; o < 32; o <<= 1) { int v = __shfl_up_sync(0xffffffffu, cum, o); if (lane >= o) cum += v; }
+        const int total = __shfl_sync(0xffffffffu, cum, 31);
+        const int off = cum - rows;
+        long long key = 0;
+        if (lane < cnt) {
+          key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+          S.hdr[lane] = h; S.key[lane] = key; S.rowoff[lane] = off;
+          if (key >= 0 && total <= P.BM) {
+            const float* x0 = P.kind != LOOKUP ? msg_x(C, P, h, key) : nullptr;
+            for (int r = 0; r < rows; r++) { S.rowmsg[off + r] = lane; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
+          }
+        }
+        const unsigned bad = __ballot_sync(0xffffffffu, lane < cnt && key < 0);
+        if (lane == 0) {
+          S.rowoff[cnt] = total;
+          BatchDesc dd; dd.sched_start = (unsigned)d0.x; dd.count = d0.y; dd.dir = d0.z; dd.flags = d0.w;
+          dd.n_upd = d1.x; dd.nrows = d1.y; dd.pad0 = dd.pad1 = 0;
+          S.desc = dd;
+          if (bad) S.ok = 0;
+          if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; }
+        }
+      }
       __syncthreads();
       const BatchDesc d = S.desc;
       my_batch++;
       AMP_PHASE(d.count > 0 ? 1 : 0);
       const int count = d.count, dir = d.dir;
-      // ---- headers, keys, row offsets ----------------------------------------------------------
-      if (tid < count) {
-        const unsigned slot = C.det ? P.sched[(d.sched_start + tid) & P.sched_mask] : 0u;
-        const int4* e = C.det ? reinterpret_cast<const int4*>(&P.ring[dir].e[slot])
-                              : reinterpret_cast<const int4*>(&P.bhdr[((my_batch - 1u) & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + tid]);
-        int4 a = __ldcg(e), b = __ldcg(e + 1);
-        Hdr h; h.inst = a.x; h.seq = a.y; h.slot = a.z; h.it = a.w; h.u = b.x; h.port = b.y; h.rows = b.z; h.flags = b.w;
-        if (h.rows <= 0) h.rows = 1;
-        S.hdr[tid] = h;
-        S.key[tid] = key_of(C, P.node, h.slot, h.it, h.u, P.U);
-      }
-      __syncthreads();
-      if (tid == 0) {
-        int o = 0;
-        for (int i = 0; i < count; i++) {
-          S.rowoff[i] = o;
-          for (int r = 0; r < S.hdr[i].rows && o + r < 64; r++) S.rowmsg[o + r] = i;
-          o += S.hdr[i].rows;
-        }
-        S.rowoff[count] = o;
-        for (int i = 0; i < count; i++) if (S.key[i] < 0) S.ok = 0;
-        if (o > P.BM) { fail(C, ST_OVERFLOW, P.node, o); S.ok = 0; }
-      }
-      __syncthreads();
       if (!S.ok) { running = false; break; }
       const int nb = S.rowoff[count];
-      if (tid < nb && P.kind != LOOKUP) {
-        const int m = S.rowmsg[tid];
-        S.rowptr[tid] = msg_x(C, P, S.hdr[m], S.key[m]) + (size_t)(tid - S.rowoff[m]) * in;
-      }
-      __syncthreads();
       const bool eval = count > 0 && (S.hdr[0].flags & HDR_EVAL);
       AMP_PHASE(2);
 
@@ -1311,7 +1327,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
         else __syncthreads();
         AMP_PHASE(5);
-        if (tile == 0 && warp == 0 && !C.det) {                         // look ahead: form the next batch now
+        if (tile == 0 && warp == 0 && !C.det && !(C.tune & 2)) {       // look ahead: form the next batch now
           unsigned bw = 0;
           if (lane == 0) bw = S.ls.batch_w;
           if (warp_uniform(bw) == my_batch) leader_try_schedule(C, P, S);
@@ -1446,7 +1462,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
           const int inst = C.slot_inst[slot];
           double tot = 0.0; int okc = 0, np = 0;
           for (int li = 0; li < C.n_loss; li++) {
-            const DevNode& L = C.nodes[C.loss_nodes[li]];
+            const DevNode& L = g_nodes[C.loss_nodes[li]];
             const long long k0 = (long long)slot * C.IT * L.U_in, k1 = k0 + (long long)C.IT * L.U_in;
             double dpart = 0.0;   // lane partial over a strided subset, then a fixed-order warp sum
             for (long long k = k0 + lane; k < k1; k += 32) {
@@ -1483,7 +1499,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
           if (S.active > C.g->max_active) C.g->max_active = S.active;
           int total = 0;
           for (int s = 0; s < C.n_sources; s++) {
-            const DevNode& sn = C.nodes[C.src_nodes[s]];
+            const DevNode& sn = g_nodes[C.src_nodes[s]];
             int cnt = 1;
             if (sn.fn == 2) cnt = (int)(I.offsets[inst + 1] - I.offsets[inst]);
             else if (sn.fn == 4) cnt = (int)(I.leaf_off[inst + 1] - I.leaf_off[inst]);
@@ -1510,7 +1526,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
       if (slot < 0) break;
       // clear the slot's loss cells (predok = -1 marks "no loss evaluated at this key")
       for (int li = 0; li < C.n_loss; li++) {
-        const DevNode& L = C.nodes[C.loss_nodes[li]];
+        const DevNode& L = g_nodes[C.loss_nodes[li]];
         const long long k0 = (long long)slot * C.IT * L.U_in, cnt = (long long)C.IT * L.U_in;
         for (long long k = tid; k < cnt; k += THREADS) { L.lossval[k0 + k] = 0.f; L.predok[k0 + k] = -1; }
       }
@@ -1524,7 +1540,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
         int s = 0;
         while (mi >= S.src_base[s + 1]) s++;
         const int k = mi - S.src_base[s];
-        const DevNode& sn = C.nodes[C.src_nodes[s]];
+        const DevNode& sn = g_nodes[C.src_nodes[s]];
         Frame f;
         f.node = sn.succ_node[0]; f.aport = sn.succ_port[0]; f.dir = FWD; f.iter = 0;
         f.inst = inst; f.seq = S.admit_seq; f.slot = slot; f.it = 0; f.u = 0; f.port = 0; f.rows = 1;
@@ -1577,9 +1593,18 @@ __global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constan
   extern __shared__ __align__(16) float dyn_smem[];
   __shared__ SharedUnion SU;
   const unsigned long long t0 = gtime();
+  {
+    const int* src = reinterpret_cast<const int*>(C.nodes);
+    int* dst = reinterpret_cast<int*>(g_nodes);
+    for (int i = threadIdx.x; i < C.n_nodes * (int)(sizeof(DevNode) / 4); i += THREADS) dst[i] = src[i];
+    src = reinterpret_cast<const int*>(C.ppts);
+    dst = reinterpret_cast<int*>(g_ppts);
+    for (int i = threadIdx.x; i < C.n_ppts * (int)(sizeof(DevPPT) / 4); i += THREADS) dst[i] = src[i];
+  }
+  __syncthreads();
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);
-  else ppt_main(C, C.ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
+  else ppt_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
 }
 
 }  // namespace amp

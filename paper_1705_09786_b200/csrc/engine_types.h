@@ -9,6 +9,8 @@ constexpr int THREADS = 256;          // threads per CTA
 constexpr int WARPS = THREADS / 32;
 constexpr int MAX_BATCH_MSGS = 32;    // messages per micro-batch (one warp schedules them)
 constexpr int BATCH_BLOCKS = 8;      // header blocks travelling with batch descriptors (asynchronous mode)
+constexpr int MAX_SMEM_NODES = 40;    // IR nodes / PPT nodes whose tables are kept in shared memory
+constexpr int MAX_SMEM_PPTS = 16;
 constexpr int MAX_TILES = 16;        // row tiles per PPT node
 constexpr int WALK_STACK = 12;        // continuation frames per walking warp
 
@@ -113,6 +115,7 @@ struct Globals {                      // mutable run state in device memory (zer
   long long n_keylog;
   unsigned retire_tail;
   int err_node, err_detail;
+  unsigned long long walk_cycles[N_NODE_TYPES * 2], walk_steps[N_NODE_TYPES * 2];   // profiling (tune bit 8)
 };
 
 struct Role { int ppt, tile; };
@@ -135,6 +138,7 @@ struct Ctx {
   // configuration
   int mak, muf, det, eval, IT;
   int wide;                           // the graph has row-wise forks (Ungroup / Group)
+  int tune;                           // experiment switches (environment AMPNET_TUNE): 2 no look-ahead, 4 no per-node counters
   float lr;
   unsigned long long timeout_ns;
 };
