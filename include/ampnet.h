@@ -164,7 +164,9 @@ ampnet_status_t ampnet_param_count(ampnet_graph_t*, int32_t node, int32_t which,
 ampnet_status_t ampnet_get_params(ampnet_graph_t*, int32_t node, int32_t which, float* dst_host, int64_t n);
 ampnet_status_t ampnet_set_params(ampnet_graph_t*, int32_t node, int32_t which, const float* src_host, int64_t n);
 
-/* Statistics of the last run.  staleness_hist: 64 bins (updates between a gradient's forward and backward).  */
+/* Statistics of the last run.  staleness_hist: 64 bins (updates between a gradient's forward and backward).
+ * fwd_msgs / bwd_msgs (messages consumed by the node) and the route fingerprint are collected in the
+ * deterministic schedule only; the asynchronous schedule counts the total of node messages.                   */
 ampnet_status_t ampnet_get_node_stats(ampnet_graph_t*, int32_t node, int64_t* n_updates, int64_t* n_grads_applied,
                                       int64_t* staleness_hist, int64_t* fwd_msgs, int64_t* bwd_msgs);
 /* Gradient count of each update of a node, in order; returns the number of updates through *n.               */
@@ -180,8 +182,10 @@ ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_t
 
 /* Where the leader tile of a node spent its SM cycles in the last run: [0] waiting for messages, [1] fetching a
  * batch descriptor, [2] loading headers, [3] staging + arithmetic, [4] local updates, [5] barrier among the node's
- * tiles, [6] emission (walking the parameter-free nodes), [7] loop overhead.  batches: micro-batches executed.   */
-ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles8, int64_t* batches);
+ * tiles, [6] emission (walking the parameter-free nodes), [7] loop overhead; [8..15] detail of the emission phase
+ * ([8] look-ahead scheduling, [9] reduction of partial gradients, [10]/[12] own walks of warps 0/1, [11]/[13] helping
+ * other warps, [14] closing barrier).  cycles16: 16 values.  batches: micro-batches executed.                    */
+ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles16, int64_t* batches);
 
 const char* ampnet_last_error(const ampnet_graph_t*); /* library-owned string */
 

@@ -230,7 +230,7 @@ class Engine:
         return n.value
 
     def phase_cycles(self, node):
-        a = np.zeros(8, np.uint64)
+        a = np.zeros(16, np.uint64)
         b = C.c_int64()
         self._check(self.lib.ampnet_get_phase_cycles(self.h, node, _p(a), C.byref(b)))
         return a, b.value

@@ -1014,7 +1014,7 @@ ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t* g, int32_t node, uint64_
   if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
   if (node < 0 || node >= (int)g->hnodes.size() || g->hnodes[node].ppt < 0) return set_err(g, AMPNET_EINVAL, "not a parameterised node");
   const PPTStats& s = g->last_stats[g->hnodes[node].ppt];
-  if (cycles8) for (int k = 0; k < 8; k++) cycles8[k] = s.phase_cycles[k];
+  if (cycles8) for (int k = 0; k < 16; k++) cycles8[k] = s.phase_cycles[k];
   if (batches) *batches = (int64_t)s.batches;
   return AMPNET_OK;
 }

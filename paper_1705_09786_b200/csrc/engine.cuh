@@ -175,8 +175,9 @@ __device__ __noinline__ void warp_copy_p(float* dst, int dld, const float* src, 
 
 #define warp_copy(dst, dld, f, rows, dim, lane) warp_copy_p((dst), (dld), (f).p, (f).ld, (f).nsum, (f).sstride, (rows), (dim), (lane))
 
-__device__ __forceinline__ void ring_push(Ring& r, const Frame& f) {   // one lane; the release store orders the payload
-  unsigned t = atomicAdd(r.tail, 1u);
+// A producer takes its ticket before it copies the payload (the two round trips overlap) and publishes afterwards.
+__device__ __forceinline__ unsigned ring_ticket(Ring& r) { return atomicAdd(r.tail, 1u); }
+__device__ __forceinline__ void ring_publish(Ring& r, unsigned t, const Frame& f) {   // one lane; the release store orders the payload
   unsigned s = t & r.mask;
   int4* d = reinterpret_cast<int4*>(&r.e[s]);
   d[0] = make_int4(f.inst, f.seq, f.slot, f.it);
@@ -289,6 +290,8 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           long long key = key_of(C, f.node, f.slot, f.it, f.u, P.U);
           if (key < 0) return;
           if (f.rows > P.rows_max) { fail(C, ST_OVERFLOW, f.node, f.rows); return; }
+          unsigned ticket = 0;
+          if (lane == 0) ticket = ring_ticket(P.ring[f.dir]);
           if (f.dir == FWD) {
             if (P.xcache) {
               float* dst = P.xcache + key * (long long)P.rows_max * P.in_dim;
@@ -298,7 +301,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             warp_copy(P.gbuf + key * (long long)P.rows_max * P.out_dim, P.out_dim, f, f.rows, P.out_dim, lane);
           }
           __syncwarp();
-          if (lane == 0) ring_push(P.ring[f.dir], f);
+          if (lane == 0) ring_publish(P.ring[f.dir], ticket, f);
         } break;
         case LOSS_CE: case LOSS_MSE: {
           long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
@@ -777,7 +780,7 @@ struct TileShared {
   unsigned tail_snap[2];
   unsigned long long stale_hist[64];
   int max_stale;
-  unsigned long long phase[8];
+  unsigned long long phase[16];
   Frame stack[WARPS][WALK_STACK];
   WalkPool pool;
 };
@@ -1044,7 +1047,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
     S.ls.log_n = 0; S.ls.n_updates = S.ls.n_grads_applied = S.ls.msgs = S.ls.batches = S.ls.batch_rows = 0;
   }
   if (tid < 64) S.stale_hist[tid] = 0;
-  if (tid < 8) S.phase[tid] = 0;
+  if (tid < 16) S.phase[tid] = 0;
   if (tid < POOL) S.pool.ready[tid] = 0;
   if (tid == 0) { S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
   __syncthreads();
@@ -1330,7 +1333,9 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         if (tile == 0 && warp == 0 && !C.det && !(C.tune & 2)) {       // look ahead: form the next batch now
           unsigned bw = 0;
           if (lane == 0) bw = S.ls.batch_w;
+          const long long tq = clock64();
           if (warp_uniform(bw) == my_batch) leader_try_schedule(C, P, S);
+          if (lane == 0) S.phase[8] += (unsigned long long)(clock64() - tq);
         }
         const bool split = C.wide && P.T > 1;          // share row-wise forks among the node's tiles
         if (dir == BWD && P.kind != LOOKUP && !(P.flags & 1) && (P.T > 1 || P.kind == GRUCELL)) {
@@ -1366,6 +1371,8 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         }
         if (tid == 0) S.pool.outstanding = split ? count : (tile < count ? (count - tile + P.T - 1) / P.T : 0);
         __syncthreads();
+        const long long tw0 = clock64();
+        if (tid == 0) S.phase[9] += (unsigned long long)(tw0 - tph);       // look-ahead + reduction + barriers
         int mine = 0;
         for (int i = 0; i < count; i++) {
           const int part = (tile - i % P.T + P.T) % P.T;
@@ -1389,9 +1396,13 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           __syncwarp();
           if (lane == 0) atomicSub(&S.pool.outstanding, 1);
         }
+        const long long tw1 = clock64();
         pool_steal(C, &S.pool, S.stack[warp], acc);
+        const long long tw2 = clock64();
+        if (lane == 0 && warp < 2) { S.phase[10 + 2 * warp] += (unsigned long long)(tw1 - tw0); S.phase[11 + 2 * warp] += (unsigned long long)(tw2 - tw1); }
         flush_acc(C, acc, lane);
         __syncthreads();
+        if (tid == 0) S.phase[14] += (unsigned long long)(clock64() - tw2);
         AMP_PHASE(6);
       }
       if (d.flags & BATCH_TERMINATE) { running = false; round_open = false; }
@@ -1415,7 +1426,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       st.max_staleness = S.max_stale; st.log_n = S.ls.log_n; st.n_updates = S.ls.n_updates;
       st.n_grads_applied = S.ls.n_grads_applied; st.msgs = S.ls.msgs; st.batches = S.ls.batches; st.batch_rows = S.ls.batch_rows;
     }
-    if (tid < 8) P.stats->phase_cycles[tid] = S.phase[tid];
+    if (tid < 16) P.stats->phase_cycles[tid] = S.phase[tid];
   }
 }
 

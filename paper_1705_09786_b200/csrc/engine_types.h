@@ -37,7 +37,7 @@ struct PPTStats {
   unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
   unsigned long long stale_hist[64];
   int max_staleness, log_n;
-  unsigned long long phase_cycles[8];   // leader tile: idle, fetch, headers, compute, update, barrier, emit
+  unsigned long long phase_cycles[16];  // leader tile: idle, fetch, headers, compute, update, barrier, emit, loop; [8..] emission detail
 };
 
 struct DevNode {
