@@ -90,6 +90,25 @@ typedef struct {
   int32_t payload_dtype;           /* 0 = fp32 (the only one executed so far) */
 } ampnet_ir_desc_t;
 
+/* IR builders for the model families of Sec. 2 / Sec. 4: multi-layer perceptron (ReLU hidden layers, softmax-CE),
+ * variable-length RNN (Fig. 2: Lookup, Concat with the hidden state from Phi, Linear, Isu(t+1), Cond(end?), loop or
+ * Linear + Loss), binary tree RNN (leaf / branch cells joined by Phi, classifier at every node, children concatenated
+ * on the way up), gated graph neural network (Fig. 3a: per-edge-type Linear messages, GRU update, `steps` iterations,
+ * sum-pool read-out with MSE).  Host only; no device is touched.  The arrays are caller-allocated HOST memory of the
+ * given capacities; *n_nodes / *n_edges always return the sizes needed, AMPNET_EOVERFLOW says the capacity was too
+ * small (call with NULL arrays to size them).                                                                   */
+ampnet_status_t ampnet_ir_mlp(const int32_t* dims, int32_t n_dims, ampnet_node_desc_t* nodes, int32_t cap_nodes,
+                              int32_t* n_nodes, ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
+ampnet_status_t ampnet_ir_rnn(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes, int32_t act,
+                              ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                              ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
+ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
+                               ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                               ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
+ampnet_status_t ampnet_ir_ggnn(int32_t n_node_types, int32_t hidden, int32_t steps, int32_t n_edge_types, int32_t readout,
+                               ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                               ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
+
 /* Device-memory allocator supplied by the caller (for example a PyTorch caching allocator).  `alloc` returns a
  * device pointer aligned to 256 bytes or NULL; `free` releases it.  Both are called from the calling thread. */
 typedef void* (*ampnet_alloc_fn)(void* ctx, size_t bytes);

@@ -12,7 +12,8 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error", "ampnet_run_epoch_static", "ampnet_get_phase_cycles"]
+           "ampnet_last_error", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
+           "ampnet_ir_tree", "ampnet_ir_ggnn"]
 
 
 class AmpnetError(RuntimeError):
@@ -93,6 +94,12 @@ def load_library():
     lib.ampnet_leftover_cache_entries.argtypes = [P, C.POINTER(C.c_int64)]
     lib.ampnet_get_placement.argtypes = [P, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.ampnet_get_phase_cycles.argtypes = [P, C.c_int32, P, C.POINTER(C.c_int64)]
+    I32, PI = C.c_int32, C.POINTER(C.c_int32)
+    tail = [P, I32, PI, P, I32, PI]
+    lib.ampnet_ir_mlp.argtypes = [P, I32] + tail
+    lib.ampnet_ir_rnn.argtypes = [I32] * 5 + tail
+    lib.ampnet_ir_tree.argtypes = [I32] * 4 + tail
+    lib.ampnet_ir_ggnn.argtypes = [I32] * 5 + tail
     lib.ampnet_last_error.argtypes = [P]
     lib.ampnet_last_error.restype = C.c_char_p
     _LIB = lib
@@ -101,6 +108,30 @@ def load_library():
 
 def _p(a):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def ir_tables(family, *args):
+    """Node and edge tables (int32 [n,8] / [m,4]) of a canonical model family from the library's IR builders.
+    family: "mlp" (dims list), "rnn" (vocab, emb, hidden, classes, act), "tree" (vocab, emb, hidden, classes),
+    "ggnn" (n_node_types, hidden, steps, n_edge_types, readout)."""
+    lib = load_library()
+    nn, ne = C.c_int32(), C.c_int32()
+
+    def call(nodes, cn, edges, ce):
+        tail = (_p(nodes), cn, C.byref(nn), _p(edges), ce, C.byref(ne))
+        if family == "mlp":
+            dims = np.ascontiguousarray(args[0], dtype=np.int32)
+            return lib.ampnet_ir_mlp(_p(dims), len(dims), *tail)
+        return getattr(lib, "ampnet_ir_" + family)(*[int(a) for a in args], *tail)
+
+    rc = call(None, 0, None, 0)
+    if rc not in (0, 5):
+        raise AmpnetError(rc, f"ampnet_ir_{family} rejected its arguments")
+    nodes, edges = np.zeros((nn.value, 8), np.int32), np.zeros((ne.value, 4), np.int32)
+    rc = call(nodes, nn.value, edges, ne.value)
+    if rc != 0:
+        raise AmpnetError(rc, f"ampnet_ir_{family} failed")
+    return nodes, edges
 
 
 class Engine:

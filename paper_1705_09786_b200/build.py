@@ -4,7 +4,8 @@ import subprocess
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(_DIR, "csrc", "ampnet.cu")
-DEPS = [SRC, os.path.join(_DIR, "csrc", "engine.cuh"), os.path.join(_DIR, "csrc", "engine_types.h"),
+SRC_HOST = os.path.join(_DIR, "csrc", "ir_builders.cpp")
+DEPS = [SRC, SRC_HOST, os.path.join(_DIR, "csrc", "engine.cuh"), os.path.join(_DIR, "csrc", "engine_types.h"),
         os.path.join(os.path.dirname(_DIR), "include", "ampnet.h")]
 LIB = os.path.join(_DIR, "libampnet.so")
 
@@ -19,7 +20,7 @@ def build(force=False, verbose=False):
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-           "-Xcompiler", "-fPIC", "-shared", "-o", tmp, SRC]
+           "-Xcompiler", "-fPIC", "-shared", "-o", tmp, SRC, SRC_HOST]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)

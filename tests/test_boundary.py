@@ -78,3 +78,21 @@ def test_product_does_not_import_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 text = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in text.lower(), f"{f} mentions the oracle"
+
+
+def test_library_ir_builders_emit_the_canonical_graphs(lib):
+    """The host IR builders of the library and the tables of the shared input module describe the same graphs."""
+    import numpy as np
+    import paper_1705_09786_b200 as amp
+    from workloads import ir
+    cases = [("mlp", ([784, 256, 256, 10],), ir.mlp()), ("mlp", ([5, 3],), ir.mlp((5, 3))),
+             ("rnn", (14, 128, 128, 10, ir.ACT_TANH), ir.rnn()), ("tree", (20000, 300, 150, 5), ir.tree()),
+             ("ggnn", (15, 100, 4, 4, 100), ir.ggnn()), ("ggnn", (7, 8, 2, 3, 5), ir.ggnn(7, 8, 2, 3, 5))]
+    for family, args, want in cases:
+        nodes, edges = amp.ir_tables(family, *args)
+        np.testing.assert_array_equal(nodes, want.nodes)
+        np.testing.assert_array_equal(edges, want.edges)
+    with pytest.raises(amp.AmpnetError):
+        amp.ir_tables("rnn", 14, 64, 128, 10, ir.ACT_TANH)       # Concat ports need one common width
+    with pytest.raises(amp.AmpnetError):
+        amp.ir_tables("mlp", [784])
