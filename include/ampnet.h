@@ -87,7 +87,9 @@ typedef struct {
   int32_t n_nodes, n_edges;
   const ampnet_node_desc_t* nodes; /* host */
   const ampnet_edge_desc_t* edges; /* host */
-  int32_t payload_dtype;           /* 0 = fp32 (the only one executed so far) */
+  int32_t payload_dtype;           /* 0 = fp32 messages; 1 = bf16 messages: every emitted payload is rounded to bfloat16
+                                      (round to nearest even), weights, accumulators and cached-activation arithmetic
+                                      stay fp32                                                              */
 } ampnet_ir_desc_t;
 
 /* IR builders for the model families of Sec. 2 / Sec. 4: multi-layer perceptron (ReLU hidden layers, softmax-CE),

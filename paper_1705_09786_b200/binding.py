@@ -137,7 +137,7 @@ def ir_tables(family, *args):
 class Engine:
     """One IR graph on one GPU.  graph: an object with int32 tables `.nodes` [n,8] and `.edges` [m,4]."""
 
-    def __init__(self, graph, seed=1, device=0, use_torch_allocator=True):
+    def __init__(self, graph, seed=1, device=0, use_torch_allocator=True, payload_bf16=False):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("the AMPNet engine needs a CUDA device (no CPU fallback)")
@@ -165,7 +165,7 @@ class Engine:
             self._alloc_struct = Allocator(self._alloc_cb, self._free_cb, None)
         nodes = np.ascontiguousarray(graph.nodes, dtype=np.int32)
         edges = np.ascontiguousarray(graph.edges, dtype=np.int32)
-        ir = IRDesc(len(nodes), len(edges), _p(nodes), _p(edges), 0)
+        ir = IRDesc(len(nodes), len(edges), _p(nodes), _p(edges), 1 if payload_bf16 else 0)
         self.stream = torch.cuda.current_stream(self.device)
         h = C.c_void_p()
         rc = self.lib.ampnet_graph_create(C.byref(ir), seed, C.c_void_p(self.stream.cuda_stream),

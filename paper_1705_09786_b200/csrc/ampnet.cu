@@ -58,6 +58,7 @@ struct ampnet_graph {
   std::vector<HostPPT> ppts;
   std::vector<int> sources, losses;
   bool has_it = false; int it_steps = 0;
+  bool payload_bf16 = false;
   ampnet_allocator_t alloc{};
   cudaStream_t stream = nullptr;
   int device = 0, n_sms = 0, max_smem = 0;
@@ -359,7 +360,7 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   size_t static_smem = 40 * 1024;
   if (cudaFuncGetAttributes(&fa, ampnet_engine) == cudaSuccess) static_smem = fa.sharedSizeBytes;
   const size_t budget = ((size_t)g->max_smem - static_smem - 1024) / sizeof(float);
-  int max_tiles = 16;
+  int max_tiles = 16;      // default; a node whose tile does not fit in shared memory gets more, up to MAX_TILES
   if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, std::min(MAX_TILES, atoi(e)));
   double total_w = 0;
   for (auto& P : g->ppts) if (P.kind != LOOKUP) total_w += (double)P.nmat * P.in * P.out;
@@ -382,7 +383,7 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
       int bm = BM;
       while (tile_smem_floats(P, R, bm) > budget && bm > std::max(rows_max, 4)) bm = std::max(std::max(rows_max, 4), bm / 2);
       if (tile_smem_floats(P, R, bm) <= budget) { P.R = R; P.BM = bm; P.T = (P.out + R - 1) / R; break; }
-      if (R == 1) return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory even at one row per tile", P.node);
+      if (R == 1 || T >= MAX_TILES) return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory with %d row tiles", P.node, T);
       T = std::min(P.out, T + 1);
     }
     P.smem_floats = tile_smem_floats(P, P.R, P.BM);
@@ -447,7 +448,8 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     }
     P.vcache = B.take<int>(keys);
     const unsigned cap = pow2_at_least(2ull * keys);
-    if (cap > (1u << 20)) return set_err(g, AMPNET_EINVAL, "node %d: queue capacity %u above the supported 2^20 (lower max_active_keys)", H.node, cap);
+    if (cap > (det ? (1u << 20) : (1u << 23)))
+      return set_err(g, AMPNET_EINVAL, "node %d: queue capacity %u above the supported 2^%d (lower max_active_keys)", H.node, cap, det ? 20 : 23);
     for (int d = 0; d < 2; d++) {
       P.ring[d].e = B.take<Hdr>(cap);
       P.ring[d].seq = C.take<unsigned>(cap);
@@ -558,6 +560,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   X.loss_out = B.take<float>((size_t)std::max<long long>(D.n, 1));
   X.wide = 0;
   for (auto& hn : g->hnodes) if (hn.type == UNGROUP || hn.type == GROUP) X.wide = 1;
+  X.bf16 = g->payload_bf16 ? 1 : 0;
   X.tune = 0;
   if (const char* e = getenv("AMPNET_TUNE")) X.tune = atoi(e);
   if (X.tune & 1) X.wide = 0;
@@ -684,12 +687,13 @@ ampnet_status_t ampnet_graph_create(const ampnet_ir_desc_t* ir, uint64_t init_se
   if (!out) return AMPNET_EINVAL;
   *out = nullptr;
   if (!ir || !ir->nodes || ir->n_nodes < 1 || ir->n_edges < 0 || (ir->n_edges > 0 && !ir->edges)) return AMPNET_EINVAL;
-  if (ir->payload_dtype != 0) return AMPNET_EINVAL;
+  if (ir->payload_dtype != 0 && ir->payload_dtype != 1) return AMPNET_EINVAL;
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) return AMPNET_ECUDA;
   ampnet_graph* g = new ampnet_graph();
   g->nodes.assign(ir->nodes, ir->nodes + ir->n_nodes);
   if (ir->n_edges) g->edges.assign(ir->edges, ir->edges + ir->n_edges);
+  g->payload_bf16 = ir->payload_dtype == 1;
   if (allocator) g->alloc = *allocator;
   g->stream = (cudaStream_t)cuda_stream;
   ampnet_status_t st = AMPNET_OK;

@@ -8,6 +8,7 @@
 // Group, Ungroup, Flatmap, row sum, Loss, Sink) are executed by the warp that emits a message: it walks
 // the IR graph until the message lands in the input cache and queue of the next PPT node.
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include "engine_types.h"
 
@@ -94,6 +95,11 @@ __device__ __forceinline__ unsigned long long mix64(unsigned long long x) {
 // Per-CTA copies of the node and PPT tables (read on every step of a walk): shared memory instead of device memory.
 __shared__ DevNode g_nodes[MAX_SMEM_NODES];
 __shared__ DevPPT g_ppts[MAX_SMEM_PPTS];
+__shared__ int g_bf16;      // payloads are rounded to bfloat16 (round to nearest even) where they are emitted
+
+// What a node emits as a payload passes through here: identity for fp32 messages, bf16 rounding otherwise.
+// Weights, accumulators and the arithmetic on cached activations stay fp32.
+__device__ __forceinline__ float emit_round(float v) { return g_bf16 ? __bfloat162float(__float2bfloat16_rn(v)) : v; }
 
 // ------------------------------------------------------------------------------------------------
 // walking warp: executes the parameter-free nodes between two PPT nodes
@@ -122,7 +128,7 @@ struct WalkAcc { unsigned long long msgs, hash; };
 __device__ __forceinline__ float ld_payload(const float* p, int nsum, int sstride, size_t off) {
   float s = __ldcg(p + off);
   for (int j = 1; j < nsum; j++) s += __ldcg(p + (size_t)j * sstride + off);     // addend order
-  return s;
+  return nsum > 1 ? emit_round(s) : s;
 }
 // Copy payload rows into a cache; a lazy sum is evaluated on the way.  The rows are flattened so that every lane keeps
 // four (vector) loads in flight whatever the row length.
@@ -144,6 +150,10 @@ __device__ __forceinline__ void warp_copy_v(float* dst, int dld, const float* sr
           if (V == 4) { const float4 t = __ldcg(reinterpret_cast<const float4*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; v[k][2 % V] += t.z; v[k][3 % V] += t.w; }
           else if (V == 2) { const float2 t = __ldcg(reinterpret_cast<const float2*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; }
           else v[k][0] += __ldcg(a);
+        }
+        if (nsum > 1) {
+#pragma unroll
+          for (int q = 0; q < V; q++) v[k][q] = emit_round(v[k][q]);
         }
       }
     }
@@ -319,12 +329,12 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             for (int j = lane; j < n.in_dim; j += 32) s += expf(ld_payload(f.p, f.nsum, f.sstride, j) - mx);
             for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
             float lse = mx + logf(s);
-            for (int j = lane; j < n.in_dim; j += 32) g[j] = expf(ld_payload(f.p, f.nsum, f.sstride, j) - lse) - (j == label ? 1.f : 0.f);
+            for (int j = lane; j < n.in_dim; j += 32) g[j] = emit_round(expf(ld_payload(f.p, f.nsum, f.sstride, j) - lse) - (j == label ? 1.f : 0.f));
             if (lane == 0) { n.lossval[key] = lse - ld_payload(f.p, f.nsum, f.sstride, label); n.predok[key] = (arg == label) ? 1 : 0; }
           } else {
             if (lane == 0) {
               float d = ld_payload(f.p, f.nsum, f.sstride, 0) - I.labels_f[f.inst];
-              n.lossval[key] = d * d; g[0] = 2.f * d; n.predok[key] = 0;
+              n.lossval[key] = d * d; g[0] = emit_round(2.f * d); n.predok[key] = 0;
             }
           }
           if (f.flags & HDR_EVAL) { __syncwarp(); if (lane == 0) retire_push(C, f.slot); }
@@ -531,7 +541,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             for (int i = lane; i < n.in_dim; i += 32) {
               float s = 0.f;
               for (int r = 0; r < f.rows; r++) s += f.p ? ld_payload(f.p, f.nsum, f.sstride, (size_t)r * f.ld + i) : 0.f;   // row order
-              out[i] = s;
+              out[i] = emit_round(s);
             }
             if (lane == 0 && !(f.flags & HDR_EVAL)) n.rowcnt[key] = f.rows;
             __syncwarp();
@@ -1156,7 +1166,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
             const float y = act_fwd(P.act, M.Ys[b * P.R + r] + M.bs[r]);
-            P.ycache[(S.key[m] * P.rows_max + (b - S.rowoff[m])) * out + r_begin + r] = y;
+            P.ycache[(S.key[m] * P.rows_max + (b - S.rowoff[m])) * out + r_begin + r] = emit_round(y);
           }
         } else {
           for (int idx = tid; idx < nb * R; idx += THREADS) {
@@ -1214,7 +1224,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
             const float cnd = tanhf(M.Ys[2 * BR + b * SR + r] + M.bs[2 * SR + r]);
             const float z = M.Ys[b * SR + r];
             P.cc[o] = cnd;
-            P.ycache[o] = (1.f - z) * M.Xs[b * in + H + r_begin + r] + z * cnd;
+            P.ycache[o] = emit_round((1.f - z) * M.Xs[b * in + H + r_begin + r] + z * cnd);
           }
         } else {
           const size_t pstride = (size_t)P.BM * in;
@@ -1273,7 +1283,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
             const Hdr& h = S.hdr[m];
             const int pos = I.kind == 3 ? (b - S.rowoff[m]) : h.u;
             const int id = I.tokens[I.offsets[h.inst] + pos];
-            P.stage[idx] = ((unsigned)id < (unsigned)in) ? P.W[(size_t)id * out + c] : 0.f;
+            P.stage[idx] = ((unsigned)id < (unsigned)in) ? emit_round(P.W[(size_t)id * out + c]) : 0.f;
           }
         } else {
           for (int c = tid; c < out; c += THREADS)
@@ -1337,6 +1347,10 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           if (warp_uniform(bw) == my_batch) leader_try_schedule(C, P, S);
           if (lane == 0) S.phase[8] += (unsigned long long)(clock64() - tq);
         }
+        if (g_bf16 && dir == BWD && P.kind == LINEAR && P.T == 1 && !(P.flags & 1)) {
+          for (int idx = tid; idx < nb * in; idx += THREADS) P.stage[idx] = emit_round(P.stage[idx]);
+          __syncthreads();
+        }
         const bool split = C.wide && P.T > 1;          // share row-wise forks among the node's tiles
         if (dir == BWD && P.kind != LOOKUP && !(P.flags & 1) && (P.T > 1 || P.kind == GRUCELL)) {
           // Sum the tiles' partial input gradients (tile order) for the rows this tile emits; every thread keeps
@@ -1354,17 +1368,19 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
               if (part != 0 && row % P.T != part) continue;
               const size_t e = (size_t)ro * in + k;
               const int c = k - row * in;
-              float v[MAX_TILES], w[MAX_TILES];
-#pragma unroll
-              for (int t = 0; t < MAX_TILES; t++) {
-                v[t] = t < P.T ? __ldcg(pa + (size_t)t * pstride + e) : 0.f;
-                w[t] = (pb && c < H && t < P.T) ? __ldcg(pb + (size_t)t * pstride + e) : 0.f;
-              }
               float sum = 0.f;
+              for (int t0 = 0; t0 < P.T; t0 += 8) {          // eight tiles' partials in flight, added in tile order
+                float v[8], w[8];
 #pragma unroll
-              for (int t = 0; t < MAX_TILES; t++) { sum += v[t]; sum += w[t]; }
+                for (int t = 0; t < 8; t++) {
+                  v[t] = t0 + t < P.T ? __ldcg(pa + (size_t)(t0 + t) * pstride + e) : 0.f;
+                  w[t] = (pb && c < H && t0 + t < P.T) ? __ldcg(pb + (size_t)(t0 + t) * pstride + e) : 0.f;
+                }
+#pragma unroll
+                for (int t = 0; t < 8; t++) { sum += v[t]; sum += w[t]; }
+              }
               if (pb && c >= H) sum += __ldcg(dirb + (size_t)(ro + row) * H + (c - H));
-              P.stage[e] = sum;
+              P.stage[e] = emit_round(sum);
             }
           }
           __syncthreads();
@@ -1612,6 +1628,7 @@ __global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constan
     dst = reinterpret_cast<int*>(g_ppts);
     for (int i = threadIdx.x; i < C.n_ppts * (int)(sizeof(DevPPT) / 4); i += THREADS) dst[i] = src[i];
   }
+  if (threadIdx.x == 0) g_bf16 = C.bf16;
   __syncthreads();
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);

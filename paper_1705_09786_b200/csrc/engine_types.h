@@ -11,7 +11,7 @@ constexpr int MAX_BATCH_MSGS = 32;    // messages per micro-batch (one warp sche
 constexpr int BATCH_BLOCKS = 8;      // header blocks travelling with batch descriptors (asynchronous mode)
 constexpr int MAX_SMEM_NODES = 40;    // IR nodes / PPT nodes whose tables are kept in shared memory
 constexpr int MAX_SMEM_PPTS = 16;
-constexpr int MAX_TILES = 16;        // row tiles per PPT node
+constexpr int MAX_TILES = 32;        // row tiles per PPT node
 constexpr int WALK_STACK = 12;        // continuation frames per walking warp
 
 enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, CONCAT, SPLIT,
@@ -138,6 +138,7 @@ struct Ctx {
   // configuration
   int mak, muf, det, eval, IT;
   int wide;                           // the graph has row-wise forks (Ungroup / Group)
+  int bf16;                           // payloads rounded to bfloat16 at emission
   int tune;                           // experiment switches (environment AMPNET_TUNE): 2 no look-ahead, 4 no per-node counters
   float lr;
   unsigned long long timeout_ns;

@@ -2,20 +2,20 @@
 import numpy as np
 
 
-def run_both(oracle_mod, graph, inst, params, mak, muf, lr, order=None, timeout_s=60.0, **engine_kw):
+def run_both(oracle_mod, graph, inst, params, mak, muf, lr, order=None, timeout_s=60.0, payload_bf16=False, **engine_kw):
     import paper_1705_09786_b200 as amp
-    o = oracle_mod.Oracle(graph)
+    o = oracle_mod.Oracle(graph, payload_bf16=payload_bf16)
     o.load_instances(inst)
     o.set_params(params)
     ost, oloss = o.run_epoch(mak=mak, muf=muf, lr=lr, order=order)
-    e = amp.Engine(graph)
+    e = amp.Engine(graph, payload_bf16=payload_bf16)
     e.load_instances(inst)
     e.set_params(params)
     est, eloss = e.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=True, order=order, timeout_s=timeout_s, **engine_kw)
     return o, ost, oloss, e, est, eloss
 
 
-def assert_parity(graph, o, ost, oloss, e, est, eloss, param_rtol=1e-4, loss_rtol=1e-5, loss_atol=2e-6):
+def assert_parity(graph, o, ost, oloss, e, est, eloss, param_rtol=1e-4, loss_rtol=1e-5, loss_atol=2e-6, param_floor=1e-30):
     """Integer bookkeeping bit-exact; parameters within max relative error 1e-4 (relative to the largest
     magnitude of the tensor, with elementwise slack for entries near zero); per-instance losses within 1e-5."""
     # routing, key bookkeeping, update counts: exact
@@ -42,7 +42,7 @@ def assert_parity(graph, o, ost, oloss, e, est, eloss, param_rtol=1e-4, loss_rto
     worst = 0.0
     ep, op = e.get_params(), o.get_params()
     for k in op:
-        scale = np.abs(op[k]).max() + 1e-30
+        scale = max(np.abs(op[k]).max(), param_floor)
         err = np.abs(ep[k].astype(np.float64) - op[k]).max() / scale
         worst = max(worst, err)
         assert err <= param_rtol, (graph.names[k[0]], k[1], err)

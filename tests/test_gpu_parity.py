@@ -99,6 +99,27 @@ def test_per_node_update_threshold(oracle_mod):
     r[3].close()
 
 
+@pytest.mark.parametrize("family,n,mak,muf,lr", [("tree", 30, 16, 20, 0.02), ("rnn", 60, 8, 10, 0.02),
+                                                ("ggnn", 20, 16, 40, 0.003), ("mlp", 40, 4, 8, 0.01)])
+def test_bf16_payloads_match_oracle(oracle_mod, family, n, mak, muf, lr):
+    """bf16 messages: every emitted payload rounded to bfloat16 on both sides.  Bookkeeping stays bit-exact.  A value
+    that lies within fp32 rounding of a bf16 rounding boundary can round the other way on the GPU (fp32) than in
+    the oracle (fp64) and then differs by one bf16 ulp (2^-8 relative), so the float tolerance is a few bf16 ulps."""
+    g, inst = _case(family, n)
+    p = wp.init_params(g)
+    r = parity.run_both(oracle_mod, g, inst, p, mak, muf, lr, payload_bf16=True)
+    # biases that are still ~1e-4 after one short epoch are compared on an absolute scale of 1e-3
+    parity.assert_parity(g, *r, param_rtol=2e-2, loss_rtol=2e-2, loss_atol=2e-3, param_floor=1e-3)
+    # and the rounding is really applied: the fp32-message run gives different losses
+    e2 = __import__("paper_1705_09786_b200").Engine(g)
+    e2.load_instances(inst)
+    e2.set_params(p)
+    _, l32 = e2.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=True, timeout_s=60)
+    assert np.abs(l32 - r[5]).max() > 0
+    e2.close()
+    r[3].close()
+
+
 @pytest.mark.parametrize("family,n", [("mlp", 64), ("rnn", 80), ("tree", 40), ("ggnn", 30)])
 def test_eval_matches_oracle(oracle_mod, family, n):
     import paper_1705_09786_b200 as amp
