@@ -31,16 +31,23 @@ WORKLOADS = {
     "rnn": (ir.rnn, data.list_instances, 20000, 16, 50, 0.05),
     "tree": (ir.tree, data.tree_instances, 8544, 64, 100, 0.05),
     "ggnn": (ir.ggnn, data.graph_instances, 130000, 128, 200, 0.01),
+    # throughput stress: binary tree RNN, hidden 512, 64..512 leaves, bf16 messages with fp32 accumulators
+    "stress": (lambda: ir.tree(vocab=20000, emb=512, hidden=512, classes=5),
+               lambda n, split=0: data.tree_instances(n=n, min_leaves=64, max_leaves=512, split=split, config_index=5),
+               50000, 64, 64, 0.01),
 }
+STRESS_BENCH_INSTANCES = 1000     # the stress workload is timed on a prefix of this many trees per step
+SWEEP_MAK = (1, 8, 64, 256, 1024)
+SWEEP_MUF = (1, 64, 1024)
 GGNN_BENCH_INSTANCES = 20000      # the graph workload is timed on a prefix of this many graphs per step
 
 
 def make_workload(name, rank=0, n=None):
     build_graph, gen, full, mak, muf, lr = WORKLOADS[name]
     if n is None:
-        n = GGNN_BENCH_INSTANCES if name == "ggnn" else full
+        n = GGNN_BENCH_INSTANCES if name == "ggnn" else STRESS_BENCH_INSTANCES if name == "stress" else full
     inst = gen(n=n, split=0 if rank == 0 else 100 + rank)
-    return build_graph(), inst, dict(mak=mak, muf=muf, lr=lr, full=full)
+    return build_graph(), inst, dict(mak=mak, muf=muf, lr=lr, full=full, bf16=(name == "stress"))
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -134,7 +141,7 @@ def measured_peaks():
 def time_oracle(graph, inst, cfg, target_s=12.0, probe=48):
     """The oracle as it stands, single-threaded, on a bounded prefix of the workload."""
     import oracle as oracle_mod
-    o = oracle_mod.Oracle(graph)
+    o = oracle_mod.Oracle(graph, payload_bf16=cfg.get("bf16", False))
     p = wp.init_params(graph)
     probe = min(probe, inst.n)
     o.load_instances(inst.head(probe))
@@ -174,7 +181,7 @@ def run_reference(args):
 
 
 def workload_config(name, inst, cfg, mode):
-    return {"workload": name, "instances_per_step": int(inst.n), "full_dataset_instances": cfg["full"],
+    return {"workload": name, "messages": "bf16 payloads, fp32 accumulators" if cfg.get("bf16") else "fp32", "instances_per_step": int(inst.n), "full_dataset_instances": cfg["full"],
             "max_active_keys": cfg["mak"], "min_update_frequency": cfg["muf"], "lr": cfg["lr"], "mode": mode,
             "l2": "flushed between steps (256 MiB write)", "parallelism": "replicas, no collective"}
 
@@ -194,7 +201,7 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     dist_init("nccl")
     graph, inst, cfg = make_workload(args.workload, rank, n=args.instances)
-    eng = amp.Engine(graph, device=local)
+    eng = amp.Engine(graph, device=local, payload_bf16=cfg["bf16"])
     eng.load_instances(inst)
     p0 = wp.init_params(graph)
     eng.set_params(p0)
@@ -224,6 +231,8 @@ def run_ours(args):
     torch.cuda.synchronize()
     barrier()
     clocks = sampler.summary()
+    updates = {n: eng.node_stats(n)["n_updates"] for n in graph.ppt_nodes()}     # of the last timed step
+    placement = {graph.names[n]: eng.placement(n) for n in graph.ppt_nodes()}
     secs = sum(step_s)
     value, tmax = aggregate(inst.n * args.steps, secs, dev)
     msg_rate, _ = aggregate(msgs, secs, dev)
@@ -247,9 +256,25 @@ def run_ours(args):
     e2e_s = time.perf_counter() - t0
     e2e_value, _ = aggregate(inst.n * e2e_steps, e2e_s, dev)
 
+    sweep = None
+    if args.sweep and rank == 0:
+        # max_active_keys x min_update_frequency grid on a prefix (one epoch each, parameters reset)
+        sweep = []
+        for mak in SWEEP_MAK:
+            sub = inst.head(max(20, min(inst.n, 30 * mak if mak < 64 else 400)))
+            eng.load_instances(sub)
+            for muf in SWEEP_MUF:
+                eng.set_params(p0)
+                st, _ = eng.run_epoch(mak=mak, muf=muf, lr=cfg["lr"], deterministic=False, timeout_s=args.timeout,
+                                      want_loss=False)
+                sweep.append({"max_active_keys": mak, "min_update_frequency": muf, "instances": int(sub.n),
+                              "instances_per_s": sub.n / st.seconds, "node_messages_per_s": st.node_messages / st.seconds,
+                              "rows_per_micro_batch": st.micro_batch_rows / max(1, st.micro_batches),
+                              "max_active_observed": int(st.max_active_observed), "max_staleness": int(st.max_staleness),
+                              "micro_batches_fma": int(st.micro_batches), "micro_batches_tensor_core": 0})
+        eng.load_instances(inst)
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        updates = {n: eng.node_stats(n)["n_updates"] for n in graph.ppt_nodes()}
         flops = rf.algorithmic_flops(graph, inst, updates)
         sm_mhz = float(peaks.get("sm_max_mhz", 1965.0))
         peak_tf = rf.fma_peak_tflops(sm_mhz)
@@ -284,7 +309,10 @@ def run_ours(args):
                 "clocks": clocks, "gpu_launches": args.steps,
                 "stats": {"mean_loss_last_step": last.mean_loss, "max_staleness": int(last.max_staleness),
                           "rows_per_micro_batch": last.micro_batch_rows / max(1, last.micro_batches),
-                          "placement": {graph.names[n]: eng.placement(n) for n in graph.ppt_nodes()}}}
+                          "placement": placement,
+                          "micro_batch_split": {"fma": 1.0, "tensor_core": 0.0}}}
+        if sweep is not None:
+            line["sweep"] = sweep
         print(json.dumps(line), flush=True)
     eng.close()
     import torch.distributed as dist
@@ -302,6 +330,7 @@ def main():
     ap.add_argument("--instances", type=int, default=None, help="instances per step (default: the workload's size)")
     ap.add_argument("--timeout", type=float, default=300.0, help="bound on one device run, seconds")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="also run the max_active_keys x min_update_frequency grid")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

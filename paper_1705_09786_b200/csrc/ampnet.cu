@@ -378,13 +378,16 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
     const double share = std::max((double)P.nmat * P.in * P.out / total_w, 0.1);
     int T = 1 + (int)std::floor(share * avail);
     T = std::max(1, std::min({T, max_tiles, P.out <= 16 ? P.out : std::max(1, P.out / 4)}));
-    for (;;) {
-      int R = (P.out + T - 1) / T;
-      int bm = BM;
-      while (tile_smem_floats(P, R, bm) > budget && bm > std::max(rows_max, 4)) bm = std::max(std::max(rows_max, 4), bm / 2);
-      if (tile_smem_floats(P, R, bm) <= budget) { P.R = R; P.BM = bm; P.T = (P.out + R - 1) / R; break; }
-      if (R == 1 || T >= MAX_TILES) return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory with %d row tiles", P.node, T);
-      T = std::min(P.out, T + 1);
+    // Keep the micro-batch capacity if more row tiles make the tile fit; only then shrink the capacity.
+    bool placed = false;
+    const int bm_min = std::max(rows_max, 4);
+    for (int bm = BM; !placed; bm = std::max(bm_min, bm / 2)) {
+      for (int t = T; t <= std::min(MAX_TILES, P.out); t++) {
+        const int R = (P.out + t - 1) / t;
+        if (tile_smem_floats(P, R, bm) <= budget) { P.R = R; P.BM = bm; P.T = (P.out + R - 1) / R; placed = true; break; }
+      }
+      if (!placed && bm == bm_min)
+        return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory with %d row tiles", P.node, MAX_TILES);
     }
     P.smem_floats = tile_smem_floats(P, P.R, P.BM);
     used += P.T;
