@@ -137,32 +137,36 @@ __device__ __forceinline__ void warp_copy_v(float* dst, int dld, const float* sr
   const int wv = dim / V, total = rows * wv;
   for (int base = lane; base < total; base += 128) {
     float v[4][V];
+    size_t off[4], doff[4];
 #pragma unroll
     for (int k = 0; k < 4; k++) {
       const int idx = base + 32 * k;
-      if (idx < total) {
-        const int r = idx / wv, c = idx - r * wv;
-        const size_t off = (size_t)r * sld + (size_t)c * V;
+      int r = 0, c = idx;
+      if (rows > 1) { r = idx / wv; c = idx - r * wv; }
+      off[k] = (size_t)r * sld + (size_t)c * V;
+      doff[k] = (size_t)r * dld + (size_t)c * V;
 #pragma unroll
-        for (int q = 0; q < V; q++) v[k][q] = 0.f;
-        for (int j = 0; j < nsum; j++) {                       // addend order
-          const float* a = src + (size_t)j * sstride + off;
-          if (V == 4) { const float4 t = __ldcg(reinterpret_cast<const float4*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; v[k][2 % V] += t.z; v[k][3 % V] += t.w; }
-          else if (V == 2) { const float2 t = __ldcg(reinterpret_cast<const float2*>(a)); v[k][0] += t.x; v[k][1 % V] += t.y; }
-          else v[k][0] += __ldcg(a);
-        }
-        if (nsum > 1) {
+      for (int q = 0; q < V; q++) v[k][q] = 0.f;
+    }
+    for (int j = 0; j < nsum; j++) {                             // addend order; the four loads of one addend overlap
+      const float* a = src + (size_t)j * sstride;
 #pragma unroll
-          for (int q = 0; q < V; q++) v[k][q] = emit_round(v[k][q]);
+      for (int k = 0; k < 4; k++) {
+        if (base + 32 * k < total) {
+          if (V == 4) { const float4 t = __ldcg(reinterpret_cast<const float4*>(a + off[k])); v[k][0] += t.x; v[k][1 % V] += t.y; v[k][2 % V] += t.z; v[k][3 % V] += t.w; }
+          else if (V == 2) { const float2 t = __ldcg(reinterpret_cast<const float2*>(a + off[k])); v[k][0] += t.x; v[k][1 % V] += t.y; }
+          else v[k][0] += __ldcg(a + off[k]);
         }
       }
     }
 #pragma unroll
     for (int k = 0; k < 4; k++) {
-      const int idx = base + 32 * k;
-      if (idx < total) {
-        const int r = idx / wv, c = idx - r * wv;
-        float* d = dst + (size_t)r * dld + (size_t)c * V;
+      if (base + 32 * k < total) {
+        if (nsum > 1) {
+#pragma unroll
+          for (int q = 0; q < V; q++) v[k][q] = emit_round(v[k][q]);
+        }
+        float* d = dst + doff[k];
         if (V == 4) *reinterpret_cast<float4*>(d) = make_float4(v[k][0], v[k][1 % V], v[k][2 % V], v[k][3 % V]);
         else if (V == 2) *reinterpret_cast<float2*>(d) = make_float2(v[k][0], v[k][1 % V]);
         else d[0] = v[k][0];
@@ -301,6 +305,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (key < 0) return;
           if (f.rows > P.rows_max) { fail(C, ST_OVERFLOW, f.node, f.rows); return; }
           unsigned ticket = 0;
+          const long long tq0 = (C.tune & 8) ? clock64() : 0;
           if (lane == 0) ticket = ring_ticket(P.ring[f.dir]);
           if (f.dir == FWD) {
             if (P.xcache) {
@@ -311,7 +316,14 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             warp_copy(P.gbuf + key * (long long)P.rows_max * P.out_dim, P.out_dim, f, f.rows, P.out_dim, lane);
           }
           __syncwarp();
+          const long long tq1 = (C.tune & 8) ? clock64() : 0;
           if (lane == 0) ring_publish(P.ring[f.dir], ticket, f);
+          if ((C.tune & 8) && lane == 0) {      // profile: SPLIT slots = copy (+ticket) / publish, SOURCE FWD slot = before
+            const long long tq2 = clock64();
+            atomicAdd(&C.g->walk_cycles[SPLIT * 2], (unsigned long long)(tq1 - tq0)); atomicAdd(&C.g->walk_steps[SPLIT * 2], 1ull);
+            atomicAdd(&C.g->walk_cycles[SPLIT * 2 + 1], (unsigned long long)(tq2 - tq1)); atomicAdd(&C.g->walk_steps[SPLIT * 2 + 1], 1ull);
+            atomicAdd(&C.g->walk_cycles[SOURCE * 2], (unsigned long long)(tq0 - tstep)); atomicAdd(&C.g->walk_steps[SOURCE * 2], 1ull);
+          }
         } break;
         case LOSS_CE: case LOSS_MSE: {
           long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
