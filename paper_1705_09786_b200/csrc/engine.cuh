@@ -1275,7 +1275,13 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
             dirbuf[(size_t)b * H + r_begin + r] = dirp[b * SR + r] + dq * rg;
           }
           __syncthreads();
-          AMP_DISPATCH_J(P.J, (tile_dW<J>(dpz, SR, nb, Wz, in, R, in, part2)));
+          // this tile's share of da_c joins its second partial here, so that emission sums one partial array per tile
+          for (int idx = tid; idx < nb * in; idx += THREADS) {
+            const int c = idx % in;
+            part2[idx] = c < H ? __ldcg(part1 + idx) : 0.f;
+          }
+          __syncthreads();
+          AMP_DISPATCH_J(P.J, (tile_dW<J, true>(dpz, SR, nb, Wz, in, R, in, part2)));
           AMP_DISPATCH_J(P.J, (tile_dW<J, true>(dpr, SR, nb, Wr, in, R, in, part2)));
           tile_accum(dpz, SR, nb, M.Xs, in, M.As, in, R, in);
           tile_accum(dpr, SR, nb, M.Xs, in, M.As + SR * in, in, R, in);
@@ -1381,15 +1387,12 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
               const size_t e = (size_t)ro * in + k;
               const int c = k - row * in;
               float sum = 0.f;
-              for (int t0 = 0; t0 < P.T; t0 += 8) {          // eight tiles' partials in flight, added in tile order
-                float v[8], w[8];
+              for (int t0 = 0; t0 < P.T; t0 += 16) {         // sixteen tiles' partials in flight, added in tile order
+                float v[16];
 #pragma unroll
-                for (int t = 0; t < 8; t++) {
-                  v[t] = t0 + t < P.T ? __ldcg(pa + (size_t)(t0 + t) * pstride + e) : 0.f;
-                  w[t] = (pb && c < H && t0 + t < P.T) ? __ldcg(pb + (size_t)(t0 + t) * pstride + e) : 0.f;
-                }
+                for (int t = 0; t < 16; t++) v[t] = t0 + t < P.T ? __ldcg(pa + (size_t)(t0 + t) * pstride + e) : 0.f;
 #pragma unroll
-                for (int t = 0; t < 8; t++) { sum += v[t]; sum += w[t]; }
+                for (int t = 0; t < 16; t++) sum += v[t];
               }
               if (pb && c >= H) sum += __ldcg(dirb + (size_t)(ro + row) * H + (c - H));
               P.stage[e] = emit_round(sum);
