@@ -355,13 +355,14 @@ size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
 
 // Placement: row tiles per PPT node.  Enough tiles that a tile's weights + accumulators + staging fit in
 // shared memory, then the remaining CTAs in proportion to the nodes' multiply-add volume.
-ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles) {
+ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles, bool emitters, int tiles_cap) {
   cudaFuncAttributes fa{};
   size_t static_smem = 40 * 1024;
   if (cudaFuncGetAttributes(&fa, ampnet_engine) == cudaSuccess) static_smem = fa.sharedSizeBytes;
   const size_t budget = ((size_t)g->max_smem - static_smem - 1024) / sizeof(float);
   int max_tiles = 16;      // default; a node whose tile does not fit in shared memory gets more, up to MAX_TILES
   if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, std::min(MAX_TILES, atoi(e)));
+  if (tiles_cap > 0) max_tiles = std::min(max_tiles, tiles_cap);
   double total_w = 0;
   for (auto& P : g->ppts) if (P.kind != LOOKUP) total_w += (double)P.nmat * P.in * P.out;
   const int avail = std::max(1, n_ctas - 1 - (int)g->ppts.size());
@@ -394,9 +395,14 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   }
   if (used > n_ctas) return set_err(g, AMPNET_EINVAL, "placement needs %d CTAs but only %d are available", used, n_ctas);
   roles.clear();
-  roles.push_back(Role{-1, 0});
+  roles.push_back(Role{-1, 0, 0, 0});
   for (int p = 0; p < (int)g->ppts.size(); p++)
-    for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t});
+    for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t, 0, 0});
+  if (emitters) {
+    if (2 * used - 1 > n_ctas) return AMPNET_EOVERFLOW;          // the caller retries with fewer tiles or without emitters
+    for (int p = 0; p < (int)g->ppts.size(); p++)
+      for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t, 1, 0});
+  }
   return AMPNET_OK;
 }
 
@@ -415,8 +421,15 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   infer_domains(g, D);
   const int IT = g->has_it ? g->it_steps + 1 : 1;
   int n_ctas = cfg && cfg->n_ctas > 0 ? std::min(cfg->n_ctas, g->n_sms) : g->n_sms;
-  ampnet_status_t st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles);
+  // Asynchronous runs pair every tile with an emitter CTA when the SMs allow it (with fewer tiles if need be).
+  int tune = 0;
+  if (const char* e = getenv("AMPNET_TUNE")) tune = atoi(e);
+  bool emitters = !det && !(tune & 32);
+  ampnet_status_t st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles, emitters, 0);
+  if (st == AMPNET_EOVERFLOW && emitters) st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles, true, 8);
+  if (st == AMPNET_EOVERFLOW && emitters) { emitters = false; st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles, false, 0); }
   if (st != AMPNET_OK) return st;
+  R.ctx.emit_ctas = emitters ? 1 : 0;
   n_ctas = (int)R.roles.size();
   DeviceArena &C = g->ctl, &B = g->bulk;
   C.used = B.used = 0;
@@ -465,7 +478,10 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.bhdr = B.take<Hdr>((size_t)BATCH_BLOCKS * MAX_BATCH_MSGS);
     P.sortbuf = B.take<unsigned long long>(cap);
     if ((P.T > 1 && H.kind != LOOKUP) || H.kind == GRUCELL) P.dxpart = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
-    P.stage = B.take<float>((size_t)P.BM * std::max(P.in_dim, P.out_dim));
+    P.stage_floats = (long long)P.BM * std::max(P.in_dim, P.out_dim);
+    P.stage = B.take<float>((size_t)2 * P.stage_floats);
+    P.emit_pub = C.take<unsigned>(P.T);
+    P.emit_done = C.take<unsigned>(P.T);
     P.nbar = C.take<unsigned>(1);
     P.stats = C.take<PPTStats>(1);
     P.update_log = B.take<int>(g->update_log_cap); P.update_log_cap = g->update_log_cap;

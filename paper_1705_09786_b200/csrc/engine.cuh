@@ -1035,6 +1035,130 @@ __device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, con
   return C.inst.dense + (long long)h.inst * C.inst.dense_dim;         // fed directly by a dense-row source
 }
 
+// Warp 0 of a CTA: descriptor, headers, keys, row offsets and row pointers of batch `batch` into shared memory.
+__device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared& S, const unsigned my_batch) {
+  const int lane = threadIdx.x & 31;
+  const int in = P.in_dim;
+    const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]);
+    const int4 d0 = __ldcg(dp), d1 = __ldcg(dp + 1);          // same address in every lane
+    int4 ha = make_int4(0, 0, 0, 0), hb = make_int4(0, 0, 0, 0);
+    if (!C.det) {                                             // headers travel with the descriptor: load both at once
+      const int4* e = reinterpret_cast<const int4*>(&P.bhdr[(my_batch & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + lane]);
+      ha = __ldcg(e); hb = __ldcg(e + 1);
+    }
+    const int cnt = d0.y, ddir = d0.z;
+    if (C.det && lane < cnt) {
+      const unsigned slot = P.sched[((unsigned)d0.x + lane) & P.sched_mask];
+      const int4* e = reinterpret_cast<const int4*>(&P.ring[ddir].e[slot]);
+      ha = __ldcg(e); hb = __ldcg(e + 1);
+    }
+    Hdr h; h.inst = ha.x; h.seq = ha.y; h.slot = ha.z; h.it = ha.w; h.u = hb.x; h.port = hb.y; h.rows = hb.z; h.flags = hb.w;
+    if (h.rows <= 0) h.rows = 1;
+    const int rows = lane < cnt ? h.rows : 0;
+    int cum = rows;
+    for (int o = 1; o < 32; o <<= 1) { int v = __shfl_up_sync(0xffffffffu, cum, o); if (lane >= o) cum += v; }
+    const int total = __shfl_sync(0xffffffffu, cum, 31);
+    const int off = cum - rows;
+    long long key = 0;
+    if (lane < cnt) {
+      key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      S.hdr[lane] = h; S.key[lane] = key; S.rowoff[lane] = off;
+      if (key >= 0 && total <= P.BM) {
+        const float* x0 = P.kind != LOOKUP ? msg_x(C, P, h, key) : nullptr;
+        for (int r = 0; r < rows; r++) { S.rowmsg[off + r] = lane; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
+      }
+    }
+    const unsigned bad = __ballot_sync(0xffffffffu, lane < cnt && key < 0);
+    if (lane == 0) {
+      S.rowoff[cnt] = total;
+      BatchDesc dd; dd.sched_start = (unsigned)d0.x; dd.count = d0.y; dd.dir = d0.z; dd.flags = d0.w;
+      dd.n_upd = d1.x; dd.nrows = d1.y; dd.pad0 = dd.pad1 = 0;
+      S.desc = dd;
+      if (bad) S.ok = 0;
+      if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; }
+    }
+
+}
+
+// Emission of a batch by one CTA: reduce the tiles' partial input gradients for the rows this CTA emits, then walk
+// the messages through the parameter-free nodes.  `parity` selects the per-batch buffers, `stage` the staging rows.
+__device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile, TileShared& S, const BatchDesc d,
+                                        const unsigned parity, float* stage, WalkAcc& acc) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const DevNode& N = g_nodes[P.node];
+  const int in = P.in_dim, out = P.out_dim, count = d.count, dir = d.dir;
+  const int nb = S.rowoff[count];
+  const unsigned my_batch = parity;
+    if (g_bf16 && dir == BWD && P.kind == LINEAR && P.T == 1 && !(P.flags & 1)) {
+      for (int idx = tid; idx < nb * in; idx += THREADS) stage[idx] = emit_round(stage[idx]);
+      __syncthreads();
+    }
+    const bool split = C.wide && P.T > 1;          // share row-wise forks among the node's tiles
+    if (dir == BWD && P.kind != LOOKUP && !(P.flags & 1) && (P.T > 1 || P.kind == GRUCELL)) {
+      // Sum the tiles' partial input gradients (tile order) for the rows this tile emits; every thread keeps
+      // all T loads of an element in flight.
+      const size_t pstride = (size_t)P.BM * in;
+      const float* pa = P.dxpart + (size_t)(my_batch & 1) * P.T * pstride;
+      const float* pb = P.kind == GRUCELL ? P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride : nullptr;
+      const float* dirb = pb ? pb + (size_t)P.T * pstride : nullptr;
+      const int H = out;
+      for (int i = split ? 0 : tile; i < count; i += split ? 1 : P.T) {
+        const int part = (tile - i % P.T + P.T) % P.T;
+        const int ro = S.rowoff[i], ne = S.hdr[i].rows * in;
+        for (int k = tid; k < ne; k += THREADS) {
+          const int row = k / in;
+          if (part != 0 && row % P.T != part) continue;
+          const size_t e = (size_t)ro * in + k;
+          const int c = k - row * in;
+          float sum = 0.f;
+          for (int t0 = 0; t0 < P.T; t0 += 16) {         // sixteen tiles' partials in flight, added in tile order
+            float v[16];
+#pragma unroll
+            for (int t = 0; t < 16; t++) v[t] = t0 + t < P.T ? __ldcg(pa + (size_t)(t0 + t) * pstride + e) : 0.f;
+#pragma unroll
+            for (int t = 0; t < 16; t++) sum += v[t];
+          }
+          if (pb && c >= H) sum += __ldcg(dirb + (size_t)(ro + row) * H + (c - H));
+          stage[e] = emit_round(sum);
+        }
+      }
+      __syncthreads();
+    }
+    if (tid == 0) S.pool.outstanding = split ? count : (tile < count ? (count - tile + P.T - 1) / P.T : 0);
+    __syncthreads();
+    const long long tw0 = clock64();
+    int mine = 0;
+    for (int i = 0; i < count; i++) {
+      const int part = (tile - i % P.T + P.T) % P.T;
+      if (!split && part != 0) continue;
+      if ((mine++ % WARPS) != warp) continue;
+      const Hdr& h = S.hdr[i];
+      Frame f;
+      f.iter = 0; f.inst = h.inst; f.seq = h.seq; f.slot = h.slot; f.it = h.it; f.u = h.u; f.port = h.port;
+      f.rows = h.rows; f.flags = h.flags; f.nsum = 1; f.sstride = 0;
+      f.part = split ? part : 0; f.nparts = split ? P.T : 1;
+      if (dir == FWD) {
+        f.node = N.succ_node[0]; f.aport = N.succ_port[0]; f.dir = FWD; f.dim = out; f.ld = out;
+        f.p = P.kind == LOOKUP ? stage + (size_t)S.rowoff[i] * out
+                               : P.ycache + (size_t)S.key[i] * P.rows_max * out;
+      } else {
+        f.node = N.pred_node[0]; f.aport = N.pred_port[0]; f.dir = BWD; f.dim = in; f.ld = in;
+        if (P.kind == LOOKUP || (P.flags & 1)) { f.p = nullptr; f.dim = 0; f.rows = 1; }
+        else f.p = stage + (size_t)S.rowoff[i] * in;
+      }
+      walk(C, f, S.stack[warp], acc, &S.pool);
+      __syncwarp();
+      if (lane == 0) atomicSub(&S.pool.outstanding, 1);
+    }
+    const long long tw1 = clock64();
+    pool_steal(C, &S.pool, S.stack[warp], acc);
+    const long long tw2 = clock64();
+    if (lane == 0 && warp < 2) { S.phase[10 + 2 * warp] += (unsigned long long)(tw1 - tw0); S.phase[11 + 2 * warp] += (unsigned long long)(tw2 - tw1); }
+    flush_acc(C, acc, lane);
+    __syncthreads();
+    if (tid == 0) S.phase[14] += (unsigned long long)(clock64() - tw2);
+}
+
 __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileShared& S,
                          const unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -1117,53 +1241,20 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       }
       __syncthreads();
       if (!S.ok || aborted(C)) { running = false; break; }
-      // ---- descriptor, headers, keys, row offsets, row pointers: one warp, one block barrier --------------
-      if (warp == 0) {
-        const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]);
-        const int4 d0 = __ldcg(dp), d1 = __ldcg(dp + 1);          // same address in every lane
-        int4 ha = make_int4(0, 0, 0, 0), hb = make_int4(0, 0, 0, 0);
-        if (!C.det) {                                             // headers travel with the descriptor: load both at once
-          const int4* e = reinterpret_cast<const int4*>(&P.bhdr[(my_batch & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + lane]);
-          ha = __ldcg(e); hb = __ldcg(e + 1);
-        }
-        const int cnt = d0.y, ddir = d0.z;
-        if (C.det && lane < cnt) {
-          const unsigned slot = P.sched[((unsigned)d0.x + lane) & P.sched_mask];
-          const int4* e = reinterpret_cast<const int4*>(&P.ring[ddir].e[slot]);
-          ha = __ldcg(e); hb = __ldcg(e + 1);
-        }
-        Hdr h; h.inst = ha.x; h.seq = ha.y; h.slot = ha.z; h.it = ha.w; h.u = hb.x; h.port = hb.y; h.rows = hb.z; h.flags = hb.w;
-        if (h.rows <= 0) h.rows = 1;
-        const int rows = lane < cnt ? h.rows : 0;
-        int cum = rows;
-        for (int o = 1; o < 32; o <<= 1) { int v = __shfl_up_sync(0xffffffffu, cum, o); if (lane >= o) cum += v; }
-        const int total = __shfl_sync(0xffffffffu, cum, 31);
-        const int off = cum - rows;
-        long long key = 0;
-        if (lane < cnt) {
-          key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
-          S.hdr[lane] = h; S.key[lane] = key; S.rowoff[lane] = off;
-          if (key >= 0 && total <= P.BM) {
-            const float* x0 = P.kind != LOOKUP ? msg_x(C, P, h, key) : nullptr;
-            for (int r = 0; r < rows; r++) { S.rowmsg[off + r] = lane; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
-          }
-        }
-        const unsigned bad = __ballot_sync(0xffffffffu, lane < cnt && key < 0);
-        if (lane == 0) {
-          S.rowoff[cnt] = total;
-          BatchDesc dd; dd.sched_start = (unsigned)d0.x; dd.count = d0.y; dd.dir = d0.z; dd.flags = d0.w;
-          dd.n_upd = d1.x; dd.nrows = d1.y; dd.pad0 = dd.pad1 = 0;
-          S.desc = dd;
-          if (bad) S.ok = 0;
-          if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; }
-        }
-      }
+      if (warp == 0) load_batch_ctx(C, P, S, my_batch);
       __syncthreads();
       const BatchDesc d = S.desc;
       my_batch++;
       AMP_PHASE(d.count > 0 ? 1 : 0);
       const int count = d.count, dir = d.dir;
       if (!S.ok) { running = false; break; }
+      float* const stage_k = P.stage + (size_t)(my_batch & 1) * P.stage_floats;
+      if (C.emit_ctas && count > 0) {
+        // the per-batch buffers of this parity were last used two batches ago: wait until that batch has been emitted
+        if (tid == 0 && !spin_until(C, t0, [&] { return ld_acq(&P.emit_done[tile]) + 2u >= my_batch; })) S.ok = 0;
+        __syncthreads();
+        if (!S.ok) { running = false; break; }
+      }
       const int nb = S.rowoff[count];
       const bool eval = count > 0 && (S.hdr[0].flags & HDR_EVAL);
       AMP_PHASE(2);
@@ -1188,7 +1279,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           }
           __syncthreads();
           if (!(P.flags & 1)) {
-            float* dst = P.T > 1 ? P.dxpart + ((size_t)(my_batch & 1) * P.T + tile) * P.BM * in : P.stage;
+            float* dst = P.T > 1 ? P.dxpart + ((size_t)(my_batch & 1) * P.T + tile) * P.BM * in : stage_k;
             AMP_DISPATCH_J(P.J, (tile_dW<J>(M.Ds, P.R, nb, M.Ws, in, R, in, dst)));
           }
           tile_accum(M.Ds, P.R, nb, M.Xs, in, M.As, in, R, in);
@@ -1301,7 +1392,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
             const Hdr& h = S.hdr[m];
             const int pos = I.kind == 3 ? (b - S.rowoff[m]) : h.u;
             const int id = I.tokens[I.offsets[h.inst] + pos];
-            P.stage[idx] = ((unsigned)id < (unsigned)in) ? emit_round(P.W[(size_t)id * out + c]) : 0.f;
+            stage_k[idx] = ((unsigned)id < (unsigned)in) ? emit_round(P.W[(size_t)id * out + c]) : 0.f;
           }
         } else {
           for (int c = tid; c < out; c += THREADS)
@@ -1365,77 +1456,10 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           if (warp_uniform(bw) == my_batch) leader_try_schedule(C, P, S);
           if (lane == 0) S.phase[8] += (unsigned long long)(clock64() - tq);
         }
-        if (g_bf16 && dir == BWD && P.kind == LINEAR && P.T == 1 && !(P.flags & 1)) {
-          for (int idx = tid; idx < nb * in; idx += THREADS) P.stage[idx] = emit_round(P.stage[idx]);
-          __syncthreads();
-        }
-        const bool split = C.wide && P.T > 1;          // share row-wise forks among the node's tiles
-        if (dir == BWD && P.kind != LOOKUP && !(P.flags & 1) && (P.T > 1 || P.kind == GRUCELL)) {
-          // Sum the tiles' partial input gradients (tile order) for the rows this tile emits; every thread keeps
-          // all T loads of an element in flight.
-          const size_t pstride = (size_t)P.BM * in;
-          const float* pa = P.dxpart + (size_t)(my_batch & 1) * P.T * pstride;
-          const float* pb = P.kind == GRUCELL ? P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride : nullptr;
-          const float* dirb = pb ? pb + (size_t)P.T * pstride : nullptr;
-          const int H = out;
-          for (int i = split ? 0 : tile; i < count; i += split ? 1 : P.T) {
-            const int part = (tile - i % P.T + P.T) % P.T;
-            const int ro = S.rowoff[i], ne = S.hdr[i].rows * in;
-            for (int k = tid; k < ne; k += THREADS) {
-              const int row = k / in;
-              if (part != 0 && row % P.T != part) continue;
-              const size_t e = (size_t)ro * in + k;
-              const int c = k - row * in;
-              float sum = 0.f;
-              for (int t0 = 0; t0 < P.T; t0 += 16) {         // sixteen tiles' partials in flight, added in tile order
-                float v[16];
-#pragma unroll
-                for (int t = 0; t < 16; t++) v[t] = t0 + t < P.T ? __ldcg(pa + (size_t)(t0 + t) * pstride + e) : 0.f;
-#pragma unroll
-                for (int t = 0; t < 16; t++) sum += v[t];
-              }
-              if (pb && c >= H) sum += __ldcg(dirb + (size_t)(ro + row) * H + (c - H));
-              P.stage[e] = emit_round(sum);
-            }
-          }
-          __syncthreads();
-        }
-        if (tid == 0) S.pool.outstanding = split ? count : (tile < count ? (count - tile + P.T - 1) / P.T : 0);
-        __syncthreads();
-        const long long tw0 = clock64();
-        if (tid == 0) S.phase[9] += (unsigned long long)(tw0 - tph);       // look-ahead + reduction + barriers
-        int mine = 0;
-        for (int i = 0; i < count; i++) {
-          const int part = (tile - i % P.T + P.T) % P.T;
-          if (!split && part != 0) continue;
-          if ((mine++ % WARPS) != warp) continue;
-          const Hdr& h = S.hdr[i];
-          Frame f;
-          f.iter = 0; f.inst = h.inst; f.seq = h.seq; f.slot = h.slot; f.it = h.it; f.u = h.u; f.port = h.port;
-          f.rows = h.rows; f.flags = h.flags; f.nsum = 1; f.sstride = 0;
-          f.part = split ? part : 0; f.nparts = split ? P.T : 1;
-          if (dir == FWD) {
-            f.node = N.succ_node[0]; f.aport = N.succ_port[0]; f.dir = FWD; f.dim = out; f.ld = out;
-            f.p = P.kind == LOOKUP ? P.stage + (size_t)S.rowoff[i] * out
-                                   : P.ycache + (size_t)S.key[i] * P.rows_max * out;
-          } else {
-            f.node = N.pred_node[0]; f.aport = N.pred_port[0]; f.dir = BWD; f.dim = in; f.ld = in;
-            if (P.kind == LOOKUP || (P.flags & 1)) { f.p = nullptr; f.dim = 0; f.rows = 1; }
-            else f.p = P.stage + (size_t)S.rowoff[i] * in;
-          }
-          walk(C, f, S.stack[warp], acc, &S.pool);
-          __syncwarp();
-          if (lane == 0) atomicSub(&S.pool.outstanding, 1);
-        }
-        const long long tw1 = clock64();
-        pool_steal(C, &S.pool, S.stack[warp], acc);
-        const long long tw2 = clock64();
-        if (lane == 0 && warp < 2) { S.phase[10 + 2 * warp] += (unsigned long long)(tw1 - tw0); S.phase[11 + 2 * warp] += (unsigned long long)(tw2 - tw1); }
-        flush_acc(C, acc, lane);
-        __syncthreads();
-        if (tid == 0) S.phase[14] += (unsigned long long)(clock64() - tw2);
+        if (!C.emit_ctas) emit_batch(C, P, tile, S, d, my_batch, stage_k, acc);
         AMP_PHASE(6);
       }
+      if (C.emit_ctas && tid == 0) st_rel(&P.emit_pub[tile], my_batch);     // hand the batch to this tile's emitter CTA
       if (d.flags & BATCH_TERMINATE) { running = false; round_open = false; }
       if (d.flags & BATCH_END_ROUND) round_open = false;
       (void)eval;
@@ -1458,6 +1482,34 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       st.n_grads_applied = S.ls.n_grads_applied; st.msgs = S.ls.msgs; st.batches = S.ls.batches; st.batch_rows = S.ls.batch_rows;
     }
     if (tid < 16) P.stats->phase_cycles[tid] = S.phase[tid];
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// emitter CTA (asynchronous mode): the partner of one tile.  It emits the tile's share of every batch while the tile
+// already stages and computes the next one.
+// ------------------------------------------------------------------------------------------------
+__device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int tile, TileShared& S, const unsigned long long t0) {
+  const int tid = threadIdx.x, warp = tid >> 5;
+  if (tid < POOL) S.pool.ready[tid] = 0;
+  if (tid < 16) S.phase[tid] = 0;
+  if (tid == 0) { S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
+  __syncthreads();
+  unsigned my_batch = 0;
+  WalkAcc acc = {0, 0};
+  for (;;) {
+    if (tid == 0) { S.ok = 1; if (!spin_until(C, t0, [&] { return ld_acq(&P.emit_pub[tile]) > my_batch; })) S.ok = 0; }
+    __syncthreads();
+    if (!S.ok) break;
+    if (warp == 0) load_batch_ctx(C, P, S, my_batch);
+    __syncthreads();
+    const BatchDesc d = S.desc;
+    my_batch++;
+    if (!S.ok) break;
+    if (d.count > 0) emit_batch(C, P, tile, S, d, my_batch, P.stage + (size_t)(my_batch & 1) * P.stage_floats, acc);
+    __syncthreads();
+    if (tid == 0) { __threadfence(); st_rel(&P.emit_done[tile], my_batch); }
+    if (d.flags & BATCH_TERMINATE) break;
   }
 }
 
@@ -1647,6 +1699,7 @@ __global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constan
   __syncthreads();
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);
+  else if (role.kind == 1) emitter_main(C, g_ppts[role.ppt], role.tile, SU.t, t0);
   else ppt_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
 }
 

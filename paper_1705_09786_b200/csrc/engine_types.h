@@ -75,7 +75,9 @@ struct DevPPT {
   Hdr* bhdr;                          // [BATCH_BLOCKS][MAX_BATCH_MSGS] headers of the most recent batches
   unsigned long long* sortbuf;
   float* dxpart;                      // [2][T][BM][in_dim] partial input gradients of the row tiles
-  float* stage;                       // [BM][max(in_dim, out_dim)] reduced input gradients / gathered rows
+  float* stage;                       // [2][BM][max(in_dim, out_dim)] reduced input gradients / gathered rows, by batch parity
+  long long stage_floats;
+  unsigned *emit_pub, *emit_done;     // per tile: batches handed to / finished by the tile's emitter CTA
   float* part2;                       // GRUCELL scratch
   unsigned* nbar;                     // barrier counter of the node's tiles
   PPTStats* stats;
@@ -118,7 +120,7 @@ struct Globals {                      // mutable run state in device memory (zer
   unsigned long long walk_cycles[N_NODE_TYPES * 2], walk_steps[N_NODE_TYPES * 2];   // profiling (tune bit 8)
 };
 
-struct Role { int ppt, tile; };
+struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: its emitter CTA
 
 struct Ctx {
   DevNode* nodes; int n_nodes;
@@ -139,6 +141,7 @@ struct Ctx {
   int mak, muf, det, eval, IT;
   int wide;                           // the graph has row-wise forks (Ungroup / Group)
   int bf16;                           // payloads rounded to bfloat16 at emission
+  int emit_ctas;                      // every tile has a partner CTA that emits its batches
   int tune;                           // experiment switches (environment AMPNET_TUNE): 2 no look-ahead, 4 no per-node counters
   float lr;
   unsigned long long timeout_ns;
