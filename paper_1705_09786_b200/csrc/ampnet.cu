@@ -355,7 +355,7 @@ size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
 
 // Placement: row tiles per PPT node.  Enough tiles that a tile's weights + accumulators + staging fit in
 // shared memory, then the remaining CTAs in proportion to the nodes' multiply-add volume.
-ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles, bool emitters, int tiles_cap) {
+ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles, int emitters, int tiles_cap) {
   cudaFuncAttributes fa{};
   size_t static_smem = 40 * 1024;
   if (cudaFuncGetAttributes(&fa, ampnet_engine) == cudaSuccess) static_smem = fa.sharedSizeBytes;
@@ -398,10 +398,11 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   roles.push_back(Role{-1, 0, 0, 0});
   for (int p = 0; p < (int)g->ppts.size(); p++)
     for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t, 0, 0});
-  if (emitters) {
-    if (2 * used - 1 > n_ctas) return AMPNET_EOVERFLOW;          // the caller retries with fewer tiles or without emitters
+  if (emitters > 0) {
+    if (1 + (used - 1) * (1 + emitters) > n_ctas) return AMPNET_EOVERFLOW;   // the caller retries with fewer emitters / tiles
     for (int p = 0; p < (int)g->ppts.size(); p++)
-      for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t, 1, 0});
+      for (int t = 0; t < g->ppts[p].T; t++)
+        for (int e = 0; e < emitters; e++) roles.push_back(Role{p, t, 1, e});
   }
   return AMPNET_OK;
 }
@@ -424,12 +425,22 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   // Asynchronous runs pair every tile with an emitter CTA when the SMs allow it (with fewer tiles if need be).
   int tune = 0;
   if (const char* e = getenv("AMPNET_TUNE")) tune = atoi(e);
-  bool emitters = !det && !(tune & 32);
-  ampnet_status_t st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles, emitters, 0);
-  if (st == AMPNET_EOVERFLOW && emitters) st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles, true, 8);
-  if (st == AMPNET_EOVERFLOW && emitters) { emitters = false; st = place(g, n_ctas, cfg ? cfg->max_batch_rows : 0, R.roles, false, 0); }
+  int emit_ctas = (!det && !(tune & 32)) ? ((tune & 64) ? 1 : 2) : 0;
+  const int mbr = cfg ? cfg->max_batch_rows : 0;
+  // Two emitter CTAs per tile if the SMs allow it, with as many tiles per node as fit; then one; then none.
+  ampnet_status_t st = AMPNET_EOVERFLOW;
+  const int caps[] = {0, 12, 10, 8, 7, 6, 5, 4};
+  for (; emit_ctas > 0 && st == AMPNET_EOVERFLOW; emit_ctas--) {
+    for (int cap : caps) {
+      st = place(g, n_ctas, mbr, R.roles, emit_ctas, cap);
+      if (st != AMPNET_EOVERFLOW) break;
+    }
+    if (st != AMPNET_EOVERFLOW) break;
+  }
+  if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0, 0); }
   if (st != AMPNET_OK) return st;
-  R.ctx.emit_ctas = emitters ? 1 : 0;
+  const int depth = emit_ctas > 0 ? emit_ctas + 1 : 2;
+  R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth;
   n_ctas = (int)R.roles.size();
   DeviceArena &C = g->ctl, &B = g->bulk;
   C.used = B.used = 0;
@@ -460,7 +471,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
       P.zc = B.take<float>(keys * P.rows_max * P.out_dim);
       P.rc = B.take<float>(keys * P.rows_max * P.out_dim);
       P.cc = B.take<float>(keys * P.rows_max * P.out_dim);
-      P.part2 = B.take<float>((size_t)2 * (P.T + 1) * P.BM * P.in_dim);
+      P.part2 = B.take<float>((size_t)depth * (P.T + 1) * P.BM * P.in_dim);
     }
     P.vcache = B.take<int>(keys);
     const unsigned cap = pow2_at_least(2ull * keys);
@@ -477,11 +488,12 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.batch_pub = C.take<unsigned>(1);
     P.bhdr = B.take<Hdr>((size_t)BATCH_BLOCKS * MAX_BATCH_MSGS);
     P.sortbuf = B.take<unsigned long long>(cap);
-    if ((P.T > 1 && H.kind != LOOKUP) || H.kind == GRUCELL) P.dxpart = B.take<float>((size_t)2 * P.T * P.BM * P.in_dim);
+    if ((P.T > 1 && H.kind != LOOKUP) || H.kind == GRUCELL) P.dxpart = B.take<float>((size_t)depth * P.T * P.BM * P.in_dim);
     P.stage_floats = (long long)P.BM * std::max(P.in_dim, P.out_dim);
-    P.stage = B.take<float>((size_t)2 * P.stage_floats);
+    P.stage = B.take<float>((size_t)depth * P.stage_floats);
     P.emit_pub = C.take<unsigned>(P.T);
-    P.emit_done = C.take<unsigned>(P.T);
+    P.emit_fin = C.take<unsigned>(P.T);
+    P.emit_done = C.take<unsigned>((size_t)P.T * std::max(1, emit_ctas));
     P.nbar = C.take<unsigned>(1);
     P.stats = C.take<PPTStats>(1);
     P.update_log = B.take<int>(g->update_log_cap); P.update_log_cap = g->update_log_cap;

@@ -1098,8 +1098,8 @@ __device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile,
       // Sum the tiles' partial input gradients (tile order) for the rows this tile emits; every thread keeps
       // all T loads of an element in flight.
       const size_t pstride = (size_t)P.BM * in;
-      const float* pa = P.dxpart + (size_t)(my_batch & 1) * P.T * pstride;
-      const float* pb = P.kind == GRUCELL ? P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride : nullptr;
+      const float* pa = P.dxpart + (size_t)(my_batch % (unsigned)C.depth) * P.T * pstride;
+      const float* pb = P.kind == GRUCELL ? P.part2 + (size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) * pstride : nullptr;
       const float* dirb = pb ? pb + (size_t)P.T * pstride : nullptr;
       const int H = out;
       for (int i = split ? 0 : tile; i < count; i += split ? 1 : P.T) {
@@ -1248,10 +1248,14 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       AMP_PHASE(d.count > 0 ? 1 : 0);
       const int count = d.count, dir = d.dir;
       if (!S.ok) { running = false; break; }
-      float* const stage_k = P.stage + (size_t)(my_batch & 1) * P.stage_floats;
+      float* const stage_k = P.stage + (size_t)(my_batch % (unsigned)C.depth) * P.stage_floats;
       if (C.emit_ctas && count > 0) {
-        // the per-batch buffers of this parity were last used two batches ago: wait until that batch has been emitted
-        if (tid == 0 && !spin_until(C, t0, [&] { return ld_acq(&P.emit_done[tile]) + 2u >= my_batch; })) S.ok = 0;
+        // the per-batch buffers are reused every `depth` batches: wait until their previous user has been emitted
+        if (tid == 0 && my_batch > (unsigned)C.depth) {
+          const unsigned j = my_batch - 1u - (unsigned)C.depth;           // the batch that used these buffers before
+          const unsigned* done = &P.emit_done[tile * C.emit_ctas + (int)(j % (unsigned)C.emit_ctas)];
+          if (!spin_until(C, t0, [&] { return ld_acq(done) >= j + 1u; })) S.ok = 0;
+        }
         __syncthreads();
         if (!S.ok) { running = false; break; }
       }
@@ -1279,7 +1283,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           }
           __syncthreads();
           if (!(P.flags & 1)) {
-            float* dst = P.T > 1 ? P.dxpart + ((size_t)(my_batch & 1) * P.T + tile) * P.BM * in : stage_k;
+            float* dst = P.T > 1 ? P.dxpart + ((size_t)(my_batch % (unsigned)C.depth) * P.T + tile) * P.BM * in : stage_k;
             AMP_DISPATCH_J(P.J, (tile_dW<J>(M.Ds, P.R, nb, M.Ws, in, R, in, dst)));
           }
           tile_accum(M.Ds, P.R, nb, M.Xs, in, M.As, in, R, in);
@@ -1331,10 +1335,10 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           }
         } else {
           const size_t pstride = (size_t)P.BM * in;
-          float* part1 = P.part2 + ((size_t)(my_batch & 1) * (P.T + 1) + tile) * pstride;
-          const float* part1_all = P.part2 + (size_t)(my_batch & 1) * (P.T + 1) * pstride;
-          float* dirbuf = P.part2 + ((size_t)(my_batch & 1) * (P.T + 1) + P.T) * pstride;     // [BM][H]
-          float* part2 = P.dxpart + ((size_t)(my_batch & 1) * P.T + tile) * pstride;
+          float* part1 = P.part2 + ((size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) + tile) * pstride;
+          const float* part1_all = P.part2 + (size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) * pstride;
+          float* dirbuf = P.part2 + ((size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) + P.T) * pstride;     // [BM][H]
+          float* part2 = P.dxpart + ((size_t)(my_batch % (unsigned)C.depth) * P.T + tile) * pstride;
           float *dpz = M.Ds, *dpr = M.Ds + BR, *dpc = M.Ds + 2 * BR, *dirp = M.Ds + 3 * BR;
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
@@ -1459,7 +1463,10 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         if (!C.emit_ctas) emit_batch(C, P, tile, S, d, my_batch, stage_k, acc);
         AMP_PHASE(6);
       }
-      if (C.emit_ctas && tid == 0) st_rel(&P.emit_pub[tile], my_batch);     // hand the batch to this tile's emitter CTA
+      if (C.emit_ctas && tid == 0) {                                        // hand the batch to this tile's emitter CTAs
+        st_rel(&P.emit_pub[tile], my_batch);
+        if (d.flags & BATCH_TERMINATE) st_rel(&P.emit_fin[tile], 1u);
+      }
       if (d.flags & BATCH_TERMINATE) { running = false; round_open = false; }
       if (d.flags & BATCH_END_ROUND) round_open = false;
       (void)eval;
@@ -1489,27 +1496,31 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
 // emitter CTA (asynchronous mode): the partner of one tile.  It emits the tile's share of every batch while the tile
 // already stages and computes the next one.
 // ------------------------------------------------------------------------------------------------
-__device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int tile, TileShared& S, const unsigned long long t0) {
+__device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int tile, const int which, TileShared& S,
+                                          const unsigned long long t0) {
   const int tid = threadIdx.x, warp = tid >> 5;
   if (tid < POOL) S.pool.ready[tid] = 0;
   if (tid < 16) S.phase[tid] = 0;
   if (tid == 0) { S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
   __syncthreads();
-  unsigned my_batch = 0;
+  unsigned my_batch = (unsigned)which;          // this emitter takes batches which, which + E, which + 2E, ...
   WalkAcc acc = {0, 0};
   for (;;) {
-    if (tid == 0) { S.ok = 1; if (!spin_until(C, t0, [&] { return ld_acq(&P.emit_pub[tile]) > my_batch; })) S.ok = 0; }
+    // every emitter of the tile sees the terminating batch: emit_pub counts all batches, the last one is the marker
+    if (tid == 0) { S.ok = 1; if (!spin_until(C, t0, [&] { return ld_acq(&P.emit_pub[tile]) > my_batch || ld_acq(&P.emit_fin[tile]) != 0u; })) S.ok = 0; }
     __syncthreads();
     if (!S.ok) break;
+    if (tid == 0) S.tail_snap[0] = ld_acq(&P.emit_pub[tile]);
+    __syncthreads();
+    if (S.tail_snap[0] <= my_batch) break;                     // finished and nothing left for this emitter
     if (warp == 0) load_batch_ctx(C, P, S, my_batch);
     __syncthreads();
     const BatchDesc d = S.desc;
-    my_batch++;
     if (!S.ok) break;
-    if (d.count > 0) emit_batch(C, P, tile, S, d, my_batch, P.stage + (size_t)(my_batch & 1) * P.stage_floats, acc);
+    if (d.count > 0) emit_batch(C, P, tile, S, d, my_batch + 1u, P.stage + (size_t)((my_batch + 1u) % (unsigned)C.depth) * P.stage_floats, acc);
     __syncthreads();
-    if (tid == 0) { __threadfence(); st_rel(&P.emit_done[tile], my_batch); }
-    if (d.flags & BATCH_TERMINATE) break;
+    if (tid == 0) { __threadfence(); st_rel(&P.emit_done[tile * C.emit_ctas + which], my_batch + 1u); }
+    my_batch += (unsigned)C.emit_ctas;
   }
 }
 
@@ -1699,7 +1710,7 @@ __global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constan
   __syncthreads();
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);
-  else if (role.kind == 1) emitter_main(C, g_ppts[role.ppt], role.tile, SU.t, t0);
+  else if (role.kind == 1) emitter_main(C, g_ppts[role.ppt], role.tile, role.pad, SU.t, t0);
   else ppt_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
 }
 

@@ -77,7 +77,8 @@ struct DevPPT {
   float* dxpart;                      // [2][T][BM][in_dim] partial input gradients of the row tiles
   float* stage;                       // [2][BM][max(in_dim, out_dim)] reduced input gradients / gathered rows, by batch parity
   long long stage_floats;
-  unsigned *emit_pub, *emit_done;     // per tile: batches handed to / finished by the tile's emitter CTA
+  unsigned *emit_pub, *emit_fin;      // per tile: batches handed to its emitter CTAs; set once the last one is out
+  unsigned* emit_done;                // [tile][emitter]: last batch (index + 1) the emitter has finished
   float* part2;                       // GRUCELL scratch
   unsigned* nbar;                     // barrier counter of the node's tiles
   PPTStats* stats;
@@ -120,7 +121,7 @@ struct Globals {                      // mutable run state in device memory (zer
   unsigned long long walk_cycles[N_NODE_TYPES * 2], walk_steps[N_NODE_TYPES * 2];   // profiling (tune bit 8)
 };
 
-struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: its emitter CTA
+struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of its emitter CTAs (pad = which one)
 
 struct Ctx {
   DevNode* nodes; int n_nodes;
@@ -141,7 +142,8 @@ struct Ctx {
   int mak, muf, det, eval, IT;
   int wide;                           // the graph has row-wise forks (Ungroup / Group)
   int bf16;                           // payloads rounded to bfloat16 at emission
-  int emit_ctas;                      // every tile has a partner CTA that emits its batches
+  int emit_ctas;                      // emitter CTAs per tile (0: tiles emit themselves)
+  int depth;                          // per-batch buffers (partials, staging rows) are reused every `depth` batches
   int tune;                           // experiment switches (environment AMPNET_TUNE): 2 no look-ahead, 4 no per-node counters
   float lr;
   unsigned long long timeout_ns;
