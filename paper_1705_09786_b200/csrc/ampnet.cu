@@ -399,7 +399,8 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   for (int p = 0; p < (int)g->ppts.size(); p++)
     for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t, 0, 0});
   if (emitters > 0) {
-    if (1 + (used - 1) * (1 + emitters) > n_ctas) return AMPNET_EOVERFLOW;   // the caller retries with fewer emitters / tiles
+    if (1 + (used - 1) * (1 + emitters) + (int)g->ppts.size() > n_ctas) return AMPNET_EOVERFLOW;   // retried with fewer emitters / tiles
+    for (int p = 0; p < (int)g->ppts.size(); p++) roles.push_back(Role{p, 0, 2, 0});                 // one scheduler CTA per node
     for (int p = 0; p < (int)g->ppts.size(); p++)
       for (int t = 0; t < g->ppts[p].T; t++)
         for (int e = 0; e < emitters; e++) roles.push_back(Role{p, t, 1, e});
@@ -440,7 +441,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0, 0); }
   if (st != AMPNET_OK) return st;
   const int depth = emit_ctas > 0 ? emit_ctas + 1 : 2;
-  R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth;
+  R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth; R.ctx.sched_ctas = emit_ctas > 0 ? 1 : 0;
   n_ctas = (int)R.roles.size();
   DeviceArena &C = g->ctl, &B = g->bulk;
   C.used = B.used = 0;
@@ -493,6 +494,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.stage = B.take<float>((size_t)depth * P.stage_floats);
     P.emit_pub = C.take<unsigned>(P.T);
     P.emit_fin = C.take<unsigned>(P.T);
+    P.fetched = C.take<unsigned>(1);
     P.emit_done = C.take<unsigned>((size_t)P.T * std::max(1, emit_ctas));
     P.nbar = C.take<unsigned>(1);
     P.stats = C.take<PPTStats>(1);

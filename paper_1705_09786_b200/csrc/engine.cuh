@@ -1035,6 +1035,25 @@ __device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, con
   return C.inst.dense + (long long)h.inst * C.inst.dense_dim;         // fed directly by a dense-row source
 }
 
+__device__ __forceinline__ void write_leader_stats(DevPPT& P, TileShared& S) {      // whole CTA
+  const int tid = threadIdx.x;
+  if (tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
+  if (tid == 0) {
+    PPTStats& st = *P.stats;
+    st.max_staleness = S.max_stale; st.log_n = S.ls.log_n; st.n_updates = S.ls.n_updates;
+    st.n_grads_applied = S.ls.n_grads_applied; st.msgs = S.ls.msgs; st.batches = S.ls.batches; st.batch_rows = S.ls.batch_rows;
+  }
+}
+
+__device__ __forceinline__ void init_leader_state(TileShared& S) {                 // whole CTA, before a barrier
+  const int tid = threadIdx.x;
+  if (tid == 0) {
+    S.ls.head[0] = S.ls.head[1] = 0; S.ls.sched_w = S.ls.batch_w = 0; S.ls.n_acc = 0; S.ls.version = 0; S.max_stale = 0;
+    S.ls.log_n = 0; S.ls.n_updates = S.ls.n_grads_applied = S.ls.msgs = S.ls.batches = S.ls.batch_rows = 0;
+  }
+  if (tid < 64) S.stale_hist[tid] = 0;
+}
+
 // Warp 0 of a CTA: descriptor, headers, keys, row offsets and row pointers of batch `batch` into shared memory.
 __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared& S, const unsigned my_batch) {
   const int lane = threadIdx.x & 31;
@@ -1217,7 +1236,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       AMP_PHASE(7);
       if (tid == 0) S.ok = 1;
       __syncthreads();
-      if (tile == 0) {
+      if (tile == 0 && !C.sched_ctas) {
         if (warp == 0) {
           unsigned it = 0;
           for (;;) {
@@ -1242,6 +1261,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       __syncthreads();
       if (!S.ok || aborted(C)) { running = false; break; }
       if (warp == 0) load_batch_ctx(C, P, S, my_batch);
+      if (C.sched_ctas && tile == 0 && tid == 0) st_rel(P.fetched, my_batch + 1u);   // the scheduler may form the next batch
       __syncthreads();
       const BatchDesc d = S.desc;
       my_batch++;
@@ -1453,7 +1473,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
         else __syncthreads();
         AMP_PHASE(5);
-        if (tile == 0 && warp == 0 && !C.det && !(C.tune & 2)) {       // look ahead: form the next batch now
+        if (tile == 0 && warp == 0 && !C.det && !C.sched_ctas && !(C.tune & 2)) {   // look ahead: form the next batch now
           unsigned bw = 0;
           if (lane == 0) bw = S.ls.batch_w;
           const long long tq = clock64();
@@ -1482,12 +1502,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       for (int i = tid; i < R; i += THREADS) P.b[m * out + r_begin + i] = M.bs[m * P.R + i];
     }
   if (tile == 0) {
-    if (tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
-    if (tid == 0) {
-      PPTStats& st = *P.stats;
-      st.max_staleness = S.max_stale; st.log_n = S.ls.log_n; st.n_updates = S.ls.n_updates;
-      st.n_grads_applied = S.ls.n_grads_applied; st.msgs = S.ls.msgs; st.batches = S.ls.batches; st.batch_rows = S.ls.batch_rows;
-    }
+    if (!C.sched_ctas) write_leader_stats(P, S);
     if (tid < 16) P.stats->phase_cycles[tid] = S.phase[tid];
   }
 }
@@ -1522,6 +1537,42 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int til
     if (tid == 0) { __threadfence(); st_rel(&P.emit_done[tile * C.emit_ctas + which], my_batch + 1u); }
     my_batch += (unsigned)C.emit_ctas;
   }
+}
+
+// ------------------------------------------------------------------------------------------------
+// scheduler CTA (asynchronous mode): the leader of one PPT node on an SM of its own.  It forms the next micro-batch
+// as soon as tile 0 has fetched the previous one, so that batch formation overlaps the tiles' work.
+// ------------------------------------------------------------------------------------------------
+__device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared& S, const unsigned long long t0) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  init_leader_state(S);
+  __syncthreads();
+  if (warp == 0) {
+    unsigned it = 0;
+    for (;;) {
+      // at most one batch ahead of what tile 0 has fetched
+      unsigned go = 0, bw = 0;
+      if (lane == 0) { bw = S.ls.batch_w; go = ld_acq(P.fetched) >= bw; }
+      bw = warp_uniform(bw);
+      bool progressed = false;
+      if (warp_uniform(go)) {
+        progressed = leader_try_schedule(C, P, S);
+        unsigned fin = 0;
+        if (lane == 0) fin = progressed && (P.batches[bw & P.batch_mask].flags & BATCH_TERMINATE);
+        if (warp_uniform(fin)) break;
+      }
+      if (progressed) { it = 0; continue; }
+      if ((++it & 15u) == 0) {
+        if (aborted_warp(C)) break;
+        unsigned late = 0;
+        if (lane == 0) late = gtime() - t0 > C.timeout_ns;
+        if (warp_uniform(late)) { if (lane == 0) fail(C, ST_TIMEOUT, P.node, 3); break; }
+      }
+      __nanosleep(it < 16 ? 20 : 100);
+    }
+  }
+  __syncthreads();
+  write_leader_stats(P, S);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1711,6 +1762,7 @@ __global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constan
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);
   else if (role.kind == 1) emitter_main(C, g_ppts[role.ppt], role.tile, role.pad, SU.t, t0);
+  else if (role.kind == 2) scheduler_main(C, g_ppts[role.ppt], SU.t, t0);
   else ppt_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
 }
 

@@ -79,6 +79,7 @@ struct DevPPT {
   long long stage_floats;
   unsigned *emit_pub, *emit_fin;      // per tile: batches handed to its emitter CTAs; set once the last one is out
   unsigned* emit_done;                // [tile][emitter]: last batch (index + 1) the emitter has finished
+  unsigned* fetched;                  // batches tile 0 has fetched (paces the scheduler CTA)
   float* part2;                       // GRUCELL scratch
   unsigned* nbar;                     // barrier counter of the node's tiles
   PPTStats* stats;
@@ -121,7 +122,7 @@ struct Globals {                      // mutable run state in device memory (zer
   unsigned long long walk_cycles[N_NODE_TYPES * 2], walk_steps[N_NODE_TYPES * 2];   // profiling (tune bit 8)
 };
 
-struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of its emitter CTAs (pad = which one)
+struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of its emitter CTAs (pad = which one), 2: the node's scheduler CTA
 
 struct Ctx {
   DevNode* nodes; int n_nodes;
@@ -143,6 +144,7 @@ struct Ctx {
   int wide;                           // the graph has row-wise forks (Ungroup / Group)
   int bf16;                           // payloads rounded to bfloat16 at emission
   int emit_ctas;                      // emitter CTAs per tile (0: tiles emit themselves)
+  int sched_ctas;                     // every PPT node has a scheduler CTA (its leader) of its own
   int depth;                          // per-batch buffers (partials, staging rows) are reused every `depth` batches
   int tune;                           // experiment switches (environment AMPNET_TUNE): 2 no look-ahead, 4 no per-node counters
   float lr;
