@@ -109,6 +109,7 @@ struct Frame {
   int inst, seq, slot, it, u, port, rows, flags;
   int dim, ld;
   int nsum, sstride;    // payload element (r, i) = sum over j < nsum of p[j * sstride + r * ld + i]
+  long long ibase, ebase; // first position / first edge of the instance in the structure tables (loaded once per message)
   int part, nparts;     // nparts > 1: the rows of the first row-wise fork are shared among nparts CTAs; this walker takes
                         // rows j = part (mod nparts); until that fork only part 0 has side effects (the others are shadows)
   const float* p;       // payload rows (device memory); nullptr = zeros
@@ -330,7 +331,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (key < 0) return;
           float* g = n.jbuf + key * n.jstride;
           if (n.type == LOSS_CE) {
-            int label = I.labels_i[I.labels_per_node ? IBASE(f.inst) + f.u : f.inst];
+            int label = I.labels_i[I.labels_per_node ? f.ibase + f.u : f.inst];
             float mx = -3.4e38f; int arg = 0x7fffffff;
             for (int j = lane; j < n.in_dim; j += 32) { float v = ld_payload(f.p, f.nsum, f.sstride, j); if (v > mx) { mx = v; arg = j; } }
             for (int o = 16; o; o >>= 1) {
@@ -360,8 +361,8 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (f.dir == FWD) {
             int k = 0;
             switch (n.fn) {
-              case 1: k = f.u < (int)(I.offsets[f.inst + 1] - IBASE(f.inst)) ? 0 : 1; break;
-              case 2: k = f.u == I.root[f.inst] ? 0 : 1; break;
+              case 1: k = f.u < (int)(I.offsets[f.inst + 1] - f.ibase) ? 0 : 1; break;
+              case 2: k = I.parent[f.ibase + f.u] < 0 ? 0 : 1; break;      // the root has no parent
               case 3: k = f.u; break;
               case 4: k = f.it < n.fn_arg ? 0 : 1; break;
             }
@@ -392,12 +393,12 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
         case ISU:
           if (f.dir == FWD) {
             if (n.fn == 1) f.u += 1;
-            else if (n.fn == 2) { f.port = I.child_slot[IBASE(f.inst) + f.u]; f.u = I.parent[IBASE(f.inst) + f.u]; }
+            else if (n.fn == 2) { f.port = I.child_slot[f.ibase + f.u]; f.u = I.parent[f.ibase + f.u]; }
             else f.it += 1;
             to_succ(f, n, 0);
           } else {
             if (n.fn == 1) f.u -= 1;
-            else if (n.fn == 2) { f.u = f.port == 0 ? I.left[IBASE(f.inst) + f.u] : I.right[IBASE(f.inst) + f.u]; f.port = 0; }
+            else if (n.fn == 2) { f.u = f.port == 0 ? I.left[f.ibase + f.u] : I.right[f.ibase + f.u]; f.port = 0; }
             else f.it -= 1;
             to_pred(f, n, 0);
           }
@@ -451,12 +452,12 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
         case GROUP:
           if (f.dir == FWD) {
             int gkey = 0, member = 0, count = 1;
-            const long long ebase = I.edge_off ? I.edge_off[f.inst] : 0;
+            const long long ebase = f.ebase;
             if (n.fn == 1) { int c = I.etype[ebase + f.u]; gkey = c; member = I.rank_type[ebase + f.u];
                              const long long* to = I.type_off + (long long)f.inst * I.NT + c; count = (int)(to[1] - to[0]); }
             else if (n.fn == 2) { int v = I.edst[ebase + f.u]; gkey = v; member = I.rank_in[ebase + f.u];
-                                  count = (int)(I.in_off[IBASE(f.inst) + v + 1] - I.in_off[IBASE(f.inst) + v]); }
-            else { gkey = 0; member = f.u; count = (int)(I.offsets[f.inst + 1] - IBASE(f.inst)); }
+                                  count = (int)(I.in_off[f.ibase + v + 1] - I.in_off[f.ibase + v]); }
+            else { gkey = 0; member = f.u; count = (int)(I.offsets[f.inst + 1] - f.ibase); }
             long long key = key_of(C, f.node, f.slot, f.it, gkey, n.U_out);
             if (key < 0) return;
             if (member >= n.rows_out || count > n.rows_out) { fail(C, ST_OVERFLOW, f.node, member); return; }
@@ -474,10 +475,10 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
               if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             f.nparts = 1; f.part = 0;
-            const long long ebase = I.edge_off ? I.edge_off[f.inst] : 0;
+            const long long ebase = f.ebase;
             int mu;
             if (n.fn == 1) mu = I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i];
-            else if (n.fn == 2) mu = I.in_list[I.in_off[IBASE(f.inst) + f.u] + i];
+            else if (n.fn == 2) mu = I.in_list[I.in_off[f.ibase + f.u] + i];
             else mu = i;
             (void)ebase;
             f.p = f.p ? f.p + (size_t)i * f.ld : nullptr; f.rows = 1; f.u = mu;
@@ -499,9 +500,9 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             cont = true;
           } else {
             int gkey, row, expected;
-            if (n.fn == 2) { const long long ebase = I.edge_off[f.inst]; gkey = I.etype[ebase + f.u]; row = I.rank_type[ebase + f.u];
+            if (n.fn == 2) { const long long ebase = f.ebase; gkey = I.etype[ebase + f.u]; row = I.rank_type[ebase + f.u];
                              const long long* to = I.type_off + (long long)f.inst * I.NT + gkey; expected = (int)(to[1] - to[0]); }
-            else { gkey = 0; row = f.u; expected = (int)(I.offsets[f.inst + 1] - IBASE(f.inst)); }
+            else { gkey = 0; row = f.u; expected = (int)(I.offsets[f.inst + 1] - f.ibase); }
             long long key = key_of(C, f.node, f.slot, f.it, gkey, n.U_in);
             if (key < 0) return;
             if (row >= n.rows_in) { fail(C, ST_OVERFLOW, f.node, row); return; }
@@ -516,7 +517,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           break;
         case FLATMAP: {
           if (f.dir == FWD) {
-            const long long* oo = I.out_off + IBASE(f.inst) + f.u;
+            const long long* oo = I.out_off + f.ibase + f.u;
             int deg = (int)(oo[1] - oo[0]);
             int i = f.iter;
             if (deg > 0) {
@@ -528,9 +529,9 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
               cont = true;
             }
           } else {
-            const long long ebase = I.edge_off[f.inst];
+            const long long ebase = f.ebase;
             int v = I.esrc[ebase + f.u], member = I.rank_out[ebase + f.u];
-            int deg = (int)(I.out_off[IBASE(f.inst) + v + 1] - I.out_off[IBASE(f.inst) + v]);
+            int deg = (int)(I.out_off[f.ibase + v + 1] - I.out_off[f.ibase + v]);
             long long key = key_of(C, f.node, f.slot, f.it, v, n.U_in);
             if (key < 0) return;
             const int maxdeg = (int)(n.jstride / n.in_dim) - 1;
@@ -1156,6 +1157,7 @@ __device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile,
       f.iter = 0; f.inst = h.inst; f.seq = h.seq; f.slot = h.slot; f.it = h.it; f.u = h.u; f.port = h.port;
       f.rows = h.rows; f.flags = h.flags; f.nsum = 1; f.sstride = 0;
       f.part = split ? part : 0; f.nparts = split ? P.T : 1;
+      f.ibase = C.inst.offsets ? C.inst.offsets[h.inst] : 0; f.ebase = C.inst.edge_off ? C.inst.edge_off[h.inst] : 0;
       if (dir == FWD) {
         f.node = N.succ_node[0]; f.aport = N.succ_port[0]; f.dir = FWD; f.dim = out; f.ld = out;
         f.p = P.kind == LOOKUP ? stage + (size_t)S.rowoff[i] * out
@@ -1701,6 +1703,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
         f.node = sn.succ_node[0]; f.aport = sn.succ_port[0]; f.dir = FWD; f.iter = 0;
         f.inst = inst; f.seq = S.admit_seq; f.slot = slot; f.it = 0; f.u = 0; f.port = 0; f.rows = 1;
         f.flags = C.eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr; f.nsum = 1; f.sstride = 0; f.part = 0; f.nparts = 1;
+        f.ibase = I.offsets ? I.offsets[inst] : 0; f.ebase = I.edge_off ? I.edge_off[inst] : 0;
         switch (sn.fn) {
           case 1: f.p = I.dense + (long long)inst * I.dense_dim; f.dim = I.dense_dim; f.ld = I.dense_dim; break;
           case 2: f.u = k; break;
