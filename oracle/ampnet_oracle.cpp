@@ -180,6 +180,9 @@ struct Engine {
   // run configuration
   int mak = 1, muf = 1;
   real lr = 0;
+  // optimiser applied at a local update (App. A: SGD, momentum-SGD, Adam): 0 SGD, 1 momentum, 2 Adam
+  int opt = 0;
+  real mu = 0.9, beta1 = 0.9, beta2 = 0.999, eps = 1e-8;
   // schedule state
   std::vector<std::vector<Msg>> inbox_a, inbox_b;
   std::vector<std::vector<Msg>>* target = nullptr;
@@ -226,7 +229,31 @@ struct PPTBase : Node {
   int n_acc = 0, version = 0;
   bool is_ppt() const override { return true; }
   int muf() const { return muf_override > 0 ? muf_override : E->muf; }
-  virtual void apply(real scale) = 0;     // theta -= scale * A; A = 0
+  virtual void apply(real inv_n) = 0;     // theta <- optimiser step on the mean gradient A * inv_n; A = 0
+  // Optimiser state per parameter tensor, kept across epochs; opt_t counts this node's updates (Adam bias correction).
+  std::vector<std::vector<real>> mom, var;
+  long long opt_t = 0;
+  void reset_optimizer() { mom.clear(); var.clear(); opt_t = 0; }
+  void opt_step(std::vector<real>& P, std::vector<real>& A, int w, size_t k, real inv_n) {
+    const real g = A[k] * inv_n;
+    A[k] = 0;
+    if (E->opt == 0) { P[k] -= E->lr * g; return; }
+    if ((int)mom.size() <= w) { mom.resize(w + 1); var.resize(w + 1); }
+    if (mom[w].size() != P.size()) { mom[w].assign(P.size(), 0); var[w].assign(P.size(), 0); }
+    if (E->opt == 1) {                       // v <- mu v + g; theta <- theta - lr v
+      real& v = mom[w][k];
+      v = E->mu * v + g;
+      P[k] -= E->lr * v;
+    } else {                                 // Adam with bias correction, t = number of updates of this node
+      real& m = mom[w][k];
+      real& v = var[w][k];
+      m = E->beta1 * m + (1 - E->beta1) * g;
+      v = E->beta2 * v + (1 - E->beta2) * g * g;
+      const real mh = m / (1 - std::pow(E->beta1, (real)opt_t));
+      const real vh = v / (1 - std::pow(E->beta2, (real)opt_t));
+      P[k] -= E->lr * mh / (std::sqrt(vh) + E->eps);
+    }
+  }
   void record_staleness(int v_fwd) {
     int s = version - v_fwd;
     st.stale_hist[std::min(s, 63)]++;
@@ -236,7 +263,8 @@ struct PPTBase : Node {
   void maybe_update() { if (n_acc >= muf()) do_update(); }
   void do_update() {
     if (n_acc == 0) return;
-    apply(E->lr / (real)n_acc);
+    opt_t++;
+    apply((real)1 / (real)n_acc);
     st.n_updates++;
     st.n_grads_applied += n_acc;
     st.update_log.push_back(n_acc);
@@ -301,9 +329,9 @@ struct Linear : PPTBase {
     maybe_update();
     E->emit_bwd(id, 0, o);
   }
-  void apply(real scale) override {
-    for (size_t k = 0; k < W.size(); k++) { W[k] -= scale * AW[k]; AW[k] = 0; }
-    for (size_t k = 0; k < b.size(); k++) { b[k] -= scale * Ab[k]; Ab[k] = 0; }
+  void apply(real inv_n) override {
+    for (size_t k = 0; k < W.size(); k++) opt_step(W, AW, 0, k, inv_n);
+    for (size_t k = 0; k < b.size(); k++) opt_step(b, Ab, 1, k, inv_n);
   }
 };
 
@@ -353,13 +381,9 @@ struct Lookup : PPTBase {        // in_dim = vocabulary, out_dim = embedding wid
     Msg o; o.s = m.s;                 // no input gradient: the message goes home to the controller
     E->emit_bwd(id, 0, o);
   }
-  void apply(real scale) override {   // touched rows only
+  void apply(real inv_n) override {   // touched rows only (their moments too: untouched rows do not decay)
     for (int idx : touched_list) {
-      for (int j = 0; j < out_dim; j++) {
-        size_t k = (size_t)idx * out_dim + j;
-        Emb[k] -= scale * AE[k];
-        AE[k] = 0;
-      }
+      for (int j = 0; j < out_dim; j++) opt_step(Emb, AE, 0, (size_t)idx * out_dim + j, inv_n);
       touched[idx] = 0;
     }
     touched_list.clear();
@@ -459,11 +483,11 @@ struct GRUCell : PPTBase {       // x = [a; h], in_dim = 2H, out_dim = H
     maybe_update();
     E->emit_bwd(id, 0, o);
   }
-  void apply(real scale) override {
+  void apply(real inv_n) override {
     std::vector<real>* P[6] = {&Wz, &Wr, &Wc, &bz, &br, &bc};
     std::vector<real>* A[6] = {&AWz, &AWr, &AWc, &Abz, &Abr, &Abc};
     for (int t = 0; t < 6; t++)
-      for (size_t k = 0; k < P[t]->size(); k++) { (*P[t])[k] -= scale * (*A[t])[k]; (*A[t])[k] = 0; }
+      for (size_t k = 0; k < P[t]->size(); k++) opt_step(*P[t], *A[t], t, k, inv_n);
   }
 };
 
@@ -1099,6 +1123,16 @@ int oracle_run_epoch(void* h, int split, int mak, int muf, double lr, const int6
                      int flush, oracle_stats_t* out, double* per_instance_loss) {
   if (mak < 1 || muf < 1) return 1;
   return static_cast<Oracle*>(h)->run_epoch(split, mak, muf, lr, order, n_order, flush, out, per_instance_loss);
+}
+
+// kind: 0 SGD, 1 momentum-SGD (v <- mu v + g, theta -= lr v), 2 Adam (bias-corrected); state is kept across epochs.
+int oracle_set_optimizer(void* h, int kind, double mu, double beta1, double beta2, double eps, int reset_state) {
+  Oracle* O = static_cast<Oracle*>(h);
+  if (kind < 0 || kind > 2) return 1;
+  O->E.opt = kind; O->E.mu = (real)mu; O->E.beta1 = (real)beta1; O->E.beta2 = (real)beta2; O->E.eps = (real)eps;
+  if (reset_state)
+    for (auto& n : O->E.nodes) if (n->is_ppt()) static_cast<PPTBase*>(n.get())->reset_optimizer();
+  return 0;
 }
 
 int oracle_eval(void* h, int split, double* mean_loss, double* accuracy, double* per_instance_loss) {

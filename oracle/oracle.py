@@ -52,6 +52,7 @@ def _load(real):
     lib.oracle_run_epoch.argtypes = [P, C.c_int, C.c_int, C.c_int, C.c_double, P, C.c_int64, C.c_int,
                                      C.POINTER(OracleStats), P]
     lib.oracle_eval.argtypes = [P, C.c_int, P, P, P]
+    lib.oracle_set_optimizer.argtypes = [P, C.c_int, C.c_double, C.c_double, C.c_double, C.c_double, C.c_int]
     lib.oracle_get_node_stats.argtypes = [P, C.c_int, P, P, P, P, P]
     lib.oracle_get_update_log.restype = C.c_int64
     lib.oracle_get_update_log.argtypes = [P, C.c_int, P, C.c_int64]
@@ -130,6 +131,13 @@ class Oracle:
                                               C.byref(st), _p(loss)))
         st.seconds = time.perf_counter() - t0
         return st, loss
+
+    def set_optimizer(self, kind="sgd", momentum=0.9, beta1=0.9, beta2=0.999, eps=1e-8, reset=True):
+        k = {"sgd": 0, "momentum": 1, "adam": 2}[kind]
+        # the hyper-parameters are rounded to fp32 so that a float32 implementation uses the same numbers
+        f = lambda v: float(np.float32(v))
+        if self.lib.oracle_set_optimizer(self.h, k, f(momentum), f(beta1), f(beta2), f(eps), int(reset)) != 0:
+            raise ValueError(kind)
 
     def eval(self, split=0):
         ml, acc = C.c_double(), C.c_double()

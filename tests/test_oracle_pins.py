@@ -341,3 +341,31 @@ def test_bf16_payload_rounding_only_touches_payloads(oracle_mod):
     assert (rel > 0).any() and rel.max() < 3e-2            # bf16 has 8 bits of mantissa
     for k in p:
         np.testing.assert_array_equal(o.get_params(*k), p[k])
+
+
+# ---------------------------------------------------------------------------------------------------
+# optimisers (App. A: momentum-SGD and Adam as run-time options): against torch.optim on the textbook loop
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("kind", ["momentum", "adam"])
+def test_optimizers_match_torch_optim_on_minibatch_training(oracle_mod, kind):
+    import torch
+    g = ir.mlp((10, 8, 6, 4))
+    inst = data.mlp_instances(n=24, dim=10, classes=4)
+    p = wp.init_params(g)
+    batch, lr = 4, float(np.float32(0.05 if kind == "momentum" else 0.01))
+    o = make(oracle_mod, g, inst, p)
+    o.set_optimizer(kind)
+    for _ in range(2):                                    # two epochs: the optimiser state carries over
+        o.run_epoch(mak=1, muf=batch, lr=lr)
+    P = H.tparams(p)
+    f32 = lambda v: float(np.float32(v))
+    opt = torch.optim.SGD(P.values(), lr=lr, momentum=f32(0.9)) if kind == "momentum" else \
+        torch.optim.Adam(P.values(), lr=lr, betas=(f32(0.9), f32(0.999)), eps=f32(1e-8))
+    for _ in range(2):
+        for s in range(0, inst.n, batch):
+            opt.zero_grad()
+            loss = sum(H.mlp_loss(g, P, inst, i) for i in range(s, s + batch)) / batch
+            loss.backward()
+            opt.step()
+    for k, v in P.items():
+        np.testing.assert_allclose(o.get_params(*k), v.detach().numpy(), rtol=1e-9, atol=1e-12)
