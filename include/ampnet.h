@@ -208,6 +208,22 @@ ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_t
  * other warps, [14] closing barrier).  cycles16: 16 values.  batches: micro-batches executed.                    */
 ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles16, int64_t* batches);
 
+/* ---- update rule of the local updates (Sec. 3; App. A lists the optimiser among the run-time options) -------
+ * Every parameterised node applies the chosen rule to the MEAN of its accumulated gradients, g = A / n, whenever
+ * it updates (min_update_frequency reached, or the epoch-end flush):
+ *   AMPNET_OPT_SGD       theta <- theta - lr g                                   (the default)
+ *   AMPNET_OPT_MOMENTUM  v <- momentum v + g;  theta <- theta - lr v
+ *   AMPNET_OPT_ADAM      m <- beta1 m + (1-beta1) g;  v <- beta2 v + (1-beta2) g^2;
+ *                        theta <- theta - lr (m / (1-beta1^t)) / (sqrt(v / (1-beta2^t)) + eps),  t = updates of this node
+ * The moments are per node, owned by the handle (allocated here through the handle's allocator, one or two float
+ * arrays of the node's parameter count, in device memory), kept across epochs and touched only at updates; an
+ * embedding table moves only the rows (and their moments) that received gradients since its last update.
+ * reset_state != 0 zeroes the moments and t.  Arguments that the chosen rule does not use are ignored.
+ * Errors: AMPNET_EINVAL (unknown kind, momentum/beta outside [0,1), eps <= 0), AMPNET_ENOMEM, AMPNET_ECUDA.          */
+enum { AMPNET_OPT_SGD = 0, AMPNET_OPT_MOMENTUM = 1, AMPNET_OPT_ADAM = 2 };
+ampnet_status_t ampnet_set_optimizer(ampnet_graph_t*, int32_t kind, float momentum, float beta1, float beta2, float eps,
+                                     int32_t reset_state);
+
 const char* ampnet_last_error(const ampnet_graph_t*); /* library-owned string */
 
 /* ---- a training epoch that allocates nothing (no counterpart in the paper) ------------------------------

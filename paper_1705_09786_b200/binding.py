@@ -12,7 +12,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
+           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
            "ampnet_ir_tree", "ampnet_ir_ggnn"]
 
 
@@ -94,6 +94,7 @@ def load_library():
     lib.ampnet_leftover_cache_entries.argtypes = [P, C.POINTER(C.c_int64)]
     lib.ampnet_get_placement.argtypes = [P, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.ampnet_get_phase_cycles.argtypes = [P, C.c_int32, P, C.POINTER(C.c_int64)]
+    lib.ampnet_set_optimizer.argtypes = [P, C.c_int32, C.c_float, C.c_float, C.c_float, C.c_float, C.c_int32]
     I32, PI = C.c_int32, C.POINTER(C.c_int32)
     tail = [P, I32, PI, P, I32, PI]
     lib.ampnet_ir_mlp.argtypes = [P, I32] + tail
@@ -224,6 +225,10 @@ class Engine:
         fn = self.lib.ampnet_run_epoch_static if static_scratch else self.lib.ampnet_run_epoch
         self._check(fn(self.h, C.byref(cfg), C.byref(st), _p(loss)))
         return st, loss
+
+    def set_optimizer(self, kind="sgd", momentum=0.9, beta1=0.9, beta2=0.999, eps=1e-8, reset=True):
+        k = {"sgd": 0, "momentum": 1, "adam": 2}[kind]
+        self._check(self.lib.ampnet_set_optimizer(self.h, k, momentum, beta1, beta2, eps, int(reset)))
 
     def eval(self, split=0, mak=64):
         ml, acc = C.c_double(), C.c_double()

@@ -44,6 +44,8 @@ struct HostDataset {
 struct HostPPT {
   int node = 0, kind = 0, in = 0, out = 0, nmat = 1;
   float *W = nullptr, *b = nullptr;
+  float *om = nullptr, *ov = nullptr;   // optimiser moments (nW + nb floats each), allocated by ampnet_set_optimizer
+  long long opt_t = 0;                  // updates applied since the optimiser state was reset
   size_t nW = 0, nb = 0;
   int T = 1, R = 0, BM = 0, J = 0;
   size_t smem_floats = 0;
@@ -59,6 +61,7 @@ struct ampnet_graph {
   std::vector<int> sources, losses;
   bool has_it = false; int it_steps = 0;
   bool payload_bf16 = false;
+  int opt = 0; float opt_mu = 0.9f, opt_beta1 = 0.9f, opt_beta2 = 0.999f, opt_eps = 1e-8f;
   ampnet_allocator_t alloc{};
   cudaStream_t stream = nullptr;
   int device = 0, n_sms = 0, max_smem = 0;
@@ -463,6 +466,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.T = H.T; P.cta0 = cta; cta += H.T; P.R = H.R; P.BM = H.BM; P.J = H.J;
     P.U = h.U_in; P.rows_max = h.rows_in;
     P.W = H.W; P.b = H.b;
+    P.om = H.om; P.ov = H.ov; P.opt_t0 = H.opt_t;
     const size_t keys = (size_t)mak * IT * P.U;
     const bool source_fed = g->hnodes[h.pred_node[0]].type == SOURCE;
     if (!source_fed) P.xcache = B.take<float>(keys * P.rows_max * P.in_dim);
@@ -599,6 +603,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   if (X.tune & 1) X.wide = 0;
   X.mak = mak; X.muf = cfg ? cfg->min_update_frequency : 1; X.det = det; X.eval = eval; X.IT = IT;
   X.lr = cfg ? cfg->lr : 0.f;
+  X.opt = g->opt; X.mu = g->opt_mu; X.beta1 = g->opt_beta1; X.beta2 = g->opt_beta2; X.eps = g->opt_eps;
   double to = cfg && cfg->timeout_s > 0 ? cfg->timeout_s : 120.0;
   X.timeout_ns = (unsigned long long)(to * 1e9);
   R.smem_bytes = max_smem_floats * sizeof(float);
@@ -683,6 +688,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   CUDA_TRY(g, cudaStreamSynchronize(g->stream));
   if (dbg) fprintf(stderr, "[ampnet] done\n");
   g->have_run = true;
+  if (!eval) for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].opt_t += (long long)g->last_stats[p].n_updates;
   if (getenv("AMPNET_TUNE") && (atoi(getenv("AMPNET_TUNE")) & 8)) {
     static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK"};
     for (int t = 0; t < N_NODE_TYPES * 2; t++)
@@ -754,7 +760,7 @@ ampnet_status_t ampnet_graph_create(const ampnet_ir_desc_t* ir, uint64_t init_se
 void ampnet_graph_destroy(ampnet_graph_t* g) {
   if (!g) return;
   cudaStreamSynchronize(g->stream);
-  for (auto& P : g->ppts) { dev_free(g, P.W); dev_free(g, P.b); }
+  for (auto& P : g->ppts) { dev_free(g, P.W); dev_free(g, P.b); dev_free(g, P.om); dev_free(g, P.ov); }
   free_dataset(g, g->data[0]);
   free_dataset(g, g->data[1]);
   dev_free(g, g->ctl_mem);
@@ -762,6 +768,31 @@ void ampnet_graph_destroy(ampnet_graph_t* g) {
   if (g->ev0) cudaEventDestroy(g->ev0);
   if (g->ev1) cudaEventDestroy(g->ev1);
   delete g;
+}
+
+ampnet_status_t ampnet_set_optimizer(ampnet_graph_t* g, int32_t kind, float momentum, float beta1, float beta2, float eps,
+                                     int32_t reset_state) {
+  if (!g) return AMPNET_EINVAL;
+  if (kind < AMPNET_OPT_SGD || kind > AMPNET_OPT_ADAM) return set_err(g, AMPNET_EINVAL, "unknown optimiser %d", kind);
+  if (kind == AMPNET_OPT_MOMENTUM && !(momentum >= 0.f && momentum < 1.f)) return set_err(g, AMPNET_EINVAL, "momentum must lie in [0, 1)");
+  if (kind == AMPNET_OPT_ADAM && !(beta1 >= 0.f && beta1 < 1.f && beta2 >= 0.f && beta2 < 1.f && eps > 0.f))
+    return set_err(g, AMPNET_EINVAL, "Adam needs beta1, beta2 in [0, 1) and eps > 0");
+  CUDA_TRY(g, cudaSetDevice(g->device));
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  for (auto& P : g->ppts) {
+    const size_t bytes = (P.nW + P.nb) * sizeof(float);
+    float** want[2] = {kind >= AMPNET_OPT_MOMENTUM ? &P.om : nullptr, kind == AMPNET_OPT_ADAM ? &P.ov : nullptr};
+    for (float** w : want) {
+      if (!w) continue;
+      const bool fresh = *w == nullptr;
+      if (fresh && !(*w = (float*)dev_alloc(g, bytes))) return set_err(g, AMPNET_ENOMEM, "optimiser state allocation of %zu bytes failed", bytes);
+      if (fresh || reset_state) CUDA_TRY(g, cudaMemsetAsync(*w, 0, bytes, g->stream));
+    }
+    if (reset_state) P.opt_t = 0;
+  }
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  g->opt = kind; g->opt_mu = momentum; g->opt_beta1 = beta1; g->opt_beta2 = beta2; g->opt_eps = eps;
+  return AMPNET_OK;
 }
 
 const char* ampnet_last_error(const ampnet_graph_t* g) { return g ? g->err.c_str() : "invalid handle"; }

@@ -865,7 +865,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
   if (lane == 0) {
     BatchDesc d;
     d.sched_start = S.ls.sched_w; d.count = take; d.dir = dir; d.flags = upd ? BATCH_UPDATE : 0;
-    d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.pad0 = d.pad1 = 0;
+    d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.upd_t = upd ? (int)S.ls.n_updates + 1 : 0; d.pad1 = 0;
     P.batches[S.ls.batch_w & P.batch_mask] = d;
     __threadfence();
     st_rel(P.batch_pub, S.ls.batch_w + 1u);
@@ -885,9 +885,9 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
 
 __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags) {   // one thread
   BatchDesc d;
-  d.sched_start = S.ls.sched_w; d.count = 0; d.dir = BWD; d.flags = flags; d.n_upd = 0; d.nrows = 0; d.pad0 = d.pad1 = 0;
+  d.sched_start = S.ls.sched_w; d.count = 0; d.dir = BWD; d.flags = flags; d.n_upd = 0; d.nrows = 0; d.upd_t = d.pad1 = 0;
   if ((flags & BATCH_TERMINATE) && S.ls.n_acc > 0 && !C.eval) {      // epoch-end flush of the leftover gradients
-    d.flags |= BATCH_UPDATE; d.n_upd = S.ls.n_acc;
+    d.flags |= BATCH_UPDATE; d.n_upd = S.ls.n_acc; d.upd_t = (int)S.ls.n_updates + 1;
     LeaderState& st = S.ls;
     if (st.log_n < P.update_log_cap) P.update_log[st.log_n] = d.n_upd;
     st.log_n++; st.n_updates++; st.n_grads_applied += d.n_upd;
@@ -1092,7 +1092,7 @@ __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared&
     if (lane == 0) {
       S.rowoff[cnt] = total;
       BatchDesc dd; dd.sched_start = (unsigned)d0.x; dd.count = d0.y; dd.dir = d0.z; dd.flags = d0.w;
-      dd.n_upd = d1.x; dd.nrows = d1.y; dd.pad0 = dd.pad1 = 0;
+      dd.n_upd = d1.x; dd.nrows = d1.y; dd.upd_t = d1.z; dd.pad1 = 0;
       S.desc = dd;
       if (bad) S.ok = 0;
       if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; }
@@ -1180,10 +1180,39 @@ __device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile,
     if (tid == 0) S.phase[14] += (unsigned long long)(clock64() - tw2);
 }
 
+// Local update of one parameter from its accumulated gradient (Sec. 3; the update rule is a run-time option, App. A):
+// g = A / n, then SGD, momentum-SGD (v <- mu v + g, theta <- theta - lr v) or Adam with bias correction, where t counts
+// the updates of this node.  The moments live in device memory and are touched only here.
+struct OptStep {
+  int opt; float lr, inv_n, mu, b1, b2, eps, c1, c2; float *om, *ov;
+  __device__ OptStep(const Ctx& C, const DevPPT& P, const BatchDesc& d)
+      : opt(C.opt), lr(C.lr), inv_n(1.f / (float)d.n_upd), mu(C.mu), b1(C.beta1), b2(C.beta2), eps(C.eps), c1(1.f), c2(1.f),
+        om(P.om), ov(P.ov) {
+    if (opt == 2) {
+      const double t = (double)(P.opt_t0 + d.upd_t);
+      c1 = (float)(1.0 / (1.0 - pow((double)b1, t)));
+      c2 = (float)(1.0 / (1.0 - pow((double)b2, t)));
+    }
+  }
+  __device__ __forceinline__ void apply(float& w, float& a, const size_t k) const {
+    if (opt == 0) { w = fmaf(-(lr * inv_n), a, w); a = 0.f; return; }
+    const float g = a * inv_n;
+    a = 0.f;
+    if (opt == 1) {
+      const float v = fmaf(mu, om[k], g);
+      om[k] = v;
+      w = fmaf(-lr, v, w);
+    } else {
+      const float m = fmaf(b1, om[k], (1.f - b1) * g), v = fmaf(b2, ov[k], (1.f - b2) * g * g);
+      om[k] = m; ov[k] = v;
+      w -= lr * (m * c1) / (sqrtf(v * c2) + eps);
+    }
+  }
+};
+
 __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileShared& S,
                          const unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const DevNode& N = g_nodes[P.node];
   const int in = P.in_dim, out = P.out_dim;
   const int r_begin = tile * P.R;
   const int R = P.kind == LOOKUP ? 0 : max(0, min(P.R, out - r_begin));
@@ -1438,31 +1467,29 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       AMP_PHASE(3);
       // ---- local update (Sec. 3): theta -= lr * A / n, accumulator cleared --------------------------
       if (d.flags & BATCH_UPDATE) {
-        const float scale = C.lr / (float)d.n_upd;
+        const OptStep os(C, P, d);
         if (P.kind == LOOKUP) {
           __threadfence_block();
           const int nt = *P.touched_n;
           for (int idx = tid; idx < nt * out; idx += THREADS) {
             const int id = P.touched_list[idx / out], c = idx % out;
             const size_t o = (size_t)id * out + c;
-            P.W[o] = fmaf(-scale, P.A[o], P.W[o]);
-            P.A[o] = 0.f;
+            os.apply(P.W[o], P.A[o], o);
           }
           __syncthreads();
           for (int k = tid; k < nt; k += THREADS) P.touched_flag[P.touched_list[k]] = 0;
           __syncthreads();
           if (tid == 0) *P.touched_n = 0;
         } else {
+          const size_t nW = (size_t)nmat * out * in;
           for (int m = 0; m < nmat; m++) {
             for (int i = tid; i < R * in; i += THREADS) {
               const int o = m * P.R * in + i;
-              M.Ws[o] = fmaf(-scale, M.As[o], M.Ws[o]);
-              M.As[o] = 0.f;
+              os.apply(M.Ws[o], M.As[o], (size_t)m * out * in + (size_t)r_begin * in + i);
             }
             for (int i = tid; i < R; i += THREADS) {
               const int o = m * P.R + i;
-              M.bs[o] = fmaf(-scale, M.Abs[o], M.bs[o]);
-              M.Abs[o] = 0.f;
+              os.apply(M.bs[o], M.Abs[o], nW + (size_t)m * out + r_begin + i);
             }
           }
         }

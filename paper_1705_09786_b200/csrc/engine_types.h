@@ -31,7 +31,7 @@ struct Ring {            // multi-producer ring of headers; payloads live in the
   unsigned mask;
 };
 
-struct __align__(16) BatchDesc { unsigned sched_start; int count, dir, flags, n_upd, nrows, pad0, pad1; };
+struct __align__(16) BatchDesc { unsigned sched_start; int count, dir, flags, n_upd, nrows, upd_t, pad1; };   // upd_t: index (from 1) of this update within the run
 
 struct PPTStats {
   unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
@@ -63,6 +63,8 @@ struct DevPPT {
   int node, kind, in_dim, out_dim, act, flags, muf_override, pad0;
   int T, cta0, R, BM;                 // row tiles, first CTA, rows per tile, batch row capacity
   int U, rows_max, J, pad1;           // key space, max rows per message, ceil(in_dim / 32) bucket
+  float *om, *ov;                     // optimiser state (first / second moment), laid out like W followed by b
+  long long opt_t0;                   // updates of this node before the run (Adam's bias correction)
   float *W, *b;                       // LINEAR: W[out][in], b[out]; LOOKUP: W = E[V][d]; GRUCELL: W[3][H][2H], b[3][H]
   float* A;                           // LOOKUP: accumulator [V][d] in device memory
   int *touched_flag, *touched_list, *touched_n;
@@ -148,6 +150,8 @@ struct Ctx {
   int depth;                          // per-batch buffers (partials, staging rows) are reused every `depth` batches
   int tune;                           // experiment switches (environment AMPNET_TUNE): 2 no look-ahead, 4 no per-node counters
   float lr;
+  int opt;                            // update rule: 0 SGD, 1 momentum-SGD, 2 Adam
+  float mu, beta1, beta2, eps;
   unsigned long long timeout_ns;
 };
 

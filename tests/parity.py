@@ -2,15 +2,19 @@
 import numpy as np
 
 
-def run_both(oracle_mod, graph, inst, params, mak, muf, lr, order=None, timeout_s=60.0, payload_bf16=False, **engine_kw):
+def run_both(oracle_mod, graph, inst, params, mak, muf, lr, order=None, timeout_s=60.0, payload_bf16=False, optimizer=None, **engine_kw):
     import paper_1705_09786_b200 as amp
     o = oracle_mod.Oracle(graph, payload_bf16=payload_bf16)
     o.load_instances(inst)
     o.set_params(params)
+    if optimizer:
+        o.set_optimizer(**optimizer)
     ost, oloss = o.run_epoch(mak=mak, muf=muf, lr=lr, order=order)
     e = amp.Engine(graph, payload_bf16=payload_bf16)
     e.load_instances(inst)
     e.set_params(params)
+    if optimizer:
+        e.set_optimizer(**optimizer)
     est, eloss = e.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=True, order=order, timeout_s=timeout_s, **engine_kw)
     return o, ost, oloss, e, est, eloss
 

@@ -54,6 +54,33 @@ def test_shuffled_epoch_order_and_second_epoch(oracle_mod):
     e.close()
 
 
+OPT_CASES = [
+    ("mlp", 70, 4, 8, 0.01, "momentum"), ("mlp", 70, 4, 8, 0.001, "adam"),
+    ("rnn", 61, 5, 3, 0.01, "momentum"), ("rnn", 61, 5, 3, 0.001, "adam"),
+    ("tree", 31, 6, 7, 0.005, "momentum"), ("tree", 31, 6, 7, 0.001, "adam"),
+    ("ggnn", 25, 9, 40, 0.0003, "momentum"), ("ggnn", 25, 9, 40, 0.0003, "adam"),
+]
+
+
+@pytest.mark.parametrize("family,n,mak,muf,lr,kind", OPT_CASES)
+def test_momentum_and_adam_updates_match_oracle(oracle_mod, family, n, mak, muf, lr, kind):
+    """Two epochs, so that the moments and Adam's step count carry over; then a reset and a third epoch."""
+    g, inst = _case(family, n)
+    p = wp.init_params(g)
+    opt = dict(kind=kind, momentum=0.8, beta1=0.85, beta2=0.99, eps=1e-6)
+    o, ost, oloss, e, est, eloss = parity.run_both(oracle_mod, g, inst, p, mak, muf, lr, optimizer=opt)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    ost, oloss = o.run_epoch(mak=mak, muf=muf, lr=lr)
+    est, eloss = e.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=True, timeout_s=60)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    o.set_optimizer(**opt)
+    e.set_optimizer(**opt)
+    ost, oloss = o.run_epoch(mak=mak, muf=muf, lr=lr)
+    est, eloss = e.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=True, timeout_s=60)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    e.close()
+
+
 def test_partial_epoch_and_degenerate_sizes(oracle_mod):
     """One instance; mak larger than the instance count; a prefix of the data; the smallest structures."""
     g, inst = _case("rnn", 9)
