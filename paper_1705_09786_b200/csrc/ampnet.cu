@@ -691,6 +691,14 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   if (!eval) for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].opt_t += (long long)g->last_stats[p].n_updates;
   if (getenv("AMPNET_TUNE") && (atoi(getenv("AMPNET_TUNE")) & 8)) {
     static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK"};
+    const double us = 1.0 / 1965.0;
+    fprintf(stderr, "[ctrl] us: retire %.0f admit %.0f clear %.0f pump %.0f idle %.0f admissions %llu\n", G.role_cycles[0] * us, G.role_cycles[1] * us,
+            G.role_cycles[2] * us, G.role_cycles[3] * us, G.role_cycles[4] * us, G.role_cycles[5]);
+    for (size_t p = 0; p < g->ppts.size(); p++) {
+      const unsigned long long* r = G.role_cycles + 8 + 8 * p;
+      fprintf(stderr, "[role] node %2d sched us: wait-tile %.0f no-msg %.0f form %.0f | emitter(0,0) us: wait %.0f load %.0f emit %.0f batches %llu\n",
+              g->ppts[p].node, r[0] * us, r[1] * us, r[2] * us, r[3] * us, r[4] * us, r[5] * us, r[6]);
+    }
     for (int t = 0; t < N_NODE_TYPES * 2; t++)
       if (G.walk_steps[t]) fprintf(stderr, "[walk] %-8s %s steps %10llu cycles/step %8.0f\n", names[t / 2], t & 1 ? "BWD" : "FWD", G.walk_steps[t], (double)G.walk_cycles[t] / G.walk_steps[t]);
   }

@@ -200,7 +200,11 @@ __device__ __forceinline__ void ring_publish(Ring& r, unsigned t, const Frame& f
   st_rel(&r.seq[s], t + 1u);
 }
 
+// A source message came home (or, in evaluation, reached a Loss / Sink): one lane.  The arrival that completes the
+// instance tells the controller; the others only count down.
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v);
 __device__ __forceinline__ void retire_push(const Ctx& C, int slot) {
+  if (atom_add_acq_rel(&C.outstanding[slot], -1) != 1) return;
   unsigned t = atomicAdd(&C.g->retire_tail, 1u);
   unsigned s = t & C.retire_mask;
   C.retire_e[s] = (unsigned)slot;
@@ -798,6 +802,8 @@ struct TileShared {
   int rowoff[MAX_BATCH_MSGS + 1];
   int rowmsg[64];
   const float* rowptr[64];
+  int rowid[64], rownext[64];          // LOOKUP: table row of every batch row; next batch row with the same table row (-1: none)
+  int rowfirst[64];                    // LOOKUP: no earlier batch row has the same table row
   LeaderState ls;
   int ok;
   unsigned tail_snap[2];
@@ -909,10 +915,19 @@ __device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileSh
     slot[dir] = t & P.ring[dir].mask;
     mready[dir] = (ld_acq(&P.ring[dir].seq[slot[dir]]) == t + 1u) ? 1u : 0u;
   }
-  for (int dir = BWD; dir >= FWD; dir--) {
+  int nready[2];
+#pragma unroll
+  for (int dir = 0; dir < 2; dir++) {
     const unsigned m = __ballot_sync(0xffffffffu, mready[dir] != 0);
-    int n = __ffs(~m) - 1;
-    if (n < 0) n = 32;
+    nready[dir] = m == 0xffffffffu ? 32 : __ffs(~m) - 1;
+  }
+  // Backward first (App. A), but a cycle costs the same whether the batch holds 2 messages or 32: a short backward
+  // queue gives way to a longer forward queue and is taken once it has grown to half a batch, has caught up with the
+  // forward queue, or the forward queue has run dry (max_active_keys bounds the forward supply, so it always does).
+  const bool fwd_first = !(C.tune & 128) && nready[BWD] < MAX_BATCH_MSGS / 2 && nready[FWD] > nready[BWD];
+  for (int k = 0; k < 2; k++) {
+    const int dir = (k == 0) == fwd_first ? FWD : BWD;
+    const int n = nready[dir];
     if (n == 0) continue;
     int take = form_batch(C, P, S, dir, slot[dir], n);
     if (lane == 0) S.ls.head[dir] += take;
@@ -1084,8 +1099,29 @@ __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared&
       key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
       S.hdr[lane] = h; S.key[lane] = key; S.rowoff[lane] = off;
       if (key >= 0 && total <= P.BM) {
-        const float* x0 = P.kind != LOOKUP ? msg_x(C, P, h, key) : nullptr;
-        for (int r = 0; r < rows; r++) { S.rowmsg[off + r] = lane; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
+        if (P.kind != LOOKUP) {
+          const float* x0 = msg_x(C, P, h, key);
+          for (int r = 0; r < rows; r++) { S.rowmsg[off + r] = lane; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
+        } else {                                              // table rows and the rows of the incoming gradient
+          const DevInst& I = C.inst;
+          const long long base = I.offsets[h.inst];
+          const float* g0 = P.gbuf + (size_t)key * P.rows_max * P.out_dim;
+          for (int r = 0; r < rows; r++) {
+            const int id = I.tokens[base + (I.kind == 3 ? r : h.u)];
+            S.rowmsg[off + r] = lane; S.rowptr[off + r] = g0 + (size_t)r * P.out_dim;
+            S.rowid[off + r] = (unsigned)id < (unsigned)in ? id : -1;
+          }
+        }
+      }
+    }
+    if (P.kind == LOOKUP && ddir == BWD && total <= P.BM) {   // chain the batch rows that hit the same table row
+      __syncwarp();
+      for (int b = lane; b < total; b += 32) {
+        const int id = S.rowid[b];
+        int nx = -1, first = 1;
+        for (int k = b + 1; k < total; k++) if (S.rowid[k] == id) { nx = k; break; }
+        for (int k = 0; k < b; k++) if (S.rowid[k] == id) { first = 0; break; }
+        S.rownext[b] = nx; S.rowfirst[b] = id >= 0 ? first : 0;
       }
     }
     const unsigned bad = __ballot_sync(0xffffffffu, lane < cnt && key < 0);
@@ -1209,6 +1245,104 @@ struct OptStep {
     }
   }
 };
+
+// Embedding table, one batch (whole CTA).  Forward: gather the table rows into the staging rows.  Backward: accumulate
+// in message order, as if the rows arrived one by one: the first batch row of every table row adds the gradients of all
+// batch rows that hit the same table row, in order.  A warp takes whole rows and keeps ten loads per lane in flight.
+__device__ __noinline__ void lookup_batch(DevPPT& P, TileShared& S, const int dir, const int nb, float* stage_k) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, out = P.out_dim;
+  constexpr int K = 5;                                      // column chunks of 32 per pass
+  if (dir == FWD) {
+    for (int b0 = warp * 2; b0 < nb; b0 += WARPS * 2)       // two rows per pass
+      for (int c0 = 0; c0 < out; c0 += 32 * K) {
+        float v[2][K];
+#pragma unroll
+        for (int r = 0; r < 2; r++) {
+          const int id = b0 + r < nb ? S.rowid[b0 + r] : -1;
+#pragma unroll
+          for (int k = 0; k < K; k++) {
+            const int c = c0 + k * 32 + lane;
+            v[r][k] = (id >= 0 && c < out) ? P.W[(size_t)id * out + c] : 0.f;
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < 2; r++)
+#pragma unroll
+          for (int k = 0; k < K; k++) {
+            const int c = c0 + k * 32 + lane;
+            if (b0 + r < nb && c < out) stage_k[(size_t)(b0 + r) * out + c] = emit_round(v[r][k]);
+          }
+      }
+  } else {
+    for (int b = warp; b < nb; b += WARPS) {
+      if (!S.rowfirst[b]) continue;
+      const int id = S.rowid[b];
+      int fresh = 0;
+      if (lane == 0) fresh = !P.touched_flag[id];
+      float* arow = P.A + (size_t)id * out;
+      for (int c0 = 0; c0 < out; c0 += 32 * K) {
+        float a[K], g0[K];
+#pragma unroll
+        for (int k = 0; k < K; k++) {
+          const int c = c0 + k * 32 + lane;
+          a[k] = c < out ? arow[c] : 0.f;
+          g0[k] = c < out ? __ldcg(S.rowptr[b] + c) : 0.f;
+        }
+#pragma unroll
+        for (int k = 0; k < K; k++) a[k] += g0[k];
+        for (int nx = S.rownext[b]; nx >= 0; nx = S.rownext[nx]) {
+#pragma unroll
+          for (int k = 0; k < K; k++) { const int c = c0 + k * 32 + lane; g0[k] = c < out ? __ldcg(S.rowptr[nx] + c) : 0.f; }
+#pragma unroll
+          for (int k = 0; k < K; k++) a[k] += g0[k];
+        }
+#pragma unroll
+        for (int k = 0; k < K; k++) { const int c = c0 + k * 32 + lane; if (c < out) arow[c] = a[k]; }
+      }
+      if (lane == 0 && fresh) { P.touched_flag[id] = 1; P.touched_list[atomicAdd(P.touched_n, 1)] = id; }
+    }
+  }
+}
+
+// Local update of a tile's share of the node's parameters (whole CTA; ends with a block barrier).
+__device__ __noinline__ void tile_update(const Ctx& C, DevPPT& P, const TileMem& M, const BatchDesc& d, const int R,
+                                         const int r_begin) {
+  const int tid = threadIdx.x, in = P.in_dim, out = P.out_dim;
+  const int nmat = P.kind == GRUCELL ? 3 : 1;
+  const OptStep os(C, P, d);
+  if (P.kind == LOOKUP) {
+    __threadfence_block();
+    const int nt = *P.touched_n;
+    for (int base = tid; base < nt * out; base += 4 * THREADS) {       // four elements in flight per thread
+      float w[4], a[4]; size_t o[4];
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const int idx = base + j * THREADS;
+        if (idx < nt * out) { o[j] = (size_t)P.touched_list[idx / out] * out + idx % out; w[j] = P.W[o[j]]; a[j] = P.A[o[j]]; }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; j++)
+        if (base + j * THREADS < nt * out) { os.apply(w[j], a[j], o[j]); P.W[o[j]] = w[j]; P.A[o[j]] = a[j]; }
+    }
+    __syncthreads();
+    for (int k = tid; k < nt; k += THREADS) P.touched_flag[P.touched_list[k]] = 0;
+    __syncthreads();
+    if (tid == 0) *P.touched_n = 0;
+  } else {
+    const size_t nW = (size_t)nmat * out * in;
+    for (int m = 0; m < nmat; m++) {
+      for (int i = tid; i < R * in; i += THREADS) {
+        const int o = m * P.R * in + i;
+        os.apply(M.Ws[o], M.As[o], (size_t)m * out * in + (size_t)r_begin * in + i);
+      }
+      for (int i = tid; i < R; i += THREADS) {
+        const int o = m * P.R + i;
+        os.apply(M.bs[o], M.Abs[o], nW + (size_t)m * out + r_begin + i);
+      }
+    }
+  }
+  __syncthreads();
+}
 
 __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileShared& S,
                          const unsigned long long t0) {
@@ -1440,61 +1574,15 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           }
         }
       } else if (count > 0 && P.kind == LOOKUP) {
-        const DevInst& I = C.inst;
-        if (dir == FWD) {
-          for (int idx = tid; idx < nb * out; idx += THREADS) {
-            const int b = idx / out, c = idx - b * out, m = S.rowmsg[b];
-            const Hdr& h = S.hdr[m];
-            const int pos = I.kind == 3 ? (b - S.rowoff[m]) : h.u;
-            const int id = I.tokens[I.offsets[h.inst] + pos];
-            stage_k[idx] = ((unsigned)id < (unsigned)in) ? emit_round(P.W[(size_t)id * out + c]) : 0.f;
-          }
-        } else {
-          for (int c = tid; c < out; c += THREADS)
-            for (int b = 0; b < nb; b++) {
-              const int m = S.rowmsg[b];
-              const Hdr& h = S.hdr[m];
-              const int pos = I.kind == 3 ? (b - S.rowoff[m]) : h.u;
-              const int id = I.tokens[I.offsets[h.inst] + pos];
-              if ((unsigned)id >= (unsigned)in) continue;
-              const float g = __ldcg(P.gbuf + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * out + c);
-              P.A[(size_t)id * out + c] += g;
-              if (c == 0 && !P.touched_flag[id]) { P.touched_flag[id] = 1; P.touched_list[(*P.touched_n)++] = id; }
-            }
-        }
+        const long long tl0 = clock64();
+        lookup_batch(P, S, dir, nb, stage_k);
+        __syncthreads();
+        if (tid == 0) { S.phase[9 + 2 * dir] += (unsigned long long)(clock64() - tl0); S.phase[10 + 2 * dir] += (unsigned long long)nb; }
       }
       __syncthreads();
       AMP_PHASE(3);
       // ---- local update (Sec. 3): theta -= lr * A / n, accumulator cleared --------------------------
-      if (d.flags & BATCH_UPDATE) {
-        const OptStep os(C, P, d);
-        if (P.kind == LOOKUP) {
-          __threadfence_block();
-          const int nt = *P.touched_n;
-          for (int idx = tid; idx < nt * out; idx += THREADS) {
-            const int id = P.touched_list[idx / out], c = idx % out;
-            const size_t o = (size_t)id * out + c;
-            os.apply(P.W[o], P.A[o], o);
-          }
-          __syncthreads();
-          for (int k = tid; k < nt; k += THREADS) P.touched_flag[P.touched_list[k]] = 0;
-          __syncthreads();
-          if (tid == 0) *P.touched_n = 0;
-        } else {
-          const size_t nW = (size_t)nmat * out * in;
-          for (int m = 0; m < nmat; m++) {
-            for (int i = tid; i < R * in; i += THREADS) {
-              const int o = m * P.R * in + i;
-              os.apply(M.Ws[o], M.As[o], (size_t)m * out * in + (size_t)r_begin * in + i);
-            }
-            for (int i = tid; i < R; i += THREADS) {
-              const int o = m * P.R + i;
-              os.apply(M.bs[o], M.Abs[o], nW + (size_t)m * out + r_begin + i);
-            }
-          }
-        }
-        __syncthreads();
-      }
+      if (d.flags & BATCH_UPDATE) tile_update(C, P, M, d, R, r_begin);
       AMP_PHASE(4);
       // ---- all tiles of the node done with the batch, then emit ------------------------------------
       if (count > 0) {
@@ -1549,6 +1637,9 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int til
   __syncthreads();
   unsigned my_batch = (unsigned)which;          // this emitter takes batches which, which + E, which + 2E, ...
   WalkAcc acc = {0, 0};
+  unsigned long long* const rc = C.g->role_cycles + 8 + 8 * (int)(&P - g_ppts);
+  long long tp = clock64();
+#define EMIT_PHASE(k) do { if (tid == 0) { const long long tn = clock64(); S.phase[k] += (unsigned long long)(tn - tp); tp = tn; } } while (0)
   for (;;) {
     // every emitter of the tile sees the terminating batch: emit_pub counts all batches, the last one is the marker
     if (tid == 0) { S.ok = 1; if (!spin_until(C, t0, [&] { return ld_acq(&P.emit_pub[tile]) > my_batch || ld_acq(&P.emit_fin[tile]) != 0u; })) S.ok = 0; }
@@ -1557,15 +1648,21 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int til
     if (tid == 0) S.tail_snap[0] = ld_acq(&P.emit_pub[tile]);
     __syncthreads();
     if (S.tail_snap[0] <= my_batch) break;                     // finished and nothing left for this emitter
+    EMIT_PHASE(3);
     if (warp == 0) load_batch_ctx(C, P, S, my_batch);
     __syncthreads();
     const BatchDesc d = S.desc;
     if (!S.ok) break;
+    EMIT_PHASE(4);
     if (d.count > 0) emit_batch(C, P, tile, S, d, my_batch + 1u, P.stage + (size_t)((my_batch + 1u) % (unsigned)C.depth) * P.stage_floats, acc);
     __syncthreads();
+    EMIT_PHASE(5);
+    if (tid == 0) S.phase[6] += 1ull;
     if (tid == 0) { __threadfence(); st_rel(&P.emit_done[tile * C.emit_ctas + which], my_batch + 1u); }
     my_batch += (unsigned)C.emit_ctas;
   }
+  __syncthreads();
+  if (tile == 0 && which == 0 && tid >= 3 && tid < 7) rc[tid] = S.phase[tid];
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1578,14 +1675,19 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
   __syncthreads();
   if (warp == 0) {
     unsigned it = 0;
+    unsigned long long* const rc = C.g->role_cycles + 8 + 8 * (int)(&P - g_ppts);
+    long long tp = clock64();
+    unsigned long long rcl[3] = {0, 0, 0};
     for (;;) {
       // at most one batch ahead of what tile 0 has fetched
       unsigned go = 0, bw = 0;
       if (lane == 0) { bw = S.ls.batch_w; go = ld_acq(P.fetched) >= bw; }
       bw = warp_uniform(bw);
       bool progressed = false;
-      if (warp_uniform(go)) {
-        progressed = leader_try_schedule(C, P, S);
+      const bool gow = warp_uniform(go);
+      if (gow) progressed = leader_try_schedule(C, P, S);
+      if (lane == 0) { const long long tn = clock64(); rcl[!gow ? 0 : progressed ? 2 : 1] += (unsigned long long)(tn - tp); tp = tn; }
+      if (gow) {
         unsigned fin = 0;
         if (lane == 0) fin = progressed && (P.batches[bw & P.batch_mask].flags & BATCH_TERMINATE);
         if (warp_uniform(fin)) break;
@@ -1599,6 +1701,7 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
       }
       __nanosleep(it < 16 ? 20 : 100);
     }
+    if (lane == 0) { rc[0] = rcl[0]; rc[1] = rcl[1]; rc[2] = rcl[2]; }
   }
   __syncthreads();
   write_leader_stats(P, S);
@@ -1607,6 +1710,12 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
 // ------------------------------------------------------------------------------------------------
 // controller CTA: admission under max_active_keys, source messages, retirement (Sec. 3, Sec. 4)
 // ------------------------------------------------------------------------------------------------
+constexpr int OCC_SLOTS = 8192;
+__device__ __forceinline__ bool source_is_bulk(const Ctx& C, const DevNode& sn) {
+  if (C.det || (C.tune & 16) || !(sn.fn == 1 || sn.fn == 2 || sn.fn == 4)) return false;
+  const DevNode& dn = g_nodes[sn.succ_node[0]];
+  return (dn.type == LINEAR || dn.type == LOOKUP || dn.type == GRUCELL) && g_ppts[dn.ppt].xcache == nullptr && g_ppts[dn.ppt].rows_max >= 1;
+}
 struct CtrlShared {
   int ok;
   long long next, retired;
@@ -1614,6 +1723,8 @@ struct CtrlShared {
   unsigned retire_head;
   int admit_slot, admit_inst, admit_seq, n_src_msgs;
   int src_count[4], src_base[5];
+  unsigned long long prof[8];
+  unsigned occ[OCC_SLOTS / 32];          // occupied key slots (slots beyond OCC_SLOTS are found by scanning slot_inst)
   Frame stack[WARPS][WALK_STACK];
   WalkPool pool;
 };
@@ -1623,12 +1734,17 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
   const DevInst& I = C.inst;
   if (tid == 0) { S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
   if (tid < POOL) S.pool.ready[tid] = 0;
+  for (int i = tid; i < OCC_SLOTS / 32; i += THREADS) S.occ[i] = 0u;
+  if (tid < 8) S.prof[tid] = 0;
   __syncthreads();
   unsigned grid_gen = 0;
   WalkAcc acc = {0, 0};
   long long round = 0;
   unsigned idle = 0;
+  long long tp = clock64();
+#define CTRL_PHASE(k) do { if (tid == 0) { const long long tn = clock64(); S.prof[k] += (unsigned long long)(tn - tp); tp = tn; } } while (0)
   for (;; round++) {
+    CTRL_PHASE(4);
     // ---- retirements ------------------------------------------------------------------------------
     if (warp == 0) {
       for (;;) {
@@ -1639,10 +1755,8 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
         const unsigned s = h & C.retire_mask;
         const int slot = (int)__ldcg(&C.retire_e[s]);
         __syncwarp();
-        int left = 0;
-        if (lane == 0) { S.retire_head = h + 1u; left = --C.outstanding[slot]; }
-        left = __shfl_sync(0xffffffffu, left, 0);
-        if (left == 0) {
+        if (lane == 0) S.retire_head = h + 1u;
+        {
           // instance finished: sum its loss cells in key order, free the slot
           const int inst = C.slot_inst[slot];
           double tot = 0.0; int okc = 0, np = 0;
@@ -1662,6 +1776,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
             C.loss_out[inst] = (float)tot;
             C.g->total_loss += tot; C.g->correct += okc; C.g->n_pred += np;
             C.slot_inst[slot] = -1;
+            if (slot < OCC_SLOTS) S.occ[slot >> 5] &= ~(1u << (slot & 31));
             S.active--; S.retired++;
             if (C.det && C.keylog) C.keylog[C.slot_log[slot]].release = round;
           }
@@ -1670,13 +1785,19 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
       }
     }
     __syncthreads();
+    CTRL_PHASE(0);
     // ---- admission ----------------------------------------------------------------------------------
     for (;;) {
       if (tid == 0) {
         S.admit_slot = -1;
         if (S.active < C.mak && S.next < C.n_order) {
-          int slot = 0;
-          while (slot < C.mak && C.slot_inst[slot] >= 0) slot++;          // lowest free slot
+          int slot = 0;                                                   // lowest free slot
+          const int nw = (min(C.mak, OCC_SLOTS) + 31) >> 5;
+          int w = 0;
+          while (w < nw && S.occ[w] == 0xffffffffu) w++;
+          if (w < nw) slot = w * 32 + __ffs(~S.occ[w]) - 1;
+          else { slot = OCC_SLOTS; while (slot < C.mak && C.slot_inst[slot] >= 0) slot++; }
+          if (slot < OCC_SLOTS) S.occ[slot >> 5] |= 1u << (slot & 31);
           const int inst = (int)(C.order ? C.order[S.next] : S.next);
           S.admit_slot = slot; S.admit_inst = inst; S.admit_seq = (int)S.next;
           C.slot_inst[slot] = inst;
@@ -1708,6 +1829,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
       }
       __syncthreads();
       const int slot = S.admit_slot;
+      CTRL_PHASE(1);
       if (slot < 0) break;
       // clear the slot's loss cells (predok = -1 marks "no loss evaluated at this key")
       for (int li = 0; li < C.n_loss; li++) {
@@ -1719,13 +1841,44 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
       __syncthreads();
       // pump the source messages (Sec. 4: tokens / leaves / graph nodes, initial hidden state, dense row)
       const int inst = S.admit_inst;
-      if (tid == 0) S.pool.outstanding = S.n_src_msgs;
+      if (tid == 0) { S.pool.outstanding = S.n_src_msgs; S.prof[5] += 1ull; }
       __syncthreads();
+      CTRL_PHASE(2);
+      // A source that feeds a parameterised node directly (token / leaf / dense-row messages carry no payload of their
+      // own) is pumped 32 messages at a time: one ticket grab per warp, every lane publishes its own header.
+      for (int s = 0; s < C.n_sources; s++) {
+        const DevNode& sn = g_nodes[C.src_nodes[s]];
+        if (!source_is_bulk(C, sn)) continue;
+        const DevNode& dn = g_nodes[sn.succ_node[0]];
+        DevPPT& P = g_ppts[dn.ppt];
+        const int cnt = S.src_count[s];
+        for (int c0 = warp * 32; c0 < cnt; c0 += WARPS * 32) {
+          const int k = c0 + lane;
+          int u = 0;
+          if (k < cnt) u = sn.fn == 2 ? k : sn.fn == 4 ? I.leaf_ids[I.leaf_off[inst] + k] : 0;
+          const bool okm = k < cnt && key_of(C, sn.succ_node[0], slot, 0, u, P.U) >= 0;
+          const unsigned vm = __ballot_sync(0xffffffffu, okm);
+          unsigned tk = 0;
+          if (lane == 0 && vm) tk = atomicAdd(P.ring[FWD].tail, (unsigned)__popc(vm));
+          tk = __shfl_sync(0xffffffffu, tk, 0) + (unsigned)__popc(vm & ((1u << lane) - 1u));
+          if (okm) {
+            const unsigned q = tk & P.ring[FWD].mask;
+            int4* d = reinterpret_cast<int4*>(&P.ring[FWD].e[q]);
+            d[0] = make_int4(inst, S.admit_seq, slot, 0);
+            d[1] = make_int4(u, 0, 1, C.eval ? HDR_EVAL : 0);
+            st_rel(&P.ring[FWD].seq[q], tk + 1u);
+          }
+          const int n_here = min(32, cnt - c0);
+          acc.msgs += (unsigned long long)__popc(vm);
+          if (lane == 0) atomicSub(&S.pool.outstanding, n_here);
+        }
+      }
       for (int mi = warp; mi < S.n_src_msgs; mi += WARPS) {
         int s = 0;
         while (mi >= S.src_base[s + 1]) s++;
         const int k = mi - S.src_base[s];
         const DevNode& sn = g_nodes[C.src_nodes[s]];
+        if (source_is_bulk(C, sn)) continue;
         Frame f;
         f.node = sn.succ_node[0]; f.aport = sn.succ_port[0]; f.dir = FWD; f.iter = 0;
         f.inst = inst; f.seq = S.admit_seq; f.slot = slot; f.it = 0; f.u = 0; f.port = 0; f.rows = 1;
@@ -1745,6 +1898,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
       pool_steal(C, &S.pool, S.stack[warp], acc);
       flush_acc(C, acc, lane);
       __syncthreads();
+      CTRL_PHASE(3);
     }
     // ---- termination / pacing -------------------------------------------------------------------------
     const bool finished = S.retired == C.n_order;
@@ -1771,6 +1925,8 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
       if (!S.ok) break;
     }
   }
+  __syncthreads();
+  if (tid < 8) C.g->role_cycles[tid] = S.prof[tid];
 }
 
 union SharedUnion { TileShared t; CtrlShared c; };

@@ -122,6 +122,9 @@ struct Globals {                      // mutable run state in device memory (zer
   unsigned retire_tail;
   int err_node, err_detail;
   unsigned long long walk_cycles[N_NODE_TYPES * 2], walk_steps[N_NODE_TYPES * 2];   // profiling (tune bit 8)
+  // cycles by role: [0..7] controller (retire, admit, clear, pump, idle, admissions), then per PPT node p at 8 + 8 p:
+  // scheduler (waiting for tile 0, no message pending, forming) and emitters (waiting, loading, emitting, batches)
+  unsigned long long role_cycles[8 + 8 * MAX_SMEM_PPTS];
 };
 
 struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of its emitter CTAs (pad = which one), 2: the node's scheduler CTA
