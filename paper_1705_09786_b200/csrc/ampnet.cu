@@ -492,6 +492,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.batches = B.take<BatchDesc>(2 * (size_t)cap); P.batch_mask = 2 * cap - 1;
     P.batch_pub = C.take<unsigned>(1);
     P.bhdr = B.take<Hdr>((size_t)BATCH_BLOCKS * MAX_BATCH_MSGS);
+    P.ctxblk = B.take<BatchCtx>((size_t)BATCH_BLOCKS);
     P.sortbuf = B.take<unsigned long long>(cap);
     if ((P.T > 1 && H.kind != LOOKUP) || H.kind == GRUCELL) P.dxpart = B.take<float>((size_t)depth * P.T * P.BM * P.in_dim);
     P.stage_floats = (long long)P.BM * std::max(P.in_dim, P.out_dim);

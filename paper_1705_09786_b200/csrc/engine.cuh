@@ -795,15 +795,7 @@ struct LeaderState {
   unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
 };
 
-struct TileShared {
-  BatchDesc desc;
-  Hdr hdr[MAX_BATCH_MSGS];
-  long long key[MAX_BATCH_MSGS];
-  int rowoff[MAX_BATCH_MSGS + 1];
-  int rowmsg[64];
-  const float* rowptr[64];
-  int rowid[64], rownext[64];          // LOOKUP: table row of every batch row; next batch row with the same table row (-1: none)
-  int rowfirst[64];                    // LOOKUP: no earlier batch row has the same table row
+struct TileShared : BatchCtx {
   LeaderState ls;
   int ok;
   unsigned tail_snap[2];
@@ -873,8 +865,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
     d.sched_start = S.ls.sched_w; d.count = take; d.dir = dir; d.flags = upd ? BATCH_UPDATE : 0;
     d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.upd_t = upd ? (int)S.ls.n_updates + 1 : 0; d.pad1 = 0;
     P.batches[S.ls.batch_w & P.batch_mask] = d;
-    __threadfence();
-    st_rel(P.batch_pub, S.ls.batch_w + 1u);
+    if (!C.sched_ctas) { __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }   // a scheduler CTA publishes the assembled context instead
     S.ls.batch_w++;
     S.ls.sched_w += take;
     LeaderState& st = S.ls;
@@ -900,8 +891,7 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
     S.ls.n_acc = 0; S.ls.version++;
   }
   P.batches[S.ls.batch_w & P.batch_mask] = d;
-  __threadfence();
-  st_rel(P.batch_pub, S.ls.batch_w + 1u);
+  if (!C.sched_ctas) { __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
   S.ls.batch_w++;
 }
 
@@ -1129,11 +1119,30 @@ __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared&
       S.rowoff[cnt] = total;
       BatchDesc dd; dd.sched_start = (unsigned)d0.x; dd.count = d0.y; dd.dir = d0.z; dd.flags = d0.w;
       dd.n_upd = d1.x; dd.nrows = d1.y; dd.upd_t = d1.z; dd.pad1 = 0;
+      if (bad) { S.ok = 0; dd.pad1 = 1; }
+      if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; dd.pad1 = 1; }
       S.desc = dd;
-      if (bad) S.ok = 0;
-      if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; }
     }
 
+}
+
+// With scheduler CTAs: the assembled context of batch `batch`, one 16-byte piece per thread (whole CTA, no barrier).
+__device__ __forceinline__ void fetch_ctx_block(const DevPPT& P, TileShared& S, const unsigned batch) {
+  const int4* src = reinterpret_cast<const int4*>(P.ctxblk + (batch & (BATCH_BLOCKS - 1)));
+  int4* dst = reinterpret_cast<int4*>(static_cast<BatchCtx*>(&S));
+  for (int i = threadIdx.x; i < (int)(sizeof(BatchCtx) / 16); i += THREADS) dst[i] = __ldcg(src + i);
+}
+// Scheduler CTA, warp 0: assemble the context of the batch just formed and publish it.
+__device__ __noinline__ void publish_ctx_block(const Ctx& C, DevPPT& P, TileShared& S, const unsigned batch) {
+  const int lane = threadIdx.x & 31;
+  load_batch_ctx(C, P, S, batch);
+  __syncwarp();
+  const int4* src = reinterpret_cast<const int4*>(static_cast<BatchCtx*>(&S));
+  int4* dst = reinterpret_cast<int4*>(P.ctxblk + (batch & (BATCH_BLOCKS - 1)));
+  for (int i = lane; i < (int)(sizeof(BatchCtx) / 16); i += 32) dst[i] = src[i];
+  __syncwarp();
+  if (lane == 0) { __threadfence(); st_rel(P.batch_pub, batch + 1u); }
+  __syncwarp();
 }
 
 // Emission of a batch by one CTA: reduce the tiles' partial input gradients for the rows this CTA emits, then walk
@@ -1425,21 +1434,36 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       }
       __syncthreads();
       if (!S.ok || aborted(C)) { running = false; break; }
-      if (warp == 0) load_batch_ctx(C, P, S, my_batch);
-      if (C.sched_ctas && tile == 0 && tid == 0) st_rel(P.fetched, my_batch + 1u);   // the scheduler may form the next batch
+      if (C.sched_ctas) {
+        fetch_ctx_block(P, S, my_batch);
+        if (tile == 0 && tid == 0) st_rel(P.fetched, my_batch + 1u);                 // paces the scheduler
+      } else if (warp == 0) load_batch_ctx(C, P, S, my_batch);
       __syncthreads();
       const BatchDesc d = S.desc;
       my_batch++;
       AMP_PHASE(d.count > 0 ? 1 : 0);
       const int count = d.count, dir = d.dir;
-      if (!S.ok) { running = false; break; }
+      if (!S.ok || d.pad1) { running = false; break; }
       float* const stage_k = P.stage + (size_t)(my_batch % (unsigned)C.depth) * P.stage_floats;
       if (C.emit_ctas && count > 0) {
-        // the per-batch buffers are reused every `depth` batches: wait until their previous user has been emitted
-        if (tid == 0 && my_batch > (unsigned)C.depth) {
-          const unsigned j = my_batch - 1u - (unsigned)C.depth;           // the batch that used these buffers before
-          const unsigned* done = &P.emit_done[tile * C.emit_ctas + (int)(j % (unsigned)C.emit_ctas)];
-          if (!spin_until(C, t0, [&] { return ld_acq(done) >= j + 1u; })) S.ok = 0;
+        // the per-batch buffers are reused every `depth` batches and read by the emitters of every tile: wait until all
+        // of them are done with the batch that used these buffers before
+        if (warp == 0 && my_batch > (unsigned)C.depth) {
+          const unsigned j = my_batch - 1u - (unsigned)C.depth;
+          const int ne = P.T * C.emit_ctas;
+          unsigned it = 0;
+          for (;;) {
+            bool ok = true;
+            for (int e = lane; e < ne; e += 32)
+              if ((unsigned)(e % C.emit_ctas) == j % (unsigned)C.emit_ctas) ok = ok && ld_acq(&P.emit_done[e]) >= j + 1u;
+            if (__all_sync(0xffffffffu, ok)) break;
+            if ((++it & 15u) == 0) {
+              unsigned bad = 0;
+              if (lane == 0) { bad = aborted(C); if (!bad && gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, P.node, 6); bad = 1; } }
+              if (warp_uniform(bad)) { if (lane == 0) S.ok = 0; break; }
+            }
+            __nanosleep(it < 16 ? 20 : 100);
+          }
         }
         __syncthreads();
         if (!S.ok) { running = false; break; }
@@ -1587,7 +1611,8 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       // ---- all tiles of the node done with the batch, then emit ------------------------------------
       if (count > 0) {
         __threadfence();
-        if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
+        // tiles that emit themselves wait for each other here; emitter CTAs wait for all tiles instead
+        if (P.T > 1 && !C.emit_ctas) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
         else __syncthreads();
         AMP_PHASE(5);
         if (tile == 0 && warp == 0 && !C.det && !C.sched_ctas && !(C.tune & 2)) {   // look ahead: form the next batch now
@@ -1642,17 +1667,38 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int til
 #define EMIT_PHASE(k) do { if (tid == 0) { const long long tn = clock64(); S.phase[k] += (unsigned long long)(tn - tp); tp = tn; } } while (0)
   for (;;) {
     // every emitter of the tile sees the terminating batch: emit_pub counts all batches, the last one is the marker
-    if (tid == 0) { S.ok = 1; if (!spin_until(C, t0, [&] { return ld_acq(&P.emit_pub[tile]) > my_batch || ld_acq(&P.emit_fin[tile]) != 0u; })) S.ok = 0; }
+    // A batch is ready once every tile of the node has handed it over (the tiles do not wait for each other).
+    if (tid == 0) S.ok = 1;
     __syncthreads();
-    if (!S.ok) break;
-    if (tid == 0) S.tail_snap[0] = ld_acq(&P.emit_pub[tile]);
+    if (warp == 0) {
+      const int lane = tid & 31;
+      unsigned it = 0;
+      int state = 0;                                            // 1: the batch is ready, 2: finished, 3: give up
+      while (state == 0) {
+        const unsigned pub = lane < P.T ? ld_acq(&P.emit_pub[lane]) : 0xffffffffu;
+        if (__all_sync(0xffffffffu, pub > my_batch)) state = 1;
+        else {
+          unsigned fin = 0;
+          if (lane == 0) fin = ld_acq(&P.emit_fin[tile]) != 0u && ld_acq(&P.emit_pub[tile]) <= my_batch;
+          if (warp_uniform(fin)) state = 2;
+          else if ((++it & 15u) == 0) {
+            unsigned bad = 0;
+            if (lane == 0) { bad = aborted(C); if (!bad && gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, P.node, 5); bad = 1; } }
+            if (warp_uniform(bad)) state = 3;
+          }
+          if (state == 0) __nanosleep(it < 16 ? 20 : 100);
+        }
+      }
+      if (lane == 0) S.tail_snap[0] = (unsigned)state;
+    }
     __syncthreads();
-    if (S.tail_snap[0] <= my_batch) break;                     // finished and nothing left for this emitter
+    if (S.tail_snap[0] != 1u) break;                           // finished and nothing left for this emitter, or aborted
     EMIT_PHASE(3);
-    if (warp == 0) load_batch_ctx(C, P, S, my_batch);
+    if (C.sched_ctas) fetch_ctx_block(P, S, my_batch);
+    else if (warp == 0) load_batch_ctx(C, P, S, my_batch);
     __syncthreads();
     const BatchDesc d = S.desc;
-    if (!S.ok) break;
+    if (!S.ok || d.pad1) break;
     EMIT_PHASE(4);
     if (d.count > 0) emit_batch(C, P, tile, S, d, my_batch + 1u, P.stage + (size_t)((my_batch + 1u) % (unsigned)C.depth) * P.stage_floats, acc);
     __syncthreads();
@@ -1679,13 +1725,14 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
     long long tp = clock64();
     unsigned long long rcl[3] = {0, 0, 0};
     for (;;) {
-      // at most one batch ahead of what tile 0 has fetched
+      // at most two batches ahead of what tile 0 has fetched
       unsigned go = 0, bw = 0;
-      if (lane == 0) { bw = S.ls.batch_w; go = ld_acq(P.fetched) >= bw; }
+      if (lane == 0) { bw = S.ls.batch_w; go = ld_acq(P.fetched) + 1u >= bw; }
       bw = warp_uniform(bw);
       bool progressed = false;
       const bool gow = warp_uniform(go);
       if (gow) progressed = leader_try_schedule(C, P, S);
+      if (progressed) publish_ctx_block(C, P, S, bw);
       if (lane == 0) { const long long tn = clock64(); rcl[!gow ? 0 : progressed ? 2 : 1] += (unsigned long long)(tn - tp); tp = tn; }
       if (gow) {
         unsigned fin = 0;

@@ -8,7 +8,7 @@ constexpr int MAX_PORTS = 8;
 constexpr int THREADS = 256;          // threads per CTA
 constexpr int WARPS = THREADS / 32;
 constexpr int MAX_BATCH_MSGS = 32;    // messages per micro-batch (one warp schedules them)
-constexpr int BATCH_BLOCKS = 8;      // header blocks travelling with batch descriptors (asynchronous mode)
+constexpr int BATCH_BLOCKS = 16;     // batch context blocks in flight between a node's scheduler and its tiles / emitters
 constexpr int MAX_SMEM_NODES = 40;    // IR nodes / PPT nodes whose tables are kept in shared memory
 constexpr int MAX_SMEM_PPTS = 16;
 constexpr int MAX_TILES = 32;        // row tiles per PPT node
@@ -32,6 +32,20 @@ struct Ring {            // multi-producer ring of headers; payloads live in the
 };
 
 struct __align__(16) BatchDesc { unsigned sched_start; int count, dir, flags, n_upd, nrows, upd_t, pad1; };   // upd_t: index (from 1) of this update within the run
+
+// Everything a tile or an emitter needs to know about one micro-batch.  With scheduler CTAs the scheduler assembles it
+// once and the consumers copy the block; otherwise every consumer derives it from the descriptor and the headers.
+struct __align__(16) BatchCtx {
+  BatchDesc desc;                       // desc.pad1 != 0: the batch is malformed (the run is being aborted)
+  Hdr hdr[MAX_BATCH_MSGS];
+  long long key[MAX_BATCH_MSGS];
+  int rowoff[MAX_BATCH_MSGS + 4];       // first batch row of every message; [count] = rows of the batch
+  int rowmsg[64];                       // message of every batch row
+  const float* rowptr[64];              // cached input row (LOOKUP: incoming gradient row) of every batch row
+  int rowid[64], rownext[64];           // LOOKUP: table row of every batch row; next batch row with the same table row (-1: none)
+  int rowfirst[64];                     // LOOKUP: no earlier batch row has the same table row
+};
+static_assert(sizeof(BatchCtx) % 16 == 0, "batch context blocks are copied in 16-byte pieces");
 
 struct PPTStats {
   unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
@@ -75,6 +89,7 @@ struct DevPPT {
   unsigned* sched; unsigned sched_mask;
   BatchDesc* batches; unsigned batch_mask; unsigned* batch_pub;
   Hdr* bhdr;                          // [BATCH_BLOCKS][MAX_BATCH_MSGS] headers of the most recent batches
+  BatchCtx* ctxblk;                   // [BATCH_BLOCKS] assembled batch contexts (scheduler CTAs only)
   unsigned long long* sortbuf;
   float* dxpart;                      // [2][T][BM][in_dim] partial input gradients of the row tiles
   float* stage;                       // [2][BM][max(in_dim, out_dim)] reduced input gradients / gathered rows, by batch parity
