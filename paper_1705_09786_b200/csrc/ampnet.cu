@@ -48,6 +48,7 @@ struct HostPPT {
   long long opt_t = 0;                  // updates applied since the optimiser state was reset
   size_t nW = 0, nb = 0;
   int T = 1, R = 0, BM = 0, J = 0;
+  int NE = 0, G = 1;                    // emitter CTAs of the node and their batch groups
   size_t smem_floats = 0;
 };
 
@@ -373,7 +374,7 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   for (auto& P : g->ppts) {
     const DevNode& h = g->hnodes[P.node];
     const int rows_max = h.rows_in;
-    int BM = rows_max <= 32 ? 32 : 64;
+    int BM = MAX_BATCH_ROWS;
     if (max_batch_rows > 0) BM = std::max(rows_max, std::min(BM, max_batch_rows));
     if (rows_max > 64) return set_err(g, AMPNET_EINVAL, "node %d: %d payload rows per message exceed the supported 64", P.node, rows_max);
     P.J = P.kind == LOOKUP ? 4 : j_bucket(P.in);
@@ -401,12 +402,22 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   roles.push_back(Role{-1, 0, 0, 0});
   for (int p = 0; p < (int)g->ppts.size(); p++)
     for (int t = 0; t < g->ppts[p].T; t++) roles.push_back(Role{p, t, 0, 0});
+  for (auto& P : g->ppts) { P.NE = 0; P.G = 1; }
   if (emitters > 0) {
-    if (1 + (used - 1) * (1 + emitters) + (int)g->ppts.size() > n_ctas) return AMPNET_EOVERFLOW;   // retried with fewer emitters / tiles
+    const int need = 1 + (used - 1) * (1 + emitters) + (int)g->ppts.size();
+    if (need > n_ctas) return AMPNET_EOVERFLOW;                                                     // retried with fewer emitters / tiles
+    for (auto& P : g->ppts) P.NE = P.T * emitters;
+    // spare SMs become emitters of the nodes that have the fewest (a node with few row tiles emits as many messages)
+    for (int spare = n_ctas - need; spare > 0; spare--) {
+      HostPPT* best = nullptr;
+      for (auto& P : g->ppts) if (P.NE < 24 && (!best || P.NE < best->NE)) best = &P;
+      if (!best) break;
+      best->NE++;
+    }
+    for (auto& P : g->ppts) P.G = std::min(2, P.NE);
     for (int p = 0; p < (int)g->ppts.size(); p++) roles.push_back(Role{p, 0, 2, 0});                 // one scheduler CTA per node
     for (int p = 0; p < (int)g->ppts.size(); p++)
-      for (int t = 0; t < g->ppts[p].T; t++)
-        for (int e = 0; e < emitters; e++) roles.push_back(Role{p, t, 1, e});
+      for (int e = 0; e < g->ppts[p].NE; e++) roles.push_back(Role{p, 0, 1, e});
   }
   return AMPNET_OK;
 }
@@ -443,7 +454,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   }
   if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0, 0); }
   if (st != AMPNET_OK) return st;
-  const int depth = emit_ctas > 0 ? emit_ctas + 1 : 2;
+  const int depth = emit_ctas > 0 ? 3 : 2;       // emitters work in two batch groups: a tile may be two batches ahead
   R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth; R.ctx.sched_ctas = emit_ctas > 0 ? 1 : 0;
   n_ctas = (int)R.roles.size();
   DeviceArena &C = g->ctl, &B = g->bulk;
@@ -500,7 +511,8 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.emit_pub = C.take<unsigned>(P.T);
     P.emit_fin = C.take<unsigned>(P.T);
     P.fetched = C.take<unsigned>(1);
-    P.emit_done = C.take<unsigned>((size_t)P.T * std::max(1, emit_ctas));
+    P.emit_done = C.take<unsigned>((size_t)std::max(1, H.NE));
+    P.NE = H.NE; P.G = H.G;
     P.nbar = C.take<unsigned>(1);
     P.stats = C.take<PPTStats>(1);
     P.update_log = B.take<int>(g->update_log_cap); P.update_log_cap = g->update_log_cap;

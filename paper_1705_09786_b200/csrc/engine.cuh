@@ -810,44 +810,63 @@ __device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) {
   return P.muf_override > 0 ? P.muf_override : C.muf;
 }
 
-// Warp 0 of the leader tile: take up to 32 candidate messages (ring slot per lane, in processing order), cut
-// the batch at the row capacity and at the message that triggers an update (Sec. 3), publish it.
-// Returns the number of messages taken.
-__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, unsigned slot, int ncand) {
+// Inclusive prefix sums over 64 values held two per lane (v[0]: index lane, v[1]: index lane + 32).
+__device__ __forceinline__ void scan64(int (&v)[2], const int lane) {
+#pragma unroll
+  for (int j = 0; j < 2; j++)
+    for (int o = 1; o < 32; o <<= 1) { const int t = __shfl_up_sync(0xffffffffu, v[j], o); if (lane >= o) v[j] += t; }
+  v[1] += __shfl_sync(0xffffffffu, v[0], 31);
+}
+__device__ __forceinline__ unsigned long long ballot64(const bool p0, const bool p1) {
+  return (unsigned long long)__ballot_sync(0xffffffffu, p0) | ((unsigned long long)__ballot_sync(0xffffffffu, p1) << 32);
+}
+
+// Warp 0 of the leader: take up to 64 candidate messages (two ring slots per lane, in processing order: candidate
+// lane and candidate lane + 32), cut the batch at the row capacity and at the message that triggers an update (Sec. 3),
+// publish it.  Returns the number of messages taken.
+__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, const unsigned (&slot)[2], int ncand) {
   const int lane = threadIdx.x & 31;
   Ring& R = P.ring[dir];
-  Hdr h = {0, 0, 0, 0, 0, 0, 0, 0};
-  if (lane < ncand) {
-    const int4* e = reinterpret_cast<const int4*>(&R.e[slot]);
-    int4 a = __ldcg(e), b = __ldcg(e + 1);
-    h.inst = a.x; h.seq = a.y; h.slot = a.z; h.it = a.w; h.u = b.x; h.port = b.y; h.rows = b.z; h.flags = b.w;
+  Hdr h[2];
+  int cum[2];
+#pragma unroll
+  for (int j = 0; j < 2; j++) {
+    h[j] = Hdr{0, 0, 0, 0, 0, 0, 0, 0};
+    if (lane + 32 * j < ncand) {
+      const int4* e = reinterpret_cast<const int4*>(&R.e[slot[j]]);
+      int4 a = __ldcg(e), b = __ldcg(e + 1);
+      h[j].inst = a.x; h[j].seq = a.y; h[j].slot = a.z; h[j].it = a.w; h[j].u = b.x; h[j].port = b.y; h[j].rows = b.z; h[j].flags = b.w;
+    }
+    cum[j] = lane + 32 * j < ncand ? (h[j].rows > 0 ? h[j].rows : 1) : 0;
   }
-  const int rows = lane < ncand ? (h.rows > 0 ? h.rows : 1) : 0;
-  int cum = rows;
-  for (int o = 1; o < 32; o <<= 1) { int v = __shfl_up_sync(0xffffffffu, cum, o); if (lane >= o) cum += v; }
-  const bool ok = lane < ncand && cum <= P.BM;
-  unsigned okm = __ballot_sync(0xffffffffu, ok);
-  int take = __ffs(~okm) - 1;
-  if (take < 0) take = 32;
-  if (take == 0) { fail(C, ST_OVERFLOW, P.node, rows); return 0; }     // a single message larger than a batch
+  const int rows0 = cum[0];
+  scan64(cum, lane);
+  const bool ok0 = lane < ncand && cum[0] <= P.BM, ok1 = lane + 32 < ncand && cum[1] <= P.BM;
+  const unsigned long long okm = ballot64(ok0, ok1);
+  int take = okm == ~0ull ? 64 : __ffsll((long long)~okm) - 1;
+  if (take == 0) { fail(C, ST_OVERFLOW, P.node, rows0); return 0; }     // a single message larger than a batch
   bool upd = false;
-  const bool eval = (h.flags & HDR_EVAL) != 0;
-  const int eval0 = __shfl_sync(0xffffffffu, (int)eval, 0);
+  const int eval0 = __shfl_sync(0xffffffffu, (int)((h[0].flags & HDR_EVAL) != 0), 0);
   if (dir == BWD && !eval0) {
     const int muf = node_muf(C, P);
-    unsigned tm = __ballot_sync(0xffffffffu, ok && lane < take && (S.ls.n_acc + cum >= muf));
-    if (tm) { take = __ffs(tm); upd = true; }
+    const unsigned long long tm = ballot64(ok0 && lane < take && S.ls.n_acc + cum[0] >= muf,
+                                           ok1 && lane + 32 < take && S.ls.n_acc + cum[1] >= muf);
+    if (tm) { take = __ffsll((long long)tm); upd = true; }
   }
-  const int total = __shfl_sync(0xffffffffu, cum, take - 1);
-  if (lane < take) {
-    P.sched[(S.ls.sched_w + lane) & P.sched_mask] = slot;
+  const int t0v = __shfl_sync(0xffffffffu, cum[0], (take - 1) & 31), t1v = __shfl_sync(0xffffffffu, cum[1], (take - 1) & 31);
+  const int total = take > 32 ? t1v : t0v;
+#pragma unroll
+  for (int j = 0; j < 2; j++) {
+    const int i = lane + 32 * j;
+    if (i >= take) continue;
+    P.sched[(S.ls.sched_w + i) & P.sched_mask] = slot[j];
     if (!C.det) {
-      int4* b = reinterpret_cast<int4*>(&P.bhdr[(S.ls.batch_w & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + lane]);
-      b[0] = make_int4(h.inst, h.seq, h.slot, h.it);
-      b[1] = make_int4(h.u, h.port, h.rows, h.flags);
+      int4* b = reinterpret_cast<int4*>(&P.bhdr[(S.ls.batch_w & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + i]);
+      b[0] = make_int4(h[j].inst, h[j].seq, h[j].slot, h[j].it);
+      b[1] = make_int4(h[j].u, h[j].port, h[j].rows, h[j].flags);
     }
     if (!eval0) {
-      long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      long long key = key_of(C, P.node, h[j].slot, h[j].it, h[j].u, P.U);
       if (key >= 0) {
         if (dir == FWD) P.vcache[key] = S.ls.version;
         else {
@@ -898,20 +917,23 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
 // Asynchronous mode, warp 0 of the leader: whatever is pending, backward first (App. A).
 __device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
   const int lane = threadIdx.x & 31;
-  unsigned slot[2], mready[2];
+  unsigned slot[2][2];
+  bool mready[2][2];
 #pragma unroll
-  for (int dir = 0; dir < 2; dir++) {            // both rings are polled before either result is needed
-    const unsigned t = S.ls.head[dir] + lane;
-    slot[dir] = t & P.ring[dir].mask;
-    mready[dir] = (ld_acq(&P.ring[dir].seq[slot[dir]]) == t + 1u) ? 1u : 0u;
-  }
+  for (int dir = 0; dir < 2; dir++)               // both rings are polled before either result is needed
+#pragma unroll
+    for (int j = 0; j < 2; j++) {
+      const unsigned t = S.ls.head[dir] + lane + 32 * j;
+      slot[dir][j] = t & P.ring[dir].mask;
+      mready[dir][j] = ld_acq(&P.ring[dir].seq[slot[dir][j]]) == t + 1u;
+    }
   int nready[2];
 #pragma unroll
   for (int dir = 0; dir < 2; dir++) {
-    const unsigned m = __ballot_sync(0xffffffffu, mready[dir] != 0);
-    nready[dir] = m == 0xffffffffu ? 32 : __ffs(~m) - 1;
+    const unsigned long long m = ballot64(mready[dir][0], mready[dir][1]);
+    nready[dir] = m == ~0ull ? 64 : __ffsll((long long)~m) - 1;
   }
-  // Backward first (App. A), but a cycle costs the same whether the batch holds 2 messages or 32: a short backward
+  // Backward first (App. A), but a cycle costs the same whether the batch holds 2 messages or 64: a short backward
   // queue gives way to a longer forward queue and is taken once it has grown to half a batch, has caught up with the
   // forward queue, or the forward queue has run dry (max_active_keys bounds the forward supply, so it always does).
   const bool fwd_first = !(C.tune & 128) && nready[BWD] < MAX_BATCH_MSGS / 2 && nready[FWD] > nready[BWD];
@@ -919,7 +941,7 @@ __device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileSh
     const int dir = (k == 0) == fwd_first ? FWD : BWD;
     const int n = nready[dir];
     if (n == 0) continue;
-    int take = form_batch(C, P, S, dir, slot[dir], n);
+    int take = dir == FWD ? form_batch(C, P, S, FWD, slot[FWD], n) : form_batch(C, P, S, BWD, slot[BWD], n);
     if (lane == 0) S.ls.head[dir] += take;
     __syncwarp();
     return true;
@@ -979,9 +1001,11 @@ __device__ __noinline__ void leader_schedule_round(const Ctx& C, DevPPT& P, Tile
     if (warp == 0) {
       unsigned pos = 0;
       while (pos < n) {
-        int nc = (int)min(32u, n - pos);
-        unsigned slot = 0;
-        if (lane < nc) slot = (head + (unsigned)(P.sortbuf[pos + lane] & 0xfffffull)) & R.mask;
+        int nc = (int)min((unsigned)MAX_BATCH_MSGS, n - pos);
+        unsigned slot[2] = {0, 0};
+#pragma unroll
+        for (int j = 0; j < 2; j++)
+          if (lane + 32 * j < nc) slot[j] = (head + (unsigned)(P.sortbuf[pos + lane + 32 * j] & 0xfffffull)) & R.mask;
         int take = form_batch(C, P, S, dir, slot, nc);
         if (take <= 0) break;
         pos += take;
@@ -1064,66 +1088,73 @@ __device__ __forceinline__ void init_leader_state(TileShared& S) {              
 __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared& S, const unsigned my_batch) {
   const int lane = threadIdx.x & 31;
   const int in = P.in_dim;
-    const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]);
-    const int4 d0 = __ldcg(dp), d1 = __ldcg(dp + 1);          // same address in every lane
+  const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]);
+  const int4 d0 = __ldcg(dp), d1 = __ldcg(dp + 1);          // same address in every lane
+  const int cnt = d0.y, ddir = d0.z;
+  Hdr h[2];
+  int cum[2], rows[2];
+#pragma unroll
+  for (int j = 0; j < 2; j++) {                             // message lane + 32 j
+    const int i = lane + 32 * j;
     int4 ha = make_int4(0, 0, 0, 0), hb = make_int4(0, 0, 0, 0);
-    if (!C.det) {                                             // headers travel with the descriptor: load both at once
-      const int4* e = reinterpret_cast<const int4*>(&P.bhdr[(my_batch & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + lane]);
+    if (!C.det) {                                           // headers travel with the descriptor: load both at once
+      const int4* e = reinterpret_cast<const int4*>(&P.bhdr[(my_batch & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + i]);
       ha = __ldcg(e); hb = __ldcg(e + 1);
-    }
-    const int cnt = d0.y, ddir = d0.z;
-    if (C.det && lane < cnt) {
-      const unsigned slot = P.sched[((unsigned)d0.x + lane) & P.sched_mask];
+    } else if (i < cnt) {
+      const unsigned slot = P.sched[((unsigned)d0.x + i) & P.sched_mask];
       const int4* e = reinterpret_cast<const int4*>(&P.ring[ddir].e[slot]);
       ha = __ldcg(e); hb = __ldcg(e + 1);
     }
-    Hdr h; h.inst = ha.x; h.seq = ha.y; h.slot = ha.z; h.it = ha.w; h.u = hb.x; h.port = hb.y; h.rows = hb.z; h.flags = hb.w;
-    if (h.rows <= 0) h.rows = 1;
-    const int rows = lane < cnt ? h.rows : 0;
-    int cum = rows;
-    for (int o = 1; o < 32; o <<= 1) { int v = __shfl_up_sync(0xffffffffu, cum, o); if (lane >= o) cum += v; }
-    const int total = __shfl_sync(0xffffffffu, cum, 31);
-    const int off = cum - rows;
-    long long key = 0;
-    if (lane < cnt) {
-      key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
-      S.hdr[lane] = h; S.key[lane] = key; S.rowoff[lane] = off;
-      if (key >= 0 && total <= P.BM) {
-        if (P.kind != LOOKUP) {
-          const float* x0 = msg_x(C, P, h, key);
-          for (int r = 0; r < rows; r++) { S.rowmsg[off + r] = lane; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
-        } else {                                              // table rows and the rows of the incoming gradient
-          const DevInst& I = C.inst;
-          const long long base = I.offsets[h.inst];
-          const float* g0 = P.gbuf + (size_t)key * P.rows_max * P.out_dim;
-          for (int r = 0; r < rows; r++) {
-            const int id = I.tokens[base + (I.kind == 3 ? r : h.u)];
-            S.rowmsg[off + r] = lane; S.rowptr[off + r] = g0 + (size_t)r * P.out_dim;
-            S.rowid[off + r] = (unsigned)id < (unsigned)in ? id : -1;
-          }
-        }
+    h[j].inst = ha.x; h[j].seq = ha.y; h[j].slot = ha.z; h[j].it = ha.w; h[j].u = hb.x; h[j].port = hb.y; h[j].rows = hb.z; h[j].flags = hb.w;
+    if (h[j].rows <= 0) h[j].rows = 1;
+    rows[j] = i < cnt ? h[j].rows : 0;
+    cum[j] = rows[j];
+  }
+  scan64(cum, lane);
+  const int total = __shfl_sync(0xffffffffu, cum[1], 31);
+  bool badkey = false;
+#pragma unroll
+  for (int j = 0; j < 2; j++) {
+    const int i = lane + 32 * j;
+    if (i >= cnt) continue;
+    const int off = cum[j] - rows[j];
+    const long long key = key_of(C, P.node, h[j].slot, h[j].it, h[j].u, P.U);
+    S.hdr[i] = h[j]; S.key[i] = key; S.rowoff[i] = off;
+    if (key < 0) { badkey = true; continue; }
+    if (total > P.BM) continue;
+    if (P.kind != LOOKUP) {
+      const float* x0 = msg_x(C, P, h[j], key);
+      for (int r = 0; r < rows[j]; r++) { S.rowmsg[off + r] = i; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
+    } else {                                                // table rows and the rows of the incoming gradient
+      const DevInst& I = C.inst;
+      const long long base = I.offsets[h[j].inst];
+      const float* g0 = P.gbuf + (size_t)key * P.rows_max * P.out_dim;
+      for (int r = 0; r < rows[j]; r++) {
+        const int id = I.tokens[base + (I.kind == 3 ? r : h[j].u)];
+        S.rowmsg[off + r] = i; S.rowptr[off + r] = g0 + (size_t)r * P.out_dim;
+        S.rowid[off + r] = (unsigned)id < (unsigned)in ? id : -1;
       }
     }
-    if (P.kind == LOOKUP && ddir == BWD && total <= P.BM) {   // chain the batch rows that hit the same table row
-      __syncwarp();
-      for (int b = lane; b < total; b += 32) {
-        const int id = S.rowid[b];
-        int nx = -1, first = 1;
-        for (int k = b + 1; k < total; k++) if (S.rowid[k] == id) { nx = k; break; }
-        for (int k = 0; k < b; k++) if (S.rowid[k] == id) { first = 0; break; }
-        S.rownext[b] = nx; S.rowfirst[b] = id >= 0 ? first : 0;
-      }
+  }
+  if (P.kind == LOOKUP && ddir == BWD && total <= P.BM) {   // chain the batch rows that hit the same table row
+    __syncwarp();
+    for (int b = lane; b < total; b += 32) {
+      const int id = S.rowid[b];
+      int nx = -1, first = 1;
+      for (int k = b + 1; k < total; k++) if (S.rowid[k] == id) { nx = k; break; }
+      for (int k = 0; k < b; k++) if (S.rowid[k] == id) { first = 0; break; }
+      S.rownext[b] = nx; S.rowfirst[b] = id >= 0 ? first : 0;
     }
-    const unsigned bad = __ballot_sync(0xffffffffu, lane < cnt && key < 0);
-    if (lane == 0) {
-      S.rowoff[cnt] = total;
-      BatchDesc dd; dd.sched_start = (unsigned)d0.x; dd.count = d0.y; dd.dir = d0.z; dd.flags = d0.w;
-      dd.n_upd = d1.x; dd.nrows = d1.y; dd.upd_t = d1.z; dd.pad1 = 0;
-      if (bad) { S.ok = 0; dd.pad1 = 1; }
-      if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; dd.pad1 = 1; }
-      S.desc = dd;
-    }
-
+  }
+  const unsigned bad = __ballot_sync(0xffffffffu, badkey);
+  if (lane == 0) {
+    S.rowoff[cnt] = total;
+    BatchDesc dd; dd.sched_start = (unsigned)d0.x; dd.count = d0.y; dd.dir = d0.z; dd.flags = d0.w;
+    dd.n_upd = d1.x; dd.nrows = d1.y; dd.upd_t = d1.z; dd.pad1 = 0;
+    if (bad) { S.ok = 0; dd.pad1 = 1; }
+    if (total > P.BM) { fail(C, ST_OVERFLOW, P.node, total); S.ok = 0; dd.pad1 = 1; }
+    S.desc = dd;
+  }
 }
 
 // With scheduler CTAs: the assembled context of batch `batch`, one 16-byte piece per thread (whole CTA, no barrier).
@@ -1147,7 +1178,9 @@ __device__ __noinline__ void publish_ctx_block(const Ctx& C, DevPPT& P, TileShar
 
 // Emission of a batch by one CTA: reduce the tiles' partial input gradients for the rows this CTA emits, then walk
 // the messages through the parameter-free nodes.  `parity` selects the per-batch buffers, `stage` the staging rows.
-__device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile, TileShared& S, const BatchDesc d,
+// This CTA emits share `tile` of `NT` shares: message i belongs to share i % NT (row-wise forks: every share walks every
+// message and takes the rows j = part (mod NT)).
+__device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile, const int NT, TileShared& S, const BatchDesc d,
                                         const unsigned parity, float* stage, WalkAcc& acc) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const DevNode& N = g_nodes[P.node];
@@ -1158,7 +1191,7 @@ __device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile,
       for (int idx = tid; idx < nb * in; idx += THREADS) stage[idx] = emit_round(stage[idx]);
       __syncthreads();
     }
-    const bool split = C.wide && P.T > 1;          // share row-wise forks among the node's tiles
+    const bool split = C.wide && NT > 1;           // share row-wise forks among the emitting CTAs
     if (dir == BWD && P.kind != LOOKUP && !(P.flags & 1) && (P.T > 1 || P.kind == GRUCELL)) {
       // Sum the tiles' partial input gradients (tile order) for the rows this tile emits; every thread keeps
       // all T loads of an element in flight.
@@ -1167,12 +1200,12 @@ __device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile,
       const float* pb = P.kind == GRUCELL ? P.part2 + (size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) * pstride : nullptr;
       const float* dirb = pb ? pb + (size_t)P.T * pstride : nullptr;
       const int H = out;
-      for (int i = split ? 0 : tile; i < count; i += split ? 1 : P.T) {
-        const int part = (tile - i % P.T + P.T) % P.T;
+      for (int i = split ? 0 : tile; i < count; i += split ? 1 : NT) {
+        const int part = (tile - i % NT + NT) % NT;
         const int ro = S.rowoff[i], ne = S.hdr[i].rows * in;
         for (int k = tid; k < ne; k += THREADS) {
           const int row = k / in;
-          if (part != 0 && row % P.T != part) continue;
+          if (part != 0 && row % NT != part) continue;
           const size_t e = (size_t)ro * in + k;
           const int c = k - row * in;
           float sum = 0.f;
@@ -1189,19 +1222,19 @@ __device__ __noinline__ void emit_batch(const Ctx& C, DevPPT& P, const int tile,
       }
       __syncthreads();
     }
-    if (tid == 0) S.pool.outstanding = split ? count : (tile < count ? (count - tile + P.T - 1) / P.T : 0);
+    if (tid == 0) S.pool.outstanding = split ? count : (tile < count ? (count - tile + NT - 1) / NT : 0);
     __syncthreads();
     const long long tw0 = clock64();
     int mine = 0;
     for (int i = 0; i < count; i++) {
-      const int part = (tile - i % P.T + P.T) % P.T;
+      const int part = (tile - i % NT + NT) % NT;
       if (!split && part != 0) continue;
       if ((mine++ % WARPS) != warp) continue;
       const Hdr& h = S.hdr[i];
       Frame f;
       f.iter = 0; f.inst = h.inst; f.seq = h.seq; f.slot = h.slot; f.it = h.it; f.u = h.u; f.port = h.port;
       f.rows = h.rows; f.flags = h.flags; f.nsum = 1; f.sstride = 0;
-      f.part = split ? part : 0; f.nparts = split ? P.T : 1;
+      f.part = split ? part : 0; f.nparts = split ? NT : 1;
       f.ibase = C.inst.offsets ? C.inst.offsets[h.inst] : 0; f.ebase = C.inst.edge_off ? C.inst.edge_off[h.inst] : 0;
       if (dir == FWD) {
         f.node = N.succ_node[0]; f.aport = N.succ_port[0]; f.dir = FWD; f.dim = out; f.ld = out;
@@ -1450,12 +1483,11 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         // of them are done with the batch that used these buffers before
         if (warp == 0 && my_batch > (unsigned)C.depth) {
           const unsigned j = my_batch - 1u - (unsigned)C.depth;
-          const int ne = P.T * C.emit_ctas;
           unsigned it = 0;
           for (;;) {
             bool ok = true;
-            for (int e = lane; e < ne; e += 32)
-              if ((unsigned)(e % C.emit_ctas) == j % (unsigned)C.emit_ctas) ok = ok && ld_acq(&P.emit_done[e]) >= j + 1u;
+            for (int e = lane; e < P.NE; e += 32)
+              if ((unsigned)(e % P.G) == j % (unsigned)P.G) ok = ok && ld_acq(&P.emit_done[e]) >= j + 1u;
             if (__all_sync(0xffffffffu, ok)) break;
             if ((++it & 15u) == 0) {
               unsigned bad = 0;
@@ -1471,6 +1503,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       const int nb = S.rowoff[count];
       const bool eval = count > 0 && (S.hdr[0].flags & HDR_EVAL);
       AMP_PHASE(2);
+      if (tid == 0 && count > 0) { S.phase[13 + dir] += 1ull; if (d.flags & BATCH_UPDATE) S.phase[15] += 1ull; }
 
       if (count > 0 && P.kind == LINEAR) {
         // stage the cached inputs of the batch
@@ -1622,7 +1655,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           if (warp_uniform(bw) == my_batch) leader_try_schedule(C, P, S);
           if (lane == 0) S.phase[8] += (unsigned long long)(clock64() - tq);
         }
-        if (!C.emit_ctas) emit_batch(C, P, tile, S, d, my_batch, stage_k, acc);
+        if (!C.emit_ctas) emit_batch(C, P, tile, P.T, S, d, my_batch, stage_k, acc);
         AMP_PHASE(6);
       }
       if (C.emit_ctas && tid == 0) {                                        // hand the batch to this tile's emitter CTAs
@@ -1653,14 +1686,16 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
 // emitter CTA (asynchronous mode): the partner of one tile.  It emits the tile's share of every batch while the tile
 // already stages and computes the next one.
 // ------------------------------------------------------------------------------------------------
-__device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int tile, const int which, TileShared& S,
+__device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int which, TileShared& S,
                                           const unsigned long long t0) {
+  const int tile = 0;                                         // whose termination flag this emitter watches
+  const int grp = which % P.G, member = which / P.G, members = (P.NE - grp + P.G - 1) / P.G;
   const int tid = threadIdx.x, warp = tid >> 5;
   if (tid < POOL) S.pool.ready[tid] = 0;
   if (tid < 16) S.phase[tid] = 0;
   if (tid == 0) { S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
   __syncthreads();
-  unsigned my_batch = (unsigned)which;          // this emitter takes batches which, which + E, which + 2E, ...
+  unsigned my_batch = (unsigned)grp;            // this emitter's group takes batches grp, grp + G, grp + 2G, ...
   WalkAcc acc = {0, 0};
   unsigned long long* const rc = C.g->role_cycles + 8 + 8 * (int)(&P - g_ppts);
   long long tp = clock64();
@@ -1700,15 +1735,15 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int til
     const BatchDesc d = S.desc;
     if (!S.ok || d.pad1) break;
     EMIT_PHASE(4);
-    if (d.count > 0) emit_batch(C, P, tile, S, d, my_batch + 1u, P.stage + (size_t)((my_batch + 1u) % (unsigned)C.depth) * P.stage_floats, acc);
+    if (d.count > 0) emit_batch(C, P, member, members, S, d, my_batch + 1u, P.stage + (size_t)((my_batch + 1u) % (unsigned)C.depth) * P.stage_floats, acc);
     __syncthreads();
     EMIT_PHASE(5);
     if (tid == 0) S.phase[6] += 1ull;
-    if (tid == 0) { __threadfence(); st_rel(&P.emit_done[tile * C.emit_ctas + which], my_batch + 1u); }
-    my_batch += (unsigned)C.emit_ctas;
+    if (tid == 0) { __threadfence(); st_rel(&P.emit_done[which], my_batch + 1u); }
+    my_batch += (unsigned)P.G;
   }
   __syncthreads();
-  if (tile == 0 && which == 0 && tid >= 3 && tid < 7) rc[tid] = S.phase[tid];
+  if (which == 0 && tid >= 3 && tid < 7) rc[tid] = S.phase[tid];
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1994,7 +2029,7 @@ __global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constan
   __syncthreads();
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);
-  else if (role.kind == 1) emitter_main(C, g_ppts[role.ppt], role.tile, role.pad, SU.t, t0);
+  else if (role.kind == 1) emitter_main(C, g_ppts[role.ppt], role.pad, SU.t, t0);
   else if (role.kind == 2) scheduler_main(C, g_ppts[role.ppt], SU.t, t0);
   else ppt_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
 }

@@ -7,7 +7,8 @@ namespace amp {
 constexpr int MAX_PORTS = 8;
 constexpr int THREADS = 256;          // threads per CTA
 constexpr int WARPS = THREADS / 32;
-constexpr int MAX_BATCH_MSGS = 32;    // messages per micro-batch (one warp schedules them)
+constexpr int MAX_BATCH_MSGS = 64;    // messages per micro-batch (one warp schedules them, two messages per lane)
+constexpr int MAX_BATCH_ROWS = 64;    // payload rows per micro-batch
 constexpr int BATCH_BLOCKS = 16;     // batch context blocks in flight between a node's scheduler and its tiles / emitters
 constexpr int MAX_SMEM_NODES = 40;    // IR nodes / PPT nodes whose tables are kept in shared memory
 constexpr int MAX_SMEM_PPTS = 16;
@@ -40,10 +41,10 @@ struct __align__(16) BatchCtx {
   Hdr hdr[MAX_BATCH_MSGS];
   long long key[MAX_BATCH_MSGS];
   int rowoff[MAX_BATCH_MSGS + 4];       // first batch row of every message; [count] = rows of the batch
-  int rowmsg[64];                       // message of every batch row
-  const float* rowptr[64];              // cached input row (LOOKUP: incoming gradient row) of every batch row
-  int rowid[64], rownext[64];           // LOOKUP: table row of every batch row; next batch row with the same table row (-1: none)
-  int rowfirst[64];                     // LOOKUP: no earlier batch row has the same table row
+  int rowmsg[MAX_BATCH_ROWS];                       // message of every batch row
+  const float* rowptr[MAX_BATCH_ROWS];              // cached input row (LOOKUP: incoming gradient row) of every batch row
+  int rowid[MAX_BATCH_ROWS], rownext[MAX_BATCH_ROWS];           // LOOKUP: table row of every batch row; next batch row with the same table row (-1: none)
+  int rowfirst[MAX_BATCH_ROWS];                     // LOOKUP: no earlier batch row has the same table row
 };
 static_assert(sizeof(BatchCtx) % 16 == 0, "batch context blocks are copied in 16-byte pieces");
 
@@ -95,7 +96,9 @@ struct DevPPT {
   float* stage;                       // [2][BM][max(in_dim, out_dim)] reduced input gradients / gathered rows, by batch parity
   long long stage_floats;
   unsigned *emit_pub, *emit_fin;      // per tile: batches handed to its emitter CTAs; set once the last one is out
-  unsigned* emit_done;                // [tile][emitter]: last batch (index + 1) the emitter has finished
+  unsigned* emit_done;                // [emitter]: last batch (index + 1) the emitter has finished
+  int NE, G;                          // emitter CTAs of the node; groups that take batches in turn (emitter q: group q % G,
+                                      // member q / G, which emits its share of the messages of every batch of its group)
   unsigned* fetched;                  // batches tile 0 has fetched (paces the scheduler CTA)
   float* part2;                       // GRUCELL scratch
   unsigned* nbar;                     // barrier counter of the node's tiles
@@ -142,7 +145,7 @@ struct Globals {                      // mutable run state in device memory (zer
   unsigned long long role_cycles[8 + 8 * MAX_SMEM_PPTS];
 };
 
-struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of its emitter CTAs (pad = which one), 2: the node's scheduler CTA
+struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of the node's emitter CTAs (pad = which one), 2: the node's scheduler CTA
 
 struct Ctx {
   DevNode* nodes; int n_nodes;
@@ -163,7 +166,7 @@ struct Ctx {
   int mak, muf, det, eval, IT;
   int wide;                           // the graph has row-wise forks (Ungroup / Group)
   int bf16;                           // payloads rounded to bfloat16 at emission
-  int emit_ctas;                      // emitter CTAs per tile (0: tiles emit themselves)
+  int emit_ctas;                      // the nodes have emitter CTAs (0: tiles emit themselves)
   int sched_ctas;                     // every PPT node has a scheduler CTA (its leader) of its own
   int depth;                          // per-batch buffers (partials, staging rows) are reused every `depth` batches
   int tune;                           // experiment switches (environment AMPNET_TUNE): 2 no look-ahead, 4 no per-node counters
