@@ -378,7 +378,11 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
     if (max_batch_rows > 0) BM = std::max(rows_max, std::min(BM, max_batch_rows));
     if (rows_max > 64) return set_err(g, AMPNET_EINVAL, "node %d: %d payload rows per message exceed the supported 64", P.node, rows_max);
     P.J = P.kind == LOOKUP ? 4 : j_bucket(P.in);
-    if (P.kind == LOOKUP) { P.T = 1; P.R = 0; P.BM = BM; P.smem_floats = tile_smem_floats(P, 0, BM); used += 1; continue; }
+    if (P.kind == LOOKUP) {
+      // a large table means gathers and accumulations bound by DRAM latency: deal its rows to several tiles
+      P.T = (P.in >= 4096 && (tiles_cap == 0 || tiles_cap >= 8)) ? 4 : 1;
+      P.R = 0; P.BM = BM; P.smem_floats = tile_smem_floats(P, 0, BM); used += P.T; continue;
+    }
     // small nodes (a classifier) still emit one message per gradient: give them tiles for the emission work
     const double share = std::max((double)P.nmat * P.in * P.out / total_w, 0.1);
     int T = 1 + (int)std::floor(share * avail);
@@ -519,8 +523,8 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     if (H.kind == LOOKUP) {
       P.A = C.take<float>(H.nW);
       P.touched_flag = C.take<int>(H.in);
-      P.touched_list = C.take<int>(H.in);
-      P.touched_n = C.take<int>(1);
+      P.touched_list = C.take<int>((size_t)H.in + H.T);      // one segment of ceil(V / T) entries per tile
+      P.touched_n = C.take<int>(H.T);
     }
     P.smem_floats = (int)H.smem_floats;
     max_smem_floats = std::max(max_smem_floats, H.smem_floats);

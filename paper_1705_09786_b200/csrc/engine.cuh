@@ -1291,20 +1291,25 @@ struct OptStep {
 // Embedding table, one batch (whole CTA).  Forward: gather the table rows into the staging rows.  Backward: accumulate
 // in message order, as if the rows arrived one by one: the first batch row of every table row adds the gradients of all
 // batch rows that hit the same table row, in order.  A warp takes whole rows and keeps ten loads per lane in flight.
-__device__ __noinline__ void lookup_batch(DevPPT& P, TileShared& S, const int dir, const int nb, float* stage_k) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, out = P.out_dim;
+// The table rows are dealt to the node's tiles (row id belongs to tile id % T): every tile sees the whole batch and
+// handles the batch rows whose table row it owns, with a list of touched rows of its own.
+__device__ __noinline__ void lookup_batch(DevPPT& P, TileShared& S, const int dir, const int nb, float* stage_k, const int tile) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, out = P.out_dim, T = P.T;
+  int* const tlist = P.touched_list + (size_t)tile * ((P.in_dim + T - 1) / T);
   constexpr int K = 5;                                      // column chunks of 32 per pass
   if (dir == FWD) {
     for (int b0 = warp * 2; b0 < nb; b0 += WARPS * 2)       // two rows per pass
       for (int c0 = 0; c0 < out; c0 += 32 * K) {
         float v[2][K];
+        bool mine[2];
 #pragma unroll
         for (int r = 0; r < 2; r++) {
           const int id = b0 + r < nb ? S.rowid[b0 + r] : -1;
+          mine[r] = b0 + r < nb && (id >= 0 ? id % T == tile : tile == 0);      // rows outside the table read as zero
 #pragma unroll
           for (int k = 0; k < K; k++) {
             const int c = c0 + k * 32 + lane;
-            v[r][k] = (id >= 0 && c < out) ? P.W[(size_t)id * out + c] : 0.f;
+            v[r][k] = (mine[r] && id >= 0 && c < out) ? P.W[(size_t)id * out + c] : 0.f;
           }
         }
 #pragma unroll
@@ -1312,13 +1317,14 @@ __device__ __noinline__ void lookup_batch(DevPPT& P, TileShared& S, const int di
 #pragma unroll
           for (int k = 0; k < K; k++) {
             const int c = c0 + k * 32 + lane;
-            if (b0 + r < nb && c < out) stage_k[(size_t)(b0 + r) * out + c] = emit_round(v[r][k]);
+            if (mine[r] && c < out) stage_k[(size_t)(b0 + r) * out + c] = emit_round(v[r][k]);
           }
       }
   } else {
     for (int b = warp; b < nb; b += WARPS) {
       if (!S.rowfirst[b]) continue;
       const int id = S.rowid[b];
+      if (id % T != tile) continue;
       int fresh = 0;
       if (lane == 0) fresh = !P.touched_flag[id];
       float* arow = P.A + (size_t)id * out;
@@ -1341,35 +1347,38 @@ __device__ __noinline__ void lookup_batch(DevPPT& P, TileShared& S, const int di
 #pragma unroll
         for (int k = 0; k < K; k++) { const int c = c0 + k * 32 + lane; if (c < out) arow[c] = a[k]; }
       }
-      if (lane == 0 && fresh) { P.touched_flag[id] = 1; P.touched_list[atomicAdd(P.touched_n, 1)] = id; }
+      if (lane == 0 && fresh) { P.touched_flag[id] = 1; tlist[atomicAdd(P.touched_n + tile, 1)] = id; }
     }
   }
 }
 
 // Local update of a tile's share of the node's parameters (whole CTA; ends with a block barrier).
 __device__ __noinline__ void tile_update(const Ctx& C, DevPPT& P, const TileMem& M, const BatchDesc& d, const int R,
-                                         const int r_begin) {
+                                         const int r_begin, const int tile) {
   const int tid = threadIdx.x, in = P.in_dim, out = P.out_dim;
   const int nmat = P.kind == GRUCELL ? 3 : 1;
   const OptStep os(C, P, d);
   if (P.kind == LOOKUP) {
     __threadfence_block();
-    const int nt = *P.touched_n;
-    for (int base = tid; base < nt * out; base += 4 * THREADS) {       // four elements in flight per thread
-      float w[4], a[4]; size_t o[4];
+    // this tile's touched table rows, a row per warp with ten elements per lane in flight
+    int* const tlist = P.touched_list + (size_t)tile * ((P.in_dim + P.T - 1) / P.T);
+    const int nt = P.touched_n[tile];
+    const int lane = tid & 31, warp = tid >> 5;
+    constexpr int K = 5;
+    for (int k = warp; k < nt; k += WARPS) {
+      const int id = tlist[k];
+      const size_t o0 = (size_t)id * out;
+      for (int c0 = 0; c0 < out; c0 += 32 * K) {
+        float w[K], a[K];
 #pragma unroll
-      for (int j = 0; j < 4; j++) {
-        const int idx = base + j * THREADS;
-        if (idx < nt * out) { o[j] = (size_t)P.touched_list[idx / out] * out + idx % out; w[j] = P.W[o[j]]; a[j] = P.A[o[j]]; }
+        for (int j = 0; j < K; j++) { const int c = c0 + j * 32 + lane; if (c < out) { w[j] = P.W[o0 + c]; a[j] = P.A[o0 + c]; } }
+#pragma unroll
+        for (int j = 0; j < K; j++) { const int c = c0 + j * 32 + lane; if (c < out) { os.apply(w[j], a[j], o0 + c); P.W[o0 + c] = w[j]; P.A[o0 + c] = a[j]; } }
       }
-#pragma unroll
-      for (int j = 0; j < 4; j++)
-        if (base + j * THREADS < nt * out) { os.apply(w[j], a[j], o[j]); P.W[o[j]] = w[j]; P.A[o[j]] = a[j]; }
+      if (lane == 0) P.touched_flag[id] = 0;
     }
     __syncthreads();
-    for (int k = tid; k < nt; k += THREADS) P.touched_flag[P.touched_list[k]] = 0;
-    __syncthreads();
-    if (tid == 0) *P.touched_n = 0;
+    if (tid == 0) P.touched_n[tile] = 0;
   } else {
     const size_t nW = (size_t)nmat * out * in;
     for (int m = 0; m < nmat; m++) {
@@ -1632,14 +1641,14 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         }
       } else if (count > 0 && P.kind == LOOKUP) {
         const long long tl0 = clock64();
-        lookup_batch(P, S, dir, nb, stage_k);
+        lookup_batch(P, S, dir, nb, stage_k, tile);
         __syncthreads();
         if (tid == 0) { S.phase[9 + 2 * dir] += (unsigned long long)(clock64() - tl0); S.phase[10 + 2 * dir] += (unsigned long long)nb; }
       }
       __syncthreads();
       AMP_PHASE(3);
       // ---- local update (Sec. 3): theta -= lr * A / n, accumulator cleared --------------------------
-      if (d.flags & BATCH_UPDATE) tile_update(C, P, M, d, R, r_begin);
+      if (d.flags & BATCH_UPDATE) tile_update(C, P, M, d, R, r_begin, tile);
       AMP_PHASE(4);
       // ---- all tiles of the node done with the batch, then emit ------------------------------------
       if (count > 0) {
