@@ -357,47 +357,77 @@ size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
          (size_t)(2 * P.nmat + 1) * BM * R + 64;
 }
 
-// Placement: row tiles per PPT node.  Enough tiles that a tile's weights + accumulators + staging fit in
-// shared memory, then the remaining CTAs in proportion to the nodes' multiply-add volume.
-ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles, int emitters, int tiles_cap) {
+// Placement: row tiles per PPT node.  Every node starts with the fewest tiles whose weights + accumulators + staging
+// fit in shared memory; the remaining tile budget goes, one tile at a time, to the node with the most multiply-add work
+// per tile (a GRU cell counts twice: three matrices and a second, dependent stage), so that the nodes' batch cycles
+// come out alike.  A tile costs 1 + emitters CTAs; the controller and one scheduler CTA per node come off the top.
+ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vector<Role>& roles, int emitters) {
   cudaFuncAttributes fa{};
   size_t static_smem = 40 * 1024;
   if (cudaFuncGetAttributes(&fa, ampnet_engine) == cudaSuccess) static_smem = fa.sharedSizeBytes;
   const size_t budget = ((size_t)g->max_smem - static_smem - 1024) / sizeof(float);
   int max_tiles = 16;      // default; a node whose tile does not fit in shared memory gets more, up to MAX_TILES
   if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, std::min(MAX_TILES, atoi(e)));
-  if (tiles_cap > 0) max_tiles = std::min(max_tiles, tiles_cap);
-  double total_w = 0;
-  for (auto& P : g->ppts) if (P.kind != LOOKUP) total_w += (double)P.nmat * P.in * P.out;
-  const int avail = std::max(1, n_ctas - 1 - (int)g->ppts.size());
-  int used = 1;
-  for (auto& P : g->ppts) {
+  const int np = (int)g->ppts.size();
+  const int tile_budget = emitters > 0 ? (n_ctas - 1 - np) / (1 + emitters) : n_ctas - 1;
+  std::vector<int> limit(np, 1), bm_of(np, 0);
+  std::vector<double> work(np, 0.0);
+  auto fit = [&](HostPPT& P, int t_from, int bm, int& t_out) {      // fewest tiles >= t_from that fit with capacity bm
+    for (int t = t_from; t <= std::min(MAX_TILES, P.out); t++) {
+      const int R = (P.out + t - 1) / t;
+      if ((P.out + R - 1) / R < t_from) continue;
+      if (tile_smem_floats(P, R, bm) <= budget) { t_out = (P.out + R - 1) / R; return true; }
+    }
+    return false;
+  };
+  int used_tiles = 0;
+  for (int p = 0; p < np; p++) {
+    HostPPT& P = g->ppts[p];
     const DevNode& h = g->hnodes[P.node];
     const int rows_max = h.rows_in;
     int BM = MAX_BATCH_ROWS;
     if (max_batch_rows > 0) BM = std::max(rows_max, std::min(BM, max_batch_rows));
-    if (rows_max > 64) return set_err(g, AMPNET_EINVAL, "node %d: %d payload rows per message exceed the supported 64", P.node, rows_max);
+    if (rows_max > MAX_BATCH_ROWS) return set_err(g, AMPNET_EINVAL, "node %d: %d payload rows per message exceed the supported %d", P.node, rows_max, MAX_BATCH_ROWS);
     P.J = P.kind == LOOKUP ? 4 : j_bucket(P.in);
     if (P.kind == LOOKUP) {
       // a large table means gathers and accumulations bound by DRAM latency: deal its rows to several tiles
-      P.T = (P.in >= 4096 && (tiles_cap == 0 || tiles_cap >= 8)) ? 4 : 1;
-      P.R = 0; P.BM = BM; P.smem_floats = tile_smem_floats(P, 0, BM); used += P.T; continue;
+      P.T = (P.in >= 4096 && tile_budget >= 24) ? 4 : 1;
+      P.R = 0; P.BM = BM; limit[p] = P.T; bm_of[p] = BM;
+      used_tiles += P.T;
+      continue;
     }
-    // small nodes (a classifier) still emit one message per gradient: give them tiles for the emission work
-    const double share = std::max((double)P.nmat * P.in * P.out / total_w, 0.1);
-    int T = 1 + (int)std::floor(share * avail);
-    T = std::max(1, std::min({T, max_tiles, P.out <= 16 ? P.out : std::max(1, P.out / 4)}));
     // Keep the micro-batch capacity if more row tiles make the tile fit; only then shrink the capacity.
-    bool placed = false;
     const int bm_min = std::max(rows_max, 4);
+    bool placed = false;
     for (int bm = BM; !placed; bm = std::max(bm_min, bm / 2)) {
-      for (int t = T; t <= std::min(MAX_TILES, P.out); t++) {
-        const int R = (P.out + t - 1) / t;
-        if (tile_smem_floats(P, R, bm) <= budget) { P.R = R; P.BM = bm; P.T = (P.out + R - 1) / R; placed = true; break; }
-      }
-      if (!placed && bm == bm_min)
-        return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory with %d row tiles", P.node, MAX_TILES);
+      int t = 0;
+      if (fit(P, 1, bm, t)) { P.T = t; bm_of[p] = bm; placed = true; break; }
+      if (bm == bm_min) return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory with %d row tiles", P.node, MAX_TILES);
     }
+    // a node with a handful of output rows (a classifier) may still have a tile per row; others keep 4 rows per tile
+    limit[p] = std::max(P.T, std::min(max_tiles, P.out <= 16 ? P.out : std::max(1, P.out / 4)));
+    work[p] = (double)P.nmat * P.in * P.out * (P.kind == GRUCELL ? 2.0 : 1.0);
+    used_tiles += P.T;
+  }
+  if (1 + used_tiles * (1 + emitters) + (emitters > 0 ? np : 0) > n_ctas) return AMPNET_EOVERFLOW;   // retried with fewer emitters
+  for (;;) {
+    int best = -1;
+    for (int p = 0; p < np; p++) {
+      const HostPPT& P = g->ppts[p];
+      if (P.kind == LOOKUP || P.T >= limit[p]) continue;
+      if (best < 0 || work[p] / P.T > work[best] / g->ppts[best].T) best = p;
+    }
+    if (best < 0) break;
+    HostPPT& P = g->ppts[best];
+    int t = 0;
+    if (!fit(P, P.T + 1, bm_of[best], t) || t > limit[best] || t <= P.T) { limit[best] = P.T; continue; }   // rows per tile are whole: the tile count moves in steps
+    if (used_tiles + (t - P.T) > tile_budget) { limit[best] = P.T; continue; }
+    used_tiles += t - P.T; P.T = t;
+  }
+  int used = 1;
+  for (int p = 0; p < np; p++) {
+    HostPPT& P = g->ppts[p];
+    if (P.kind != LOOKUP) { P.R = (P.out + P.T - 1) / P.T; P.T = (P.out + P.R - 1) / P.R; P.BM = bm_of[p]; }
     P.smem_floats = tile_smem_floats(P, P.R, P.BM);
     used += P.T;
   }
@@ -448,15 +478,11 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   const int mbr = cfg ? cfg->max_batch_rows : 0;
   // Two emitter CTAs per tile if the SMs allow it, with as many tiles per node as fit; then one; then none.
   ampnet_status_t st = AMPNET_EOVERFLOW;
-  const int caps[] = {0, 12, 10, 8, 7, 6, 5, 4};
   for (; emit_ctas > 0 && st == AMPNET_EOVERFLOW; emit_ctas--) {
-    for (int cap : caps) {
-      st = place(g, n_ctas, mbr, R.roles, emit_ctas, cap);
-      if (st != AMPNET_EOVERFLOW) break;
-    }
+    st = place(g, n_ctas, mbr, R.roles, emit_ctas);
     if (st != AMPNET_EOVERFLOW) break;
   }
-  if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0, 0); }
+  if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0); }
   if (st != AMPNET_OK) return st;
   const int depth = emit_ctas > 0 ? 3 : 2;       // emitters work in two batch groups: a tile may be two batches ahead
   R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth; R.ctx.sched_ctas = emit_ctas > 0 ? 1 : 0;

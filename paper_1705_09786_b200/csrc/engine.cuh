@@ -740,6 +740,50 @@ __device__ __noinline__ void tile_dW(const float* __restrict__ Ds, int ldd, int 
   }
 }
 
+// dst[b][i] = (i < nbase ? base[b][i] : 0) + sum_r D1[b][r] * W1[r][i] + sum_r D2[b][r] * W2[r][i]: the second backward
+// stage of the GRU cell in one pass with one store per element (dst and base in device memory, ld = in_dim).
+template <int J>
+__device__ __noinline__ void tile_dW2(const float* __restrict__ D1, const float* __restrict__ D2, int ldd, int nb,
+                                      const float* __restrict__ W1, const float* __restrict__ W2, int ldw, int R, int in_dim,
+                                      const float* __restrict__ base, int nbase, float* __restrict__ dst) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int b0 = warp * 4; b0 < nb; b0 += WARPS * 4) {
+    float acc[4][J];
+#pragma unroll
+    for (int m = 0; m < 4; m++)
+#pragma unroll
+      for (int j = 0; j < J; j++) {
+        const int i = lane + 32 * j;
+        acc[m][j] = (b0 + m < nb && i < nbase) ? __ldcg(base + (size_t)(b0 + m) * in_dim + i) : 0.f;
+      }
+#pragma unroll
+    for (int pass = 0; pass < 2; pass++) {
+      const float* __restrict__ Ds = pass ? D2 : D1;
+      const float* __restrict__ Ws = pass ? W2 : W1;
+      for (int r = 0; r < R; r++) {
+        float d[4];
+#pragma unroll
+        for (int m = 0; m < 4; m++) d[m] = (b0 + m < nb) ? Ds[(b0 + m) * ldd + r] : 0.f;
+#pragma unroll
+        for (int j = 0; j < J; j++) {
+          const int i = lane + 32 * j;
+          const float w = i < in_dim ? Ws[r * ldw + i] : 0.f;
+#pragma unroll
+          for (int m = 0; m < 4; m++) acc[m][j] = fmaf(d[m], w, acc[m][j]);
+        }
+      }
+    }
+#pragma unroll
+    for (int m = 0; m < 4; m++)
+      if (b0 + m < nb)
+#pragma unroll
+        for (int j = 0; j < J; j++) {
+          const int i = lane + 32 * j;
+          if (i < in_dim) dst[(size_t)(b0 + m) * in_dim + i] = acc[m][j];
+        }
+  }
+}
+
 // A[r][i] += sum_b D[b][r] * X[b][i];  work unit = 4 weight rows x 4 column chunks.
 __device__ __noinline__ void tile_accum(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Xs, int ldx,
                            float* __restrict__ As, int lda, int R, int in_dim) {
@@ -1615,20 +1659,20 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R;
             float dq = 0.f;
-            for (int t = 0; t < P.T; t++) dq += __ldcg(part1_all + (size_t)t * pstride + (size_t)b * in + H + r_begin + r);
+            for (int tb = 0; tb < P.T; tb += 8) {        // eight tiles' partials in flight, added in tile order
+              float v[8];
+#pragma unroll
+              for (int t = 0; t < 8; t++) v[t] = tb + t < P.T ? __ldcg(part1_all + (size_t)(tb + t) * pstride + (size_t)b * in + H + r_begin + r) : 0.f;
+#pragma unroll
+              for (int t = 0; t < 8; t++) dq += v[t];
+            }
             const float rg = M.Ys[b * SR + r], h = M.Xs[b * in + H + r_begin + r];
             dpr[b * SR + r] = dq * h * rg * (1.f - rg);
             dirbuf[(size_t)b * H + r_begin + r] = dirp[b * SR + r] + dq * rg;
           }
           __syncthreads();
           // this tile's share of da_c joins its second partial here, so that emission sums one partial array per tile
-          for (int idx = tid; idx < nb * in; idx += THREADS) {
-            const int c = idx % in;
-            part2[idx] = c < H ? __ldcg(part1 + idx) : 0.f;
-          }
-          __syncthreads();
-          AMP_DISPATCH_J(P.J, (tile_dW<J, true>(dpz, SR, nb, Wz, in, R, in, part2)));
-          AMP_DISPATCH_J(P.J, (tile_dW<J, true>(dpr, SR, nb, Wr, in, R, in, part2)));
+          AMP_DISPATCH_J(P.J, (tile_dW2<J>(dpz, dpr, SR, nb, Wz, Wr, in, R, in, part1, H, part2)));
           tile_accum(dpz, SR, nb, M.Xs, in, M.As, in, R, in);
           tile_accum(dpr, SR, nb, M.Xs, in, M.As + SR * in, in, R, in);
           tile_accum(dpc, SR, nb, M.XC, in, M.As + 2 * SR * in, in, R, in);
