@@ -351,10 +351,12 @@ unsigned pow2_at_least(unsigned long long v) {
   return p;
 }
 
-size_t tile_smem_floats(const HostPPT& P, int R, int BM) {
+size_t tile_smem_floats(const HostPPT& P, int R, int BM) {      // mirrors the carve-up at the top of ppt_main
   if (P.kind == LOOKUP) return 64;
-  return (size_t)P.nmat * (2 * (size_t)R * P.in + 2 * R) + (size_t)BM * P.in * (P.kind == GRUCELL ? 2 : 1) +
-         (size_t)(2 * P.nmat + 1) * BM * R + 64;
+  const size_t LW = (size_t)pad_ldw(P.in), LX = (size_t)pad_ldx(P.in), RP = (size_t)((R + 3) & ~3), nm = (size_t)P.nmat;
+  auto p4 = [](size_t v) { return (v + 3) & ~(size_t)3; };
+  return 2 * nm * R * LW + 2 * p4(nm * R) + (size_t)BM * LX * (P.kind == GRUCELL ? 2 : 1) + (nm + 1) * BM * RP + p4(nm * BM * R) +
+         XWT_SCRATCH + 64;
 }
 
 // Placement: row tiles per PPT node.  Every node starts with the fewest tiles whose weights + accumulators + staging
@@ -741,6 +743,11 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
       const unsigned long long* r = G.role_cycles + 8 + 8 * p;
       fprintf(stderr, "[role] node %2d sched us: wait-tile %.0f no-msg %.0f form %.0f | emitter(0,0) us: wait %.0f load %.0f emit %.0f batches %llu\n",
               g->ppts[p].node, r[0] * us, r[1] * us, r[2] * us, r[3] * us, r[4] * us, r[5] * us, r[6]);
+    }
+    for (size_t p = 0; p < g->ppts.size(); p++) {
+      fprintf(stderr, "[step] node %2d us:", g->ppts[p].node);
+      for (int k = 0; k < 12; k++) fprintf(stderr, " %.0f", G.step_cycles[p][k] * us);
+      fprintf(stderr, "\n");
     }
     for (int t = 0; t < N_NODE_TYPES * 2; t++)
       if (G.walk_steps[t]) fprintf(stderr, "[walk] %-8s %s steps %10llu cycles/step %8.0f\n", names[t / 2], t & 1 ? "BWD" : "FWD", G.walk_steps[t], (double)G.walk_cycles[t] / G.walk_steps[t]);

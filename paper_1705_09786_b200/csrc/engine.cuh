@@ -657,49 +657,57 @@ __device__ __forceinline__ float act_grad(int a, float y) {
   }
 }
 
-// out[b][r] = sum_i X[b][i] * W[r][i]  for b < nb, r < R.  4 batch rows x 4 weight rows per warp pass; the 16
-// lane-partial sums are reduced across the warp with a halving butterfly (16 shuffles instead of 80).
-template <int J>
-__device__ __noinline__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const float* __restrict__ Ws, int ldw, int R,
-                         int in_dim, float* __restrict__ out, int ldo) {
+// Shared-memory layout of a tile's operands: weight / accumulator rows have a leading dimension of a multiple of 4 floats
+// (ldw), staged input rows one that is 4 (mod 8) floats (ldx, so that a warp whose lanes read 16 bytes each from 32
+// different rows meets no bank conflict), gradient rows D a multiple of 4 (ldd); all padding is kept at zero.
+__host__ __device__ __forceinline__ int pad_ldw(int in) { return (in + 3) & ~3; }
+__host__ __device__ __forceinline__ int pad_ldx(int in) { int l = (in + 3) & ~3; while ((l & 7) != 4) l += 4; return l; }
+constexpr int XWT_SCRATCH = WARPS * 32 * 8;      // floats: partial sums of the k-slices
+
+// out[b][r] = sum_k X[b][k] * W[r][k]  for b < nb, r < R (whole CTA; ends with a block barrier).  Lanes own batch rows:
+// warp (g, s) takes the 32 batch rows of group g and the k-slice s, keeps RB outputs per lane in registers, reads its row
+// 16 bytes at a time and the weight rows as broadcasts; the slices' partial sums meet in `scratch` and are added in
+// slice order.
+template <int RB>
+__device__ __forceinline__ void xwT_pass(const float* __restrict__ Xs, int ldx, int nb, const float* __restrict__ Ws, int ldw, int r0, int R,
+                                         int K4, float* __restrict__ scratch, int G, int S) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int nbg = (nb + 3) >> 2, nrg = (R + 3) >> 2;
-  for (int unit = warp; unit < nbg * nrg; unit += WARPS) {
-    const int b0 = (unit / nrg) * 4, r0 = (unit % nrg) * 4;
-    float acc[16];
+  const int g = warp % G, s = warp / G;
+  const int b = g * 32 + lane;
+  const int k4_per = (K4 + S - 1) / S, k4a = s * k4_per, k4b = min(K4, k4a + k4_per);
+  float acc[RB];
 #pragma unroll
-    for (int k = 0; k < 16; k++) acc[k] = 0.f;
+  for (int q = 0; q < RB; q++) acc[q] = 0.f;
+  const float4* xrow = reinterpret_cast<const float4*>(Xs + (size_t)min(b, nb - 1) * ldx);
+#pragma unroll 2
+  for (int k4 = k4a; k4 < k4b; k4++) {
+    const float4 x = xrow[k4];
 #pragma unroll
-    for (int j = 0; j < J; j++) {
-      const int i = lane + 32 * j;
-      if (i < in_dim) {
-        float x[4], w[4];
-#pragma unroll
-        for (int m = 0; m < 4; m++) x[m] = (b0 + m < nb) ? Xs[(b0 + m) * ldx + i] : 0.f;
-#pragma unroll
-        for (int q = 0; q < 4; q++) w[q] = (r0 + q < R) ? Ws[(r0 + q) * ldw + i] : 0.f;
-#pragma unroll
-        for (int m = 0; m < 4; m++)
-#pragma unroll
-          for (int q = 0; q < 4; q++) acc[m * 4 + q] = fmaf(x[m], w[q], acc[m * 4 + q]);
-      }
+    for (int q = 0; q < RB; q++) {
+      const float4 w = *reinterpret_cast<const float4*>(Ws + (size_t)min(r0 + q, R - 1) * ldw + 4 * k4);
+      acc[q] = fmaf(x.x, w.x, acc[q]); acc[q] = fmaf(x.y, w.y, acc[q]); acc[q] = fmaf(x.z, w.z, acc[q]); acc[q] = fmaf(x.w, w.w, acc[q]);
     }
-    // halving butterfly: after the step with offset o, a lane keeps the half of its values selected by bit o
+  }
+  if (b < nb) {
 #pragma unroll
-    for (int h = 8, o = 16; h >= 1; h >>= 1, o >>= 1) {
-      const bool up = (lane & o) != 0;
-#pragma unroll
-      for (int k = 0; k < h; k++) {
-        float send = up ? acc[k] : acc[k + h];
-        float keep = up ? acc[k + h] : acc[k];
-        acc[k] = keep + __shfl_xor_sync(0xffffffffu, send, o);
-      }
+    for (int q = 0; q < RB; q++) scratch[((size_t)s * 32 * G + b) * RB + q] = acc[q];
+  }
+}
+__device__ __noinline__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const float* __restrict__ Ws, int ldw, int R,
+                                      int in_dim, float* __restrict__ out, int ldo, float* __restrict__ scratch) {
+  const int G = nb > 32 ? 2 : 1, S = WARPS / G, K4 = (in_dim + 3) >> 2;
+  for (int r0 = 0; r0 < R; r0 += 8) {
+    const int rb = min(8, R - r0), RBs = rb > 4 ? 8 : 4;
+    if (rb > 4) xwT_pass<8>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
+    else xwT_pass<4>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < nb * rb; idx += THREADS) {
+      const int b = idx / rb, q = idx - b * rb;
+      float v = 0.f;
+      for (int s = 0; s < S; s++) v += scratch[((size_t)s * 32 * G + b) * RBs + q];
+      out[b * ldo + r0 + q] = v;
     }
-    float v = acc[0] + __shfl_xor_sync(0xffffffffu, acc[0], 1);
-    // lane bits (16,8,4,2) selected value index k = 8*b16 + 4*b8 + 2*b4 + b2
-    const int k = ((lane >> 4) & 1) * 8 + ((lane >> 3) & 1) * 4 + ((lane >> 2) & 1) * 2 + ((lane >> 1) & 1);
-    const int m = k >> 2, q = k & 3;
-    if ((lane & 1) == 0 && b0 + m < nb && r0 + q < R) out[(b0 + m) * ldo + r0 + q] = v;
+    __syncthreads();
   }
 }
 
@@ -784,39 +792,30 @@ __device__ __noinline__ void tile_dW2(const float* __restrict__ D1, const float*
   }
 }
 
-// A[r][i] += sum_b D[b][r] * X[b][i];  work unit = 4 weight rows x 4 column chunks.
+// A[r][k] += sum_b D[b][r] * X[b][k];  a warp's unit is 4 accumulator rows x 64 columns (a lane owns two), the four
+// gradient entries of a batch row come as one 16-byte broadcast (D rows are padded to a multiple of 4 with zeros).
 __device__ __noinline__ void tile_accum(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Xs, int ldx,
-                           float* __restrict__ As, int lda, int R, int in_dim) {
+                                        float* __restrict__ As, int lda, int R, int in_dim) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int nj = (in_dim + 31) >> 5, ncg = (nj + 3) >> 2, nrg = (R + 3) >> 2;
+  const int K = (in_dim + 1) & ~1;
+  const int nrg = (R + 3) >> 2, ncg = (K + 63) >> 6;
   for (int unit = warp; unit < nrg * ncg; unit += WARPS) {
-    const int r0 = (unit / ncg) * 4, j0 = (unit % ncg) * 4;
-    float a[4][4];
+    const int r0 = (unit / ncg) * 4, k = (unit % ncg) * 64 + 2 * lane;
+    if (k >= K) continue;
+    float2 a[4];
 #pragma unroll
-    for (int q = 0; q < 4; q++)
-#pragma unroll
-      for (int j = 0; j < 4; j++) {
-        const int i = lane + 32 * (j0 + j);
-        a[q][j] = (r0 + q < R && i < in_dim) ? As[(r0 + q) * lda + i] : 0.f;
-      }
+    for (int q = 0; q < 4; q++) a[q] = r0 + q < R ? *reinterpret_cast<const float2*>(As + (size_t)(r0 + q) * lda + k) : make_float2(0.f, 0.f);
+#pragma unroll 4
     for (int b = 0; b < nb; b++) {
-      float d[4], x[4];
-#pragma unroll
-      for (int q = 0; q < 4; q++) d[q] = (r0 + q < R) ? Ds[b * ldd + r0 + q] : 0.f;
-#pragma unroll
-      for (int j = 0; j < 4; j++) { const int i = lane + 32 * (j0 + j); x[j] = i < in_dim ? Xs[b * ldx + i] : 0.f; }
-#pragma unroll
-      for (int q = 0; q < 4; q++)
-#pragma unroll
-        for (int j = 0; j < 4; j++) a[q][j] = fmaf(d[q], x[j], a[q][j]);
+      const float4 d = *reinterpret_cast<const float4*>(Ds + (size_t)b * ldd + r0);
+      const float2 x = *reinterpret_cast<const float2*>(Xs + (size_t)b * ldx + k);
+      a[0].x = fmaf(d.x, x.x, a[0].x); a[0].y = fmaf(d.x, x.y, a[0].y);
+      a[1].x = fmaf(d.y, x.x, a[1].x); a[1].y = fmaf(d.y, x.y, a[1].y);
+      a[2].x = fmaf(d.z, x.x, a[2].x); a[2].y = fmaf(d.z, x.y, a[2].y);
+      a[3].x = fmaf(d.w, x.x, a[3].x); a[3].y = fmaf(d.w, x.y, a[3].y);
     }
 #pragma unroll
-    for (int q = 0; q < 4; q++)
-#pragma unroll
-      for (int j = 0; j < 4; j++) {
-        const int i = lane + 32 * (j0 + j);
-        if (r0 + q < R && i < in_dim) As[(r0 + q) * lda + i] = a[q][j];
-      }
+    for (int q = 0; q < 4; q++) if (r0 + q < R) *reinterpret_cast<float2*>(As + (size_t)(r0 + q) * lda + k) = a[q];
   }
 }
 
@@ -846,9 +845,12 @@ struct TileShared : BatchCtx {
   unsigned long long stale_hist[64];
   int max_stale;
   unsigned long long phase[16];
+  unsigned long long step[16];
+  long long step_t;
   Frame stack[WARPS][WALK_STACK];
   WalkPool pool;
 };
+#define AMP_STEP(k) do { if (threadIdx.x == 0) { const long long n_ = clock64(); S.step[k] += (unsigned long long)(n_ - S.step_t); S.step_t = n_; } } while (0)
 
 __device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) {
   return P.muf_override > 0 ? P.muf_override : C.muf;
@@ -1068,7 +1070,7 @@ __device__ __noinline__ void leader_schedule_round(const Ctx& C, DevPPT& P, Tile
 // Copy the cached input rows of a batch into shared memory with several loads in flight per thread.
 // rowptr[b] points at row b's `width` floats in device memory; V = 4, 2 or 1 floats per load.
 template <int V>
-__device__ __forceinline__ void stage_rows_v(float* __restrict__ Xs, const float* const* rowptr, int nb, int width) {
+__device__ __forceinline__ void stage_rows_v(float* __restrict__ Xs, int ldx, const float* const* rowptr, int nb, int width) {
   const int wv = width / V, total = nb * wv;
   for (int base = threadIdx.x; base < total; base += THREADS * 4) {
     float v[4][V];
@@ -1089,19 +1091,20 @@ __device__ __forceinline__ void stage_rows_v(float* __restrict__ Xs, const float
       if (idx < total) {
         const int b = idx / wv, c = idx - b * wv;
 #pragma unroll
-        for (int q = 0; q < V; q++) Xs[b * width + c * V + q] = v[k][q];
+        for (int q = 0; q < V; q++) Xs[b * ldx + c * V + q] = v[k][q];
       }
     }
   }
 }
-__device__ __noinline__ void stage_rows(float* Xs, const float* const* rowptr, int nb, int width, int align_floats) {
-  if ((width & 3) == 0 && (align_floats & 3) == 0) stage_rows_v<4>(Xs, rowptr, nb, width);
-  else if ((width & 1) == 0 && (align_floats & 1) == 0) stage_rows_v<2>(Xs, rowptr, nb, width);
-  else stage_rows_v<1>(Xs, rowptr, nb, width);
+__device__ __noinline__ void stage_rows(float* Xs, int ldx, const float* const* rowptr, int nb, int width, int align_floats) {
+  if ((width & 3) == 0 && (align_floats & 3) == 0) stage_rows_v<4>(Xs, ldx, rowptr, nb, width);
+  else if ((width & 1) == 0 && (align_floats & 1) == 0) stage_rows_v<2>(Xs, ldx, rowptr, nb, width);
+  else stage_rows_v<1>(Xs, ldx, rowptr, nb, width);
 }
 
 struct TileMem {           // carve-up of the dynamic shared memory of a tile (floats)
-  float *Ws, *As, *bs, *Abs, *Xs, *Ds, *Ys, *XC;
+  float *Ws, *As, *bs, *Abs, *Xs, *Ds, *Ys, *XC, *scratch;
+  int LW, LX, RP;          // leading dimensions: weight / accumulator rows, staged input rows, gradient rows
 };
 
 __device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, const Hdr& h, long long key) {
@@ -1396,6 +1399,36 @@ __device__ __noinline__ void lookup_batch(DevPPT& P, TileShared& S, const int di
   }
 }
 
+// GRU cell: XC = [a; r * h] from X = [a; h] (shared memory) and the reset gates of all tiles (device memory), a batch
+// row per warp pass with eight gate loads per lane in flight (whole CTA, no barrier).
+__device__ __noinline__ void gru_gated_input(const DevPPT& P, const TileShared& S, const float* __restrict__ Xs, float* __restrict__ XC,
+                                             const int ldx, const int nb) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, in = P.in_dim, H = P.out_dim;
+  for (int idx = threadIdx.x; idx < nb * (in - H); idx += THREADS) {
+    const int b = idx / (in - H), c = idx - b * (in - H);
+    XC[b * ldx + c] = Xs[b * ldx + c];
+  }
+  for (int b0 = warp; b0 < nb; b0 += WARPS * 4)               // four batch rows per warp pass
+    for (int c0 = 0; c0 < H; c0 += 32 * 4) {
+      float rg[4][4];
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const int b = b0 + j * WARPS;
+        const float* rrow = nullptr;
+        if (b < nb) { const int m = S.rowmsg[b]; rrow = P.rc + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H; }
+#pragma unroll
+        for (int k = 0; k < 4; k++) { const int c = c0 + k * 32 + lane; rg[j][k] = (rrow && c < H) ? __ldcg(rrow + c) : 0.f; }
+      }
+#pragma unroll
+      for (int j = 0; j < 4; j++) {
+        const int b = b0 + j * WARPS;
+        if (b >= nb) continue;
+#pragma unroll
+        for (int k = 0; k < 4; k++) { const int c = c0 + k * 32 + lane; if (c < H) XC[b * ldx + (in - H) + c] = Xs[b * ldx + (in - H) + c] * rg[j][k]; }
+      }
+    }
+}
+
 // Local update of a tile's share of the node's parameters (whole CTA; ends with a block barrier).
 __device__ __noinline__ void tile_update(const Ctx& C, DevPPT& P, const TileMem& M, const BatchDesc& d, const int R,
                                          const int r_begin, const int tile) {
@@ -1427,7 +1460,7 @@ __device__ __noinline__ void tile_update(const Ctx& C, DevPPT& P, const TileMem&
     const size_t nW = (size_t)nmat * out * in;
     for (int m = 0; m < nmat; m++) {
       for (int i = tid; i < R * in; i += THREADS) {
-        const int o = m * P.R * in + i;
+        const int r = i / in, o = (m * P.R + r) * M.LW + (i - r * in);
         os.apply(M.Ws[o], M.As[o], (size_t)m * out * in + (size_t)r_begin * in + i);
       }
       for (int i = tid; i < R; i += THREADS) {
@@ -1448,23 +1481,28 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
   const int nmat = P.kind == GRUCELL ? 3 : 1;
   TileMem M;
   {
-    float* p = smem;
-    M.Ws = p; p += (size_t)nmat * P.R * in;
-    M.As = p; p += (size_t)nmat * P.R * in;
-    M.bs = p; p += nmat * P.R;
-    M.Abs = p; p += nmat * P.R;
-    M.Xs = p; p += (size_t)P.BM * in;
-    M.Ds = p; p += (size_t)(nmat + 1) * P.BM * P.R;
-    M.Ys = p; p += (size_t)nmat * P.BM * P.R;
-    M.XC = p;   // GRUCELL only: [BM][in]
+    M.LW = pad_ldw(in); M.LX = pad_ldx(in); M.RP = (P.R + 3) & ~3;
+    float* p = smem;                                 // every array starts on a 16-byte boundary
+    M.Ws = p; p += (size_t)nmat * P.R * M.LW;
+    M.As = p; p += (size_t)nmat * P.R * M.LW;
+    M.bs = p; p += (nmat * P.R + 3) & ~3;
+    M.Abs = p; p += (nmat * P.R + 3) & ~3;
+    M.Xs = p; p += (size_t)P.BM * M.LX;
+    M.Ds = p; p += (size_t)(nmat + 1) * P.BM * M.RP;
+    M.Ys = p; p += ((size_t)nmat * P.BM * P.R + 3) & ~(size_t)3;
+    M.scratch = p; p += XWT_SCRATCH;
+    M.XC = p; p += P.kind == GRUCELL ? (size_t)P.BM * M.LX : 0;
+    if (P.kind != LOOKUP) for (float* q = smem + tid; q < p; q += THREADS) *q = 0.f;     // the padding stays zero
   }
+  __syncthreads();
+  const int LW = M.LW, LX = M.LX, RP = M.RP;
   if (P.kind != LOOKUP) {
     for (int m = 0; m < nmat; m++) {
       for (int i = tid; i < R * in; i += THREADS) {
-        M.Ws[m * P.R * in + i] = P.W[(size_t)m * out * in + (size_t)r_begin * in + i];
-        M.As[m * P.R * in + i] = 0.f;
+        const int r = i / in, c = i - r * in;
+        M.Ws[(m * P.R + r) * LW + c] = P.W[(size_t)m * out * in + (size_t)r_begin * in + i];
       }
-      for (int i = tid; i < R; i += THREADS) { M.bs[m * P.R + i] = P.b[m * out + r_begin + i]; M.Abs[m * P.R + i] = 0.f; }
+      for (int i = tid; i < R; i += THREADS) M.bs[m * P.R + i] = P.b[m * out + r_begin + i];
     }
   }
   if (tid == 0) {
@@ -1472,7 +1510,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
     S.ls.log_n = 0; S.ls.n_updates = S.ls.n_grads_applied = S.ls.msgs = S.ls.batches = S.ls.batch_rows = 0;
   }
   if (tid < 64) S.stale_hist[tid] = 0;
-  if (tid < 16) S.phase[tid] = 0;
+  if (tid < 16) { S.phase[tid] = 0; S.step[tid] = 0; }
   if (tid < POOL) S.pool.ready[tid] = 0;
   if (tid == 0) { S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
   __syncthreads();
@@ -1560,10 +1598,10 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
 
       if (count > 0 && P.kind == LINEAR) {
         // stage the cached inputs of the batch
-        stage_rows(M.Xs, S.rowptr, nb, in, P.xcache ? in : C.inst.dense_dim);
+        stage_rows(M.Xs, LX, S.rowptr, nb, in, P.xcache ? in : C.inst.dense_dim);
         if (dir == FWD) {
           __syncthreads();
-          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.Xs, in, nb, M.Ws, in, R, in, M.Ys, P.R)));
+          tile_xwT(M.Xs, LX, nb, M.Ws, LW, R, in, M.Ys, P.R, M.scratch);
           __syncthreads();
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
@@ -1574,30 +1612,32 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
             const size_t o = (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * out + r_begin + r;
-            M.Ds[b * P.R + r] = __ldcg(P.gbuf + o) * act_grad(P.act, __ldcg(P.ycache + o));
+            M.Ds[b * RP + r] = __ldcg(P.gbuf + o) * act_grad(P.act, __ldcg(P.ycache + o));
           }
           __syncthreads();
           if (!(P.flags & 1)) {
             float* dst = P.T > 1 ? P.dxpart + ((size_t)(my_batch % (unsigned)C.depth) * P.T + tile) * P.BM * in : stage_k;
-            AMP_DISPATCH_J(P.J, (tile_dW<J>(M.Ds, P.R, nb, M.Ws, in, R, in, dst)));
+            AMP_DISPATCH_J(P.J, (tile_dW<J>(M.Ds, RP, nb, M.Ws, LW, R, in, dst)));
           }
-          tile_accum(M.Ds, P.R, nb, M.Xs, in, M.As, in, R, in);
+          tile_accum(M.Ds, RP, nb, M.Xs, LX, M.As, LW, R, in);
           for (int r = tid; r < R; r += THREADS) {
             float s = M.Abs[r];
-            for (int b = 0; b < nb; b++) s += M.Ds[b * P.R + r];
+            for (int b = 0; b < nb; b++) s += M.Ds[b * RP + r];
             M.Abs[r] = s;
           }
         }
       } else if (count > 0 && P.kind == GRUCELL) {
         // x = [a; h]; the tile owns rows [r_begin, r_begin + R) of Wz, Wr, Wc (matrix m at Ws + m * P.R * in)
-        const int H = out, SR = P.R, BR = P.BM * P.R;
-        const float *Wz = M.Ws, *Wr = M.Ws + SR * in, *Wc = M.Ws + 2 * SR * in;
-        stage_rows(M.Xs, S.rowptr, nb, in, in);
+        const int H = out, SR = P.R, BR = P.BM * P.R, BRD = P.BM * RP;      // Ys arrays: [BM][SR]; D arrays: [BM][RP]
+        const float *Wz = M.Ws, *Wr = M.Ws + SR * LW, *Wc = M.Ws + 2 * SR * LW;
+        if (tid == 0) S.step_t = clock64();
+        stage_rows(M.Xs, LX, S.rowptr, nb, in, in);
         __syncthreads();
+        AMP_STEP(0);
         if (dir == FWD) {
           // phase 1: gates z, r for the tile's rows
-          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.Xs, in, nb, Wz, in, R, in, M.Ys, SR)));
-          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.Xs, in, nb, Wr, in, R, in, M.Ys + BR, SR)));
+          tile_xwT(M.Xs, LX, nb, Wz, LW, R, in, M.Ys, SR, M.scratch);
+          tile_xwT(M.Xs, LX, nb, Wr, LW, R, in, M.Ys + BR, SR, M.scratch);
           __syncthreads();
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
@@ -1607,55 +1647,53 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
             M.Ys[b * SR + r] = z;
             P.zc[o] = z; P.rc[o] = rg;
           }
+          AMP_STEP(1);
           __threadfence();
           if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
           else __syncthreads();
+          AMP_STEP(2);
           // phase 2: candidate c = tanh(Wc [a; r*h] + bc) and the new state
-          for (int idx = tid; idx < nb * in; idx += THREADS) {
-            const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
-            float v = M.Xs[idx];
-            if (c >= H) v *= __ldcg(P.rc + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + (c - H));
-            M.XC[idx] = v;
-          }
+          gru_gated_input(P, S, M.Xs, M.XC, LX, nb);
           __syncthreads();
-          AMP_DISPATCH_J(P.J, (tile_xwT<J>(M.XC, in, nb, Wc, in, R, in, M.Ys + 2 * BR, SR)));
+          AMP_STEP(3);
+          tile_xwT(M.XC, LX, nb, Wc, LW, R, in, M.Ys + 2 * BR, SR, M.scratch);
           __syncthreads();
+          AMP_STEP(4);
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
             const size_t o = (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + r_begin + r;
             const float cnd = tanhf(M.Ys[2 * BR + b * SR + r] + M.bs[2 * SR + r]);
             const float z = M.Ys[b * SR + r];
             P.cc[o] = cnd;
-            P.ycache[o] = emit_round((1.f - z) * M.Xs[b * in + H + r_begin + r] + z * cnd);
+            P.ycache[o] = emit_round((1.f - z) * M.Xs[b * LX + H + r_begin + r] + z * cnd);
           }
+          AMP_STEP(5);
         } else {
           const size_t pstride = (size_t)P.BM * in;
           float* part1 = P.part2 + ((size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) + tile) * pstride;
           const float* part1_all = P.part2 + (size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) * pstride;
           float* dirbuf = P.part2 + ((size_t)(my_batch % (unsigned)C.depth) * (P.T + 1) + P.T) * pstride;     // [BM][H]
           float* part2 = P.dxpart + ((size_t)(my_batch % (unsigned)C.depth) * P.T + tile) * pstride;
-          float *dpz = M.Ds, *dpr = M.Ds + BR, *dpc = M.Ds + 2 * BR, *dirp = M.Ds + 3 * BR;
+          float *dpz = M.Ds, *dpr = M.Ds + BRD, *dpc = M.Ds + 2 * BRD, *dirp = M.Ds + 3 * BRD;
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
             const size_t o = (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + r_begin + r;
             const float g = __ldcg(P.gbuf + o), z = __ldcg(P.zc + o), rg = __ldcg(P.rc + o), cnd = __ldcg(P.cc + o);
-            const float h = M.Xs[b * in + H + r_begin + r];
-            dpc[b * SR + r] = g * z * (1.f - cnd * cnd);
-            dpz[b * SR + r] = g * (cnd - h) * z * (1.f - z);
-            dirp[b * SR + r] = g * (1.f - z);
+            const float h = M.Xs[b * LX + H + r_begin + r];
+            dpc[b * RP + r] = g * z * (1.f - cnd * cnd);
+            dpz[b * RP + r] = g * (cnd - h) * z * (1.f - z);
+            dirp[b * RP + r] = g * (1.f - z);
             M.Ys[b * SR + r] = rg;
           }
-          for (int idx = tid; idx < nb * in; idx += THREADS) {
-            const int b = idx / in, c = idx - b * in, m = S.rowmsg[b];
-            float v = M.Xs[idx];
-            if (c >= H) v *= __ldcg(P.rc + (size_t)(S.key[m] * P.rows_max + (b - S.rowoff[m])) * H + (c - H));
-            M.XC[idx] = v;
-          }
+          gru_gated_input(P, S, M.Xs, M.XC, LX, nb);
           __syncthreads();
-          AMP_DISPATCH_J(P.J, (tile_dW<J>(dpc, SR, nb, Wc, in, R, in, part1)));      // [da_c; dq] partial
+          AMP_STEP(6);
+          AMP_DISPATCH_J(P.J, (tile_dW<J>(dpc, RP, nb, Wc, LW, R, in, part1)));      // [da_c; dq] partial
+          AMP_STEP(7);
           __threadfence();
           if (P.T > 1) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
           else __syncthreads();
+          AMP_STEP(8);
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R;
             float dq = 0.f;
@@ -1666,20 +1704,23 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
 #pragma unroll
               for (int t = 0; t < 8; t++) dq += v[t];
             }
-            const float rg = M.Ys[b * SR + r], h = M.Xs[b * in + H + r_begin + r];
-            dpr[b * SR + r] = dq * h * rg * (1.f - rg);
-            dirbuf[(size_t)b * H + r_begin + r] = dirp[b * SR + r] + dq * rg;
+            const float rg = M.Ys[b * SR + r], h = M.Xs[b * LX + H + r_begin + r];
+            dpr[b * RP + r] = dq * h * rg * (1.f - rg);
+            dirbuf[(size_t)b * H + r_begin + r] = dirp[b * RP + r] + dq * rg;
           }
           __syncthreads();
+          AMP_STEP(9);
           // this tile's share of da_c joins its second partial here, so that emission sums one partial array per tile
-          AMP_DISPATCH_J(P.J, (tile_dW2<J>(dpz, dpr, SR, nb, Wz, Wr, in, R, in, part1, H, part2)));
-          tile_accum(dpz, SR, nb, M.Xs, in, M.As, in, R, in);
-          tile_accum(dpr, SR, nb, M.Xs, in, M.As + SR * in, in, R, in);
-          tile_accum(dpc, SR, nb, M.XC, in, M.As + 2 * SR * in, in, R, in);
+          AMP_DISPATCH_J(P.J, (tile_dW2<J>(dpz, dpr, RP, nb, Wz, Wr, LW, R, in, part1, H, part2)));
+          AMP_STEP(10);
+          tile_accum(dpz, RP, nb, M.Xs, LX, M.As, LW, R, in);
+          tile_accum(dpr, RP, nb, M.Xs, LX, M.As + SR * LW, LW, R, in);
+          tile_accum(dpc, RP, nb, M.XC, LX, M.As + 2 * SR * LW, LW, R, in);
+          AMP_STEP(11);
           for (int k = tid; k < 3 * R; k += THREADS) {
             const int m = k / R, r = k - m * R;
             float sacc = M.Abs[m * SR + r];
-            for (int b = 0; b < nb; b++) sacc += M.Ds[m * BR + b * SR + r];
+            for (int b = 0; b < nb; b++) sacc += M.Ds[m * BRD + b * RP + r];
             M.Abs[m * SR + r] = sacc;
           }
         }
@@ -1726,12 +1767,13 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
   __syncthreads();
   if (P.kind != LOOKUP)
     for (int m = 0; m < nmat; m++) {
-      for (int i = tid; i < R * in; i += THREADS) P.W[(size_t)m * out * in + (size_t)r_begin * in + i] = M.Ws[m * P.R * in + i];
+      for (int i = tid; i < R * in; i += THREADS) { const int r = i / in; P.W[(size_t)m * out * in + (size_t)r_begin * in + i] = M.Ws[(m * P.R + r) * LW + (i - r * in)]; }
       for (int i = tid; i < R; i += THREADS) P.b[m * out + r_begin + i] = M.bs[m * P.R + i];
     }
   if (tile == 0) {
     if (!C.sched_ctas) write_leader_stats(P, S);
     if (tid < 16) P.stats->phase_cycles[tid] = S.phase[tid];
+    if (tid < 16) C.g->step_cycles[(int)(&P - g_ppts)][tid] = S.step[tid];
   }
 }
 

@@ -143,6 +143,7 @@ struct Globals {                      // mutable run state in device memory (zer
   // cycles by role: [0..7] controller (retire, admit, clear, pump, idle, admissions), then per PPT node p at 8 + 8 p:
   // scheduler (waiting for tile 0, no message pending, forming) and emitters (waiting, loading, emitting, batches)
   unsigned long long role_cycles[8 + 8 * MAX_SMEM_PPTS];
+  unsigned long long step_cycles[MAX_SMEM_PPTS][16];   // tile 0 of every node: cycles between the marks inside the arithmetic phase
 };
 
 struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of the node's emitter CTAs (pad = which one), 2: the node's scheduler CTA
