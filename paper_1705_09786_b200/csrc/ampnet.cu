@@ -49,6 +49,7 @@ struct HostPPT {
   size_t nW = 0, nb = 0;
   int T = 1, R = 0, BM = 0, J = 0;
   int NE = 0, G = 1;                    // emitter CTAs of the node and their batch groups
+  double emit_load = 0.0;               // emitter-seconds the node's emission took in the last asynchronous epoch (0: unknown)
   size_t smem_floats = 0;
 };
 
@@ -442,15 +443,34 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   if (emitters > 0) {
     const int need = 1 + (used - 1) * (1 + emitters) + (int)g->ppts.size();
     if (need > n_ctas) return AMPNET_EOVERFLOW;                                                     // retried with fewer emitters / tiles
-    for (auto& P : g->ppts) P.NE = P.T * emitters;
-    // spare SMs become emitters of the nodes that have the fewest (a node with few row tiles emits as many messages)
-    for (int spare = n_ctas - need; spare > 0; spare--) {
-      HostPPT* best = nullptr;
-      for (auto& P : g->ppts) if (P.NE < 24 && (!best || P.NE < best->NE)) best = &P;
-      if (!best) break;
-      best->NE++;
+    double load = 0.0;
+    for (auto& P : g->ppts) load += P.emit_load;
+    if (load > 0.0) {
+      // Feedback from the last asynchronous epoch: every node keeps two emitters, the rest of the pool is dealt out in
+      // proportion to the emitter time the nodes' emission took (largest remainder first).
+      const int pool = n_ctas - 1 - np - (used - 1);
+      int left = pool;
+      for (auto& P : g->ppts) { P.NE = 2; left -= 2; }
+      std::vector<double> want(np);
+      for (int p = 0; p < np; p++) want[p] = g->ppts[p].emit_load / load * std::max(left, 0);
+      for (int p = 0; p < np && left > 0; p++) { const int k = std::min(left, (int)std::floor(want[p])); g->ppts[p].NE += k; left -= k; want[p] -= k; }
+      while (left > 0) {
+        int best = 0;
+        for (int p = 1; p < np; p++) if (want[p] > want[best]) best = p;
+        g->ppts[best].NE++; want[best] -= 1.0; left--;
+      }
+    } else {
+      for (auto& P : g->ppts) P.NE = P.T * emitters;
+      // spare SMs become emitters of the nodes that have the fewest (a node with few row tiles emits as many messages)
+      for (int spare = n_ctas - need; spare > 0; spare--) {
+        HostPPT* best = nullptr;
+        for (auto& P : g->ppts) if (P.NE < 24 && (!best || P.NE < best->NE)) best = &P;
+        if (!best) break;
+        best->NE++;
+      }
     }
-    for (auto& P : g->ppts) P.G = std::min(2, P.NE);
+    // batch groups: a large pool works on up to four batches at a time (a batch's emission can take several tile cycles)
+    for (auto& P : g->ppts) P.G = P.NE >= 16 ? 4 : P.NE >= 9 ? 3 : std::min(2, P.NE);
     for (int p = 0; p < (int)g->ppts.size(); p++) roles.push_back(Role{p, 0, 2, 0});                 // one scheduler CTA per node
     for (int p = 0; p < (int)g->ppts.size(); p++)
       for (int e = 0; e < g->ppts[p].NE; e++) roles.push_back(Role{p, 0, 1, e});
@@ -486,7 +506,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   }
   if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0); }
   if (st != AMPNET_OK) return st;
-  const int depth = emit_ctas > 0 ? 3 : 2;       // emitters work in two batch groups: a tile may be two batches ahead
+  const int depth = emit_ctas > 0 ? 5 : 2;       // emitters work in up to four batch groups: a tile may be four batches ahead
   R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth; R.ctx.sched_ctas = emit_ctas > 0 ? 1 : 0;
   n_ctas = (int)R.roles.size();
   DeviceArena &C = g->ctl, &B = g->bulk;
@@ -734,6 +754,8 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   if (dbg) fprintf(stderr, "[ampnet] done\n");
   g->have_run = true;
   if (!eval) for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].opt_t += (long long)g->last_stats[p].n_updates;
+  if (!eval && !det && R.ctx.emit_ctas)      // emitter time of the node = time of its first emitter x emitters (they share every batch)
+    for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].emit_load = (double)G.role_cycles[8 + 8 * p + 5] * std::max(1, g->ppts[p].NE) + 1.0;
   if (getenv("AMPNET_TUNE") && (atoi(getenv("AMPNET_TUNE")) & 8)) {
     static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK"};
     const double us = 1.0 / 1965.0;
