@@ -906,7 +906,8 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
     const int i = lane + 32 * j;
     if (i >= take) continue;
     P.sched[(S.ls.sched_w + i) & P.sched_mask] = slot[j];
-    if (!C.det) {
+    if (C.sched_ctas) S.hdr[i] = h[j];                 // the scheduler CTA assembles the batch context from its own copy
+    else if (!C.det) {
       int4* b = reinterpret_cast<int4*>(&P.bhdr[(S.ls.batch_w & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + i]);
       b[0] = make_int4(h[j].inst, h[j].seq, h[j].slot, h[j].it);
       b[1] = make_int4(h[j].u, h[j].port, h[j].rows, h[j].flags);
@@ -929,8 +930,8 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
     BatchDesc d;
     d.sched_start = S.ls.sched_w; d.count = take; d.dir = dir; d.flags = upd ? BATCH_UPDATE : 0;
     d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.upd_t = upd ? (int)S.ls.n_updates + 1 : 0; d.pad1 = 0;
-    P.batches[S.ls.batch_w & P.batch_mask] = d;
-    if (!C.sched_ctas) { __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }   // a scheduler CTA publishes the assembled context instead
+    if (C.sched_ctas) S.desc = d;                      // a scheduler CTA publishes the assembled context instead
+    else { P.batches[S.ls.batch_w & P.batch_mask] = d; __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
     S.ls.batch_w++;
     S.ls.sched_w += take;
     LeaderState& st = S.ls;
@@ -955,8 +956,8 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
     st.log_n++; st.n_updates++; st.n_grads_applied += d.n_upd;
     S.ls.n_acc = 0; S.ls.version++;
   }
-  P.batches[S.ls.batch_w & P.batch_mask] = d;
-  if (!C.sched_ctas) { __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
+  if (C.sched_ctas) S.desc = d;
+  else { P.batches[S.ls.batch_w & P.batch_mask] = d; __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
   S.ls.batch_w++;
 }
 
@@ -1132,11 +1133,13 @@ __device__ __forceinline__ void init_leader_state(TileShared& S) {              
 }
 
 // Warp 0 of a CTA: descriptor, headers, keys, row offsets and row pointers of batch `batch` into shared memory.
-__device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared& S, const unsigned my_batch) {
+// local: descriptor and headers are already in this CTA's shared memory (the scheduler CTA that has just formed the batch).
+__device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared& S, const unsigned my_batch, const bool local = false) {
   const int lane = threadIdx.x & 31;
   const int in = P.in_dim;
-  const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]);
-  const int4 d0 = __ldcg(dp), d1 = __ldcg(dp + 1);          // same address in every lane
+  int4 d0, d1;
+  if (local) { const int4* dp = reinterpret_cast<const int4*>(&S.desc); d0 = dp[0]; d1 = dp[1]; }
+  else { const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]); d0 = __ldcg(dp); d1 = __ldcg(dp + 1); }
   const int cnt = d0.y, ddir = d0.z;
   Hdr h[2];
   int cum[2], rows[2];
@@ -1144,7 +1147,9 @@ __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared&
   for (int j = 0; j < 2; j++) {                             // message lane + 32 j
     const int i = lane + 32 * j;
     int4 ha = make_int4(0, 0, 0, 0), hb = make_int4(0, 0, 0, 0);
-    if (!C.det) {                                           // headers travel with the descriptor: load both at once
+    if (local) {
+      if (i < cnt) { const int4* e = reinterpret_cast<const int4*>(&S.hdr[i]); ha = e[0]; hb = e[1]; }
+    } else if (!C.det) {                                    // headers travel with the descriptor: load both at once
       const int4* e = reinterpret_cast<const int4*>(&P.bhdr[(my_batch & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + i]);
       ha = __ldcg(e); hb = __ldcg(e + 1);
     } else if (i < cnt) {
@@ -1213,7 +1218,7 @@ __device__ __forceinline__ void fetch_ctx_block(const DevPPT& P, TileShared& S, 
 // Scheduler CTA, warp 0: assemble the context of the batch just formed and publish it.
 __device__ __noinline__ void publish_ctx_block(const Ctx& C, DevPPT& P, TileShared& S, const unsigned batch) {
   const int lane = threadIdx.x & 31;
-  load_batch_ctx(C, P, S, batch);
+  load_batch_ctx(C, P, S, batch, true);
   __syncwarp();
   const int4* src = reinterpret_cast<const int4*>(static_cast<BatchCtx*>(&S));
   int4* dst = reinterpret_cast<int4*>(P.ctxblk + (batch & (BATCH_BLOCKS - 1)));
@@ -1866,7 +1871,7 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
       if (lane == 0) { const long long tn = clock64(); rcl[!gow ? 0 : progressed ? 2 : 1] += (unsigned long long)(tn - tp); tp = tn; }
       if (gow) {
         unsigned fin = 0;
-        if (lane == 0) fin = progressed && (P.batches[bw & P.batch_mask].flags & BATCH_TERMINATE);
+        if (lane == 0) fin = progressed && (S.desc.flags & BATCH_TERMINATE);
         if (warp_uniform(fin)) break;
       }
       if (progressed) { it = 0; continue; }
