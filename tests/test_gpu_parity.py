@@ -197,6 +197,35 @@ def test_async_mode_invariants(family, n, mak, muf, lr):
         assert losses[-1] < losses[0]
 
 
+@pytest.mark.parametrize("family,n,mak,muf,lr", [("tree", 8544, 64, 100, 0.05), ("ggnn", 20000, 128, 200, 0.01)])
+def test_full_size_epoch_in_the_timed_configuration(oracle_mod, family, n, mak, muf, lr):
+    """The sizes and the launch configuration that bench.py times (asynchronous mode, full dataset).  What holds for
+    every schedule is checked exactly over the whole epoch; the parameters the epoch produced are then handed to the
+    oracle, which recomputes the loss of sampled instances one by one."""
+    import paper_1705_09786_b200 as amp
+    g, inst = _case(family, n)
+    e = amp.Engine(g)
+    e.load_instances(inst)
+    e.load_instances(inst, split=1)
+    e.set_params(wp.init_params(g))
+    st, loss = e.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=False, timeout_s=120)
+    assert st.instances == inst.n and st.max_active_observed <= mak
+    assert e.leftover_cache_entries() == 0 and np.isfinite(loss).all()
+    want = parity_counts(g, inst)
+    assert st.node_messages == want["node_messages"]
+    for node, G in want["grads"].items():
+        assert e.node_stats(node)["n_grads_applied"] == G == e.update_log(node).sum()
+    # forward pass at full size against the oracle on a sample (same parameters on both sides)
+    _, _, eloss = e.eval(split=1, mak=mak)
+    idx = np.random.default_rng(5).choice(inst.n, size=48, replace=False)
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst.subset(idx), split=1)
+    o.set_params(e.get_params())
+    _, _, oloss = o.eval(split=1)
+    np.testing.assert_allclose(eloss[idx], oloss, rtol=1e-5, atol=2e-6)
+    e.close()
+
+
 def parity_counts(g, inst):
     if g.name == "mlp":
         return dict(node_messages=7 * inst.n, grads={n: inst.n for n in g.ppt_nodes()})
