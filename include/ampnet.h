@@ -67,7 +67,8 @@ enum { AMPNET_SRC_DENSE_ROW = 1, AMPNET_SRC_TOKENS = 2, AMPNET_SRC_ZERO_STATE = 
 enum { AMPNET_COND_SEQ_END = 1,   /* u < #tokens ? 0 : 1        */
        AMPNET_COND_TREE_ROOT = 2, /* u is the root ? 0 : 1      */
        AMPNET_COND_BY_U = 3,      /* successor = u              */
-       AMPNET_COND_IT_LT = 4 };   /* it < fn_arg ? 0 : 1        */
+       AMPNET_COND_IT_LT = 4,     /* it < fn_arg ? 0 : 1        */
+       AMPNET_COND_ROUND_ROBIN = 5 }; /* successor = (instance + u) mod successors: replicas of a node (Sec. 5) */
 enum { AMPNET_ISU_U_INC = 1, AMPNET_ISU_TREE_PARENT = 2, AMPNET_ISU_IT_INC = 3 };
 enum { AMPNET_CONCAT_BY_EDGE = 1, AMPNET_CONCAT_BY_STATE_PORT = 2 };
 enum { AMPNET_GROUP_EDGES_BY_TYPE = 1, AMPNET_GROUP_EDGES_BY_DST = 2, AMPNET_GROUP_ALL_NODES = 3 };
@@ -207,6 +208,19 @@ ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_t
  * ([8] look-ahead scheduling, [9] reduction of partial gradients, [10]/[12] own walks of warps 0/1, [11]/[13] helping
  * other warps, [14] closing barrier).  cycles16: 16 values.  batches: micro-batches executed.                    */
 ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles16, int64_t* batches);
+
+/* ---- replicas (Sec. 5) -------------------------------------------------------------------------------------
+ * A heavy node is replicated in full between a Cond (AMPNET_COND_ROUND_ROBIN) and a Phi; the copies train
+ * independently and are synchronised infrequently, at the end of an epoch, by averaging.  This call replaces the
+ * parameters of the n listed nodes (same type and shape, n >= 1) by their element-wise mean, on the device, between
+ * two epochs.  Optimiser state is left as it is.  nodes: host array of node indices.
+ * Errors: AMPNET_EINVAL (not a parameterised node, shapes differ), AMPNET_ECUDA.                                  */
+ampnet_status_t ampnet_average_params(ampnet_graph_t*, const int32_t* nodes, int32_t n);
+
+/* canonical RNN with Linear-1 replicated `replicas` times (replicas = 1: identical to ampnet_ir_rnn) */
+ampnet_status_t ampnet_ir_rnn_replicated(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes, int32_t act, int32_t replicas,
+                                         ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                                         ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
 
 /* ---- update rule of the local updates (Sec. 3; App. A lists the optimiser among the run-time options) -------
  * Every parameterised node applies the chosen rule to the MEAN of its accumulated gradients, g = A / n, whenever

@@ -58,7 +58,7 @@ enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS,
                 BCAST, GROUP, UNGROUP, FLATMAP, SINK, N_TYPES };
 enum Act { ACT_NONE, ACT_RELU, ACT_TANH, ACT_SIGMOID };
 enum { SRC_DENSE_ROW = 1, SRC_TOKENS, SRC_ZERO_STATE, SRC_TREE_LEAVES, SRC_GRAPH_NODES };
-enum { COND_SEQ_END = 1, COND_TREE_ROOT, COND_BY_U, COND_IT_LT };
+enum { COND_SEQ_END = 1, COND_TREE_ROOT, COND_BY_U, COND_IT_LT, COND_ROUND_ROBIN };
 enum { ISU_U_INC = 1, ISU_TREE_PARENT, ISU_IT_INC };
 enum { CONCAT_BY_EDGE = 1, CONCAT_BY_STATE_PORT };
 enum { GROUP_EDGES_BY_TYPE = 1, GROUP_EDGES_BY_DST, GROUP_ALL_NODES };
@@ -548,6 +548,7 @@ struct Cond : Node {            // routes on the state only; stateless
       case COND_TREE_ROOT: k = m.s.u == S.root ? 0 : 1; break;
       case COND_BY_U: k = m.s.u; break;
       case COND_IT_LT: k = m.s.it < fn_arg ? 0 : 1; break;
+      case COND_ROUND_ROBIN: k = (int)((m.s.inst + m.s.u) % (long long)E->succ[id].size()); break;   // replicas (Sec. 5)
       default: E->err = "Cond: unknown fn";
     }
     E->emit_fwd(id, k, m);

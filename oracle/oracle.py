@@ -139,6 +139,13 @@ class Oracle:
         if self.lib.oracle_set_optimizer(self.h, k, f(momentum), f(beta1), f(beta2), f(eps), int(reset)) != 0:
             raise ValueError(kind)
 
+    def average_params(self, nodes):
+        """End-of-epoch replica synchronisation (Sec. 5): every listed node gets the mean of their parameters."""
+        for which in (0, 1):
+            mean = sum(self._get(self.lib.oracle_get_params, n, which) for n in nodes) / len(nodes)
+            for n in nodes:
+                self.set_params({(n, which): mean})
+
     def eval(self, split=0):
         ml, acc = C.c_double(), C.c_double()
         loss = np.zeros(self.n[split], np.float64)

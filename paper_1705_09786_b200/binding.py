@@ -12,7 +12,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
+           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
            "ampnet_ir_tree", "ampnet_ir_ggnn"]
 
 
@@ -99,6 +99,8 @@ def load_library():
     tail = [P, I32, PI, P, I32, PI]
     lib.ampnet_ir_mlp.argtypes = [P, I32] + tail
     lib.ampnet_ir_rnn.argtypes = [I32] * 5 + tail
+    lib.ampnet_ir_rnn_replicated.argtypes = [I32] * 6 + tail
+    lib.ampnet_average_params.argtypes = [P, P, C.c_int32]
     lib.ampnet_ir_tree.argtypes = [I32] * 4 + tail
     lib.ampnet_ir_ggnn.argtypes = [I32] * 5 + tail
     lib.ampnet_last_error.argtypes = [P]
@@ -229,6 +231,11 @@ class Engine:
     def set_optimizer(self, kind="sgd", momentum=0.9, beta1=0.9, beta2=0.999, eps=1e-8, reset=True):
         k = {"sgd": 0, "momentum": 1, "adam": 2}[kind]
         self._check(self.lib.ampnet_set_optimizer(self.h, k, momentum, beta1, beta2, eps, int(reset)))
+
+    def average_params(self, nodes):
+        """End-of-epoch replica synchronisation (Sec. 5): the listed nodes get the mean of their parameters."""
+        a = np.ascontiguousarray(nodes, dtype=np.int32)
+        self._check(self.lib.ampnet_average_params(self.h, _p(a), len(a)))
 
     def eval(self, split=0, mak=64):
         ml, acc = C.c_double(), C.c_double()

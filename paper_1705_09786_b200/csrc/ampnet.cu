@@ -86,6 +86,20 @@ struct ampnet_graph {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
 };
 
+// End-of-epoch replica synchronisation (Sec. 5): element-wise mean of up to eight nodes' parameters, written back to all.
+struct AvgArgs { float* W[8]; float* b[8]; int n; long long nW, nb; };
+__global__ void average_params_kernel(const AvgArgs a) {
+  const long long total = a.nW + a.nb, stride = (long long)gridDim.x * blockDim.x;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+    float* const* arr = i < a.nW ? a.W : a.b;
+    const long long j = i < a.nW ? i : i - a.nW;
+    float s = 0.f;
+    for (int k = 0; k < a.n; k++) s += arr[k][j];
+    s /= (float)a.n;
+    for (int k = 0; k < a.n; k++) arr[k][j] = s;
+  }
+}
+
 namespace {
 
 ampnet_status_t set_err(ampnet_graph* g, ampnet_status_t st, const char* fmt, ...) {
@@ -217,7 +231,7 @@ ampnet_status_t build_topology(ampnet_graph* g) {
         if (st == AMPNET_OK) g->losses.push_back(i);
         break;
       case SINK: st = need(h.n_pred == 1 && h.n_succ == 0, "SINK needs one predecessor and no successor"); break;
-      case COND: st = need(h.n_pred == 1 && h.n_succ >= 1 && h.fn >= 1 && h.fn <= 4, "COND needs one predecessor and a valid fn"); break;
+      case COND: st = need(h.n_pred == 1 && h.n_succ >= 1 && h.fn >= 1 && h.fn <= 5, "COND needs one predecessor and a valid fn"); break;
       case PHI: st = need(h.n_pred >= 1 && h.n_succ == 1, "PHI needs predecessors and one successor"); break;
       case ISU:
         st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 3, "ISU needs a valid fn");
@@ -872,6 +886,30 @@ ampnet_status_t ampnet_set_optimizer(ampnet_graph_t* g, int32_t kind, float mome
   }
   CUDA_TRY(g, cudaStreamSynchronize(g->stream));
   g->opt = kind; g->opt_mu = momentum; g->opt_beta1 = beta1; g->opt_beta2 = beta2; g->opt_eps = eps;
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_average_params(ampnet_graph_t* g, const int32_t* nodes, int32_t n) {
+  if (!g) return AMPNET_EINVAL;
+  if (!nodes || n < 1 || n > 8) return set_err(g, AMPNET_EINVAL, "between 1 and 8 nodes are averaged");
+  AvgArgs a{};
+  const HostPPT* first = nullptr;
+  for (int k = 0; k < n; k++) {
+    const int node = nodes[k];
+    if (node < 0 || node >= (int)g->hnodes.size() || g->hnodes[node].ppt < 0) return set_err(g, AMPNET_EINVAL, "node %d has no parameters", node);
+    const HostPPT& P = g->ppts[g->hnodes[node].ppt];
+    if (!first) first = &P;
+    if (P.kind != first->kind || P.nW != first->nW || P.nb != first->nb) return set_err(g, AMPNET_EINVAL, "node %d differs in type or shape from node %d", node, nodes[0]);
+    for (int j = 0; j < k; j++) if (nodes[j] == node) return set_err(g, AMPNET_EINVAL, "node %d is listed twice", node);
+    a.W[k] = P.W; a.b[k] = P.b;
+  }
+  a.n = n; a.nW = (long long)first->nW; a.nb = (long long)first->nb;
+  CUDA_TRY(g, cudaSetDevice(g->device));
+  const long long total = a.nW + a.nb;
+  const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
+  average_params_kernel<<<blocks, 256, 0, g->stream>>>(a);
+  CUDA_TRY(g, cudaGetLastError());
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
   return AMPNET_OK;
 }
 

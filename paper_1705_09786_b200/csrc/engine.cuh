@@ -369,6 +369,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
               case 2: k = I.parent[f.ibase + f.u] < 0 ? 0 : 1; break;      // the root has no parent
               case 3: k = f.u; break;
               case 4: k = f.it < n.fn_arg ? 0 : 1; break;
+              case 5: k = (f.inst + f.u) % n.n_succ; break;                  // replicas of a node (Sec. 5)
             }
             if ((unsigned)k >= (unsigned)n.n_succ) { fail(C, ST_OVERFLOW, f.node, k); return; }
             to_succ(f, n, k);

@@ -52,7 +52,14 @@ ampnet_status_t ampnet_ir_mlp(const int32_t* dims, int32_t n_dims, ampnet_node_d
 ampnet_status_t ampnet_ir_rnn(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes, int32_t act,
                               ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
                               ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges) {
+  return ampnet_ir_rnn_replicated(vocab, emb, hidden, classes, act, 1, nodes, cap_nodes, n_nodes, edges, cap_edges, n_edges);
+}
+
+ampnet_status_t ampnet_ir_rnn_replicated(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes, int32_t act, int32_t replicas,
+                                         ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                                         ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges) {
   if (vocab < 1 || emb < 1 || hidden < 1 || classes < 1 || emb != hidden) return AMPNET_EINVAL;   // one width per Concat port
+  if (replicas < 1 || replicas > 8) return AMPNET_EINVAL;                                          // a Cond has at most 8 ports
   Builder b;
   int s_tok = b.node(AMPNET_SOURCE, 0, 0, 0, AMPNET_SRC_TOKENS);
   int look = b.node(AMPNET_LOOKUP, vocab, emb, 0, 0, 0, AMPNET_FLAG_SOURCE_ADJACENT);
@@ -68,8 +75,22 @@ ampnet_status_t ampnet_ir_rnn(int32_t vocab, int32_t emb, int32_t hidden, int32_
   b.edge(look, cat, 0, 0);
   b.edge(s_h0, phi, 0, 0);
   b.edge(phi, cat, 0, 1);
-  b.edge(cat, lin1);
-  b.edge(lin1, isu);
+  if (replicas > 1) {      // the copies go between a round-robin Cond and a Phi, after the canonical nodes
+    int cond_r = b.node(AMPNET_COND, emb + hidden, emb + hidden, 0, AMPNET_COND_ROUND_ROBIN);
+    int phi_r = b.node(AMPNET_PHI, hidden, hidden);
+    b.edge(cat, cond_r);
+    b.edge(cond_r, lin1, 0, 0);
+    b.edge(lin1, phi_r, 0, 0);
+    for (int k = 1; k < replicas; k++) {
+      int c = b.node(AMPNET_LINEAR, emb + hidden, hidden, act);
+      b.edge(cond_r, c, k, 0);
+      b.edge(c, phi_r, 0, k);
+    }
+    b.edge(phi_r, isu);
+  } else {
+    b.edge(cat, lin1);
+    b.edge(lin1, isu);
+  }
   b.edge(isu, cond);
   b.edge(cond, phi, 0, 1);
   b.edge(cond, lin2, 1, 0);

@@ -81,6 +81,38 @@ def test_momentum_and_adam_updates_match_oracle(oracle_mod, family, n, mak, muf,
     e.close()
 
 
+@pytest.mark.parametrize("k,mak,muf", [(2, 8, 10), (4, 16, 5)])
+def test_replicated_linear_with_end_of_epoch_averaging(oracle_mod, k, mak, muf):
+    """Linear-1 of the list RNN replicated k times between a round-robin Cond and a Phi (Sec. 5): an epoch, the
+    averaging of the copies, and a second epoch that starts from the averaged copies, on both sides."""
+    g = ir.rnn(replicas=k)
+    inst = data.list_instances(n=70)
+    p = wp.init_params(g)
+    copies = [g.index("linear1")] + [g.index(f"linear1_r{r}") for r in range(1, k)]
+    o, ost, oloss, e, est, eloss = parity.run_both(oracle_mod, g, inst, p, mak, muf, 0.02)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    T = np.diff(inst.offsets)
+    assert est.node_messages == int((17 * T + 3).sum())
+    assert all(e.node_stats(c)["fwd_msgs"] > 0 for c in copies)
+    o.average_params(copies)
+    e.average_params(copies)
+    ep, op = e.get_params(), o.get_params()
+    for c in copies:
+        for which in (0, 1):
+            np.testing.assert_array_equal(ep[(c, which)], ep[(copies[0], which)])
+            np.testing.assert_allclose(ep[(c, which)], op[(c, which)], rtol=1e-4, atol=1e-6)
+    ost, oloss = o.run_epoch(mak=mak, muf=muf, lr=0.02)
+    est, eloss = e.run_epoch(mak=mak, muf=muf, lr=0.02, deterministic=True, timeout_s=60)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    # the free-running schedule: exact accounting with replicas
+    st, loss = e.run_epoch(mak=mak, muf=muf, lr=0.02, deterministic=False, timeout_s=60)
+    assert st.node_messages == int((17 * T + 3).sum()) and e.leftover_cache_entries() == 0 and np.isfinite(loss).all()
+    assert sum(e.node_stats(c)["n_grads_applied"] for c in copies) == T.sum()
+    with pytest.raises(Exception):
+        e.average_params([copies[0], g.index("linear2")])          # shapes differ
+    e.close()
+
+
 def test_partial_epoch_and_degenerate_sizes(oracle_mod):
     """One instance; mak larger than the instance count; a prefix of the data; the smallest structures."""
     g, inst = _case("rnn", 9)

@@ -369,3 +369,61 @@ def test_optimizers_match_torch_optim_on_minibatch_training(oracle_mod, kind):
             opt.step()
     for k, v in P.items():
         np.testing.assert_allclose(o.get_params(*k), v.detach().numpy(), rtol=1e-9, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------------
+# replicas of a heavy node between a round-robin Cond and a Phi, synchronised by averaging (Sec. 5)
+# ---------------------------------------------------------------------------------------------------
+def _replicated_case(k, n=6):
+    g1 = ir.rnn(emb=6, hidden=6)
+    gk = ir.rnn(emb=6, hidden=6, replicas=k)
+    inst = data.list_instances(n=n, max_len=5)
+    p1 = wp.init_params(g1)
+    copies = [gk.index("linear1")] + [gk.index(f"linear1_r{r}") for r in range(1, k)]
+    pk = {}
+    for (node, which), v in p1.items():                  # the canonical nodes keep their indices in the replicated graph
+        pk[(node, which)] = v
+    for c in copies[1:]:
+        pk[(c, 0)], pk[(c, 1)] = p1[(g1.index("linear1"), 0)], p1[(g1.index("linear1"), 1)]
+    return g1, gk, inst, p1, pk, copies
+
+
+@pytest.mark.parametrize("k", [2, 3])
+def test_replicas_split_the_gradient_of_the_unreplicated_model(oracle_mod, k):
+    """With identical copies the model computes the same function, so the copies' accumulated gradients add up to the
+    gradient of the unreplicated model (autograd of the independent formulation), every copy serves exactly the
+    (instance, position) pairs with (instance + position) mod k = its port, and the other nodes are unaffected."""
+    g1, gk, inst, p1, pk, copies = _replicated_case(k)
+    o = make(oracle_mod, gk, inst, pk)
+    st, loss = o.run_epoch(mak=3, muf=BIG, lr=0.1, flush=False)
+    grads, losses = H.dataset_grad(g1, p1, inst)
+    np.testing.assert_allclose(loss, losses, rtol=1e-12, atol=1e-13)
+    lin1 = g1.index("linear1")
+    for which in (0, 1):
+        total = sum(o.get_accum(c, which) for c in copies)
+        np.testing.assert_allclose(total, grads[(lin1, which)], rtol=1e-9, atol=1e-12)
+    for (node, which), gr in grads.items():
+        if node != lin1:
+            np.testing.assert_allclose(o.get_accum(node, which), gr, rtol=1e-9, atol=1e-12)
+    T = np.diff(inst.offsets)
+    for r, c in enumerate(copies):
+        want = sum(1 for i in range(inst.n) for u in range(T[i]) if (i + u) % k == r)
+        assert o.node_stats(c)["fwd_msgs"] == want == o.node_stats(c)["bwd_msgs"]
+    assert st.node_messages == int((17 * T + 3).sum()) and st.leftover_cache_entries == 0
+
+
+def test_replica_averaging_is_the_mean_and_keeps_other_nodes(oracle_mod):
+    g1, gk, inst, p1, pk, copies = _replicated_case(2, n=8)
+    o = make(oracle_mod, gk, inst, pk)
+    o.run_epoch(mak=2, muf=3, lr=float(np.float32(0.05)))
+    before = o.get_params()
+    assert np.abs(before[(copies[0], 0)] - before[(copies[1], 0)]).max() > 0      # the copies have drifted apart
+    o.average_params(copies)
+    after = o.get_params()
+    for which in (0, 1):
+        mean = (before[(copies[0], which)] + before[(copies[1], which)]) / 2
+        for c in copies:
+            np.testing.assert_allclose(after[(c, which)], mean, rtol=0, atol=1e-15)
+    for key in before:
+        if key[0] not in copies:
+            np.testing.assert_array_equal(after[key], before[key])

@@ -40,6 +40,7 @@ COND_SEQ_END = 1       # u < T ? 0 : 1          (T = number of tokens of the ins
 COND_TREE_ROOT = 2     # u is the root ? 0 : 1
 COND_BY_U = 3          # successor = u
 COND_IT_LT = 4         # it < fn_arg ? 0 : 1
+COND_ROUND_ROBIN = 5   # successor = (instance + u) mod number of successors   (replicas, Sec. 5)
 # ISU.fn: invertible state update
 ISU_U_INC = 1          # u -> u + 1
 ISU_TREE_PARENT = 2    # (u, port) -> (parent(u), child slot of u); inverse picks the child
@@ -129,9 +130,11 @@ def mlp(dims=(784, 256, 256, 10)):
     return g
 
 
-def rnn(vocab=14, emb=128, hidden=128, classes=10, act=ACT_TANH):
+def rnn(vocab=14, emb=128, hidden=128, classes=10, act=ACT_TANH, replicas=1):
     """Variable-length RNN (paper Fig. 2): Lookup -> Concat(with h from Phi) -> Linear-1 -> Isu(t+1)
-    -> Cond(end?) -> Phi loop | Linear-2 -> Loss.  13T+3 node-messages for T tokens."""
+    -> Cond(end?) -> Phi loop | Linear-2 -> Loss.  13T+3 node-messages for T tokens.
+    replicas > 1: Linear-1 is replicated in full between a Cond (round robin over instance + position) and a Phi
+    (Sec. 5); the copies are "linear1", "linear1_r1", ...; 17T+3 node-messages."""
     assert emb == hidden, "Concat ports have one common width"
     g = IRGraph("rnn")
     s_tok = g.node("src_tokens", SOURCE, fn=SRC_TOKENS)
@@ -148,8 +151,18 @@ def rnn(vocab=14, emb=128, hidden=128, classes=10, act=ACT_TANH):
     g.edge(look, cat, 0, 0)
     g.edge(s_h0, phi, 0, 0)
     g.edge(phi, cat, 0, 1)
-    g.edge(cat, lin1)
-    g.edge(lin1, isu)
+    if replicas > 1:            # appended after the canonical nodes, so that those keep their indices
+        cond_r = g.node("cond_replica", COND, emb + hidden, emb + hidden, fn=COND_ROUND_ROBIN)
+        phi_r = g.node("phi_replica", PHI, hidden, hidden)
+        copies = [lin1] + [g.node(f"linear1_r{k}", LINEAR, emb + hidden, hidden, act=act) for k in range(1, replicas)]
+        g.edge(cat, cond_r)
+        for k, c in enumerate(copies):
+            g.edge(cond_r, c, k, 0)
+            g.edge(c, phi_r, 0, k)
+        g.edge(phi_r, isu)
+    else:
+        g.edge(cat, lin1)
+        g.edge(lin1, isu)
     g.edge(isu, cond)
     g.edge(cond, phi, 0, 1)     # loop
     g.edge(cond, lin2, 1, 0)    # exit
