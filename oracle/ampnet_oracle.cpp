@@ -187,6 +187,7 @@ struct Engine {
   std::vector<std::vector<Msg>> inbox_a, inbox_b;
   std::vector<std::vector<Msg>>* target = nullptr;
   std::vector<int> retire_notices;       // slots
+  std::vector<int> inflight_eval;        // per slot: forward-only messages of the slot's instance waiting in PPT inboxes
   std::vector<double> loss;              // per instance
   std::vector<int> correct, n_pred;      // eval accuracy bookkeeping
   int64_t node_messages = 0, ppt_messages = 0;
@@ -204,6 +205,7 @@ struct Engine {
     route_hash += msg_hash(node, m.dir, aport, m.s);
     if (m.dir == FWD) n->st.fwd_msgs++; else n->st.bwd_msgs++;
     if (n->is_ppt()) {
+      if (m.eval && !inflight_eval.empty()) inflight_eval[m.s.slot]++;
       (*target)[node].push_back(m);
       return;
     }
@@ -882,6 +884,7 @@ struct Oracle {
       for (auto& m : box) {
         E.ppt_messages++;
         if (m.dir == FWD) n->forward(m, 0); else n->backward(m, 0);
+        if (m.eval && !E.inflight_eval.empty()) E.inflight_eval[m.s.slot]--;      // after its successors were emitted
       }
       box.clear();
     }
@@ -891,8 +894,11 @@ struct Oracle {
     return true;
   }
 
+  // inference_only (may be null): per instance, != 0 marks an instance that is only evaluated (forward messages, nothing
+  // cached, no gradients) while the others train: concurrent inference in the same queues (Sec. 1, Sec. 6).  Such an
+  // instance is finished, and its key released in the next round, once none of its messages is left anywhere.
   int run_epoch(int split, int mak, int muf, double lr, const int64_t* order, int64_t n_order, int flush,
-                RunStats* out, double* per_instance_loss) {
+                RunStats* out, double* per_instance_loss, const uint8_t* inference_only = nullptr, double* inf_out = nullptr) {
     E.cur = &E.data[split];
     const int64_t n_inst = (int64_t)E.cur->inst.size();
     E.mak = mak; E.muf = muf; E.lr = (real)lr; E.err.clear();
@@ -903,6 +909,8 @@ struct Oracle {
     for (auto& n : E.nodes) { n->reset_run(); n->st = NodeStats(); }
     key_log.clear();
     std::vector<int> slot_inst(mak, -1), outstanding(mak, 0), slot_log(mak, -1);
+    std::vector<char> slot_eval(mak, 0);
+    E.inflight_eval.assign(inference_only ? mak : 0, 0);
     int active = 0; int64_t next = 0, max_active = 0, r = 0;
     auto* cur = &E.inbox_a; auto* nxt = &E.inbox_b;
     for (;; r++) {
@@ -921,7 +929,9 @@ struct Oracle {
         slot_inst[slot] = inst; active++;
         slot_log[slot] = (int)key_log.size();
         key_log.push_back(KeyLogEntry{inst, slot, r, -1});
-        outstanding[slot] = pump_sources(inst, (int)next, slot, false);
+        slot_eval[slot] = inference_only && inference_only[inst];
+        outstanding[slot] = pump_sources(inst, (int)next, slot, slot_eval[slot] != 0);
+        if (slot_eval[slot]) outstanding[slot] = 1;            // one notice: "nothing of this instance is left"
         next++;
       }
       max_active = std::max<int64_t>(max_active, active);
@@ -931,6 +941,8 @@ struct Oracle {
       E.target = nxt;
       process_ppt_inboxes(*cur);
       std::swap(cur, nxt);
+      for (int sl = 0; sl < mak && inference_only; sl++)
+        if (slot_inst[sl] >= 0 && slot_eval[sl] && outstanding[sl] == 1 && E.inflight_eval[sl] == 0) E.retire_notices.push_back(sl);
       if (!E.err.empty()) return 1;
       if (r > (int64_t)4e9) { E.err = "schedule did not terminate"; return 1; }
     }
@@ -938,12 +950,17 @@ struct Oracle {
     int64_t leftover = 0;
     int max_stale = 0;
     for (auto& n : E.nodes) { leftover += (int64_t)n->cache_size(); max_stale = std::max(max_stale, n->st.max_staleness); }
-    double tot = 0;
-    for (int64_t i = 0; i < n_order; i++) tot += E.loss[order[i]];
+    double tot = 0, itot = 0; int64_t n_train = 0, n_inf = 0, ic = 0, ip = 0;
+    for (int64_t i = 0; i < n_order; i++) {
+      const int64_t k = order[i];
+      if (inference_only && inference_only[k]) { itot += E.loss[k]; n_inf++; ic += E.correct[k]; ip += E.n_pred[k]; }
+      else { tot += E.loss[k]; n_train++; }
+    }
+    if (inf_out) { inf_out[0] = (double)n_inf; inf_out[1] = n_inf ? itot / n_inf : 0; inf_out[2] = ip ? (double)ic / (double)ip : 0; }
     if (per_instance_loss) for (int64_t i = 0; i < n_inst; i++) per_instance_loss[i] = E.loss[i];
     if (out) {
       out->instances = n_order; out->node_messages = E.node_messages; out->ppt_messages = E.ppt_messages;
-      out->rounds = r + 1; out->seconds = 0; out->mean_loss = n_order ? tot / n_order : 0;
+      out->rounds = r + 1; out->seconds = 0; out->mean_loss = n_train ? tot / n_train : 0;
       out->max_staleness = max_stale; out->max_active_observed = max_active; out->route_hash = E.route_hash;
       out->leftover_cache_entries = leftover;
     }
@@ -957,6 +974,7 @@ struct Oracle {
     E.err.clear();
     E.inbox_a.assign(E.nodes.size(), {}); E.inbox_b.assign(E.nodes.size(), {});
     E.loss.assign(n_inst, 0); E.correct.assign(n_inst, 0); E.n_pred.assign(n_inst, 0);
+    E.inflight_eval.clear();
     auto* cur = &E.inbox_a; auto* nxt = &E.inbox_b;
     for (int64_t i = 0; i < n_inst; i++) {
       E.target = cur;
@@ -1124,6 +1142,13 @@ int oracle_run_epoch(void* h, int split, int mak, int muf, double lr, const int6
                      int flush, oracle_stats_t* out, double* per_instance_loss) {
   if (mak < 1 || muf < 1) return 1;
   return static_cast<Oracle*>(h)->run_epoch(split, mak, muf, lr, order, n_order, flush, out, per_instance_loss);
+}
+
+// inf_out: {inference instances, their mean loss, their accuracy}
+int oracle_run_epoch_mixed(void* h, int split, int mak, int muf, double lr, const int64_t* order, int64_t n_order,
+                           int flush, const uint8_t* inference_only, oracle_stats_t* out, double* per_instance_loss, double* inf_out) {
+  if (mak < 1 || muf < 1) return 1;
+  return static_cast<Oracle*>(h)->run_epoch(split, mak, muf, lr, order, n_order, flush, out, per_instance_loss, inference_only, inf_out);
 }
 
 // kind: 0 SGD, 1 momentum-SGD (v <- mu v + g, theta -= lr v), 2 Adam (bias-corrected); state is kept across epochs.

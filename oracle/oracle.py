@@ -52,6 +52,8 @@ def _load(real):
     lib.oracle_run_epoch.argtypes = [P, C.c_int, C.c_int, C.c_int, C.c_double, P, C.c_int64, C.c_int,
                                      C.POINTER(OracleStats), P]
     lib.oracle_eval.argtypes = [P, C.c_int, P, P, P]
+    lib.oracle_run_epoch_mixed.argtypes = [P, C.c_int, C.c_int, C.c_int, C.c_double, P, C.c_int64, C.c_int, P,
+                                           C.POINTER(OracleStats), P, P]
     lib.oracle_set_optimizer.argtypes = [P, C.c_int, C.c_double, C.c_double, C.c_double, C.c_double, C.c_int]
     lib.oracle_get_node_stats.argtypes = [P, C.c_int, P, P, P, P, P]
     lib.oracle_get_update_log.restype = C.c_int64
@@ -131,6 +133,18 @@ class Oracle:
                                               C.byref(st), _p(loss)))
         st.seconds = time.perf_counter() - t0
         return st, loss
+
+    def run_epoch_mixed(self, mak, muf, lr, inference_only, order=None, flush=True, split=0):
+        """Training epoch in which the instances marked in inference_only (uint8 per instance) are only evaluated.
+        Returns (stats, per-instance loss, dict(instances, mean_loss, accuracy) of the inference instances)."""
+        n = self.n[split]
+        order = np.arange(n, dtype=np.int64) if order is None else np.ascontiguousarray(order, dtype=np.int64)
+        mask = np.ascontiguousarray(inference_only, dtype=np.uint8)
+        assert mask.shape == (n,)
+        st, loss, inf = OracleStats(), np.zeros(n, np.float64), np.zeros(3, np.float64)
+        self._check(self.lib.oracle_run_epoch_mixed(self.h, split, mak, muf, float(np.float32(lr)), _p(order), len(order),
+                                                    int(flush), _p(mask), C.byref(st), _p(loss), _p(inf)))
+        return st, loss, dict(instances=int(inf[0]), mean_loss=inf[1], accuracy=inf[2])
 
     def set_optimizer(self, kind="sgd", momentum=0.9, beta1=0.9, beta2=0.999, eps=1e-8, reset=True):
         k = {"sgd": 0, "momentum": 1, "adam": 2}[kind]

@@ -427,3 +427,38 @@ def test_replica_averaging_is_the_mean_and_keeps_other_nodes(oracle_mod):
     for key in before:
         if key[0] not in copies:
             np.testing.assert_array_equal(after[key], before[key])
+
+
+# ---------------------------------------------------------------------------------------------------
+# concurrent inference: instances that are only evaluated share the queues with training instances
+# ---------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("family", FAMILIES)
+def test_inference_instances_ride_along_without_touching_training(oracle_mod, family):
+    g, inst, p = H.tiny_case(family, n=7)
+    mask = np.array([0, 1, 0, 0, 1, 1, 0], np.uint8)
+    train = np.nonzero(mask == 0)[0]
+    # (a) gradients: the masked instances contribute nothing, the others exactly what they contribute alone
+    o = make(oracle_mod, g, inst, p)
+    st, loss, inf = o.run_epoch_mixed(mak=3, muf=BIG, lr=0.1, inference_only=mask, flush=False)
+    ref = make(oracle_mod, g, inst, p)
+    rst, rloss = ref.run_epoch(mak=3, muf=BIG, lr=0.1, order=train, flush=False)
+    for node in g.ppt_nodes():
+        for which, _ in g.param_shapes(node):
+            np.testing.assert_allclose(o.get_accum(node, which), ref.get_accum(node, which), rtol=1e-12, atol=1e-14)
+        assert o.node_stats(node)["bwd_msgs"] == ref.node_stats(node)["bwd_msgs"]
+    assert st.leftover_cache_entries == 0 and st.max_active_observed <= 3
+    # (b) losses: with unchanged parameters every instance's loss is its forward-only loss
+    e = make(oracle_mod, g, inst, p)
+    e.load_instances(inst, split=1)
+    ml, acc, eloss = e.eval(split=1)
+    np.testing.assert_allclose(loss, eloss, rtol=1e-12, atol=1e-14)
+    assert inf["instances"] == int(mask.sum())
+    assert inf["mean_loss"] == pytest.approx(eloss[mask == 1].mean(), rel=1e-12)
+    assert st.mean_loss == pytest.approx(eloss[mask == 0].mean(), rel=1e-12)
+    # (c) everything masked: a pure evaluation, no update anywhere
+    o2 = make(oracle_mod, g, inst, p)
+    st2, loss2, inf2 = o2.run_epoch_mixed(mak=2, muf=1, lr=0.5, inference_only=np.ones(7, np.uint8))
+    np.testing.assert_allclose(loss2, eloss, rtol=1e-12, atol=1e-14)
+    assert inf2["accuracy"] == pytest.approx(acc)
+    for k, v in o2.get_params().items():
+        np.testing.assert_array_equal(v, p[k].astype(np.float64))
