@@ -256,6 +256,14 @@ def run_ours(args):
     e2e_s = time.perf_counter() - t0
     e2e_value, _ = aggregate(inst.n * e2e_steps, e2e_s, dev)
 
+    # ---- forward-only throughput (the paper's inference column): the same instances, evaluation messages only -----
+    eng.eval(0, mak=cfg["mak"])
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    eng.eval(0, mak=cfg["mak"])
+    torch.cuda.synchronize()
+    inference_rate = inst.n / (time.perf_counter() - t0)
+
     sweep = None
     if args.sweep and rank == 0:
         # max_active_keys x min_update_frequency grid on a prefix (one epoch each, parameters reset)
@@ -309,7 +317,7 @@ def run_ours(args):
                 "clocks": clocks, "gpu_launches": args.steps,
                 "stats": {"mean_loss_last_step": last.mean_loss, "max_staleness": int(last.max_staleness),
                           "rows_per_micro_batch": last.micro_batch_rows / max(1, last.micro_batches),
-                          "placement": placement,
+                          "placement": placement, "inference_instances_per_s": inference_rate,
                           "micro_batch_split": {"fma": 1.0, "tensor_core": 0.0}}}
         if sweep is not None:
             line["sweep"] = sweep

@@ -209,6 +209,17 @@ ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_t
  * other warps, [14] closing barrier).  cycles16: 16 values.  batches: micro-batches executed.                    */
 ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles16, int64_t* batches);
 
+/* ---- concurrent inference (Sec. 1: inference can run while the model trains; Sec. 6 reports inference throughput) --------
+ * A training epoch in which the instances i with inference_only[i] != 0 (host array, one byte per loaded instance of
+ * the training split) are only evaluated: their messages carry the evaluation flag, travel through the same queues and
+ * micro-batch formation as the training messages (a micro-batch holds one kind only), cache nothing, produce no
+ * gradients and count towards no update; they occupy a key like any instance.  out->mean_loss is the mean over the
+ * training instances, *inference (may be NULL) receives count, mean loss and accuracy of the others;
+ * per_instance_loss is indexed by instance for both kinds.                                                        */
+typedef struct ampnet_inference_stats { int64_t instances; double mean_loss; double accuracy; } ampnet_inference_stats_t;
+ampnet_status_t ampnet_run_epoch_mixed(ampnet_graph_t*, const ampnet_run_cfg_t*, const uint8_t* inference_only,
+                                       ampnet_epoch_stats_t* out, float* per_instance_loss, ampnet_inference_stats_t* inference);
+
 /* ---- replicas (Sec. 5) -------------------------------------------------------------------------------------
  * A heavy node is replicated in full between a Cond (AMPNET_COND_ROUND_ROBIN) and a Phi; the copies train
  * independently and are synchronised infrequently, at the end of an epoch, by averaging.  This call replaces the

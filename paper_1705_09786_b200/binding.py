@@ -12,8 +12,12 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
+           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_mixed", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
            "ampnet_ir_tree", "ampnet_ir_ggnn"]
+
+
+class InferenceStats(C.Structure):
+    _fields_ = [("instances", C.c_int64), ("mean_loss", C.c_double), ("accuracy", C.c_double)]
 
 
 class AmpnetError(RuntimeError):
@@ -101,6 +105,7 @@ def load_library():
     lib.ampnet_ir_rnn.argtypes = [I32] * 5 + tail
     lib.ampnet_ir_rnn_replicated.argtypes = [I32] * 6 + tail
     lib.ampnet_average_params.argtypes = [P, P, C.c_int32]
+    lib.ampnet_run_epoch_mixed.argtypes = [P, P, P, P, P, P]
     lib.ampnet_ir_tree.argtypes = [I32] * 4 + tail
     lib.ampnet_ir_ggnn.argtypes = [I32] * 5 + tail
     lib.ampnet_last_error.argtypes = [P]
@@ -227,6 +232,19 @@ class Engine:
         fn = self.lib.ampnet_run_epoch_static if static_scratch else self.lib.ampnet_run_epoch
         self._check(fn(self.h, C.byref(cfg), C.byref(st), _p(loss)))
         return st, loss
+
+    def run_epoch_mixed(self, mak, muf, lr, inference_only, deterministic=False, order=None, timeout_s=0.0):
+        """A training epoch in which the instances marked in inference_only (uint8 per instance) are only evaluated.
+        Returns (stats, per-instance loss, dict(instances, mean_loss, accuracy) of the inference instances)."""
+        order = None if order is None else np.ascontiguousarray(order, dtype=np.int64)
+        mask = np.ascontiguousarray(inference_only, dtype=np.uint8)
+        if mask.shape != (self.n[0],):
+            raise ValueError("inference_only needs one entry per loaded training instance")
+        cfg = RunCfg(mak, muf, lr, int(deterministic), _p(order), 0 if order is None else len(order), timeout_s, 0, 0)
+        st, inf = EpochStats(), InferenceStats()
+        loss = np.zeros(self.n[0], np.float32)
+        self._check(self.lib.ampnet_run_epoch_mixed(self.h, C.byref(cfg), _p(mask), C.byref(st), _p(loss), C.byref(inf)))
+        return st, loss, dict(instances=inf.instances, mean_loss=inf.mean_loss, accuracy=inf.accuracy)
 
     def set_optimizer(self, kind="sgd", momentum=0.9, beta1=0.9, beta2=0.999, eps=1e-8, reset=True):
         k = {"sgd": 0, "momentum": 1, "adam": 2}[kind]

@@ -707,7 +707,8 @@ ampnet_status_t ensure_arenas(ampnet_graph* g, size_t ctl_need, size_t bulk_need
 }
 
 ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, const ampnet_run_cfg_t* cfg,
-                        ampnet_epoch_stats_t* out, float* per_instance_loss, double* accuracy) {
+                        ampnet_epoch_stats_t* out, float* per_instance_loss, double* accuracy,
+                        const uint8_t* inference_only = nullptr, ampnet_inference_stats_t* inference = nullptr) {
   HostDataset& D = g->data[split];
   if (!D.loaded) return set_err(g, AMPNET_ESTATE, "no instances loaded for split %d", split);
   if (mak < 1) return set_err(g, AMPNET_EINVAL, "max_active_keys must be >= 1");
@@ -728,7 +729,8 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   ampnet_status_t st = plan_run(g, split, mak, det, eval, cfg, n_order, true, R);
   if (st != AMPNET_OK) return st;
   const size_t order_bytes = order ? (size_t)n_order * sizeof(long long) : 0;
-  st = ensure_arenas(g, g->ctl.used, g->bulk.used + order_bytes + 512);
+  const size_t mask_bytes = inference_only ? (size_t)D.n : 0;
+  st = ensure_arenas(g, g->ctl.used, g->bulk.used + order_bytes + mask_bytes + 1024);
   if (st != AMPNET_OK) return st;
   st = plan_run(g, split, mak, det, eval, cfg, n_order, false, R);
   if (st != AMPNET_OK) return st;
@@ -736,6 +738,11 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
     long long* d_order = g->bulk.take<long long>((size_t)n_order);
     CUDA_TRY(g, cudaMemcpyAsync(d_order, order, order_bytes, cudaMemcpyHostToDevice, g->stream));
     R.ctx.order = d_order;
+  }
+  if (inference_only) {
+    unsigned char* d_mask = g->bulk.take<unsigned char>(mask_bytes);
+    CUDA_TRY(g, cudaMemcpyAsync(d_mask, inference_only, mask_bytes, cudaMemcpyHostToDevice, g->stream));
+    R.ctx.inference_only = d_mask;
   }
   if ((size_t)R.smem_bytes > (size_t)g->max_smem) return set_err(g, AMPNET_EINVAL, "tile needs %zu bytes of shared memory", R.smem_bytes);
   CUDA_TRY(g, cudaMemsetAsync(g->ctl_mem, 0, g->ctl.used, g->stream));
@@ -794,7 +801,8 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   if (out) {
     std::memset(out, 0, sizeof *out);
     out->instances = n_order; out->node_messages = (int64_t)G.node_messages; out->rounds = (int64_t)G.rounds;
-    out->seconds = ms * 1e-3; out->mean_loss = n_order ? G.total_loss / (double)n_order : 0.0;
+    out->seconds = ms * 1e-3; const long long n_train = n_order - (long long)G.inf_instances;
+    out->mean_loss = n_train > 0 ? G.total_loss / (double)n_train : 0.0;
     out->max_active_observed = G.max_active; out->route_hash = G.route_hash;
     for (auto& s : g->last_stats) {
       out->ppt_messages += (int64_t)s.msgs; out->max_staleness = std::max(out->max_staleness, s.max_staleness);
@@ -802,6 +810,11 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
     }
   }
   if (accuracy) *accuracy = G.n_pred ? (double)G.correct / (double)G.n_pred : 0.0;
+  if (inference) {
+    inference->instances = (int64_t)G.inf_instances;
+    inference->mean_loss = G.inf_instances ? G.inf_loss / (double)G.inf_instances : 0.0;
+    inference->accuracy = G.inf_pred ? (double)G.inf_correct / (double)G.inf_pred : 0.0;
+  }
   if (G.status == ST_TIMEOUT) return set_err(g, AMPNET_ETIMEOUT, "a bounded device wait gave up (node %d, detail %d)", G.err_node, G.err_detail);
   if (G.status == ST_OVERFLOW) return set_err(g, AMPNET_EOVERFLOW, "a queue / cache / key-space bound was exceeded (node %d, detail %d)", G.err_node, G.err_detail);
   if (G.status != 0) return set_err(g, AMPNET_ECUDA, "device status %d", G.status);
@@ -1074,6 +1087,13 @@ ampnet_status_t ampnet_run_epoch(ampnet_graph_t* g, const ampnet_run_cfg_t* cfg,
   if (!g) return AMPNET_EINVAL;
   if (!cfg) return set_err(g, AMPNET_EINVAL, "NULL run configuration");
   return execute(g, 0, cfg->max_active_keys, cfg->deterministic ? 1 : 0, 0, cfg, out, per_instance_loss, nullptr);
+}
+
+ampnet_status_t ampnet_run_epoch_mixed(ampnet_graph_t* g, const ampnet_run_cfg_t* cfg, const uint8_t* inference_only,
+                                       ampnet_epoch_stats_t* out, float* per_instance_loss, ampnet_inference_stats_t* inference) {
+  if (!g) return AMPNET_EINVAL;
+  if (!cfg || !inference_only) return set_err(g, AMPNET_EINVAL, "NULL run configuration or mask");
+  return execute(g, 0, cfg->max_active_keys, cfg->deterministic ? 1 : 0, 0, cfg, out, per_instance_loss, nullptr, inference_only, inference);
 }
 
 ampnet_status_t ampnet_eval(ampnet_graph_t* g, int32_t split, int32_t max_active_keys, double* mean_loss,

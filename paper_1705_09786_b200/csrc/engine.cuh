@@ -888,12 +888,14 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
   }
   const int rows0 = cum[0];
   scan64(cum, lane);
-  const bool ok0 = lane < ncand && cum[0] <= P.BM, ok1 = lane + 32 < ncand && cum[1] <= P.BM;
+  // a batch is all training or all forward-only messages (concurrent inference): cut where the flag changes
+  const int eval0 = __shfl_sync(0xffffffffu, (int)((h[0].flags & HDR_EVAL) != 0), 0);
+  const bool ok0 = lane < ncand && cum[0] <= P.BM && (int)((h[0].flags & HDR_EVAL) != 0) == eval0,
+             ok1 = lane + 32 < ncand && cum[1] <= P.BM && (int)((h[1].flags & HDR_EVAL) != 0) == eval0;
   const unsigned long long okm = ballot64(ok0, ok1);
   int take = okm == ~0ull ? 64 : __ffsll((long long)~okm) - 1;
   if (take == 0) { fail(C, ST_OVERFLOW, P.node, rows0); return 0; }     // a single message larger than a batch
   bool upd = false;
-  const int eval0 = __shfl_sync(0xffffffffu, (int)((h[0].flags & HDR_EVAL) != 0), 0);
   if (dir == BWD && !eval0) {
     const int muf = node_muf(C, P);
     const unsigned long long tm = ballot64(ok0 && lane < take && S.ls.n_acc + cum[0] >= muf,
@@ -1904,7 +1906,7 @@ struct CtrlShared {
   long long next, retired;
   int active;
   unsigned retire_head;
-  int admit_slot, admit_inst, admit_seq, n_src_msgs;
+  int admit_slot, admit_inst, admit_seq, n_src_msgs, admit_eval;
   int src_count[4], src_base[5];
   unsigned long long prof[8];
   unsigned occ[OCC_SLOTS / 32];          // occupied key slots (slots beyond OCC_SLOTS are found by scanning slot_inst)
@@ -1957,7 +1959,8 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
           for (int o = 16; o; o >>= 1) { okc += __shfl_xor_sync(0xffffffffu, okc, o); np += __shfl_xor_sync(0xffffffffu, np, o); }
           if (lane == 0) {
             C.loss_out[inst] = (float)tot;
-            C.g->total_loss += tot; C.g->correct += okc; C.g->n_pred += np;
+            if (C.inference_only && C.inference_only[inst]) { C.g->inf_loss += tot; C.g->inf_instances += 1; C.g->inf_correct += okc; C.g->inf_pred += np; }
+            else { C.g->total_loss += tot; C.g->correct += okc; C.g->n_pred += np; }
             C.slot_inst[slot] = -1;
             if (slot < OCC_SLOTS) S.occ[slot >> 5] &= ~(1u << (slot & 31));
             S.active--; S.retired++;
@@ -1996,7 +1999,8 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
           }
           S.src_base[C.n_sources] = total;
           S.n_src_msgs = total;
-          if (C.eval) {      // forward only: the instance is finished when every Loss / Sink has been reached
+          S.admit_eval = C.eval || (C.inference_only && C.inference_only[inst]);
+          if (S.admit_eval) {      // forward only: the instance is finished when every Loss / Sink has been reached
             int exp = 1;
             if (I.kind == 2) exp = (int)(I.offsets[inst + 1] - I.offsets[inst]) + 1;
             C.outstanding[slot] = exp;
@@ -2048,7 +2052,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
             const unsigned q = tk & P.ring[FWD].mask;
             int4* d = reinterpret_cast<int4*>(&P.ring[FWD].e[q]);
             d[0] = make_int4(inst, S.admit_seq, slot, 0);
-            d[1] = make_int4(u, 0, 1, C.eval ? HDR_EVAL : 0);
+            d[1] = make_int4(u, 0, 1, S.admit_eval ? HDR_EVAL : 0);
             st_rel(&P.ring[FWD].seq[q], tk + 1u);
           }
           const int n_here = min(32, cnt - c0);
@@ -2065,7 +2069,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
         Frame f;
         f.node = sn.succ_node[0]; f.aport = sn.succ_port[0]; f.dir = FWD; f.iter = 0;
         f.inst = inst; f.seq = S.admit_seq; f.slot = slot; f.it = 0; f.u = 0; f.port = 0; f.rows = 1;
-        f.flags = C.eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr; f.nsum = 1; f.sstride = 0; f.part = 0; f.nparts = 1;
+        f.flags = S.admit_eval ? HDR_EVAL : 0; f.dim = 0; f.ld = 0; f.p = nullptr; f.nsum = 1; f.sstride = 0; f.part = 0; f.nparts = 1;
         f.ibase = I.offsets ? I.offsets[inst] : 0; f.ebase = I.edge_off ? I.edge_off[inst] : 0;
         switch (sn.fn) {
           case 1: f.p = I.dense + (long long)inst * I.dense_dim; f.dim = I.dense_dim; f.ld = I.dense_dim; break;

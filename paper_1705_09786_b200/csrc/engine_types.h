@@ -136,6 +136,7 @@ struct Globals {                      // mutable run state in device memory (zer
   long long max_active;
   unsigned long long correct, n_pred;
   double total_loss;
+  double inf_loss; unsigned long long inf_instances, inf_correct, inf_pred;   // instances that were only evaluated (concurrent inference)
   long long n_keylog;
   unsigned retire_tail;
   int err_node, err_detail;
@@ -162,6 +163,7 @@ struct Ctx {
   KeyLog* keylog;
   unsigned* retire_e; unsigned* retire_seq; unsigned retire_mask;
   const long long* order; long long n_order;
+  const unsigned char* inference_only;  // per instance: only evaluated while the others train (may be null)
   float* loss_out;
   // configuration
   int mak, muf, det, eval, IT;

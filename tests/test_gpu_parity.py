@@ -113,6 +113,37 @@ def test_replicated_linear_with_end_of_epoch_averaging(oracle_mod, k, mak, muf):
     e.close()
 
 
+@pytest.mark.parametrize("family,n,mak,muf,lr", [("tree", 30, 6, 7, 0.01), ("ggnn", 24, 9, 40, 0.003), ("rnn", 60, 5, 3, 0.02),
+                                                ("mlp", 40, 4, 8, 0.01)])
+def test_concurrent_inference_matches_oracle(oracle_mod, family, n, mak, muf, lr):
+    """A third of the instances are only evaluated while the others train, in the same queues (deterministic schedule:
+    bookkeeping bit-exact, floats within the usual tolerances), then the same in the free-running schedule."""
+    import paper_1705_09786_b200 as amp
+    g, inst = _case(family, n)
+    p = wp.init_params(g)
+    mask = (np.arange(inst.n) % 3 == 1).astype(np.uint8)
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst)
+    o.set_params(p)
+    ost, oloss, oinf = o.run_epoch_mixed(mak=mak, muf=muf, lr=lr, inference_only=mask)
+    e = amp.Engine(g)
+    e.load_instances(inst)
+    e.set_params(p)
+    est, eloss, einf = e.run_epoch_mixed(mak=mak, muf=muf, lr=lr, inference_only=mask, deterministic=True, timeout_s=60)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    assert einf["instances"] == oinf["instances"] == int(mask.sum())
+    assert einf["mean_loss"] == pytest.approx(oinf["mean_loss"], rel=1e-5, abs=2e-6)
+    assert einf["accuracy"] == pytest.approx(oinf["accuracy"], abs=1e-12)
+    assert est.mean_loss == pytest.approx(ost.mean_loss, rel=1e-5, abs=2e-6)
+    # free-running: the training instances' gradients are applied exactly once, the others contribute none
+    st, loss, inf = e.run_epoch_mixed(mak=mak, muf=muf, lr=lr, inference_only=mask, deterministic=False, timeout_s=60)
+    want = parity_counts(g, inst.subset(np.nonzero(mask == 0)[0]))
+    for node, G in want["grads"].items():
+        assert e.node_stats(node)["n_grads_applied"] == G
+    assert inf["instances"] == int(mask.sum()) and np.isfinite(loss).all() and e.leftover_cache_entries() == 0
+    e.close()
+
+
 def test_partial_epoch_and_degenerate_sizes(oracle_mod):
     """One instance; mak larger than the instance count; a prefix of the data; the smallest structures."""
     g, inst = _case("rnn", 9)
