@@ -49,6 +49,7 @@ struct HostPPT {
   size_t nW = 0, nb = 0;
   int T = 1, R = 0, BM = 0, J = 0;
   int NE = 0, G = 1;                    // emitter CTAs of the node and their batch groups
+  bool a_global = false;                // the tiles' gradient accumulators live in device memory (frees shared memory for staging rows)
   double emit_load = 0.0;               // emitter-seconds the node's emission took in the last asynchronous epoch (0: unknown)
   size_t smem_floats = 0;
 };
@@ -366,11 +367,11 @@ unsigned pow2_at_least(unsigned long long v) {
   return p;
 }
 
-size_t tile_smem_floats(const HostPPT& P, int R, int BM) {      // mirrors the carve-up at the top of ppt_main
+size_t tile_smem_floats(const HostPPT& P, int R, int BM, bool a_global = false) {      // mirrors the carve-up at the top of ppt_main
   if (P.kind == LOOKUP) return 64;
   const size_t LW = (size_t)pad_ldw(P.in), LX = (size_t)pad_ldx(P.in), RP = (size_t)((R + 3) & ~3), nm = (size_t)P.nmat;
   auto p4 = [](size_t v) { return (v + 3) & ~(size_t)3; };
-  return 2 * nm * R * LW + 2 * p4(nm * R) + (size_t)BM * LX * (P.kind == GRUCELL ? 2 : 1) + (nm + 1) * BM * RP + p4(nm * BM * R) +
+  return (a_global ? 1 : 2) * nm * R * LW + 2 * p4(nm * R) + (size_t)BM * LX * (P.kind == GRUCELL ? 2 : 1) + (nm + 1) * BM * RP + p4(nm * BM * R) +
          XWT_SCRATCH + 64;
 }
 
@@ -393,7 +394,7 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
     for (int t = t_from; t <= std::min(MAX_TILES, P.out); t++) {
       const int R = (P.out + t - 1) / t;
       if ((P.out + R - 1) / R < t_from) continue;
-      if (tile_smem_floats(P, R, bm) <= budget) { t_out = (P.out + R - 1) / R; return true; }
+      if (tile_smem_floats(P, R, bm, P.a_global) <= budget) { t_out = (P.out + R - 1) / R; return true; }
     }
     return false;
   };
@@ -416,10 +417,22 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
     // Keep the micro-batch capacity if more row tiles make the tile fit; only then shrink the capacity.
     const int bm_min = std::max(rows_max, 4);
     bool placed = false;
+    P.a_global = false;
     for (int bm = BM; !placed; bm = std::max(bm_min, bm / 2)) {
       int t = 0;
       if (fit(P, 1, bm, t)) { P.T = t; bm_of[p] = bm; placed = true; break; }
       if (bm == bm_min) return set_err(g, AMPNET_EINVAL, "node %d does not fit in shared memory with %d row tiles", P.node, MAX_TILES);
+    }
+    // A node so wide that fewer than 32 rows can be staged beside its weight and accumulator tiles keeps the accumulators
+    // in device memory instead (read and written once per backward batch) if that buys a larger micro-batch.
+    if (bm_of[p] < 32 && bm_of[p] < BM) {
+      P.a_global = true;
+      bool better = false;
+      for (int bm = BM; bm > bm_of[p]; bm /= 2) {
+        int t = 0;
+        if (fit(P, 1, bm, t)) { P.T = t; bm_of[p] = bm; better = true; break; }
+      }
+      if (!better) P.a_global = false;
     }
     // a node with a handful of output rows (a classifier) may still have a tile per row; others keep 4 rows per tile
     limit[p] = std::max(P.T, std::min(max_tiles, P.out <= 16 ? P.out : std::max(1, P.out / 4)));
@@ -445,7 +458,7 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
     if (P.kind != LOOKUP) { P.R = (P.out + P.T - 1) / P.T; P.T = (P.out + P.R - 1) / P.R; P.BM = bm_of[p]; }
-    P.smem_floats = tile_smem_floats(P, P.R, P.BM);
+    P.smem_floats = tile_smem_floats(P, P.R, P.BM, P.a_global);
     used += P.T;
   }
   if (used > n_ctas) return set_err(g, AMPNET_EINVAL, "placement needs %d CTAs but only %d are available", used, n_ctas);
@@ -582,6 +595,8 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.nbar = C.take<unsigned>(1);
     P.stats = C.take<PPTStats>(1);
     P.update_log = B.take<int>(g->update_log_cap); P.update_log_cap = g->update_log_cap;
+    P.a_global = H.a_global ? 1 : 0;
+    if (H.a_global) P.A = C.take<float>((size_t)H.T * H.nmat * H.R * pad_ldw(H.in));
     if (H.kind == LOOKUP) {
       P.A = C.take<float>(H.nW);
       P.touched_flag = C.take<int>(H.in);

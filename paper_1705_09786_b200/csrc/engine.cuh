@@ -1492,7 +1492,8 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
     M.LW = pad_ldw(in); M.LX = pad_ldx(in); M.RP = (P.R + 3) & ~3;
     float* p = smem;                                 // every array starts on a 16-byte boundary
     M.Ws = p; p += (size_t)nmat * P.R * M.LW;
-    M.As = p; p += (size_t)nmat * P.R * M.LW;
+    if (P.a_global) M.As = P.A + (size_t)tile * nmat * P.R * M.LW;       // zeroed with the run state
+    else { M.As = p; p += (size_t)nmat * P.R * M.LW; }
     M.bs = p; p += (nmat * P.R + 3) & ~3;
     M.Abs = p; p += (nmat * P.R + 3) & ~3;
     M.Xs = p; p += (size_t)P.BM * M.LX;

@@ -81,7 +81,9 @@ struct DevPPT {
   float *om, *ov;                     // optimiser state (first / second moment), laid out like W followed by b
   long long opt_t0;                   // updates of this node before the run (Adam's bias correction)
   float *W, *b;                       // LINEAR: W[out][in], b[out]; LOOKUP: W = E[V][d]; GRUCELL: W[3][H][2H], b[3][H]
-  float* A;                           // LOOKUP: accumulator [V][d] in device memory
+  float* A;                           // LOOKUP: accumulator [V][d] in device memory; a node whose tiles keep their accumulators in
+                                      // device memory (a_global): [tile][nmat][R][ldw]
+  int a_global, pad2;
   int *touched_flag, *touched_list, *touched_n;
   float *xcache, *ycache, *gbuf;      // [key][rows_max][in | out | out]
   float *zc, *rc, *cc;                // GRUCELL caches [key][rows_max][H]

@@ -144,6 +144,18 @@ def test_concurrent_inference_matches_oracle(oracle_mod, family, n, mak, muf, lr
     e.close()
 
 
+def test_wide_cells_that_keep_their_accumulators_in_device_memory(oracle_mod):
+    """Hidden size 512 (the stress configuration's cells): the branch cell's tiles cannot stage 32 rows beside weights and
+    accumulators, so placement moves the accumulators to device memory.  Same parity bar."""
+    g = ir.tree(vocab=300, emb=512, hidden=512, classes=5)
+    inst = data.tree_instances(n=10, min_leaves=3, max_leaves=12, vocab=300)
+    p = wp.init_params(g)
+    r = parity.run_both(oracle_mod, g, inst, p, 4, 9, 0.01)
+    parity.assert_parity(g, *r)
+    assert r[3].placement(g.index("branch_cell"))[1] < 64        # the reduced staging capacity that triggers the path
+    r[3].close()
+
+
 def test_partial_epoch_and_degenerate_sizes(oracle_mod):
     """One instance; mak larger than the instance count; a prefix of the data; the smallest structures."""
     g, inst = _case("rnn", 9)
