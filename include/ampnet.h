@@ -185,6 +185,10 @@ ampnet_status_t ampnet_eval(ampnet_graph_t*, int32_t split, int32_t max_active_k
 ampnet_status_t ampnet_param_count(ampnet_graph_t*, int32_t node, int32_t which, int64_t* n);
 ampnet_status_t ampnet_get_params(ampnet_graph_t*, int32_t node, int32_t which, float* dst_host, int64_t n);
 ampnet_status_t ampnet_set_params(ampnet_graph_t*, int32_t node, int32_t which, const float* src_host, int64_t n);
+/* Device address of the same array (*n floats), owned by the handle and valid until it is destroyed.  Between two
+ * epochs the caller may read or write it on the handle's stream or after synchronising with it: this is how replicas of
+ * the whole model on several GPUs are averaged in place at the end of an epoch (Sec. 5) by a collective library.     */
+ampnet_status_t ampnet_param_device_ptr(ampnet_graph_t*, int32_t node, int32_t which, float** dev, int64_t* n);
 
 /* Statistics of the last run.  staleness_hist: 64 bins (updates between a gradient's forward and backward).
  * fwd_msgs / bwd_msgs (messages consumed by the node) and the route fingerprint are collected in the

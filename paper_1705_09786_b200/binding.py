@@ -12,7 +12,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_mixed", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
+           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_mixed", "ampnet_param_device_ptr", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
            "ampnet_ir_tree", "ampnet_ir_ggnn"]
 
 
@@ -106,6 +106,7 @@ def load_library():
     lib.ampnet_ir_rnn_replicated.argtypes = [I32] * 6 + tail
     lib.ampnet_average_params.argtypes = [P, P, C.c_int32]
     lib.ampnet_run_epoch_mixed.argtypes = [P, P, P, P, P, P]
+    lib.ampnet_param_device_ptr.argtypes = [P, C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64)]
     lib.ampnet_ir_tree.argtypes = [I32] * 4 + tail
     lib.ampnet_ir_ggnn.argtypes = [I32] * 5 + tail
     lib.ampnet_last_error.argtypes = [P]
@@ -218,6 +219,22 @@ class Engine:
         a = np.empty(n.value, np.float32)
         self._check(self.lib.ampnet_get_params(self.h, node, which, _p(a), n.value))
         return a.reshape(dict(self.graph.param_shapes(node))[which])
+
+    def param_tensors(self):
+        """{(node, which): torch tensor} aliasing the parameter arrays in device memory (no copies)."""
+        import torch
+
+        class _View:                          # what torch.as_tensor needs to wrap a raw device pointer
+            def __init__(self, ptr, n):
+                self.__cuda_array_interface__ = {"shape": (n,), "typestr": "<f4", "data": (ptr, False), "version": 2}
+
+        out = {}
+        for i in self.graph.ppt_nodes():
+            for w, shape in self.graph.param_shapes(i):
+                ptr, n = C.c_void_p(), C.c_int64()
+                self._check(self.lib.ampnet_param_device_ptr(self.h, i, w, C.byref(ptr), C.byref(n)))
+                out[(i, w)] = torch.as_tensor(_View(ptr.value, n.value), device=self.device).view(*shape)
+        return out
 
     def run_epoch(self, mak, muf, lr, deterministic=False, order=None, timeout_s=0.0, max_batch_rows=0, n_ctas=0,
                   want_loss=True, static_scratch=False):

@@ -1157,6 +1157,15 @@ ampnet_status_t ampnet_get_params(ampnet_graph_t* g, int32_t node, int32_t which
   CUDA_TRY(g, cudaStreamSynchronize(g->stream));
   return AMPNET_OK;
 }
+ampnet_status_t ampnet_param_device_ptr(ampnet_graph_t* g, int32_t node, int32_t which, float** dev, int64_t* n) {
+  HostPPT* P = find_ppt(g, node);
+  float* b; size_t c;
+  if (!P || !dev || !param_slice(*P, which, &b, &c)) return g ? set_err(g, AMPNET_EINVAL, "no parameter (%d, %d)", node, which) : AMPNET_EINVAL;
+  CUDA_TRY(g, cudaStreamSynchronize(g->stream));
+  *dev = b;
+  if (n) *n = (int64_t)c;
+  return AMPNET_OK;
+}
 ampnet_status_t ampnet_set_params(ampnet_graph_t* g, int32_t node, int32_t which, const float* src, int64_t n) {
   HostPPT* P = find_ppt(g, node);
   float* b; size_t c;

@@ -65,6 +65,12 @@ def _worker(rank, world, port, q):
     _, inst, _ = bench.make_workload("rnn", rank, n=50)          # every rank draws its own shard
     bench.barrier()
     value, tmax = bench.aggregate(units_this_rank=100 * (rank + 1), seconds_this_rank=1.0 + rank)
+    # end-of-epoch averaging of the replicas' parameters (Sec. 5): rank r holds r + 1 and 10 (r + 1)
+    import torch
+    from paper_1705_09786_b200.replicas import average_across_ranks
+    params = [torch.full((3, 2), float(rank + 1)), torch.full((5,), 10.0 * (rank + 1))]
+    n = average_across_ranks(params)
+    assert n == world and torch.all(params[0] == 1.5) and torch.all(params[1] == 15.0)
     q.put((rank, value, tmax, int(inst.tokens[:64].sum())))
     import torch.distributed as dist
     dist.destroy_process_group()

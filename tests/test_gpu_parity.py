@@ -4,6 +4,8 @@ Bar: routing multiset, key log, update counts and gradient counts bit-exact in t
 parameters within max relative error 1e-4, per-instance losses within 1e-5 (relative, with an absolute
 floor of 2e-6 for losses near zero: fp32 log-sum-exp has ~1e-7 absolute error per term).
 """
+import os
+
 import numpy as np
 import pytest
 
@@ -154,6 +156,39 @@ def test_wide_cells_that_keep_their_accumulators_in_device_memory(oracle_mod):
     parity.assert_parity(g, *r)
     assert r[3].placement(g.index("branch_cell"))[1] < 64        # the reduced staging capacity that triggers the path
     r[3].close()
+
+
+def test_parameter_tensors_alias_device_memory_for_replica_averaging():
+    """engine.param_tensors() are views of the arrays the engine trains (no copies), which is what lets a collective
+    library average whole-model replicas in place; a single-rank NCCL group exercises the call path."""
+    import torch
+    import torch.distributed as dist
+    import paper_1705_09786_b200 as amp
+    from paper_1705_09786_b200.replicas import average_across_ranks
+    g = ir.mlp((12, 9, 4))
+    e = amp.Engine(g)
+    p = wp.init_params(g)
+    e.set_params(p)
+    views = e.param_tensors()
+    for k, v in p.items():
+        np.testing.assert_array_equal(views[k].cpu().numpy(), v.astype(np.float32))
+    k0 = (g.ppt_nodes()[0], 0)
+    views[k0].mul_(2.0)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(e.get_params(*k0), 2 * p[k0].astype(np.float32))
+    assert average_across_ranks(list(views.values())) == 1            # no process group: nothing to do
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT="29533")
+    dist.init_process_group("nccl", rank=0, world_size=1)
+    try:
+        before = {k: v.clone() for k, v in views.items()}
+        assert average_across_ranks(list(views.values())) == 1
+        t = views[k0]
+        dist.all_reduce(t)                                               # the collective runs on the aliased memory
+        torch.cuda.synchronize()
+        assert torch.equal(t, before[k0])
+    finally:
+        dist.destroy_process_group()
+    e.close()
 
 
 def test_partial_epoch_and_degenerate_sizes(oracle_mod):
