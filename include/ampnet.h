@@ -53,7 +53,7 @@ enum {
   AMPNET_PHI = 8,         /* join: records the origin keyed on the state, backpropagates to it           */
   AMPNET_ISU = 9,         /* invertible state update (fn = AMPNET_ISU_*)                                 */
   AMPNET_CONCAT = 10,     /* fn_arg ports of width in_dim -> one payload of width out_dim                */
-  AMPNET_SPLIT = 11,      /* inverse of CONCAT (declared; not executed by the device engine yet)         */
+  AMPNET_SPLIT = 11,      /* inverse of CONCAT: fn_arg successors, successor k gets columns [k w, (k+1) w) */
   AMPNET_BCAST = 12,      /* same payload to fn_arg successors; backward = sum in successor order        */
   AMPNET_GROUP = 13,      /* collect messages by state into one matrix payload (fn = AMPNET_GROUP_*)     */
   AMPNET_UNGROUP = 14,    /* one message per row (fn = AMPNET_UNGROUP_*)                                 */

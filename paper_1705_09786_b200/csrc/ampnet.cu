@@ -180,7 +180,6 @@ ampnet_status_t build_topology(ampnet_graph* g) {
   for (int i = 0; i < n; i++) {
     const auto& d = g->nodes[i];
     if (d.type < 0 || d.type >= N_NODE_TYPES) return set_err(g, AMPNET_EINVAL, "node %d: unknown type %d", i, d.type);
-    if (d.type == SPLIT) return set_err(g, AMPNET_EINVAL, "node %d: SPLIT is not executed by the device engine", i);
     if (d.in_dim < 0 || d.out_dim < 0) return set_err(g, AMPNET_EINVAL, "node %d: negative dimension", i);
     DevNode& h = g->hnodes[i];
     h.type = d.type; h.in_dim = d.in_dim; h.out_dim = d.out_dim; h.act = d.act; h.fn = d.fn; h.fn_arg = d.fn_arg;
@@ -242,6 +241,10 @@ ampnet_status_t build_topology(ampnet_graph* g) {
                   ((h.fn == 1 && h.n_pred == h.fn_arg) || (h.fn == 2 && h.n_pred == 1)), "CONCAT ports / widths inconsistent");
         break;
       case BCAST: st = need(h.n_pred == 1 && h.fn_arg >= 1 && h.n_succ == h.fn_arg, "BCAST needs fn_arg successors"); break;
+      case SPLIT:
+        st = need(h.n_pred == 1 && h.fn_arg >= 1 && h.fn_arg <= MAX_PORTS && h.n_succ == h.fn_arg && h.in_dim == h.fn_arg * h.out_dim,
+                  "SPLIT needs fn_arg successors of width in_dim / fn_arg");
+        break;
       case GROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 3, "GROUP needs a valid fn"); break;
       case UNGROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 2, "UNGROUP needs a valid fn"); break;
       case FLATMAP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn == 1, "FLATMAP needs a valid fn"); break;
@@ -255,7 +258,7 @@ ampnet_status_t build_topology(ampnet_graph* g) {
   if (g->losses.empty() || g->losses.size() > 4) return set_err(g, AMPNET_EINVAL, "the graph needs 1..4 LOSS nodes");
   // widths along the edges
   auto out_width = [&](const DevNode& h) {
-    if (h.type == LINEAR || h.type == LOOKUP || h.type == GRUCELL || h.type == CONCAT) return h.out_dim;
+    if (h.type == LINEAR || h.type == LOOKUP || h.type == GRUCELL || h.type == CONCAT || h.type == SPLIT) return h.out_dim;
     if (h.type == SOURCE) return (h.fn == 1 || h.fn == 3) ? h.out_dim : 0;
     return h.in_dim;
   };
@@ -624,6 +627,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
         n.jcnt = C.take<int>(kout); track(n.jcnt, kout * sizeof(int));
         break;
       case UNGROUP:
+      case SPLIT:            // the backward join of the parts' gradients
         n.jstride = (long long)n.rows_in * n.in_dim;
         n.jbuf = B.take<float>(kin * n.jstride);
         n.jcnt = C.take<int>(kin); track(n.jcnt, kin * sizeof(int));

@@ -286,7 +286,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
     const bool shadow = f.nparts > 1 && f.part > 0;
     const bool dies_as_shadow = shadow && !(n.type == COND || n.type == PHI || n.type == ISU) && (n.type == LINEAR || n.type == LOOKUP || n.type == GRUCELL || n.type == LOSS_CE ||
                                            n.type == LOSS_MSE || n.type == SINK || n.type == SOURCE || n.type == NPT_SUMROWS ||
-                                           (n.type == BCAST && f.dir == BWD) || (n.type == CONCAT && f.dir == FWD) ||
+                                           (n.type == BCAST && f.dir == BWD) || (n.type == CONCAT && f.dir == FWD) || (n.type == SPLIT && f.dir == BWD) ||
                                            (n.type == GROUP && f.dir == FWD) || (n.type == UNGROUP && f.dir == BWD) ||
                                            (n.type == FLATMAP && f.dir == BWD));
     if (dies_as_shadow) {
@@ -452,6 +452,29 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             f.p = f.p ? f.p + k * n.in_dim : nullptr; f.dim = n.in_dim;
             if (n.fn == 2) { f.port = k; to_pred(f, n, 0); } else to_pred(f, n, k);
             cont = true;
+          }
+          break;
+        case SPLIT:                               // inverse of Concat: successor k gets the columns [k w, (k + 1) w)
+          if (f.dir == FWD) {
+            const int k = f.iter;
+            if (k + 1 < n.fn_arg) { Frame c = f; c.iter = k + 1;
+              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                             if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
+            f.p = f.p ? f.p + k * n.out_dim : nullptr; f.dim = n.out_dim;
+            to_succ(f, n, k);
+            cont = true;
+          } else {                                // the parts' gradients meet again, keyed on the state
+            const int port = f.aport;
+            long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
+            if (key < 0) return;
+            if ((unsigned)port >= (unsigned)n.fn_arg || f.rows > n.rows_in) { fail(C, ST_OVERFLOW, f.node, port); return; }
+            float* base = n.jbuf + key * n.jstride;
+            warp_copy(base + port * n.out_dim, n.in_dim, f, f.rows, n.out_dim, lane);
+            if (join_arrive(&n.jcnt[key], n.fn_arg, lane)) {
+              f.p = base; f.nsum = 1; f.dim = n.in_dim; f.ld = n.in_dim;
+              to_pred(f, n, 0);
+              cont = true;
+            }
           }
           break;
         case GROUP:

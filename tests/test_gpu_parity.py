@@ -191,6 +191,40 @@ def test_parameter_tensors_alias_device_memory_for_replica_averaging():
     e.close()
 
 
+def _split_graph():
+    """Dense rows -> Linear(12 -> 8, tanh) -> Split into two halves -> two classifiers with a loss each."""
+    g = ir.IRGraph("split_heads")
+    src = g.node("src", ir.SOURCE, out_dim=12, fn=ir.SRC_DENSE_ROW)
+    l1 = g.node("linear1", ir.LINEAR, 12, 8, act=ir.ACT_TANH, flags=ir.FLAG_SOURCE_ADJACENT)
+    sp = g.node("split", ir.SPLIT, 8, 4, fn_arg=2)
+    heads = []
+    for k in range(2):
+        h = g.node(f"head{k}", ir.LINEAR, 4, 3)
+        ls = g.node(f"loss{k}", ir.LOSS_CE, 3, 0, fn=ir.LABEL_PER_INSTANCE)
+        heads.append((h, ls))
+    g.edge(src, l1)
+    g.edge(l1, sp)
+    for k, (h, ls) in enumerate(heads):
+        g.edge(sp, h, k, 0)
+        g.edge(h, ls)
+    return g
+
+
+@pytest.mark.parametrize("mak,muf", [(1, 1), (5, 4)])
+def test_split_node_matches_oracle(oracle_mod, mak, muf):
+    """Split (inverse of Concat): forward slices of the payload to several successors, backward join of their gradients."""
+    g = _split_graph()
+    inst = data.mlp_instances(n=37, dim=12, classes=3)
+    p = wp.init_params(g)
+    r = parity.run_both(oracle_mod, g, inst, p, mak, muf, 0.02)
+    parity.assert_parity(g, *r)
+    e = r[3]
+    st, loss = e.run_epoch(mak=mak, muf=muf, lr=0.02, deterministic=False, timeout_s=60)
+    assert e.leftover_cache_entries() == 0 and np.isfinite(loss).all()
+    assert e.node_stats(g.index("linear1"))["n_grads_applied"] == inst.n
+    e.close()
+
+
 def test_partial_epoch_and_degenerate_sizes(oracle_mod):
     """One instance; mak larger than the instance count; a prefix of the data; the smallest structures."""
     g, inst = _case("rnn", 9)

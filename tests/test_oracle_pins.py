@@ -462,3 +462,42 @@ def test_inference_instances_ride_along_without_touching_training(oracle_mod, fa
     assert inf2["accuracy"] == pytest.approx(acc)
     for k, v in o2.get_params().items():
         np.testing.assert_array_equal(v, p[k].astype(np.float64))
+
+
+# ---------------------------------------------------------------------------------------------------
+# Split (inverse of Concat): slices forward, joins the parts' gradients backward
+# ---------------------------------------------------------------------------------------------------
+def test_split_gradients_equal_autograd(oracle_mod):
+    import torch
+    g = ir.IRGraph("split_heads")
+    src = g.node("src", ir.SOURCE, out_dim=6, fn=ir.SRC_DENSE_ROW)
+    l1 = g.node("linear1", ir.LINEAR, 6, 8, act=ir.ACT_TANH, flags=ir.FLAG_SOURCE_ADJACENT)
+    sp = g.node("split", ir.SPLIT, 8, 4, fn_arg=2)
+    g.edge(src, l1)
+    g.edge(l1, sp)
+    heads = []
+    for k in range(2):
+        h = g.node(f"head{k}", ir.LINEAR, 4, 3)
+        ls = g.node(f"loss{k}", ir.LOSS_CE, 3, 0, fn=ir.LABEL_PER_INSTANCE)
+        g.edge(sp, h, k, 0)
+        g.edge(h, ls)
+        heads.append(h)
+    inst = data.mlp_instances(n=5, dim=6, classes=3)
+    p = wp.init_params(g)
+    o = make(oracle_mod, g, inst, p)
+    st, loss = o.run_epoch(mak=2, muf=BIG, lr=0.1, flush=False)
+    P = {k: torch.tensor(v, dtype=torch.float64, requires_grad=True) for k, v in p.items()}
+    total = 0
+    for i in range(inst.n):
+        x = torch.tensor(inst.dense[i], dtype=torch.float64)
+        hid = torch.tanh(P[(l1, 0)] @ x + P[(l1, 1)])
+        li = 0
+        for k, h in enumerate(heads):
+            y = P[(h, 0)] @ hid[4 * k:4 * k + 4] + P[(h, 1)]
+            li = li + torch.logsumexp(y, 0) - y[int(inst.labels_i[i])]
+        assert float(li) == pytest.approx(loss[i], rel=1e-12)
+        total = total + li
+    total.backward()
+    for k, v in P.items():
+        np.testing.assert_allclose(o.get_accum(*k), v.grad.numpy(), rtol=1e-9, atol=1e-12)
+    assert st.leftover_cache_entries == 0
