@@ -370,6 +370,27 @@ def test_full_size_epoch_in_the_timed_configuration(oracle_mod, family, n, mak, 
     e.close()
 
 
+@pytest.mark.parametrize("family,n,mak,muf", [("tree", 200, 32, 50), ("ggnn", 150, 32, 50)])
+def test_reduced_cta_budgets_keep_the_accounting_exact(family, n, mak, muf):
+    """Fewer CTAs than SMs (n_ctas): placement falls back to fewer tiles, one emitter per tile, and finally tiles that
+    emit their own batches; every fallback still applies every gradient exactly once."""
+    import paper_1705_09786_b200 as amp
+    g, inst = _case(family, n)
+    want = parity_counts(g, inst)
+    shapes = set()
+    for n_ctas in (100, 60, 36, 20):
+        e = amp.Engine(g)
+        e.load_instances(inst)
+        e.set_params(wp.init_params(g))
+        st, loss = e.run_epoch(mak=mak, muf=muf, lr=0.01, deterministic=False, timeout_s=60, n_ctas=n_ctas)
+        assert st.node_messages == want["node_messages"] and e.leftover_cache_entries() == 0 and np.isfinite(loss).all()
+        for node, G in want["grads"].items():
+            assert e.node_stats(node)["n_grads_applied"] == G
+        shapes.add(tuple(e.placement(i)[0] for i in g.ppt_nodes()))
+        e.close()
+    assert len(shapes) >= 2          # the budgets really produced different placements
+
+
 def parity_counts(g, inst):
     if g.name == "mlp":
         return dict(node_messages=7 * inst.n, grads={n: inst.n for n in g.ppt_nodes()})
