@@ -495,7 +495,7 @@ def test_split_gradients_equal_autograd(oracle_mod):
         for k, h in enumerate(heads):
             y = P[(h, 0)] @ hid[4 * k:4 * k + 4] + P[(h, 1)]
             li = li + torch.logsumexp(y, 0) - y[int(inst.labels_i[i])]
-        assert float(li) == pytest.approx(loss[i], rel=1e-12)
+        assert float(li.detach()) == pytest.approx(loss[i], rel=1e-12)
         total = total + li
     total.backward()
     for k, v in P.items():
