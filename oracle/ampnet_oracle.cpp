@@ -54,8 +54,9 @@ typedef ORACLE_REAL real;
 
 namespace {
 
+enum { LSTM_LEAF = 1, LSTM_BRANCH = 2 };
 enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, CONCAT, SPLIT,
-                BCAST, GROUP, UNGROUP, FLATMAP, SINK, N_TYPES };
+                BCAST, GROUP, UNGROUP, FLATMAP, SINK, NPT_LSTM, N_TYPES };
 enum Act { ACT_NONE, ACT_RELU, ACT_TANH, ACT_SIGMOID };
 enum { SRC_DENSE_ROW = 1, SRC_TOKENS, SRC_ZERO_STATE, SRC_TREE_LEAVES, SRC_GRAPH_NODES };
 enum { COND_SEQ_END = 1, COND_TREE_ROOT, COND_BY_U, COND_IT_LT, COND_ROUND_ROBIN };
@@ -813,6 +814,71 @@ struct SumRows : Node {         // non-parameterised payload transform: sum of t
   }
 };
 
+// LSTM gate combination (Sec. 6: the Tree-LSTM is split into a leaf and a branch cell).  Parameter-free: the gate
+// pre-activations come from an ordinary Linear node on port 0, the children's cell states [cL; cR] on port 1 (branch).
+//   leaf:   i = s(pi), o = s(po), u = tanh(pu);                 c = i u;                 h = o tanh(c)
+//   branch: i, fL, fR, o = s(.), u = tanh(pu);                  c = i u + fL cL + fR cR;  h = o tanh(c)
+// Output payload [h; c]; H = out_dim / 2.  The inputs are cached keyed on the state for the backward pass.
+struct LstmGate : Node {
+  struct In { std::vector<real> pre, cells; int got = 0; };
+  std::map<Key, In> in;
+  size_t cache_size() const override { return in.size(); }
+  static real sg(real x) { return (real)1 / ((real)1 + std::exp(-x)); }
+  void forward(Msg& m, int port) override {
+    const int H = out_dim / 2, need = fn == LSTM_BRANCH ? 2 : 1;
+    In& c = in[key_of(m.s)];
+    if (port == 0) c.pre = m.p; else c.cells = m.p;
+    if (++c.got < need) return;
+    Msg o; o.eval = m.eval; o.s = m.s; o.rows = 1; o.dim = out_dim; o.p.assign(out_dim, 0);
+    for (int j = 0; j < H; j++) {
+      real cj, oj;
+      if (fn == LSTM_LEAF) { cj = sg(c.pre[j]) * std::tanh(c.pre[2 * H + j]); oj = sg(c.pre[H + j]); }
+      else {
+        cj = sg(c.pre[j]) * std::tanh(c.pre[4 * H + j]) + sg(c.pre[H + j]) * c.cells[j] + sg(c.pre[2 * H + j]) * c.cells[H + j];
+        oj = sg(c.pre[3 * H + j]);
+      }
+      o.p[j] = oj * std::tanh(cj);
+      o.p[H + j] = cj;
+    }
+    if (m.eval) in.erase(key_of(m.s)); else c.got = 0;
+    E->round_payload(o);
+    E->emit_fwd(id, 0, o);
+  }
+  void backward(Msg& m, int) override {
+    const int H = out_dim / 2;
+    auto it = in.find(key_of(m.s));
+    if (it == in.end()) { E->err = "LstmGate: backward without cached inputs"; return; }
+    const In c = it->second;
+    in.erase(it);
+    Msg dp; dp.s = m.s; dp.rows = 1; dp.dim = in_dim; dp.p.assign(in_dim, 0);
+    Msg dc; dc.s = m.s; dc.rows = 1; dc.dim = out_dim; dc.p.assign(out_dim, 0);
+    for (int j = 0; j < H; j++) {
+      const real gh = m.p[j], gc = m.p[H + j];
+      if (fn == LSTM_LEAF) {
+        const real i = sg(c.pre[j]), o = sg(c.pre[H + j]), u = std::tanh(c.pre[2 * H + j]);
+        const real cj = i * u, tc = std::tanh(cj), d = gc + gh * o * (1 - tc * tc);
+        dp.p[j] = d * u * i * (1 - i);
+        dp.p[H + j] = gh * tc * o * (1 - o);
+        dp.p[2 * H + j] = d * i * (1 - u * u);
+      } else {
+        const real i = sg(c.pre[j]), fl = sg(c.pre[H + j]), fr = sg(c.pre[2 * H + j]), o = sg(c.pre[3 * H + j]), u = std::tanh(c.pre[4 * H + j]);
+        const real cl = c.cells[j], cr = c.cells[H + j];
+        const real cj = i * u + fl * cl + fr * cr, tc = std::tanh(cj), d = gc + gh * o * (1 - tc * tc);
+        dp.p[j] = d * u * i * (1 - i);
+        dp.p[H + j] = d * cl * fl * (1 - fl);
+        dp.p[2 * H + j] = d * cr * fr * (1 - fr);
+        dp.p[3 * H + j] = gh * tc * o * (1 - o);
+        dp.p[4 * H + j] = d * i * (1 - u * u);
+        dc.p[j] = d * fl;
+        dc.p[H + j] = d * fr;
+      }
+    }
+    E->round_payload(dp);
+    E->emit_bwd(id, 0, dp);
+    if (fn == LSTM_BRANCH) { E->round_payload(dc); E->emit_bwd(id, 1, dc); }
+  }
+};
+
 struct SourceNode : Node {
   void forward(Msg&, int) override {}
   void backward(Msg&, int) override {}
@@ -1022,6 +1088,7 @@ void* oracle_create(const int32_t* nodes, int n_nodes, const int32_t* edges, int
       case GRUCELL: n = make<GRUCell>(&E); break;
       case LOSS_CE: case LOSS_MSE: n = make<Loss>(&E); break;
       case NPT_SUMROWS: n = make<SumRows>(&E); break;
+      case NPT_LSTM: n = make<LstmGate>(&E); break;
       case COND: n = make<Cond>(&E); break;
       case PHI: n = make<Phi>(&E); break;
       case ISU: n = make<Isu>(&E); break;

@@ -69,6 +69,30 @@ def tree_loss(g, P, inst, i):
     return total
 
 
+def tree_lstm_loss(g, P, inst, i):
+    """Binary Tree-LSTM (Tai et al., N = 2) with separate leaf and branch cells; classifier on h at every node."""
+    look, leaf, br, cls = (g.index(k) for k in ("lookup", "leaf_gates", "branch_gates", "classifier"))
+    o = int(inst.offsets[i])
+    m = int(inst.offsets[i + 1]) - o
+    total = 0.0
+
+    def rec(u):
+        nonlocal total
+        if inst.left[o + u] < 0:
+            pi, po, pu = torch.chunk(P[(leaf, 0)] @ P[(look, 0)][int(inst.tokens[o + u])] + P[(leaf, 1)], 3)
+            c = torch.sigmoid(pi) * torch.tanh(pu)
+        else:
+            (hl, cl), (hr, cr) = rec(int(inst.left[o + u])), rec(int(inst.right[o + u]))
+            pi, pfl, pfr, po, pu = torch.chunk(P[(br, 0)] @ torch.cat([hl, hr]) + P[(br, 1)], 5)
+            c = torch.sigmoid(pi) * torch.tanh(pu) + torch.sigmoid(pfl) * cl + torch.sigmoid(pfr) * cr
+        h = torch.sigmoid(po) * torch.tanh(c)
+        total = total + ce(P[(cls, 0)] @ h + P[(cls, 1)], int(inst.labels_i[o + u]))
+        return h, c
+
+    rec(m - 1)
+    return total
+
+
 def ggnn_loss(g, P, inst, i, steps=4):
     """Dense-adjacency formulation: a = sum_c A_c H W_c^T with A_c[dst, src] = #edges of type c."""
     look, gru, r1, r2 = (g.index(k) for k in ("lookup", "gru", "readout1", "readout2"))
@@ -96,7 +120,7 @@ def ggnn_loss(g, P, inst, i, steps=4):
     return (y[0] - float(inst.labels_f[i])) ** 2
 
 
-LOSS_FNS = {"mlp": mlp_loss, "rnn": rnn_loss, "tree": tree_loss, "ggnn": ggnn_loss}
+LOSS_FNS = {"mlp": mlp_loss, "rnn": rnn_loss, "tree": tree_loss, "ggnn": ggnn_loss, "tree_lstm": tree_lstm_loss}
 
 
 def dataset_grad(g, params, inst):
@@ -120,6 +144,9 @@ def tiny_case(family, n=3, seed=0):
         inst = data.list_instances(n=n, max_len=4)
     elif family == "tree":
         g = ir.tree(vocab=12, emb=5, hidden=4, classes=3)
+        inst = data.tree_instances(n=n, min_leaves=2, max_leaves=5, vocab=12, classes=3)
+    elif family == "tree_lstm":
+        g = ir.tree_lstm(vocab=12, emb=5, hidden=4, classes=3)
         inst = data.tree_instances(n=n, min_leaves=2, max_leaves=5, vocab=12, classes=3)
     else:
         g = ir.ggnn(n_node_types=15, hidden=4, steps=4, readout=3)

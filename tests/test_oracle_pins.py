@@ -12,7 +12,7 @@ from workloads import ir, data, params as wp
 import helpers as H
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
-FAMILIES = ["mlp", "rnn", "tree", "ggnn"]
+FAMILIES = ["mlp", "rnn", "tree", "ggnn", "tree_lstm"]
 BIG = 1 << 30
 
 

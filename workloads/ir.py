@@ -20,10 +20,15 @@ import numpy as np
 
 # ---- node types -----------------------------------------------------------
 SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, \
-    CONCAT, SPLIT, BCAST, GROUP, UNGROUP, FLATMAP, SINK = range(17)
+    CONCAT, SPLIT, BCAST, GROUP, UNGROUP, FLATMAP, SINK, NPT_LSTM = range(18)
 TYPE_NAMES = ["SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "NPT_SUMROWS",
-              "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK"]
+              "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK", "NPT_LSTM"]
 PPT_TYPES = (LINEAR, LOOKUP, GRUCELL)
+
+# NPT_LSTM.fn: which LSTM gate combination the parameter-free node applies to the gate pre-activations on port 0
+LSTM_LEAF = 1          # [pi, po, pu] (3H): c = s(pi) tanh(pu), h = s(po) tanh(c); output [h; c]
+LSTM_BRANCH = 2        # [pi, pfL, pfR, po, pu] (5H) and the children's cells [cL; cR] on port 1:
+                       # c = s(pi) tanh(pu) + s(pfL) cL + s(pfR) cR, h = s(po) tanh(c)
 
 # ---- activations fused into a PPT node -------------------------------------
 ACT_NONE, ACT_RELU, ACT_TANH, ACT_SIGMOID = range(4)
@@ -167,6 +172,55 @@ def rnn(vocab=14, emb=128, hidden=128, classes=10, act=ACT_TANH, replicas=1):
     g.edge(cond, phi, 0, 1)     # loop
     g.edge(cond, lin2, 1, 0)    # exit
     g.edge(lin2, loss)
+    return g
+
+
+def tree_lstm(vocab=20000, emb=300, hidden=150, classes=5):
+    """Binary Tree-LSTM split into a leaf and a branch cell (Sec. 6, sentiment model).  A cell is an ordinary Linear node that
+    produces the gate pre-activations (leaf: emb -> 3H, branch: [hL; hR] -> 5H) followed by a parameter-free gate node;
+    a cell's output [h; c] is split into an h stream (classifier at every node, parent's [hL; hR]) and a c stream
+    (parent's [cL; cR]); both streams end in a Sink at the root."""
+    g = IRGraph("tree_lstm")
+    H = hidden
+    src = g.node("src_leaves", SOURCE, fn=SRC_TREE_LEAVES)
+    look = g.node("lookup", LOOKUP, vocab, emb, flags=FLAG_SOURCE_ADJACENT)
+    leaf = g.node("leaf_gates", LINEAR, emb, 3 * H)
+    leaf_g = g.node("leaf_lstm", NPT_LSTM, 3 * H, 2 * H, fn=LSTM_LEAF)
+    phi = g.node("phi", PHI, 2 * H, 2 * H)
+    sp = g.node("split_hc", SPLIT, 2 * H, H, fn_arg=2)
+    bc = g.node("bcast", BCAST, H, H, fn_arg=2)
+    cls = g.node("classifier", LINEAR, H, classes)
+    loss = g.node("loss", LOSS_CE, classes, 0, fn=LABEL_PER_TREE_NODE)
+    cond_h = g.node("cond_root_h", COND, H, H, fn=COND_TREE_ROOT)
+    sink_h = g.node("sink_h", SINK, H, 0)
+    isu_h = g.node("isu_parent_h", ISU, H, H, fn=ISU_TREE_PARENT)
+    cat_h = g.node("concat_h", CONCAT, H, 2 * H, fn=CONCAT_BY_STATE_PORT, fn_arg=2)
+    br = g.node("branch_gates", LINEAR, 2 * H, 5 * H)
+    cond_c = g.node("cond_root_c", COND, H, H, fn=COND_TREE_ROOT)
+    sink_c = g.node("sink_c", SINK, H, 0)
+    isu_c = g.node("isu_parent_c", ISU, H, H, fn=ISU_TREE_PARENT)
+    cat_c = g.node("concat_c", CONCAT, H, 2 * H, fn=CONCAT_BY_STATE_PORT, fn_arg=2)
+    br_g = g.node("branch_lstm", NPT_LSTM, 5 * H, 2 * H, fn=LSTM_BRANCH)
+    g.edge(src, look)
+    g.edge(look, leaf)
+    g.edge(leaf, leaf_g)
+    g.edge(leaf_g, phi, 0, 0)
+    g.edge(br_g, phi, 0, 1)
+    g.edge(phi, sp)
+    g.edge(sp, bc, 0, 0)            # h
+    g.edge(bc, cls, 0, 0)
+    g.edge(cls, loss)
+    g.edge(bc, cond_h, 1, 0)
+    g.edge(cond_h, sink_h, 0, 0)
+    g.edge(cond_h, isu_h, 1, 0)
+    g.edge(isu_h, cat_h)
+    g.edge(cat_h, br)
+    g.edge(br, br_g, 0, 0)
+    g.edge(sp, cond_c, 1, 0)        # c
+    g.edge(cond_c, sink_c, 0, 0)
+    g.edge(cond_c, isu_c, 1, 0)
+    g.edge(isu_c, cat_c)
+    g.edge(cat_c, br_g, 0, 1)
     return g
 
 
