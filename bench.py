@@ -31,6 +31,8 @@ WORKLOADS = {
     "rnn": (ir.rnn, data.list_instances, 20000, 16, 50, 0.05),
     "tree": (ir.tree, data.tree_instances, 8544, 64, 100, 0.05),
     "ggnn": (ir.ggnn, data.graph_instances, 130000, 128, 200, 0.01),
+    # the paper's sentiment model proper: binary Tree-LSTM (leaf and branch cells) on the same trees as "tree"
+    "tree_lstm": (ir.tree_lstm, data.tree_instances, 8544, 64, 100, 0.05),
     # throughput stress: binary tree RNN, hidden 512, 64..512 leaves, bf16 messages with fp32 accumulators
     "stress": (lambda: ir.tree(vocab=20000, emb=512, hidden=512, classes=5),
                lambda n, split=0: data.tree_instances(n=n, min_leaves=64, max_leaves=512, split=split, config_index=5),

@@ -58,12 +58,16 @@ enum {
   AMPNET_GROUP = 13,      /* collect messages by state into one matrix payload (fn = AMPNET_GROUP_*)     */
   AMPNET_UNGROUP = 14,    /* one message per row (fn = AMPNET_UNGROUP_*)                                 */
   AMPNET_FLATMAP = 15,    /* one message per generated state, payload replicated (fn = AMPNET_FLATMAP_*) */
-  AMPNET_SINK = 16        /* answers a forward message with a zero gradient                              */
+  AMPNET_SINK = 16,       /* answers a forward message with a zero gradient                              */
+  AMPNET_NPT_LSTM = 17    /* non-parameterised LSTM gate combination (fn = AMPNET_LSTM_*): gate pre-activations from a
+                             LINEAR node on port 0 (and the children's cells [cL; cR] on port 1) -> [h; c]          */
 };
 enum { AMPNET_ACT_NONE = 0, AMPNET_ACT_RELU = 1, AMPNET_ACT_TANH = 2, AMPNET_ACT_SIGMOID = 3 };
 /* state functions; the message state is (inst, seq, slot, it, u, port)                                     */
 enum { AMPNET_SRC_DENSE_ROW = 1, AMPNET_SRC_TOKENS = 2, AMPNET_SRC_ZERO_STATE = 3, AMPNET_SRC_TREE_LEAVES = 4,
        AMPNET_SRC_GRAPH_NODES = 5 };
+enum { AMPNET_LSTM_LEAF = 1,   /* [pi, po, pu] (3H): c = s(pi) tanh(pu), h = s(po) tanh(c)                                   */
+       AMPNET_LSTM_BRANCH = 2 }; /* [pi, pfL, pfR, po, pu] (5H), [cL; cR]: c = s(pi) tanh(pu) + s(pfL) cL + s(pfR) cR, h = s(po) tanh(c) */
 enum { AMPNET_COND_SEQ_END = 1,   /* u < #tokens ? 0 : 1        */
        AMPNET_COND_TREE_ROOT = 2, /* u is the root ? 0 : 1      */
        AMPNET_COND_BY_U = 3,      /* successor = u              */
@@ -105,6 +109,10 @@ ampnet_status_t ampnet_ir_mlp(const int32_t* dims, int32_t n_dims, ampnet_node_d
 ampnet_status_t ampnet_ir_rnn(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes, int32_t act,
                               ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
                               ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
+/* binary Tree-LSTM (Sec. 6): leaf and branch cells built from a LINEAR node (gate pre-activations) and an NPT_LSTM node */
+ampnet_status_t ampnet_ir_tree_lstm(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
+                                    ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                                    ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
 ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
                                ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
                                ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);

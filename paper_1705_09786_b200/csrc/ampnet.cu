@@ -249,6 +249,10 @@ ampnet_status_t build_topology(ampnet_graph* g) {
       case UNGROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 2, "UNGROUP needs a valid fn"); break;
       case FLATMAP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn == 1, "FLATMAP needs a valid fn"); break;
       case NPT_SUMROWS: st = need(h.n_pred == 1 && h.n_succ == 1, "NPT_SUMROWS needs one predecessor and one successor"); break;
+      case NPT_LSTM:
+        st = need(h.n_succ == 1 && (h.fn == 1 || h.fn == 2) && h.n_pred == h.fn && h.out_dim > 0 && h.out_dim % 2 == 0 &&
+                  h.in_dim == (h.fn == 1 ? 3 : 5) * (h.out_dim / 2), "NPT_LSTM needs fn 1 (3H -> 2H, one port) or 2 (5H and 2H -> 2H, two ports)");
+        break;
     }
     if (st != AMPNET_OK) return st;
     if (h.type == ISU && h.fn == 3) g->has_it = true;
@@ -258,7 +262,7 @@ ampnet_status_t build_topology(ampnet_graph* g) {
   if (g->losses.empty() || g->losses.size() > 4) return set_err(g, AMPNET_EINVAL, "the graph needs 1..4 LOSS nodes");
   // widths along the edges
   auto out_width = [&](const DevNode& h) {
-    if (h.type == LINEAR || h.type == LOOKUP || h.type == GRUCELL || h.type == CONCAT || h.type == SPLIT) return h.out_dim;
+    if (h.type == LINEAR || h.type == LOOKUP || h.type == GRUCELL || h.type == CONCAT || h.type == SPLIT || h.type == NPT_LSTM) return h.out_dim;
     if (h.type == SOURCE) return (h.fn == 1 || h.fn == 3) ? h.out_dim : 0;
     return h.in_dim;
   };
@@ -267,7 +271,8 @@ ampnet_status_t build_topology(ampnet_graph* g) {
     const int w = out_width(s);
     if (d.type == LOOKUP || w == 0) continue;
     if (d.type == SINK) continue;
-    if (w != d.in_dim) return set_err(g, AMPNET_EINVAL, "edge %zu: width %d does not match the destination's in_dim %d", k, w, d.in_dim);
+    const int want = (d.type == NPT_LSTM && g->edges[k].dst_port == 1) ? d.out_dim : d.in_dim;    // port 1 of the gate node takes [cL; cR]
+    if (w != want) return set_err(g, AMPNET_EINVAL, "edge %zu: width %d does not match the destination's input width %d", k, w, want);
   }
   // every cycle must pass through a PHI: the graph without PHI nodes is acyclic
   std::vector<int> indeg(n, 0);
@@ -626,6 +631,11 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
         n.jstride = (long long)n.rows_out * n.in_dim;
         n.jcnt = C.take<int>(kout); track(n.jcnt, kout * sizeof(int));
         break;
+      case NPT_LSTM:         // per key: gate pre-activations, the children's cells, the output [h; c]
+        n.jstride = (long long)n.in_dim + 2 * n.out_dim;
+        n.jbuf = B.take<float>(kin * n.jstride);
+        n.jcnt = C.take<int>(kin); track(n.jcnt, kin * sizeof(int));
+        break;
       case UNGROUP:
       case SPLIT:            // the backward join of the parts' gradients
         n.jstride = (long long)n.rows_in * n.in_dim;
@@ -681,6 +691,13 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   X.n_sources = (int)g->sources.size();
   for (size_t k = 0; k < g->sources.size(); k++) X.src_nodes[k] = g->sources[k];
   X.n_loss = (int)g->losses.size();
+  // A forward-only instance is finished when it has reached every end of the graph: a Loss with one label per instance
+  // and a Sink are reached once, a Loss with a label per position (tree node) once per position.
+  X.ends_per_instance = X.ends_per_position = 0;
+  for (auto& hn : g->hnodes) {
+    if (hn.type == SINK) X.ends_per_instance++;
+    if (hn.type == LOSS_CE || hn.type == LOSS_MSE) { if (hn.type == LOSS_CE && hn.fn == 2) X.ends_per_position++; else X.ends_per_instance++; }
+  }
   for (size_t k = 0; k < g->losses.size(); k++) X.loss_nodes[k] = g->losses[k];
   X.slot_inst = B.take<int>(mak);
   X.outstanding = C.take<int>(mak);
@@ -797,7 +814,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   if (!eval && !det && R.ctx.emit_ctas)      // emitter time of the node = time of its first emitter x emitters (they share every batch)
     for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].emit_load = (double)G.role_cycles[8 + 8 * p + 5] * std::max(1, g->ppts[p].NE) + 1.0;
   if (getenv("AMPNET_TUNE") && (atoi(getenv("AMPNET_TUNE")) & 8)) {
-    static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK"};
+    static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK", "LSTM"};
     const double us = 1.0 / 1965.0;
     fprintf(stderr, "[ctrl] us: retire %.0f admit %.0f clear %.0f pump %.0f idle %.0f admissions %llu\n", G.role_cycles[0] * us, G.role_cycles[1] * us,
             G.role_cycles[2] * us, G.role_cycles[3] * us, G.role_cycles[4] * us, G.role_cycles[5]);

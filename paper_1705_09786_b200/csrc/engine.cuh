@@ -263,6 +263,8 @@ __device__ __forceinline__ void to_pred(Frame& f, const DevNode& n, int j) {
   f.node = n.pred_node[j]; f.aport = n.pred_port[j]; f.dir = BWD; f.iter = 0;
 }
 
+__device__ __forceinline__ float sigm(float v) { return 1.f / (1.f + expf(-v)); }
+
 // first position (token / tree node / graph node) of an instance
 #define IBASE(inst) (I.offsets ? I.offsets[(inst)] : 0)
 __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& acc, WalkPool* Q) {
@@ -286,7 +288,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
     const bool shadow = f.nparts > 1 && f.part > 0;
     const bool dies_as_shadow = shadow && !(n.type == COND || n.type == PHI || n.type == ISU) && (n.type == LINEAR || n.type == LOOKUP || n.type == GRUCELL || n.type == LOSS_CE ||
                                            n.type == LOSS_MSE || n.type == SINK || n.type == SOURCE || n.type == NPT_SUMROWS ||
-                                           (n.type == BCAST && f.dir == BWD) || (n.type == CONCAT && f.dir == FWD) || (n.type == SPLIT && f.dir == BWD) ||
+                                           (n.type == BCAST && f.dir == BWD) || (n.type == CONCAT && f.dir == FWD) || (n.type == SPLIT && f.dir == BWD) || n.type == NPT_LSTM ||
                                            (n.type == GROUP && f.dir == FWD) || (n.type == UNGROUP && f.dir == BWD) ||
                                            (n.type == FLATMAP && f.dir == BWD));
     if (dies_as_shadow) {
@@ -454,6 +456,72 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             cont = true;
           }
           break;
+        case NPT_LSTM: {                          // LSTM gate combination; cache per key: [pre-activations | cells | output]
+          const int H = n.out_dim / 2;
+          long long key = key_of(C, f.node, f.slot, f.it, f.u, n.U_in);
+          if (key < 0) return;
+          if (f.rows != 1) { fail(C, ST_OVERFLOW, f.node, f.rows); return; }
+          float* base = n.jbuf + key * n.jstride;
+          float* cells = base + n.in_dim;
+          if (f.dir == FWD) {
+            if (f.aport == 0) warp_copy(base, n.in_dim, f, 1, n.in_dim, lane);
+            else warp_copy(cells, n.out_dim, f, 1, n.out_dim, lane);
+            if (n.fn == 2) { if (!join_arrive(&n.jcnt[key], 2, lane)) break; }       // the other port's message is still under way
+            else __syncwarp();
+            float* outp = cells + n.out_dim;
+            for (int j = lane; j < H; j += 32) {
+              float cj, oj;
+              if (n.fn == 1) { cj = sigm(base[j]) * tanhf(base[2 * H + j]); oj = sigm(base[H + j]); }
+              else {
+                cj = sigm(base[j]) * tanhf(base[4 * H + j]) + sigm(base[H + j]) * cells[j] + sigm(base[2 * H + j]) * cells[H + j];
+                oj = sigm(base[3 * H + j]);
+              }
+              outp[j] = emit_round(oj * tanhf(cj));
+              outp[H + j] = emit_round(cj);
+            }
+            __syncwarp();
+            f.p = outp; f.nsum = 1; f.sstride = 0; f.dim = n.out_dim; f.ld = n.out_dim;
+            to_succ(f, n, 0);
+            cont = true;
+          } else if (f.iter == 0) {
+            // gradients in place: d pre-activations over the cached pre-activations, [dcL; dcR] over the cached cells
+            for (int j = lane; j < H; j += 32) {
+              const float gh = ld_payload(f.p, f.nsum, f.sstride, j), gc = ld_payload(f.p, f.nsum, f.sstride, H + j);
+              if (n.fn == 1) {
+                const float i = sigm(base[j]), o = sigm(base[H + j]), u = tanhf(base[2 * H + j]);
+                const float tc = tanhf(i * u), d = gc + gh * o * (1.f - tc * tc);
+                base[j] = emit_round(d * u * i * (1.f - i));
+                base[H + j] = emit_round(gh * tc * o * (1.f - o));
+                base[2 * H + j] = emit_round(d * i * (1.f - u * u));
+              } else {
+                const float i = sigm(base[j]), fl = sigm(base[H + j]), fr = sigm(base[2 * H + j]),
+                            o = sigm(base[3 * H + j]), u = tanhf(base[4 * H + j]);
+                const float cl = cells[j], cr = cells[H + j];
+                const float tc = tanhf(i * u + fl * cl + fr * cr), d = gc + gh * o * (1.f - tc * tc);
+                base[j] = emit_round(d * u * i * (1.f - i));
+                base[H + j] = emit_round(d * cl * fl * (1.f - fl));
+                base[2 * H + j] = emit_round(d * cr * fr * (1.f - fr));
+                base[3 * H + j] = emit_round(gh * tc * o * (1.f - o));
+                base[4 * H + j] = emit_round(d * i * (1.f - u * u));
+                cells[j] = emit_round(d * fl);
+                cells[H + j] = emit_round(d * fr);
+              }
+            }
+            __syncwarp();
+            if (n.fn == 2) {                      // second message: the cells' gradient to port 1
+              Frame c = f; c.iter = 1;
+              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+                                             if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
+            }
+            f.p = base; f.nsum = 1; f.sstride = 0; f.dim = n.in_dim; f.ld = n.in_dim;
+            to_pred(f, n, 0);
+            cont = true;
+          } else {
+            f.p = cells; f.nsum = 1; f.sstride = 0; f.dim = n.out_dim; f.ld = n.out_dim;
+            to_pred(f, n, 1);
+            cont = true;
+          }
+        } break;
         case SPLIT:                               // inverse of Concat: successor k gets the columns [k w, (k + 1) w)
           if (f.dir == FWD) {
             const int k = f.iter;
@@ -2025,8 +2093,8 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
           S.n_src_msgs = total;
           S.admit_eval = C.eval || (C.inference_only && C.inference_only[inst]);
           if (S.admit_eval) {      // forward only: the instance is finished when every Loss / Sink has been reached
-            int exp = 1;
-            if (I.kind == 2) exp = (int)(I.offsets[inst + 1] - I.offsets[inst]) + 1;
+            int exp = C.ends_per_instance;
+            if (C.ends_per_position) exp += C.ends_per_position * (int)(I.offsets[inst + 1] - I.offsets[inst]);
             C.outstanding[slot] = exp;
           } else C.outstanding[slot] = total;
           if (C.det && C.keylog) {

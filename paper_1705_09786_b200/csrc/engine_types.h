@@ -16,7 +16,7 @@ constexpr int MAX_TILES = 32;        // row tiles per PPT node
 constexpr int WALK_STACK = 12;        // continuation frames per walking warp
 
 enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, CONCAT, SPLIT,
-                BCAST, GROUP, UNGROUP, FLATMAP, SINK, N_NODE_TYPES };
+                BCAST, GROUP, UNGROUP, FLATMAP, SINK, NPT_LSTM, N_NODE_TYPES };
 enum { FWD = 0, BWD = 1 };
 enum { HDR_EVAL = 1 };
 enum { BATCH_UPDATE = 1, BATCH_END_ROUND = 2, BATCH_TERMINATE = 4 };
@@ -161,6 +161,7 @@ struct Ctx {
   // controller
   int n_sources; int src_nodes[4];
   int n_loss; int loss_nodes[4];
+  int ends_per_instance, ends_per_position;   // forward-only instances: Loss / Sink arrivals that finish one = a + b x positions
   int* slot_inst; int* outstanding; int* slot_log;
   KeyLog* keylog;
   unsigned* retire_e; unsigned* retire_seq; unsigned retire_mask;

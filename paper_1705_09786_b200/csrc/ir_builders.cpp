@@ -130,6 +130,54 @@ ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32
   return b.emit(nodes, cap_nodes, n_nodes, edges, cap_edges, n_edges);
 }
 
+ampnet_status_t ampnet_ir_tree_lstm(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
+                                    ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                                    ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges) {
+  if (vocab < 1 || emb < 1 || hidden < 1 || classes < 1) return AMPNET_EINVAL;
+  Builder b;
+  const int H = hidden;
+  int src = b.node(AMPNET_SOURCE, 0, 0, 0, AMPNET_SRC_TREE_LEAVES);
+  int look = b.node(AMPNET_LOOKUP, vocab, emb, 0, 0, 0, AMPNET_FLAG_SOURCE_ADJACENT);
+  int leaf = b.node(AMPNET_LINEAR, emb, 3 * H);                                   // leaf cell: gate pre-activations i, o, u
+  int leaf_g = b.node(AMPNET_NPT_LSTM, 3 * H, 2 * H, 0, AMPNET_LSTM_LEAF);
+  int phi = b.node(AMPNET_PHI, 2 * H, 2 * H);
+  int sp = b.node(AMPNET_SPLIT, 2 * H, H, 0, 0, 2);                               // [h; c] -> h stream, c stream
+  int bc = b.node(AMPNET_BCAST, H, H, 0, 0, 2);
+  int cls = b.node(AMPNET_LINEAR, H, classes);
+  int loss = b.node(AMPNET_LOSS_CE, classes, 0, 0, AMPNET_LABEL_PER_TREE_NODE);
+  int cond_h = b.node(AMPNET_COND, H, H, 0, AMPNET_COND_TREE_ROOT);
+  int sink_h = b.node(AMPNET_SINK, H, 0);
+  int isu_h = b.node(AMPNET_ISU, H, H, 0, AMPNET_ISU_TREE_PARENT);
+  int cat_h = b.node(AMPNET_CONCAT, H, 2 * H, 0, AMPNET_CONCAT_BY_STATE_PORT, 2);
+  int br = b.node(AMPNET_LINEAR, 2 * H, 5 * H);                                   // branch cell: i, fL, fR, o, u from [hL; hR]
+  int cond_c = b.node(AMPNET_COND, H, H, 0, AMPNET_COND_TREE_ROOT);
+  int sink_c = b.node(AMPNET_SINK, H, 0);
+  int isu_c = b.node(AMPNET_ISU, H, H, 0, AMPNET_ISU_TREE_PARENT);
+  int cat_c = b.node(AMPNET_CONCAT, H, 2 * H, 0, AMPNET_CONCAT_BY_STATE_PORT, 2);
+  int br_g = b.node(AMPNET_NPT_LSTM, 5 * H, 2 * H, 0, AMPNET_LSTM_BRANCH);
+  b.edge(src, look);
+  b.edge(look, leaf);
+  b.edge(leaf, leaf_g);
+  b.edge(leaf_g, phi, 0, 0);
+  b.edge(br_g, phi, 0, 1);
+  b.edge(phi, sp);
+  b.edge(sp, bc, 0, 0);
+  b.edge(bc, cls, 0, 0);
+  b.edge(cls, loss);
+  b.edge(bc, cond_h, 1, 0);
+  b.edge(cond_h, sink_h, 0, 0);
+  b.edge(cond_h, isu_h, 1, 0);
+  b.edge(isu_h, cat_h);
+  b.edge(cat_h, br);
+  b.edge(br, br_g, 0, 0);
+  b.edge(sp, cond_c, 1, 0);
+  b.edge(cond_c, sink_c, 0, 0);
+  b.edge(cond_c, isu_c, 1, 0);
+  b.edge(isu_c, cat_c);
+  b.edge(cat_c, br_g, 0, 1);
+  return b.emit(nodes, cap_nodes, n_nodes, edges, cap_edges, n_edges);
+}
+
 ampnet_status_t ampnet_ir_ggnn(int32_t n_node_types, int32_t hidden, int32_t steps, int32_t n_edge_types, int32_t readout,
                                ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
                                ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges) {

@@ -44,6 +44,10 @@ def gradient_rows(graph, inst):
         L = (np.diff(inst.offsets) + 1) // 2
         return {graph.index("lookup"): int(L.sum()), graph.index("leaf_cell"): int(L.sum()),
                 graph.index("branch_cell"): int((L - 1).sum()), graph.index("classifier"): int((2 * L - 1).sum())}
+    if name == "tree_lstm":
+        L = (np.diff(inst.offsets) + 1) // 2
+        return {graph.index("lookup"): int(L.sum()), graph.index("leaf_gates"): int(L.sum()),
+                graph.index("branch_gates"): int((L - 1).sum()), graph.index("classifier"): int((2 * L - 1).sum())}
     if name == "ggnn":
         steps = int(graph.nodes[graph.index("cond_it")][5])
         N = int(np.diff(inst.offsets).sum())
@@ -67,6 +71,9 @@ def node_messages(graph, inst):
     if name == "tree":
         L = (np.diff(inst.offsets) + 1) // 2
         return int((33 * L - 18).sum())
+    if name == "tree_lstm":
+        L = (np.diff(inst.offsets) + 1) // 2
+        return int((55 * L - 32).sum())
     if name == "ggnn":
         steps = int(graph.nodes[graph.index("cond_it")][5])
         N, D = np.diff(inst.offsets), np.diff(inst.edge_offsets)

@@ -16,6 +16,8 @@ pytestmark = pytest.mark.gpu
 
 
 def _case(family, n):
+    if family == "tree_lstm":
+        return ir.tree_lstm(), data.tree_instances(n=n)
     if family == "mlp":
         return ir.mlp((784, 256, 256, 10)), data.mlp_instances(n=n)
     if family == "rnn":
@@ -31,6 +33,7 @@ CASES = [
     ("rnn", 90, 1, 1, 0.02), ("rnn", 90, 16, 50, 0.05), ("rnn", 61, 5, 3, 0.02),
     ("tree", 24, 1, 1, 0.002), ("tree", 40, 64, 100, 0.05), ("tree", 31, 6, 7, 0.01),
     ("ggnn", 12, 1, 1, 0.0005), ("ggnn", 40, 128, 200, 0.01), ("ggnn", 25, 9, 40, 0.005),
+    ("tree_lstm", 16, 1, 1, 0.002), ("tree_lstm", 36, 64, 100, 0.05), ("tree_lstm", 27, 6, 7, 0.01),
 ]
 
 
@@ -116,7 +119,7 @@ def test_replicated_linear_with_end_of_epoch_averaging(oracle_mod, k, mak, muf):
 
 
 @pytest.mark.parametrize("family,n,mak,muf,lr", [("tree", 30, 6, 7, 0.01), ("ggnn", 24, 9, 40, 0.003), ("rnn", 60, 5, 3, 0.02),
-                                                ("mlp", 40, 4, 8, 0.01)])
+                                                ("mlp", 40, 4, 8, 0.01), ("tree_lstm", 24, 6, 7, 0.01)])
 def test_concurrent_inference_matches_oracle(oracle_mod, family, n, mak, muf, lr):
     """A third of the instances are only evaluated while the others train, in the same queues (deterministic schedule:
     bookkeeping bit-exact, floats within the usual tolerances), then the same in the free-running schedule."""
@@ -271,7 +274,7 @@ def test_per_node_update_threshold(oracle_mod):
 
 
 @pytest.mark.parametrize("family,n,mak,muf,lr", [("tree", 30, 16, 20, 0.02), ("rnn", 60, 8, 10, 0.02),
-                                                ("ggnn", 20, 16, 40, 0.003), ("mlp", 40, 4, 8, 0.01)])
+                                                ("ggnn", 20, 16, 40, 0.003), ("mlp", 40, 4, 8, 0.01), ("tree_lstm", 24, 16, 20, 0.02)])
 def test_bf16_payloads_match_oracle(oracle_mod, family, n, mak, muf, lr):
     """bf16 messages: every emitted payload rounded to bfloat16 on both sides.  Bookkeeping stays bit-exact.  A value
     that lies within fp32 rounding of a bf16 rounding boundary can round the other way on the GPU (fp32) than in
@@ -293,7 +296,7 @@ def test_bf16_payloads_match_oracle(oracle_mod, family, n, mak, muf, lr):
     r[3].close()
 
 
-@pytest.mark.parametrize("family,n", [("mlp", 64), ("rnn", 80), ("tree", 40), ("ggnn", 30)])
+@pytest.mark.parametrize("family,n", [("mlp", 64), ("rnn", 80), ("tree", 40), ("ggnn", 30), ("tree_lstm", 30)])
 def test_eval_matches_oracle(oracle_mod, family, n):
     import paper_1705_09786_b200 as amp
     g, inst = _case(family, n)
@@ -317,7 +320,8 @@ def test_eval_matches_oracle(oracle_mod, family, n):
 
 
 @pytest.mark.parametrize("family,n,mak,muf,lr", [("mlp", 512, 4, 32, 0.01), ("rnn", 1500, 16, 50, 0.05),
-                                                ("tree", 400, 64, 100, 0.05), ("ggnn", 600, 128, 200, 0.003)])
+                                                ("tree", 400, 64, 100, 0.05), ("ggnn", 600, 128, 200, 0.003),
+                                                ("tree_lstm", 300, 64, 100, 0.05)])
 def test_async_mode_invariants(family, n, mak, muf, lr):
     """The free-running schedule is timing dependent; what holds for every schedule is checked exactly."""
     import paper_1705_09786_b200 as amp
@@ -398,6 +402,11 @@ def parity_counts(g, inst):
         T = np.diff(inst.offsets)
         return dict(node_messages=int((13 * T + 3).sum()),
                     grads={g.index("lookup"): T.sum(), g.index("linear1"): T.sum(), g.index("linear2"): inst.n})
+    if g.name == "tree_lstm":
+        L = (np.diff(inst.offsets) + 1) // 2
+        return dict(node_messages=int((55 * L - 32).sum()),
+                    grads={g.index("lookup"): L.sum(), g.index("leaf_gates"): L.sum(),
+                           g.index("branch_gates"): (L - 1).sum(), g.index("classifier"): (2 * L - 1).sum()})
     if g.name == "tree":
         L = (np.diff(inst.offsets) + 1) // 2
         return dict(node_messages=int((33 * L - 18).sum()),
