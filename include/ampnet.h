@@ -261,6 +261,11 @@ enum { AMPNET_OPT_SGD = 0, AMPNET_OPT_MOMENTUM = 1, AMPNET_OPT_ADAM = 2 };
 ampnet_status_t ampnet_set_optimizer(ampnet_graph_t*, int32_t kind, float momentum, float beta1, float beta2, float eps,
                                      int32_t reset_state);
 
+/* FP32 multiply-add rate of the device, measured with a register-only FMA kernel (16 independent chains per thread, 8
+ * blocks of 256 threads per SM, best of three timed launches on the default stream): the denominator of the roofline
+ * fraction of this path, which is bound by plain FP32 arithmetic.  Needs no handle.  Errors: AMPNET_ECUDA, AMPNET_ENOMEM. */
+ampnet_status_t ampnet_measure_fma_peak(int32_t device, double* tflops);
+
 const char* ampnet_last_error(const ampnet_graph_t*); /* library-owned string */
 
 /* ---- a training epoch that allocates nothing (no counterpart in the paper) ------------------------------

@@ -4,4 +4,4 @@ Every step of the hot path runs in the CUDA library (libampnet.so); this package
 arguments.  PyTorch supplies device memory (through the allocator callbacks) and the CUDA stream.
 There is no CPU fallback: without the built library or without a CUDA device the calls raise.
 """
-from .binding import Engine, EpochStats, AmpnetError, load_library, RunCfg, ir_tables  # noqa: F401
+from .binding import Engine, EpochStats, AmpnetError, load_library, RunCfg, ir_tables, measure_fma_peak  # noqa: F401

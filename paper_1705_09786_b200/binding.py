@@ -13,7 +13,7 @@ EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
            "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_mixed", "ampnet_param_device_ptr", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_ir_mlp", "ampnet_ir_rnn",
-           "ampnet_ir_tree", "ampnet_ir_ggnn", "ampnet_ir_tree_lstm"]
+           "ampnet_ir_tree", "ampnet_ir_ggnn", "ampnet_ir_tree_lstm", "ampnet_measure_fma_peak"]
 
 
 class InferenceStats(C.Structure):
@@ -109,6 +109,7 @@ def load_library():
     lib.ampnet_param_device_ptr.argtypes = [P, C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64)]
     lib.ampnet_ir_tree.argtypes = [I32] * 4 + tail
     lib.ampnet_ir_tree_lstm.argtypes = [I32] * 4 + tail
+    lib.ampnet_measure_fma_peak.argtypes = [C.c_int32, C.POINTER(C.c_double)]
     lib.ampnet_ir_ggnn.argtypes = [I32] * 5 + tail
     lib.ampnet_last_error.argtypes = [P]
     lib.ampnet_last_error.restype = C.c_char_p
@@ -118,6 +119,15 @@ def load_library():
 
 def _p(a):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def measure_fma_peak(device=0):
+    """Measured FP32 FMA rate of the device in TFLOP/s (register-only kernel of the library)."""
+    v = C.c_double()
+    rc = load_library().ampnet_measure_fma_peak(device, C.byref(v))
+    if rc != 0:
+        raise AmpnetError(rc, "ampnet_measure_fma_peak failed")
+    return v.value
 
 
 def ir_tables(family, *args):

@@ -87,6 +87,22 @@ struct ampnet_graph {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
 };
 
+// FP32 FMA issue rate of the device, measured: every thread runs 16 independent FMA chains from registers.
+__global__ void __launch_bounds__(256) fma_peak_kernel(float* sink, int iters) {
+  float a[16];
+#pragma unroll
+  for (int k = 0; k < 16; k++) a[k] = 1.0f + 1e-3f * (float)(threadIdx.x + k);
+  const float m = 1.0000001f, c = 1e-7f;
+  for (int i = 0; i < iters; i++) {
+#pragma unroll
+    for (int k = 0; k < 16; k++) a[k] = fmaf(a[k], m, c);
+  }
+  float s = 0.f;
+#pragma unroll
+  for (int k = 0; k < 16; k++) s += a[k];
+  if (s == 12345.678f) sink[0] = s;          // keeps the chains alive
+}
+
 // End-of-epoch replica synchronisation (Sec. 5): element-wise mean of up to eight nodes' parameters, written back to all.
 struct AvgArgs { float* W[8]; float* b[8]; int n; long long nW, nb; };
 __global__ void average_params_kernel(const AvgArgs a) {
@@ -960,6 +976,32 @@ ampnet_status_t ampnet_average_params(ampnet_graph_t* g, const int32_t* nodes, i
   CUDA_TRY(g, cudaGetLastError());
   CUDA_TRY(g, cudaStreamSynchronize(g->stream));
   return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_measure_fma_peak(int32_t device, double* tflops) {
+  if (!tflops) return AMPNET_EINVAL;
+  cudaDeviceProp prop{};
+  if (cudaSetDevice(device) != cudaSuccess || cudaGetDeviceProperties(&prop, device) != cudaSuccess) return AMPNET_ECUDA;
+  float* sink = nullptr;
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  if (cudaMalloc(&sink, 256) != cudaSuccess) return AMPNET_ENOMEM;
+  ampnet_status_t rc = AMPNET_OK;
+  const int blocks = prop.multiProcessorCount * 8, iters = 1 << 16;
+  float best_ms = 1e30f;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) rc = AMPNET_ECUDA;
+  for (int rep = 0; rep < 4 && rc == AMPNET_OK; rep++) {        // the first repetition warms up
+    cudaEventRecord(e0, 0);
+    fma_peak_kernel<<<blocks, 256>>>(sink, iters);
+    cudaEventRecord(e1, 0);
+    float ms = 0.f;
+    if (cudaEventSynchronize(e1) != cudaSuccess || cudaEventElapsedTime(&ms, e0, e1) != cudaSuccess) rc = AMPNET_ECUDA;
+    else if (rep > 0) best_ms = std::min(best_ms, ms);
+  }
+  if (rc == AMPNET_OK) *tflops = (double)blocks * 256.0 * 16.0 * 2.0 * (double)iters / (best_ms * 1e-3) / 1e12;
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  cudaFree(sink);
+  return rc;
 }
 
 const char* ampnet_last_error(const ampnet_graph_t* g) { return g ? g->err.c_str() : "invalid handle"; }
