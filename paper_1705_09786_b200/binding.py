@@ -232,7 +232,8 @@ class Engine:
         return a.reshape(dict(self.graph.param_shapes(node))[which])
 
     def param_tensors(self):
-        """{(node, which): torch tensor} aliasing the parameter arrays in device memory (no copies)."""
+        """{(node, which): torch tensor} aliasing the parameter arrays in device memory (no copies).  The arrays belong to
+        the engine: the tensors must not be used after close(), and not while an epoch is running."""
         import torch
 
         class _View:                          # what torch.as_tensor needs to wrap a raw device pointer
