@@ -146,6 +146,17 @@ def test_concurrent_inference_matches_oracle(oracle_mod, family, n, mak, muf, lr
     for node, G in want["grads"].items():
         assert e.node_stats(node)["n_grads_applied"] == G
     assert inf["instances"] == int(mask.sum()) and np.isfinite(loss).all() and e.leftover_cache_entries() == 0
+    # every instance forward-only: a pure evaluation inside the training entry point, no parameter moves
+    before = e.get_params()
+    _, _, want_loss = e.eval(0, mak=mak)
+    st, loss, inf = e.run_epoch_mixed(mak=mak, muf=1, lr=0.5, inference_only=np.ones(inst.n, np.uint8), timeout_s=60)
+    np.testing.assert_allclose(loss, want_loss, rtol=1e-4, atol=1e-6)      # two free-running passes: summation orders differ
+    assert inf["instances"] == inst.n and all(e.node_stats(n)["n_updates"] == 0 for n in g.ppt_nodes())
+    for k, v in e.get_params().items():
+        np.testing.assert_array_equal(v, before[k])
+    # and an empty epoch
+    st, loss = e.run_epoch(mak=mak, muf=muf, lr=lr, order=np.zeros(0, np.int64), timeout_s=60)
+    assert st.instances == 0 and st.node_messages == 0
     e.close()
 
 
