@@ -466,6 +466,40 @@ def test_async_convergence_matches_synchronous_oracle(oracle_mod):
     e.close()
 
 
+def test_replicated_model_converges_with_a_larger_effective_minibatch():
+    """Sec. 6 on replicas: two copies of Linear-1, averaged at the end of every epoch, learn the list reduction task;
+    every copy still updates after 50 gradients of its own, i.e. the effective minibatch doubles (the paper's
+    explanation of its slowdown with 4 copies), so the replicated model may need a few more epochs for the same
+    accuracy: at most four more than the six of the unreplicated one."""
+    import paper_1705_09786_b200 as amp
+    train, valid = data.list_instances(n=3000), data.list_instances(n=1000, split=1)
+
+    def run(k, epochs, target=None):
+        g = ir.rnn(replicas=k)
+        copies = [g.index("linear1")] + [g.index(f"linear1_r{r}") for r in range(1, k)]
+        e = amp.Engine(g)
+        e.load_instances(train)
+        e.load_instances(valid, split=1)
+        p = wp.init_params(g)
+        for c in copies[1:]:                               # the copies start equal
+            p[(c, 0)], p[(c, 1)] = p[(copies[0], 0)], p[(copies[0], 1)]
+        e.set_params(p)
+        best = 0.0
+        for _ in range(epochs):
+            e.run_epoch(mak=16, muf=50, lr=0.05, deterministic=False, timeout_s=120)
+            if k > 1:
+                e.average_params(copies)
+            best = max(best, e.eval(split=1)[1])
+            if target is not None and best >= target:
+                break
+        e.close()
+        return best
+
+    a1 = run(1, 6)
+    assert a1 > 0.3                                         # chance is 0.1
+    assert run(2, 10, target=a1 - 0.02) >= a1 - 0.02
+
+
 # ---------------------------------------------------------------------------------------------------
 # failure paths: every one returns a status, none faults or hangs the device
 # ---------------------------------------------------------------------------------------------------
