@@ -1837,7 +1837,9 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       AMP_PHASE(4);
       // ---- all tiles of the node done with the batch, then emit ------------------------------------
       if (count > 0) {
-        __threadfence();
+        // With emitter CTAs the block barrier below orders every thread's writes before thread 0's release store of
+        // the hand-over counter (a release is cumulative over the barrier); only the barrier among tiles needs the fence.
+        if (!C.emit_ctas) __threadfence();
         // tiles that emit themselves wait for each other here; emitter CTAs wait for all tiles instead
         if (P.T > 1 && !C.emit_ctas) { if (!cta_barrier(C, t0, P.nbar, (unsigned)P.T, node_gen, &S.ok)) { running = false; break; } }
         else __syncthreads();
