@@ -927,6 +927,7 @@ __device__ __noinline__ void tile_accum(const float* __restrict__ Ds, int ldd, i
 struct LeaderState {
   unsigned head[2], sched_w, batch_w;
   int n_acc, version, log_n;
+  int ver_form;                        // version when the last batch was formed (staleness is accounted after it is published)
   unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
 };
 
@@ -1010,7 +1011,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
       long long key = key_of(C, P.node, h[j].slot, h[j].it, h[j].u, P.U);
       if (key >= 0) {
         if (dir == FWD) P.vcache[key] = S.ls.version;
-        else {
+        else if (!C.sched_ctas) {             // a scheduler CTA accounts staleness after it has published the batch
           int s = S.ls.version - P.vcache[key];
           if (s < 0) s = 0;
           atomicAdd(&S.stale_hist[s > 63 ? 63 : s], 1ull);
@@ -1021,6 +1022,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
   }
   __syncwarp();
   if (lane == 0) {
+    S.ls.ver_form = S.ls.version;
     BatchDesc d;
     d.sched_start = S.ls.sched_w; d.count = take; d.dir = dir; d.flags = upd ? BATCH_UPDATE : 0;
     d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.upd_t = upd ? (int)S.ls.n_updates + 1 : 0; d.pad1 = 0;
@@ -1964,7 +1966,18 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
       bool progressed = false;
       const bool gow = warp_uniform(go);
       if (gow) progressed = leader_try_schedule(C, P, S);
-      if (progressed) publish_ctx_block(C, P, S, bw);
+      if (progressed) {
+        publish_ctx_block(C, P, S, bw);
+        if (S.desc.dir == BWD && S.desc.count > 0 && !(S.hdr[0].flags & HDR_EVAL)) {     // staleness of the batch just published
+          for (int i = lane; i < S.desc.count; i += 32) {
+            int st = S.ls.ver_form - P.vcache[S.key[i]];
+            if (st < 0) st = 0;
+            atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
+            atomicMax(&S.max_stale, st);
+          }
+          __syncwarp();
+        }
+      }
       if (lane == 0) { const long long tn = clock64(); rcl[!gow ? 0 : progressed ? 2 : 1] += (unsigned long long)(tn - tp); tp = tn; }
       if (gow) {
         unsigned fin = 0;
