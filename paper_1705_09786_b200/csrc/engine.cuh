@@ -1320,7 +1320,7 @@ __device__ __noinline__ void publish_ctx_block(const Ctx& C, DevPPT& P, TileShar
   int4* dst = reinterpret_cast<int4*>(P.ctxblk + (batch & (BATCH_BLOCKS - 1)));
   for (int i = lane; i < (int)(sizeof(BatchCtx) / 16); i += 32) dst[i] = src[i];
   __syncwarp();
-  if (lane == 0) { __threadfence(); st_rel(P.batch_pub, batch + 1u); }
+  if (lane == 0) st_rel(P.batch_pub, batch + 1u);     // the release store is cumulative over the warp barrier above
   __syncwarp();
 }
 
@@ -1938,7 +1938,7 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int whi
     __syncthreads();
     EMIT_PHASE(5);
     if (tid == 0) S.phase[6] += 1ull;
-    if (tid == 0) { __threadfence(); st_rel(&P.emit_done[which], my_batch + 1u); }
+    if (tid == 0) st_rel(&P.emit_done[which], my_batch + 1u);          // after the block barrier above
     my_batch += (unsigned)P.G;
   }
   __syncthreads();
