@@ -1900,39 +1900,48 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int whi
   long long tp = clock64();
 #define EMIT_PHASE(k) do { if (tid == 0) { const long long tn = clock64(); S.phase[k] += (unsigned long long)(tn - tp); tp = tn; } } while (0)
   for (;;) {
-    // every emitter of the tile sees the terminating batch: emit_pub counts all batches, the last one is the marker
-    // A batch is ready once every tile of the node has handed it over (the tiles do not wait for each other).
-    if (tid == 0) S.ok = 1;
-    __syncthreads();
-    if (warp == 0) {
-      const int lane = tid & 31;
-      unsigned it = 0;
-      int state = 0;                                            // 1: the batch is ready, 2: finished, 3: give up
-      while (state == 0) {
-        const unsigned pub = lane < P.T ? ld_acq(&P.emit_pub[lane]) : 0xffffffffu;
-        if (__all_sync(0xffffffffu, pub > my_batch)) state = 1;
-        else {
-          unsigned fin = 0;
-          if (lane == 0) fin = ld_acq(&P.emit_fin[tile]) != 0u && ld_acq(&P.emit_pub[tile]) <= my_batch;
-          if (warp_uniform(fin)) state = 2;
-          else if ((++it & 15u) == 0) {
-            unsigned bad = 0;
-            if (lane == 0) { bad = aborted(C); if (!bad && gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, P.node, 5); bad = 1; } }
-            if (warp_uniform(bad)) state = 3;
+    // (1) As soon as the scheduler has published the batch its context is copied: that overlaps the tiles' work on it.
+    // (2) The batch is emitted once every tile of the node has handed it over (the tiles do not wait for each other).
+    // Both waits end when tile 0 has seen the terminating batch and nothing is left for this emitter.
+    BatchDesc d;
+    bool stop = false;
+    for (int phase = 0; phase < 2 && !stop; phase++) {
+      if (tid == 0) S.ok = 1;
+      __syncthreads();
+      if (warp == 0) {
+        const int lane = tid & 31;
+        unsigned it = 0;
+        int state = 0;                                          // 1: ready, 2: finished, 3: give up
+        while (state == 0) {
+          bool ready;
+          if (phase == 0) { unsigned pub = 0; if (lane == 0) pub = ld_acq(P.batch_pub); ready = warp_uniform(pub) > my_batch; }
+          else { const unsigned pub = lane < P.T ? ld_acq(&P.emit_pub[lane]) : 0xffffffffu; ready = __all_sync(0xffffffffu, pub > my_batch); }
+          if (ready) state = 1;
+          else {
+            unsigned fin = 0;
+            if (lane == 0) fin = ld_acq(&P.emit_fin[tile]) != 0u && ld_acq(&P.emit_pub[tile]) <= my_batch;
+            if (warp_uniform(fin)) state = 2;
+            else if ((++it & 15u) == 0) {
+              unsigned bad = 0;
+              if (lane == 0) { bad = aborted(C); if (!bad && gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, P.node, 5); bad = 1; } }
+              if (warp_uniform(bad)) state = 3;
+            }
+            if (state == 0) __nanosleep(it < 16 ? 20 : 100);
           }
-          if (state == 0) __nanosleep(it < 16 ? 20 : 100);
         }
+        if (lane == 0) S.tail_snap[0] = (unsigned)state;
       }
-      if (lane == 0) S.tail_snap[0] = (unsigned)state;
+      __syncthreads();
+      if (S.tail_snap[0] != 1u) { stop = true; break; }        // finished and nothing left for this emitter, or aborted
+      if (phase == 0) {
+        EMIT_PHASE(3);
+        fetch_ctx_block(P, S, my_batch);
+        __syncthreads();
+        d = S.desc;
+        if (!S.ok || d.pad1) stop = true;
+      }
     }
-    __syncthreads();
-    if (S.tail_snap[0] != 1u) break;                           // finished and nothing left for this emitter, or aborted
-    EMIT_PHASE(3);
-    if (C.sched_ctas) fetch_ctx_block(P, S, my_batch);
-    else if (warp == 0) load_batch_ctx(C, P, S, my_batch);
-    __syncthreads();
-    const BatchDesc d = S.desc;
-    if (!S.ok || d.pad1) break;
+    if (stop) break;
     EMIT_PHASE(4);
     if (d.count > 0) emit_batch(C, P, member, members, S, d, my_batch + 1u, P.stage + (size_t)((my_batch + 1u) % (unsigned)C.depth) * P.stage_floats, acc);
     __syncthreads();
