@@ -1655,27 +1655,12 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           }
           __syncwarp();
         }
-      } else if (tid == 0) {
-        if (!spin_until(C, t0, [&] { return ld_acq(P.batch_pub) > my_batch; })) S.ok = 0;
-      }
-      __syncthreads();
-      if (!S.ok || aborted(C)) { running = false; break; }
-      if (C.sched_ctas) {
-        fetch_ctx_block(P, S, my_batch);
-        if (tile == 0 && tid == 0) st_rel(P.fetched, my_batch + 1u);                 // paces the scheduler
-      } else if (warp == 0) load_batch_ctx(C, P, S, my_batch);
-      __syncthreads();
-      const BatchDesc d = S.desc;
-      my_batch++;
-      AMP_PHASE(d.count > 0 ? 1 : 0);
-      const int count = d.count, dir = d.dir;
-      if (!S.ok || d.pad1) { running = false; break; }
-      float* const stage_k = P.stage + (size_t)(my_batch % (unsigned)C.depth) * P.stage_floats;
-      if (C.emit_ctas && count > 0) {
-        // the per-batch buffers are reused every `depth` batches and read by the emitters of every tile: wait until all
-        // of them are done with the batch that used these buffers before
-        if (warp == 0 && my_batch > (unsigned)C.depth) {
-          const unsigned j = my_batch - 1u - (unsigned)C.depth;
+      } else {
+        if (tid == 0) { if (!spin_until(C, t0, [&] { return ld_acq(P.batch_pub) > my_batch; })) S.ok = 0; }
+        // Meanwhile warp 1 makes sure that the per-batch buffers of this batch are free: they are reused every `depth`
+        // batches and read by the emitters of every tile, all of which must be done with their previous user.
+        if (warp == 1 && C.emit_ctas && my_batch >= (unsigned)C.depth) {
+          const unsigned j = my_batch - (unsigned)C.depth;
           unsigned it = 0;
           for (;;) {
             bool ok = true;
@@ -1690,9 +1675,20 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
             __nanosleep(it < 16 ? 20 : 100);
           }
         }
-        __syncthreads();
-        if (!S.ok) { running = false; break; }
       }
+      __syncthreads();
+      if (!S.ok) { running = false; break; }
+      if (C.sched_ctas) {
+        fetch_ctx_block(P, S, my_batch);
+        if (tile == 0 && tid == 0) st_rel(P.fetched, my_batch + 1u);                 // paces the scheduler
+      } else if (warp == 0) load_batch_ctx(C, P, S, my_batch);
+      __syncthreads();
+      const BatchDesc d = S.desc;
+      my_batch++;
+      AMP_PHASE(d.count > 0 ? 1 : 0);
+      const int count = d.count, dir = d.dir;
+      if (!S.ok || d.pad1) { running = false; break; }
+      float* const stage_k = P.stage + (size_t)(my_batch % (unsigned)C.depth) * P.stage_floats;
       const int nb = S.rowoff[count];
       const bool eval = count > 0 && (S.hdr[0].flags & HDR_EVAL);
       AMP_PHASE(2);
