@@ -940,6 +940,8 @@ struct TileShared : BatchCtx {
   unsigned long long phase[16];
   unsigned long long step[16];
   long long step_t;
+  unsigned long long mbar;             // transaction barrier of the bulk copies that stage a batch's input rows
+  unsigned mbar_parity;
   Frame stack[WARPS][WALK_STACK];
   WalkPool pool;
 };
@@ -1192,6 +1194,31 @@ __device__ __forceinline__ void stage_rows_v(float* __restrict__ Xs, int ldx, co
       }
     }
   }
+}
+// Bulk-copy staging (TMA, untiled): one cp.async.bulk per input row, issued by the row's thread, completion counted in
+// bytes on a shared-memory transaction barrier that every thread then waits for (bounded).  Needs rows that start on 16
+// bytes and are a multiple of 16 bytes long in device memory.  The proxy fence orders the issuing thread's view of the
+// rows (written by other SMs with ordinary stores and acquired through the queues) before the asynchronous read.
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+__device__ __noinline__ void stage_rows_bulk(const Ctx& C, TileShared& S, float* Xs, int ldx, const float* const* rowptr, int nb, int width,
+                                             int node, unsigned long long t0) {
+  const int tid = threadIdx.x;
+  const unsigned bar = smem_u32(&S.mbar), parity = S.mbar_parity;
+  if (tid == 0) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((unsigned)(nb * width * 4)) : "memory");
+  __syncthreads();
+  if (tid < nb) {
+    asm volatile("fence.proxy.async;" ::: "memory");
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(smem_u32(Xs + (size_t)tid * ldx)), "l"(rowptr[tid]), "r"((unsigned)(width * 4)), "r"(bar) : "memory");
+  }
+  unsigned done = 0, spins = 0;
+  for (;;) {
+    asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) break;
+    if ((++spins & 1023u) == 0 && (aborted(C) || gtime() - t0 > C.timeout_ns)) { if (tid == 0) fail(C, ST_TIMEOUT, node, 7); break; }
+  }
+  __syncthreads();
+  if (tid == 0) S.mbar_parity = parity ^ 1u;
 }
 __device__ __noinline__ void stage_rows(float* Xs, int ldx, const float* const* rowptr, int nb, int width, int align_floats) {
   if ((width & 3) == 0 && (align_floats & 3) == 0) stage_rows_v<4>(Xs, ldx, rowptr, nb, width);
@@ -1615,6 +1642,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
   if (tid < 16) { S.phase[tid] = 0; S.step[tid] = 0; }
   if (tid < POOL) S.pool.ready[tid] = 0;
   if (tid == 0) { S.pool.head = S.pool.tail = 0; S.pool.outstanding = 0; }
+  if (tid == 0) { asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&S.mbar)) : "memory"); S.mbar_parity = 0; }
   __syncthreads();
 #define AMP_PHASE(k) do { if (tid == 0) { long long now_ = clock64(); S.phase[k] += (unsigned long long)(now_ - tph); tph = now_; } } while (0)
   long long tph = clock64();
@@ -1696,7 +1724,8 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
 
       if (count > 0 && P.kind == LINEAR) {
         // stage the cached inputs of the batch
-        stage_rows(M.Xs, LX, S.rowptr, nb, in, P.xcache ? in : C.inst.dense_dim);
+        if (((in | (P.xcache ? in : C.inst.dense_dim)) & 3) == 0 && nb <= THREADS) stage_rows_bulk(C, S, M.Xs, LX, S.rowptr, nb, in, P.node, t0);
+        else stage_rows(M.Xs, LX, S.rowptr, nb, in, P.xcache ? in : C.inst.dense_dim);
         if (dir == FWD) {
           __syncthreads();
           tile_xwT(M.Xs, LX, nb, M.Ws, LW, R, in, M.Ys, P.R, M.scratch);
@@ -1729,7 +1758,8 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         const int H = out, SR = P.R, BR = P.BM * P.R, BRD = P.BM * RP;      // Ys arrays: [BM][SR]; D arrays: [BM][RP]
         const float *Wz = M.Ws, *Wr = M.Ws + SR * LW, *Wc = M.Ws + 2 * SR * LW;
         if (tid == 0) S.step_t = clock64();
-        stage_rows(M.Xs, LX, S.rowptr, nb, in, in);
+        if ((in & 3) == 0) stage_rows_bulk(C, S, M.Xs, LX, S.rowptr, nb, in, P.node, t0);
+        else stage_rows(M.Xs, LX, S.rowptr, nb, in, in);
         __syncthreads();
         AMP_STEP(0);
         if (dir == FWD) {
