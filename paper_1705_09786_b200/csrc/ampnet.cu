@@ -75,6 +75,7 @@ struct ampnet_graph {
   void *ctl_mem = nullptr, *bulk_mem = nullptr;
   size_t ctl_cap = 0, bulk_cap = 0;
   std::vector<std::pair<size_t, size_t>> leftover_regions;   // (offset, bytes) inside ctl
+  std::vector<std::pair<void*, size_t>> zero_regions;        // parts of the bulk arena that must start a run at zero
   std::vector<PPTStats*> d_stats;
   std::vector<int*> d_update_log;
   unsigned long long* d_node_msgs = nullptr;
@@ -564,6 +565,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   C.used = B.used = 0;
   if (dry) { C.base = B.base = nullptr; } else { C.base = (char*)g->ctl_mem; B.base = (char*)g->bulk_mem; }
   g->leftover_regions.clear();
+  g->zero_regions.clear();
   auto track = [&](void* p, size_t bytes) { if (!dry) g->leftover_regions.push_back({(size_t)((char*)p - C.base), bytes}); };
   R.nodes = g->hnodes;
   R.ppts.assign(g->ppts.size(), DevPPT{});
@@ -583,7 +585,11 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.om = H.om; P.ov = H.ov; P.opt_t0 = H.opt_t;
     const size_t keys = (size_t)mak * IT * P.U;
     const bool source_fed = g->hnodes[h.pred_node[0]].type == SOURCE;
-    if (!source_fed) P.xcache = B.take<float>(keys * P.rows_max * P.in_dim);
+    P.xld = pad_ldw(P.in_dim);
+    if (!source_fed) {
+      P.xcache = B.take<float>(keys * P.rows_max * P.xld);
+      if (P.xld != P.in_dim && !dry) g->zero_regions.push_back({P.xcache, keys * P.rows_max * P.xld * sizeof(float)});   // the row padding
+    }
     if (H.kind != LOOKUP) P.ycache = B.take<float>(keys * P.rows_max * P.out_dim);
     P.gbuf = B.take<float>(keys * P.rows_max * P.out_dim);
     if (H.kind == GRUCELL) {
@@ -639,7 +645,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
         n.jstride = (long long)n.rows_in * n.out_dim;
         n.jcnt = C.take<int>(kout); track(n.jcnt, kout * sizeof(int));
         const DevNode& s = R.nodes[n.succ_node[0]];
-        if (is_ppt_type(s.type) && R.ppts[s.ppt].xcache && s.U_in == n.U_out && s.rows_in == n.rows_in) { n.jbuf = R.ppts[s.ppt].xcache; n.jalias = 1; }
+        if (is_ppt_type(s.type) && R.ppts[s.ppt].xcache && R.ppts[s.ppt].xld == s.in_dim && s.U_in == n.U_out && s.rows_in == n.rows_in) { n.jbuf = R.ppts[s.ppt].xcache; n.jalias = 1; }
         else n.jbuf = B.take<float>(kout * n.jstride);
       } break;
       case GROUP:
@@ -798,6 +804,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   }
   if ((size_t)R.smem_bytes > (size_t)g->max_smem) return set_err(g, AMPNET_EINVAL, "tile needs %zu bytes of shared memory", R.smem_bytes);
   CUDA_TRY(g, cudaMemsetAsync(g->ctl_mem, 0, g->ctl.used, g->stream));
+  for (auto& z : g->zero_regions) CUDA_TRY(g, cudaMemsetAsync(z.first, 0, z.second, g->stream));
   CUDA_TRY(g, cudaMemsetAsync(R.ctx.slot_inst, 0xFF, (size_t)mak * sizeof(int), g->stream));
   CUDA_TRY(g, cudaMemsetAsync(R.ctx.loss_out, 0, (size_t)std::max<long long>(D.n, 1) * sizeof(float), g->stream));
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.nodes, R.nodes.data(), R.nodes.size() * sizeof(DevNode), cudaMemcpyHostToDevice, g->stream));

@@ -316,8 +316,8 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (lane == 0) ticket = ring_ticket(P.ring[f.dir]);
           if (f.dir == FWD) {
             if (P.xcache) {
-              float* dst = P.xcache + key * (long long)P.rows_max * P.in_dim;
-              if (f.p != dst) warp_copy(dst, P.in_dim, f, f.rows, P.in_dim, lane);
+              float* dst = P.xcache + key * (long long)P.rows_max * P.xld;
+              if (f.p != dst) warp_copy(dst, P.xld, f, f.rows, P.in_dim, lane);
             }
           } else if (n.type != LOOKUP || f.dim > 0) {
             warp_copy(P.gbuf + key * (long long)P.rows_max * P.out_dim, P.out_dim, f, f.rows, P.out_dim, lane);
@@ -1232,7 +1232,7 @@ struct TileMem {           // carve-up of the dynamic shared memory of a tile (f
 };
 
 __device__ __forceinline__ const float* msg_x(const Ctx& C, const DevPPT& P, const Hdr& h, long long key) {
-  if (P.xcache) return P.xcache + key * (long long)P.rows_max * P.in_dim;
+  if (P.xcache) return P.xcache + key * (long long)P.rows_max * P.xld;
   return C.inst.dense + (long long)h.inst * C.inst.dense_dim;         // fed directly by a dense-row source
 }
 
@@ -1299,7 +1299,7 @@ __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared&
     if (total > P.BM) continue;
     if (P.kind != LOOKUP) {
       const float* x0 = msg_x(C, P, h[j], key);
-      for (int r = 0; r < rows[j]; r++) { S.rowmsg[off + r] = i; S.rowptr[off + r] = x0 ? x0 + (size_t)r * in : nullptr; }
+      for (int r = 0; r < rows[j]; r++) { S.rowmsg[off + r] = i; S.rowptr[off + r] = x0 ? x0 + (size_t)r * P.xld : nullptr; }
     } else {                                                // table rows and the rows of the incoming gradient
       const DevInst& I = C.inst;
       const long long base = I.offsets[h[j].inst];
@@ -1724,7 +1724,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
 
       if (count > 0 && P.kind == LINEAR) {
         // stage the cached inputs of the batch
-        if (((in | (P.xcache ? in : C.inst.dense_dim)) & 3) == 0 && nb <= THREADS) stage_rows_bulk(C, S, M.Xs, LX, S.rowptr, nb, in, P.node, t0);
+        if (P.xcache || (in & 3) == 0) stage_rows_bulk(C, S, M.Xs, LX, S.rowptr, nb, P.xcache ? P.xld : in, P.node, t0);
         else stage_rows(M.Xs, LX, S.rowptr, nb, in, P.xcache ? in : C.inst.dense_dim);
         if (dir == FWD) {
           __syncthreads();
@@ -1758,7 +1758,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         const int H = out, SR = P.R, BR = P.BM * P.R, BRD = P.BM * RP;      // Ys arrays: [BM][SR]; D arrays: [BM][RP]
         const float *Wz = M.Ws, *Wr = M.Ws + SR * LW, *Wc = M.Ws + 2 * SR * LW;
         if (tid == 0) S.step_t = clock64();
-        if ((in & 3) == 0) stage_rows_bulk(C, S, M.Xs, LX, S.rowptr, nb, in, P.node, t0);
+        if (P.xcache) stage_rows_bulk(C, S, M.Xs, LX, S.rowptr, nb, P.xld, P.node, t0);
         else stage_rows(M.Xs, LX, S.rowptr, nb, in, in);
         __syncthreads();
         AMP_STEP(0);

@@ -77,7 +77,8 @@ struct DevNode {
 struct DevPPT {
   int node, kind, in_dim, out_dim, act, flags, muf_override, pad0;
   int T, cta0, R, BM;                 // row tiles, first CTA, rows per tile, batch row capacity
-  int U, rows_max, J, pad1;           // key space, max rows per message, ceil(in_dim / 32) bucket
+  int U, rows_max, J, xld;            // key space, max rows per message, ceil(in_dim / 32) bucket, row stride of xcache (in_dim
+                                      // rounded up to 4 floats, padding kept at zero: rows start on 16 bytes for bulk copies)
   float *om, *ov;                     // optimiser state (first / second moment), laid out like W followed by b
   long long opt_t0;                   // updates of this node before the run (Adam's bias correction)
   float *W, *b;                       // LINEAR: W[out][in], b[out]; LOOKUP: W = E[V][d]; GRUCELL: W[3][H][2H], b[3][H]
