@@ -50,6 +50,7 @@ struct HostPPT {
   int T = 1, R = 0, BM = 0, J = 0;
   int NE = 0, G = 1;                    // emitter CTAs of the node and their batch groups
   bool a_global = false;                // the tiles' gradient accumulators live in device memory (frees shared memory for staging rows)
+  int xwt_rb = 8;                       // output rows per pass of X.W^T: 16 where the larger scratch still fits
   double emit_load = 0.0;               // emitter-seconds the node's emission took in the last asynchronous epoch (0: unknown)
   size_t smem_floats = 0;
 };
@@ -392,12 +393,12 @@ unsigned pow2_at_least(unsigned long long v) {
   return p;
 }
 
-size_t tile_smem_floats(const HostPPT& P, int R, int BM, bool a_global = false) {      // mirrors the carve-up at the top of ppt_main
+size_t tile_smem_floats(const HostPPT& P, int R, int BM, bool a_global = false, int xwt_rb = 8) {      // mirrors the carve-up at the top of ppt_main
   if (P.kind == LOOKUP) return 64;
   const size_t LW = (size_t)pad_ldw(P.in), LX = (size_t)pad_ldx(P.in), RP = (size_t)((R + 3) & ~3), nm = (size_t)P.nmat;
   auto p4 = [](size_t v) { return (v + 3) & ~(size_t)3; };
   return (a_global ? 1 : 2) * nm * R * LW + 2 * p4(nm * R) + (size_t)BM * LX * (P.kind == GRUCELL ? 2 : 1) + (nm + 1) * BM * RP + p4(nm * BM * R) +
-         XWT_SCRATCH + 64;
+         xwt_scratch_floats(xwt_rb) + 64;
 }
 
 // Placement: row tiles per PPT node.  Every node starts with the fewest tiles whose weights + accumulators + staging
@@ -483,7 +484,8 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
     if (P.kind != LOOKUP) { P.R = (P.out + P.T - 1) / P.T; P.T = (P.out + P.R - 1) / P.R; P.BM = bm_of[p]; }
-    P.smem_floats = tile_smem_floats(P, P.R, P.BM, P.a_global);
+    P.xwt_rb = (P.kind != LOOKUP && P.R > 8 && tile_smem_floats(P, P.R, P.BM, P.a_global, 16) <= budget) ? 16 : 8;
+    P.smem_floats = tile_smem_floats(P, P.R, P.BM, P.a_global, P.xwt_rb);
     used += P.T;
   }
   if (used > n_ctas) return set_err(g, AMPNET_EINVAL, "placement needs %d CTAs but only %d are available", used, n_ctas);
@@ -557,6 +559,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     if (st != AMPNET_EOVERFLOW) break;
   }
   if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0); }
+  if (st == AMPNET_EOVERFLOW) return set_err(g, AMPNET_EINVAL, "the model needs more CTAs than the %d available (one per row tile + the controller)", n_ctas);
   if (st != AMPNET_OK) return st;
   const int depth = emit_ctas > 0 ? 5 : 2;       // emitters work in up to four batch groups: a tile may be four batches ahead
   R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth; R.ctx.sched_ctas = emit_ctas > 0 ? 1 : 0;
@@ -626,6 +629,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.stats = C.take<PPTStats>(1);
     P.update_log = B.take<int>(g->update_log_cap); P.update_log_cap = g->update_log_cap;
     P.a_global = H.a_global ? 1 : 0;
+    P.xwt_rb = H.xwt_rb;
     if (H.a_global) P.A = C.take<float>((size_t)H.T * H.nmat * H.R * pad_ldw(H.in));
     if (H.kind == LOOKUP) {
       P.A = C.take<float>(H.nW);

@@ -754,7 +754,7 @@ __device__ __forceinline__ float act_grad(int a, float y) {
 // different rows meets no bank conflict), gradient rows D a multiple of 4 (ldd); all padding is kept at zero.
 __host__ __device__ __forceinline__ int pad_ldw(int in) { return (in + 3) & ~3; }
 __host__ __device__ __forceinline__ int pad_ldx(int in) { int l = (in + 3) & ~3; while ((l & 7) != 4) l += 4; return l; }
-constexpr int XWT_SCRATCH = WARPS * 32 * 8;      // floats: partial sums of the k-slices
+__host__ __device__ __forceinline__ int xwt_scratch_floats(int rb) { return WARPS * 32 * rb; }     // partial sums of the k-slices
 
 // out[b][r] = sum_k X[b][k] * W[r][k]  for b < nb, r < R (whole CTA; ends with a block barrier).  Lanes own batch rows:
 // warp (g, s) takes the 32 batch rows of group g and the k-slice s, keeps RB outputs per lane in registers, reads its row
@@ -786,11 +786,13 @@ __device__ __forceinline__ void xwT_pass(const float* __restrict__ Xs, int ldx, 
   }
 }
 __device__ __noinline__ void tile_xwT(const float* __restrict__ Xs, int ldx, int nb, const float* __restrict__ Ws, int ldw, int R,
-                                      int in_dim, float* __restrict__ out, int ldo, float* __restrict__ scratch) {
+                                      int in_dim, float* __restrict__ out, int ldo, float* __restrict__ scratch, int rb_max) {
   const int G = nb > 32 ? 2 : 1, S = WARPS / G, K4 = (in_dim + 3) >> 2;
-  for (int r0 = 0; r0 < R; r0 += 8) {
-    const int rb = min(8, R - r0), RBs = rb > 4 ? 8 : 4;
-    if (rb > 4) xwT_pass<8>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
+  for (int r0 = 0; r0 < R; r0 += rb_max) {                 // up to rb_max (8 or 16) output rows per pass over the staged inputs
+    const int rb = min(rb_max, R - r0), RBs = rb > 12 ? 16 : rb > 8 ? 12 : rb > 4 ? 8 : 4;
+    if (RBs == 16) xwT_pass<16>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
+    else if (RBs == 12) xwT_pass<12>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
+    else if (RBs == 8) xwT_pass<8>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
     else xwT_pass<4>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
     __syncthreads();
     for (int idx = threadIdx.x; idx < nb * rb; idx += THREADS) {
@@ -1619,7 +1621,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
     M.Xs = p; p += (size_t)P.BM * M.LX;
     M.Ds = p; p += (size_t)(nmat + 1) * P.BM * M.RP;
     M.Ys = p; p += ((size_t)nmat * P.BM * P.R + 3) & ~(size_t)3;
-    M.scratch = p; p += XWT_SCRATCH;
+    M.scratch = p; p += xwt_scratch_floats(P.xwt_rb);
     M.XC = p; p += P.kind == GRUCELL ? (size_t)P.BM * M.LX : 0;
     if (P.kind != LOOKUP) for (float* q = smem + tid; q < p; q += THREADS) *q = 0.f;     // the padding stays zero
   }
@@ -1728,7 +1730,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         else stage_rows(M.Xs, LX, S.rowptr, nb, in, P.xcache ? in : C.inst.dense_dim);
         if (dir == FWD) {
           __syncthreads();
-          tile_xwT(M.Xs, LX, nb, M.Ws, LW, R, in, M.Ys, P.R, M.scratch);
+          tile_xwT(M.Xs, LX, nb, M.Ws, LW, R, in, M.Ys, P.R, M.scratch, P.xwt_rb);
           __syncthreads();
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
@@ -1764,8 +1766,8 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
         AMP_STEP(0);
         if (dir == FWD) {
           // phase 1: gates z, r for the tile's rows
-          tile_xwT(M.Xs, LX, nb, Wz, LW, R, in, M.Ys, SR, M.scratch);
-          tile_xwT(M.Xs, LX, nb, Wr, LW, R, in, M.Ys + BR, SR, M.scratch);
+          tile_xwT(M.Xs, LX, nb, Wz, LW, R, in, M.Ys, SR, M.scratch, P.xwt_rb);
+          tile_xwT(M.Xs, LX, nb, Wr, LW, R, in, M.Ys + BR, SR, M.scratch, P.xwt_rb);
           __syncthreads();
           for (int idx = tid; idx < nb * R; idx += THREADS) {
             const int b = idx / R, r = idx - b * R, m = S.rowmsg[b];
@@ -1784,7 +1786,7 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
           gru_gated_input(P, S, M.Xs, M.XC, LX, nb);
           __syncthreads();
           AMP_STEP(3);
-          tile_xwT(M.XC, LX, nb, Wc, LW, R, in, M.Ys + 2 * BR, SR, M.scratch);
+          tile_xwT(M.XC, LX, nb, Wc, LW, R, in, M.Ys + 2 * BR, SR, M.scratch, P.xwt_rb);
           __syncthreads();
           AMP_STEP(4);
           for (int idx = tid; idx < nb * R; idx += THREADS) {

@@ -84,7 +84,7 @@ struct DevPPT {
   float *W, *b;                       // LINEAR: W[out][in], b[out]; LOOKUP: W = E[V][d]; GRUCELL: W[3][H][2H], b[3][H]
   float* A;                           // LOOKUP: accumulator [V][d] in device memory; a node whose tiles keep their accumulators in
                                       // device memory (a_global): [tile][nmat][R][ldw]
-  int a_global, pad2;
+  int a_global, xwt_rb;               // xwt_rb: output rows per pass of X.W^T (8 or 16; sizes the k-slice scratch)
   int *touched_flag, *touched_list, *touched_n;
   float *xcache, *ycache, *gbuf;      // [key][rows_max][in | out | out]
   float *zc, *rc, *cc;                // GRUCELL caches [key][rows_max][H]
