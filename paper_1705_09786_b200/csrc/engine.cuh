@@ -943,6 +943,7 @@ struct TileShared : BatchCtx {
   unsigned long long step[16];
   long long step_t;
   unsigned long long mbar;             // transaction barrier of the bulk copies that stage a batch's input rows
+  int mylist[MAX_BATCH_ROWS], mycount; // embedding node: the batch rows this tile handles
   unsigned mbar_parity;
   Frame stack[WARPS][WALK_STACK];
   WalkPool pool;
@@ -1473,35 +1474,45 @@ struct OptStep {
 __device__ __noinline__ void lookup_batch(DevPPT& P, TileShared& S, const int dir, const int nb, float* stage_k, const int tile) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, out = P.out_dim, T = P.T;
   int* const tlist = P.touched_list + (size_t)tile * ((P.in_dim + T - 1) / T);
-  constexpr int K = 5;                                      // column chunks of 32 per pass
+  constexpr int K = 10;                                     // column chunks of 32 per pass: a 320-wide row in one round trip
+  // the batch rows this tile handles (forward: rows whose table row it owns; backward: the owned chain heads), compacted
+  if (warp == 0) {
+    int n = 0;
+    for (int b0 = 0; b0 < nb; b0 += 32) {
+      const int b = b0 + lane;
+      bool m = false;
+      if (b < nb) {
+        const int id = S.rowid[b];
+        m = dir == FWD ? (id >= 0 ? id % T == tile : tile == 0) : (S.rowfirst[b] && id % T == tile);     // rows outside the table read as zero
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, m);
+      if (m) S.mylist[n + __popc(bal & ((1u << lane) - 1u))] = b;
+      n += __popc(bal);
+    }
+    if (lane == 0) S.mycount = n;
+  }
+  __syncthreads();
+  const int mine = S.mycount;
   if (dir == FWD) {
-    for (int b0 = warp * 2; b0 < nb; b0 += WARPS * 2)       // two rows per pass
+    for (int k0 = warp; k0 < mine; k0 += WARPS) {
+      const int b = S.mylist[k0], id = S.rowid[b];
       for (int c0 = 0; c0 < out; c0 += 32 * K) {
-        float v[2][K];
-        bool mine[2];
+        float v[K];
 #pragma unroll
-        for (int r = 0; r < 2; r++) {
-          const int id = b0 + r < nb ? S.rowid[b0 + r] : -1;
-          mine[r] = b0 + r < nb && (id >= 0 ? id % T == tile : tile == 0);      // rows outside the table read as zero
-#pragma unroll
-          for (int k = 0; k < K; k++) {
-            const int c = c0 + k * 32 + lane;
-            v[r][k] = (mine[r] && id >= 0 && c < out) ? P.W[(size_t)id * out + c] : 0.f;
-          }
+        for (int k = 0; k < K; k++) {
+          const int c = c0 + k * 32 + lane;
+          v[k] = (id >= 0 && c < out) ? P.W[(size_t)id * out + c] : 0.f;
         }
 #pragma unroll
-        for (int r = 0; r < 2; r++)
-#pragma unroll
-          for (int k = 0; k < K; k++) {
-            const int c = c0 + k * 32 + lane;
-            if (mine[r] && c < out) stage_k[(size_t)(b0 + r) * out + c] = emit_round(v[r][k]);
-          }
+        for (int k = 0; k < K; k++) {
+          const int c = c0 + k * 32 + lane;
+          if (c < out) stage_k[(size_t)b * out + c] = emit_round(v[k]);
+        }
       }
+    }
   } else {
-    for (int b = warp; b < nb; b += WARPS) {
-      if (!S.rowfirst[b]) continue;
-      const int id = S.rowid[b];
-      if (id % T != tile) continue;
+    for (int k0 = warp; k0 < mine; k0 += WARPS) {
+      const int b = S.mylist[k0], id = S.rowid[b];
       int fresh = 0;
       if (lane == 0) fresh = !P.touched_flag[id];
       float* arow = P.A + (size_t)id * out;
