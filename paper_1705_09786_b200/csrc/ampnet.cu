@@ -574,7 +574,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   R.ppts.assign(g->ppts.size(), DevPPT{});
   g->d_stats.assign(g->ppts.size(), nullptr);
   g->d_update_log.assign(g->ppts.size(), nullptr);
-  size_t max_smem_floats = 64;
+  size_t max_smem_floats = 2048;        // at least the two batch slots of a scheduler CTA
   int cta = 1;
   for (size_t p = 0; p < g->ppts.size(); p++) {
     const HostPPT& H = g->ppts[p];
@@ -847,8 +847,8 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
             G.role_cycles[2] * us, G.role_cycles[3] * us, G.role_cycles[4] * us, G.role_cycles[5]);
     for (size_t p = 0; p < g->ppts.size(); p++) {
       const unsigned long long* r = G.role_cycles + 8 + 8 * p;
-      fprintf(stderr, "[role] node %2d sched us: wait-tile %.0f no-msg %.0f form %.0f | emitter(0,0) us: wait %.0f load %.0f emit %.0f batches %llu\n",
-              g->ppts[p].node, r[0] * us, r[1] * us, r[2] * us, r[3] * us, r[4] * us, r[5] * us, r[6]);
+      fprintf(stderr, "[role] node %2d sched us: wait-tile %.0f no-msg %.0f form %.0f (context %.0f) | emitter(0,0) us: wait %.0f load %.0f emit %.0f batches %llu\n",
+              g->ppts[p].node, r[0] * us, r[1] * us, r[2] * us, r[7] * us, r[3] * us, r[4] * us, r[5] * us, r[6]);
     }
     for (size_t p = 0; p < g->ppts.size(); p++) {
       fprintf(stderr, "[step] node %2d us:", g->ppts[p].node);

@@ -22,6 +22,14 @@ __device__ __forceinline__ unsigned ld_acq(const unsigned* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+// Several independent flags polled at once: relaxed loads overlap in flight where acquire loads would not; one fence
+// after them orders everything read afterwards behind all of them.
+__device__ __forceinline__ unsigned ld_rlx(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_acq() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
 __device__ __forceinline__ void st_rel(unsigned* p, unsigned v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
@@ -929,7 +937,6 @@ __device__ __noinline__ void tile_accum(const float* __restrict__ Ds, int ldd, i
 struct LeaderState {
   unsigned head[2], sched_w, batch_w;
   int n_acc, version, log_n;
-  int ver_form;                        // version when the last batch was formed (staleness is accounted after it is published)
   unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows;
 };
 
@@ -948,6 +955,16 @@ struct TileShared : BatchCtx {
   Frame stack[WARPS][WALK_STACK];
   WalkPool pool;
 };
+// Scheduler CTA: a batch formed by warp 0 waits here for warp 1, which assembles and publishes its context while warp 0
+// polls for the next one.  full = batch number + 1 while occupied (shared memory, written behind a block-level fence).
+struct SchedSlot {
+  BatchDesc desc;
+  int ver_form;
+  unsigned full;
+  int pad[2];
+  Hdr hdr[MAX_BATCH_MSGS];
+};
+static_assert(2 * sizeof(SchedSlot) <= 2048 * sizeof(float), "the launch reserves 2048 floats of dynamic shared memory at least");
 #define AMP_STEP(k) do { if (threadIdx.x == 0) { const long long n_ = clock64(); S.step[k] += (unsigned long long)(n_ - S.step_t); S.step_t = n_; } } while (0)
 
 __device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) {
@@ -968,7 +985,8 @@ __device__ __forceinline__ unsigned long long ballot64(const bool p0, const bool
 // Warp 0 of the leader: take up to 64 candidate messages (two ring slots per lane, in processing order: candidate
 // lane and candidate lane + 32), cut the batch at the row capacity and at the message that triggers an update (Sec. 3),
 // publish it.  Returns the number of messages taken.
-__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, const unsigned (&slot)[2], int ncand) {
+__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, int dir, const unsigned (&slot)[2], int ncand,
+                                       SchedSlot* q = nullptr) {
   const int lane = threadIdx.x & 31;
   Ring& R = P.ring[dir];
   Hdr h[2];
@@ -1006,7 +1024,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
     const int i = lane + 32 * j;
     if (i >= take) continue;
     P.sched[(S.ls.sched_w + i) & P.sched_mask] = slot[j];
-    if (C.sched_ctas) S.hdr[i] = h[j];                 // the scheduler CTA assembles the batch context from its own copy
+    if (q) q->hdr[i] = h[j];                           // the scheduler CTA assembles the batch context from its own copy
     else if (!C.det) {
       int4* b = reinterpret_cast<int4*>(&P.bhdr[(S.ls.batch_w & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + i]);
       b[0] = make_int4(h[j].inst, h[j].seq, h[j].slot, h[j].it);
@@ -1016,7 +1034,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
       long long key = key_of(C, P.node, h[j].slot, h[j].it, h[j].u, P.U);
       if (key >= 0) {
         if (dir == FWD) P.vcache[key] = S.ls.version;
-        else if (!C.sched_ctas) {             // a scheduler CTA accounts staleness after it has published the batch
+        else if (!q) {                        // a scheduler CTA accounts staleness after it has published the batch
           int s = S.ls.version - P.vcache[key];
           if (s < 0) s = 0;
           atomicAdd(&S.stale_hist[s > 63 ? 63 : s], 1ull);
@@ -1027,11 +1045,10 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
   }
   __syncwarp();
   if (lane == 0) {
-    S.ls.ver_form = S.ls.version;
     BatchDesc d;
     d.sched_start = S.ls.sched_w; d.count = take; d.dir = dir; d.flags = upd ? BATCH_UPDATE : 0;
     d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.upd_t = upd ? (int)S.ls.n_updates + 1 : 0; d.pad1 = 0;
-    if (C.sched_ctas) S.desc = d;                      // a scheduler CTA publishes the assembled context instead
+    if (q) { q->desc = d; q->ver_form = S.ls.version; }   // a scheduler CTA publishes the assembled context instead
     else { P.batches[S.ls.batch_w & P.batch_mask] = d; __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
     S.ls.batch_w++;
     S.ls.sched_w += take;
@@ -1047,7 +1064,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
   return take;
 }
 
-__device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags) {   // one thread
+__device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags, SchedSlot* q = nullptr) {   // one thread
   BatchDesc d;
   d.sched_start = S.ls.sched_w; d.count = 0; d.dir = BWD; d.flags = flags; d.n_upd = 0; d.nrows = 0; d.upd_t = d.pad1 = 0;
   if ((flags & BATCH_TERMINATE) && S.ls.n_acc > 0 && !C.eval) {      // epoch-end flush of the leftover gradients
@@ -1057,24 +1074,35 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
     st.log_n++; st.n_updates++; st.n_grads_applied += d.n_upd;
     S.ls.n_acc = 0; S.ls.version++;
   }
-  if (C.sched_ctas) S.desc = d;
+  if (q) { q->desc = d; q->ver_form = S.ls.version; }
   else { P.batches[S.ls.batch_w & P.batch_mask] = d; __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
   S.ls.batch_w++;
 }
 
 // Asynchronous mode, warp 0 of the leader: whatever is pending, backward first (App. A).
-__device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S) {
+// gate (optional): a counter read together with the ring polls; the call does nothing and returns false with *open = 0
+// while gate + 1 < gate_min (the scheduler's look-ahead limit).
+__device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileShared& S, const unsigned* gate = nullptr,
+                                                 unsigned gate_min = 0, bool* open = nullptr, SchedSlot* q = nullptr) {
   const int lane = threadIdx.x & 31;
   unsigned slot[2][2];
   bool mready[2][2];
+  unsigned gv = 0;
+  if (gate && lane == 0) gv = ld_rlx(gate);
 #pragma unroll
   for (int dir = 0; dir < 2; dir++)               // both rings are polled before either result is needed
 #pragma unroll
     for (int j = 0; j < 2; j++) {
       const unsigned t = S.ls.head[dir] + lane + 32 * j;
       slot[dir][j] = t & P.ring[dir].mask;
-      mready[dir][j] = ld_acq(&P.ring[dir].seq[slot[dir][j]]) == t + 1u;
+      mready[dir][j] = ld_rlx(&P.ring[dir].seq[slot[dir][j]]) == t + 1u;
     }
+  fence_acq();
+  if (gate) {
+    const bool go = warp_uniform(gv) + 1u >= gate_min;
+    *open = go;
+    if (!go) return false;
+  }
   int nready[2];
 #pragma unroll
   for (int dir = 0; dir < 2; dir++) {
@@ -1089,7 +1117,7 @@ __device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileSh
     const int dir = (k == 0) == fwd_first ? FWD : BWD;
     const int n = nready[dir];
     if (n == 0) continue;
-    int take = dir == FWD ? form_batch(C, P, S, FWD, slot[FWD], n) : form_batch(C, P, S, BWD, slot[BWD], n);
+    int take = dir == FWD ? form_batch(C, P, S, FWD, slot[FWD], n, q) : form_batch(C, P, S, BWD, slot[BWD], n, q);
     if (lane == 0) S.ls.head[dir] += take;
     __syncwarp();
     return true;
@@ -1097,7 +1125,7 @@ __device__ __noinline__ bool leader_try_schedule(const Ctx& C, DevPPT& P, TileSh
   unsigned fin = 0;
   if (lane == 0) fin = ld_acq(&C.g->done);
   if (warp_uniform(fin)) {
-    if (lane == 0) publish_marker(C, P, S, BATCH_TERMINATE);
+    if (lane == 0) publish_marker(C, P, S, BATCH_TERMINATE, q);
     __syncwarp();
     return true;
   }
@@ -1259,12 +1287,13 @@ __device__ __forceinline__ void init_leader_state(TileShared& S) {              
 }
 
 // Warp 0 of a CTA: descriptor, headers, keys, row offsets and row pointers of batch `batch` into shared memory.
-// local: descriptor and headers are already in this CTA's shared memory (the scheduler CTA that has just formed the batch).
-__device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared& S, const unsigned my_batch, const bool local = false) {
+// q: descriptor and headers are already in this CTA's shared memory (the scheduler CTA that has just formed the batch).
+__device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared& S, const unsigned my_batch, const SchedSlot* q = nullptr) {
+  const bool local = q != nullptr;
   const int lane = threadIdx.x & 31;
   const int in = P.in_dim;
   int4 d0, d1;
-  if (local) { const int4* dp = reinterpret_cast<const int4*>(&S.desc); d0 = dp[0]; d1 = dp[1]; }
+  if (local) { const int4* dp = reinterpret_cast<const int4*>(&q->desc); d0 = dp[0]; d1 = dp[1]; }
   else { const int4* dp = reinterpret_cast<const int4*>(&P.batches[my_batch & P.batch_mask]); d0 = __ldcg(dp); d1 = __ldcg(dp + 1); }
   const int cnt = d0.y, ddir = d0.z;
   Hdr h[2];
@@ -1274,7 +1303,7 @@ __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared&
     const int i = lane + 32 * j;
     int4 ha = make_int4(0, 0, 0, 0), hb = make_int4(0, 0, 0, 0);
     if (local) {
-      if (i < cnt) { const int4* e = reinterpret_cast<const int4*>(&S.hdr[i]); ha = e[0]; hb = e[1]; }
+      if (i < cnt) { const int4* e = reinterpret_cast<const int4*>(&q->hdr[i]); ha = e[0]; hb = e[1]; }
     } else if (!C.det) {                                    // headers travel with the descriptor: load both at once
       const int4* e = reinterpret_cast<const int4*>(&P.bhdr[(my_batch & (BATCH_BLOCKS - 1)) * MAX_BATCH_MSGS + i]);
       ha = __ldcg(e); hb = __ldcg(e + 1);
@@ -1341,10 +1370,10 @@ __device__ __forceinline__ void fetch_ctx_block(const DevPPT& P, TileShared& S, 
   int4* dst = reinterpret_cast<int4*>(static_cast<BatchCtx*>(&S));
   for (int i = threadIdx.x; i < (int)(sizeof(BatchCtx) / 16); i += THREADS) dst[i] = __ldcg(src + i);
 }
-// Scheduler CTA, warp 0: assemble the context of the batch just formed and publish it.
-__device__ __noinline__ void publish_ctx_block(const Ctx& C, DevPPT& P, TileShared& S, const unsigned batch) {
+// Scheduler CTA, one warp: assemble the context of the batch formed into slot q and publish it.
+__device__ __noinline__ void publish_ctx_block(const Ctx& C, DevPPT& P, TileShared& S, const unsigned batch, const SchedSlot* q) {
   const int lane = threadIdx.x & 31;
-  load_batch_ctx(C, P, S, batch, true);
+  load_batch_ctx(C, P, S, batch, q);
   __syncwarp();
   const int4* src = reinterpret_cast<const int4*>(static_cast<BatchCtx*>(&S));
   int4* dst = reinterpret_cast<int4*>(P.ctxblk + (batch & (BATCH_BLOCKS - 1)));
@@ -1997,41 +2026,35 @@ __device__ __noinline__ void emitter_main(const Ctx& C, DevPPT& P, const int whi
 // scheduler CTA (asynchronous mode): the leader of one PPT node on an SM of its own.  It forms the next micro-batch
 // as soon as tile 0 has fetched the previous one, so that batch formation overlaps the tiles' work.
 // ------------------------------------------------------------------------------------------------
-__device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared& S, const unsigned long long t0) {
+__device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared& S, float* smem, const unsigned long long t0) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  SchedSlot* const Q = reinterpret_cast<SchedSlot*>(smem);
   init_leader_state(S);
+  if (tid < 2) Q[tid].full = 0u;
   __syncthreads();
-  if (warp == 0) {
+  unsigned long long* const rc = C.g->role_cycles + 8 + 8 * (int)(&P - g_ppts);
+  if (warp == 0) {                       // polls the rings and forms batches, at most two ahead of what tile 0 has fetched
     unsigned it = 0;
-    unsigned long long* const rc = C.g->role_cycles + 8 + 8 * (int)(&P - g_ppts);
     long long tp = clock64();
     unsigned long long rcl[3] = {0, 0, 0};
     for (;;) {
-      // at most two batches ahead of what tile 0 has fetched
-      unsigned go = 0, bw = 0;
-      if (lane == 0) { bw = S.ls.batch_w; go = ld_acq(P.fetched) + 1u >= bw; }
+      unsigned bw = 0, busy = 0;
+      if (lane == 0) { bw = S.ls.batch_w; busy = *reinterpret_cast<volatile unsigned*>(&Q[bw & 1u].full); }
       bw = warp_uniform(bw);
-      bool progressed = false;
-      const bool gow = warp_uniform(go);
-      if (gow) progressed = leader_try_schedule(C, P, S);
+      SchedSlot* const q = &Q[bw & 1u];
+      bool gow = false, progressed = false;
+      if (!warp_uniform(busy)) progressed = leader_try_schedule(C, P, S, P.fetched, bw, &gow, q);
+      unsigned fin = 0;
       if (progressed) {
-        publish_ctx_block(C, P, S, bw);
-        if (S.desc.dir == BWD && S.desc.count > 0 && !(S.hdr[0].flags & HDR_EVAL)) {     // staleness of the batch just published
-          for (int i = lane; i < S.desc.count; i += 32) {
-            int st = S.ls.ver_form - P.vcache[S.key[i]];
-            if (st < 0) st = 0;
-            atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
-            atomicMax(&S.max_stale, st);
-          }
-          __syncwarp();
+        __syncwarp();
+        if (lane == 0) {
+          fin = q->desc.flags & BATCH_TERMINATE;
+          __threadfence_block();
+          *reinterpret_cast<volatile unsigned*>(&q->full) = bw + 1u;
         }
       }
       if (lane == 0) { const long long tn = clock64(); rcl[!gow ? 0 : progressed ? 2 : 1] += (unsigned long long)(tn - tp); tp = tn; }
-      if (gow) {
-        unsigned fin = 0;
-        if (lane == 0) fin = progressed && (S.desc.flags & BATCH_TERMINATE);
-        if (warp_uniform(fin)) break;
-      }
+      if (warp_uniform(fin)) break;
       if (progressed) { it = 0; continue; }
       if ((++it & 15u) == 0) {
         if (aborted_warp(C)) break;
@@ -2042,6 +2065,48 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
       __nanosleep(it < 16 ? 20 : 100);
     }
     if (lane == 0) { rc[0] = rcl[0]; rc[1] = rcl[1]; rc[2] = rcl[2]; }
+  } else if (warp == 1) {                // assembles and publishes the contexts, in batch order
+    unsigned long long busy_cycles = 0;
+    for (unsigned b = 0;; b++) {
+      SchedSlot* const q = &Q[b & 1u];
+      unsigned it = 0, stop = 0;
+      for (;;) {
+        unsigned f = 0;
+        if (lane == 0) f = *reinterpret_cast<volatile unsigned*>(&q->full) == b + 1u;
+        if (warp_uniform(f)) break;
+        if ((++it & 63u) == 0) {
+          if (aborted_warp(C)) { stop = 1; break; }
+          unsigned late = 0;
+          if (lane == 0) late = gtime() - t0 > C.timeout_ns;
+          if (warp_uniform(late)) { if (lane == 0) fail(C, ST_TIMEOUT, P.node, 8); stop = 1; break; }
+        }
+        __nanosleep(20);
+      }
+      if (stop) break;
+      __threadfence_block();
+      long long tf = 0;
+      if (lane == 0) tf = clock64();
+      publish_ctx_block(C, P, S, b, q);
+      if (S.desc.dir == BWD && S.desc.count > 0 && !(S.hdr[0].flags & HDR_EVAL)) {     // staleness of the batch just published
+        const int ver = q->ver_form;
+        for (int i = lane; i < S.desc.count; i += 32) {
+          int st = ver - P.vcache[S.key[i]];
+          if (st < 0) st = 0;
+          atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
+          atomicMax(&S.max_stale, st);
+        }
+      }
+      __syncwarp();
+      unsigned fin = 0;
+      if (lane == 0) {
+        fin = q->desc.flags & BATCH_TERMINATE;
+        __threadfence_block();
+        *reinterpret_cast<volatile unsigned*>(&q->full) = 0u;
+        busy_cycles += (unsigned long long)(clock64() - tf);
+      }
+      if (warp_uniform(fin)) break;
+    }
+    if (lane == 0) rc[7] = busy_cycles;
   }
   __syncthreads();
   write_leader_stats(P, S);
@@ -2290,7 +2355,7 @@ __global__ void __launch_bounds__(THREADS, 1) ampnet_engine(const __grid_constan
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);
   else if (role.kind == 1) emitter_main(C, g_ppts[role.ppt], role.pad, SU.t, t0);
-  else if (role.kind == 2) scheduler_main(C, g_ppts[role.ppt], SU.t, t0);
+  else if (role.kind == 2) scheduler_main(C, g_ppts[role.ppt], SU.t, dyn_smem, t0);
   else ppt_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
 }
 
