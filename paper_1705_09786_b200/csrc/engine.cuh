@@ -2033,7 +2033,10 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
   if (tid < 2) Q[tid].full = 0u;
   __syncthreads();
   unsigned long long* const rc = C.g->role_cycles + 8 + 8 * (int)(&P - g_ppts);
-  if (warp == 0) {                       // polls the rings and forms batches, at most two ahead of what tile 0 has fetched
+  // Warp 0 polls the rings and forms batches, one ahead of the batch tile 0 is working on: the batch is formed as late
+  // as still keeps the tile fed, so that messages arriving meanwhile join it (a second batch of look-ahead adds a tile
+  // cycle to every hop; AMPNET_TUNE bit 256 restores it).
+  if (warp == 0) {
     unsigned it = 0;
     long long tp = clock64();
     unsigned long long rcl[3] = {0, 0, 0};
@@ -2043,7 +2046,7 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
       bw = warp_uniform(bw);
       SchedSlot* const q = &Q[bw & 1u];
       bool gow = false, progressed = false;
-      if (!warp_uniform(busy)) progressed = leader_try_schedule(C, P, S, P.fetched, bw, &gow, q);
+      if (!warp_uniform(busy)) progressed = leader_try_schedule(C, P, S, P.fetched, bw + ((C.tune & 256) ? 0u : 1u), &gow, q);
       unsigned fin = 0;
       if (progressed) {
         __syncwarp();
