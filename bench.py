@@ -39,6 +39,7 @@ WORKLOADS = {
                50000, 64, 64, 0.01),
 }
 STRESS_BENCH_INSTANCES = 1000     # the stress workload is timed on a prefix of this many trees per step
+BASELINE_CONFIGS = ("mlp", "rnn", "tree", "ggnn", "stress")      # the five configurations of the benchmark set
 SWEEP_MAK = (1, 8, 64, 256, 1024)
 SWEEP_MUF = (1, 64, 1024)
 GGNN_BENCH_INSTANCES = 20000      # the graph workload is timed on a prefix of this many graphs per step
@@ -285,6 +286,34 @@ def run_ours(args):
     rate_one_key = n1 / st1.seconds
     eng.load_instances(inst)
 
+    # ---- the other configurations of the benchmark set, briefly (single GPU only): same timing rules, fewer steps ----
+    others = None
+    if world == 1 and not args.no_other_configs and args.instances is None:
+        eng.close()
+        eng = None
+        others = {}
+        for name in BASELINE_CONFIGS:
+            if name == args.workload:
+                continue
+            g2, inst2, cfg2 = make_workload(name, rank)
+            e2 = amp.Engine(g2, device=local, payload_bf16=cfg2["bf16"])
+            e2.load_instances(inst2)
+            e2.set_params(wp.init_params(g2))
+            ks, ms = [], 0
+            for k in range(3 + 2):                               # three warm-up epochs, two timed
+                flush_buf.fill_(1)
+                st2, _ = e2.run_epoch(mak=cfg2["mak"], muf=cfg2["muf"], lr=cfg2["lr"], deterministic=False,
+                                      timeout_s=args.timeout, want_loss=False)
+                if k >= 3:
+                    ks.append(st2.seconds); ms += st2.node_messages
+            fl = rf.algorithmic_flops(g2, inst2, {n: e2.node_stats(n)["n_updates"] for n in g2.ppt_nodes()})
+            others[name] = {"instances_per_s": 2 * inst2.n / sum(ks), "node_messages_per_s": ms / sum(ks),
+                            "tflops": fl / (sum(ks) / 2) / 1e12, "instances_per_step": int(inst2.n),
+                            "full_dataset_instances": cfg2["full"], "max_active_keys": cfg2["mak"],
+                            "min_update_frequency": cfg2["muf"], "steps": 2, "warmup": 3,
+                            "timing": "device time of the persistent kernel (CUDA events around the launch)"}
+            e2.close()
+
     sweep = None
     if args.sweep and rank == 0:
         # max_active_keys x min_update_frequency grid on a prefix (one epoch each, parameters reset)
@@ -350,8 +379,13 @@ def run_ours(args):
                           "micro_batch_split": {"fma": 1.0, "tensor_core": 0.0}}}
         if sweep is not None:
             line["sweep"] = sweep
+        if others is not None:
+            for o in others.values():
+                o["frac_of_fma_peak"] = o["tflops"] / peak_tf
+            line["other_configs"] = others
         print(json.dumps(line), flush=True)
-    eng.close()
+    if eng is not None:
+        eng.close()
     import torch.distributed as dist
     if dist.is_initialized():
         dist.destroy_process_group()
@@ -367,6 +401,7 @@ def main():
     ap.add_argument("--instances", type=int, default=None, help="instances per step (default: the workload's size)")
     ap.add_argument("--timeout", type=float, default=300.0, help="bound on one device run, seconds")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the brief runs of the other configurations")
     ap.add_argument("--sweep", action="store_true", help="also run the max_active_keys x min_update_frequency grid")
     args = ap.parse_args()
     if args.impl == "reference":
