@@ -637,11 +637,18 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     P.update_log = B.take<int>(g->update_log_cap); P.update_log_cap = g->update_log_cap;
     P.a_global = H.a_global ? 1 : 0;
     P.xwt_rb = H.xwt_rb;
-    if (H.a_global) P.A = C.take<float>((size_t)H.T * H.nmat * H.R * pad_ldw(H.in));
+    // accumulators kept in device memory start every run at zero; they live beside the caches so that the control arena
+    // stays small (queues and counters only)
+    auto zeroed = [&](size_t n_floats) {
+      float* a = B.take<float>(n_floats);
+      if (!dry) g->zero_regions.push_back({a, n_floats * sizeof(float)});
+      return a;
+    };
+    if (H.a_global) P.A = zeroed((size_t)H.T * H.nmat * H.R * pad_ldw(H.in));
     if (H.kind == LOOKUP) {
-      P.A = C.take<float>(H.nW);
-      P.touched_flag = C.take<int>(H.in);
-      P.touched_list = C.take<int>((size_t)H.in + H.T);      // one segment of ceil(V / T) entries per tile
+      P.A = zeroed(H.nW);
+      P.touched_flag = reinterpret_cast<int*>(zeroed(H.in));
+      P.touched_list = reinterpret_cast<int*>(zeroed((size_t)H.in + H.T));      // one segment of ceil(V / T) entries per tile
       P.touched_n = C.take<int>(H.T);
     }
     P.smem_floats = (int)H.smem_floats;
@@ -814,6 +821,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   const bool ctl_own = g->ctl_cand[0] && (g->ctl_mem == g->ctl_cand[0] || g->ctl_mem == g->ctl_cand[1]);
   const bool ctl_trial = ctl_own && g->ctl_choice < 0 && !det && !eval && !getenv("AMPNET_NO_ARENA_TRIAL");
   if (ctl_own) g->ctl_mem = g->ctl_cand[g->ctl_choice >= 0 ? g->ctl_choice : (ctl_trial && g->ctl_trials >= 2) ? 1 : 0];
+  if (ctl_own && getenv("AMPNET_ARENA_POS")) g->ctl_mem = g->ctl_cand[atoi(getenv("AMPNET_ARENA_POS")) & 1];
   st = plan_run(g, split, mak, det, eval, cfg, n_order, false, R);
   if (st != AMPNET_OK) return st;
   if (order) {
