@@ -12,7 +12,7 @@ from workloads import ir   # integer codes of the IR format only
 SM_COUNT = 148             # B200: 2 dies x 74 SMs
 # dram__bytes_read.sum + dram__bytes_write.sum of ampnet_engine per instance, from the ncu captures summarised under
 # profiles/ (captured on a small case; traffic grows in proportion to the instances processed)
-MEASURED_DRAM_BYTES_PER_INSTANCE = {"tree": 99461.0, "ggnn": 860920.0}
+MEASURED_DRAM_BYTES_PER_INSTANCE = {"tree": 101860.0, "ggnn": 858646.0}
 FP32_LANES_PER_SM = 128
 
 
