@@ -172,6 +172,35 @@ def test_wide_cells_that_keep_their_accumulators_in_device_memory(oracle_mod):
     r[3].close()
 
 
+def test_deterministic_parity_after_the_control_arena_has_moved(oracle_mod):
+    """A small control arena is tried at two positions during the first asynchronous epochs (epochs 0, 1 at the first,
+    epoch 2 at the second, then the faster).  Every such epoch keeps the accounting exact, and a deterministic epoch from
+    the same start on the same handle afterwards still matches the oracle: nothing of the run state depends on where the
+    arena was."""
+    import paper_1705_09786_b200 as amp
+    g, inst = ir.rnn(), data.list_instances(n=120)
+    p = wp.init_params(g)
+    e = amp.Engine(g)
+    e.load_instances(inst)
+    counts = parity_counts(g, inst)
+    for epoch in range(5):
+        e.set_params(p)
+        st, loss = e.run_epoch(mak=8, muf=10, lr=0.02, deterministic=False, timeout_s=60)
+        assert st.instances == inst.n and e.leftover_cache_entries() == 0, epoch
+        assert st.node_messages == counts["node_messages"], epoch
+        for n, rows in counts["grads"].items():
+            assert e.node_stats(n)["n_grads_applied"] == rows, (epoch, g.names[n])
+        assert np.isfinite(loss).all()
+    e.set_params(p)
+    est, eloss = e.run_epoch(mak=8, muf=10, lr=0.02, deterministic=True, timeout_s=60)
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst)
+    o.set_params(p)
+    ost, oloss = o.run_epoch(mak=8, muf=10, lr=0.02)
+    parity.assert_parity(g, o, ost, oloss, e, est, eloss)
+    e.close()
+
+
 def test_parameter_tensors_alias_device_memory_for_replica_averaging():
     """engine.param_tensors() are views of the arrays the engine trains (no copies), which is what lets a collective
     library average whole-model replicas in place; a single-rank NCCL group exercises the call path."""
