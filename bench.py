@@ -354,6 +354,8 @@ def run_ours(args):
                     "kernel": "ampnet_engine (one persistent launch per step)", "kernel_ms": kavg * 1e3,
                     "algorithmic_flop_per_launch": flops, "flop_per_instance": F, "payload_bytes_per_instance": B,
                     "resident_weight_roofline_instances_per_s": roof_inst,
+                    "weight_reload_roofline_instances_per_s": float(peaks.get("hbm_gbs", 6650.0)) * 1e9 / (rf.reload_bytes(graph, inst) / inst.n),
+                    "weight_reload_roofline_kind": "a per-message mat-vec that reads W forward and backward and updates the accumulator in device memory (context)",
                     "frac_of_resident_weight_roofline": (inst.n / kavg) / roof_inst}
         cpu = None
         if not args.no_cpu_baseline:
@@ -373,6 +375,8 @@ def run_ours(args):
                 "e2e": {"value": e2e_value, "unit": "instances/s", "h2d_bytes_per_step": input_bytes(inst),
                         "d2h_bytes_per_step": int(inst.n * 4 + 512), "steps": e2e_steps},
                 "clocks": clocks, "gpu_launches": args.steps,
+                "step_ms": {"all": [round(1e3 * v, 3) for v in step_s], "best": 1e3 * min(step_s), "median": 1e3 * float(np.median(step_s)),
+                            "note": "this rank's steps (CUDA events around launch + averaging)"},
                 "stats": {"mean_loss_last_step": last.mean_loss, "max_staleness": int(last.max_staleness),
                           "rows_per_micro_batch": last.micro_batch_rows / max(1, last.micro_batches),
                           "placement": placement, "inference_instances_per_s": inference_rate,
@@ -394,7 +398,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="tree", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

@@ -116,6 +116,21 @@ def payload_bytes(graph, inst):
     return total
 
 
+def reload_bytes(graph, inst):
+    """Device-memory bytes of a design that reloads the weights for every message (the per-message mat-vec the paper
+    argues existing frameworks are bound by): W read forward, W read backward, accumulator read and written, per
+    payload row and matrix."""
+    rows = gradient_rows(graph, inst)
+    nodes = graph.nodes
+    total = 0.0
+    for n, r in rows.items():
+        t, din, dout = int(nodes[n][0]), int(nodes[n][1]), int(nodes[n][2])
+        if t == ir.LOOKUP:
+            continue
+        total += r * 4.0 * 4 * din * dout * (3 if t == ir.GRUCELL else 1)
+    return total
+
+
 def roofline_instances_per_s(graph, inst, sm_mhz, hbm_gbs):
     """On-chip-resident-weight roofline: weights never reloaded; bound by FP32 FMA or by payload traffic."""
     F = algorithmic_flops(graph, inst) / inst.n
