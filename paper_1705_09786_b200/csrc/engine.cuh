@@ -813,27 +813,35 @@ __device__ __noinline__ void tile_xwT(const float* __restrict__ Xs, int ldx, int
   }
 }
 
-// dx[b][i] = sum_r D[b][r] * W[r][i], written to dst (device memory, ld = in_dim).
+// dx[b][i] = sum_r D[b][r] * W[r][i], written to dst (device memory, ld = in_dim).  The gradient rows are read four
+// outputs at a time as 16-byte broadcasts (their stride ldd is a multiple of four and the padding beyond R is zero) and
+// the loop carries no predicate: weight rows beyond R, columns beyond in_dim and batch rows beyond nb are read from
+// whatever follows in shared memory (finite numbers), multiplied by zero or never stored.
 template <int J, bool ACCUM = false>
 __device__ __noinline__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Ws, int ldw, int R,
                         int in_dim, float* __restrict__ dst) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int R4 = (R + 3) >> 2, ld4 = ldd >> 2;
   for (int b0 = warp * 4; b0 < nb; b0 += WARPS * 4) {
     float acc[4][J];
 #pragma unroll
     for (int m = 0; m < 4; m++)
 #pragma unroll
       for (int j = 0; j < J; j++) acc[m][j] = 0.f;
-    for (int r = 0; r < R; r++) {
-      float d[4];
+    const float4* dp = reinterpret_cast<const float4*>(Ds + (size_t)b0 * ldd);
+    const float* wp = Ws + lane;
+    for (int c = 0; c < R4; c++, wp += 4 * ldw) {
+      float4 d[4];
 #pragma unroll
-      for (int m = 0; m < 4; m++) d[m] = (b0 + m < nb) ? Ds[(b0 + m) * ldd + r] : 0.f;
+      for (int m = 0; m < 4; m++) d[m] = dp[m * ld4 + c];
 #pragma unroll
       for (int j = 0; j < J; j++) {
-        const int i = lane + 32 * j;
-        const float w = i < in_dim ? Ws[r * ldw + i] : 0.f;
+        const float w0 = wp[32 * j], w1 = wp[ldw + 32 * j], w2 = wp[2 * ldw + 32 * j], w3 = wp[3 * ldw + 32 * j];
 #pragma unroll
-        for (int m = 0; m < 4; m++) acc[m][j] = fmaf(d[m], w, acc[m][j]);
+        for (int m = 0; m < 4; m++) {
+          acc[m][j] = fmaf(d[m].x, w0, acc[m][j]); acc[m][j] = fmaf(d[m].y, w1, acc[m][j]);
+          acc[m][j] = fmaf(d[m].z, w2, acc[m][j]); acc[m][j] = fmaf(d[m].w, w3, acc[m][j]);
+        }
       }
     }
 #pragma unroll
