@@ -797,9 +797,10 @@ __device__ __noinline__ void tile_xwT(const float* __restrict__ Xs, int ldx, int
                                       int in_dim, float* __restrict__ out, int ldo, float* __restrict__ scratch, int rb_max) {
   const int G = nb > 32 ? 2 : 1, S = WARPS / G, K4 = (in_dim + 3) >> 2;
   for (int r0 = 0; r0 < R; r0 += rb_max) {                 // up to rb_max (8 or 16) output rows per pass over the staged inputs
-    const int rb = min(rb_max, R - r0), RBs = rb > 12 ? 16 : rb > 8 ? 12 : rb > 4 ? 8 : 4;
+    const int rb = min(rb_max, R - r0), RBs = rb > 12 ? 16 : rb > 10 ? 12 : rb > 8 ? 10 : rb > 4 ? 8 : 4;
     if (RBs == 16) xwT_pass<16>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
     else if (RBs == 12) xwT_pass<12>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
+    else if (RBs == 10) xwT_pass<10>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
     else if (RBs == 8) xwT_pass<8>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
     else xwT_pass<4>(Xs, ldx, nb, Ws, ldw, r0, R, K4, scratch, G, S);
     __syncthreads();
