@@ -45,6 +45,11 @@ def test_work_model_counts(oracle_mod):
     want = inst.n * (2 * 48 * 2 + 2 * 36 * 3 + 2 * 18 * 3)
     assert rf.algorithmic_flops(g, inst) == want
     assert rf.fma_peak_tflops(1965.0) == pytest.approx(74.45, rel=1e-3)
+    # weight-reload bytes: every message pair reads W twice and reads + writes the accumulator (4 x 4 bytes x in x out)
+    assert rf.reload_bytes(g, inst) == inst.n * 16 * (48 + 36 + 18)
+    gt, it = cases[2]
+    L = (np.diff(it.offsets) + 1) // 2
+    assert rf.reload_bytes(gt, it) == 16 * (L.sum() * 6 * 5 + (L - 1).sum() * 10 * 5 + (2 * L - 1).sum() * 5 * 3)
 
 
 def _free_port():
