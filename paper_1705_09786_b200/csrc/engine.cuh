@@ -1057,8 +1057,11 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileShared& S, i
     BatchDesc d;
     d.sched_start = S.ls.sched_w; d.count = take; d.dir = dir; d.flags = upd ? BATCH_UPDATE : 0;
     d.n_upd = upd ? S.ls.n_acc + total : 0; d.nrows = total; d.upd_t = upd ? (int)S.ls.n_updates + 1 : 0; d.pad1 = 0;
-    if (q) { q->desc = d; q->ver_form = S.ls.version; }   // a scheduler CTA publishes the assembled context instead
-    else { P.batches[S.ls.batch_w & P.batch_mask] = d; __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
+    if (q) {                                              // a scheduler CTA: hand the batch to the warp that assembles and publishes
+      q->desc = d; q->ver_form = S.ls.version;            // its context before the bookkeeping below (that warp is waiting)
+      __threadfence_block();
+      *reinterpret_cast<volatile unsigned*>(&q->full) = S.ls.batch_w + 1u;
+    } else { P.batches[S.ls.batch_w & P.batch_mask] = d; __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
     S.ls.batch_w++;
     S.ls.sched_w += take;
     LeaderState& st = S.ls;
@@ -1083,7 +1086,7 @@ __device__ void publish_marker(const Ctx& C, DevPPT& P, TileShared& S, int flags
     st.log_n++; st.n_updates++; st.n_grads_applied += d.n_upd;
     S.ls.n_acc = 0; S.ls.version++;
   }
-  if (q) { q->desc = d; q->ver_form = S.ls.version; }
+  if (q) { q->desc = d; q->ver_form = S.ls.version; __threadfence_block(); *reinterpret_cast<volatile unsigned*>(&q->full) = S.ls.batch_w + 1u; }
   else { P.batches[S.ls.batch_w & P.batch_mask] = d; __threadfence(); st_rel(P.batch_pub, S.ls.batch_w + 1u); }
   S.ls.batch_w++;
 }
@@ -2057,13 +2060,9 @@ __device__ __noinline__ void scheduler_main(const Ctx& C, DevPPT& P, TileShared&
       bool gow = false, progressed = false;
       if (!warp_uniform(busy)) progressed = leader_try_schedule(C, P, S, P.fetched, bw + ((C.tune & 256) ? 0u : 1u), &gow, q);
       unsigned fin = 0;
-      if (progressed) {
+      if (progressed) {                  // (the slot was handed to warp 1 as soon as its descriptor was written)
         __syncwarp();
-        if (lane == 0) {
-          fin = q->desc.flags & BATCH_TERMINATE;
-          __threadfence_block();
-          *reinterpret_cast<volatile unsigned*>(&q->full) = bw + 1u;
-        }
+        if (lane == 0) fin = q->desc.flags & BATCH_TERMINATE;
       }
       if (lane == 0) { const long long tn = clock64(); rcl[!gow ? 0 : progressed ? 2 : 1] += (unsigned long long)(tn - tp); tp = tn; }
       if (warp_uniform(fin)) break;
