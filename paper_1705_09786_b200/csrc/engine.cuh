@@ -1761,8 +1761,8 @@ __device__ __noinline__ void ppt_main(const Ctx& C, DevPPT& P, const int tile, f
       __syncthreads();
       if (!S.ok) { running = false; break; }
       if (C.sched_ctas) {
+        if (tile == 0 && tid == 0) *reinterpret_cast<volatile unsigned*>(P.fetched) = my_batch + 1u;   // paces the scheduler: a hint, ordered with nothing
         fetch_ctx_block(P, S, my_batch);
-        if (tile == 0 && tid == 0) st_rel(P.fetched, my_batch + 1u);                 // paces the scheduler
       } else if (warp == 0) load_batch_ctx(C, P, S, my_batch);
       __syncthreads();
       const BatchDesc d = S.desc;
