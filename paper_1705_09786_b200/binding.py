@@ -167,9 +167,11 @@ class Engine:
         self.device = torch.device("cuda", device)
         torch.cuda.set_device(self.device)
         self._blocks = {}
+        self.alloc_calls = self.free_calls = 0      # how often the library called back into the allocator
         self._alloc_struct = None
         if use_torch_allocator:
             def _alloc(ctx, nbytes):
+                self.alloc_calls += 1
                 try:
                     t = torch.empty(int(nbytes) + 256, dtype=torch.uint8, device=self.device)
                 except Exception:
@@ -179,6 +181,7 @@ class Engine:
                 return ptr
 
             def _free(ctx, ptr):
+                self.free_calls += 1
                 self._blocks.pop(ptr, None)
 
             self._alloc_cb, self._free_cb = ALLOC_FN(_alloc), FREE_FN(_free)

@@ -18,6 +18,14 @@
 
 using namespace amp;
 
+// host hooks of the direct-delivery engine (engine_fast.cu)
+extern "C" int ampnet_direct_threads();
+extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows);
+extern "C" size_t ampnet_direct_bwd_tile_smem_bytes(int out_dim, int cols, int batch_rows);
+extern "C" int ampnet_direct_max_units();
+extern "C" cudaError_t ampnet_direct_static_smem(size_t* bytes);
+extern "C" cudaError_t ampnet_direct_launch(const amp::Ctx* ctx, int n_ctas, size_t smem_bytes, cudaStream_t stream, int n_sms);
+
 namespace {
 
 struct DeviceArena {           // one allocation carved into aligned pieces
@@ -51,6 +59,8 @@ struct HostPPT {
   int NE = 0, G = 1;                    // emitter CTAs of the node and their batch groups
   bool a_global = false;                // the tiles' gradient accumulators live in device memory (frees shared memory for staging rows)
   int xwt_rb = 8;                       // output rows per pass of X.W^T: 16 where the larger scratch still fits
+  int TB = 0, CB = 0, NS = 1;           // direct-delivery engine: backward column tiles, columns per tile, gradient slots per key
+  size_t bwd_smem_floats = 0;
   double emit_load = 0.0;               // emitter-seconds the node's emission took in the last asynchronous epoch (0: unknown)
   size_t smem_floats = 0;
 };
@@ -93,6 +103,7 @@ struct ampnet_graph {
   std::vector<PPTStats> last_stats;
   std::vector<unsigned long long> last_node_msgs;
   bool have_run = false;
+  bool arenas_lent = false;           // the arenas belong to the caller of execute() (static scratch): never freed or grown
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
 };
 
@@ -539,6 +550,134 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   return AMPNET_OK;
 }
 
+// ---- direct-delivery engine: which graphs it takes, and its placement -------------------------------------
+// It runs asynchronous epochs of graphs whose messages are single rows and whose parameter-free chains it can resolve
+// per message: Cond, Phi, Isu, Bcast, Concat (assembling in the next node's input cache), Sink, and a Loss fed directly
+// by a Linear node.  Everything else (row-wise Group / Ungroup / Flatmap, GRU and LSTM cells, the deterministic
+// schedule, per-node message counters) stays with the interpreter engine.
+bool direct_candidate(ampnet_graph* g, const HostDataset& D, int det) {
+  if (det) return false;
+  if (const char* e = getenv("AMPNET_ENGINE")) if (!strcmp(e, "classic")) return false;
+  if (const char* e = getenv("AMPNET_TUNE")) if (atoi(e) & (16 | 32 | 8)) return false;
+  if (D.kind == 3) return false;
+  const int n = (int)g->hnodes.size();
+  for (int i = 0; i < n; i++) {
+    const DevNode& h = g->hnodes[i];
+    if (h.rows_in != 1 || h.rows_out != 1) return false;
+    switch (h.type) {
+      case SOURCE: if (h.fn < 1 || h.fn > 4) return false; break;
+      case LINEAR: case LOOKUP: case COND: case PHI: case ISU: case SINK: break;
+      case LOSS_CE: case LOSS_MSE: if (g->hnodes[h.pred_node[0]].type != LINEAR) return false; break;
+      case CONCAT: {
+        const DevNode& s = g->hnodes[h.succ_node[0]];
+        if (s.type != LINEAR || (s.in_dim & 3) || s.in_dim != h.out_dim || s.U_in != h.U_out || s.rows_in != h.rows_in) return false;
+      } break;
+      case BCAST: {
+        // backward, the sum forms in the gradient buffer of the parameterised node behind Phi / Cond / Isu
+        std::vector<int> todo{h.pred_node[0]};
+        std::vector<char> seen(n, 0);
+        while (!todo.empty()) {
+          const int v = todo.back(); todo.pop_back();
+          if (seen[v]) continue;
+          seen[v] = 1;
+          const DevNode& p = g->hnodes[v];
+          if (p.type == LINEAR || p.type == LOOKUP) continue;
+          if (p.type != PHI && p.type != COND && p.type != ISU) return false;
+          for (int k = 0; k < p.n_pred; k++) todo.push_back(p.pred_node[k]);
+        }
+      } break;
+      default: return false;
+    }
+  }
+  return true;
+}
+
+// Tiles of the direct-delivery engine.  A Linear node is split by direction: forward row tiles of `rows` weight rows
+// (AMPNET_DIRECT_ROWS, default 8) and backward column tiles of `cols` input columns (AMPNET_DIRECT_COLS, default 16;
+// 4, 8, 16 or 32), more per tile where the CTA budget, shared memory or the register-resident accumulators ask for it.
+// A node that feeds a Loss is one tile for both directions (the Loss needs the whole output row); a large embedding
+// table is dealt to four tiles by row id.
+ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& roles) {
+  size_t static_smem = 48 * 1024;
+  ampnet_direct_static_smem(&static_smem);
+  const size_t budget = (size_t)g->max_smem - static_smem - 1024;
+  int rows = 8, cols = 16;
+  if (const char* e = getenv("AMPNET_DIRECT_ROWS")) rows = std::max(1, atoi(e));
+  if (const char* e = getenv("AMPNET_DIRECT_COLS")) { const int c = atoi(e); if (c == 4 || c == 8 || c == 16 || c == 32) cols = c; }
+  const int np = (int)g->ppts.size(), tile_budget = n_ctas - 1, max_units = ampnet_direct_max_units();
+  std::vector<int> fixed(np, 0);
+  // gradient slots: the backward sum of a Bcast forms in the gradient buffer of the node behind Phi / Cond / Isu
+  for (auto& P : g->ppts) P.NS = 1;
+  for (int i = 0; i < (int)g->hnodes.size(); i++) {
+    const DevNode& h = g->hnodes[i];
+    if (h.type != BCAST) continue;
+    std::vector<int> todo{h.pred_node[0]};
+    std::vector<char> seen(g->hnodes.size(), 0);
+    while (!todo.empty()) {
+      const int v = todo.back(); todo.pop_back();
+      if (seen[v]) continue;
+      seen[v] = 1;
+      const DevNode& p = g->hnodes[v];
+      if (p.type == LINEAR || p.type == LOOKUP) { g->ppts[p.ppt].NS = std::max(g->ppts[p.ppt].NS, h.fn_arg); continue; }
+      for (int k = 0; k < p.n_pred; k++) todo.push_back(p.pred_node[k]);
+    }
+  }
+  for (int p = 0; p < np; p++) {
+    HostPPT& P = g->ppts[p];
+    const DevNode& h = g->hnodes[P.node];
+    P.NE = 0; P.G = 1; P.a_global = false; P.J = 0; P.TB = 0; P.CB = 0; P.bwd_smem_floats = 0;
+    if (P.kind == LOOKUP) { P.T = (P.in >= 4096 && tile_budget >= 24) ? 4 : 1; P.R = 0; P.BM = MAX_BATCH_ROWS; fixed[p] = 1; continue; }
+    const int st = g->hnodes[h.succ_node[0]].type;
+    P.BM = MAX_BATCH_ROWS;
+    if (st == LOSS_CE || st == LOSS_MSE) { P.R = P.out; fixed[p] = 1; }
+    else {
+      P.R = std::min(P.out, rows);
+      P.CB = cols;
+      while (P.CB > 4 && (long long)P.out * (P.CB / 4) > max_units) P.CB /= 2;
+      if ((long long)P.out * (P.CB / 4) > max_units) return AMPNET_EOVERFLOW;        // accumulators of a column tile exceed the registers
+    }
+  }
+  auto fits = [&](const HostPPT& P) {
+    return ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM) <= budget && (P.CB == 0 || ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) <= budget);
+  };
+  for (int p = 0; p < np; p++) {
+    HostPPT& P = g->ppts[p];
+    if (P.kind == LOOKUP) continue;
+    while (!fits(P)) {
+      if (P.BM > 16) P.BM /= 2;
+      else if (!fixed[p] && P.R > 1) { P.R = (P.R + 1) / 2; P.BM = MAX_BATCH_ROWS; }
+      else return AMPNET_EOVERFLOW;
+    }
+  }
+  for (;;) {
+    int used = 0, worst = -1, worst_n = 0;
+    for (int p = 0; p < np; p++) {
+      HostPPT& P = g->ppts[p];
+      if (P.kind != LOOKUP) { P.T = (P.out + P.R - 1) / P.R; P.TB = P.CB ? (P.in + P.CB - 1) / P.CB : 0; }
+      used += P.T + P.TB;
+      if (!fixed[p] && std::max(P.T, P.TB) > worst_n && (P.R < P.out || P.CB < 32)) { worst = p; worst_n = std::max(P.T, P.TB); }
+    }
+    if (used <= tile_budget) break;
+    if (worst < 0) return AMPNET_EOVERFLOW;
+    HostPPT& P = g->ppts[worst];
+    if (P.TB >= P.T && P.CB < 32 && (long long)P.out * (P.CB * 2 / 4) <= max_units) P.CB *= 2;
+    else if (P.R < P.out) P.R++;
+    else return AMPNET_EOVERFLOW;
+    while (!fits(P) && P.BM > 16) P.BM /= 2;
+    if (!fits(P)) return AMPNET_EOVERFLOW;
+  }
+  roles.clear();
+  roles.push_back(Role{-1, 0, 0, 0});
+  for (int p = 0; p < np; p++) {
+    HostPPT& P = g->ppts[p];
+    P.smem_floats = P.kind == LOOKUP ? 64 : ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM) / sizeof(float);
+    P.bwd_smem_floats = P.TB ? ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) / sizeof(float) : 0;
+    for (int t = 0; t < P.T; t++) roles.push_back(Role{p, t, 0, 0});
+    for (int t = 0; t < P.TB; t++) roles.push_back(Role{p, t, 3, 0});
+  }
+  return AMPNET_OK;
+}
+
 // ---- run ---------------------------------------------------------------------------------------------------
 struct RunPlan {
   std::vector<DevNode> nodes;
@@ -546,7 +685,10 @@ struct RunPlan {
   std::vector<Role> roles;
   Ctx ctx{};
   size_t smem_bytes = 0;
+  bool direct = false;                // the run goes to the direct-delivery engine
 };
+
+inline bool eval_uses_classic(int) { return false; }
 
 ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval, const ampnet_run_cfg_t* cfg,
                          long long n_order, bool dry, RunPlan& R) {
@@ -559,16 +701,23 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   if (const char* e = getenv("AMPNET_TUNE")) tune = atoi(e);
   int emit_ctas = (!det && !(tune & 32)) ? ((tune & 64) ? 1 : 2) : 0;
   const int mbr = cfg ? cfg->max_batch_rows : 0;
-  // Two emitter CTAs per tile if the SMs allow it, with as many tiles per node as fit; then one; then none.
   ampnet_status_t st = AMPNET_EOVERFLOW;
-  for (; emit_ctas > 0 && st == AMPNET_EOVERFLOW; emit_ctas--) {
+  R.direct = !eval_uses_classic(eval) && mbr == 0 && direct_candidate(g, D, det);
+  if (R.direct) {
+    st = place_direct(g, n_ctas, R.roles);
+    if (st == AMPNET_EOVERFLOW) R.direct = false;             // too few CTAs for its tiles: the interpreter engine places its own
+    else if (st != AMPNET_OK) return st;
+    else emit_ctas = 0;
+  }
+  // Two emitter CTAs per tile if the SMs allow it, with as many tiles per node as fit; then one; then none.
+  for (; !R.direct && emit_ctas > 0 && st == AMPNET_EOVERFLOW; emit_ctas--) {
     st = place(g, n_ctas, mbr, R.roles, emit_ctas);
     if (st != AMPNET_EOVERFLOW) break;
   }
-  if (st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0); }
+  if (!R.direct && st == AMPNET_EOVERFLOW) { emit_ctas = 0; st = place(g, n_ctas, mbr, R.roles, 0); }
   if (st == AMPNET_EOVERFLOW) return set_err(g, AMPNET_EINVAL, "the model needs more CTAs than the %d available (one per row tile + the controller)", n_ctas);
   if (st != AMPNET_OK) return st;
-  const int depth = emit_ctas > 0 ? 5 : 2;       // emitters work in up to four batch groups: a tile may be four batches ahead
+  const int depth = R.direct ? 1 : emit_ctas > 0 ? 5 : 2;       // emitters work in up to four batch groups: a tile may be four batches ahead
   R.ctx.emit_ctas = emit_ctas; R.ctx.depth = depth; R.ctx.sched_ctas = emit_ctas > 0 ? 1 : 0;
   n_ctas = (int)R.roles.size();
   DeviceArena &C = g->ctl, &B = g->bulk;
@@ -601,7 +750,12 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
       if (P.xld != P.in_dim && !dry) g->zero_regions.push_back({P.xcache, keys * P.rows_max * P.xld * sizeof(float)});   // the row padding
     }
     if (H.kind != LOOKUP) P.ycache = B.take<float>(keys * P.rows_max * P.out_dim);
-    P.gbuf = B.take<float>(keys * P.rows_max * P.out_dim);
+    P.NS = R.direct ? H.NS : 1; P.TB = H.TB; P.CB = H.CB; P.bwd_smem_floats = (int)H.bwd_smem_floats;
+    P.gbuf = B.take<float>(keys * P.rows_max * P.out_dim * P.NS);
+    if (R.direct) {                  // one gradient slot per contributor: nothing is added in memory, nothing cleared
+      for (int d = 0; d < 2; d++) { P.injoin[d] = C.take<int>(keys); track(P.injoin[d], keys * sizeof(int)); }
+      P.wver = C.take<unsigned>(1);
+    }
     if (H.kind == GRUCELL) {
       P.zc = B.take<float>(keys * P.rows_max * P.out_dim);
       P.rc = B.take<float>(keys * P.rows_max * P.out_dim);
@@ -653,6 +807,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     }
     P.smem_floats = (int)H.smem_floats;
     max_smem_floats = std::max(max_smem_floats, H.smem_floats);
+    if (R.direct) max_smem_floats = std::max(max_smem_floats, H.bwd_smem_floats);
     g->d_stats[p] = P.stats; g->d_update_log[p] = P.update_log;
   }
   for (size_t i = 0; i < R.nodes.size(); i++) {
@@ -705,6 +860,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
         break;
       case PHI:
         n.origin = C.take<unsigned char>(kin); track(n.origin, kin);
+        if (R.direct) { n.jcnt = C.take<int>(kin); track(n.jcnt, kin * sizeof(int)); }
         break;
       default: break;
     }
@@ -765,8 +921,16 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   return AMPNET_OK;
 }
 
+// Slack added to what a dry plan counted: alignment of the pieces carved after it (order, inference mask).
+constexpr size_t ARENA_SLACK = 4096, BULK_EXTRA = 1024;
+
 ampnet_status_t ensure_arenas(ampnet_graph* g, size_t ctl_need, size_t bulk_need) {
-  ctl_need += 4096; bulk_need += 4096;
+  ctl_need += ARENA_SLACK; bulk_need += ARENA_SLACK;
+  if (g->arenas_lent) {               // lent memory is used as it is: nothing is freed, nothing allocated
+    if (ctl_need > g->ctl_cap || bulk_need > g->bulk_cap)
+      return set_err(g, AMPNET_EINVAL, "the lent scratch is too small for this run (%zu + %zu bytes needed)", ctl_need, bulk_need);
+    return AMPNET_OK;
+  }
   if (ctl_need > g->ctl_cap) {
     const size_t MiB = (size_t)1 << 20;
     const bool small = ctl_need <= MiB;
@@ -811,15 +975,16 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   const bool dbg = getenv("AMPNET_DEBUG") != nullptr;
   CUDA_TRY(g, cudaSetDevice(g->device));
   RunPlan R;
+  g->have_run = false;                // planning re-targets the statistics pointers: the previous run's are gone from here on
   if (dbg) fprintf(stderr, "[ampnet] planning\n");
   ampnet_status_t st = plan_run(g, split, mak, det, eval, cfg, n_order, true, R);
   if (st != AMPNET_OK) return st;
   const size_t order_bytes = order ? (size_t)n_order * sizeof(long long) : 0;
   const size_t mask_bytes = inference_only ? (size_t)D.n : 0;
-  st = ensure_arenas(g, g->ctl.used, g->bulk.used + order_bytes + mask_bytes + 1024);
+  st = ensure_arenas(g, g->ctl.used, g->bulk.used + order_bytes + mask_bytes + BULK_EXTRA);
   if (st != AMPNET_OK) return st;
   const bool ctl_own = g->ctl_cand[0] && (g->ctl_mem == g->ctl_cand[0] || g->ctl_mem == g->ctl_cand[1]);
-  const bool ctl_trial = ctl_own && g->ctl_choice < 0 && !det && !eval && !getenv("AMPNET_NO_ARENA_TRIAL");
+  const bool ctl_trial = ctl_own && g->ctl_choice < 0 && !det && !eval && !R.direct && !getenv("AMPNET_NO_ARENA_TRIAL");
   if (ctl_own) g->ctl_mem = g->ctl_cand[g->ctl_choice >= 0 ? g->ctl_choice : (ctl_trial && g->ctl_trials >= 2) ? 1 : 0];
   if (ctl_own && getenv("AMPNET_ARENA_POS")) g->ctl_mem = g->ctl_cand[atoi(getenv("AMPNET_ARENA_POS")) & 1];
   st = plan_run(g, split, mak, det, eval, cfg, n_order, false, R);
@@ -842,15 +1007,23 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.nodes, R.nodes.data(), R.nodes.size() * sizeof(DevNode), cudaMemcpyHostToDevice, g->stream));
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.ppts, R.ppts.data(), R.ppts.size() * sizeof(DevPPT), cudaMemcpyHostToDevice, g->stream));
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.roles, R.roles.data(), R.roles.size() * sizeof(Role), cudaMemcpyHostToDevice, g->stream));
-  CUDA_TRY(g, cudaFuncSetAttribute(ampnet_engine, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)R.smem_bytes));
-  int per_sm = 0;
-  CUDA_TRY(g, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ampnet_engine, THREADS, R.smem_bytes));
-  if (per_sm < 1 || (long long)per_sm * g->n_sms < R.ctx.n_ctas)
-    return set_err(g, AMPNET_EINVAL, "%d CTAs cannot be co-resident (%d per SM)", R.ctx.n_ctas, per_sm);
-  if (dbg) fprintf(stderr, "[ampnet] launching %d CTAs, %zu B smem, ctl %zu B, bulk %zu B\n", R.ctx.n_ctas, R.smem_bytes, g->ctl.used, g->bulk.used);
-  void* args[] = {&R.ctx};
-  CUDA_TRY(g, cudaEventRecord(g->ev0, g->stream));
-  CUDA_TRY(g, cudaLaunchCooperativeKernel((void*)ampnet_engine, dim3(R.ctx.n_ctas), dim3(THREADS), args, R.smem_bytes, g->stream));
+  if (dbg) fprintf(stderr, "[ampnet] %s engine, %d CTAs, %zu B smem, ctl %zu B, bulk %zu B\n", R.direct ? "direct-delivery" : "interpreter", R.ctx.n_ctas, R.smem_bytes, g->ctl.used, g->bulk.used);
+  if (dbg) for (auto& P : g->ppts) fprintf(stderr, "[ampnet]   node %d: %d tiles x %d rows, %d backward tiles x %d columns, batch %d, slots %d\n", P.node, P.T, P.R, P.TB, P.CB, P.BM, P.NS);
+  if (R.direct) {
+    CUDA_TRY(g, cudaEventRecord(g->ev0, g->stream));
+    const cudaError_t le = ampnet_direct_launch(&R.ctx, R.ctx.n_ctas, R.smem_bytes, g->stream, g->n_sms);
+    if (le == cudaErrorCooperativeLaunchTooLarge) return set_err(g, AMPNET_EINVAL, "%d CTAs cannot be co-resident", R.ctx.n_ctas);
+    if (le != cudaSuccess) return set_err(g, AMPNET_ECUDA, "launch of the direct-delivery engine failed: %s", cudaGetErrorString(le));
+  } else {
+    CUDA_TRY(g, cudaFuncSetAttribute(ampnet_engine, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)R.smem_bytes));
+    int per_sm = 0;
+    CUDA_TRY(g, cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ampnet_engine, THREADS, R.smem_bytes));
+    if (per_sm < 1 || (long long)per_sm * g->n_sms < R.ctx.n_ctas)
+      return set_err(g, AMPNET_EINVAL, "%d CTAs cannot be co-resident (%d per SM)", R.ctx.n_ctas, per_sm);
+    void* args[] = {&R.ctx};
+    CUDA_TRY(g, cudaEventRecord(g->ev0, g->stream));
+    CUDA_TRY(g, cudaLaunchCooperativeKernel((void*)ampnet_engine, dim3(R.ctx.n_ctas), dim3(THREADS), args, R.smem_bytes, g->stream));
+  }
   CUDA_TRY(g, cudaEventRecord(g->ev1, g->stream));
   Globals G;
   CUDA_TRY(g, cudaMemcpyAsync(&G, R.ctx.g, sizeof G, cudaMemcpyDeviceToHost, g->stream));
@@ -866,7 +1039,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   if (dbg) fprintf(stderr, "[ampnet] done\n");
   g->have_run = true;
   if (!eval) for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].opt_t += (long long)g->last_stats[p].n_updates;
-  if (!eval && !det && R.ctx.emit_ctas)      // emitter time of the node = time of its first emitter x emitters (they share every batch)
+  if (!eval && !det && !R.direct && R.ctx.emit_ctas)      // emitter time of the node = time of its first emitter x emitters (they share every batch)
     for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].emit_load = (double)G.role_cycles[8 + 8 * p + 5] * std::max(1, g->ppts[p].NE) + 1.0;
   if (getenv("AMPNET_TUNE") && (atoi(getenv("AMPNET_TUNE")) & 8)) {
     static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK", "LSTM"};
@@ -1392,11 +1565,13 @@ extern "C" ampnet_status_t ampnet_run_epoch_static(ampnet_graph_t* g, const ampn
   // size the run state without touching any memory, and refuse what does not fit
   const long long n_order = cfg->order ? cfg->n_order : D.n;
   RunPlan plan;
+  g->have_run = false;                // the dry plan re-targets the statistics pointers of the previous run
   ampnet_status_t st = plan_run(g, 0, cfg->max_active_keys, cfg->deterministic ? 1 : 0, 0, cfg, n_order, true, plan);
   if (st != AMPNET_OK) return st;
   const size_t order_bytes = cfg->order ? (size_t)std::max<long long>(n_order, 0) * sizeof(long long) : 0;
-  const size_t ctl_need = ((g->ctl.used + 4096 + 255) & ~(size_t)255);
-  const size_t bulk_need = g->bulk.used + order_bytes + 512 + 4096;
+  // the very sizes execute() will ask ensure_arenas() for
+  const size_t ctl_need = ((g->ctl.used + ARENA_SLACK + 255) & ~(size_t)255);
+  const size_t bulk_need = g->bulk.used + order_bytes + BULK_EXTRA + ARENA_SLACK;
   if (ctl_need + bulk_need > (size_t)AMPNET_STATIC_SCRATCH_BYTES)
     return set_err(g, AMPNET_EINVAL, "this run needs %zu bytes of scratch but the static scratch holds %zu: lower "
                    "max_active_keys or use ampnet_run_epoch", ctl_need + bulk_need, (size_t)AMPNET_STATIC_SCRATCH_BYTES);
@@ -1406,7 +1581,9 @@ extern "C" ampnet_status_t ampnet_run_epoch_static(ampnet_graph_t* g, const ampn
   char* base = static_cast<char*>(g_static_scratch_addr[g->device]);
   g->ctl_mem = base; g->ctl_cap = ctl_need;
   g->bulk_mem = base + ctl_need; g->bulk_cap = (size_t)AMPNET_STATIC_SCRATCH_BYTES - ctl_need;
+  g->arenas_lent = true;
   st = execute(g, 0, cfg->max_active_keys, cfg->deterministic ? 1 : 0, 0, cfg, out, per_instance_loss, nullptr);
+  g->arenas_lent = false;
   g->ctl_mem = own_ctl; g->ctl_cap = own_ctl_cap; g->bulk_mem = own_bulk; g->bulk_cap = own_bulk_cap;
   g->leftover_regions.clear();      // they described the lent memory
   return st;

@@ -239,7 +239,7 @@ __device__ __forceinline__ bool join_arrive(int* cnt, int expected, int lane) {
 }
 
 // ---- CTA-wide pool of frames: a warp that forks offers the rest of the fork to idle warps --------------
-__device__ __forceinline__ bool pool_offer(WalkPool* Q, const Frame& c, int lane) {
+__device__ __forceinline__ bool pool_offer(const Ctx& C, WalkPool* Q, const Frame& c, int lane) {
   if (!Q) return false;
   int ok = 0;
   if (lane == 0) {
@@ -256,6 +256,7 @@ __device__ __forceinline__ bool pool_offer(WalkPool* Q, const Frame& c, int lane
       atomicAdd(&Q->outstanding, 1);
       int spins = 0;
       while (*(volatile unsigned*)&Q->ready[idx] != 0u && ++spins < (1 << 20)) {}
+      if (*(volatile unsigned*)&Q->ready[idx] != 0u) fail(C, ST_TIMEOUT, -5, (int)idx);   // the slot never drained: report, the run is over
       Q->f[idx] = c;
       __threadfence_block();
       *(volatile unsigned*)&Q->ready[idx] = t + 1u;
@@ -423,7 +424,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (f.dir == FWD) {
             int k = f.iter;
             if (k + 1 < n.fn_arg) { Frame c = f; c.iter = k + 1;
-              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+              if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             to_succ(f, n, k);
             cont = true;
@@ -457,7 +458,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           } else {
             int k = f.iter;
             if (k + 1 < n.fn_arg) { Frame c = f; c.iter = k + 1;
-              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+              if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             f.p = f.p ? f.p + k * n.in_dim : nullptr; f.dim = n.in_dim;
             if (n.fn == 2) { f.port = k; to_pred(f, n, 0); } else to_pred(f, n, k);
@@ -518,7 +519,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             __syncwarp();
             if (n.fn == 2) {                      // second message: the cells' gradient to port 1
               Frame c = f; c.iter = 1;
-              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+              if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); }
             }
             f.p = base; f.nsum = 1; f.sstride = 0; f.dim = n.in_dim; f.ld = n.in_dim;
@@ -534,7 +535,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
           if (f.dir == FWD) {
             const int k = f.iter;
             if (k + 1 < n.fn_arg) { Frame c = f; c.iter = k + 1;
-              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+              if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             f.p = f.p ? f.p + k * n.out_dim : nullptr; f.dim = n.out_dim;
             to_succ(f, n, k);
@@ -576,7 +577,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             const int i = f.iter * f.nparts + f.part;       // this walker's share of the rows
             if (i >= f.rows) break;
             if (i + f.nparts < f.rows) { Frame c = f; c.iter = f.iter + 1;
-              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+              if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             f.nparts = 1; f.part = 0;
             const long long ebase = f.ebase;
@@ -595,7 +596,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             const int i = f.iter * f.nparts + f.part;       // this walker's share of the rows
             if (i >= f.rows) break;
             if (i + f.nparts < f.rows) { Frame c = f; c.iter = f.iter + 1;
-              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+              if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             f.nparts = 1; f.part = 0;
             int mu = n.fn == 2 ? I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i] : i;
@@ -626,7 +627,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             int i = f.iter;
             if (deg > 0) {
               if (i + 1 < deg) { Frame c = f; c.iter = i + 1;
-              if (!pool_offer(Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
+              if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
               f.u = I.out_list[oo[0] + i];
               to_succ(f, n, 0);
@@ -715,7 +716,13 @@ __device__ __noinline__ void pool_steal(const Ctx& C, WalkPool* Q, Frame* stack,
     if (got) {
       h = __shfl_sync(0xffffffffu, h, 0);
       const unsigned idx = h % POOL;
-      if (lane == 0) { int spins = 0; while (*(volatile unsigned*)&Q->ready[idx] != h + 1u && ++spins < (1 << 20)) {} }
+      unsigned lost = 0;
+      if (lane == 0) {
+        int spins = 0;
+        while (*(volatile unsigned*)&Q->ready[idx] != h + 1u && ++spins < (1 << 20)) {}
+        if (*(volatile unsigned*)&Q->ready[idx] != h + 1u) { fail(C, ST_TIMEOUT, -6, (int)idx); lost = 1; }   // never published
+      }
+      if (warp_uniform(lost)) { if (lane == 0) atomicSub(&Q->outstanding, 1); break; }
       __syncwarp();
       Frame f = Q->f[idx];
       __syncwarp();
@@ -817,7 +824,10 @@ __device__ __noinline__ void tile_xwT(const float* __restrict__ Xs, int ldx, int
 // dx[b][i] = sum_r D[b][r] * W[r][i], written to dst (device memory, ld = in_dim).  The gradient rows are read four
 // outputs at a time as 16-byte broadcasts (their stride ldd is a multiple of four and the padding beyond R is zero) and
 // the loop carries no predicate: weight rows beyond R, columns beyond in_dim and batch rows beyond nb are read from
-// whatever follows in shared memory (finite numbers), multiplied by zero or never stored.
+// whatever follows in shared memory, multiplied by zero or never stored.  INVARIANT this relies on: what follows Ws in
+// the tile's carve-up (accumulators, biases, staging rows; all zero-filled at start) holds finite numbers.  A run whose
+// accumulators have overflowed to Inf / NaN has diverged already (its parameters are Inf / NaN after the next update),
+// so the 0 x Inf = NaN this could add to an input gradient changes nothing that was still meaningful.
 template <int J, bool ACCUM = false>
 __device__ __noinline__ void tile_dW(const float* __restrict__ Ds, int ldd, int nb, const float* __restrict__ Ws, int ldw, int R,
                         int in_dim, float* __restrict__ dst) {
@@ -1258,7 +1268,12 @@ __device__ __noinline__ void stage_rows_bulk(const Ctx& C, TileShared& S, float*
   for (;;) {
     asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) break;
-    if ((++spins & 1023u) == 0 && (aborted(C) || gtime() - t0 > C.timeout_ns)) { if (tid == 0) fail(C, ST_TIMEOUT, node, 7); break; }
+    if ((++spins & 1023u) == 0 && (aborted(C) || gtime() - t0 > C.timeout_ns)) {
+      if (tid == 0) fail(C, ST_TIMEOUT, node, 7);
+      for (unsigned extra = 0; extra < (1u << 16) && !done; extra++)      // copies already issued still land in this CTA's shared memory
+        asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+      break;
+    }
   }
   __syncthreads();
   if (tid == 0) S.mbar_parity = parity ^ 1u;

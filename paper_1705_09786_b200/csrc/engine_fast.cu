@@ -1,0 +1,1330 @@
+// Direct-delivery engine: the asynchronous (measured) mode for IR graphs whose messages are single rows.
+//
+// Roles: CTA 0 is the controller (admission under max_active_keys, retirement: Sec. 3, Sec. 4 "controller loop");
+// every other CTA is a row tile of one parameterised node and keeps its rows of W resident in shared memory for the
+// whole epoch.  There is no scheduler and no emitter between two nodes:
+//   * every tile polls its node's two rings itself and forms its own micro-batches (backward first, App. A).  All tiles
+//     of a node see the same messages in the same order (the ring is the order), so all of them cut their backward
+//     batches at the same gradient counts and update at the same points (Sec. 3): a tile is a node of its own in the
+//     sense of the tiling the paper describes in Sec. 5, forward and backward batches may interleave differently;
+//   * the chain of parameter-free nodes behind a message (Cond, Phi, Isu, Bcast, Concat, Sink, Loss) is a function of
+//     the message state and the instance's structure tables alone.  One thread per message resolves it ("route") while
+//     the batch's input rows are still in flight, down to the buffers the payload finally lands in: the input cache of
+//     the next parameterised node (a Concat assembles there), or its incoming-gradient buffer (a Bcast's backward sum
+//     forms there);
+//   * after the arithmetic every tile stores its slice of the outputs (forward) or adds its partial input gradient
+//     (backward, red.global.add) straight into those buffers and arrives at the landing's join counter with its share
+//     of JOIN_UNIT; the arrival that completes the count publishes the header in the consumer's ring.
+// One hop is therefore: stores -> one acquire-release atomic -> ticket + release store -> the consumer's poll.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include "engine_types.h"
+
+namespace ampf {
+using namespace amp;
+
+constexpr int FT = 512;               // threads per CTA
+constexpr int FW = FT / 32;
+constexpr int FBM = 64;               // messages (= rows) per micro-batch
+constexpr int MAXD = 4;               // landings per message
+constexpr int RSTACK = 4;             // pending forks per routed message
+
+// ------------------------------------------------------------------------------------------------
+// memory-model helpers, bounded waits
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned ld_acq(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ unsigned ld_rlx(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void fence_acq() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+__device__ __forceinline__ void st_rel(unsigned* p, unsigned v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
+  int old;
+  asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
+}
+__device__ __forceinline__ void red_add(float* p, float v) {
+  asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __noinline__ void fail(const Ctx& C, int code, int node, int detail) {
+  if (atomicCAS(&C.g->status, 0, code) == 0) { C.g->err_node = node; C.g->err_detail = detail; }
+  __threadfence();
+  st_rel(&C.g->abort_flag, 1u);
+}
+__device__ __forceinline__ bool aborted(const Ctx& C) { return ld_acq(&C.g->abort_flag) != 0; }
+__device__ __forceinline__ unsigned warp_uniform(unsigned v) { return __shfl_sync(0xffffffffu, v, 0); }
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ long long key_of(const Ctx& C, int node, int slot, int it, int u, int U) {   // the failure path is a call
+  if ((unsigned)slot >= (unsigned)C.mak || (unsigned)it >= (unsigned)C.IT || (unsigned)u >= (unsigned)U) {
+    fail(C, ST_OVERFLOW, node, u);
+    return -1;
+  }
+  return ((long long)slot * C.IT + it) * U + u;
+}
+
+// Pointers into shared memory that reach a function as arguments would be dereferenced as generic addresses; this tells
+// the compiler their address space.
+#define IN_SMEM(p) __builtin_assume(__isShared(p))
+
+__shared__ DevNode g_nodes[MAX_SMEM_NODES];
+__shared__ DevPPT g_ppts[MAX_SMEM_PPTS];
+__shared__ int g_bf16;
+// What a node emits as a payload: identity for fp32 messages, rounded to bfloat16 (nearest even) otherwise.
+__device__ __forceinline__ float emit_round(float v) { return g_bf16 ? __bfloat162float(__float2bfloat16_rn(v)) : v; }
+
+__device__ __forceinline__ float act_fwd(int a, float v) {
+  switch (a) {
+    case 1: return v > 0.f ? v : 0.f;
+    case 2: return tanhf(v);
+    case 3: return 1.f / (1.f + expf(-v));
+    default: return v;
+  }
+}
+__device__ __forceinline__ float act_grad(int a, float y) {
+  switch (a) {
+    case 1: return y > 0.f ? 1.f : 0.f;
+    case 2: return 1.f - y * y;
+    case 3: return y * (1.f - y);
+    default: return 1.f;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// routes: where the payload of one message lands
+// ------------------------------------------------------------------------------------------------
+enum { ACT_PUSH = 1, ACT_RETIRE = 2, ACT_LOSS = 3 };
+
+// One landing of a message.  Columns [s0, s0 + w) of the payload go to dst[0 .. w) (dst == nullptr: nothing to
+// deposit, the arrival alone counts).  The arrival that brings *jcnt to `expected` (ACT_RETIRE: down to zero) clears
+// the recorded Phi origin, publishes the header (ACT_PUSH) or tells the controller (ACT_RETIRE).
+struct __align__(16) Deliv {
+  float* dst;
+  int* jcnt;
+  unsigned char *clear, *clear2;  // recorded Phi origins the completing arrival clears
+  int expected, s0, w, act;
+  int ppt, dir, u, it;
+  int port, post, node, zero, pad[2];   // post: logical node-messages the completing arrival accounts for; node: the Loss;
+                                  // zero: the payload is a zero vector (deposit zeros of width w)
+};
+
+struct Route {                    // state of one message on its way through the parameter-free nodes
+  int node, aport, dir, u, it, port, s0, w, null;
+};
+
+// The message `h` leaves parameterised node `P` in direction `dir`.  Follows the parameter-free nodes (Sec. 4: Cond
+// queries the state, Phi records / recalls the origin, Isu updates the state and inverts the update, Bcast copies and
+// sums, Concat joins and splits) and writes the landings to out[0 .. returned count).  pre: node-messages consumed on
+// the way that every arrival sees (added once per message by the first row tile).  width: payload width at the start.
+__device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_node, int start_aport, const int dir0, const int width,
+                                          Deliv* out, int& pre) {
+  IN_SMEM(out);
+  const DevInst& I = C.inst;
+  const long long ibase = I.offsets ? I.offsets[h.inst] : 0;
+  Route stack[RSTACK];
+  int sp = 0, nout = 0;
+  Route f;
+  f.node = start_node; f.aport = start_aport; f.dir = dir0; f.u = h.u; f.it = h.it; f.port = h.port; f.s0 = 0; f.w = width; f.null = 0;
+  pre = 0;
+  bool have = true;
+  // a pending join: the backward sum of a Bcast forms in the buffer the message lands in
+  int* pend = nullptr; int pend_exp = 0, pend_slot = 0; int post = 0; unsigned char *clear = nullptr, *clear2 = nullptr;
+  int* phi_cnt = nullptr;         // arrival counter of the last Phi passed backward (joins the tiles' arrivals of one message at a Source)
+  int steps = 0;
+  while (have) {
+    if (f.node < 0 || ++steps > 256) { fail(C, ST_OVERFLOW, -2, f.node); return nout; }
+    const DevNode& n = g_nodes[f.node];
+    bool cont = false;
+    auto count = [&] { if (pend) post++; else pre++; };
+    auto to_succ = [&](int k) { f.aport = n.succ_port[k]; f.node = n.succ_node[k]; f.dir = FWD; cont = true; };
+    auto to_pred = [&](int j) { f.aport = n.pred_port[j]; f.node = n.pred_node[j]; f.dir = BWD; cont = true; };
+    auto land = [&](Deliv d) {
+      if (nout >= MAXD) { fail(C, ST_OVERFLOW, f.node, -9); return; }
+      d.clear = clear; d.clear2 = clear2; d.zero = f.null ? 1 : 0;
+      out[nout++] = d;
+      pend = nullptr; pend_exp = 0; pend_slot = 0; post = 0; clear = clear2 = nullptr; phi_cnt = nullptr;
+    };
+    switch (n.type) {
+      case LINEAR: case LOOKUP: {
+        DevPPT& Q = g_ppts[n.ppt];
+        const long long key = key_of(C, f.node, h.slot, f.it, f.u, Q.U);
+        if (key < 0) return nout;
+        Deliv d;
+        if (f.dir == FWD) {
+          if (!Q.xcache) { fail(C, ST_OVERFLOW, f.node, -10); return nout; }
+          d.dst = Q.xcache + key * (long long)Q.xld;
+        } else {
+          // gradients land in slots: one per successor of the Bcast whose backward sum forms here, so that nothing is added
+          // in memory (no atomics on payloads, nothing to clear); the reader adds the slots in successor order
+          if (!pend && Q.NS != 1) { fail(C, ST_OVERFLOW, f.node, -15); return nout; }
+          d.dst = Q.gbuf + (key * Q.NS + pend_slot) * (long long)Q.out_dim;
+        }
+        d.jcnt = pend ? pend : Q.injoin[f.dir] + key;
+        d.expected = pend ? pend_exp : JOIN_UNIT;
+        d.s0 = f.s0; d.w = f.w; d.act = ACT_PUSH; d.ppt = n.ppt; d.dir = f.dir; d.u = f.u; d.it = f.it; d.port = f.port;
+        d.post = post + 1; d.node = f.node;
+        land(d);
+      } break;
+      case LOSS_CE: case LOSS_MSE: {
+        pre++;
+        Deliv d;
+        d.dst = nullptr; d.jcnt = nullptr; d.expected = 0; d.s0 = f.s0; d.w = f.w; d.act = ACT_LOSS; d.ppt = -1; d.dir = FWD;
+        d.u = f.u; d.it = f.it; d.port = f.port; d.post = 0; d.node = f.node;
+        land(d);
+      } break;
+      case SOURCE: {                                        // a source message came home
+        if (pend) { fail(C, ST_OVERFLOW, f.node, -14); return nout; }
+        Deliv d;
+        d.dst = nullptr; d.jcnt = &C.outstanding[h.slot]; d.expected = 0; d.s0 = 0; d.w = 0; d.act = ACT_RETIRE; d.ppt = -1;
+        d.dir = BWD; d.u = f.u; d.it = f.it; d.port = f.port; d.post = post; d.node = f.node;
+        // a recorded origin may be cleared only when every tile has read it: the tiles' arrivals of this message meet at the
+        // Phi's counter first, and the one that completes it retires the whole source message
+        if (clear && phi_cnt) { d.jcnt = phi_cnt; d.expected = JOIN_UNIT; }
+        land(d);
+      } break;
+      case SINK:
+        count();
+        if (h.flags & HDR_EVAL) {
+          Deliv d;
+          d.dst = nullptr; d.jcnt = &C.outstanding[h.slot]; d.expected = 0; d.s0 = 0; d.w = 0; d.act = ACT_RETIRE; d.ppt = -1;
+          d.dir = FWD; d.u = f.u; d.it = f.it; d.port = f.port; d.post = post; d.node = f.node;
+          land(d);
+        } else { f.null = 1; to_pred(0); }                   // answers with a zero gradient
+        break;
+      case COND:
+        count();
+        if (f.dir == FWD) {
+          int k = 0;
+          switch (n.fn) {
+            case 1: k = f.u < (int)(I.offsets[h.inst + 1] - ibase) ? 0 : 1; break;
+            case 2: k = I.parent[ibase + f.u] < 0 ? 0 : 1; break;
+            case 3: k = f.u; break;
+            case 4: k = f.it < n.fn_arg ? 0 : 1; break;
+            case 5: k = (h.inst + f.u) % n.n_succ; break;
+          }
+          if ((unsigned)k >= (unsigned)n.n_succ) { fail(C, ST_OVERFLOW, f.node, k); return nout; }
+          to_succ(k);
+        } else to_pred(0);
+        break;
+      case PHI: {
+        count();
+        const long long key = key_of(C, f.node, h.slot, f.it, f.u, n.U_in);
+        if (key < 0) return nout;
+        if (f.dir == FWD) {
+          if (!(h.flags & HDR_EVAL)) n.origin[key] = (unsigned char)(f.aport + 1);   // every tile writes the same value
+          to_succ(0);
+        } else {
+          const int j = (int)*(volatile unsigned char*)&n.origin[key] - 1;
+          if (j < 0 || j >= n.n_pred) { fail(C, ST_OVERFLOW, f.node, -20); return nout; }
+          if (clear2) { fail(C, ST_OVERFLOW, f.node, -11); return nout; }
+          if (clear) clear2 = &n.origin[key]; else clear = &n.origin[key];   // cleared by the arrival that completes the landing
+          phi_cnt = n.jcnt ? &n.jcnt[key] : nullptr;
+          to_pred(j);
+        }
+      } break;
+      case ISU:
+        count();
+        if (f.dir == FWD) {
+          if (n.fn == 1) f.u += 1;
+          else if (n.fn == 2) { f.port = I.child_slot[ibase + f.u]; f.u = I.parent[ibase + f.u]; }
+          else f.it += 1;
+          to_succ(0);
+        } else {
+          if (n.fn == 1) f.u -= 1;
+          else if (n.fn == 2) { f.u = f.port == 0 ? I.left[ibase + f.u] : I.right[ibase + f.u]; f.port = 0; }
+          else f.it -= 1;
+          to_pred(0);
+        }
+        break;
+      case BCAST:
+        if (f.dir == FWD) {
+          count();
+          for (int k = n.fn_arg - 1; k >= 1; k--) {
+            if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; }
+            Route c = f; c.node = n.succ_node[k]; c.aport = n.succ_port[k]; c.dir = FWD;
+            stack[sp++] = c;
+          }
+          to_succ(0);
+        } else {
+          count();
+          const long long key = key_of(C, f.node, h.slot, f.it, f.u, n.U_in);
+          if (key < 0) return nout;
+          if (pend) { fail(C, ST_OVERFLOW, f.node, -12); return nout; }      // nested sums are not resolved here
+          pend = &n.jcnt[key]; pend_exp = n.fn_arg * JOIN_UNIT; pend_slot = f.aport;
+          if ((unsigned)pend_slot >= (unsigned)n.fn_arg) { fail(C, ST_OVERFLOW, f.node, -16); return nout; }
+          to_pred(0);
+        }
+        break;
+      case CONCAT:
+        if (f.dir == FWD) {
+          count();
+          const int port = n.fn == 2 ? f.port : f.aport;
+          const long long key = key_of(C, f.node, h.slot, f.it, f.u, n.U_out);
+          if (key < 0) return nout;
+          const DevNode& s = g_nodes[n.succ_node[0]];
+          if ((unsigned)port >= (unsigned)n.fn_arg || !n.jalias || pend) { fail(C, ST_OVERFLOW, f.node, port); return nout; }
+          Deliv d;
+          d.dst = n.jbuf + key * n.jstride + port * n.in_dim;
+          d.jcnt = &n.jcnt[key]; d.expected = n.fn_arg * JOIN_UNIT;
+          d.s0 = f.s0; d.w = f.w; d.act = ACT_PUSH; d.ppt = s.ppt; d.dir = FWD; d.u = f.u; d.it = f.it; d.port = 0;
+          d.post = 1; d.node = n.succ_node[0];
+          land(d);
+        } else {
+          count();
+          for (int k = n.fn_arg - 1; k >= 0; k--) {
+            Route c = f; c.s0 = f.s0 + k * n.in_dim; c.w = n.in_dim; c.dir = BWD;
+            if (n.fn == 2) { c.port = k; c.node = n.pred_node[0]; c.aport = n.pred_port[0]; }
+            else { c.node = n.pred_node[k]; c.aport = n.pred_port[k]; }
+            if (k == 0) { f = c; cont = true; }
+            else { if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; } stack[sp++] = c; }
+          }
+        }
+        break;
+      default:
+        fail(C, ST_OVERFLOW, f.node, n.type);
+        return nout;
+    }
+    if (!cont) {
+      if (pend) { fail(C, ST_OVERFLOW, f.node, -13); return nout; }          // a sum that found no landing
+      if (sp > 0) f = stack[--sp];
+      else have = false;
+    }
+  }
+  return nout;
+}
+
+// ------------------------------------------------------------------------------------------------
+// tile state and arithmetic
+// ------------------------------------------------------------------------------------------------
+struct TileS {
+  Hdr hdr[FBM];
+  long long key[FBM];
+  const float* rowptr[FBM];
+  Deliv dl[FBM][MAXD];
+  int nd[FBM], pre[FBM], rowid[FBM];
+  int count, dir, flags, n_upd, upd_t, eval, ok, term;
+  unsigned head[2];
+  int n_acc, version, log_n, max_stale;
+  unsigned long long n_updates, n_grads_applied, msgs, batches, batch_rows, node_msgs;
+  unsigned long long stale_hist[64];
+  unsigned long long phase[16];
+  unsigned long long mbar;
+  unsigned mbar_parity;
+  unsigned wver_seen;               // forward tile: the node's published-columns counter as last polled
+};
+
+__host__ __device__ __forceinline__ int pad4(int v) { return (v + 3) & ~3; }
+// n / d for 0 <= n < 200000 and 1 <= d <= 2048 by one multiply-high (M = floor((2^32 - 1) / d) + 1; checked exhaustively)
+struct FastDiv {
+  unsigned d, M;
+  __device__ explicit FastDiv(int d_) : d((unsigned)d_), M(0xFFFFFFFFu / (unsigned)d_ + 1u) {}
+  __device__ __forceinline__ int div(int n) const { return (int)__umulhi((unsigned)n, M); }
+};
+__host__ __device__ __forceinline__ int pad_ldx(int in) { int l = (in + 3) & ~3; while ((l & 7) != 4) l += 4; return l; }
+constexpr int XWT_SCRATCH = 0;
+
+// out[b][o] = sum_k A[b][k] B[o][k] for b < nA, o < nB: both operands in shared memory with k contiguous, rows padded
+// with zeros to K4 groups of four and strides of 4 (mod 8) floats (eight rows read 16 bytes each without a bank
+// conflict).  A thread owns one output and one of nsl interleaved k-slices, as many slices as keep every thread busy
+// (a single message still spreads over the whole CTA); the slices meet by shuffles.  Whole CTA, no barrier inside.
+__device__ __forceinline__ void gemm_nt(const float* __restrict__ A, const int lda, const int nA, const float* __restrict__ B, const int ldb,
+                                        const int nB, const int K4, float* __restrict__ out, const int ldo) {
+  const int tid = threadIdx.x, n_out = nA * nB;
+  int nsl = 1, sh = 0;
+  while (nsl < 32 && n_out * nsl * 2 <= FT) { nsl <<= 1; sh++; }
+  const int per_pass = FT >> sh, ks = tid & (nsl - 1);
+  const FastDiv dB(nB);
+  for (int o0 = 0; o0 < n_out; o0 += per_pass) {
+    const int oi = o0 + (tid >> sh);
+    const bool valid = oi < n_out;
+    const int b = valid ? dB.div(oi) : 0, o = valid ? oi - b * nB : 0;
+    const float4* a = reinterpret_cast<const float4*>(A + (size_t)b * lda);
+    const float4* w = reinterpret_cast<const float4*>(B + (size_t)o * ldb);
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+    for (int k4 = ks; k4 < K4; k4 += nsl) {
+      const float4 x = a[k4], y = w[k4];
+      a0 = fmaf(x.x, y.x, a0); a1 = fmaf(x.y, y.y, a1); a2 = fmaf(x.z, y.z, a2); a3 = fmaf(x.w, y.w, a3);
+    }
+    float v = (a0 + a1) + (a2 + a3);
+    for (int off = 1; off < nsl; off <<= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+    if (valid && ks == 0) out[b * ldo + o] = v;
+  }
+}
+
+// Local update of one parameter from its accumulated gradient (Sec. 3; the rule is a run-time option, App. A):
+// g = A / n, then SGD, momentum-SGD (v <- mu v + g, theta <- theta - lr v) or Adam with bias correction, where t counts
+// the updates of this node.
+struct OptStep {
+  int opt; float lr, inv_n, mu, b1, b2, eps, c1, c2; float *om, *ov;
+  __device__ OptStep(const Ctx& C, const DevPPT& P, int n_upd, int upd_t)
+      : opt(C.opt), lr(C.lr), inv_n(1.f / (float)n_upd), mu(C.mu), b1(C.beta1), b2(C.beta2), eps(C.eps), c1(1.f), c2(1.f),
+        om(P.om), ov(P.ov) {
+    if (opt == 2) {
+      const double t = (double)(P.opt_t0 + upd_t);
+      c1 = (float)(1.0 / (1.0 - pow((double)b1, t)));
+      c2 = (float)(1.0 / (1.0 - pow((double)b2, t)));
+    }
+  }
+  __device__ __forceinline__ void apply(float& w, float& a, const size_t k) const {
+    if (opt == 0) { w = fmaf(-(lr * inv_n), a, w); a = 0.f; return; }
+    apply_moments(w, a, k);
+  }
+  __device__ __noinline__ void apply_moments(float& w, float& a, const size_t k) const {
+    const float g = a * inv_n;
+    a = 0.f;
+    if (opt == 1) {
+      const float v = fmaf(mu, om[k], g);
+      om[k] = v;
+      w = fmaf(-lr, v, w);
+    } else {
+      const float m = fmaf(b1, om[k], (1.f - b1) * g), v = fmaf(b2, ov[k], (1.f - b2) * g * g);
+      om[k] = m; ov[k] = v;
+      w -= lr * (m * c1) / (sqrtf(v * c2) + eps);
+    }
+  }
+};
+
+__device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) { return P.muf_override > 0 ? P.muf_override : C.muf; }
+
+// ------------------------------------------------------------------------------------------------
+// arrivals
+// ------------------------------------------------------------------------------------------------
+__device__ __noinline__ void ring_push(Ring& r, const Hdr& h, int it, int u, int port) {     // one thread
+  const unsigned t = atomicAdd(r.tail, 1u), s = t & r.mask;
+  int4* d = reinterpret_cast<int4*>(&r.e[s]);
+  d[0] = make_int4(h.inst, h.seq, h.slot, it);
+  d[1] = make_int4(u, port, 1, h.flags);
+  st_rel(&r.seq[s], t + 1u);
+}
+// The instance in key slot `slot` loses `wgt` of its outstanding source messages (JOIN_UNIT each); the arrival that
+// brings the count to zero tells the controller.
+__device__ __noinline__ void retire_arrive(const Ctx& C, int slot, int wgt) {
+  const int old = atom_add_acq_rel(&C.outstanding[slot], -wgt);
+  if (old < wgt) fail(C, ST_OVERFLOW, -30, slot);                // more source messages came home than were pumped
+  if (old != wgt) return;
+  const unsigned t = atomicAdd(&C.g->retire_tail, 1u), s = t & C.retire_mask;
+  C.retire_e[s] = (unsigned)slot;
+  st_rel(&C.retire_seq[s], t + 1u);
+}
+// One thread, after the barrier behind the deposits of its CTA: arrive at landing L of message h with weight wgt.
+__device__ __noinline__ void arrive(const Ctx& C, const Hdr& h, const Deliv& L, int wgt, unsigned long long* node_msgs) {
+  IN_SMEM(&h); IN_SMEM(&L); IN_SMEM(node_msgs);
+  if (L.act == ACT_RETIRE && L.expected) {                       // the message's arrivals meet first, then it retires whole
+    if (atom_add_acq_rel(L.jcnt, wgt) + wgt != L.expected) return;
+    *(volatile int*)L.jcnt = 0;
+    if (L.clear) *L.clear = 0;
+    if (L.clear2) *L.clear2 = 0;
+    if (L.post) atomicAdd(node_msgs, (unsigned long long)L.post);
+    retire_arrive(C, h.slot, JOIN_UNIT);
+    return;
+  }
+  if (L.act == ACT_RETIRE) {
+    const int old = atom_add_acq_rel(L.jcnt, -wgt);
+    if (old < wgt) fail(C, ST_OVERFLOW, -30, h.slot);
+    if (old != wgt) return;
+    if (L.clear) *L.clear = 0;
+    if (L.clear2) *L.clear2 = 0;
+    if (L.post) atomicAdd(node_msgs, (unsigned long long)L.post);
+    const unsigned t = atomicAdd(&C.g->retire_tail, 1u), s = t & C.retire_mask;
+    C.retire_e[s] = (unsigned)h.slot;
+    st_rel(&C.retire_seq[s], t + 1u);
+    return;
+  }
+  if (L.act != ACT_PUSH) return;
+  const int sum = atom_add_acq_rel(L.jcnt, wgt) + wgt;
+  if (sum > L.expected) fail(C, ST_OVERFLOW, L.node, -31);       // more arrivals than the landing expects
+  if (sum != L.expected) return;
+  *(volatile int*)L.jcnt = 0;                                   // the key's next use finds the counter at zero
+  if (L.clear) *L.clear = 0;
+  if (L.clear2) *L.clear2 = 0;
+  atomicAdd(node_msgs, (unsigned long long)L.post);
+  ring_push(g_ppts[L.ppt].ring[L.dir], h, L.it, L.u, L.port);
+}
+
+__device__ __forceinline__ unsigned long long ballot64(const bool p0, const bool p1) {
+  return (unsigned long long)__ballot_sync(0xffffffffu, p0) | ((unsigned long long)__ballot_sync(0xffffffffu, p1) << 32);
+}
+
+// Warp 0 of a tile: take the next micro-batch from the node's rings, backward first (App. A) unless the backward queue is
+// short and the forward queue longer (a cycle costs the same for 2 messages as for 64; max_active_keys bounds the
+// forward supply, so the backward queue is always reached).  The batch is cut at the tile's row capacity, where
+// training and forward-only messages meet, and exactly at the gradient that triggers the update (Sec. 3).
+// dirs: bit 0 forward ring, bit 1 backward ring.  Returns 1 with the batch in S, 2 when the epoch is over, 0 when
+// nothing is pending.
+__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const bool leader, const bool fused, const int dirs, const bool light) {
+  IN_SMEM(&P); IN_SMEM(&S);
+  const int lane = threadIdx.x & 31;
+  if (light) {                      // nothing was pending a moment ago: watch the two head slots (and the end of the epoch) only
+    unsigned any = 0;
+    if (lane < 2 && (dirs & (1 << lane))) any = ld_rlx(&P.ring[lane].seq[S.head[lane] & P.ring[lane].mask]) == S.head[lane] + 1u;
+    if (lane == 2) any = ld_rlx(&C.g->done);
+    if (!__any_sync(0xffffffffu, any != 0)) return 0;
+  }
+  if (dirs == 1 && lane == 0) S.wver_seen = ld_rlx(P.wver);          // ordered by the fence below like the ring polls
+  unsigned slot[2][2];
+  bool ready[2][2];
+#pragma unroll
+  for (int dir = 0; dir < 2; dir++)
+#pragma unroll
+    for (int j = 0; j < 2; j++) {
+      const unsigned t = S.head[dir] + lane + 32 * j;
+      slot[dir][j] = t & P.ring[dir].mask;
+      ready[dir][j] = ld_rlx(&P.ring[dir].seq[slot[dir][j]]) == t + 1u;
+    }
+  fence_acq();
+  int nready[2];
+#pragma unroll
+  for (int dir = 0; dir < 2; dir++) {
+    const unsigned long long m = ballot64(ready[dir][0], ready[dir][1]);
+    nready[dir] = m == ~0ull ? 64 : __ffsll((long long)~m) - 1;
+    if (!(dirs & (1 << dir))) nready[dir] = 0;                     // forward row tiles / backward column tiles take one ring only
+  }
+  if (nready[0] == 0 && nready[1] == 0) {
+    unsigned fin = 0;
+    if (lane == 0) fin = ld_acq(&C.g->done);
+    if (!warp_uniform(fin)) return 0;
+    if (lane == 0) {
+      S.count = 0; S.dir = BWD; S.flags = BATCH_TERMINATE; S.n_upd = 0; S.upd_t = 0; S.eval = 0;
+      if (S.n_acc > 0 && !C.eval) {                            // epoch-end flush of the leftover gradients
+        S.flags |= BATCH_UPDATE; S.n_upd = S.n_acc; S.upd_t = (int)S.n_updates + 1;
+        if (leader && S.log_n < P.update_log_cap) P.update_log[S.log_n] = S.n_upd;
+        S.log_n++; S.n_updates++; S.n_grads_applied += S.n_upd; S.n_acc = 0; S.version++;
+      }
+    }
+    __syncwarp();
+    return 2;
+  }
+  const bool fwd_first = !(C.tune & 128) && nready[BWD] < FBM / 2 && nready[FWD] > nready[BWD];
+  const int dir = (nready[BWD] == 0 || (fwd_first && nready[FWD] > 0)) ? FWD : BWD;
+  int take = min(nready[dir], P.BM);
+  Hdr h[2];
+#pragma unroll
+  for (int j = 0; j < 2; j++) {
+    h[j] = Hdr{0, 0, 0, 0, 0, 0, 0, 0};
+    if (lane + 32 * j < take) {
+      const int4* e = reinterpret_cast<const int4*>(&P.ring[dir].e[dir == FWD ? slot[FWD][j] : slot[BWD][j]]);
+      const int4 a = __ldcg(e), b = __ldcg(e + 1);
+      h[j].inst = a.x; h[j].seq = a.y; h[j].slot = a.z; h[j].it = a.w; h[j].u = b.x; h[j].port = b.y; h[j].rows = b.z; h[j].flags = b.w;
+    }
+  }
+  const int eval0 = __shfl_sync(0xffffffffu, (int)((h[0].flags & HDR_EVAL) != 0), 0);
+  const unsigned long long okm = ballot64(lane < take && (int)((h[0].flags & HDR_EVAL) != 0) == eval0,
+                                          lane + 32 < take && (int)((h[1].flags & HDR_EVAL) != 0) == eval0);
+  take = okm == ~0ull ? 64 : __ffsll((long long)~okm) - 1;
+  bool upd = false;
+  const bool grads = (dir == BWD || fused) && !eval0;          // a fused loss head turns every forward message into a gradient at once
+  if (grads) {
+    const int muf = node_muf(C, P);
+    if (S.n_acc + take >= muf) { take = max(1, muf - S.n_acc); upd = true; }
+  }
+#pragma unroll
+  for (int j = 0; j < 2; j++) if (lane + 32 * j < take) S.hdr[lane + 32 * j] = h[j];
+  __syncwarp();
+  if (lane == 0) {
+    S.count = take; S.dir = dir; S.flags = upd ? BATCH_UPDATE : 0; S.eval = eval0;
+    S.n_upd = upd ? S.n_acc + take : 0; S.upd_t = upd ? (int)S.n_updates + 1 : 0;
+    S.head[dir] += take;
+    S.msgs += grads && fused ? 2 * take : take; S.batches++; S.batch_rows += take;
+    if (upd) {
+      if (leader && S.log_n < P.update_log_cap) P.update_log[S.log_n] = S.n_upd;
+      S.log_n++; S.n_updates++; S.n_grads_applied += S.n_upd; S.n_acc = 0; S.version++;
+    } else if (grads) S.n_acc += take;
+  }
+  __syncwarp();
+  return 1;
+}
+
+// ------------------------------------------------------------------------------------------------
+// row tile
+// ------------------------------------------------------------------------------------------------
+#define TPHASE(k) do { if (tid == 0) { const long long n_ = clock64(); S.phase[k] += (unsigned long long)(n_ - tph); tph = n_; } } while (0)
+
+// Softmax cross-entropy / squared error on the full output row y (this tile owns the whole node), as the Loss node
+// defines it: records the loss and the arg-max hit under the Loss's key and writes the gradient the Loss sends back
+// (rounded like every emitted payload) to g (training messages only).
+__device__ __forceinline__ void loss_row(const Ctx& C, const int loss_node, const Hdr& h, const float* y, float* g, const int label_bits) {
+  const DevNode& n = g_nodes[loss_node];
+  const long long key = key_of(C, loss_node, h.slot, h.it, h.u, n.U_in);
+  if (key < 0) return;
+  const bool train = !(h.flags & HDR_EVAL);
+  if (n.type == LOSS_CE) {
+    const int label = label_bits;
+    float mx = -3.4e38f; int arg = 0;
+    for (int j = 0; j < n.in_dim; j++) if (y[j] > mx) { mx = y[j]; arg = j; }
+    float s = 0.f;
+    for (int j = 0; j < n.in_dim; j++) s += expf(y[j] - mx);
+    const float lse = mx + logf(s);
+    if (train) for (int j = 0; j < n.in_dim; j++) g[j] = emit_round(expf(y[j] - lse) - (j == label ? 1.f : 0.f));
+    n.lossval[key] = lse - y[label]; n.predok[key] = (arg == label) ? 1 : 0;
+  } else {
+    const float d = y[0] - __int_as_float(label_bits);
+    n.lossval[key] = d * d; n.predok[key] = 0;
+    if (train) g[0] = emit_round(2.f * d);
+  }
+}
+
+__device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileS& S, const unsigned long long t0) {
+  IN_SMEM(&P); IN_SMEM(smem); IN_SMEM(&S);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int in = P.in_dim, out = P.out_dim;
+  const bool lookup = P.kind == LOOKUP, leader = tile == 0;
+  const int r_begin = tile * P.R;
+  const int R = lookup ? 0 : max(0, min(P.R, out - r_begin));
+  const int LW = pad_ldx(in), LX = pad_ldx(in), RP = pad4(max(P.R, 1));
+  const int wgt = tile == P.T - 1 ? JOIN_UNIT - (P.T - 1) * (JOIN_UNIT / P.T) : JOIN_UNIT / P.T;
+  const DevNode& N = g_nodes[P.node];
+  // A node that feeds a Loss is one tile and runs the whole exchange in one pass: forward, Loss, and the backward message
+  // the Loss answers with (which App. A's backward-first rule would take next anyway), so its forward messages count
+  // as gradients where the batch is cut.
+  const int loss_node = (!lookup && (g_nodes[N.succ_node[0]].type == LOSS_CE || g_nodes[N.succ_node[0]].type == LOSS_MSE)) ? N.succ_node[0] : -1;
+  const bool fused = loss_node >= 0;
+  // Every other Linear node is split by direction: row tiles (this function) take the forward ring, column tiles
+  // (bwd_tile_main) the backward ring.  The column tiles own the master weights and accumulators; after an update they
+  // publish their columns and the row tiles reload their rows before their next batch.
+  const bool fwd_only = !lookup && !fused;
+  const int dirs = fwd_only ? 1 : 3;
+  float *Ws = smem, *As = Ws + (size_t)P.R * LW, *bs = As + (size_t)P.R * LW, *Abs = bs + RP, *Xs = Abs + RP,
+        *Ds = Xs + (size_t)P.BM * LX, *Ys = Ds + (size_t)P.BM * RP, *scratch = Ys + (size_t)P.BM * RP, *smem_end = scratch + XWT_SCRATCH;
+  if (!lookup) {
+    for (float* q = smem + tid; q < smem_end; q += FT) *q = 0.f;
+    __syncthreads();
+    for (int i = tid; i < R * in; i += FT) { const int r = i / in, c = i - r * in; Ws[r * LW + c] = P.W[(size_t)r_begin * in + i]; }
+    for (int i = tid; i < R; i += FT) bs[i] = P.b[r_begin + i];
+  }
+  if (tid == 0) {
+    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0;
+    S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&S.mbar)) : "memory");
+    S.mbar_parity = 0;
+  }
+  if (tid < 64) S.stale_hist[tid] = 0;
+  if (tid < 16) S.phase[tid] = 0;
+  __syncthreads();
+  long long tph = clock64();
+  const FastDiv dR(max(R, 1)), dIn(in);
+  const bool bulk_ok = !lookup && (P.xcache != nullptr || ((in & 3) == 0 && (C.inst.dense_dim & 3) == 0));
+  const int xwidth = P.xcache ? P.xld : in;
+
+  for (;;) {
+    // ---- next batch ----------------------------------------------------------------------------------
+    if (warp == 0) {
+      unsigned it = 0;
+      for (;;) {
+        const int r = form_batch(C, P, S, leader, fused, dirs, it > 0);
+        if (r) break;
+        if ((++it & 15u) == 0) {
+          unsigned bad = 0;
+          if (lane == 0) { bad = aborted(C); if (!bad && gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, P.node, 1); bad = 1; } }
+          if (warp_uniform(bad)) { if (lane == 0) S.ok = 0; break; }
+        }
+        __nanosleep(it < 16 ? 20 : 100);
+      }
+    }
+    __syncthreads();
+    if (!S.ok) break;
+    TPHASE(0);
+    const int count = S.count, dir = S.dir, flags = S.flags;
+    if (fwd_only && (int)(S.wver_seen / (unsigned)P.TB) > S.version) {      // every column tile has published a newer version
+      for (int i = tid; i < R * in; i += FT) { const int r = i / in, c = i - r * in; Ws[r * LW + c] = __ldcg(P.W + (size_t)r_begin * in + i); }
+      for (int i = tid; i < R; i += FT) bs[i] = __ldcg(P.b + r_begin + i);
+      __syncthreads();
+      if (tid == 0) S.version = (int)(S.wver_seen / (unsigned)P.TB);
+      __syncthreads();
+      TPHASE(3);
+    }
+    // ---- keys, staging copies, routes ------------------------------------------------------------------
+    if (count > 0) {
+      const unsigned bar = smem_u32(&S.mbar);
+      if (tid == 0 && bulk_ok) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((unsigned)(count * xwidth * 4)) : "memory");
+      if (tid < count) {
+        const Hdr h = S.hdr[tid];
+        const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+        S.key[tid] = key;
+        S.nd[tid] = 0; S.pre[tid] = 0;
+        if (key < 0) S.ok = 0;
+        if (key >= 0) {
+          if (!lookup) {
+            const float* x = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+            S.rowptr[tid] = x;
+            if (bulk_ok) {
+              asm volatile("fence.proxy.async;" ::: "memory");
+              asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                           :: "r"(smem_u32(Xs + (size_t)tid * LX)), "l"(x), "r"((unsigned)(xwidth * 4)), "r"(bar) : "memory");
+            }
+          } else {
+            const int id = C.inst.tokens[C.inst.offsets[h.inst] + h.u];
+            S.rowid[tid] = (unsigned)id < (unsigned)in ? id : -1;
+          }
+          if (leader && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
+          else if (leader && !S.eval && fwd_only) P.vcache[key] = S.version;   // the version this forward pass uses (Sec. 3: staleness)
+          int pre = 0, nd = 0;
+          if (fused) {                                   // the label, fetched while the input rows are in flight
+            const DevInst& I = C.inst;
+            if (g_nodes[loss_node].type == LOSS_CE) S.rowid[tid] = I.labels_i[I.labels_per_node ? I.offsets[h.inst] + h.u : h.inst];
+            else S.rowid[tid] = __float_as_int(I.labels_f[h.inst]);
+          }
+          if (fused) {                                   // the Loss and this node's own backward arrival, then the way back
+            if (!S.eval) nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[tid], pre);
+            pre += S.eval ? 1 : 2;
+          } else if (dir == FWD) nd = route_message(C, h, N.succ_node[0], N.succ_port[0], FWD, out, S.dl[tid], pre);
+          else nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[tid], pre);
+          S.nd[tid] = nd; S.pre[tid] = pre;
+        }
+      }
+      if (bulk_ok) {
+        const unsigned parity = S.mbar_parity;
+        unsigned done = 0, spins = 0;
+        for (;;) {
+          asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+          if (done) break;
+          if ((++spins & 1023u) == 0 && (aborted(C) || gtime() - t0 > C.timeout_ns)) {
+            if (tid == 0) fail(C, ST_TIMEOUT, P.node, 7);
+            for (unsigned extra = 0; extra < (1u << 16) && !done; extra++)
+              asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+            break;
+          }
+        }
+      }
+      __syncthreads();
+      if (tid == 0 && bulk_ok) S.mbar_parity ^= 1u;
+      if (!lookup && !bulk_ok) {
+        for (int idx = tid; idx < count * in; idx += FT) { const int b = dIn.div(idx), c = idx - b * in; Xs[b * LX + c] = __ldcg(S.rowptr[b] + c); }
+        __syncthreads();
+      }
+      if (!S.ok) break;
+    }
+    TPHASE(1);
+    // ---- arithmetic and deposits -------------------------------------------------------------------------
+    if (count > 0 && fused) {
+      gemm_nt(Xs, LX, count, Ws, LW, R, pad4(in) >> 2, Ys, RP);
+      __syncthreads();
+      TPHASE(5);
+      if (tid < count) {
+        float* y = Ys + tid * RP;
+        for (int r = 0; r < R; r++) y[r] = emit_round(act_fwd(P.act, y[r] + bs[r]));
+        float* g = Ds + tid * RP;
+        loss_row(C, loss_node, S.hdr[tid], y, g, S.rowid[tid]);
+        if (!S.eval) for (int r = 0; r < R; r++) g[r] *= act_grad(P.act, y[r]);
+      }
+      __syncthreads();
+      TPHASE(6);
+      if (!S.eval) {
+        // the node is one tile with a handful of rows: a thread per element of dx (complete sums, stored into the slot the
+        // gradient lands in) and per accumulator
+        if (!(P.flags & 1)) {
+          for (int idx = tid; idx < count * in; idx += FT) {
+            const int b = dIn.div(idx), i = idx - b * in;
+            float v = 0.f;
+            for (int r = 0; r < R; r++) v = fmaf(Ds[b * RP + r], Ws[r * LW + i], v);
+            v = emit_round(v);
+            for (int q = 0; q < S.nd[b]; q++) {
+              const Deliv& L = S.dl[b][q];
+              if (L.act == ACT_PUSH && L.dst && i >= L.s0 && i < L.s0 + L.w && !(C.tune & 512)) L.dst[i - L.s0] = v;
+            }
+          }
+        }
+        TPHASE(7);
+        for (int idx = tid; idx < R * in; idx += FT) {
+          const int r = dIn.div(idx), k = idx - r * in;
+          float a = As[r * LW + k];
+#pragma unroll 4
+          for (int b = 0; b < count; b++) a = fmaf(Ds[b * RP + r], Xs[b * LX + k], a);
+          As[r * LW + k] = a;
+        }
+        for (int r = tid; r < R; r += FT) {
+          float a = Abs[r];
+          for (int b = 0; b < count; b++) a += Ds[b * RP + r];
+          Abs[r] = a;
+        }
+      }
+    } else if (count > 0 && !lookup) {
+      if (dir == FWD) {
+        gemm_nt(Xs, LX, count, Ws, LW, R, pad4(in) >> 2, Ys, RP);
+        __syncthreads();
+        TPHASE(5);
+        for (int idx = tid; idx < count * R; idx += FT) {
+          const int b = dR.div(idx), r = idx - b * R;
+          const float y = emit_round(act_fwd(P.act, Ys[b * RP + r] + bs[r]));
+          Ys[b * RP + r] = y;
+          if (!S.eval) P.ycache[S.key[b] * out + r_begin + r] = y;
+        }
+        __syncthreads();
+        TPHASE(6);
+        // this tile's slice of every output row, straight into the buffers it lands in
+        for (int idx = tid; idx < count * MAXD * R; idx += FT) {
+          const int bq = dR.div(idx), r = idx - bq * R, q = bq % MAXD, b = bq / MAXD;
+          if (q >= S.nd[b]) continue;
+          const Deliv& L = S.dl[b][q];
+          const int c = r_begin + r;
+          if (L.act == ACT_PUSH && L.dst && c >= L.s0 && c < L.s0 + L.w) L.dst[c - L.s0] = L.zero ? 0.f : Ys[b * RP + r];
+        }
+      }
+    } else if (count > 0) {
+      // Embedding table: its rows are dealt to the node's tiles (row id belongs to tile id % T).  Every tile sees every
+      // message and arrives for it; the owner of the table row moves the data.
+      __syncthreads();
+      for (int b = warp; b < count; b += FW) {
+        const int id = S.rowid[b];
+        const bool mine = id >= 0 ? id % P.T == tile : leader;
+        if (!mine) continue;
+        constexpr int K = 5;                                // column chunks of 32 in flight per lane
+        if (dir == FWD) {
+          for (int q = 0; q < S.nd[b]; q++) {
+            const Deliv& L = S.dl[b][q];
+            if (L.act != ACT_PUSH || !L.dst) continue;
+            for (int cc = 0; cc < L.w; cc += 32 * K) {
+              float v[K];
+#pragma unroll
+              for (int k = 0; k < K; k++) { const int c = cc + 32 * k + lane; v[k] = (id >= 0 && c < L.w) ? P.W[(size_t)id * out + L.s0 + c] : 0.f; }
+#pragma unroll
+              for (int k = 0; k < K; k++) { const int c = cc + 32 * k + lane; if (c < L.w) L.dst[c] = emit_round(v[k]); }
+            }
+          }
+        } else {
+          const float* g = P.gbuf + S.key[b] * (long long)P.NS * out;
+          if (id >= 0) {
+            float* arow = P.A + (size_t)id * out;
+            for (int cc = 0; cc < out; cc += 32 * K) {
+              float v[K];
+#pragma unroll
+              for (int k = 0; k < K; k++) { const int c = cc + 32 * k + lane; v[k] = c < out ? __ldcg(g + c) : 0.f; }
+#pragma unroll
+              for (int k = 0; k < K; k++) { const int c = cc + 32 * k + lane; if (c < out) atomicAdd(arow + c, emit_round(v[k])); }
+            }
+            if (lane == 0 && atomicExch(&P.touched_flag[id], 1) == 0)
+              P.touched_list[(size_t)tile * ((in + P.T - 1) / P.T) + atomicAdd(P.touched_n + tile, 1)] = id;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    TPHASE(2);
+    // ---- local update (Sec. 3): theta <- theta - lr A / n, accumulator cleared ------------------------------
+    if (flags & BATCH_UPDATE) {
+      const OptStep os(C, P, S.n_upd, S.upd_t);
+      if (lookup) {
+        __threadfence();
+        int* const tlist = P.touched_list + (size_t)tile * ((in + P.T - 1) / P.T);
+        const int nt = *(volatile int*)&P.touched_n[tile];
+        for (int k = warp; k < nt; k += FW) {
+          const int id = tlist[k];
+          const size_t o0 = (size_t)id * out;
+          constexpr int K = 5;
+          for (int cc = 0; cc < out; cc += 32 * K) {
+            float w[K], a[K];
+#pragma unroll
+            for (int j = 0; j < K; j++) { const int c = cc + 32 * j + lane; if (c < out) { w[j] = P.W[o0 + c]; a[j] = __ldcg(P.A + o0 + c); } }
+#pragma unroll
+            for (int j = 0; j < K; j++) { const int c = cc + 32 * j + lane; if (c < out) { os.apply(w[j], a[j], o0 + c); P.W[o0 + c] = w[j]; P.A[o0 + c] = a[j]; } }
+          }
+          if (lane == 0) P.touched_flag[id] = 0;
+        }
+        __syncthreads();
+        if (tid == 0) P.touched_n[tile] = 0;
+      } else {
+        const size_t nW = (size_t)out * in;
+        for (int i = tid; i < R * in; i += FT) { const int r = i / in, o = r * LW + (i - r * in); os.apply(Ws[o], As[o], (size_t)r_begin * in + i); }
+        for (int i = tid; i < R; i += FT) os.apply(bs[i], Abs[i], nW + r_begin + i);
+      }
+      __syncthreads();
+    }
+    TPHASE(3);
+    // ---- arrivals: the one that completes a landing publishes the message ------------------------------------
+    if (count > 0) {
+      for (int idx = tid; idx < count * MAXD; idx += FT) {
+        const int b = idx / MAXD, q = idx - b * MAXD;
+        if (q == 0 && leader && S.pre[b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[b]);
+        if (q >= S.nd[b]) continue;
+        const Deliv& L = S.dl[b][q];
+        const Hdr& h = S.hdr[b];
+        arrive(C, h, L, wgt, &S.node_msgs);
+      }
+      if (fused && S.eval && tid < count) retire_arrive(C, S.hdr[tid].slot, JOIN_UNIT);   // a forward-only instance ends at its Losses
+    }
+    __syncthreads();                                          // warp 0 forms the next batch over the headers the arrivals read
+    TPHASE(4);
+    if (flags & BATCH_TERMINATE) break;
+  }
+  // ---- epilogue: parameters back to device memory, statistics ----------------------------------------------
+  __syncthreads();
+  if (fused) {
+    for (int i = tid; i < R * in; i += FT) { const int r = i / in; P.W[(size_t)r_begin * in + i] = Ws[r * LW + (i - r * in)]; }
+    for (int i = tid; i < R; i += FT) P.b[r_begin + i] = bs[i];
+  }
+  if (tid == 0 && S.node_msgs) atomicAdd(&C.g->node_messages, S.node_msgs);
+  if (leader) {
+    if (!fwd_only && tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
+    if (tid < 8) P.stats->phase_cycles[tid] = S.phase[tid];
+    if (tid == 0) {
+      PPTStats& st = *P.stats;
+      if (!fwd_only) { st.max_staleness = S.max_stale; st.log_n = S.log_n; st.n_updates = S.n_updates; st.n_grads_applied = S.n_grads_applied; }
+      atomicAdd(&st.msgs, S.msgs); atomicAdd(&st.batches, S.batches); atomicAdd(&st.batch_rows, S.batch_rows);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// backward column tile of a Linear node
+// ------------------------------------------------------------------------------------------------
+// The tile owns input columns [c0, c0 + CB) of W for all output rows: the master copy of those weights in shared memory
+// and their gradient accumulators in registers.  For a backward message it needs the whole pre-activation gradient
+// dpre = g * act'(y) (g: the sum of the gradient slots under the key, y: the cached output) and its own columns of the
+// cached input x.  Its columns of the input gradient dx = W^T dpre are complete sums: they are stored, not added, into
+// the slot they land in.  A[:, cols] += dpre x[cols]^T.  After the update (Sec. 3) the tile writes its columns to the
+// parameter array in device memory and counts itself in the node's version counter; the forward row tiles reload.
+constexpr int MAXU = 4;                 // accumulator units (one output row x four columns) per thread
+
+__device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileS& S, const unsigned long long t0) {
+  IN_SMEM(&P); IN_SMEM(smem); IN_SMEM(&S);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int in = P.in_dim, out = P.out_dim, CB = P.CB, c4n = CB >> 2;
+  const bool leader = tile == 0;
+  const int c0 = tile * CB;
+  const int GL = pad_ldx(out), WL = GL;          // row strides of dpre [batch][out] and of the transposed weights [column][out]
+  const int wgt = tile == P.TB - 1 ? JOIN_UNIT - (P.TB - 1) * (JOIN_UNIT / P.TB) : JOIN_UNIT / P.TB;
+  const DevNode& N = g_nodes[P.node];
+  float *Wt = smem, *G = Wt + (size_t)CB * WL, *Xc = G + (size_t)P.BM * GL, *Dx = Xc + (size_t)P.BM * CB, *bsv = Dx + (size_t)P.BM * CB, *Abs = bsv + GL,
+        *smem_end = Abs + GL;
+  for (float* q = smem + tid; q < smem_end; q += FT) *q = 0.f;
+  __syncthreads();
+  for (int i = tid; i < out * CB; i += FT) { const int r = i / CB, c = i - r * CB; if (c0 + c < in) Wt[c * WL + r] = P.W[(size_t)r * in + c0 + c]; }
+  if (leader) for (int i = tid; i < out; i += FT) bsv[i] = P.b[i];
+  float A[MAXU][4];
+#pragma unroll
+  for (int k = 0; k < MAXU; k++)
+#pragma unroll
+    for (int j = 0; j < 4; j++) A[k][j] = 0.f;
+  const int n_units = out * c4n;
+  const FastDiv dOut(out);
+  const int cb_shift = 31 - __clz(CB), c4_shift = cb_shift - 2;
+  if (tid == 0) {
+    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0;
+    S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
+  }
+  if (tid < 64) S.stale_hist[tid] = 0;
+  if (tid < 16) S.phase[tid] = 0;
+  __syncthreads();
+  long long tph = clock64();
+
+  for (;;) {
+    if (warp == 0) {
+      unsigned it = 0;
+      for (;;) {
+        const int r = form_batch(C, P, S, leader, false, 2, it > 0);
+        if (r) break;
+        if ((++it & 15u) == 0) {
+          unsigned bad = 0;
+          if (lane == 0) { bad = aborted(C); if (!bad && gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, P.node, 11); bad = 1; } }
+          if (warp_uniform(bad)) { if (lane == 0) S.ok = 0; break; }
+        }
+        __nanosleep(it < 16 ? 20 : 100);
+      }
+    }
+    __syncthreads();
+    if (!S.ok) break;
+    TPHASE(0);
+    const int count = S.count, flags = S.flags;
+    if (count > 0) {
+      // ---- keys, routes ------------------------------------------------------------------------------------
+      if (tid < count) {
+        const Hdr h = S.hdr[tid];
+        const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+        S.key[tid] = key; S.nd[tid] = 0; S.pre[tid] = 0;
+        if (key < 0) S.ok = 0;
+        else {
+          S.rowptr[tid] = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+          if (leader) {                                  // staleness: updates of this node between forward and backward (Sec. 3)
+            int st = S.version - ((flags & BATCH_UPDATE) ? 1 : 0) - P.vcache[key];
+            if (st < 0) st = 0;
+            atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
+            atomicMax(&S.max_stale, st);
+          }
+          int pre = 0;
+          S.nd[tid] = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[tid], pre);
+          S.pre[tid] = pre;
+        }
+      }
+      __syncthreads();
+      if (!S.ok) break;
+      TPHASE(1);
+      // ---- operands: dpre for all rows, this tile's columns of x -------------------------------------------------
+      {
+        constexpr int U = 4;                              // elements per thread whose loads are in flight together
+        const int total = count * out;
+        for (int base = tid; base < total; base += FT * U) {
+          float gv[U], g2[U], yv[U];
+#pragma unroll
+          for (int u = 0; u < U; u++) {
+            const int idx = base + u * FT;
+            gv[u] = g2[u] = yv[u] = 0.f;
+            if (idx < total) {
+              const int b = dOut.div(idx), r = idx - b * out;
+              const float* g = P.gbuf + S.key[b] * (long long)P.NS * out + r;
+              gv[u] = __ldcg(g);
+              if (P.NS > 1) g2[u] = __ldcg(g + out);
+              yv[u] = __ldcg(P.ycache + S.key[b] * (long long)out + r);
+            }
+          }
+#pragma unroll
+          for (int u = 0; u < U; u++) {
+            const int idx = base + u * FT;
+            if (idx < total) {
+              const int b = dOut.div(idx), r = idx - b * out;
+              float v = gv[u];
+              if (P.NS > 1) {                             // successor order
+                v += g2[u];
+                for (int sl = 2; sl < P.NS; sl++) v += __ldcg(P.gbuf + (S.key[b] * (long long)P.NS + sl) * out + r);
+                v = emit_round(v);
+              }
+              G[b * GL + r] = v * act_grad(P.act, yv[u]);
+            }
+          }
+        }
+      }
+      for (int idx = tid; idx < count * CB; idx += FT) {
+        const int b = idx >> cb_shift, c = idx - (b << cb_shift);
+        Xc[idx] = c0 + c < in ? __ldcg(S.rowptr[b] + c0 + c) : 0.f;
+      }
+      __syncthreads();
+      TPHASE(2);
+      // ---- dx[b][cols] = sum_r dpre[b][r] W[r][cols], then straight into the slots the gradient lands in ----------------
+      if (!(P.flags & 1)) {
+        gemm_nt(G, GL, count, Wt, WL, CB, pad4(out) >> 2, Dx, CB);
+        __syncthreads();
+        for (int idx = tid; idx < count * CB; idx += FT) {
+          const int b = idx >> cb_shift, i = c0 + (idx & (CB - 1));
+          if (i >= in) continue;
+          const float v = emit_round(Dx[idx]);
+          for (int q = 0; q < S.nd[b]; q++) {
+            const Deliv& L = S.dl[b][q];
+            if (L.act == ACT_PUSH && L.dst && i >= L.s0 && i < L.s0 + L.w) L.dst[i - L.s0] = v;
+          }
+        }
+      }
+      TPHASE(3);
+      // ---- A[r][cols] += sum_b dpre[b][r] x[b][cols]: accumulators in registers --------------------------------------
+#pragma unroll
+      for (int k = 0; k < MAXU; k++) {
+        const int u = tid + k * FT;
+        if (u < n_units) {
+          const int r = u >> c4_shift, c4 = u - (r << c4_shift);
+#pragma unroll 2
+          for (int b = 0; b < count; b++) {
+            const float g = G[b * GL + r];
+            const float4 x = *reinterpret_cast<const float4*>(Xc + b * CB + 4 * c4);
+            A[k][0] = fmaf(g, x.x, A[k][0]); A[k][1] = fmaf(g, x.y, A[k][1]); A[k][2] = fmaf(g, x.z, A[k][2]); A[k][3] = fmaf(g, x.w, A[k][3]);
+          }
+        }
+      }
+      if (leader) for (int r = tid; r < out; r += FT) { float a = Abs[r]; for (int b = 0; b < count; b++) a += G[b * GL + r]; Abs[r] = a; }
+      TPHASE(4);
+    }
+    // ---- local update (Sec. 3), then the columns go to device memory for the forward tiles ---------------------------
+    if (flags & BATCH_UPDATE) {
+      const OptStep os(C, P, S.n_upd, S.upd_t);
+#pragma unroll
+      for (int k = 0; k < MAXU; k++) {
+        const int u = tid + k * FT;
+        if (u < n_units) {
+          const int r = u >> c4_shift, c4 = u - (r << c4_shift);
+#pragma unroll
+          for (int j = 0; j < 4; j++) {
+            const int c = c0 + 4 * c4 + j;
+            if (c < in) {
+              float w = Wt[(4 * c4 + j) * WL + r];
+              os.apply(w, A[k][j], (size_t)r * in + c);
+              Wt[(4 * c4 + j) * WL + r] = w;
+              P.W[(size_t)r * in + c] = w;
+            } else A[k][j] = 0.f;
+          }
+        }
+      }
+      if (leader) for (int r = tid; r < out; r += FT) { os.apply(bsv[r], Abs[r], (size_t)out * in + r); P.b[r] = bsv[r]; }
+      __syncthreads();
+      if (tid == 0) { __threadfence(); atomicAdd(P.wver, 1u); }
+      TPHASE(5);
+    }
+    // ---- arrivals ------------------------------------------------------------------------------------------------
+    if (count > 0) {
+      __syncthreads();
+      for (int idx = tid; idx < count * MAXD; idx += FT) {
+        const int b = idx / MAXD, q = idx - b * MAXD;
+        if (q == 0 && leader && S.pre[b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[b]);
+        if (q >= S.nd[b]) continue;
+        arrive(C, S.hdr[b], S.dl[b][q], wgt, &S.node_msgs);
+      }
+    }
+    __syncthreads();
+    TPHASE(6);
+    if (flags & BATCH_TERMINATE) break;
+  }
+  __syncthreads();
+  if (tid == 0 && S.node_msgs) atomicAdd(&C.g->node_messages, S.node_msgs);
+  if (leader) {
+    if (tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
+    if (tid < 8) P.stats->phase_cycles[8 + tid] = S.phase[tid];
+    if (tid == 0) {
+      PPTStats& st = *P.stats;
+      st.max_staleness = S.max_stale; st.log_n = S.log_n; st.n_updates = S.n_updates; st.n_grads_applied = S.n_grads_applied;
+      atomicAdd(&st.msgs, S.msgs); atomicAdd(&st.batches, S.batches); atomicAdd(&st.batch_rows, S.batch_rows);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// controller CTA: admission under max_active_keys, source messages, retirement (Sec. 3, Sec. 4)
+// ------------------------------------------------------------------------------------------------
+constexpr int OCC_SLOTS = 8192;
+struct CtrlS {
+  int ok;
+  long long next, retired;
+  int active;
+  unsigned retire_head;
+  int admit_slot, admit_inst, admit_seq, admit_eval;
+  int src_count[4];
+  unsigned long long node_msgs;
+  unsigned occ[OCC_SLOTS / 32];
+  Deliv dl[MAXD];
+};
+
+// A source whose messages carry no payload of their own and feed a parameterised node directly (token ids, leaf ids,
+// the dense feature row): its headers go straight into that node's forward ring.
+__device__ __forceinline__ bool source_is_direct(const DevNode& sn) {
+  if (!(sn.fn == 1 || sn.fn == 2 || sn.fn == 4)) return false;
+  const DevNode& dn = g_nodes[sn.succ_node[0]];
+  return (dn.type == LINEAR || dn.type == LOOKUP) && g_ppts[dn.ppt].xcache == nullptr;
+}
+
+__device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsigned long long t0) {
+  IN_SMEM(&S);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const DevInst& I = C.inst;
+  if (tid == 0) { S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; S.node_msgs = 0; }
+  for (int i = tid; i < OCC_SLOTS / 32; i += FT) S.occ[i] = 0u;
+  __syncthreads();
+  unsigned idle = 0;
+  for (;;) {
+    // ---- retirements: sum the instance's loss cells in key order, free the slot ------------------------------
+    if (warp == 0) {
+      for (;;) {
+        unsigned h = 0, ready = 0;
+        if (lane == 0) { h = S.retire_head; ready = ld_acq(&C.retire_seq[h & C.retire_mask]) == h + 1u; }
+        h = warp_uniform(h);
+        if (!warp_uniform(ready)) break;
+        const int slot = (int)__ldcg(&C.retire_e[h & C.retire_mask]);
+        __syncwarp();
+        if (lane == 0) S.retire_head = h + 1u;
+        const int inst = C.slot_inst[slot];
+        double tot = 0.0; int okc = 0, np = 0;
+        for (int li = 0; li < C.n_loss; li++) {
+          const DevNode& L = g_nodes[C.loss_nodes[li]];
+          const long long k0 = (long long)slot * C.IT * L.U_in, k1 = k0 + (long long)C.IT * L.U_in;
+          double dpart = 0.0;
+          for (long long k = k0 + lane; k < k1; k += 32) {
+            const int pk = __ldcg(&L.predok[k]);
+            if (pk >= 0) { dpart += (double)__ldcg(&L.lossval[k]); okc += pk; np += 1; }
+          }
+          for (int o = 16; o; o >>= 1) dpart += __shfl_xor_sync(0xffffffffu, dpart, o);
+          tot += dpart;
+        }
+        for (int o = 16; o; o >>= 1) { okc += __shfl_xor_sync(0xffffffffu, okc, o); np += __shfl_xor_sync(0xffffffffu, np, o); }
+        if (lane == 0) {
+          C.loss_out[inst] = (float)tot;
+          if (C.inference_only && C.inference_only[inst]) { C.g->inf_loss += tot; C.g->inf_instances += 1; C.g->inf_correct += okc; C.g->inf_pred += np; }
+          else { C.g->total_loss += tot; C.g->correct += okc; C.g->n_pred += np; }
+          C.slot_inst[slot] = -1;
+          if (slot < OCC_SLOTS) S.occ[slot >> 5] &= ~(1u << (slot & 31));
+          S.active--; S.retired++;
+        }
+        __syncwarp();
+      }
+    }
+    __syncthreads();
+    // ---- admission -------------------------------------------------------------------------------------------
+    for (;;) {
+      if (tid == 0) {
+        S.admit_slot = -1;
+        if (S.active < C.mak && S.next < C.n_order) {
+          int slot = 0;                                                   // lowest free slot
+          const int nw = (min(C.mak, OCC_SLOTS) + 31) >> 5;
+          int w = 0;
+          while (w < nw && S.occ[w] == 0xffffffffu) w++;
+          if (w < nw) slot = w * 32 + __ffs(~S.occ[w]) - 1;
+          else { slot = OCC_SLOTS; while (slot < C.mak && C.slot_inst[slot] >= 0) slot++; }
+          if (slot < OCC_SLOTS) S.occ[slot >> 5] |= 1u << (slot & 31);
+          const int inst = (int)(C.order ? C.order[S.next] : S.next);
+          if (C.slot_inst[slot] >= 0) fail(C, ST_OVERFLOW, -32, slot);
+          S.admit_slot = slot; S.admit_inst = inst; S.admit_seq = (int)S.next;
+          C.slot_inst[slot] = inst;
+          S.active++;
+          if (S.active > C.g->max_active) C.g->max_active = S.active;
+          int total = 0;
+          for (int s = 0; s < C.n_sources; s++) {
+            const DevNode& sn = g_nodes[C.src_nodes[s]];
+            int cnt = 1;
+            if (sn.fn == 2) cnt = (int)(I.offsets[inst + 1] - I.offsets[inst]);
+            else if (sn.fn == 4) cnt = (int)(I.leaf_off[inst + 1] - I.leaf_off[inst]);
+            S.src_count[s] = cnt; total += cnt;
+          }
+          S.admit_eval = C.eval || (C.inference_only && C.inference_only[inst]);
+          if (S.admit_eval) {      // forward only: the instance is finished when every Loss / Sink has been reached
+            int exp = C.ends_per_instance;
+            if (C.ends_per_position) exp += C.ends_per_position * (int)(I.offsets[inst + 1] - I.offsets[inst]);
+            C.outstanding[slot] = exp * JOIN_UNIT;
+          } else C.outstanding[slot] = total * JOIN_UNIT;
+          S.next++;
+        }
+      }
+      __syncthreads();
+      const int slot = S.admit_slot;
+      if (slot < 0) break;
+      // clear the slot's loss cells (predok = -1 marks "no loss evaluated at this key")
+      for (int li = 0; li < C.n_loss; li++) {
+        const DevNode& L = g_nodes[C.loss_nodes[li]];
+        const long long k0 = (long long)slot * C.IT * L.U_in, cnt = (long long)C.IT * L.U_in;
+        for (long long k = tid; k < cnt; k += FT) { L.lossval[k0 + k] = 0.f; L.predok[k0 + k] = -1; }
+      }
+      __threadfence();
+      __syncthreads();
+      // pump the source messages (Sec. 4: tokens / leaves, initial hidden state, dense row)
+      const int inst = S.admit_inst;
+      Hdr h; h.inst = inst; h.seq = S.admit_seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = 1; h.flags = S.admit_eval ? HDR_EVAL : 0;
+      for (int s = 0; s < C.n_sources; s++) {
+        const DevNode& sn = g_nodes[C.src_nodes[s]];
+        const int cnt = S.src_count[s];
+        if (source_is_direct(sn)) {
+          DevPPT& P = g_ppts[g_nodes[sn.succ_node[0]].ppt];
+          for (int c0 = warp * 32; c0 < cnt; c0 += FW * 32) {
+            const int k = c0 + lane;
+            int u = 0;
+            if (k < cnt) u = sn.fn == 2 ? k : sn.fn == 4 ? I.leaf_ids[I.leaf_off[inst] + k] : 0;
+            const bool okm = k < cnt && key_of(C, sn.succ_node[0], slot, 0, u, P.U) >= 0;
+            const unsigned vm = __ballot_sync(0xffffffffu, okm);
+            unsigned tk = 0;
+            if (lane == 0 && vm) tk = atomicAdd(P.ring[FWD].tail, (unsigned)__popc(vm));
+            tk = __shfl_sync(0xffffffffu, tk, 0) + (unsigned)__popc(vm & ((1u << lane) - 1u));
+            if (okm) {
+              const unsigned q = tk & P.ring[FWD].mask;
+              int4* d = reinterpret_cast<int4*>(&P.ring[FWD].e[q]);
+              d[0] = make_int4(inst, S.admit_seq, slot, 0);
+              d[1] = make_int4(u, 0, 1, h.flags);
+              st_rel(&P.ring[FWD].seq[q], tk + 1u);
+            }
+            if (lane == 0 && vm) atomicAdd(&S.node_msgs, (unsigned long long)__popc(vm));
+          }
+        } else if (warp == 0) {                     // a zero vector (initial hidden state) routed to where it lands
+          int pre = 0, nd = 0;
+          if (lane == 0) {
+            nd = route_message(C, h, sn.succ_node[0], sn.succ_port[0], FWD, sn.out_dim, S.dl, pre);
+            for (int q = 0; q < nd; q++) S.dl[q].zero = 1;
+          }
+          nd = (int)warp_uniform((unsigned)nd);
+          __syncwarp();
+          for (int q = 0; q < nd; q++) {
+            const Deliv& L = S.dl[q];
+            if (L.act == ACT_PUSH && L.dst) for (int c = lane; c < L.w; c += 32) L.dst[c] = 0.f;
+          }
+          __syncwarp();
+          if (lane == 0) {
+            if (pre) atomicAdd(&S.node_msgs, (unsigned long long)pre);
+            for (int q = 0; q < nd; q++) arrive(C, h, S.dl[q], JOIN_UNIT, &S.node_msgs);
+          }
+          __syncwarp();
+        }
+      }
+      __syncthreads();
+    }
+    // ---- termination / pacing ---------------------------------------------------------------------------------
+    const bool finished = S.retired == C.n_order;
+    if (finished) {
+      if (tid == 0) { C.g->rounds = 0; atomicAdd(&C.g->node_messages, S.node_msgs); __threadfence(); st_rel(&C.g->done, 1u); }
+      break;
+    }
+    if (tid == 0) {
+      S.ok = 1;
+      if ((++idle & 15u) == 0) {
+        if (aborted(C)) S.ok = 0;
+        else if (gtime() - t0 > C.timeout_ns) { fail(C, ST_TIMEOUT, -1, 2); S.ok = 0; }
+      }
+      const unsigned hh = S.retire_head;
+      unsigned spins = 0;
+      while (ld_acq(&C.retire_seq[hh & C.retire_mask]) != hh + 1u && spins < 64) { __nanosleep(50); spins++; }
+    }
+    __syncthreads();
+    if (!S.ok) break;
+  }
+}
+
+union FastShared { TileS t; CtrlS c; };
+
+}  // namespace ampf
+
+__global__ void __launch_bounds__(ampf::FT, 1) ampnet_engine_direct(const __grid_constant__ amp::Ctx C) {
+  using namespace ampf;
+  extern __shared__ __align__(16) float dyn_smem[];
+  __shared__ FastShared SU;
+  const unsigned long long t0 = gtime();
+  {
+    const int* src = reinterpret_cast<const int*>(C.nodes);
+    int* dst = reinterpret_cast<int*>(g_nodes);
+    for (int i = threadIdx.x; i < C.n_nodes * (int)(sizeof(DevNode) / 4); i += FT) dst[i] = src[i];
+    src = reinterpret_cast<const int*>(C.ppts);
+    dst = reinterpret_cast<int*>(g_ppts);
+    for (int i = threadIdx.x; i < C.n_ppts * (int)(sizeof(DevPPT) / 4); i += FT) dst[i] = src[i];
+  }
+  if (threadIdx.x == 0) g_bf16 = C.bf16;
+  __syncthreads();
+  const Role role = C.roles[blockIdx.x];
+  if (role.ppt < 0) controller_main(C, SU.c, t0);
+  else if (role.kind == 3) bwd_tile_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
+  else tile_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side: what the launch needs to know
+// ------------------------------------------------------------------------------------------------
+namespace ampf {
+size_t tile_smem_floats(int in, int R, int BM) {
+  const size_t LW = pad_ldx(in), LX = pad_ldx(in), RP = pad4(R > 0 ? R : 1);
+  return 2 * (size_t)R * LW + 2 * RP + (size_t)BM * LX + 2 * (size_t)BM * RP + XWT_SCRATCH;
+}
+}  // namespace ampf
+
+namespace ampf {
+size_t bwd_tile_smem_floats(int out, int cb, int BM) { const size_t GL = pad_ldx(out); return (size_t)cb * GL + (size_t)BM * GL + 2 * (size_t)BM * cb + 2 * GL; }
+}  // namespace ampf
+extern "C" size_t ampnet_direct_bwd_tile_smem_bytes(int out_dim, int cols, int batch_rows) { return ampf::bwd_tile_smem_floats(out_dim, cols, batch_rows) * sizeof(float) + 64; }
+extern "C" int ampnet_direct_max_units() { return ampf::MAXU * ampf::FT; }
+extern "C" int ampnet_direct_threads() { return ampf::FT; }
+extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows) { return ampf::tile_smem_floats(in_dim, rows, batch_rows) * sizeof(float) + 64; }
+extern "C" cudaError_t ampnet_direct_static_smem(size_t* bytes) {
+  cudaFuncAttributes fa{};
+  const cudaError_t e = cudaFuncGetAttributes(&fa, ampnet_engine_direct);
+  *bytes = fa.sharedSizeBytes;
+  return e;
+}
+extern "C" cudaError_t ampnet_direct_launch(const amp::Ctx* ctx, int n_ctas, size_t smem_bytes, cudaStream_t stream, int n_sms) {
+  cudaError_t e = cudaFuncSetAttribute(ampnet_engine_direct, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+  if (e != cudaSuccess) return e;
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, ampnet_engine_direct, ampf::FT, smem_bytes);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1 || (long long)per_sm * n_sms < n_ctas) return cudaErrorCooperativeLaunchTooLarge;
+  void* args[] = {const_cast<amp::Ctx*>(ctx)};
+  return cudaLaunchCooperativeKernel((void*)ampnet_engine_direct, dim3(n_ctas), dim3(ampf::FT), args, smem_bytes, stream);
+}

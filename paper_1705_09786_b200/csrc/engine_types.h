@@ -14,6 +14,7 @@ constexpr int MAX_SMEM_NODES = 40;    // IR nodes / PPT nodes whose tables are k
 constexpr int MAX_SMEM_PPTS = 16;
 constexpr int MAX_TILES = 32;        // row tiles per PPT node
 constexpr int WALK_STACK = 12;        // continuation frames per walking warp
+constexpr int JOIN_UNIT = 4096;       // direct-delivery engine: one whole message in a join counter; a row tile arrives with its share
 
 enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, CONCAT, SPLIT,
                 BCAST, GROUP, UNGROUP, FLATMAP, SINK, NPT_LSTM, N_NODE_TYPES };
@@ -108,6 +109,10 @@ struct DevPPT {
   PPTStats* stats;
   int* update_log; int update_log_cap;
   int smem_floats;
+  int* injoin[2];                     // direct-delivery engine: arrival counter per key and direction (in units of JOIN_UNIT per message)
+  int TB, CB, NS, bwd_smem_floats;    // direct-delivery engine: backward column tiles and input columns per tile; gradient slots per key
+                                      // in gbuf ([key][NS][out]: one per successor of the Bcast whose backward sum forms there)
+  unsigned* wver;                     // backward tiles that have published their columns, summed over the updates (TB per update)
 };
 
 struct DevInst {                      // instances + routing tables produced by the structure encoder
@@ -150,7 +155,8 @@ struct Globals {                      // mutable run state in device memory (zer
   unsigned long long step_cycles[MAX_SMEM_PPTS][16];   // tile 0 of every node: cycles between the marks inside the arithmetic phase
 };
 
-struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of the node's emitter CTAs (pad = which one), 2: the node's scheduler CTA
+struct Role { int ppt, tile, kind, pad; };   // kind 0: row tile, 1: one of the node's emitter CTAs (pad = which one), 2: the node's scheduler CTA,
+                                             // 3: backward column tile (direct-delivery engine)
 
 struct Ctx {
   DevNode* nodes; int n_nodes;

@@ -23,9 +23,13 @@ def test_static_scratch_epoch_matches_the_allocating_epoch_twice_in_a_row():
     for e in (a, b):
         e.load_instances(inst)
         e.set_params(p)
+    order = np.random.default_rng(3).permutation(inst.n)
     for call in range(2):
-        sa, la = a.run_epoch(mak=16, muf=50, lr=0.05, deterministic=True, timeout_s=60)
-        sb, lb = b.run_epoch(mak=16, muf=50, lr=0.05, deterministic=True, timeout_s=60, static_scratch=True)
+        od = None if call == 0 else order          # the second call also carries an epoch order (part of the size check)
+        sa, la = a.run_epoch(mak=16, muf=50, lr=0.05, deterministic=True, timeout_s=60, order=od)
+        calls = (b.alloc_calls, b.free_calls, len(b._blocks))
+        sb, lb = b.run_epoch(mak=16, muf=50, lr=0.05, deterministic=True, timeout_s=60, static_scratch=True, order=od)
+        assert (b.alloc_calls, b.free_calls, len(b._blocks)) == calls, "the static epoch went to the allocator"
         assert (sb.node_messages, sb.ppt_messages, sb.rounds, sb.route_hash) == \
                (sa.node_messages, sa.ppt_messages, sa.rounds, sa.route_hash), call
         np.testing.assert_allclose(lb, la, rtol=1e-5, atol=2e-6)
@@ -41,6 +45,29 @@ def test_static_scratch_epoch_matches_the_allocating_epoch_twice_in_a_row():
     np.testing.assert_allclose(lb, la, rtol=1e-5, atol=2e-6)
     a.close()
     b.close()
+
+
+def test_static_scratch_never_allocates_near_its_size_limit():
+    """Runs whose scratch lands just under and just over the fixed array's size: the first must run without a single
+    allocator call, the second must be refused before anything runs (never served from allocator memory)."""
+    import paper_1705_09786_b200 as amp
+    g = ir.rnn()
+    inst = data.list_instances(n=40)
+    fits, refused = 0, 0
+    for mak in (256, 512, 768, 1024, 1280, 1536, 2048, 3072):      # scratch grows with the keys in flight
+        e = amp.Engine(g)
+        e.load_instances(inst)
+        calls = (e.alloc_calls, e.free_calls, len(e._blocks))
+        try:
+            st, _ = e.run_epoch(mak=mak, muf=50, lr=0.05, timeout_s=60, static_scratch=True)
+            assert st.instances == inst.n
+            fits += 1
+        except amp.AmpnetError as err:
+            assert err.status == 1 and "bytes" in str(err)
+            refused += 1
+        assert (e.alloc_calls, e.free_calls, len(e._blocks)) == calls, mak
+        e.close()
+    assert fits >= 1 and refused >= 1
 
 
 def test_static_scratch_refuses_runs_that_do_not_fit():
