@@ -20,9 +20,10 @@ using namespace amp;
 
 // host hooks of the direct-delivery engine (engine_fast.cu)
 extern "C" int ampnet_direct_threads();
-extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows);
+extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows, int loss_head);
 extern "C" size_t ampnet_direct_bwd_tile_smem_bytes(int out_dim, int cols, int batch_rows);
 extern "C" int ampnet_direct_max_units();
+extern "C" void ampnet_direct_limits(int* max_nodes, int* max_ppts, int* max_landings, int* batch_rows);
 extern "C" cudaError_t ampnet_direct_static_smem(size_t* bytes);
 extern "C" cudaError_t ampnet_direct_launch(const amp::Ctx* ctx, int n_ctas, size_t smem_bytes, cudaStream_t stream, int n_sms);
 
@@ -561,6 +562,9 @@ bool direct_candidate(ampnet_graph* g, const HostDataset& D, int det) {
   if (const char* e = getenv("AMPNET_TUNE")) if (atoi(e) & (16 | 32 | 8)) return false;
   if (D.kind == 3) return false;
   const int n = (int)g->hnodes.size();
+  int max_nodes = 0, max_ppts = 0, max_landings = 0, batch_rows = 0;
+  ampnet_direct_limits(&max_nodes, &max_ppts, &max_landings, &batch_rows);
+  if (n > max_nodes || (int)g->ppts.size() > max_ppts) return false;
   for (int i = 0; i < n; i++) {
     const DevNode& h = g->hnodes[i];
     if (h.rows_in != 1 || h.rows_out != 1) return false;
@@ -570,9 +574,11 @@ bool direct_candidate(ampnet_graph* g, const HostDataset& D, int det) {
       case LOSS_CE: case LOSS_MSE: if (g->hnodes[h.pred_node[0]].type != LINEAR) return false; break;
       case CONCAT: {
         const DevNode& s = g->hnodes[h.succ_node[0]];
+        if (h.fn_arg > max_landings) return false;
         if (s.type != LINEAR || (s.in_dim & 3) || s.in_dim != h.out_dim || s.U_in != h.U_out || s.rows_in != h.rows_in) return false;
       } break;
       case BCAST: {
+        if (h.fn_arg > max_landings) return false;
         // backward, the sum forms in the gradient buffer of the parameterised node behind Phi / Cond / Isu
         std::vector<int> todo{h.pred_node[0]};
         std::vector<char> seen(n, 0);
@@ -605,6 +611,8 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   if (const char* e = getenv("AMPNET_DIRECT_ROWS")) rows = std::max(1, atoi(e));
   if (const char* e = getenv("AMPNET_DIRECT_COLS")) { const int c = atoi(e); if (c == 4 || c == 8 || c == 16 || c == 32) cols = c; }
   const int np = (int)g->ppts.size(), tile_budget = n_ctas - 1, max_units = ampnet_direct_max_units();
+  int lim_nodes = 0, lim_ppts = 0, lim_landings = 0, BATCH = MAX_BATCH_ROWS;
+  ampnet_direct_limits(&lim_nodes, &lim_ppts, &lim_landings, &BATCH);
   std::vector<int> fixed(np, 0);
   // gradient slots: the backward sum of a Bcast forms in the gradient buffer of the node behind Phi / Cond / Isu
   for (auto& P : g->ppts) P.NS = 1;
@@ -626,9 +634,9 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
     HostPPT& P = g->ppts[p];
     const DevNode& h = g->hnodes[P.node];
     P.NE = 0; P.G = 1; P.a_global = false; P.J = 0; P.TB = 0; P.CB = 0; P.bwd_smem_floats = 0;
-    if (P.kind == LOOKUP) { P.T = (P.in >= 4096 && tile_budget >= 24) ? 4 : 1; P.R = 0; P.BM = MAX_BATCH_ROWS; fixed[p] = 1; continue; }
+    if (P.kind == LOOKUP) { P.T = (P.in >= 4096 && tile_budget >= 24) ? 4 : 1; P.R = 0; P.BM = BATCH; fixed[p] = 1; continue; }
     const int st = g->hnodes[h.succ_node[0]].type;
-    P.BM = MAX_BATCH_ROWS;
+    P.BM = BATCH;
     if (st == LOSS_CE || st == LOSS_MSE) { P.R = P.out; fixed[p] = 1; }
     else {
       P.R = std::min(P.out, rows);
@@ -638,14 +646,14 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
     }
   }
   auto fits = [&](const HostPPT& P) {
-    return ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM) <= budget && (P.CB == 0 || ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) <= budget);
+    return ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM, P.CB == 0) <= budget && (P.CB == 0 || ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) <= budget);
   };
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
     if (P.kind == LOOKUP) continue;
     while (!fits(P)) {
       if (P.BM > 16) P.BM /= 2;
-      else if (!fixed[p] && P.R > 1) { P.R = (P.R + 1) / 2; P.BM = MAX_BATCH_ROWS; }
+      else if (!fixed[p] && P.R > 1) { P.R = (P.R + 1) / 2; P.BM = BATCH; }
       else return AMPNET_EOVERFLOW;
     }
   }
@@ -670,7 +678,7 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   roles.push_back(Role{-1, 0, 0, 0});
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
-    P.smem_floats = P.kind == LOOKUP ? 64 : ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM) / sizeof(float);
+    P.smem_floats = P.kind == LOOKUP ? 64 : ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM, P.CB == 0) / sizeof(float);
     P.bwd_smem_floats = P.TB ? ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) / sizeof(float) : 0;
     for (int t = 0; t < P.T; t++) roles.push_back(Role{p, t, 0, 0});
     for (int t = 0; t < P.TB; t++) roles.push_back(Role{p, t, 3, 0});
@@ -917,6 +925,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   X.opt = g->opt; X.mu = g->opt_mu; X.beta1 = g->opt_beta1; X.beta2 = g->opt_beta2; X.eps = g->opt_eps;
   double to = cfg && cfg->timeout_s > 0 ? cfg->timeout_s : 120.0;
   X.timeout_ns = (unsigned long long)(to * 1e9);
+  X.ctl_base = C.base;
   R.smem_bytes = max_smem_floats * sizeof(float);
   return AMPNET_OK;
 }

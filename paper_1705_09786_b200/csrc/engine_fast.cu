@@ -26,8 +26,8 @@ using namespace amp;
 
 constexpr int FT = 512;               // threads per CTA
 constexpr int FW = FT / 32;
-constexpr int FBM = 64;               // messages (= rows) per micro-batch
-constexpr int MAXD = 4;               // landings per message
+constexpr int FBM = 128;              // messages (= rows) per micro-batch
+constexpr int MAXD = 2;               // landings per message
 constexpr int RSTACK = 4;             // pending forks per routed message
 
 // ------------------------------------------------------------------------------------------------
@@ -81,8 +81,9 @@ __device__ __forceinline__ long long key_of(const Ctx& C, int node, int slot, in
 // the compiler their address space.
 #define IN_SMEM(p) __builtin_assume(__isShared(p))
 
-__shared__ DevNode g_nodes[MAX_SMEM_NODES];
-__shared__ DevPPT g_ppts[MAX_SMEM_PPTS];
+constexpr int DIRECT_MAX_NODES = 24, DIRECT_MAX_PPTS = 12;      // the graphs this engine takes are small (checked on the host)
+__shared__ DevNode g_nodes[DIRECT_MAX_NODES];
+__shared__ DevPPT g_ppts[DIRECT_MAX_PPTS];
 __shared__ int g_bf16;
 // What a node emits as a payload: identity for fp32 messages, rounded to bfloat16 (nearest even) otherwise.
 __device__ __forceinline__ float emit_round(float v) { return g_bf16 ? __bfloat162float(__float2bfloat16_rn(v)) : v; }
@@ -122,6 +123,29 @@ struct __align__(16) Deliv {
                                   // zero: the payload is a zero vector (deposit zeros of width w)
 };
 
+// The same, as it is kept per message in shared memory (48 bytes): counters and origins live in the control arena and
+// are addressed by their byte offsets from its start (0: none).
+struct __align__(16) Landing {
+  float* dst;
+  unsigned jcnt_off, clear_off, clear2_off;
+  int expected;
+  unsigned short s0, w;
+  int u;
+  unsigned char act, dir, ppt, port, zero, post, it, pad0;
+  short node, pad1;
+};
+__device__ __forceinline__ Landing pack_landing(const Ctx& C, const Deliv& d) {
+  Landing L;
+  L.dst = d.dst;
+  L.jcnt_off = d.jcnt ? (unsigned)((char*)d.jcnt - C.ctl_base) : 0u;
+  L.clear_off = d.clear ? (unsigned)((char*)d.clear - C.ctl_base) : 0u;
+  L.clear2_off = d.clear2 ? (unsigned)((char*)d.clear2 - C.ctl_base) : 0u;
+  L.expected = d.expected; L.s0 = (unsigned short)d.s0; L.w = (unsigned short)d.w; L.u = d.u;
+  L.act = (unsigned char)d.act; L.dir = (unsigned char)d.dir; L.ppt = (unsigned char)d.ppt; L.port = (unsigned char)d.port;
+  L.zero = (unsigned char)d.zero; L.post = (unsigned char)d.post; L.it = (unsigned char)d.it; L.pad0 = 0; L.node = (short)d.node; L.pad1 = 0;
+  return L;
+}
+
 struct Route {                    // state of one message on its way through the parameter-free nodes
   int node, aport, dir, u, it, port, s0, w, null;
 };
@@ -131,7 +155,7 @@ struct Route {                    // state of one message on its way through the
 // sums, Concat joins and splits) and writes the landings to out[0 .. returned count).  pre: node-messages consumed on
 // the way that every arrival sees (added once per message by the first row tile).  width: payload width at the start.
 __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_node, int start_aport, const int dir0, const int width,
-                                          Deliv* out, int& pre) {
+                                          Landing* out, int& pre) {
   IN_SMEM(out);
   const DevInst& I = C.inst;
   const long long ibase = I.offsets ? I.offsets[h.inst] : 0;
@@ -155,7 +179,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
     auto land = [&](Deliv d) {
       if (nout >= MAXD) { fail(C, ST_OVERFLOW, f.node, -9); return; }
       d.clear = clear; d.clear2 = clear2; d.zero = f.null ? 1 : 0;
-      out[nout++] = d;
+      out[nout++] = pack_landing(C, d);
       pend = nullptr; pend_exp = 0; pend_slot = 0; post = 0; clear = clear2 = nullptr; phi_cnt = nullptr;
     };
     switch (n.type) {
@@ -311,11 +335,17 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
 // tile state and arithmetic
 // ------------------------------------------------------------------------------------------------
 struct TileS {
-  Hdr hdr[FBM];
+  // Two batches are in flight in a tile: while most warps arrive for batch n, four warps already form batch n + 1 and
+  // resolve its routes.  Headers, landings and counts are kept per batch parity.
+  Hdr hdr[2][FBM];
+  Landing dl[2][FBM][MAXD];
+  unsigned char nd[2][FBM];
+  short pre[2][FBM];
   long long key[FBM];
   const float* rowptr[FBM];
-  Deliv dl[FBM][MAXD];
-  int nd[FBM], pre[FBM], rowid[FBM];
+  int rowid[FBM];
+  int fpb;                          // parity of the batch being formed
+  unsigned arr_done;                // arrival warps that have finished, summed over the batches
   int count, dir, flags, n_upd, upd_t, eval, ok, term;
   unsigned head[2];
   int n_acc, version, log_n, max_stale;
@@ -335,34 +365,81 @@ struct FastDiv {
   __device__ __forceinline__ int div(int n) const { return (int)__umulhi((unsigned)n, M); }
 };
 __host__ __device__ __forceinline__ int pad_ldx(int in) { int l = (in + 3) & ~3; while ((l & 7) != 4) l += 4; return l; }
-constexpr int XWT_SCRATCH = 0;
-
 // out[b][o] = sum_k A[b][k] B[o][k] for b < nA, o < nB: both operands in shared memory with k contiguous, rows padded
-// with zeros to K4 groups of four and strides of 4 (mod 8) floats (eight rows read 16 bytes each without a bank
-// conflict).  A thread owns one output and one of nsl interleaved k-slices, as many slices as keep every thread busy
-// (a single message still spreads over the whole CTA); the slices meet by shuffles.  Whole CTA, no barrier inside.
+// with zeros to K4 groups of four and strides of 4 (mod 8) floats.  A thread owns a 4 x 4 block of outputs (eight 16-byte
+// loads feed 64 multiply-adds: two bytes of shared-memory traffic per multiply-add instead of eight) and one of nsl
+// interleaved k-slices, as many slices as keep every thread busy (a single message still spreads over the CTA); the
+// slices meet by shuffles.  Whole CTA, no barrier inside.
+template <int TA>
+__device__ __forceinline__ void gemm_nt_t(const float* __restrict__ A, const int lda, const int nA, const float* __restrict__ B, const int ldb,
+                                          const int nB, const int K4, float* __restrict__ out, const int ldo) {
+  const int tid = threadIdx.x;
+  const int tA = (nA + TA - 1) / TA, tB = (nB + 3) >> 2, n_tiles = tA * tB;
+  int nsl = 1, sh = 0;
+  while (nsl < 32 && n_tiles * nsl * 2 <= FT) { nsl <<= 1; sh++; }
+  const int per_pass = FT >> sh, ks = tid & (nsl - 1);
+  const FastDiv dB(tB);
+  for (int t0 = 0; t0 < n_tiles; t0 += per_pass) {
+    const int ti = t0 + (tid >> sh);
+    const bool valid = ti < n_tiles;
+    const int bt = valid ? dB.div(ti) : 0, ot = valid ? ti - bt * tB : 0;
+    const float4* const A4 = reinterpret_cast<const float4*>(A);
+    const float4* const B4 = reinterpret_cast<const float4*>(B);
+    const int lda4 = lda >> 2, ldb4 = ldb >> 2;
+    const int a0 = min(TA * bt, nA - 1) * lda4, a1 = min(TA * bt + 1, nA - 1) * lda4, a2 = min(TA * bt + 2, nA - 1) * lda4, a3 = min(TA * bt + 3, nA - 1) * lda4;
+    const int w0 = min(4 * ot, nB - 1) * ldb4, w1 = min(4 * ot + 1, nB - 1) * ldb4, w2 = min(4 * ot + 2, nB - 1) * ldb4, w3 = min(4 * ot + 3, nB - 1) * ldb4;
+    float acc[TA][4];
+#pragma unroll
+    for (int m = 0; m < TA; m++)
+#pragma unroll
+      for (int j = 0; j < 4; j++) acc[m][j] = 0.f;
+#pragma unroll 2
+    for (int k4 = ks; k4 < K4; k4 += nsl) {
+      float4 x[4];
+      x[0] = A4[a0 + k4];
+      if (TA > 1) { x[1] = A4[a1 + k4]; x[2] = A4[a2 + k4]; x[3] = A4[a3 + k4]; }
+      const float4 y[4] = {B4[w0 + k4], B4[w1 + k4], B4[w2 + k4], B4[w3 + k4]};
+#pragma unroll
+      for (int m = 0; m < TA; m++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+          acc[m][j] = fmaf(x[m].x, y[j].x, acc[m][j]); acc[m][j] = fmaf(x[m].y, y[j].y, acc[m][j]);
+          acc[m][j] = fmaf(x[m].z, y[j].z, acc[m][j]); acc[m][j] = fmaf(x[m].w, y[j].w, acc[m][j]);
+        }
+    }
+    for (int off = 1; off < nsl; off <<= 1)
+#pragma unroll
+      for (int m = 0; m < TA; m++)
+#pragma unroll
+        for (int j = 0; j < 4; j++) acc[m][j] += __shfl_xor_sync(0xffffffffu, acc[m][j], off);
+    if (valid && ks == 0) {
+#pragma unroll
+      for (int m = 0; m < TA; m++)
+#pragma unroll
+        for (int j = 0; j < 4; j++)
+          if (TA * bt + m < nA && 4 * ot + j < nB) out[(TA * bt + m) * ldo + 4 * ot + j] = acc[m][j];
+    }
+  }
+}
+// A handful of messages: one row of A per thread (nothing is spent on padding rows); otherwise 4 x 4 blocks.
 __device__ __forceinline__ void gemm_nt(const float* __restrict__ A, const int lda, const int nA, const float* __restrict__ B, const int ldb,
                                         const int nB, const int K4, float* __restrict__ out, const int ldo) {
-  const int tid = threadIdx.x, n_out = nA * nB;
-  int nsl = 1, sh = 0;
-  while (nsl < 32 && n_out * nsl * 2 <= FT) { nsl <<= 1; sh++; }
-  const int per_pass = FT >> sh, ks = tid & (nsl - 1);
-  const FastDiv dB(nB);
-  for (int o0 = 0; o0 < n_out; o0 += per_pass) {
-    const int oi = o0 + (tid >> sh);
-    const bool valid = oi < n_out;
-    const int b = valid ? dB.div(oi) : 0, o = valid ? oi - b * nB : 0;
-    const float4* a = reinterpret_cast<const float4*>(A + (size_t)b * lda);
-    const float4* w = reinterpret_cast<const float4*>(B + (size_t)o * ldb);
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll 4
-    for (int k4 = ks; k4 < K4; k4 += nsl) {
-      const float4 x = a[k4], y = w[k4];
-      a0 = fmaf(x.x, y.x, a0); a1 = fmaf(x.y, y.y, a1); a2 = fmaf(x.z, y.z, a2); a3 = fmaf(x.w, y.w, a3);
+  if (nA <= 8) gemm_nt_t<1>(A, lda, nA, B, ldb, nB, K4, out, ldo);
+  else gemm_nt_t<4>(A, lda, nA, B, ldb, nB, K4, out, ldo);
+}
+
+// Columns [col0, col0 + ncols) of every message's payload are in M (shared memory, one row per message): a warp per
+// message copies what falls into each landing's column range, rounded like every emitted payload.
+__device__ __forceinline__ void deliver_cols(const TileS& S, const int pb, const float* __restrict__ M, const int ldm, const int count, const int col0, const int ncols) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int b = warp; b < count; b += FW) {
+    const int nd = S.nd[pb][b];
+    for (int q = 0; q < nd; q++) {
+      const Landing& L = S.dl[pb][b][q];
+      if (L.act != ACT_PUSH || !L.dst) continue;
+      const int lo = max(L.s0, col0), hi = min(L.s0 + L.w, col0 + ncols);
+      for (int i = lo + lane; i < hi; i += 32) L.dst[i - L.s0] = emit_round(M[b * ldm + (i - col0)]);
     }
-    float v = (a0 + a1) + (a2 + a3);
-    for (int off = 1; off < nsl; off <<= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
-    if (valid && ks == 0) out[b * ldo + o] = v;
   }
 }
 
@@ -422,36 +499,37 @@ __device__ __noinline__ void retire_arrive(const Ctx& C, int slot, int wgt) {
   st_rel(&C.retire_seq[s], t + 1u);
 }
 // One thread, after the barrier behind the deposits of its CTA: arrive at landing L of message h with weight wgt.
-__device__ __noinline__ void arrive(const Ctx& C, const Hdr& h, const Deliv& L, int wgt, unsigned long long* node_msgs) {
-  IN_SMEM(&h); IN_SMEM(&L); IN_SMEM(node_msgs);
+__device__ __noinline__ void arrive(const Ctx& C, const int inst, const int seq, const int slot, const int flags, const Landing& L, int wgt,
+                                    unsigned long long* node_msgs) {
+  IN_SMEM(&L); IN_SMEM(node_msgs);
+  int* const jcnt = reinterpret_cast<int*>(C.ctl_base + L.jcnt_off);
+  Hdr h; h.inst = inst; h.seq = seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = 1; h.flags = flags;
   if (L.act == ACT_RETIRE && L.expected) {                       // the message's arrivals meet first, then it retires whole
-    if (atom_add_acq_rel(L.jcnt, wgt) + wgt != L.expected) return;
-    *(volatile int*)L.jcnt = 0;
-    if (L.clear) *L.clear = 0;
-    if (L.clear2) *L.clear2 = 0;
+    if (atom_add_acq_rel(jcnt, wgt) + wgt != L.expected) return;
+    *(volatile int*)jcnt = 0;
+    if (L.clear_off) *reinterpret_cast<unsigned char*>(C.ctl_base + L.clear_off) = 0;
+    if (L.clear2_off) *reinterpret_cast<unsigned char*>(C.ctl_base + L.clear2_off) = 0;
     if (L.post) atomicAdd(node_msgs, (unsigned long long)L.post);
-    retire_arrive(C, h.slot, JOIN_UNIT);
+    retire_arrive(C, slot, JOIN_UNIT);
     return;
   }
   if (L.act == ACT_RETIRE) {
-    const int old = atom_add_acq_rel(L.jcnt, -wgt);
-    if (old < wgt) fail(C, ST_OVERFLOW, -30, h.slot);
+    const int old = atom_add_acq_rel(jcnt, -wgt);
+    if (old < wgt) fail(C, ST_OVERFLOW, -30, slot);
     if (old != wgt) return;
-    if (L.clear) *L.clear = 0;
-    if (L.clear2) *L.clear2 = 0;
     if (L.post) atomicAdd(node_msgs, (unsigned long long)L.post);
     const unsigned t = atomicAdd(&C.g->retire_tail, 1u), s = t & C.retire_mask;
-    C.retire_e[s] = (unsigned)h.slot;
+    C.retire_e[s] = (unsigned)slot;
     st_rel(&C.retire_seq[s], t + 1u);
     return;
   }
   if (L.act != ACT_PUSH) return;
-  const int sum = atom_add_acq_rel(L.jcnt, wgt) + wgt;
+  const int sum = atom_add_acq_rel(jcnt, wgt) + wgt;
   if (sum > L.expected) fail(C, ST_OVERFLOW, L.node, -31);       // more arrivals than the landing expects
   if (sum != L.expected) return;
-  *(volatile int*)L.jcnt = 0;                                   // the key's next use finds the counter at zero
-  if (L.clear) *L.clear = 0;
-  if (L.clear2) *L.clear2 = 0;
+  *(volatile int*)jcnt = 0;                                     // the key's next use finds the counter at zero
+  if (L.clear_off) *reinterpret_cast<unsigned char*>(C.ctl_base + L.clear_off) = 0;
+  if (L.clear2_off) *reinterpret_cast<unsigned char*>(C.ctl_base + L.clear2_off) = 0;
   atomicAdd(node_msgs, (unsigned long long)L.post);
   ring_push(g_ppts[L.ppt].ring[L.dir], h, L.it, L.u, L.port);
 }
@@ -466,7 +544,7 @@ __device__ __forceinline__ unsigned long long ballot64(const bool p0, const bool
 // training and forward-only messages meet, and exactly at the gradient that triggers the update (Sec. 3).
 // dirs: bit 0 forward ring, bit 1 backward ring.  Returns 1 with the batch in S, 2 when the epoch is over, 0 when
 // nothing is pending.
-__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const bool leader, const bool fused, const int dirs, const bool light) {
+__device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const bool leader, const bool fused, const int dirs, const bool light, const int min_take) {
   IN_SMEM(&P); IN_SMEM(&S);
   const int lane = threadIdx.x & 31;
   if (light) {                      // nothing was pending a moment ago: watch the two head slots (and the end of the epoch) only
@@ -476,24 +554,33 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
     if (!__any_sync(0xffffffffu, any != 0)) return 0;
   }
   if (dirs == 1 && lane == 0) S.wver_seen = ld_rlx(P.wver);          // ordered by the fence below like the ring polls
-  unsigned slot[2][2];
-  bool ready[2][2];
+  constexpr int NPL = FBM / 32;                                      // ring slots per lane
+  auto leading = [](const unsigned (&m)[NPL]) {                      // length of the run of set bits from candidate 0 on
+    int n = 0;
 #pragma unroll
-  for (int dir = 0; dir < 2; dir++)
-#pragma unroll
-    for (int j = 0; j < 2; j++) {
-      const unsigned t = S.head[dir] + lane + 32 * j;
-      slot[dir][j] = t & P.ring[dir].mask;
-      ready[dir][j] = ld_rlx(&P.ring[dir].seq[slot[dir][j]]) == t + 1u;
-    }
-  fence_acq();
+    for (int j = 0; j < NPL; j++) { if (m[j] == 0xffffffffu) n += 32; else { n += __ffs((int)~m[j]) - 1; break; } }
+    return n;
+  };
+  unsigned slot[2][NPL];
   int nready[2];
 #pragma unroll
   for (int dir = 0; dir < 2; dir++) {
-    const unsigned long long m = ballot64(ready[dir][0], ready[dir][1]);
-    nready[dir] = m == ~0ull ? 64 : __ffsll((long long)~m) - 1;
-    if (!(dirs & (1 << dir))) nready[dir] = 0;                     // forward row tiles / backward column tiles take one ring only
+    bool ready[NPL];
+#pragma unroll
+    for (int j = 0; j < NPL; j++) {
+      const unsigned t = S.head[dir] + lane + 32 * j;
+      slot[dir][j] = t & P.ring[dir].mask;
+      ready[j] = (dirs & (1 << dir)) && ld_rlx(&P.ring[dir].seq[slot[dir][j]]) == t + 1u;
+    }
+    unsigned m[NPL];
+#pragma unroll
+    for (int j = 0; j < NPL; j++) m[j] = __ballot_sync(0xffffffffu, ready[j]);
+    nready[dir] = leading(m);
   }
+  fence_acq();
+  // A batch costs nearly the same whether it holds 2 messages or 100.  While the previous batch's arrivals are still under
+  // way the next one is taken only if at least min_take messages wait; the caller drops the threshold once they are done.
+  if (max(nready[0], nready[1]) < min_take && max(nready[0], nready[1]) > 0) return 0;
   if (nready[0] == 0 && nready[1] == 0) {
     unsigned fin = 0;
     if (lane == 0) fin = ld_acq(&C.g->done);
@@ -509,12 +596,13 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
     __syncwarp();
     return 2;
   }
-  const bool fwd_first = !(C.tune & 128) && nready[BWD] < FBM / 2 && nready[FWD] > nready[BWD];
+  const bool fwd_first = !(C.tune & 128) && nready[BWD] < 32 && nready[FWD] > nready[BWD];
   const int dir = (nready[BWD] == 0 || (fwd_first && nready[FWD] > 0)) ? FWD : BWD;
   int take = min(nready[dir], P.BM);
-  Hdr h[2];
+  Hdr h[NPL];
+  unsigned em[NPL];
 #pragma unroll
-  for (int j = 0; j < 2; j++) {
+  for (int j = 0; j < NPL; j++) {
     h[j] = Hdr{0, 0, 0, 0, 0, 0, 0, 0};
     if (lane + 32 * j < take) {
       const int4* e = reinterpret_cast<const int4*>(&P.ring[dir].e[dir == FWD ? slot[FWD][j] : slot[BWD][j]]);
@@ -523,9 +611,9 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
     }
   }
   const int eval0 = __shfl_sync(0xffffffffu, (int)((h[0].flags & HDR_EVAL) != 0), 0);
-  const unsigned long long okm = ballot64(lane < take && (int)((h[0].flags & HDR_EVAL) != 0) == eval0,
-                                          lane + 32 < take && (int)((h[1].flags & HDR_EVAL) != 0) == eval0);
-  take = okm == ~0ull ? 64 : __ffsll((long long)~okm) - 1;
+#pragma unroll
+  for (int j = 0; j < NPL; j++) em[j] = __ballot_sync(0xffffffffu, lane + 32 * j < take && (int)((h[j].flags & HDR_EVAL) != 0) == eval0);
+  take = leading(em);
   bool upd = false;
   const bool grads = (dir == BWD || fused) && !eval0;          // a fused loss head turns every forward message into a gradient at once
   if (grads) {
@@ -533,7 +621,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
     if (S.n_acc + take >= muf) { take = max(1, muf - S.n_acc); upd = true; }
   }
 #pragma unroll
-  for (int j = 0; j < 2; j++) if (lane + 32 * j < take) S.hdr[lane + 32 * j] = h[j];
+  for (int j = 0; j < NPL; j++) if (lane + 32 * j < take) S.hdr[S.fpb][lane + 32 * j] = h[j];
   __syncwarp();
   if (lane == 0) {
     S.count = take; S.dir = dir; S.flags = upd ? BATCH_UPDATE : 0; S.eval = eval0;
@@ -585,7 +673,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   const bool lookup = P.kind == LOOKUP, leader = tile == 0;
   const int r_begin = tile * P.R;
   const int R = lookup ? 0 : max(0, min(P.R, out - r_begin));
-  const int LW = pad_ldx(in), LX = pad_ldx(in), RP = pad4(max(P.R, 1));
+  const int LW = pad_ldx(in), LX = pad_ldx(in), RP = pad_ldx(max(P.R, 1)), DXL = LX;
   const int wgt = tile == P.T - 1 ? JOIN_UNIT - (P.T - 1) * (JOIN_UNIT / P.T) : JOIN_UNIT / P.T;
   const DevNode& N = g_nodes[P.node];
   // A node that feeds a Loss is one tile and runs the whole exchange in one pass: forward, Loss, and the backward message
@@ -598,16 +686,22 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   // publish their columns and the row tiles reload their rows before their next batch.
   const bool fwd_only = !lookup && !fused;
   const int dirs = fwd_only ? 1 : 3;
-  float *Ws = smem, *As = Ws + (size_t)P.R * LW, *bs = As + (size_t)P.R * LW, *Abs = bs + RP, *Xs = Abs + RP,
-        *Ds = Xs + (size_t)P.BM * LX, *Ys = Ds + (size_t)P.BM * RP, *scratch = Ys + (size_t)P.BM * RP, *smem_end = scratch + XWT_SCRATCH;
+  float *Ws = smem, *bs = Ws + (size_t)P.R * LW, *Abs = bs + RP, *Xs = Abs + RP, *Ys = Xs + (size_t)P.BM * LX, *Ds = Ys + (size_t)P.BM * RP,
+        *As = Ds + (fused ? (size_t)P.BM * RP : 0), *Wt = As + (fused ? (size_t)P.R * LW : 0), *Dx = Xs,
+        *smem_end = Wt + (fused ? (size_t)in * RP : 0);      // gradients, accumulators, transposed weights: loss head only; its input
+                                                             // gradients take the place of the staged rows once those are used up
   if (!lookup) {
     for (float* q = smem + tid; q < smem_end; q += FT) *q = 0.f;
     __syncthreads();
     for (int i = tid; i < R * in; i += FT) { const int r = i / in, c = i - r * in; Ws[r * LW + c] = P.W[(size_t)r_begin * in + i]; }
     for (int i = tid; i < R; i += FT) bs[i] = P.b[r_begin + i];
+    if (fused) {
+      __syncthreads();
+      for (int i = tid; i < R * in; i += FT) { const int r = i / in, c = i - r * in; Wt[c * RP + r] = Ws[r * LW + c]; }
+    }
   }
   if (tid == 0) {
-    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0;
+    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0; S.arr_done = 0;
     S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&S.mbar)) : "memory");
     S.mbar_parity = 0;
@@ -620,12 +714,19 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   const bool bulk_ok = !lookup && (P.xcache != nullptr || ((in & 3) == 0 && (C.inst.dense_dim & 3) == 0));
   const int xwidth = P.xcache ? P.xld : in;
 
-  for (;;) {
-    // ---- next batch ----------------------------------------------------------------------------------
+  // Front end of a batch (warps 0-3, 128 threads = one per message): warp 0 takes the batch from the rings, then every
+  // message gets its key, its staging copy is issued and its route resolved.  It runs for batch n + 1 while the other warps
+  // arrive for batch n.
+  unsigned arr_target = 0;          // value of S.arr_done once the arrivals of every batch so far are done
+  auto front = [&](const int pbn, const unsigned done_when) {
     if (warp == 0) {
+      if (lane == 0) S.fpb = pbn;
+      __syncwarp();
       unsigned it = 0;
       for (;;) {
-        const int r = form_batch(C, P, S, leader, fused, dirs, it > 0);
+        const bool arrivals_pending = false;       // the next batch is taken as soon as the arithmetic of this one is done
+        (void)done_when;
+        const int r = form_batch(C, P, S, leader, fused, dirs, it > 0 && !arrivals_pending, 1);
         if (r) break;
         if ((++it & 15u) == 0) {
           unsigned bad = 0;
@@ -635,58 +736,70 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         __nanosleep(it < 16 ? 20 : 100);
       }
     }
-    __syncthreads();
-    if (!S.ok) break;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
     TPHASE(0);
-    const int count = S.count, dir = S.dir, flags = S.flags;
+    if (!S.ok) return;
+    const int count = S.count, dir = S.dir;
+    if (count == 0) return;
+    const unsigned bar = smem_u32(&S.mbar);
+    if (tid == 0 && bulk_ok) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((unsigned)(count * xwidth * 4)) : "memory");
+    if (tid < count) {
+      const Hdr h = S.hdr[pbn][tid];
+      const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      S.key[tid] = key;
+      S.nd[pbn][tid] = 0; S.pre[pbn][tid] = 0;
+      if (key < 0) S.ok = 0;
+      if (key >= 0) {
+        if (!lookup) {
+          const float* x = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+          S.rowptr[tid] = x;
+          if (bulk_ok) {
+            asm volatile("fence.proxy.async;" ::: "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         :: "r"(smem_u32(Xs + (size_t)tid * LX)), "l"(x), "r"((unsigned)(xwidth * 4)), "r"(bar) : "memory");
+          }
+        } else {
+          const int id = C.inst.tokens[C.inst.offsets[h.inst] + h.u];
+          S.rowid[tid] = (unsigned)id < (unsigned)in ? id : -1;
+        }
+        if (leader && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
+        else if (leader && !S.eval && fwd_only) P.vcache[key] = max(S.version, (int)(S.wver_seen / (unsigned)P.TB));   // the version this forward pass uses (Sec. 3: staleness)
+        int pre = 0, nd = 0;
+        if (fused) {                                   // the label, fetched while the input rows are in flight
+          const DevInst& I = C.inst;
+          if (g_nodes[loss_node].type == LOSS_CE) S.rowid[tid] = I.labels_i[I.labels_per_node ? I.offsets[h.inst] + h.u : h.inst];
+          else S.rowid[tid] = __float_as_int(I.labels_f[h.inst]);
+        }
+        if (fused) {                                   // the Loss and this node's own backward arrival, then the way back
+          if (!S.eval) nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][tid], pre);
+          pre += S.eval ? 1 : 2;
+        } else if (dir == FWD) nd = route_message(C, h, N.succ_node[0], N.succ_port[0], FWD, out, S.dl[pbn][tid], pre);
+        else nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][tid], pre);
+        S.nd[pbn][tid] = (unsigned char)nd; S.pre[pbn][tid] = (short)pre;
+      }
+    }
+    __syncwarp();
+    TPHASE(1);
+  };
+
+  int pb = 0;
+  if (warp < 4) front(0, 0u);
+  __syncthreads();
+  for (;;) {
+    if (!S.ok) break;
+    TPHASE(4);
+    const int count = S.count, dir = S.dir, flags = S.flags, eval_n = S.eval, n_upd = S.n_upd, upd_t = S.upd_t;
     if (fwd_only && (int)(S.wver_seen / (unsigned)P.TB) > S.version) {      // every column tile has published a newer version
-      for (int i = tid; i < R * in; i += FT) { const int r = i / in, c = i - r * in; Ws[r * LW + c] = __ldcg(P.W + (size_t)r_begin * in + i); }
+      for (int i = tid; i < R * in; i += FT) { const int r = dIn.div(i), c = i - r * in; Ws[r * LW + c] = __ldcg(P.W + (size_t)r_begin * in + i); }
       for (int i = tid; i < R; i += FT) bs[i] = __ldcg(P.b + r_begin + i);
       __syncthreads();
       if (tid == 0) S.version = (int)(S.wver_seen / (unsigned)P.TB);
-      __syncthreads();
       TPHASE(3);
     }
-    // ---- keys, staging copies, routes ------------------------------------------------------------------
+    // ---- the staged input rows of this batch ---------------------------------------------------------------
     if (count > 0) {
-      const unsigned bar = smem_u32(&S.mbar);
-      if (tid == 0 && bulk_ok) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((unsigned)(count * xwidth * 4)) : "memory");
-      if (tid < count) {
-        const Hdr h = S.hdr[tid];
-        const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
-        S.key[tid] = key;
-        S.nd[tid] = 0; S.pre[tid] = 0;
-        if (key < 0) S.ok = 0;
-        if (key >= 0) {
-          if (!lookup) {
-            const float* x = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
-            S.rowptr[tid] = x;
-            if (bulk_ok) {
-              asm volatile("fence.proxy.async;" ::: "memory");
-              asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                           :: "r"(smem_u32(Xs + (size_t)tid * LX)), "l"(x), "r"((unsigned)(xwidth * 4)), "r"(bar) : "memory");
-            }
-          } else {
-            const int id = C.inst.tokens[C.inst.offsets[h.inst] + h.u];
-            S.rowid[tid] = (unsigned)id < (unsigned)in ? id : -1;
-          }
-          if (leader && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
-          else if (leader && !S.eval && fwd_only) P.vcache[key] = S.version;   // the version this forward pass uses (Sec. 3: staleness)
-          int pre = 0, nd = 0;
-          if (fused) {                                   // the label, fetched while the input rows are in flight
-            const DevInst& I = C.inst;
-            if (g_nodes[loss_node].type == LOSS_CE) S.rowid[tid] = I.labels_i[I.labels_per_node ? I.offsets[h.inst] + h.u : h.inst];
-            else S.rowid[tid] = __float_as_int(I.labels_f[h.inst]);
-          }
-          if (fused) {                                   // the Loss and this node's own backward arrival, then the way back
-            if (!S.eval) nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[tid], pre);
-            pre += S.eval ? 1 : 2;
-          } else if (dir == FWD) nd = route_message(C, h, N.succ_node[0], N.succ_port[0], FWD, out, S.dl[tid], pre);
-          else nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[tid], pre);
-          S.nd[tid] = nd; S.pre[tid] = pre;
-        }
-      }
       if (bulk_ok) {
+        const unsigned bar = smem_u32(&S.mbar);
         const unsigned parity = S.mbar_parity;
         unsigned done = 0, spins = 0;
         for (;;) {
@@ -718,38 +831,81 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         float* y = Ys + tid * RP;
         for (int r = 0; r < R; r++) y[r] = emit_round(act_fwd(P.act, y[r] + bs[r]));
         float* g = Ds + tid * RP;
-        loss_row(C, loss_node, S.hdr[tid], y, g, S.rowid[tid]);
-        if (!S.eval) for (int r = 0; r < R; r++) g[r] *= act_grad(P.act, y[r]);
+        loss_row(C, loss_node, S.hdr[pb][tid], y, g, S.rowid[tid]);
+        if (!eval_n) for (int r = 0; r < R; r++) g[r] *= act_grad(P.act, y[r]);
       }
       __syncthreads();
       TPHASE(6);
-      if (!S.eval) {
-        // the node is one tile with a handful of rows: a thread per element of dx (complete sums, stored into the slot the
-        // gradient lands in) and per accumulator
-        if (!(P.flags & 1)) {
-          for (int idx = tid; idx < count * in; idx += FT) {
-            const int b = dIn.div(idx), i = idx - b * in;
-            float v = 0.f;
-            for (int r = 0; r < R; r++) v = fmaf(Ds[b * RP + r], Ws[r * LW + i], v);
-            v = emit_round(v);
-            for (int q = 0; q < S.nd[b]; q++) {
-              const Deliv& L = S.dl[b][q];
-              if (L.act == ACT_PUSH && L.dst && i >= L.s0 && i < L.s0 + L.w && !(C.tune & 512)) L.dst[i - L.s0] = v;
+      if (!eval_n) {
+        // A[r][k] += sum_b D[b][r] X[b][k]: a thread per (row, four columns) and slice of the batch; the slices meet in A
+        {
+          const int K4 = pad4(in) >> 2, units = R * K4;
+          const int nsl = max(1, min(8, FT / max(units, 1)));
+          for (int u0 = 0; u0 < units; u0 += FT / nsl) {
+            const int u = u0 + tid / nsl, sl = tid % nsl;
+            if (u < units && tid / nsl < FT / nsl) {
+              const int r = u / K4, k4 = u - r * K4;
+              float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 2
+              for (int b = sl; b < count; b += nsl) {
+                const float d = Ds[b * RP + r];
+                const float4 x = *reinterpret_cast<const float4*>(Xs + b * LX + 4 * k4);
+                a0 = fmaf(d, x.x, a0); a1 = fmaf(d, x.y, a1); a2 = fmaf(d, x.z, a2); a3 = fmaf(d, x.w, a3);
+              }
+              float* arow = As + r * LW + 4 * k4;
+              atomicAdd(arow, a0); atomicAdd(arow + 1, a1); atomicAdd(arow + 2, a2); atomicAdd(arow + 3, a3);
             }
           }
         }
-        TPHASE(7);
-        for (int idx = tid; idx < R * in; idx += FT) {
-          const int r = dIn.div(idx), k = idx - r * in;
-          float a = As[r * LW + k];
-#pragma unroll 4
-          for (int b = 0; b < count; b++) a = fmaf(Ds[b * RP + r], Xs[b * LX + k], a);
-          As[r * LW + k] = a;
+        __syncthreads();                                    // the staged rows are used up: dx takes their place
+        TPHASE(15);
+        // dx = D W (complete sums: the node is one tile), stored into the slots it lands in.  With a handful of rows a thread
+        // keeps its column of W in registers and walks a strip of the batch: one 16-byte broadcast of D per four rows, one
+        // coalesced store per message.  Wider heads go through the transposed weights and the staging rows.
+        if (!(P.flags & 1) && R <= 16) {
+          if (tid < count) {                                // the common landing: the whole row to one place
+            const Landing& L = S.dl[pb][tid][0];
+            const bool simple = S.nd[pb][tid] == 1 && L.act == ACT_PUSH && L.dst && L.s0 == 0 && L.w == in;
+            S.rowptr[tid] = simple ? L.dst : nullptr;
+          }
+          __syncthreads();
+          const int nstr = in < FT ? FT / in : 1;
+          for (int ib = 0; ib < in; ib += FT) {
+            const int st = in < FT ? dIn.div(tid) : 0, i = in < FT ? tid - st * in : ib + tid;
+            if (st >= nstr || i >= in) continue;
+            float w[16];
+#pragma unroll
+            for (int r = 0; r < 16; r++) w[r] = r < R ? Ws[r * LW + i] : 0.f;
+            for (int b = st; b < count; b += nstr) {
+              const float4* d4 = reinterpret_cast<const float4*>(Ds + b * RP);
+              float v = 0.f;
+#pragma unroll
+              for (int q = 0; q < 4; q++)
+                if (4 * q < R) {
+                  const float4 d = d4[q];
+                  v = fmaf(d.x, w[4 * q], v); v = fmaf(d.y, w[4 * q + 1], v); v = fmaf(d.z, w[4 * q + 2], v); v = fmaf(d.w, w[4 * q + 3], v);
+                }
+              v = emit_round(v);
+              float* const row = const_cast<float*>(S.rowptr[b]);
+              if (row) row[i] = v;
+              else
+                for (int q = 0; q < S.nd[pb][b]; q++) {
+                  const Landing& L = S.dl[pb][b][q];
+                  if (L.act == ACT_PUSH && L.dst && i >= L.s0 && i < L.s0 + L.w) L.dst[i - L.s0] = v;
+                }
+            }
+          }
+        } else if (!(P.flags & 1)) {
+          gemm_nt(Ds, RP, count, Wt, RP, in, RP >> 2, Dx, DXL);
+          __syncthreads();
+          deliver_cols(S, pb, Dx, DXL, count, 0, in);
         }
-        for (int r = tid; r < R; r += FT) {
-          float a = Abs[r];
-          for (int b = 0; b < count; b++) a += Ds[b * RP + r];
-          Abs[r] = a;
+        TPHASE(7);
+        for (int r = warp; r < R; r += FW) {
+          float a = 0.f;
+          for (int b = lane; b < count; b += 32) a += Ds[b * RP + r];
+          for (int o = 16; o; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+          if (lane == 0) Abs[r] += a;
         }
       }
     } else if (count > 0 && !lookup) {
@@ -761,15 +917,15 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
           const int b = dR.div(idx), r = idx - b * R;
           const float y = emit_round(act_fwd(P.act, Ys[b * RP + r] + bs[r]));
           Ys[b * RP + r] = y;
-          if (!S.eval) P.ycache[S.key[b] * out + r_begin + r] = y;
+          if (!eval_n) P.ycache[S.key[b] * out + r_begin + r] = y;
         }
         __syncthreads();
         TPHASE(6);
         // this tile's slice of every output row, straight into the buffers it lands in
         for (int idx = tid; idx < count * MAXD * R; idx += FT) {
           const int bq = dR.div(idx), r = idx - bq * R, q = bq % MAXD, b = bq / MAXD;
-          if (q >= S.nd[b]) continue;
-          const Deliv& L = S.dl[b][q];
+          if (q >= S.nd[pb][b]) continue;
+          const Landing& L = S.dl[pb][b][q];
           const int c = r_begin + r;
           if (L.act == ACT_PUSH && L.dst && c >= L.s0 && c < L.s0 + L.w) L.dst[c - L.s0] = L.zero ? 0.f : Ys[b * RP + r];
         }
@@ -784,8 +940,8 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         if (!mine) continue;
         constexpr int K = 5;                                // column chunks of 32 in flight per lane
         if (dir == FWD) {
-          for (int q = 0; q < S.nd[b]; q++) {
-            const Deliv& L = S.dl[b][q];
+          for (int q = 0; q < S.nd[pb][b]; q++) {
+            const Landing& L = S.dl[pb][b][q];
             if (L.act != ACT_PUSH || !L.dst) continue;
             for (int cc = 0; cc < L.w; cc += 32 * K) {
               float v[K];
@@ -816,7 +972,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     TPHASE(2);
     // ---- local update (Sec. 3): theta <- theta - lr A / n, accumulator cleared ------------------------------
     if (flags & BATCH_UPDATE) {
-      const OptStep os(C, P, S.n_upd, S.upd_t);
+      const OptStep os(C, P, n_upd, upd_t);
       if (lookup) {
         __threadfence();
         int* const tlist = P.touched_list + (size_t)tile * ((in + P.T - 1) / P.T);
@@ -838,27 +994,34 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         if (tid == 0) P.touched_n[tile] = 0;
       } else {
         const size_t nW = (size_t)out * in;
-        for (int i = tid; i < R * in; i += FT) { const int r = i / in, o = r * LW + (i - r * in); os.apply(Ws[o], As[o], (size_t)r_begin * in + i); }
+        for (int i = tid; i < R * in; i += FT) { const int r = dIn.div(i), o = r * LW + (i - r * in); os.apply(Ws[o], As[o], (size_t)r_begin * in + i); }
         for (int i = tid; i < R; i += FT) os.apply(bs[i], Abs[i], nW + r_begin + i);
+        if (fused) {
+          __syncthreads();
+          for (int i = tid; i < R * in; i += FT) { const int r = dIn.div(i), c = i - r * in; Wt[c * RP + r] = Ws[r * LW + c]; }
+        }
       }
       __syncthreads();
     }
     TPHASE(3);
-    // ---- arrivals: the one that completes a landing publishes the message ------------------------------------
-    if (count > 0) {
-      for (int idx = tid; idx < count * MAXD; idx += FT) {
-        const int b = idx / MAXD, q = idx - b * MAXD;
-        if (q == 0 && leader && S.pre[b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[b]);
-        if (q >= S.nd[b]) continue;
-        const Deliv& L = S.dl[b][q];
-        const Hdr& h = S.hdr[b];
-        arrive(C, h, L, wgt, &S.node_msgs);
-      }
-      if (fused && S.eval && tid < count) retire_arrive(C, S.hdr[tid].slot, JOIN_UNIT);   // a forward-only instance ends at its Losses
-    }
-    __syncthreads();                                          // warp 0 forms the next batch over the headers the arrivals read
-    TPHASE(4);
+    // ---- arrivals of this batch (warps 4-15) while warps 0-3 take the next batch and resolve its routes -------------------
     if (flags & BATCH_TERMINATE) break;
+    if (warp < 4) front(pb ^ 1, arr_target + (unsigned)(FW - 4));
+    else if (count > 0) {
+      for (int idx = tid - 128; idx < count * MAXD; idx += FT - 128) {
+        const int b = idx / MAXD, q = idx - b * MAXD;
+        if (q == 0 && leader && S.pre[pb][b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[pb][b]);
+        if (q == 0 && fused && eval_n) retire_arrive(C, S.hdr[pb][b].slot, JOIN_UNIT);   // a forward-only instance ends at its Losses
+        if (q >= S.nd[pb][b]) continue;
+        const Hdr& h = S.hdr[pb][b];
+        arrive(C, h.inst, h.seq, h.slot, h.flags, S.dl[pb][b][q], wgt, &S.node_msgs);
+      }
+    }
+    if (warp >= 4) { __syncwarp(); if (lane == 0) atomicAdd(&S.arr_done, 1u); }
+    __syncthreads();
+    TPHASE(4);
+    arr_target += FW - 4;
+    pb ^= 1;
   }
   // ---- epilogue: parameters back to device memory, statistics ----------------------------------------------
   __syncthreads();
@@ -887,7 +1050,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
 // cached input x.  Its columns of the input gradient dx = W^T dpre are complete sums: they are stored, not added, into
 // the slot they land in.  A[:, cols] += dpre x[cols]^T.  After the update (Sec. 3) the tile writes its columns to the
 // parameter array in device memory and counts itself in the node's version counter; the forward row tiles reload.
-constexpr int MAXU = 4;                 // accumulator units (one output row x four columns) per thread
+constexpr int MAXU = 1;                 // accumulator units (four output rows x four columns) per thread
 
 __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileS& S, const unsigned long long t0) {
   IN_SMEM(&P); IN_SMEM(smem); IN_SMEM(&S);
@@ -904,16 +1067,17 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
   __syncthreads();
   for (int i = tid; i < out * CB; i += FT) { const int r = i / CB, c = i - r * CB; if (c0 + c < in) Wt[c * WL + r] = P.W[(size_t)r * in + c0 + c]; }
   if (leader) for (int i = tid; i < out; i += FT) bsv[i] = P.b[i];
-  float A[MAXU][4];
+  float A[4][4];                          // this thread's accumulators: rows 4 r4 .. 4 r4 + 3, columns 4 c4 .. 4 c4 + 3 of the tile
 #pragma unroll
-  for (int k = 0; k < MAXU; k++)
+  for (int k = 0; k < 4; k++)
 #pragma unroll
     for (int j = 0; j < 4; j++) A[k][j] = 0.f;
-  const int n_units = out * c4n;
+  const int n_units = ((out + 3) >> 2) * c4n;
+  const int ur4 = tid >> (31 - __clz(c4n)), uc4 = tid & (c4n - 1);
   const FastDiv dOut(out);
-  const int cb_shift = 31 - __clz(CB), c4_shift = cb_shift - 2;
+  const int cb_shift = 31 - __clz(CB);
   if (tid == 0) {
-    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0;
+    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0; S.arr_done = 0;
     S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
   }
   if (tid < 64) S.stale_hist[tid] = 0;
@@ -921,11 +1085,18 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
   __syncthreads();
   long long tph = clock64();
 
-  for (;;) {
+  // Front end of a batch (warps 0-3): warp 0 takes the batch from the backward ring, then every message gets its key and
+  // its route.  It runs for batch n + 1 while the other warps arrive for batch n.
+  unsigned arr_target = 0;          // value of S.arr_done once the arrivals of every batch so far are done
+  auto front = [&](const int pbn, const unsigned done_when) {
     if (warp == 0) {
+      if (lane == 0) S.fpb = pbn;
+      __syncwarp();
       unsigned it = 0;
       for (;;) {
-        const int r = form_batch(C, P, S, leader, false, 2, it > 0);
+        const bool arrivals_pending = false;       // the next batch is taken as soon as the arithmetic of this one is done
+        (void)done_when;
+        const int r = form_batch(C, P, S, leader, false, 2, it > 0 && !arrivals_pending, 1);
         if (r) break;
         if ((++it & 15u) == 0) {
           unsigned bad = 0;
@@ -935,32 +1106,40 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
         __nanosleep(it < 16 ? 20 : 100);
       }
     }
-    __syncthreads();
-    if (!S.ok) break;
+    asm volatile("bar.sync 1, 128;" ::: "memory");
     TPHASE(0);
+    if (!S.ok) return;
     const int count = S.count, flags = S.flags;
-    if (count > 0) {
-      // ---- keys, routes ------------------------------------------------------------------------------------
-      if (tid < count) {
-        const Hdr h = S.hdr[tid];
-        const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
-        S.key[tid] = key; S.nd[tid] = 0; S.pre[tid] = 0;
-        if (key < 0) S.ok = 0;
-        else {
-          S.rowptr[tid] = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
-          if (leader) {                                  // staleness: updates of this node between forward and backward (Sec. 3)
-            int st = S.version - ((flags & BATCH_UPDATE) ? 1 : 0) - P.vcache[key];
-            if (st < 0) st = 0;
-            atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
-            atomicMax(&S.max_stale, st);
-          }
-          int pre = 0;
-          S.nd[tid] = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[tid], pre);
-          S.pre[tid] = pre;
+    if (tid < count) {
+      const Hdr h = S.hdr[pbn][tid];
+      const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      S.key[tid] = key; S.nd[pbn][tid] = 0; S.pre[pbn][tid] = 0;
+      if (key < 0) S.ok = 0;
+      else {
+        S.rowptr[tid] = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+        if (leader) {                                  // staleness: updates of this node between forward and backward (Sec. 3)
+          int st = S.version - ((flags & BATCH_UPDATE) ? 1 : 0) - P.vcache[key];
+          if (st < 0) st = 0;
+          atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
+          atomicMax(&S.max_stale, st);
         }
+        int pre = 0;
+        S.nd[pbn][tid] = (unsigned char)route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][tid], pre);
+        S.pre[pbn][tid] = (short)pre;
       }
-      __syncthreads();
-      if (!S.ok) break;
+    }
+    __syncwarp();
+    TPHASE(1);
+  };
+
+  int pb = 0;
+  if (warp < 4) front(0, 0u);
+  __syncthreads();
+  for (;;) {
+    if (!S.ok) break;
+    TPHASE(6);
+    const int count = S.count, flags = S.flags, n_upd = S.n_upd, upd_t = S.upd_t;
+    if (count > 0) {
       TPHASE(1);
       // ---- operands: dpre for all rows, this tile's columns of x -------------------------------------------------
       {
@@ -1006,72 +1185,66 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
       if (!(P.flags & 1)) {
         gemm_nt(G, GL, count, Wt, WL, CB, pad4(out) >> 2, Dx, CB);
         __syncthreads();
-        for (int idx = tid; idx < count * CB; idx += FT) {
-          const int b = idx >> cb_shift, i = c0 + (idx & (CB - 1));
-          if (i >= in) continue;
-          const float v = emit_round(Dx[idx]);
-          for (int q = 0; q < S.nd[b]; q++) {
-            const Deliv& L = S.dl[b][q];
-            if (L.act == ACT_PUSH && L.dst && i >= L.s0 && i < L.s0 + L.w) L.dst[i - L.s0] = v;
-          }
-        }
+        deliver_cols(S, pb, Dx, CB, count, c0, min(CB, in - c0));
       }
       TPHASE(3);
       // ---- A[r][cols] += sum_b dpre[b][r] x[b][cols]: accumulators in registers --------------------------------------
-#pragma unroll
-      for (int k = 0; k < MAXU; k++) {
-        const int u = tid + k * FT;
-        if (u < n_units) {
-          const int r = u >> c4_shift, c4 = u - (r << c4_shift);
+      if (tid < n_units) {
 #pragma unroll 2
-          for (int b = 0; b < count; b++) {
-            const float g = G[b * GL + r];
-            const float4 x = *reinterpret_cast<const float4*>(Xc + b * CB + 4 * c4);
-            A[k][0] = fmaf(g, x.x, A[k][0]); A[k][1] = fmaf(g, x.y, A[k][1]); A[k][2] = fmaf(g, x.z, A[k][2]); A[k][3] = fmaf(g, x.w, A[k][3]);
-          }
+        for (int b = 0; b < count; b++) {
+          const float4 g = *reinterpret_cast<const float4*>(G + b * GL + 4 * ur4);      // columns beyond `out` are zero
+          const float4 x = *reinterpret_cast<const float4*>(Xc + b * CB + 4 * uc4);
+          A[0][0] = fmaf(g.x, x.x, A[0][0]); A[0][1] = fmaf(g.x, x.y, A[0][1]); A[0][2] = fmaf(g.x, x.z, A[0][2]); A[0][3] = fmaf(g.x, x.w, A[0][3]);
+          A[1][0] = fmaf(g.y, x.x, A[1][0]); A[1][1] = fmaf(g.y, x.y, A[1][1]); A[1][2] = fmaf(g.y, x.z, A[1][2]); A[1][3] = fmaf(g.y, x.w, A[1][3]);
+          A[2][0] = fmaf(g.z, x.x, A[2][0]); A[2][1] = fmaf(g.z, x.y, A[2][1]); A[2][2] = fmaf(g.z, x.z, A[2][2]); A[2][3] = fmaf(g.z, x.w, A[2][3]);
+          A[3][0] = fmaf(g.w, x.x, A[3][0]); A[3][1] = fmaf(g.w, x.y, A[3][1]); A[3][2] = fmaf(g.w, x.z, A[3][2]); A[3][3] = fmaf(g.w, x.w, A[3][3]);
         }
       }
-      if (leader) for (int r = tid; r < out; r += FT) { float a = Abs[r]; for (int b = 0; b < count; b++) a += G[b * GL + r]; Abs[r] = a; }
+      if (leader) for (int r = tid; r < out; r += FT) { float a = Abs[r];
+#pragma unroll 4
+        for (int b = 0; b < count; b++) a += G[b * GL + r]; Abs[r] = a; }
       TPHASE(4);
     }
     // ---- local update (Sec. 3), then the columns go to device memory for the forward tiles ---------------------------
     if (flags & BATCH_UPDATE) {
-      const OptStep os(C, P, S.n_upd, S.upd_t);
+      const OptStep os(C, P, n_upd, upd_t);
+      if (tid < n_units) {
 #pragma unroll
-      for (int k = 0; k < MAXU; k++) {
-        const int u = tid + k * FT;
-        if (u < n_units) {
-          const int r = u >> c4_shift, c4 = u - (r << c4_shift);
+        for (int k = 0; k < 4; k++)
 #pragma unroll
           for (int j = 0; j < 4; j++) {
-            const int c = c0 + 4 * c4 + j;
-            if (c < in) {
-              float w = Wt[(4 * c4 + j) * WL + r];
+            const int r = 4 * ur4 + k, c = c0 + 4 * uc4 + j;
+            if (r < out && c < in) {
+              float w = Wt[(4 * uc4 + j) * WL + r];
               os.apply(w, A[k][j], (size_t)r * in + c);
-              Wt[(4 * c4 + j) * WL + r] = w;
+              Wt[(4 * uc4 + j) * WL + r] = w;
               P.W[(size_t)r * in + c] = w;
             } else A[k][j] = 0.f;
           }
-        }
       }
       if (leader) for (int r = tid; r < out; r += FT) { os.apply(bsv[r], Abs[r], (size_t)out * in + r); P.b[r] = bsv[r]; }
       __syncthreads();
       if (tid == 0) { __threadfence(); atomicAdd(P.wver, 1u); }
       TPHASE(5);
     }
-    // ---- arrivals ------------------------------------------------------------------------------------------------
-    if (count > 0) {
-      __syncthreads();
-      for (int idx = tid; idx < count * MAXD; idx += FT) {
+    // ---- arrivals of this batch (warps 4-15) while warps 0-3 take the next batch and resolve its routes -------------------
+    __syncthreads();
+    if (flags & BATCH_TERMINATE) break;
+    if (warp < 4) front(pb ^ 1, arr_target + (unsigned)(FW - 4));
+    else if (count > 0) {
+      for (int idx = tid - 128; idx < count * MAXD; idx += FT - 128) {
         const int b = idx / MAXD, q = idx - b * MAXD;
-        if (q == 0 && leader && S.pre[b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[b]);
-        if (q >= S.nd[b]) continue;
-        arrive(C, S.hdr[b], S.dl[b][q], wgt, &S.node_msgs);
+        if (q == 0 && leader && S.pre[pb][b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[pb][b]);
+        if (q >= S.nd[pb][b]) continue;
+        const Hdr& h = S.hdr[pb][b];
+        arrive(C, h.inst, h.seq, h.slot, h.flags, S.dl[pb][b][q], wgt, &S.node_msgs);
       }
     }
+    if (warp >= 4) { __syncwarp(); if (lane == 0) atomicAdd(&S.arr_done, 1u); }
     __syncthreads();
     TPHASE(6);
-    if (flags & BATCH_TERMINATE) break;
+    arr_target += FW - 4;
+    pb ^= 1;
   }
   __syncthreads();
   if (tid == 0 && S.node_msgs) atomicAdd(&C.g->node_messages, S.node_msgs);
@@ -1099,7 +1272,7 @@ struct CtrlS {
   int src_count[4];
   unsigned long long node_msgs;
   unsigned occ[OCC_SLOTS / 32];
-  Deliv dl[MAXD];
+  Landing dl[MAXD];
 };
 
 // A source whose messages carry no payload of their own and feed a parameterised node directly (token ids, leaf ids,
@@ -1236,13 +1409,13 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
           nd = (int)warp_uniform((unsigned)nd);
           __syncwarp();
           for (int q = 0; q < nd; q++) {
-            const Deliv& L = S.dl[q];
+            const Landing& L = S.dl[q];
             if (L.act == ACT_PUSH && L.dst) for (int c = lane; c < L.w; c += 32) L.dst[c] = 0.f;
           }
           __syncwarp();
           if (lane == 0) {
             if (pre) atomicAdd(&S.node_msgs, (unsigned long long)pre);
-            for (int q = 0; q < nd; q++) arrive(C, h, S.dl[q], JOIN_UNIT, &S.node_msgs);
+            for (int q = 0; q < nd; q++) arrive(C, h.inst, h.seq, h.slot, h.flags, S.dl[q], JOIN_UNIT, &S.node_msgs);
           }
           __syncwarp();
         }
@@ -1299,9 +1472,10 @@ __global__ void __launch_bounds__(ampf::FT, 1) ampnet_engine_direct(const __grid
 // host side: what the launch needs to know
 // ------------------------------------------------------------------------------------------------
 namespace ampf {
-size_t tile_smem_floats(int in, int R, int BM) {
-  const size_t LW = pad_ldx(in), LX = pad_ldx(in), RP = pad4(R > 0 ? R : 1);
-  return 2 * (size_t)R * LW + 2 * RP + (size_t)BM * LX + 2 * (size_t)BM * RP + XWT_SCRATCH;
+size_t tile_smem_floats(int in, int R, int BM, int loss_head) {
+  const size_t LW = pad_ldx(in), LX = pad_ldx(in), RP = pad_ldx(R > 0 ? R : 1);
+  return (size_t)R * LW + 2 * RP + (size_t)BM * LX + (size_t)BM * RP +
+         (loss_head ? (size_t)BM * RP + (size_t)R * LW + (size_t)in * RP : 0);
 }
 }  // namespace ampf
 
@@ -1309,9 +1483,14 @@ namespace ampf {
 size_t bwd_tile_smem_floats(int out, int cb, int BM) { const size_t GL = pad_ldx(out); return (size_t)cb * GL + (size_t)BM * GL + 2 * (size_t)BM * cb + 2 * GL; }
 }  // namespace ampf
 extern "C" size_t ampnet_direct_bwd_tile_smem_bytes(int out_dim, int cols, int batch_rows) { return ampf::bwd_tile_smem_floats(out_dim, cols, batch_rows) * sizeof(float) + 64; }
-extern "C" int ampnet_direct_max_units() { return ampf::MAXU * ampf::FT; }
+extern "C" int ampnet_direct_max_units() { return 4 * ampf::FT; }    // out_dim x (columns / 4) of a backward tile may not exceed this
 extern "C" int ampnet_direct_threads() { return ampf::FT; }
-extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows) { return ampf::tile_smem_floats(in_dim, rows, batch_rows) * sizeof(float) + 64; }
+extern "C" void ampnet_direct_limits(int* max_nodes, int* max_ppts, int* max_landings, int* batch_rows) {
+  *max_nodes = ampf::DIRECT_MAX_NODES; *max_ppts = ampf::DIRECT_MAX_PPTS; *max_landings = ampf::MAXD; *batch_rows = ampf::FBM;
+}
+extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows, int loss_head) {
+  return ampf::tile_smem_floats(in_dim, rows, batch_rows, loss_head) * sizeof(float) + 64;
+}
 extern "C" cudaError_t ampnet_direct_static_smem(size_t* bytes) {
   cudaFuncAttributes fa{};
   const cudaError_t e = cudaFuncGetAttributes(&fa, ampnet_engine_direct);

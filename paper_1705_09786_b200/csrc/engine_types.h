@@ -187,6 +187,7 @@ struct Ctx {
   int opt;                            // update rule: 0 SGD, 1 momentum-SGD, 2 Adam
   float mu, beta1, beta2, eps;
   unsigned long long timeout_ns;
+  char* ctl_base;                     // start of the control arena (counters are addressed by 32-bit offsets from here)
 };
 
 }  // namespace amp
