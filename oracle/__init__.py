@@ -2,4 +2,4 @@
 
 `Oracle` is a ctypes wrapper around ampnet_oracle.cpp; `build()` compiles it with g++.
 """
-from .oracle import Oracle, build, OracleStats  # noqa: F401
+from .oracle import Oracle, build, OracleStats, round_bf16  # noqa: F401

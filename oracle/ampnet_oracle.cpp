@@ -1262,4 +1262,9 @@ int64_t oracle_get_key_log(void* h, int64_t* inst, int32_t* slot, int64_t* admit
   return n;
 }
 
+// The bf16 rounding applied to emitted payloads, exposed so that a test can pin it against an independent conversion.
+void oracle_round_bf16(const double* in, double* out, int64_t n) {
+  for (int64_t i = 0; i < n; i++) out[i] = (double)round_bf16((real)in[i]);
+}
+
 }  // extern "C"

@@ -56,6 +56,7 @@ def _load(real):
                                            C.POINTER(OracleStats), P, P]
     lib.oracle_set_optimizer.argtypes = [P, C.c_int, C.c_double, C.c_double, C.c_double, C.c_double, C.c_int]
     lib.oracle_get_node_stats.argtypes = [P, C.c_int, P, P, P, P, P]
+    lib.oracle_round_bf16.argtypes = [P, P, C.c_int64]
     lib.oracle_get_update_log.restype = C.c_int64
     lib.oracle_get_update_log.argtypes = [P, C.c_int, P, C.c_int64]
     lib.oracle_get_key_log.restype = C.c_int64
@@ -66,6 +67,14 @@ def _load(real):
 
 def _p(a):
     return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def round_bf16(values, real="f64"):
+    """The oracle's payload rounding (to bfloat16, nearest even) applied to an array of float32-representable values."""
+    a = np.ascontiguousarray(values, dtype=np.float64)
+    out = np.empty_like(a)
+    _load(real).oracle_round_bf16(_p(a), _p(out), a.size)
+    return out
 
 
 class Oracle:

@@ -158,3 +158,46 @@ def tiny_case(family, n=3, seed=0):
         if p[k].ndim == 1:
             p[k] = rng.uniform(-0.3, 0.3, size=p[k].shape)
     return g, inst, p
+
+
+# ---- predictions of the independent forward passes (for the accuracy the oracle reports) -----------------------
+def _logit_rows(g, P, inst, i):
+    """Every (logits, label) pair the model's classification loss sees for instance i, by direct recursion."""
+    name = g.name
+    if name == "mlp":
+        x = torch.tensor(inst.dense[i], dtype=torch.float64)
+        for n in g.ppt_nodes():
+            x = act(int(g.nodes[n][3]), P[(n, 0)] @ x + P[(n, 1)])
+        return [(x, int(inst.labels_i[i]))]
+    if name == "rnn":
+        look, l1, l2 = g.index("lookup"), g.index("linear1"), g.index("linear2")
+        h = torch.zeros(P[(l1, 0)].shape[0], dtype=torch.float64)
+        for t in inst.tokens[inst.offsets[i]:inst.offsets[i + 1]]:
+            h = act(int(g.nodes[l1][3]), P[(l1, 0)] @ torch.cat([P[(look, 0)][int(t)], h]) + P[(l1, 1)])
+        return [(P[(l2, 0)] @ h + P[(l2, 1)], int(inst.labels_i[i]))]
+    assert name == "tree"
+    look, leaf, br, cls = (g.index(k) for k in ("lookup", "leaf_cell", "branch_cell", "classifier"))
+    o = int(inst.offsets[i])
+    rows = []
+
+    def rec(u):
+        if inst.left[o + u] < 0:
+            h = torch.tanh(P[(leaf, 0)] @ P[(look, 0)][int(inst.tokens[o + u])] + P[(leaf, 1)])
+        else:
+            h = torch.tanh(P[(br, 0)] @ torch.cat([rec(int(inst.left[o + u])), rec(int(inst.right[o + u]))]) + P[(br, 1)])
+        rows.append((P[(cls, 0)] @ h + P[(cls, 1)], int(inst.labels_i[o + u])))
+        return h
+
+    rec(int(inst.offsets[i + 1]) - o - 1)
+    return rows
+
+
+def accuracy(g, params, inst):
+    """Fraction of classification decisions (arg-max, lowest index on ties) that hit the label, over the dataset."""
+    P = {k: torch.tensor(v, dtype=torch.float64) for k, v in params.items()}
+    hit = n = 0
+    for i in range(inst.n):
+        for logits, label in _logit_rows(g, P, inst, i):
+            hit += int(int(torch.argmax(logits)) == label)
+            n += 1
+    return hit / n

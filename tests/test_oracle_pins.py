@@ -501,3 +501,127 @@ def test_split_gradients_equal_autograd(oracle_mod):
     for k, v in P.items():
         np.testing.assert_allclose(o.get_accum(*k), v.grad.numpy(), rtol=1e-9, atol=1e-12)
     assert st.leftover_cache_entries == 0
+
+
+# ---------------------------------------------------------------------------------------------------
+# bf16 payload rounding, reported accuracy, sparse-row optimiser state of the embedding table
+# ---------------------------------------------------------------------------------------------------
+def test_bf16_rounding_is_round_to_nearest_even(oracle_mod):
+    """The oracle's payload rounding against torch's float32 -> bfloat16 conversion: random values of every magnitude,
+    exact ties with an even and with an odd kept mantissa (truncation, round-half-up and round-half-away all fail
+    here), values just off a tie, subnormals, signed zeros, infinities and NaN."""
+    import torch
+    rng = np.random.default_rng(7)
+    bits = rng.integers(0, 1 << 32, size=200000, dtype=np.uint64).astype(np.uint32)
+    rand = bits.view(np.float32)
+    rand = rand[np.isfinite(rand)]
+    hi = rng.integers(0, 1 << 16, size=4096, dtype=np.uint32) << 16
+    hi = hi[((hi >> 23) & 0xff) != 0xff]
+    ties = (hi | 0x8000).view(np.float32)                        # exactly half way between two bfloat16 neighbours
+    above, below = (hi | 0x8001).view(np.float32), (hi | 0x7fff).view(np.float32)
+    special = np.array([0.0, -0.0, np.inf, -np.inf, 1e-40, -1e-40, 1.17549435e-38, 3.3895314e38, -3.3895314e38, 1.0,
+                        1.00390625, 1.01171875], np.float32)     # the last two: ties at 1 + 2^-8 (down) and 1 + 3 2^-8 (up)
+    x = np.concatenate([rand, ties, above, below, special])
+    want = torch.from_numpy(x.copy()).to(torch.bfloat16).to(torch.float32).numpy()
+    got = oracle_mod.round_bf16(x).astype(np.float32)
+    np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert np.isnan(oracle_mod.round_bf16(np.array([np.nan], np.float32))[0])
+    # the two textbook ties, by value: 1 + 2^-8 -> 1 (even below), 1 + 3 2^-8 -> 1 + 2^-6 (even above)
+    np.testing.assert_array_equal(oracle_mod.round_bf16(np.array([1.00390625, 1.01171875])), [1.0, 1.015625])
+
+
+@pytest.mark.parametrize("family", ["mlp", "rnn", "tree"])
+def test_reported_accuracy_is_the_argmax_of_an_independent_forward_pass(oracle_mod, family):
+    """eval()'s accuracy (and its count of predictions) against the arg-max of the direct recursive forward pass."""
+    g, inst, p = H.tiny_case(family, n=40 if family != "tree" else 12, seed=4)
+    o = make(oracle_mod, g, inst, p)
+    _, acc, _ = o.eval()
+    want = H.accuracy(g, p, inst)
+    assert 0.0 < want < 1.0                      # the case decides something: neither all right nor all wrong
+    assert acc == pytest.approx(want, abs=1e-12)
+    # a different parameter set moves both numbers together
+    p2 = {k: v * (-1.0 if len(v.shape) == 1 else 1.0) + 0.1 for k, v in p.items()}
+    o.set_params(p2)
+    assert o.eval()[1] == pytest.approx(H.accuracy(g, p2, inst), abs=1e-12)
+
+
+def _sparse_rows_reference(kind, E, grads_and_rows, lr, beta=(0.9, 0.999), eps=1e-8, mu=0.9):
+    """Momentum-SGD / Adam on an embedding table in which an update moves only the rows that received a gradient since
+    the previous update, and only their moments (plain numpy, written from the textbook update rules)."""
+    E = E.copy()
+    m, v = np.zeros_like(E), np.zeros_like(E)
+    f32 = lambda x: float(np.float32(x))
+    b1, b2, eps, mu = f32(beta[0]), f32(beta[1]), f32(eps), f32(mu)
+    for t, (g, rows) in enumerate(grads_and_rows, start=1):
+        for r in rows:
+            if kind == "momentum":
+                m[r] = mu * m[r] + g[r]
+                E[r] -= lr * m[r]
+            else:
+                m[r] = b1 * m[r] + (1 - b1) * g[r]
+                v[r] = b2 * v[r] + (1 - b2) * g[r] * g[r]
+                E[r] -= lr * (m[r] / (1 - b1 ** t)) / (np.sqrt(v[r] / (1 - b2 ** t)) + eps)
+    return E
+
+
+@pytest.mark.parametrize("kind", ["momentum", "adam"])
+def test_embedding_rows_move_only_when_touched_under_momentum_and_adam(oracle_mod, kind):
+    """Two updates of the list model's embedding table (one per epoch: the threshold is never reached, the flush at the
+    end of the epoch applies the mean gradient).  (1) When every table row is touched before each update the result is
+    torch.optim's dense optimiser.  (2) When the second epoch's lists leave rows untouched, those rows and their moments
+    stay as they were (no decay), which differs from the dense optimiser and equals a few lines of numpy."""
+    import torch
+    g = ir.rnn(vocab=14, emb=5, hidden=5, classes=10)
+    look = g.index("lookup")
+    p = wp.init_params(g, seed=3, emb_std=0.5)
+    lr = float(np.float32(0.05))
+    full = data.list_instances(n=60, max_len=6)                  # touches all 14 rows (digits 0-9 and the four ops)
+    toks = full.tokens
+    assert len(np.unique(toks)) == 14
+
+    def epoch_grad(params, inst):
+        grads, _ = H.dataset_grad(g, params, inst)
+        n_tok = len(inst.tokens)                                 # one gradient per token reaches the table
+        return grads[(look, 0)] / n_tok
+
+    # (1) dense coincidence: both epochs on the full set
+    o = make(oracle_mod, g, full, p)
+    o.set_optimizer(kind)
+    E = torch.tensor(p[(look, 0)], dtype=torch.float64, requires_grad=True)
+    f32 = lambda x: float(np.float32(x))
+    opt = torch.optim.SGD([E], lr=lr, momentum=f32(0.9)) if kind == "momentum" else \
+        torch.optim.Adam([E], lr=lr, betas=(f32(0.9), f32(0.999)), eps=f32(1e-8))
+    for _ in range(2):
+        cur = o.get_params()
+        opt.zero_grad()
+        E.grad = torch.tensor(epoch_grad(cur, full))
+        o.run_epoch(mak=1, muf=BIG, lr=lr)
+        opt.step()
+        np.testing.assert_allclose(o.get_params(look, 0), E.detach().numpy(), rtol=1e-9, atol=1e-12)
+
+    # (2) the second epoch touches only some rows
+    keep = [i for i in range(full.n) if set(toks[full.offsets[i]:full.offsets[i + 1]]) <= {0, 1, 2, 3, 10, 11}]
+    assert len(keep) >= 1
+    part = full.subset(np.array(keep))
+    rows2 = sorted(set(part.tokens.tolist()))
+    assert 0 < len(rows2) < 14
+    o = make(oracle_mod, g, full, p)
+    o.set_optimizer(kind)
+    g1 = epoch_grad(o.get_params(), full)
+    o.run_epoch(mak=1, muf=BIG, lr=lr)
+    o.load_instances(part)
+    g2 = epoch_grad(o.get_params(), part)
+    o.run_epoch(mak=1, muf=BIG, lr=lr)
+    want = _sparse_rows_reference(kind, p[(look, 0)], [(g1, range(14)), (g2, rows2)], lr)
+    got = o.get_params(look, 0)
+    np.testing.assert_allclose(got, want, rtol=1e-9, atol=1e-12)
+    untouched = [r for r in range(14) if r not in rows2]
+    after_first = _sparse_rows_reference(kind, p[(look, 0)], [(g1, range(14))], lr)
+    np.testing.assert_allclose(got[untouched], after_first[untouched], rtol=1e-12, atol=0)
+    # ... and a dense optimiser would have moved them (momentum / first moment carry over): the two readings differ here
+    dense = torch.tensor(p[(look, 0)], dtype=torch.float64, requires_grad=True)
+    dopt = torch.optim.SGD([dense], lr=lr, momentum=f32(0.9)) if kind == "momentum" else \
+        torch.optim.Adam([dense], lr=lr, betas=(f32(0.9), f32(0.999)), eps=f32(1e-8))
+    for gg in (g1, g2):
+        dopt.zero_grad(); dense.grad = torch.tensor(gg); dopt.step()
+    assert np.abs(dense.detach().numpy()[untouched] - got[untouched]).max() > 1e-6
