@@ -603,6 +603,11 @@ bool direct_candidate(ampnet_graph* g, const HostDataset& D, int det) {
 // 4, 8, 16 or 32), more per tile where the CTA budget, shared memory or the register-resident accumulators ask for it.
 // A node that feeds a Loss is one tile for both directions (the Loss needs the whole output row); a large embedding
 // table is dealt to four tiles by row id.
+static ampnet_status_t direct_overflow(int where) {
+  if (getenv("AMPNET_DEBUG")) fprintf(stderr, "[ampnet] direct-delivery placement does not fit (check %d): interpreter engine\n", where);
+  return AMPNET_EOVERFLOW;
+}
+
 ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& roles) {
   size_t static_smem = 48 * 1024;
   ampnet_direct_static_smem(&static_smem);
@@ -642,7 +647,7 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
       P.R = std::min(P.out, rows);
       P.CB = cols;
       while (P.CB > 4 && (long long)P.out * (P.CB / 4) > max_units) P.CB /= 2;
-      if ((long long)P.out * (P.CB / 4) > max_units) return AMPNET_EOVERFLOW;        // accumulators of a column tile exceed the registers
+      if ((long long)P.out * (P.CB / 4) > max_units) return direct_overflow(1);        // accumulators of a column tile exceed the registers
     }
   }
   auto fits = [&](const HostPPT& P) {
@@ -654,25 +659,30 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
     while (!fits(P)) {
       if (P.BM > 16) P.BM /= 2;
       else if (!fixed[p] && P.R > 1) { P.R = (P.R + 1) / 2; P.BM = BATCH; }
-      else return AMPNET_EOVERFLOW;
+      else return direct_overflow(2);
     }
   }
+  // over the budget: grow the tiles of whichever node has the most tiles of a kind that can still grow (rows per forward
+  // tile while its weights and a few staged rows still fit; columns per backward tile while the accumulators fit the registers)
+  std::vector<char> rows_stuck(np, 0);
   for (;;) {
-    int used = 0, worst = -1, worst_n = 0;
+    int used = 0, best = -1, best_n = 0; bool best_cols = false;
     for (int p = 0; p < np; p++) {
       HostPPT& P = g->ppts[p];
       if (P.kind != LOOKUP) { P.T = (P.out + P.R - 1) / P.R; P.TB = P.CB ? (P.in + P.CB - 1) / P.CB : 0; }
       used += P.T + P.TB;
-      if (!fixed[p] && std::max(P.T, P.TB) > worst_n && (P.R < P.out || P.CB < 32)) { worst = p; worst_n = std::max(P.T, P.TB); }
+      if (fixed[p]) continue;
+      if (!rows_stuck[p] && P.R < P.out && P.T > best_n) { best = p; best_n = P.T; best_cols = false; }
+      if (P.CB && P.CB < 32 && (long long)P.out * (P.CB * 2 / 4) <= max_units && P.TB > best_n) { best = p; best_n = P.TB; best_cols = true; }
     }
     if (used <= tile_budget) break;
-    if (worst < 0) return AMPNET_EOVERFLOW;
-    HostPPT& P = g->ppts[worst];
-    if (P.TB >= P.T && P.CB < 32 && (long long)P.out * (P.CB * 2 / 4) <= max_units) P.CB *= 2;
-    else if (P.R < P.out) P.R++;
-    else return AMPNET_EOVERFLOW;
-    while (!fits(P) && P.BM > 16) P.BM /= 2;
-    if (!fits(P)) return AMPNET_EOVERFLOW;
+    if (best < 0) return direct_overflow(4);
+    HostPPT& P = g->ppts[best];
+    if (best_cols) { P.CB *= 2; while (!fits(P) && P.BM > 8) P.BM /= 2; if (!fits(P)) return direct_overflow(5); continue; }
+    const int r0 = P.R, bm0 = P.BM;
+    P.R++;
+    while (!fits(P) && P.BM > 8) P.BM /= 2;
+    if (!fits(P)) { P.R = r0; P.BM = bm0; rows_stuck[best] = 1; }
   }
   roles.clear();
   roles.push_back(Role{-1, 0, 0, 0});

@@ -358,11 +358,12 @@ struct TileS {
 };
 
 __host__ __device__ __forceinline__ int pad4(int v) { return (v + 3) & ~3; }
-// n / d for 0 <= n < 200000 and 1 <= d <= 2048 by one multiply-high (M = floor((2^32 - 1) / d) + 1; checked exhaustively)
+// n / d for 0 <= n < 200000 and 1 <= d <= 2048 by one multiply-high (M = floor((2^32 - 1) / d) + 1; checked exhaustively
+// for 2 <= d; d = 1 would need M = 2^32 and is handled apart)
 struct FastDiv {
   unsigned d, M;
-  __device__ explicit FastDiv(int d_) : d((unsigned)d_), M(0xFFFFFFFFu / (unsigned)d_ + 1u) {}
-  __device__ __forceinline__ int div(int n) const { return (int)__umulhi((unsigned)n, M); }
+  __device__ explicit FastDiv(int d_) : d((unsigned)d_), M(d_ > 1 ? 0xFFFFFFFFu / (unsigned)d_ + 1u : 0u) {}
+  __device__ __forceinline__ int div(int n) const { return d > 1 ? (int)__umulhi((unsigned)n, M) : n; }
 };
 __host__ __device__ __forceinline__ int pad_ldx(int in) { int l = (in + 3) & ~3; while ((l & 7) != 4) l += 4; return l; }
 // out[b][o] = sum_k A[b][k] B[o][k] for b < nA, o < nB: both operands in shared memory with k contiguous, rows padded
@@ -927,7 +928,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
           if (q >= S.nd[pb][b]) continue;
           const Landing& L = S.dl[pb][b][q];
           const int c = r_begin + r;
-          if (L.act == ACT_PUSH && L.dst && c >= L.s0 && c < L.s0 + L.w) L.dst[c - L.s0] = L.zero ? 0.f : Ys[b * RP + r];
+          if (L.act == ACT_PUSH && L.dst && c >= L.s0 && c < L.s0 + L.w) __stcg(L.dst + (c - L.s0), L.zero ? 0.f : Ys[b * RP + r]);
         }
       }
     } else if (count > 0) {

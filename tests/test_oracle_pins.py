@@ -625,3 +625,40 @@ def test_embedding_rows_move_only_when_touched_under_momentum_and_adam(oracle_mo
     for gg in (g1, g2):
         dopt.zero_grad(); dense.grad = torch.tensor(gg); dopt.step()
     assert np.abs(dense.detach().numpy()[untouched] - got[untouched]).max() > 1e-6
+
+
+# bf16 messages: what any fp32 implementation differs by from the fp64 oracle.  A payload that lies within fp32 rounding
+# of a bf16 boundary rounds the other way (one bf16 ulp, 2^-8 relative), and behind a ReLU threshold that switches a whole
+# gradient row.  The oracle measures this on itself (fp32 build against fp64 build, both with bf16 payloads); the tolerances
+# of the GPU's bf16 parity test are these gaps with head room, not free parameters.
+BF16_TOL = dict(param_rtol=2e-2, loss_rtol=2e-2, loss_atol=2e-3, param_floor=1e-2)
+BF16_CASES = [("tree", 30, 16, 20, 0.02), ("rnn", 60, 8, 10, 0.02), ("ggnn", 20, 16, 40, 0.003), ("mlp", 40, 4, 8, 0.01),
+              ("tree_lstm", 24, 16, 20, 0.02)]
+
+
+def _bf16_case(family, n):
+    gen = {"mlp": (ir.mlp, data.mlp_instances), "rnn": (ir.rnn, data.list_instances), "tree": (ir.tree, data.tree_instances),
+           "ggnn": (ir.ggnn, data.graph_instances), "tree_lstm": (ir.tree_lstm, data.tree_instances)}[family]
+    return gen[0](), gen[1](n=n)
+
+
+def test_bf16_tolerances_come_from_the_oracles_own_fp32_gap(oracle_mod):
+    worst_p = worst_l = 0.0
+    for family, n, mak, muf, lr in BF16_CASES:
+        g, inst = _bf16_case(family, n)
+        p = wp.init_params(g)
+        res = {}
+        for real in ("f64", "f32"):
+            o = oracle_mod.Oracle(g, real=real, payload_bf16=True)
+            o.load_instances(inst)
+            o.set_params(p)
+            _, loss = o.run_epoch(mak=mak, muf=muf, lr=lr)
+            res[real] = (o.get_params(), loss)
+        (pa, la), (pb, lb) = res["f64"], res["f32"]
+        gp = max(np.abs(pa[k] - pb[k].astype(np.float64)).max() / max(np.abs(pa[k]).max(), BF16_TOL["param_floor"]) for k in pa)
+        gl = (np.abs(la - lb) / (np.abs(la) + BF16_TOL["loss_atol"] / BF16_TOL["loss_rtol"])).max()
+        print(f"bf16 gap fp32 vs fp64 oracle, {family}: parameters {gp:.2e}, losses {gl:.2e}")
+        assert gp <= BF16_TOL["param_rtol"] and gl <= BF16_TOL["loss_rtol"], family
+        worst_p, worst_l = max(worst_p, gp), max(worst_l, gl)
+    # head room, not slack: the tolerances stay within an order of magnitude of the largest gap measured
+    assert BF16_TOL["param_rtol"] <= 10 * worst_p and BF16_TOL["loss_rtol"] <= 10 * worst_l
