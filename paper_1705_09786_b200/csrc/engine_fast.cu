@@ -28,7 +28,7 @@ constexpr int FT = 512;               // threads per CTA
 constexpr int FW = FT / 32;
 constexpr int FBM = 128;              // messages (= rows) per micro-batch
 constexpr int MAXD = 2;               // landings per message
-constexpr int RSTACK = 4;             // pending forks per routed message
+constexpr int RSTACK = 2;             // pending forks per routed message (two named slots: an indexed array would live in local memory)
 
 // ------------------------------------------------------------------------------------------------
 // memory-model helpers, bounded waits
@@ -158,8 +158,11 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
                                           Landing* out, int& pre) {
   IN_SMEM(out);
   const DevInst& I = C.inst;
-  const long long ibase = I.offsets ? I.offsets[h.inst] : 0;
-  Route stack[RSTACK];
+  const long long ibase = h.rows;          // every message is one row here: the field carries the instance's first position instead
+  // the tree tables of the message's own position, fetched together (one round trip instead of one per node on the way)
+  int own_parent = 0, own_slot = 0, own_left = 0, own_right = 0;
+  if (I.parent) { const long long o = ibase + h.u; own_parent = I.parent[o]; own_slot = I.child_slot[o]; own_left = I.left[o]; own_right = I.right[o]; }
+  Route stack0, stack1;
   int sp = 0, nout = 0;
   Route f;
   f.node = start_node; f.aport = start_aport; f.dir = dir0; f.u = h.u; f.it = h.it; f.port = h.port; f.s0 = 0; f.w = width; f.null = 0;
@@ -235,7 +238,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
           int k = 0;
           switch (n.fn) {
             case 1: k = f.u < (int)(I.offsets[h.inst + 1] - ibase) ? 0 : 1; break;
-            case 2: k = I.parent[ibase + f.u] < 0 ? 0 : 1; break;
+            case 2: k = (f.u == h.u ? own_parent : I.parent[ibase + f.u]) < 0 ? 0 : 1; break;
             case 3: k = f.u; break;
             case 4: k = f.it < n.fn_arg ? 0 : 1; break;
             case 5: k = (h.inst + f.u) % n.n_succ; break;
@@ -264,12 +267,12 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
         count();
         if (f.dir == FWD) {
           if (n.fn == 1) f.u += 1;
-          else if (n.fn == 2) { f.port = I.child_slot[ibase + f.u]; f.u = I.parent[ibase + f.u]; }
+          else if (n.fn == 2) { const bool own = f.u == h.u; f.port = own ? own_slot : I.child_slot[ibase + f.u]; f.u = own ? own_parent : I.parent[ibase + f.u]; }
           else f.it += 1;
           to_succ(0);
         } else {
           if (n.fn == 1) f.u -= 1;
-          else if (n.fn == 2) { f.u = f.port == 0 ? I.left[ibase + f.u] : I.right[ibase + f.u]; f.port = 0; }
+          else if (n.fn == 2) { const bool own = f.u == h.u; f.u = f.port == 0 ? (own ? own_left : I.left[ibase + f.u]) : (own ? own_right : I.right[ibase + f.u]); f.port = 0; }
           else f.it -= 1;
           to_pred(0);
         }
@@ -280,7 +283,8 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
           for (int k = n.fn_arg - 1; k >= 1; k--) {
             if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; }
             Route c = f; c.node = n.succ_node[k]; c.aport = n.succ_port[k]; c.dir = FWD;
-            stack[sp++] = c;
+            if (sp == 0) stack0 = c; else stack1 = c;
+            sp++;
           }
           to_succ(0);
         } else {
@@ -314,7 +318,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
             if (n.fn == 2) { c.port = k; c.node = n.pred_node[0]; c.aport = n.pred_port[0]; }
             else { c.node = n.pred_node[k]; c.aport = n.pred_port[k]; }
             if (k == 0) { f = c; cont = true; }
-            else { if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; } stack[sp++] = c; }
+            else { if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; } if (sp == 0) stack0 = c; else stack1 = c; sp++; }
           }
         }
         break;
@@ -324,7 +328,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
     }
     if (!cont) {
       if (pend) { fail(C, ST_OVERFLOW, f.node, -13); return nout; }          // a sum that found no landing
-      if (sp > 0) f = stack[--sp];
+      if (sp > 0) { sp--; f = sp == 0 ? stack0 : stack1; }
       else have = false;
     }
   }
@@ -486,7 +490,7 @@ __device__ __noinline__ void ring_push(Ring& r, const Hdr& h, int it, int u, int
   const unsigned t = atomicAdd(r.tail, 1u), s = t & r.mask;
   int4* d = reinterpret_cast<int4*>(&r.e[s]);
   d[0] = make_int4(h.inst, h.seq, h.slot, it);
-  d[1] = make_int4(u, port, 1, h.flags);
+  d[1] = make_int4(u, port, h.rows, h.flags);
   st_rel(&r.seq[s], t + 1u);
 }
 // The instance in key slot `slot` loses `wgt` of its outstanding source messages (JOIN_UNIT each); the arrival that
@@ -500,11 +504,11 @@ __device__ __noinline__ void retire_arrive(const Ctx& C, int slot, int wgt) {
   st_rel(&C.retire_seq[s], t + 1u);
 }
 // One thread, after the barrier behind the deposits of its CTA: arrive at landing L of message h with weight wgt.
-__device__ __noinline__ void arrive(const Ctx& C, const int inst, const int seq, const int slot, const int flags, const Landing& L, int wgt,
+__device__ __noinline__ void arrive(const Ctx& C, const int inst, const int seq, const int slot, const int flags, const int ibase, const Landing& L, int wgt,
                                     unsigned long long* node_msgs) {
   IN_SMEM(&L); IN_SMEM(node_msgs);
   int* const jcnt = reinterpret_cast<int*>(C.ctl_base + L.jcnt_off);
-  Hdr h; h.inst = inst; h.seq = seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = 1; h.flags = flags;
+  Hdr h; h.inst = inst; h.seq = seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = ibase; h.flags = flags;
   if (L.act == ACT_RETIRE && L.expected) {                       // the message's arrivals meet first, then it retires whole
     if (atom_add_acq_rel(jcnt, wgt) + wgt != L.expected) return;
     *(volatile int*)jcnt = 0;
@@ -715,6 +719,21 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   const bool bulk_ok = !lookup && (P.xcache != nullptr || ((in & 3) == 0 && (C.inst.dense_dim & 3) == 0));
   const int xwidth = P.xcache ? P.xld : in;
 
+  // The cached input rows of the batch, copied asynchronously (16 bytes per cp.async, straight from L2) by the front warps
+  // once the keys are known; they wait for their own copies at the end of the front end, the block barrier does the rest.
+  auto stage_async = [&](void) {
+    asm volatile("bar.sync 1, 128;" ::: "memory");                    // the row pointers of the batch are in place
+    const int count = S.count;
+    if (!S.ok || count == 0 || !bulk_ok) return;
+    const int c4 = xwidth >> 2, total = count * c4;
+    const FastDiv dC(c4);
+    for (int idx = tid; idx < total; idx += 128) {
+      const int b = dC.div(idx), c = idx - b * c4;
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(smem_u32(Xs + (size_t)b * LX + 4 * c)), "l"(S.rowptr[b] + 4 * c) : "memory");
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  auto stage_wait = [&](void) { asm volatile("cp.async.wait_all;" ::: "memory"); };
   // Front end of a batch (warps 0-3, 128 threads = one per message): warp 0 takes the batch from the rings, then every
   // message gets its key, its staging copy is issued and its route resolved.  It runs for batch n + 1 while the other warps
   // arrive for batch n.
@@ -741,26 +760,22 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     TPHASE(0);
     if (!S.ok) return;
     const int count = S.count, dir = S.dir;
-    if (count == 0) return;
-    const unsigned bar = smem_u32(&S.mbar);
-    if (tid == 0 && bulk_ok) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((unsigned)(count * xwidth * 4)) : "memory");
+    if (count == 0) return;                         // (uniform over the front warps: nobody reaches the staging barrier)
+    long long key = -1;
+    Hdr h = Hdr{0, 0, 0, 0, 0, 0, 0, 0};
     if (tid < count) {
-      const Hdr h = S.hdr[pbn][tid];
-      const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      h = S.hdr[pbn][tid];
+      key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
       S.key[tid] = key;
       S.nd[pbn][tid] = 0; S.pre[pbn][tid] = 0;
       if (key < 0) S.ok = 0;
+      else if (!lookup) S.rowptr[tid] = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+    }
+    stage_async();                                  // the rows are on their way while the routes are resolved
+    if (tid < count) {
       if (key >= 0) {
-        if (!lookup) {
-          const float* x = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
-          S.rowptr[tid] = x;
-          if (bulk_ok) {
-            asm volatile("fence.proxy.async;" ::: "memory");
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         :: "r"(smem_u32(Xs + (size_t)tid * LX)), "l"(x), "r"((unsigned)(xwidth * 4)), "r"(bar) : "memory");
-          }
-        } else {
-          const int id = C.inst.tokens[C.inst.offsets[h.inst] + h.u];
+        if (lookup) {
+          const int id = C.inst.tokens[(long long)h.rows + h.u];
           S.rowid[tid] = (unsigned)id < (unsigned)in ? id : -1;
         }
         if (leader && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
@@ -768,7 +783,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         int pre = 0, nd = 0;
         if (fused) {                                   // the label, fetched while the input rows are in flight
           const DevInst& I = C.inst;
-          if (g_nodes[loss_node].type == LOSS_CE) S.rowid[tid] = I.labels_i[I.labels_per_node ? I.offsets[h.inst] + h.u : h.inst];
+          if (g_nodes[loss_node].type == LOSS_CE) S.rowid[tid] = I.labels_i[I.labels_per_node ? (long long)h.rows + h.u : h.inst];
           else S.rowid[tid] = __float_as_int(I.labels_f[h.inst]);
         }
         if (fused) {                                   // the Loss and this node's own backward arrival, then the way back
@@ -779,6 +794,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         S.nd[pbn][tid] = (unsigned char)nd; S.pre[pbn][tid] = (short)pre;
       }
     }
+    stage_wait();
     __syncwarp();
     TPHASE(1);
   };
@@ -799,23 +815,6 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     }
     // ---- the staged input rows of this batch ---------------------------------------------------------------
     if (count > 0) {
-      if (bulk_ok) {
-        const unsigned bar = smem_u32(&S.mbar);
-        const unsigned parity = S.mbar_parity;
-        unsigned done = 0, spins = 0;
-        for (;;) {
-          asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-          if (done) break;
-          if ((++spins & 1023u) == 0 && (aborted(C) || gtime() - t0 > C.timeout_ns)) {
-            if (tid == 0) fail(C, ST_TIMEOUT, P.node, 7);
-            for (unsigned extra = 0; extra < (1u << 16) && !done; extra++)
-              asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-            break;
-          }
-        }
-      }
-      __syncthreads();
-      if (tid == 0 && bulk_ok) S.mbar_parity ^= 1u;
       if (!lookup && !bulk_ok) {
         for (int idx = tid; idx < count * in; idx += FT) { const int b = dIn.div(idx), c = idx - b * in; Xs[b * LX + c] = __ldcg(S.rowptr[b] + c); }
         __syncthreads();
@@ -1015,7 +1014,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         if (q == 0 && fused && eval_n) retire_arrive(C, S.hdr[pb][b].slot, JOIN_UNIT);   // a forward-only instance ends at its Losses
         if (q >= S.nd[pb][b]) continue;
         const Hdr& h = S.hdr[pb][b];
-        arrive(C, h.inst, h.seq, h.slot, h.flags, S.dl[pb][b][q], wgt, &S.node_msgs);
+        arrive(C, h.inst, h.seq, h.slot, h.flags, h.rows, S.dl[pb][b][q], wgt, &S.node_msgs);
       }
     }
     if (warp >= 4) { __syncwarp(); if (lane == 0) atomicAdd(&S.arr_done, 1u); }
@@ -1033,7 +1032,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   if (tid == 0 && S.node_msgs) atomicAdd(&C.g->node_messages, S.node_msgs);
   if (leader) {
     if (!fwd_only && tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
-    if (tid < 8) P.stats->phase_cycles[tid] = S.phase[tid];
+    if (tid < (fwd_only ? 8 : 16)) P.stats->phase_cycles[tid] = S.phase[tid];
     if (tid == 0) {
       PPTStats& st = *P.stats;
       if (!fwd_only) { st.max_staleness = S.max_stale; st.log_n = S.log_n; st.n_updates = S.n_updates; st.n_grads_applied = S.n_grads_applied; }
@@ -1238,7 +1237,7 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
         if (q == 0 && leader && S.pre[pb][b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[pb][b]);
         if (q >= S.nd[pb][b]) continue;
         const Hdr& h = S.hdr[pb][b];
-        arrive(C, h.inst, h.seq, h.slot, h.flags, S.dl[pb][b][q], wgt, &S.node_msgs);
+        arrive(C, h.inst, h.seq, h.slot, h.flags, h.rows, S.dl[pb][b][q], wgt, &S.node_msgs);
       }
     }
     if (warp >= 4) { __syncwarp(); if (lane == 0) atomicAdd(&S.arr_done, 1u); }
@@ -1377,7 +1376,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
       __syncthreads();
       // pump the source messages (Sec. 4: tokens / leaves, initial hidden state, dense row)
       const int inst = S.admit_inst;
-      Hdr h; h.inst = inst; h.seq = S.admit_seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = 1; h.flags = S.admit_eval ? HDR_EVAL : 0;
+      Hdr h; h.inst = inst; h.seq = S.admit_seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = (int)(I.offsets ? I.offsets[inst] : 0); h.flags = S.admit_eval ? HDR_EVAL : 0;
       for (int s = 0; s < C.n_sources; s++) {
         const DevNode& sn = g_nodes[C.src_nodes[s]];
         const int cnt = S.src_count[s];
@@ -1396,7 +1395,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
               const unsigned q = tk & P.ring[FWD].mask;
               int4* d = reinterpret_cast<int4*>(&P.ring[FWD].e[q]);
               d[0] = make_int4(inst, S.admit_seq, slot, 0);
-              d[1] = make_int4(u, 0, 1, h.flags);
+              d[1] = make_int4(u, 0, h.rows, h.flags);
               st_rel(&P.ring[FWD].seq[q], tk + 1u);
             }
             if (lane == 0 && vm) atomicAdd(&S.node_msgs, (unsigned long long)__popc(vm));
@@ -1416,7 +1415,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
           __syncwarp();
           if (lane == 0) {
             if (pre) atomicAdd(&S.node_msgs, (unsigned long long)pre);
-            for (int q = 0; q < nd; q++) arrive(C, h.inst, h.seq, h.slot, h.flags, S.dl[q], JOIN_UNIT, &S.node_msgs);
+            for (int q = 0; q < nd; q++) arrive(C, h.inst, h.seq, h.slot, h.flags, h.rows, S.dl[q], JOIN_UNIT, &S.node_msgs);
           }
           __syncwarp();
         }
