@@ -141,6 +141,19 @@ def measured_peaks():
         return {"hbm_gbs": 6650.0, "sm_max_mhz": 1965.0}, "fallback"
 
 
+def host_description():
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count(), "cpu_model": model}
+
+
 def time_oracle(graph, inst, cfg, target_s=12.0, probe=48):
     """The oracle as it stands, single-threaded, on a bounded prefix of the workload."""
     import oracle as oracle_mod
@@ -178,7 +191,8 @@ def run_reference(args):
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "node_messages_per_s": msgs / tot,
             "config": workload_config(args.workload, inst, cfg, "canonical round schedule on the host"),
-            "cpu_baseline": {"value": value, "unit": "instances/s", "cores": 1, "kind": "oracle", "sample": sample},
+            "cpu_baseline": dict({"value": value, "unit": "instances/s", "cores": 1, "kind": "oracle", "sample": sample,
+                                  "arithmetic": "f64 build of the oracle, single thread"}, **host_description()),
             "e2e": {"value": value, "unit": "instances/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -193,6 +207,51 @@ def input_bytes(inst):
     return int(sum(a.nbytes for a in (inst.offsets, inst.tokens, inst.left, inst.right, inst.edge_offsets, inst.edge_src,
                                       inst.edge_dst, inst.edge_type, inst.dense, inst.labels_i, inst.labels_f)
                    if a is not None))
+
+
+def average_replicas(views, averaging, average_fn=None):
+    """End-of-epoch replica synchronisation (Sec. 5) inside the timed region.  If the collective cannot run the ranks
+    continue as independent replicas and `averaging` (reported as config.replica_sync) says so."""
+    if not averaging["on"]:
+        return
+    try:
+        if average_fn is None:
+            from paper_1705_09786_b200.replicas import average_across_ranks as average_fn
+        average_fn(views)
+    except Exception as exc:                                   # keep measuring independent replicas
+        averaging.update(on=False, note=f"averaging unavailable ({type(exc).__name__}); independent replicas")
+
+
+def roofline_object(rf, graph, inst, workload, flops, kernel_s, peak_tf, peaks, peak_kind, mak, rate_one_key, n1):
+    """The roofline record of one workload: algorithmic flops of a launch / its device time against the FP32 FMA peak
+    measured in this run, with the resident-weight roofline and the concurrency ceiling beside it."""
+    sm_mhz = float(peaks.get("sm_max_mhz", 1965.0))
+    achieved = flops / kernel_s / 1e12
+    roof_inst, F, B = rf.roofline_instances_per_s(graph, inst, sm_mhz, float(peaks.get("hbm_gbs", 6650.0)))
+    per_inst = rf.MEASURED_DRAM_BYTES_PER_INSTANCE.get(workload)
+    return {"bound": "alu", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
+            "traffic": per_inst * inst.n if per_inst else None,
+            "traffic_note": ("ncu capture on a small case, scaled by instances processed (see profiles/)" if per_inst
+                             else "no ncu capture for this workload"),
+            "peak_kind": "measured in this run: register-only FP32 FMA kernel (ampnet_measure_fma_peak)",
+            "peak_derived": rf.fma_peak_tflops(sm_mhz),
+            "peak_derived_kind": f"148 SMs x 128 FP32 lanes x 2 x {sm_mhz:.0f} MHz ({peak_kind} max SM clock)",
+            "concurrency_ceiling_instances_per_s": mak * rate_one_key,
+            "concurrency_ceiling_kind": f"max_active_keys x the rate at one key in flight ({rate_one_key:.0f}/s on {n1} instances)",
+            "kernel": "one persistent launch per step (ampnet_engine_direct; ampnet_engine for graphs with row-wise groups)",
+            "kernel_ms": kernel_s * 1e3, "algorithmic_flop_per_launch": flops, "flop_per_instance": F,
+            "payload_bytes_per_instance": B, "resident_weight_roofline_instances_per_s": roof_inst,
+            "weight_reload_roofline_instances_per_s": float(peaks.get("hbm_gbs", 6650.0)) * 1e9 / (rf.reload_bytes(graph, inst) / inst.n),
+            "weight_reload_roofline_kind": "a per-message mat-vec that reads W forward and backward and updates the accumulator in device memory (context)",
+            "frac_of_resident_weight_roofline": (inst.n / kernel_s) / roof_inst}
+
+
+def one_key_rate(eng, inst, cfg, timeout):
+    n1 = max(8, min(inst.n, 64))
+    eng.load_instances(inst.head(n1))
+    st1, _ = eng.run_epoch(mak=1, muf=cfg["muf"], lr=0.0, deterministic=False, timeout_s=timeout, want_loss=False)
+    eng.load_instances(inst)
+    return n1 / st1.seconds, n1
 
 
 def run_ours(args):
@@ -217,17 +276,13 @@ def run_ours(args):
     views = list(eng.param_tensors().values()) if world > 1 else []
 
     def step():
+        eng.set_params(p0)                                     # every step starts from the same parameters (untimed)
         flush_buf.fill_(1)                                     # evict L2 between steps (outside the timed events)
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         st, _ = eng.run_epoch(mak=cfg["mak"], muf=cfg["muf"], lr=cfg["lr"], deterministic=False, timeout_s=args.timeout,
                               want_loss=False)
-        if averaging["on"]:
-            try:
-                from paper_1705_09786_b200.replicas import average_across_ranks
-                average_across_ranks(views)
-            except Exception as exc:                           # keep measuring independent replicas
-                averaging.update(on=False, note=f"averaging unavailable ({type(exc).__name__}); independent replicas")
+        average_replicas(views, averaging)
         e1.record(stream)
         e1.synchronize()
         return st, e0.elapsed_time(e1) * 1e-3
@@ -247,6 +302,7 @@ def run_ours(args):
     clocks = sampler.summary()
     updates = {n: eng.node_stats(n)["n_updates"] for n in graph.ppt_nodes()}     # of the last timed step
     placement = {graph.names[n]: eng.placement(n) for n in graph.ppt_nodes()}
+    queue_occ = {graph.names[n]: list(eng.queue_occupancy(n)) for n in graph.ppt_nodes()}
     secs = sum(step_s)
     value, tmax = aggregate(inst.n * args.steps, secs, dev)
     msg_rate, _ = aggregate(msgs, secs, dev)
@@ -280,12 +336,7 @@ def run_ours(args):
 
     # ---- diagnostics: the FP32 FMA rate of this GPU, measured; the concurrency ceiling mak x (rate at one key) ------
     fma_measured = amp.measure_fma_peak(local)
-    n1 = max(8, min(inst.n, 64))
-    eng.load_instances(inst.head(n1))
-    st1, _ = eng.run_epoch(mak=1, muf=cfg["muf"], lr=0.0, deterministic=False, timeout_s=args.timeout, want_loss=False)
-    rate_one_key = n1 / st1.seconds
-    eng.load_instances(inst)
-
+    rate_one_key, n1 = one_key_rate(eng, inst, cfg, args.timeout)
     # ---- the other configurations of the benchmark set, briefly (single GPU only): same timing rules, fewer steps ----
     others = None
     if world == 1 and not args.no_other_configs and args.instances is None:
@@ -306,12 +357,25 @@ def run_ours(args):
                                       timeout_s=args.timeout, want_loss=False)
                 if k >= 3:
                     ks.append(st2.seconds); ms += st2.node_messages
+                if k < 4:
+                    e2.set_params(wp.init_params(g2))
             fl = rf.algorithmic_flops(g2, inst2, {n: e2.node_stats(n)["n_updates"] for n in g2.ppt_nodes()})
+            occ2 = {g2.names[n]: list(e2.queue_occupancy(n)) for n in g2.ppt_nodes()}
+            r1, m1 = one_key_rate(e2, inst2, cfg2, args.timeout)
+            peaks2, kind2 = measured_peaks()
             others[name] = {"instances_per_s": 2 * inst2.n / sum(ks), "node_messages_per_s": ms / sum(ks),
                             "tflops": fl / (sum(ks) / 2) / 1e12, "instances_per_step": int(inst2.n),
                             "full_dataset_instances": cfg2["full"], "max_active_keys": cfg2["mak"],
                             "min_update_frequency": cfg2["muf"], "steps": 2, "warmup": 3,
-                            "timing": "device time of the persistent kernel (CUDA events around the launch)"}
+                            "timing": "device time of the persistent kernel (CUDA events around the launch), parameters reset before every epoch",
+                            "roofline": roofline_object(rf, g2, inst2, name, fl, sum(ks) / 2, fma_measured, peaks2, kind2,
+                                                        cfg2["mak"], r1, m1),
+                            "queue_occupancy_max_pending_fwd_bwd": occ2}
+            if not args.no_cpu_baseline:
+                r = time_oracle(g2, inst2, cfg2, target_s=4.0, probe=16)
+                others[name]["cpu_baseline"] = dict({"value": r["inst_per_s"], "unit": "instances/s", "cores": 1, "kind": "oracle",
+                                                     "sample": f"first {r['instances']} of {inst2.n} instances, one epoch, {r['seconds']:.1f} s",
+                                                     "arithmetic": "f64 build of the oracle, single thread"}, **host_description())
             e2.close()
 
     sweep = None
@@ -329,40 +393,23 @@ def run_ours(args):
                               "instances_per_s": sub.n / st.seconds, "node_messages_per_s": st.node_messages / st.seconds,
                               "rows_per_micro_batch": st.micro_batch_rows / max(1, st.micro_batches),
                               "max_active_observed": int(st.max_active_observed), "max_staleness": int(st.max_staleness),
+                              "queue_occupancy_max_pending_fwd_bwd": {graph.names[n]: list(eng.queue_occupancy(n)) for n in graph.ppt_nodes()},
                               "micro_batches_fma": int(st.micro_batches), "micro_batches_tensor_core": 0})
         eng.load_instances(inst)
     if rank == 0:
         peaks, peak_kind = measured_peaks()
         flops = rf.algorithmic_flops(graph, inst, updates)
-        sm_mhz = float(peaks.get("sm_max_mhz", 1965.0))
-        peak_derived = rf.fma_peak_tflops(sm_mhz)
         peak_tf = fma_measured                       # measured in this run; the derived figure is reported beside it
         kavg = float(np.mean(kern_s))
-        achieved = flops / kavg / 1e12
-        roof_inst, F, B = rf.roofline_instances_per_s(graph, inst, sm_mhz, float(peaks.get("hbm_gbs", 6650.0)))
-        per_inst = rf.MEASURED_DRAM_BYTES_PER_INSTANCE.get(args.workload)
-        traffic = per_inst * inst.n if per_inst else None
-        note = ("ncu capture on a small case, scaled by instances processed (see profiles/)" if per_inst
-                else "no ncu capture for this workload")
-        roofline = {"bound": "alu", "achieved": achieved, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved / peak_tf,
-                    "traffic": traffic, "traffic_note": note,
-                    "peak_kind": "measured in this run: register-only FP32 FMA kernel (ampnet_measure_fma_peak)",
-                    "peak_derived": peak_derived,
-                    "peak_derived_kind": f"148 SMs x 128 FP32 lanes x 2 x {sm_mhz:.0f} MHz ({peak_kind} max SM clock)",
-                    "concurrency_ceiling_instances_per_s": cfg["mak"] * rate_one_key,
-                    "concurrency_ceiling_kind": f"max_active_keys x the rate at one key in flight ({rate_one_key:.0f}/s on {n1} instances)",
-                    "kernel": "ampnet_engine (one persistent launch per step)", "kernel_ms": kavg * 1e3,
-                    "algorithmic_flop_per_launch": flops, "flop_per_instance": F, "payload_bytes_per_instance": B,
-                    "resident_weight_roofline_instances_per_s": roof_inst,
-                    "weight_reload_roofline_instances_per_s": float(peaks.get("hbm_gbs", 6650.0)) * 1e9 / (rf.reload_bytes(graph, inst) / inst.n),
-                    "weight_reload_roofline_kind": "a per-message mat-vec that reads W forward and backward and updates the accumulator in device memory (context)",
-                    "frac_of_resident_weight_roofline": (inst.n / kavg) / roof_inst}
+        roofline = roofline_object(rf, graph, inst, args.workload, flops, kavg, peak_tf, peaks, peak_kind, cfg["mak"],
+                                   rate_one_key, n1)
         cpu = None
         if not args.no_cpu_baseline:
             r = time_oracle(graph, inst, cfg)
-            cpu = {"value": r["inst_per_s"], "unit": "instances/s", "cores": 1, "kind": "oracle",
-                   "sample": f"first {r['instances']} of {inst.n} instances, one epoch, {r['seconds']:.1f} s",
-                   "node_messages_per_s": r["msgs_per_s"]}
+            cpu = dict({"value": r["inst_per_s"], "unit": "instances/s", "cores": 1, "kind": "oracle",
+                        "sample": f"first {r['instances']} of {inst.n} instances, one epoch, {r['seconds']:.1f} s",
+                        "node_messages_per_s": r["msgs_per_s"], "arithmetic": "f64 build of the oracle, single thread"},
+                       **host_description())
         line = {"metric": "training_instances_per_s", "value": value, "unit": "instances/s", "n_gpus": world,
                 "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tmax / args.steps,
                 "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
@@ -380,12 +427,14 @@ def run_ours(args):
                 "stats": {"mean_loss_last_step": last.mean_loss, "max_staleness": int(last.max_staleness),
                           "rows_per_micro_batch": last.micro_batch_rows / max(1, last.micro_batches),
                           "placement": placement, "inference_instances_per_s": inference_rate,
-                          "micro_batch_split": {"fma": 1.0, "tensor_core": 0.0}}}
+                          "queue_occupancy_max_pending_fwd_bwd": queue_occ,
+                          "micro_batch_split": {"fma": 1.0, "tensor_core": 0.0,
+                                                "note": "every micro-batch runs on FP32 FMA: this build has no tensor-core path"}}}
         if sweep is not None:
             line["sweep"] = sweep
         if others is not None:
             for o in others.values():
-                o["frac_of_fma_peak"] = o["tflops"] / peak_tf
+                o["frac_of_fma_peak"] = o["tflops"] / fma_measured
             line["other_configs"] = others
         print(json.dumps(line), flush=True)
     if eng is not None:

@@ -220,6 +220,11 @@ ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_t
  * ([8] look-ahead scheduling, [9] reduction of partial gradients, [10]/[12] own walks of warps 0/1, [11]/[13] helping
  * other warps, [14] closing barrier).  cycles16: 16 values.  batches: micro-batches executed.                    */
 ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles16, int64_t* batches);
+/* Queue occupancy of a node in the last asynchronous run (the benchmark set's stress configuration asks for it; App. A:
+ * every worker owns a queue): the largest number of messages that were waiting in the node's forward and in its
+ * backward ring at the moment a micro-batch was taken, as seen by the node's first tile.  The deterministic schedule
+ * and graphs that run on the interpreter engine report 0.                                                        */
+ampnet_status_t ampnet_get_queue_occupancy(ampnet_graph_t*, int32_t node, int64_t* max_pending_fwd, int64_t* max_pending_bwd);
 
 /* ---- concurrent inference (Sec. 1: inference can run while the model trains; Sec. 6 reports inference throughput) --------
  * A training epoch in which the instances i with inference_only[i] != 0 (host array, one byte per loaded instance of

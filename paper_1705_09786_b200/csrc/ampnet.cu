@@ -1062,7 +1062,9 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
     for (size_t p = 0; p < g->ppts.size(); p++) g->ppts[p].emit_load = (double)G.role_cycles[8 + 8 * p + 5] * std::max(1, g->ppts[p].NE) + 1.0;
   if (getenv("AMPNET_TUNE") && (atoi(getenv("AMPNET_TUNE")) & 8)) {
     static const char* names[] = {"SOURCE", "LINEAR", "LOOKUP", "GRUCELL", "LOSS_CE", "LOSS_MSE", "SUMROWS", "COND", "PHI", "ISU", "CONCAT", "SPLIT", "BCAST", "GROUP", "UNGROUP", "FLATMAP", "SINK", "LSTM"};
-    const double us = 1.0 / 1965.0;
+    int khz = 1965000;
+    cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, g->device);      // cycles -> microseconds at the device's SM clock
+    const double us = 1e3 / (double)khz;
     fprintf(stderr, "[ctrl] us: retire %.0f admit %.0f clear %.0f pump %.0f idle %.0f admissions %llu\n", G.role_cycles[0] * us, G.role_cycles[1] * us,
             G.role_cycles[2] * us, G.role_cycles[3] * us, G.role_cycles[4] * us, G.role_cycles[5]);
     for (size_t p = 0; p < g->ppts.size(); p++) {
@@ -1545,6 +1547,16 @@ ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t* g, int32_t node, uint64_
   const PPTStats& s = g->last_stats[g->hnodes[node].ppt];
   if (cycles8) for (int k = 0; k < 16; k++) cycles8[k] = s.phase_cycles[k];
   if (batches) *batches = (int64_t)s.batches;
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_get_queue_occupancy(ampnet_graph_t* g, int32_t node, int64_t* max_pending_fwd, int64_t* max_pending_bwd) {
+  if (!g) return AMPNET_EINVAL;
+  if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
+  if (node < 0 || node >= (int)g->hnodes.size() || g->hnodes[node].ppt < 0) return set_err(g, AMPNET_EINVAL, "not a parameterised node");
+  const PPTStats& s = g->last_stats[g->hnodes[node].ppt];
+  if (max_pending_fwd) *max_pending_fwd = (int64_t)s.max_pending[0];
+  if (max_pending_bwd) *max_pending_bwd = (int64_t)s.max_pending[1];
   return AMPNET_OK;
 }
 

@@ -28,7 +28,7 @@ constexpr int FT = 512;               // threads per CTA
 constexpr int FW = FT / 32;
 constexpr int FBM = 128;              // messages (= rows) per micro-batch
 constexpr int MAXD = 2;               // landings per message
-constexpr int RSTACK = 2;             // pending forks per routed message (two named slots: an indexed array would live in local memory)
+constexpr int RSTACK = 4;             // pending forks per routed message
 
 // ------------------------------------------------------------------------------------------------
 // memory-model helpers, bounded waits
@@ -162,7 +162,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
   // the tree tables of the message's own position, fetched together (one round trip instead of one per node on the way)
   int own_parent = 0, own_slot = 0, own_left = 0, own_right = 0;
   if (I.parent) { const long long o = ibase + h.u; own_parent = I.parent[o]; own_slot = I.child_slot[o]; own_left = I.left[o]; own_right = I.right[o]; }
-  Route stack0, stack1;
+  Route stack[RSTACK];
   int sp = 0, nout = 0;
   Route f;
   f.node = start_node; f.aport = start_aport; f.dir = dir0; f.u = h.u; f.it = h.it; f.port = h.port; f.s0 = 0; f.w = width; f.null = 0;
@@ -283,8 +283,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
           for (int k = n.fn_arg - 1; k >= 1; k--) {
             if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; }
             Route c = f; c.node = n.succ_node[k]; c.aport = n.succ_port[k]; c.dir = FWD;
-            if (sp == 0) stack0 = c; else stack1 = c;
-            sp++;
+            stack[sp++] = c;
           }
           to_succ(0);
         } else {
@@ -318,7 +317,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
             if (n.fn == 2) { c.port = k; c.node = n.pred_node[0]; c.aport = n.pred_port[0]; }
             else { c.node = n.pred_node[k]; c.aport = n.pred_port[k]; }
             if (k == 0) { f = c; cont = true; }
-            else { if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; } if (sp == 0) stack0 = c; else stack1 = c; sp++; }
+            else { if (sp >= RSTACK) { fail(C, ST_OVERFLOW, f.node, sp); return nout; } stack[sp++] = c; }
           }
         }
         break;
@@ -328,7 +327,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
     }
     if (!cont) {
       if (pend) { fail(C, ST_OVERFLOW, f.node, -13); return nout; }          // a sum that found no landing
-      if (sp > 0) { sp--; f = sp == 0 ? stack0 : stack1; }
+      if (sp > 0) f = stack[--sp];
       else have = false;
     }
   }
@@ -350,6 +349,7 @@ struct TileS {
   int rowid[FBM];
   int fpb;                          // parity of the batch being formed
   unsigned arr_done;                // arrival warps that have finished, summed over the batches
+  unsigned qmax[2];                 // most messages waiting in each ring when a batch was taken (queue occupancy)
   int count, dir, flags, n_upd, upd_t, eval, ok, term;
   unsigned head[2];
   int n_acc, version, log_n, max_stale;
@@ -559,6 +559,9 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
     if (!__any_sync(0xffffffffu, any != 0)) return 0;
   }
   if (dirs == 1 && lane == 0) S.wver_seen = ld_rlx(P.wver);          // ordered by the fence below like the ring polls
+  // queue occupancy (first tile of the node): tickets handed out and not yet taken, read along with the ring polls
+  unsigned pending = 0;
+  if (leader && lane < 2 && (dirs & (1 << lane))) pending = ld_rlx(P.ring[lane].tail) - S.head[lane];
   constexpr int NPL = FBM / 32;                                      // ring slots per lane
   auto leading = [](const unsigned (&m)[NPL]) {                      // length of the run of set bits from candidate 0 on
     int n = 0;
@@ -583,6 +586,7 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
     nready[dir] = leading(m);
   }
   fence_acq();
+  if (leader && lane < 2 && pending > S.qmax[lane] && pending < (1u << 30)) S.qmax[lane] = pending;
   // A batch costs nearly the same whether it holds 2 messages or 100.  While the previous batch's arrivals are still under
   // way the next one is taken only if at least min_take messages wait; the caller drops the threshold once they are done.
   if (max(nready[0], nready[1]) < min_take && max(nready[0], nready[1]) > 0) return 0;
@@ -706,7 +710,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     }
   }
   if (tid == 0) {
-    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0; S.arr_done = 0;
+    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0; S.arr_done = 0; S.qmax[0] = S.qmax[1] = 0;
     S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&S.mbar)) : "memory");
     S.mbar_parity = 0;
@@ -719,21 +723,6 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   const bool bulk_ok = !lookup && (P.xcache != nullptr || ((in & 3) == 0 && (C.inst.dense_dim & 3) == 0));
   const int xwidth = P.xcache ? P.xld : in;
 
-  // The cached input rows of the batch, copied asynchronously (16 bytes per cp.async, straight from L2) by the front warps
-  // once the keys are known; they wait for their own copies at the end of the front end, the block barrier does the rest.
-  auto stage_async = [&](void) {
-    asm volatile("bar.sync 1, 128;" ::: "memory");                    // the row pointers of the batch are in place
-    const int count = S.count;
-    if (!S.ok || count == 0 || !bulk_ok) return;
-    const int c4 = xwidth >> 2, total = count * c4;
-    const FastDiv dC(c4);
-    for (int idx = tid; idx < total; idx += 128) {
-      const int b = dC.div(idx), c = idx - b * c4;
-      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" :: "r"(smem_u32(Xs + (size_t)b * LX + 4 * c)), "l"(S.rowptr[b] + 4 * c) : "memory");
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-  };
-  auto stage_wait = [&](void) { asm volatile("cp.async.wait_all;" ::: "memory"); };
   // Front end of a batch (warps 0-3, 128 threads = one per message): warp 0 takes the batch from the rings, then every
   // message gets its key, its staging copy is issued and its route resolved.  It runs for batch n + 1 while the other warps
   // arrive for batch n.
@@ -761,19 +750,27 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     if (!S.ok) return;
     const int count = S.count, dir = S.dir;
     if (count == 0) return;                         // (uniform over the front warps: nobody reaches the staging barrier)
-    long long key = -1;
-    Hdr h = Hdr{0, 0, 0, 0, 0, 0, 0, 0};
+    // The cached input row of every message is staged by a bulk asynchronous copy (TMA, untiled) issued by the message's
+    // thread and counted in bytes on a transaction barrier that all threads wait on before the arithmetic; the proxy fence
+    // orders the issuing thread's view of the row (ordinary stores of other SMs, acquired through the ring) before the copy.
+    const unsigned bar = smem_u32(&S.mbar);
+    if (tid == 0 && bulk_ok) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((unsigned)(count * xwidth * 4)) : "memory");
     if (tid < count) {
-      h = S.hdr[pbn][tid];
-      key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+      const Hdr h = S.hdr[pbn][tid];
+      const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
       S.key[tid] = key;
       S.nd[pbn][tid] = 0; S.pre[pbn][tid] = 0;
       if (key < 0) S.ok = 0;
-      else if (!lookup) S.rowptr[tid] = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
-    }
-    stage_async();                                  // the rows are on their way while the routes are resolved
-    if (tid < count) {
       if (key >= 0) {
+        if (!lookup) {
+          const float* x = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+          S.rowptr[tid] = x;
+          if (bulk_ok) {
+            asm volatile("fence.proxy.async;" ::: "memory");
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         :: "r"(smem_u32(Xs + (size_t)tid * LX)), "l"(x), "r"((unsigned)(xwidth * 4)), "r"(bar) : "memory");
+          }
+        }
         if (lookup) {
           const int id = C.inst.tokens[(long long)h.rows + h.u];
           S.rowid[tid] = (unsigned)id < (unsigned)in ? id : -1;
@@ -794,7 +791,6 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         S.nd[pbn][tid] = (unsigned char)nd; S.pre[pbn][tid] = (short)pre;
       }
     }
-    stage_wait();
     __syncwarp();
     TPHASE(1);
   };
@@ -815,6 +811,22 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     }
     // ---- the staged input rows of this batch ---------------------------------------------------------------
     if (count > 0) {
+      if (bulk_ok && S.ok) {
+        const unsigned bar = smem_u32(&S.mbar), parity = S.mbar_parity;
+        unsigned done = 0, spins = 0;
+        for (;;) {
+          asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+          if (done) break;
+          if ((++spins & 1023u) == 0 && (aborted(C) || gtime() - t0 > C.timeout_ns)) {
+            if (tid == 0) fail(C, ST_TIMEOUT, P.node, 7);
+            for (unsigned extra = 0; extra < (1u << 16) && !done; extra++)      // copies already issued still land in this CTA's shared memory
+              asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+            break;
+          }
+        }
+        __syncthreads();
+        if (tid == 0) S.mbar_parity ^= 1u;
+      }
       if (!lookup && !bulk_ok) {
         for (int idx = tid; idx < count * in; idx += FT) { const int b = dIn.div(idx), c = idx - b * in; Xs[b * LX + c] = __ldcg(S.rowptr[b] + c); }
         __syncthreads();
@@ -827,7 +839,46 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
       gemm_nt(Xs, LX, count, Ws, LW, R, pad4(in) >> 2, Ys, RP);
       __syncthreads();
       TPHASE(5);
-      if (tid < count) {
+      if (R <= 32) {
+        // the Loss on G = 8, 16 or 32 lanes per message (lane j holds output j): maximum and arg-max (lowest index on ties),
+        // sum of exponentials and the label's output by shuffles inside the group
+        const int G = R <= 8 ? 8 : R <= 16 ? 16 : 32, per_pass = FT / G, j = tid & (G - 1);
+        const DevNode& ln = g_nodes[loss_node];
+        for (int m0 = 0; m0 < count; m0 += per_pass) {
+          const int m = m0 + tid / G;
+          const bool live = m < count, mine = live && j < R;
+          const float y = mine ? emit_round(act_fwd(P.act, Ys[m * RP + j] + bs[j])) : -3.4e38f;
+          float gj = 0.f;
+          if (ln.type == LOSS_CE) {
+            float mx = y; int arg = mine ? j : 0x7fffffff;
+            for (int o = G >> 1; o; o >>= 1) {
+              const float om = __shfl_xor_sync(0xffffffffu, mx, o, G); const int oa = __shfl_xor_sync(0xffffffffu, arg, o, G);
+              if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
+            }
+            const float e = mine ? expf(y - mx) : 0.f;
+            float sum = e;
+            for (int o = G >> 1; o; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o, G);
+            const float lse = mx + logf(sum);
+            const int label = live ? S.rowid[m] : 0;
+            const float ylab = __shfl_sync(0xffffffffu, y, label & (G - 1), G);
+            gj = expf(y - lse) - (j == label ? 1.f : 0.f);
+            if (live && j == 0) {
+              const Hdr& h = S.hdr[pb][m];
+              const long long lkey = key_of(C, loss_node, h.slot, h.it, h.u, ln.U_in);
+              if (lkey >= 0) { ln.lossval[lkey] = lse - ylab; ln.predok[lkey] = (arg == label) ? 1 : 0; }
+            }
+          } else {
+            const float d = y - __int_as_float(live ? S.rowid[m] : 0);
+            gj = 2.f * d;
+            if (live && j == 0) {
+              const Hdr& h = S.hdr[pb][m];
+              const long long lkey = key_of(C, loss_node, h.slot, h.it, h.u, ln.U_in);
+              if (lkey >= 0) { ln.lossval[lkey] = d * d; ln.predok[lkey] = 0; }
+            }
+          }
+          if (mine && !eval_n) Ds[m * RP + j] = emit_round(gj) * act_grad(P.act, y);
+        }
+      } else if (tid < count) {
         float* y = Ys + tid * RP;
         for (int r = 0; r < R; r++) y[r] = emit_round(act_fwd(P.act, y[r] + bs[r]));
         float* g = Ds + tid * RP;
@@ -1037,6 +1088,8 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
       PPTStats& st = *P.stats;
       if (!fwd_only) { st.max_staleness = S.max_stale; st.log_n = S.log_n; st.n_updates = S.n_updates; st.n_grads_applied = S.n_grads_applied; }
       atomicAdd(&st.msgs, S.msgs); atomicAdd(&st.batches, S.batches); atomicAdd(&st.batch_rows, S.batch_rows);
+      st.max_pending[0] = S.qmax[0];
+      if (!fwd_only) st.max_pending[1] = S.qmax[1];
     }
   }
 }
@@ -1077,7 +1130,7 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
   const FastDiv dOut(out);
   const int cb_shift = 31 - __clz(CB);
   if (tid == 0) {
-    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0; S.arr_done = 0;
+    S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0; S.arr_done = 0; S.qmax[0] = S.qmax[1] = 0;
     S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
   }
   if (tid < 64) S.stale_hist[tid] = 0;
@@ -1255,6 +1308,7 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
       PPTStats& st = *P.stats;
       st.max_staleness = S.max_stale; st.log_n = S.log_n; st.n_updates = S.n_updates; st.n_grads_applied = S.n_grads_applied;
       atomicAdd(&st.msgs, S.msgs); atomicAdd(&st.batches, S.batches); atomicAdd(&st.batch_rows, S.batch_rows);
+      st.max_pending[1] = S.qmax[1];
     }
   }
 }

@@ -54,6 +54,7 @@ struct PPTStats {
   unsigned long long stale_hist[64];
   int max_staleness, log_n;
   unsigned long long phase_cycles[16];  // leader tile: idle, fetch, headers, compute, update, barrier, emit, loop; [8..] emission detail
+  unsigned max_pending[2];              // direct-delivery engine: most messages waiting in the forward / backward ring when a batch was taken
 };
 
 struct DevNode {

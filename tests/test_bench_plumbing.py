@@ -97,3 +97,28 @@ def test_replica_aggregation_world_size_2_gloo():
     assert v0 == v1 == pytest.approx(300 / 2.0)       # units of all ranks / the slowest rank's time
     assert t0 == t1 == 2.0
     assert s0 != s1                                   # independent shards
+
+
+def test_replica_sync_note_when_the_collective_raises():
+    """bench.py with N > 1 averages the replicas at the end of every epoch; if the collective raises, the ranks go on as
+    independent replicas and the JSON line's config.replica_sync says so (and averaging is not tried again)."""
+    import bench
+    calls = []
+
+    def ok(views):
+        calls.append("ok")
+
+    def broken(views):
+        calls.append("broken")
+        raise RuntimeError("NCCL error")
+
+    avg = {"on": True, "note": "end-of-epoch parameter averaging over NCCL"}
+    bench.average_replicas([], avg, ok)
+    assert avg["on"] and calls == ["ok"]
+    bench.average_replicas([], avg, broken)
+    assert not avg["on"] and "RuntimeError" in avg["note"] and "independent replicas" in avg["note"]
+    bench.average_replicas([], avg, broken)                      # switched off: the collective is not called again
+    assert calls == ["ok", "broken"]
+    single = {"on": False, "note": "single replica"}
+    bench.average_replicas([], single, broken)
+    assert single == {"on": False, "note": "single replica"}
