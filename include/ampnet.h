@@ -211,14 +211,22 @@ ampnet_status_t ampnet_get_key_log(ampnet_graph_t*, int64_t* inst, int32_t* slot
 /* Number of keyed cache entries (join counters, recorded origins) still set after the last run; the
  * forward/backward state invariant of Sec. 4 makes this 0.                                                   */
 ampnet_status_t ampnet_leftover_cache_entries(ampnet_graph_t*, int64_t* n);
-/* Placement chosen for a parameterised node: number of row tiles (CTAs) and micro-batch row capacity.        */
+/* Placement chosen for a parameterised node: number of row tiles (CTAs) and micro-batch row capacity.  Asynchronous
+ * runs of graphs that the direct-delivery engine takes (single-row messages; Cond, Phi, Isu, Bcast, Concat, Sink and a
+ * Loss fed by a Linear node) report the forward row tiles; a Linear node has as many backward column tiles again
+ * (none for a node that feeds a Loss: that is one tile doing both directions).                                   */
 ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_tiles, int32_t* batch_rows);
 
 /* Where the leader tile of a node spent its SM cycles in the last run: [0] waiting for messages, [1] fetching a
  * batch descriptor, [2] loading headers, [3] staging + arithmetic, [4] local updates, [5] barrier among the node's
  * tiles, [6] emission (walking the parameter-free nodes), [7] loop overhead; [8..15] detail of the emission phase
  * ([8] look-ahead scheduling, [9] reduction of partial gradients, [10]/[12] own walks of warps 0/1, [11]/[13] helping
- * other warps, [14] closing barrier).  cycles16: 16 values.  batches: micro-batches executed.                    */
+ * other warps, [14] closing barrier).  After a run of the direct-delivery engine the 16 values are diagnostic marks of
+ * the node's first forward tile ([0] waiting for and taking messages, [1] keys, routes and staging of the input rows,
+ * [2] rest of the arithmetic phase, [3] update / reload of the weights, [4] arrivals and closing barrier, [5] products,
+ * [6] activation and stores / Loss and gradients of a loss head, [7] delivery of those gradients) and, for a Linear node with column tiles, [8..14] of its first backward
+ * tile in the same order of work (wait, routes and staging, incoming gradient, input gradient and delivery,
+ * accumulation, update and publication, arrivals).  cycles16: 16 values.  batches: micro-batches executed.        */
 ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t* cycles16, int64_t* batches);
 /* Queue occupancy of a node in the last asynchronous run (the benchmark set's stress configuration asks for it; App. A:
  * every worker owns a queue): the largest number of messages that were waiting in the node's forward and in its
