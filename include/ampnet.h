@@ -233,6 +233,13 @@ ampnet_status_t ampnet_get_phase_cycles(ampnet_graph_t*, int32_t node, uint64_t*
  * backward ring at the moment a micro-batch was taken, as seen by the node's first tile.  The deterministic schedule
  * and graphs that run on the interpreter engine report 0.                                                        */
 ampnet_status_t ampnet_get_queue_occupancy(ampnet_graph_t*, int32_t node, int64_t* max_pending_fwd, int64_t* max_pending_bwd);
+/* Micro-batches of a node in the last run by the unit that ran their product (the stress configuration of the benchmark
+ * set asks for this split): tensor_core_batches = forward micro-batches whose product Y^T = W X^T ran as tcgen05
+ * instructions (bf16 runs on the direct-delivery engine: nodes with out_dim a multiple of 64 and in_dim a multiple of
+ * 16; W and the batch as bfloat16 operands in shared memory, fp32 accumulator in tensor memory; the master weights,
+ * the input gradient and the accumulation stay fp32), fma_batches = all others (counted like micro_batches of the epoch
+ * statistics: by the node's first forward and first backward tile).  Either pointer may be NULL.                 */
+ampnet_status_t ampnet_get_micro_batch_split(ampnet_graph_t*, int32_t node, int64_t* fma_batches, int64_t* tensor_core_batches);
 
 /* ---- concurrent inference (Sec. 1: inference can run while the model trains; Sec. 6 reports inference throughput) --------
  * A training epoch in which the instances i with inference_only[i] != 0 (host array, one byte per loaded instance of

@@ -12,7 +12,7 @@ STATUS = {0: "OK", 1: "EINVAL", 2: "ENOMEM", 3: "ECUDA", 4: "ETIMEOUT", 5: "EOVE
 EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances", "ampnet_run_epoch", "ampnet_eval",
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
-           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_mixed", "ampnet_param_device_ptr", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_get_queue_occupancy", "ampnet_ir_mlp", "ampnet_ir_rnn",
+           "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_mixed", "ampnet_param_device_ptr", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_get_queue_occupancy", "ampnet_get_micro_batch_split", "ampnet_ir_mlp", "ampnet_ir_rnn",
            "ampnet_ir_tree", "ampnet_ir_ggnn", "ampnet_ir_tree_lstm", "ampnet_measure_fma_peak"]
 
 
@@ -99,6 +99,7 @@ def load_library():
     lib.ampnet_get_placement.argtypes = [P, C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]
     lib.ampnet_get_phase_cycles.argtypes = [P, C.c_int32, P, C.POINTER(C.c_int64)]
     lib.ampnet_get_queue_occupancy.argtypes = [P, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    lib.ampnet_get_micro_batch_split.argtypes = [P, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
     lib.ampnet_set_optimizer.argtypes = [P, C.c_int32, C.c_float, C.c_float, C.c_float, C.c_float, C.c_int32]
     I32, PI = C.c_int32, C.POINTER(C.c_int32)
     tail = [P, I32, PI, P, I32, PI]
@@ -334,6 +335,12 @@ class Engine:
         f, b = C.c_int64(), C.c_int64()
         self._check(self.lib.ampnet_get_queue_occupancy(self.h, node, C.byref(f), C.byref(b)))
         return f.value, b.value
+
+    def micro_batch_split(self, node):
+        """(FMA, tensor-core) micro-batches of the node in the last run."""
+        f, t = C.c_int64(), C.c_int64()
+        self._check(self.lib.ampnet_get_micro_batch_split(self.h, node, C.byref(f), C.byref(t)))
+        return f.value, t.value
 
     def placement(self, node):
         t, b = C.c_int32(), C.c_int32()

@@ -22,6 +22,8 @@ using namespace amp;
 extern "C" int ampnet_direct_threads();
 extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows, int loss_head);
 extern "C" size_t ampnet_direct_bwd_tile_smem_bytes(int out_dim, int cols, int batch_rows);
+extern "C" size_t ampnet_direct_tc_tile_smem_bytes(int in_dim, int batch_rows);
+extern "C" void ampnet_direct_tc_limits(int* rows, int* max_batch_rows, int* k_multiple);
 extern "C" int ampnet_direct_max_units();
 extern "C" void ampnet_direct_limits(int* max_nodes, int* max_ppts, int* max_landings, int* batch_rows);
 extern "C" cudaError_t ampnet_direct_static_smem(size_t* bytes);
@@ -61,6 +63,7 @@ struct HostPPT {
   bool a_global = false;                // the tiles' gradient accumulators live in device memory (frees shared memory for staging rows)
   int xwt_rb = 8;                       // output rows per pass of X.W^T: 16 where the larger scratch still fits
   int TB = 0, CB = 0, NS = 1;           // direct-delivery engine: backward column tiles, columns per tile, gradient slots per key
+  int tc = 0;                           // direct-delivery engine: forward tiles of 64 rows on the tensor cores (bf16 runs)
   size_t bwd_smem_floats = 0;
   double emit_load = 0.0;               // emitter-seconds the node's emission took in the last asynchronous epoch (0: unknown)
   size_t smem_floats = 0;
@@ -619,6 +622,11 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   int lim_nodes = 0, lim_ppts = 0, lim_landings = 0, BATCH = MAX_BATCH_ROWS;
   ampnet_direct_limits(&lim_nodes, &lim_ppts, &lim_landings, &BATCH);
   std::vector<int> fixed(np, 0);
+  std::vector<char> fixed_rows(np, 0);
+  int tc_rows = 64, tc_bm = 64, tc_k = 16;
+  ampnet_direct_tc_limits(&tc_rows, &tc_bm, &tc_k);
+  bool use_tc = true;
+  if (const char* e = getenv("AMPNET_TENSOR_CORES")) use_tc = atoi(e) != 0;
   // gradient slots: the backward sum of a Bcast forms in the gradient buffer of the node behind Phi / Cond / Isu
   for (auto& P : g->ppts) P.NS = 1;
   for (int i = 0; i < (int)g->hnodes.size(); i++) {
@@ -638,33 +646,38 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
     const DevNode& h = g->hnodes[P.node];
-    P.NE = 0; P.G = 1; P.a_global = false; P.J = 0; P.TB = 0; P.CB = 0; P.bwd_smem_floats = 0;
+    P.NE = 0; P.G = 1; P.a_global = false; P.J = 0; P.TB = 0; P.CB = 0; P.bwd_smem_floats = 0; P.tc = 0;
     if (P.kind == LOOKUP) { P.T = (P.in >= 4096 && tile_budget >= 24) ? 4 : 1; P.R = 0; P.BM = BATCH; fixed[p] = 1; continue; }
     const int st = g->hnodes[h.succ_node[0]].type;
     P.BM = BATCH;
     if (st == LOSS_CE || st == LOSS_MSE) { P.R = P.out; fixed[p] = 1; }
     else {
       P.R = std::min(P.out, rows);
+      // bf16 runs: a node whose shape fits the instruction (rows in whole tiles of 64, input width a multiple of 16) runs its
+      // forward products on the tensor cores (AMPNET_TENSOR_CORES=0 keeps them on the FMA units)
+      if (g->payload_bf16 && use_tc && P.kind == LINEAR && P.out % tc_rows == 0 && P.in % tc_k == 0) { P.tc = 1; P.R = tc_rows; P.BM = std::min(P.BM, tc_bm); fixed_rows[p] = 1; }
       P.CB = cols;
       while (P.CB > 4 && (long long)P.out * (P.CB / 4) > max_units) P.CB /= 2;
       if ((long long)P.out * (P.CB / 4) > max_units) return direct_overflow(1);        // accumulators of a column tile exceed the registers
     }
   }
   auto fits = [&](const HostPPT& P) {
-    return ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM, P.CB == 0) <= budget && (P.CB == 0 || ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) <= budget);
+    const size_t fwd = P.tc ? ampnet_direct_tc_tile_smem_bytes(P.in, P.BM) : ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM, P.CB == 0);
+    return fwd <= budget && (P.CB == 0 || ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) <= budget);
   };
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
     if (P.kind == LOOKUP) continue;
     while (!fits(P)) {
       if (P.BM > 16) P.BM /= 2;
+      else if (P.tc) { P.tc = 0; fixed_rows[p] = 0; P.R = std::min(P.out, rows); P.BM = BATCH; }       // the weights alone do not fit as one 64-row tile
       else if (!fixed[p] && P.R > 1) { P.R = (P.R + 1) / 2; P.BM = BATCH; }
       else return direct_overflow(2);
     }
   }
   // over the budget: grow the tiles of whichever node has the most tiles of a kind that can still grow (rows per forward
   // tile while its weights and a few staged rows still fit; columns per backward tile while the accumulators fit the registers)
-  std::vector<char> rows_stuck(np, 0);
+  std::vector<char> rows_stuck(fixed_rows);
   for (;;) {
     int used = 0, best = -1, best_n = 0; bool best_cols = false;
     for (int p = 0; p < np; p++) {
@@ -688,7 +701,7 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   roles.push_back(Role{-1, 0, 0, 0});
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
-    P.smem_floats = P.kind == LOOKUP ? 64 : ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM, P.CB == 0) / sizeof(float);
+    P.smem_floats = P.kind == LOOKUP ? 64 : (P.tc ? ampnet_direct_tc_tile_smem_bytes(P.in, P.BM) : ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM, P.CB == 0)) / sizeof(float);
     P.bwd_smem_floats = P.TB ? ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) / sizeof(float) : 0;
     for (int t = 0; t < P.T; t++) roles.push_back(Role{p, t, 0, 0});
     for (int t = 0; t < P.TB; t++) roles.push_back(Role{p, t, 3, 0});
@@ -768,7 +781,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
       if (P.xld != P.in_dim && !dry) g->zero_regions.push_back({P.xcache, keys * P.rows_max * P.xld * sizeof(float)});   // the row padding
     }
     if (H.kind != LOOKUP) P.ycache = B.take<float>(keys * P.rows_max * P.out_dim);
-    P.NS = R.direct ? H.NS : 1; P.TB = H.TB; P.CB = H.CB; P.bwd_smem_floats = (int)H.bwd_smem_floats;
+    P.NS = R.direct ? H.NS : 1; P.tc = R.direct ? H.tc : 0; P.TB = H.TB; P.CB = H.CB; P.bwd_smem_floats = (int)H.bwd_smem_floats;
     P.gbuf = B.take<float>(keys * P.rows_max * P.out_dim * P.NS);
     if (R.direct) {                  // one gradient slot per contributor: nothing is added in memory, nothing cleared
       for (int d = 0; d < 2; d++) { P.injoin[d] = C.take<int>(keys); track(P.injoin[d], keys * sizeof(int)); }
@@ -1027,7 +1040,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.ppts, R.ppts.data(), R.ppts.size() * sizeof(DevPPT), cudaMemcpyHostToDevice, g->stream));
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.roles, R.roles.data(), R.roles.size() * sizeof(Role), cudaMemcpyHostToDevice, g->stream));
   if (dbg) fprintf(stderr, "[ampnet] %s engine, %d CTAs, %zu B smem, ctl %zu B, bulk %zu B\n", R.direct ? "direct-delivery" : "interpreter", R.ctx.n_ctas, R.smem_bytes, g->ctl.used, g->bulk.used);
-  if (dbg) for (auto& P : g->ppts) fprintf(stderr, "[ampnet]   node %d: %d tiles x %d rows, %d backward tiles x %d columns, batch %d, slots %d\n", P.node, P.T, P.R, P.TB, P.CB, P.BM, P.NS);
+  if (dbg) for (auto& P : g->ppts) fprintf(stderr, "[ampnet]   node %d: %d tiles x %d rows%s, %d backward tiles x %d columns, batch %d, slots %d\n", P.node, P.T, P.R, P.tc ? " (tensor cores)" : "", P.TB, P.CB, P.BM, P.NS);
   if (R.direct) {
     CUDA_TRY(g, cudaEventRecord(g->ev0, g->stream));
     const cudaError_t le = ampnet_direct_launch(&R.ctx, R.ctx.n_ctas, R.smem_bytes, g->stream, g->n_sms);
@@ -1557,6 +1570,16 @@ ampnet_status_t ampnet_get_queue_occupancy(ampnet_graph_t* g, int32_t node, int6
   const PPTStats& s = g->last_stats[g->hnodes[node].ppt];
   if (max_pending_fwd) *max_pending_fwd = (int64_t)s.max_pending[0];
   if (max_pending_bwd) *max_pending_bwd = (int64_t)s.max_pending[1];
+  return AMPNET_OK;
+}
+
+ampnet_status_t ampnet_get_micro_batch_split(ampnet_graph_t* g, int32_t node, int64_t* fma_batches, int64_t* tensor_core_batches) {
+  if (!g) return AMPNET_EINVAL;
+  if (!g->have_run) return set_err(g, AMPNET_ESTATE, "no run yet");
+  if (node < 0 || node >= (int)g->hnodes.size() || g->hnodes[node].ppt < 0) return set_err(g, AMPNET_EINVAL, "not a parameterised node");
+  const PPTStats& s = g->last_stats[g->hnodes[node].ppt];
+  if (fma_batches) *fma_batches = (int64_t)(s.batches - s.tc_batches);
+  if (tensor_core_batches) *tensor_core_batches = (int64_t)s.tc_batches;
   return AMPNET_OK;
 }
 

@@ -20,6 +20,7 @@
 #include <cuda_runtime.h>
 
 #include "engine_types.h"
+#include "tc_tile.cuh"
 
 namespace ampf {
 using namespace amp;
@@ -359,6 +360,10 @@ struct TileS {
   unsigned long long mbar;
   unsigned mbar_parity;
   unsigned wver_seen;               // forward tile: the node's published-columns counter as last polled
+  // tensor-core forward tile: address of its tensor-memory columns, the mbarrier its products are committed to (and the
+  // parity to wait for next), micro-batches run this way
+  unsigned tmem, tc_parity;
+  unsigned long long tc_mbar, tc_batches;
 };
 
 __host__ __device__ __forceinline__ int pad4(int v) { return (v + 3) & ~3; }
@@ -695,11 +700,23 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   // publish their columns and the row tiles reload their rows before their next batch.
   const bool fwd_only = !lookup && !fused;
   const int dirs = fwd_only ? 1 : 3;
-  float *Ws = smem, *bs = Ws + (size_t)P.R * LW, *Abs = bs + RP, *Xs = Abs + RP, *Ys = Xs + (size_t)P.BM * LX, *Ds = Ys + (size_t)P.BM * RP,
+  // A tensor-core tile (bf16 runs, 64 rows, in_dim a multiple of 16) keeps its rows and the staged batch as bfloat16 in
+  // the operand layout of the tensor cores; the master weights stay fp32 in the column tiles and in device memory.
+  const bool tcm = fwd_only && P.tc;
+  const int NT = (P.BM + 15) & ~15;                          // accumulator columns of a tensor-core product
+  const size_t ws_floats = tcm ? (size_t)tc::M * in / 2 : (size_t)P.R * LW, xs_floats = tcm ? (size_t)NT * in / 2 : (size_t)P.BM * LX;
+  float *Ws = smem, *bs = Ws + ws_floats, *Abs = bs + RP, *Xs = Abs + RP, *Ys = Xs + xs_floats, *Ds = Ys + (size_t)P.BM * RP,
         *As = Ds + (fused ? (size_t)P.BM * RP : 0), *Wt = As + (fused ? (size_t)P.R * LW : 0), *Dx = Xs,
         *smem_end = Wt + (fused ? (size_t)in * RP : 0);      // gradients, accumulators, transposed weights: loss head only; its input
                                                              // gradients take the place of the staged rows once those are used up
-  if (!lookup) {
+  unsigned char *const Wb = reinterpret_cast<unsigned char*>(Ws), *const Xb = reinterpret_cast<unsigned char*>(Xs);
+  if (tcm) {
+    for (float* q = smem + tid; q < smem_end; q += FT) *q = 0.f;
+    __syncthreads();
+    tc::fill_operand(Wb, R, in, [&](const int r) { return P.W + (size_t)(r_begin + r) * in; }, tid, FT);
+    for (int i = tid; i < R; i += FT) bs[i] = P.b[r_begin + i];
+    tc::fence_operands();
+  } else if (!lookup) {
     for (float* q = smem + tid; q < smem_end; q += FT) *q = 0.f;
     __syncthreads();
     for (int i = tid; i < R * in; i += FT) { const int r = i / in, c = i - r * in; Ws[r * LW + c] = P.W[(size_t)r_begin * in + i]; }
@@ -714,13 +731,15 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
     asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&S.mbar)) : "memory");
     S.mbar_parity = 0;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" :: "r"(smem_u32(&S.tc_mbar)) : "memory");
+    S.tc_parity = 0; S.tc_batches = 0;
   }
   if (tid < 64) S.stale_hist[tid] = 0;
   if (tid < 16) S.phase[tid] = 0;
   __syncthreads();
   long long tph = clock64();
   const FastDiv dR(max(R, 1)), dIn(in);
-  const bool bulk_ok = !lookup && (P.xcache != nullptr || ((in & 3) == 0 && (C.inst.dense_dim & 3) == 0));
+  const bool bulk_ok = !tcm && !lookup && (P.xcache != nullptr || ((in & 3) == 0 && (C.inst.dense_dim & 3) == 0));
   const int xwidth = P.xcache ? P.xld : in;
 
   // Front end of a batch (warps 0-3, 128 threads = one per message): warp 0 takes the batch from the rings, then every
@@ -802,7 +821,14 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     if (!S.ok) break;
     TPHASE(4);
     const int count = S.count, dir = S.dir, flags = S.flags, eval_n = S.eval, n_upd = S.n_upd, upd_t = S.upd_t;
-    if (fwd_only && (int)(S.wver_seen / (unsigned)P.TB) > S.version) {      // every column tile has published a newer version
+    if (tcm && (int)(S.wver_seen / (unsigned)P.TB) > S.version) {
+      tc::fill_operand(Wb, R, in, [&](const int r) { return P.W + (size_t)(r_begin + r) * in; }, tid, FT);
+      for (int i = tid; i < R; i += FT) bs[i] = __ldcg(P.b + r_begin + i);
+      tc::fence_operands();
+      __syncthreads();
+      if (tid == 0) S.version = (int)(S.wver_seen / (unsigned)P.TB);
+      TPHASE(3);
+    } else if (fwd_only && (int)(S.wver_seen / (unsigned)P.TB) > S.version) {      // every column tile has published a newer version
       for (int i = tid; i < R * in; i += FT) { const int r = dIn.div(i), c = i - r * in; Ws[r * LW + c] = __ldcg(P.W + (size_t)r_begin * in + i); }
       for (int i = tid; i < R; i += FT) bs[i] = __ldcg(P.b + r_begin + i);
       __syncthreads();
@@ -827,7 +853,11 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         __syncthreads();
         if (tid == 0) S.mbar_parity ^= 1u;
       }
-      if (!lookup && !bulk_ok) {
+      if (tcm) {                                              // the batch as the second operand: fp32 rows from the cache, stored as bfloat16
+        tc::fill_operand(Xb, count, in, [&](const int b) { return S.rowptr[b]; }, tid, FT);
+        tc::fence_operands();
+        __syncthreads();
+      } else if (!lookup && !bulk_ok) {
         for (int idx = tid; idx < count * in; idx += FT) { const int b = dIn.div(idx), c = idx - b * in; Xs[b * LX + c] = __ldcg(S.rowptr[b] + c); }
         __syncthreads();
       }
@@ -961,8 +991,30 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
       }
     } else if (count > 0 && !lookup) {
       if (dir == FWD) {
-        gemm_nt(Xs, LX, count, Ws, LW, R, pad4(in) >> 2, Ys, RP);
-        __syncthreads();
+        if (tcm) {
+          // Y^T = W X^T on the tensor cores: one thread issues in_dim / 16 instructions, everybody waits for the commit
+          // (bounded like every wait here), warps 0-3 move the accumulator from tensor memory to Ys[message][row].
+          const unsigned bar = smem_u32(&S.tc_mbar), parity = S.tc_parity;
+          if (tid == 0) { tc::issue(S.tmem, Wb, Xb, in, NT, bar); S.tc_batches++; }
+          unsigned done = 0, spins = 0;
+          for (;;) {
+            asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+            if (done) break;
+            if ((++spins & 1023u) == 0 && (aborted(C) || gtime() - t0 > C.timeout_ns)) {
+              if (tid == 0) { fail(C, ST_TIMEOUT, P.node, 8); S.ok = 0; }
+              for (unsigned extra = 0; extra < (1u << 16) && !done; extra++)        // instructions already issued still write the accumulator
+                asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}" : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+              break;
+            }
+          }
+          if (__all_sync(0xffffffffu, done != 0)) tc::read_accumulator(S.tmem, NT, count, Ys, RP, R);
+          __syncthreads();
+          if (tid == 0) S.tc_parity ^= 1u;
+          if (!S.ok) break;
+        } else {
+          gemm_nt(Xs, LX, count, Ws, LW, R, pad4(in) >> 2, Ys, RP);
+          __syncthreads();
+        }
         TPHASE(5);
         for (int idx = tid; idx < count * R; idx += FT) {
           const int b = dR.div(idx), r = idx - b * R;
@@ -1088,6 +1140,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
       PPTStats& st = *P.stats;
       if (!fwd_only) { st.max_staleness = S.max_stale; st.log_n = S.log_n; st.n_updates = S.n_updates; st.n_grads_applied = S.n_grads_applied; }
       atomicAdd(&st.msgs, S.msgs); atomicAdd(&st.batches, S.batches); atomicAdd(&st.batch_rows, S.batch_rows);
+      st.tc_batches = tcm ? S.tc_batches : 0;
       st.max_pending[0] = S.qmax[0];
       if (!fwd_only) st.max_pending[1] = S.qmax[1];
     }
@@ -1519,7 +1572,23 @@ __global__ void __launch_bounds__(ampf::FT, 1) ampnet_engine_direct(const __grid
   const Role role = C.roles[blockIdx.x];
   if (role.ppt < 0) controller_main(C, SU.c, t0);
   else if (role.kind == 3) bwd_tile_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
-  else tile_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
+  else {
+    // a tensor-core tile holds tensor-memory columns for its accumulator for the whole run; every way out of
+    // tile_main comes back here, so they are always given back
+    const bool tcm = g_ppts[role.ppt].tc != 0 && g_ppts[role.ppt].kind == LINEAR;
+    if (tcm) {
+      if (threadIdx.x < 32) tc::tmem_alloc(&SU.t.tmem);
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncthreads();
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    }
+    tile_main(C, g_ppts[role.ppt], role.tile, dyn_smem, SU.t, t0);
+    if (tcm) {
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncthreads();
+      if (threadIdx.x < 32) tc::tmem_free(SU.t.tmem);
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1542,6 +1611,12 @@ extern "C" int ampnet_direct_threads() { return ampf::FT; }
 extern "C" void ampnet_direct_limits(int* max_nodes, int* max_ppts, int* max_landings, int* batch_rows) {
   *max_nodes = ampf::DIRECT_MAX_NODES; *max_ppts = ampf::DIRECT_MAX_PPTS; *max_landings = ampf::MAXD; *batch_rows = ampf::FBM;
 }
+// shared memory of a tensor-core forward tile: 64 rows and the batch (rounded up to 16 messages) as bfloat16, bias, outputs
+extern "C" size_t ampnet_direct_tc_tile_smem_bytes(int in_dim, int batch_rows) {
+  const size_t RP = ampf::pad_ldx(tc::M), NT = (size_t)((batch_rows + 15) & ~15);
+  return (size_t)tc::M * in_dim * 2 + 2 * RP * sizeof(float) + NT * in_dim * 2 + (size_t)batch_rows * RP * sizeof(float) + 64;
+}
+extern "C" void ampnet_direct_tc_limits(int* rows, int* max_batch_rows, int* k_multiple) { *rows = tc::M; *max_batch_rows = tc::TMEM_COLS; *k_multiple = 16; }
 extern "C" size_t ampnet_direct_tile_smem_bytes(int in_dim, int rows, int batch_rows, int loss_head) {
   return ampf::tile_smem_floats(in_dim, rows, batch_rows, loss_head) * sizeof(float) + 64;
 }

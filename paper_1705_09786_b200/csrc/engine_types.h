@@ -55,6 +55,7 @@ struct PPTStats {
   int max_staleness, log_n;
   unsigned long long phase_cycles[16];  // leader tile: idle, fetch, headers, compute, update, barrier, emit, loop; [8..] emission detail
   unsigned max_pending[2];              // direct-delivery engine: most messages waiting in the forward / backward ring when a batch was taken
+  unsigned long long tc_batches;        // micro-batches (of those counted in `batches`) whose product ran on the tensor cores
 };
 
 struct DevNode {
@@ -77,7 +78,8 @@ struct DevNode {
 };
 
 struct DevPPT {
-  int node, kind, in_dim, out_dim, act, flags, muf_override, pad0;
+  int node, kind, in_dim, out_dim, act, flags, muf_override;
+  int tc;                             // direct-delivery engine: the forward row tiles (64 rows each) run their products on the tensor cores
   int T, cta0, R, BM;                 // row tiles, first CTA, rows per tile, batch row capacity
   int U, rows_max, J, xld;            // key space, max rows per message, ceil(in_dim / 32) bucket, row stride of xcache (in_dim
                                       // rounded up to 4 floats, padding kept at zero: rows start on 16 bytes for bulk copies)
