@@ -209,6 +209,25 @@ def input_bytes(inst):
                    if a is not None))
 
 
+def split_counts(eng, graph):
+    """Micro-batches of the last run by the unit that ran their product, counted on the device (first forward and first
+    backward tile of every node)."""
+    fma = tensor = 0
+    for n in graph.ppt_nodes():
+        f, t = eng.micro_batch_split(n)
+        fma += f
+        tensor += t
+    return {"micro_batches_fma": int(fma), "micro_batches_tensor_core": int(tensor)}
+
+
+def micro_batch_split(eng, graph):
+    c = split_counts(eng, graph)
+    total = max(1, c["micro_batches_fma"] + c["micro_batches_tensor_core"])
+    return {"fma": c["micro_batches_fma"] / total, "tensor_core": c["micro_batches_tensor_core"] / total, **c,
+            "note": "tensor cores (tcgen05, bf16 operands, fp32 accumulation) run the forward products of nodes with out_dim % 64 == 0 "
+                    "and in_dim % 16 == 0 in bf16 runs (the stress configuration's cells); everything else runs on FP32 FMA"}
+
+
 def average_replicas(views, averaging, average_fn=None):
     """End-of-epoch replica synchronisation (Sec. 5) inside the timed region.  If the collective cannot run the ranks
     continue as independent replicas and `averaging` (reported as config.replica_sync) says so."""
@@ -303,6 +322,7 @@ def run_ours(args):
     updates = {n: eng.node_stats(n)["n_updates"] for n in graph.ppt_nodes()}     # of the last timed step
     placement = {graph.names[n]: eng.placement(n) for n in graph.ppt_nodes()}
     queue_occ = {graph.names[n]: list(eng.queue_occupancy(n)) for n in graph.ppt_nodes()}
+    split = micro_batch_split(eng, graph)
     secs = sum(step_s)
     value, tmax = aggregate(inst.n * args.steps, secs, dev)
     msg_rate, _ = aggregate(msgs, secs, dev)
@@ -361,6 +381,8 @@ def run_ours(args):
                     e2.set_params(wp.init_params(g2))
             fl = rf.algorithmic_flops(g2, inst2, {n: e2.node_stats(n)["n_updates"] for n in g2.ppt_nodes()})
             occ2 = {g2.names[n]: list(e2.queue_occupancy(n)) for n in g2.ppt_nodes()}
+            split2 = micro_batch_split(e2, g2)
+            split2.pop("note")
             r1, m1 = one_key_rate(e2, inst2, cfg2, args.timeout)
             peaks2, kind2 = measured_peaks()
             others[name] = {"instances_per_s": 2 * inst2.n / sum(ks), "node_messages_per_s": ms / sum(ks),
@@ -370,7 +392,7 @@ def run_ours(args):
                             "timing": "device time of the persistent kernel (CUDA events around the launch), parameters reset before every epoch",
                             "roofline": roofline_object(rf, g2, inst2, name, fl, sum(ks) / 2, fma_measured, peaks2, kind2,
                                                         cfg2["mak"], r1, m1),
-                            "queue_occupancy_max_pending_fwd_bwd": occ2}
+                            "queue_occupancy_max_pending_fwd_bwd": occ2, "micro_batch_split": split2}
             if not args.no_cpu_baseline:
                 r = time_oracle(g2, inst2, cfg2, target_s=4.0, probe=16)
                 others[name]["cpu_baseline"] = dict({"value": r["inst_per_s"], "unit": "instances/s", "cores": 1, "kind": "oracle",
@@ -394,7 +416,7 @@ def run_ours(args):
                               "rows_per_micro_batch": st.micro_batch_rows / max(1, st.micro_batches),
                               "max_active_observed": int(st.max_active_observed), "max_staleness": int(st.max_staleness),
                               "queue_occupancy_max_pending_fwd_bwd": {graph.names[n]: list(eng.queue_occupancy(n)) for n in graph.ppt_nodes()},
-                              "micro_batches_fma": int(st.micro_batches), "micro_batches_tensor_core": 0})
+                              **split_counts(eng, graph)})
         eng.load_instances(inst)
     if rank == 0:
         peaks, peak_kind = measured_peaks()
@@ -428,8 +450,7 @@ def run_ours(args):
                           "rows_per_micro_batch": last.micro_batch_rows / max(1, last.micro_batches),
                           "placement": placement, "inference_instances_per_s": inference_rate,
                           "queue_occupancy_max_pending_fwd_bwd": queue_occ,
-                          "micro_batch_split": {"fma": 1.0, "tensor_core": 0.0,
-                                                "note": "every micro-batch runs on FP32 FMA: this build has no tensor-core path"}}}
+                          "micro_batch_split": split}}
         if sweep is not None:
             line["sweep"] = sweep
         if others is not None:

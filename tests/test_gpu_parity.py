@@ -401,6 +401,38 @@ def test_asynchronous_epoch_without_updates_matches_oracle(oracle_mod, monkeypat
     e.close()
 
 
+@pytest.mark.parametrize("tensor_cores", [1, 0])
+def test_stress_shape_without_updates_matches_oracle_on_tensor_cores_and_on_fma(oracle_mod, monkeypatch, tensor_cores):
+    """The asynchronous path of the stress configuration (hidden 512, bf16 messages) element by element against the oracle,
+    where the schedule cannot matter (no update before the flush at the end of the epoch): once with the forward products of
+    the two cells on the tensor cores (W and the micro-batch as bfloat16 operands, fp32 accumulation; the oracle keeps W in
+    fp32, which the bf16 tolerances cover) and once with every product on the FMA units.  The split counters must say which
+    of the two ran."""
+    import paper_1705_09786_b200 as amp
+    from test_oracle_pins import BF16_TOL
+    monkeypatch.setenv("AMPNET_TENSOR_CORES", str(tensor_cores))
+    g, inst = _stress_case(4, 64, 200)
+    p = wp.init_params(g)
+    o = oracle_mod.Oracle(g, payload_bf16=True)
+    o.load_instances(inst)
+    o.set_params(p)
+    _, oloss = o.run_epoch(mak=1, muf=1 << 30, lr=0.05)
+    e = amp.Engine(g, payload_bf16=True)
+    e.load_instances(inst)
+    e.set_params(p)
+    st, eloss = e.run_epoch(mak=64, muf=1 << 30, lr=0.05, deterministic=False, timeout_s=120)
+    np.testing.assert_allclose(eloss, oloss, rtol=BF16_TOL["loss_rtol"], atol=BF16_TOL["loss_atol"])
+    ep, op = e.get_params(), o.get_params()
+    for k in op:
+        scale = max(np.abs(op[k]).max(), BF16_TOL["param_floor"])
+        assert np.abs(ep[k] - op[k]).max() / scale <= BF16_TOL["param_rtol"], (g.names[k[0]], k[1])
+    for name in ("leaf_cell", "branch_cell"):
+        fma, tensor = e.micro_batch_split(g.index(name))
+        assert (tensor > 0) == bool(tensor_cores) and fma > 0          # the backward batches stay on the FMA units
+    assert e.micro_batch_split(g.index("classifier"))[1] == 0 and e.micro_batch_split(g.index("lookup"))[1] == 0
+    e.close()
+
+
 def test_tree_with_256_keys_in_flight(oracle_mod):
     """The tree workload with more keys than the benchmark uses (every instance of the set in flight at once)."""
     g, inst = _case("tree", 300)
