@@ -64,6 +64,7 @@ struct HostPPT {
   int xwt_rb = 8;                       // output rows per pass of X.W^T: 16 where the larger scratch still fits
   int TB = 0, CB = 0, NS = 1;           // direct-delivery engine: backward column tiles, columns per tile, gradient slots per key
   int tc = 0;                           // direct-delivery engine: forward tiles of 64 rows on the tensor cores (bf16 runs)
+  int LT = 1;                           // direct-delivery engine: tiles that share the messages of a node that feeds a Loss
   size_t bwd_smem_floats = 0;
   double emit_load = 0.0;               // emitter-seconds the node's emission took in the last asynchronous epoch (0: unknown)
   size_t smem_floats = 0;
@@ -435,6 +436,7 @@ ampnet_status_t place(ampnet_graph* g, int n_ctas, int max_batch_rows, std::vect
   int max_tiles = 16;      // default; a node whose tile does not fit in shared memory gets more, up to MAX_TILES
   if (const char* e = getenv("AMPNET_MAX_TILES")) max_tiles = std::max(1, std::min(MAX_TILES, atoi(e)));
   const int np = (int)g->ppts.size();
+  for (auto& P : g->ppts) { P.LT = 1; P.tc = 0; }                // (choices of the direct-delivery engine)
   const int tile_budget = emitters > 0 ? (n_ctas - 1 - np) / (1 + emitters) : n_ctas - 1;
   std::vector<int> limit(np, 1), bm_of(np, 0);
   std::vector<double> work(np, 0.0);
@@ -646,7 +648,7 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
     const DevNode& h = g->hnodes[P.node];
-    P.NE = 0; P.G = 1; P.a_global = false; P.J = 0; P.TB = 0; P.CB = 0; P.bwd_smem_floats = 0; P.tc = 0;
+    P.NE = 0; P.G = 1; P.a_global = false; P.J = 0; P.TB = 0; P.CB = 0; P.bwd_smem_floats = 0; P.tc = 0; P.LT = 1;
     if (P.kind == LOOKUP) { P.T = (P.in >= 4096 && tile_budget >= 24) ? 4 : 1; P.R = 0; P.BM = BATCH; fixed[p] = 1; continue; }
     const int st = g->hnodes[h.succ_node[0]].type;
     P.BM = BATCH;
@@ -697,13 +699,25 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
     while (!fits(P) && P.BM > 8) P.BM /= 2;
     if (!fits(P)) { P.R = r0; P.BM = bm0; rows_stuck[best] = 1; }
   }
+  // CTAs left over go to the loss heads: their tiles share the node's messages (every tree node, every list, passes
+  // through that one node) and meet at its updates
+  {
+    int used = 0, heads = 0, want = 4;
+    if (const char* e = getenv("AMPNET_LOSS_TILES")) want = std::max(1, std::min(16, atoi(e)));
+    for (int p = 0; p < np; p++) { used += g->ppts[p].T + g->ppts[p].TB; heads += fixed[p] && g->ppts[p].kind != LOOKUP; }
+    for (int p = 0; p < np && heads > 0; p++) {
+      HostPPT& P = g->ppts[p];
+      if (!fixed[p] || P.kind == LOOKUP) continue;
+      P.LT = std::max(1, std::min(want, 1 + (tile_budget - used) / heads));
+    }
+  }
   roles.clear();
   roles.push_back(Role{-1, 0, 0, 0});
   for (int p = 0; p < np; p++) {
     HostPPT& P = g->ppts[p];
     P.smem_floats = P.kind == LOOKUP ? 64 : (P.tc ? ampnet_direct_tc_tile_smem_bytes(P.in, P.BM) : ampnet_direct_tile_smem_bytes(P.in, P.R, P.BM, P.CB == 0)) / sizeof(float);
     P.bwd_smem_floats = P.TB ? ampnet_direct_bwd_tile_smem_bytes(P.out, P.CB, P.BM) / sizeof(float) : 0;
-    for (int t = 0; t < P.T; t++) roles.push_back(Role{p, t, 0, 0});
+    for (int t = 0; t < (P.LT > 1 ? P.LT : P.T); t++) roles.push_back(Role{p, t, 0, 0});
     for (int t = 0; t < P.TB; t++) roles.push_back(Role{p, t, 3, 0});
   }
   return AMPNET_OK;
@@ -786,7 +800,14 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
     if (R.direct) {                  // one gradient slot per contributor: nothing is added in memory, nothing cleared
       for (int d = 0; d < 2; d++) { P.injoin[d] = C.take<int>(keys); track(P.injoin[d], keys * sizeof(int)); }
       P.wver = C.take<unsigned>(1);
-    }
+      P.LT = H.LT;
+      if (H.LT > 1) {
+        const size_t PS = (size_t)H.out * H.in + H.out;
+        P.lh_count = C.take<int>(1);
+        P.lh_part = B.take<float>(2 * (size_t)H.LT * PS);
+        P.lh_mom = B.take<float>(2 * (size_t)(H.LT - 1) * PS);
+      }
+    } else P.LT = 1;
     if (H.kind == GRUCELL) {
       P.zc = B.take<float>(keys * P.rows_max * P.out_dim);
       P.rc = B.take<float>(keys * P.rows_max * P.out_dim);
@@ -1040,7 +1061,7 @@ ampnet_status_t execute(ampnet_graph* g, int split, int mak, int det, int eval, 
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.ppts, R.ppts.data(), R.ppts.size() * sizeof(DevPPT), cudaMemcpyHostToDevice, g->stream));
   CUDA_TRY(g, cudaMemcpyAsync(R.ctx.roles, R.roles.data(), R.roles.size() * sizeof(Role), cudaMemcpyHostToDevice, g->stream));
   if (dbg) fprintf(stderr, "[ampnet] %s engine, %d CTAs, %zu B smem, ctl %zu B, bulk %zu B\n", R.direct ? "direct-delivery" : "interpreter", R.ctx.n_ctas, R.smem_bytes, g->ctl.used, g->bulk.used);
-  if (dbg) for (auto& P : g->ppts) fprintf(stderr, "[ampnet]   node %d: %d tiles x %d rows%s, %d backward tiles x %d columns, batch %d, slots %d\n", P.node, P.T, P.R, P.tc ? " (tensor cores)" : "", P.TB, P.CB, P.BM, P.NS);
+  if (dbg) for (auto& P : g->ppts) fprintf(stderr, "[ampnet]   node %d: %d tiles x %d rows%s, %d backward tiles x %d columns, batch %d, slots %d\n", P.node, P.LT > 1 ? P.LT : P.T, P.R, P.tc ? " (tensor cores)" : P.LT > 1 ? " (shared loss head)" : "", P.TB, P.CB, P.BM, P.NS);
   if (R.direct) {
     CUDA_TRY(g, cudaEventRecord(g->ev0, g->stream));
     const cudaError_t le = ampnet_direct_launch(&R.ctx, R.ctx.n_ctas, R.smem_bytes, g->stream, g->n_sms);
@@ -1586,7 +1607,7 @@ ampnet_status_t ampnet_get_micro_batch_split(ampnet_graph_t* g, int32_t node, in
 ampnet_status_t ampnet_get_placement(ampnet_graph_t* g, int32_t node, int32_t* n_tiles, int32_t* batch_rows) {
   HostPPT* P = find_ppt(g, node);
   if (!P) return g ? set_err(g, AMPNET_EINVAL, "not a parameterised node") : AMPNET_EINVAL;
-  if (n_tiles) *n_tiles = P->T;
+  if (n_tiles) *n_tiles = P->LT > 1 ? P->LT : P->T;
   if (batch_rows) *batch_rows = P->BM;
   return AMPNET_OK;
 }

@@ -651,6 +651,99 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
   return 1;
 }
 
+// Loss head shared by LT tiles: tile t takes the tickets t, t + LT, t + 2 LT, ... of the node's forward ring (a message is
+// handled by exactly one tile), so S.head[FWD] counts own tickets.  Every ticket is one gradient (no forward-only message
+// travels in such a run), so update number k falls due exactly when the tickets below k x muf have been handled (Sec. 3);
+// a tile that has handled its own takes part in the exchange of the partial sums as soon as that ticket has been handed
+// out, or, at the end of the epoch, in the flush of what is left.  Returns like form_batch; a batch may be empty
+// (update only).
+__device__ __noinline__ int form_batch_split(const Ctx& C, DevPPT& P, TileS& S, const bool leader, const int LT, const int t, const bool light) {
+  IN_SMEM(&P); IN_SMEM(&S);
+  const int lane = threadIdx.x & 31;
+  const Ring& rg = P.ring[FWD];
+  const bool training = !C.eval;
+  const unsigned k0 = S.head[FWD], own_next = k0 * (unsigned)LT + (unsigned)t;
+  const unsigned muf = (unsigned)node_muf(C, P);
+  const unsigned long long done_grads = S.n_updates * (unsigned long long)muf, bnd = done_grads + muf;     // tickets below bnd belong to the next update
+  unsigned probe = 0;
+  if (lane == 0) probe = ld_rlx(rg.tail);
+  if (lane == 1) probe = ld_rlx(&rg.seq[own_next & rg.mask]) == own_next + 1u;
+  if (lane == 2) probe = ld_rlx(&C.g->done);
+  const unsigned tail = __shfl_sync(0xffffffffu, probe, 0), head_ready = __shfl_sync(0xffffffffu, probe, 1), fin0 = __shfl_sync(0xffffffffu, probe, 2);
+  const bool at_boundary = training && own_next >= bnd;
+  if (light && !fin0 && !(at_boundary ? tail >= bnd : head_ready != 0)) return 0;
+  if (leader && lane == 0 && tail - own_next < (1u << 30) && tail - own_next > S.qmax[FWD]) S.qmax[FWD] = tail - own_next;
+  auto close_epoch = [&]() {                       // after `done`: the ring's tail is final
+    unsigned fin_tail = 0;
+    if (lane == 0) { fence_acq(); fin_tail = ld_rlx(rg.tail); }
+    fin_tail = __shfl_sync(0xffffffffu, fin_tail, 0);
+    if (lane == 0) {
+      S.count = 0; S.dir = FWD; S.flags = BATCH_TERMINATE; S.n_upd = 0; S.upd_t = 0; S.eval = 0;
+      const long long left = training ? (long long)fin_tail - (long long)done_grads : 0;
+      if (left > 0) {                                          // epoch-end flush of the leftover gradients
+        S.flags |= BATCH_UPDATE; S.n_upd = (int)left; S.upd_t = (int)S.n_updates + 1;
+        if (leader && S.log_n < P.update_log_cap) P.update_log[S.log_n] = S.n_upd;
+        S.log_n++; S.n_updates++; S.n_grads_applied += S.n_upd; S.version++;
+      }
+    }
+    __syncwarp();
+    return 2;
+  };
+  auto count_update = [&]() {                      // lane 0: the update that closes the period
+    S.flags = BATCH_UPDATE; S.n_upd = (int)muf; S.upd_t = (int)S.n_updates + 1;
+    if (leader && S.log_n < P.update_log_cap) P.update_log[S.log_n] = S.n_upd;
+    S.log_n++; S.n_updates++; S.n_grads_applied += S.n_upd; S.version++;
+  };
+  if (at_boundary) {
+    if (tail >= bnd) {
+      if (lane == 0) { S.count = 0; S.dir = FWD; S.eval = 0; count_update(); }
+      __syncwarp();
+      return 1;
+    }
+    unsigned fin = 0;
+    if (lane == 0) fin = ld_acq(&C.g->done);
+    if (!warp_uniform(fin)) return 0;
+    return close_epoch();
+  }
+  constexpr int NPL = FBM / 32;
+  unsigned slot[NPL], m[NPL];
+#pragma unroll
+  for (int j = 0; j < NPL; j++) {
+    const unsigned tk = (k0 + lane + 32 * j) * (unsigned)LT + (unsigned)t;
+    slot[j] = tk & rg.mask;
+    const bool ready = (!training || tk < bnd) && ld_rlx(&rg.seq[slot[j]]) == tk + 1u;
+    m[j] = __ballot_sync(0xffffffffu, ready);
+  }
+  fence_acq();
+  int nready = 0;
+#pragma unroll
+  for (int j = 0; j < NPL; j++) { if (m[j] == 0xffffffffu) nready += 32; else { nready += __ffs((int)~m[j]) - 1; break; } }
+  if (nready == 0) {
+    unsigned fin = 0;
+    if (lane == 0) fin = ld_acq(&C.g->done);
+    if (!warp_uniform(fin)) return 0;
+    return close_epoch();
+  }
+  const int take = min(nready, P.BM);
+#pragma unroll
+  for (int j = 0; j < NPL; j++)
+    if (lane + 32 * j < take) {
+      const int4* e = reinterpret_cast<const int4*>(&rg.e[slot[j]]);
+      const int4 a = __ldcg(e), b = __ldcg(e + 1);
+      S.hdr[S.fpb][lane + 32 * j] = Hdr{a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    }
+  __syncwarp();
+  if (lane == 0) {
+    const int eval0 = (S.hdr[S.fpb][0].flags & HDR_EVAL) != 0;
+    S.count = take; S.dir = FWD; S.flags = 0; S.eval = eval0; S.n_upd = 0; S.upd_t = 0;
+    S.head[FWD] = k0 + (unsigned)take;
+    S.msgs += training ? 2 * take : take; S.batches++; S.batch_rows += take;
+    if (training && (k0 + (unsigned)take) * (unsigned)LT + (unsigned)t >= bnd && tail >= bnd) count_update();   // this tile's last tickets of the period
+  }
+  __syncwarp();
+  return 1;
+}
+
 // ------------------------------------------------------------------------------------------------
 // row tile
 // ------------------------------------------------------------------------------------------------
@@ -685,16 +778,31 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int in = P.in_dim, out = P.out_dim;
   const bool lookup = P.kind == LOOKUP, leader = tile == 0;
-  const int r_begin = tile * P.R;
-  const int R = lookup ? 0 : max(0, min(P.R, out - r_begin));
-  const int LW = pad_ldx(in), LX = pad_ldx(in), RP = pad_ldx(max(P.R, 1)), DXL = LX;
-  const int wgt = tile == P.T - 1 ? JOIN_UNIT - (P.T - 1) * (JOIN_UNIT / P.T) : JOIN_UNIT / P.T;
   const DevNode& N = g_nodes[P.node];
   // A node that feeds a Loss is one tile and runs the whole exchange in one pass: forward, Loss, and the backward message
   // the Loss answers with (which App. A's backward-first rule would take next anyway), so its forward messages count
   // as gradients where the batch is cut.
   const int loss_node = (!lookup && (g_nodes[N.succ_node[0]].type == LOSS_CE || g_nodes[N.succ_node[0]].type == LOSS_MSE)) ? N.succ_node[0] : -1;
   const bool fused = loss_node >= 0;
+  // Several tiles may share a loss head: each takes every LT-th message and owns it whole (all rows, the Loss, the way
+  // back); the partial gradient sums meet at every update.  Runs with forward-only instances among the training ones
+  // (whose messages are no gradients, so tickets do not count them) leave the node to its first tile.
+  const int LT = fused ? max(1, P.LT) : 1;
+  const bool split = LT > 1 && C.inference_only == nullptr;
+  const int r_begin = fused ? 0 : tile * P.R;
+  const int R = lookup ? 0 : max(0, min(P.R, out - r_begin));
+  const int LW = pad_ldx(in), LX = pad_ldx(in), RP = pad_ldx(max(P.R, 1)), DXL = LX;
+  const int wgt = fused ? JOIN_UNIT : tile == P.T - 1 ? JOIN_UNIT - (P.T - 1) * (JOIN_UNIT / P.T) : JOIN_UNIT / P.T;
+  if (fused && LT > 1 && !split && tile > 0) {                 // nothing to do in this run: wait for its end
+    if (tid == 0) {
+      for (unsigned it = 0; !ld_acq(&C.g->done); it++) {
+        if ((it & 63u) == 63u && (aborted(C) || gtime() - t0 > C.timeout_ns)) break;
+        __nanosleep(500);
+      }
+    }
+    __syncthreads();
+    return;
+  }
   // Every other Linear node is split by direction: row tiles (this function) take the forward ring, column tiles
   // (bwd_tile_main) the backward ring.  The column tiles own the master weights and accumulators; after an update they
   // publish their columns and the row tiles reload their rows before their next batch.
@@ -726,6 +834,11 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
       for (int i = tid; i < R * in; i += FT) { const int r = i / in, c = i - r * in; Wt[c * RP + r] = Ws[r * LW + c]; }
     }
   }
+  if (split && tile > 0 && P.om) {                               // private copy of the optimiser moments (all tiles step alike)
+    const size_t PS = (size_t)out * in + out;
+    float* const m = P.lh_mom + (size_t)(tile - 1) * 2 * PS;
+    for (size_t i = tid; i < PS; i += FT) { m[i] = P.om[i]; m[PS + i] = P.ov ? P.ov[i] : 0.f; }
+  }
   if (tid == 0) {
     S.head[0] = S.head[1] = 0; S.n_acc = 0; S.version = 0; S.log_n = 0; S.max_stale = 0; S.ok = 1; S.term = 0; S.arr_done = 0; S.qmax[0] = S.qmax[1] = 0;
     S.n_updates = S.n_grads_applied = S.msgs = S.batches = S.batch_rows = S.node_msgs = 0;
@@ -754,7 +867,8 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
       for (;;) {
         const bool arrivals_pending = false;       // the next batch is taken as soon as the arithmetic of this one is done
         (void)done_when;
-        const int r = form_batch(C, P, S, leader, fused, dirs, it > 0 && !arrivals_pending, 1);
+        const int r = split ? form_batch_split(C, P, S, leader, LT, tile, it > 0)
+                            : form_batch(C, P, S, leader, fused, dirs, it > 0 && !arrivals_pending, 1);
         if (r) break;
         if ((++it & 15u) == 0) {
           unsigned bad = 0;
@@ -794,7 +908,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
           const int id = C.inst.tokens[(long long)h.rows + h.u];
           S.rowid[tid] = (unsigned)id < (unsigned)in ? id : -1;
         }
-        if (leader && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
+        if ((leader || split) && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
         else if (leader && !S.eval && fwd_only) P.vcache[key] = max(S.version, (int)(S.wver_seen / (unsigned)P.TB));   // the version this forward pass uses (Sec. 3: staleness)
         int pre = 0, nd = 0;
         if (fused) {                                   // the label, fetched while the input rows are in flight
@@ -1075,7 +1189,11 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     TPHASE(2);
     // ---- local update (Sec. 3): theta <- theta - lr A / n, accumulator cleared ------------------------------
     if (flags & BATCH_UPDATE) {
-      const OptStep os(C, P, n_upd, upd_t);
+      OptStep os(C, P, n_upd, upd_t);
+      if (split && tile > 0 && P.om) {                       // tiles 1.. of a shared loss head keep their own (identical) moments
+        os.om = P.lh_mom + (size_t)(tile - 1) * 2 * ((size_t)out * in + out);
+        os.ov = os.om + ((size_t)out * in + out);
+      }
       if (lookup) {
         __threadfence();
         int* const tlist = P.touched_list + (size_t)tile * ((in + P.T - 1) / P.T);
@@ -1097,6 +1215,40 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
         if (tid == 0) P.touched_n[tile] = 0;
       } else {
         const size_t nW = (size_t)out * in;
+        if (split) {
+          // The tiles of a shared loss head put their partial sums side by side (two sets of buffers, by update parity: a
+          // tile can be at most one exchange ahead of the slowest), count themselves, wait for the others and add the
+          // partials in tile order, so that every tile applies the same update to its copy of the weights.
+          const size_t PS = nW + (size_t)out;
+          float* const mine = P.lh_part + ((size_t)(upd_t & 1) * LT + tile) * PS;
+          for (int i = tid; i < R * in; i += FT) { const int r = dIn.div(i); mine[i] = As[r * LW + (i - r * in)]; }
+          for (int i = tid; i < R; i += FT) mine[nW + i] = Abs[i];
+          __syncthreads();
+          if (tid == 0) {
+            __threadfence();
+            atom_add_acq_rel(P.lh_count, 1);
+            const unsigned target = (unsigned)LT * (unsigned)upd_t;
+            for (unsigned it = 0; ld_acq(reinterpret_cast<const unsigned*>(P.lh_count)) < target; it++) {
+              if ((it & 63u) == 63u && (aborted(C) || gtime() - t0 > C.timeout_ns)) { fail(C, ST_TIMEOUT, P.node, 9); S.ok = 0; break; }
+              __nanosleep(40);
+            }
+          }
+          __syncthreads();
+          if (!S.ok) break;
+          const float* const all = P.lh_part + (size_t)(upd_t & 1) * LT * PS;
+          for (int i = tid; i < R * in; i += FT) {
+            float a = 0.f;
+            for (int tt = 0; tt < LT; tt++) a += __ldcg(all + tt * PS + i);
+            const int r = dIn.div(i);
+            As[r * LW + (i - r * in)] = a;
+          }
+          for (int i = tid; i < R; i += FT) {
+            float a = 0.f;
+            for (int tt = 0; tt < LT; tt++) a += __ldcg(all + tt * PS + nW + i);
+            Abs[i] = a;
+          }
+          __syncthreads();
+        }
         for (int i = tid; i < R * in; i += FT) { const int r = dIn.div(i), o = r * LW + (i - r * in); os.apply(Ws[o], As[o], (size_t)r_begin * in + i); }
         for (int i = tid; i < R; i += FT) os.apply(bs[i], Abs[i], nW + r_begin + i);
         if (fused) {
@@ -1113,7 +1265,7 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     else if (count > 0) {
       for (int idx = tid - 128; idx < count * MAXD; idx += FT - 128) {
         const int b = idx / MAXD, q = idx - b * MAXD;
-        if (q == 0 && leader && S.pre[pb][b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[pb][b]);
+        if (q == 0 && (leader || split) && S.pre[pb][b]) atomicAdd(&S.node_msgs, (unsigned long long)S.pre[pb][b]);
         if (q == 0 && fused && eval_n) retire_arrive(C, S.hdr[pb][b].slot, JOIN_UNIT);   // a forward-only instance ends at its Losses
         if (q >= S.nd[pb][b]) continue;
         const Hdr& h = S.hdr[pb][b];
@@ -1128,13 +1280,19 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
   }
   // ---- epilogue: parameters back to device memory, statistics ----------------------------------------------
   __syncthreads();
-  if (fused) {
+  if (fused && leader) {
     for (int i = tid; i < R * in; i += FT) { const int r = i / in; P.W[(size_t)r_begin * in + i] = Ws[r * LW + (i - r * in)]; }
     for (int i = tid; i < R; i += FT) P.b[r_begin + i] = bs[i];
   }
   if (tid == 0 && S.node_msgs) atomicAdd(&C.g->node_messages, S.node_msgs);
+  if (split && !leader && tid == 0) {                          // the node's counts are the sums over its tiles
+    PPTStats& st = *P.stats;
+    atomicAdd(&st.stale_hist[0], S.stale_hist[0]);
+    atomicAdd(&st.msgs, S.msgs); atomicAdd(&st.batches, S.batches); atomicAdd(&st.batch_rows, S.batch_rows);
+  }
   if (leader) {
-    if (!fwd_only && tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
+    if (split) { if (tid == 0) atomicAdd(&P.stats->stale_hist[0], S.stale_hist[0]); }
+    else if (!fwd_only && tid < 64) P.stats->stale_hist[tid] = S.stale_hist[tid];
     if (tid < (fwd_only ? 8 : 16)) P.stats->phase_cycles[tid] = S.phase[tid];
     if (tid == 0) {
       PPTStats& st = *P.stats;

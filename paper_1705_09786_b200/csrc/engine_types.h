@@ -116,6 +116,12 @@ struct DevPPT {
   int TB, CB, NS, bwd_smem_floats;    // direct-delivery engine: backward column tiles and input columns per tile; gradient slots per key
                                       // in gbuf ([key][NS][out]: one per successor of the Bcast whose backward sum forms there)
   unsigned* wver;                     // backward tiles that have published their columns, summed over the updates (TB per update)
+  // direct-delivery engine, node that feeds a Loss: LT tiles share its messages (tile t takes the tickets t, t + LT, ... of
+  // the forward ring) and exchange their partial gradient sums at every update: lh_part[2][LT][out * in + out] by update
+  // parity, lh_count = arrivals at the exchanges so far (LT per update), lh_mom = private optimiser moments of tiles 1..LT-1
+  int LT, pad1;
+  int* lh_count;
+  float *lh_part, *lh_mom;
 };
 
 struct DevInst {                      // instances + routing tables produced by the structure encoder
