@@ -1105,7 +1105,13 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
       }
     } else if (count > 0 && !lookup) {
       if (dir == FWD) {
-        if (tcm) {
+        if (tcm && count <= tc::SMALL_ROWS) {
+          // a handful of messages is no dense contraction: FMA units, same bfloat16 operands
+          for (int i = tid; i < count * RP; i += FT) Ys[i] = 0.f;
+          __syncthreads();
+          tc::small_product(Wb, Xb, in, count, Ys, RP, tid);
+          __syncthreads();
+        } else if (tcm) {
           // Y^T = W X^T on the tensor cores: one thread issues in_dim / 16 instructions, everybody waits for the commit
           // (bounded like every wait here), warps 0-3 move the accumulator from tensor memory to Ys[message][row].
           const unsigned bar = smem_u32(&S.tc_mbar), parity = S.tc_parity;

@@ -115,4 +115,33 @@ __device__ __forceinline__ void read_accumulator(const unsigned taddr, const int
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
 
+// ---- a handful of messages: the same product on the FMA units ------------------------------------------------------
+// Below SMALL_ROWS + 1 messages the product is no dense contraction: 512 threads take (row, one of eight k-slices) and
+// read the same bfloat16 operands (so a tile computes with the same weights whatever the size of the batch); the slices
+// meet by shared-memory adds in out[n * ldo + row], which the caller has zeroed.
+constexpr int SMALL_ROWS = 4;
+__device__ __forceinline__ void small_product(const unsigned char* Wb, const unsigned char* Xb, const int K, const int count, float* out, const int ldo, const int tid) {
+  const int r = tid & (M - 1), s = tid >> 6, K8 = K >> 3;
+  float acc[SMALL_ROWS];
+#pragma unroll
+  for (int b = 0; b < SMALL_ROWS; b++) acc[b] = 0.f;
+  for (int c = s; c < K8; c += 8) {
+    const uint4 w = *reinterpret_cast<const uint4*>(Wb + elem_off(r, 8 * c, K));
+    const unsigned wu[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int b = 0; b < SMALL_ROWS; b++) {
+      if (b >= count) break;
+      const uint4 x = *reinterpret_cast<const uint4*>(Xb + elem_off(b, 8 * c, K));
+      const unsigned xu[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+      for (int q = 0; q < 4; q++) {
+        acc[b] = fmaf(__uint_as_float(wu[q] << 16), __uint_as_float(xu[q] << 16), acc[b]);
+        acc[b] = fmaf(__uint_as_float(wu[q] & 0xffff0000u), __uint_as_float(xu[q] & 0xffff0000u), acc[b]);
+      }
+    }
+  }
+#pragma unroll
+  for (int b = 0; b < SMALL_ROWS; b++) if (b < count) atomicAdd(out + b * ldo + r, acc[b]);
+}
+
 }  // namespace tc
