@@ -213,8 +213,8 @@ ampnet_status_t ampnet_get_key_log(ampnet_graph_t*, int64_t* inst, int32_t* slot
 ampnet_status_t ampnet_leftover_cache_entries(ampnet_graph_t*, int64_t* n);
 /* Placement chosen for a parameterised node: number of row tiles (CTAs) and micro-batch row capacity.  Asynchronous
  * runs of graphs that the direct-delivery engine takes (single-row messages; Cond, Phi, Isu, Bcast, Concat, Sink and a
- * Loss fed by a Linear node) report the forward row tiles; a Linear node has as many backward column tiles again
- * (none for a node that feeds a Loss: that is one tile doing both directions).                                   */
+ * Loss fed by a Linear node) report the forward row tiles; a Linear node has backward column tiles besides (none for a
+ * node that feeds a Loss: each of its tiles holds all rows, does both directions and takes its share of the messages). */
 ampnet_status_t ampnet_get_placement(ampnet_graph_t*, int32_t node, int32_t* n_tiles, int32_t* batch_rows);
 
 /* Where the leader tile of a node spent its SM cycles in the last run: [0] waiting for messages, [1] fetching a
