@@ -820,6 +820,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
       return set_err(g, AMPNET_EINVAL, "node %d: queue capacity %u above the supported 2^%d (lower max_active_keys)", H.node, cap, det ? 20 : 23);
     for (int d = 0; d < 2; d++) {
       P.ring[d].e = B.take<Hdr>(cap);
+      if (R.direct && !dry) g->zero_regions.push_back({P.ring[d].e, (size_t)cap * sizeof(Hdr)});     // entries carry their ticket: none may survive a run
       P.ring[d].seq = C.take<unsigned>(cap);
       P.ring[d].tail = C.take<unsigned>(1);
       P.ring[d].mask = cap - 1;

@@ -53,6 +53,23 @@ __device__ __forceinline__ int atom_add_acq_rel(int* p, int v) {
   asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
   return old;
 }
+// Ring entries of this engine carry their own ticket, so that one round trip brings a message: two 16-byte halves
+// {inst, seq, slot, tag} and {u, base position, it | port << 16 | flags << 24, tag} with tag = ticket + 1 (16-byte stores
+// are single transactions; an entry is taken when both tags match).  The second half is stored with release and loaded
+// with acquire semantics: what the producer wrote before (payloads, the arrivals it has acquired) is visible to the
+// thread that takes the message.  Entries are zeroed before every run (tickets start over).
+__device__ __forceinline__ void entry_store(Hdr* e, int inst, int seq, int slot, int it, int u, int port, int rows, int flags, unsigned tag) {
+  asm volatile("st.relaxed.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};" :: "l"(e), "r"(inst), "r"(seq), "r"(slot), "r"(tag) : "memory");
+  asm volatile("st.release.gpu.global.v4.u32 [%0], {%1, %2, %3, %4};" :: "l"(reinterpret_cast<char*>(e) + 16), "r"(u), "r"(rows), "r"(it | (port << 16) | (flags << 24)), "r"(tag) : "memory");
+}
+__device__ __forceinline__ bool entry_load(const Hdr* e, unsigned tag, Hdr& h) {
+  unsigned a0, a1, a2, a3, b0, b1, b2, b3;
+  asm volatile("ld.relaxed.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(a0), "=r"(a1), "=r"(a2), "=r"(a3) : "l"(e) : "memory");
+  asm volatile("ld.acquire.gpu.global.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(b0), "=r"(b1), "=r"(b2), "=r"(b3) : "l"(reinterpret_cast<const char*>(e) + 16) : "memory");
+  h.inst = (int)a0; h.seq = (int)a1; h.slot = (int)a2; h.u = (int)b0; h.rows = (int)b1;
+  h.it = (int)(b2 & 0xffffu); h.port = (int)((b2 >> 16) & 0xffu); h.flags = (int)(b2 >> 24);
+  return a3 == tag && b3 == tag;
+}
 __device__ __forceinline__ void red_add(float* p, float v) {
   asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
@@ -403,8 +420,9 @@ __device__ __forceinline__ void gemm_nt_t(const float* __restrict__ A, const int
     for (int m = 0; m < TA; m++)
 #pragma unroll
       for (int j = 0; j < 4; j++) acc[m][j] = 0.f;
+    // (threads past the last block take part in the shuffles only: their loads would cost shared-memory bandwidth)
 #pragma unroll 2
-    for (int k4 = ks; k4 < K4; k4 += nsl) {
+    for (int k4 = valid ? ks : K4; k4 < K4; k4 += nsl) {
       float4 x[4];
       x[0] = A4[a0 + k4];
       if (TA > 1) { x[1] = A4[a1 + k4]; x[2] = A4[a2 + k4]; x[3] = A4[a3 + k4]; }
@@ -492,11 +510,8 @@ __device__ __forceinline__ int node_muf(const Ctx& C, const DevPPT& P) { return 
 // arrivals
 // ------------------------------------------------------------------------------------------------
 __device__ __noinline__ void ring_push(Ring& r, const Hdr& h, int it, int u, int port) {     // one thread
-  const unsigned t = atomicAdd(r.tail, 1u), s = t & r.mask;
-  int4* d = reinterpret_cast<int4*>(&r.e[s]);
-  d[0] = make_int4(h.inst, h.seq, h.slot, it);
-  d[1] = make_int4(u, port, h.rows, h.flags);
-  st_rel(&r.seq[s], t + 1u);
+  const unsigned t = atomicAdd(r.tail, 1u);
+  entry_store(&r.e[t & r.mask], h.inst, h.seq, h.slot, it, u, port, h.rows, h.flags, t + 1u);
 }
 // The instance in key slot `slot` loses `wgt` of its outstanding source messages (JOIN_UNIT each); the arrival that
 // brings the count to zero tells the controller.
@@ -557,13 +572,7 @@ __device__ __forceinline__ unsigned long long ballot64(const bool p0, const bool
 __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const bool leader, const bool fused, const int dirs, const bool light, const int min_take) {
   IN_SMEM(&P); IN_SMEM(&S);
   const int lane = threadIdx.x & 31;
-  if (light) {                      // nothing was pending a moment ago: watch the two head slots (and the end of the epoch) only
-    unsigned any = 0;
-    if (lane < 2 && (dirs & (1 << lane))) any = ld_rlx(&P.ring[lane].seq[S.head[lane] & P.ring[lane].mask]) == S.head[lane] + 1u;
-    if (lane == 2) any = ld_rlx(&C.g->done);
-    if (!__any_sync(0xffffffffu, any != 0)) return 0;
-  }
-  if (dirs == 1 && lane == 0) S.wver_seen = ld_rlx(P.wver);          // ordered by the fence below like the ring polls
+  if (dirs == 1 && lane == 0) S.wver_seen = ld_acq(P.wver);          // (acquire: the published columns are read after this)
   // queue occupancy (first tile of the node): tickets handed out and not yet taken, read along with the ring polls
   unsigned pending = 0;
   if (leader && lane < 2 && (dirs & (1 << lane))) pending = ld_rlx(P.ring[lane].tail) - S.head[lane];
@@ -574,31 +583,34 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
     for (int j = 0; j < NPL; j++) { if (m[j] == 0xffffffffu) n += 32; else { n += __ffs((int)~m[j]) - 1; break; } }
     return n;
   };
-  unsigned slot[2][NPL];
+  // First wave: the W entries at the head of each ring, one per lane (a tile that found nothing a moment ago watches
+  // eight; the end of the epoch is polled along).  One round trip brings the messages themselves.
+  const int W = light ? 8 : 32;
+  Hdr hh[2];
   int nready[2];
+  unsigned fin0 = 0;
+  if (light && lane == 31) fin0 = ld_rlx(&C.g->done);
 #pragma unroll
   for (int dir = 0; dir < 2; dir++) {
-    bool ready[NPL];
-#pragma unroll
-    for (int j = 0; j < NPL; j++) {
-      const unsigned t = S.head[dir] + lane + 32 * j;
-      slot[dir][j] = t & P.ring[dir].mask;
-      ready[j] = (dirs & (1 << dir)) && ld_rlx(&P.ring[dir].seq[slot[dir][j]]) == t + 1u;
+    bool ready = false;
+    if ((dirs & (1 << dir)) && lane < W) {
+      const unsigned t = S.head[dir] + (unsigned)lane;
+      ready = entry_load(&P.ring[dir].e[t & P.ring[dir].mask], t + 1u, hh[dir]);
     }
-    unsigned m[NPL];
-#pragma unroll
-    for (int j = 0; j < NPL; j++) m[j] = __ballot_sync(0xffffffffu, ready[j]);
-    nready[dir] = leading(m);
+    const unsigned m = __ballot_sync(0xffffffffu, ready);
+    nready[dir] = m == 0xffffffffu ? 32 : __ffs((int)~m) - 1;
   }
-  fence_acq();
+  if (light && nready[0] == 0 && nready[1] == 0 && !__shfl_sync(0xffffffffu, fin0, 31)) return 0;
   if (leader && lane < 2 && pending > S.qmax[lane] && pending < (1u << 30)) S.qmax[lane] = pending;
-  // A batch costs nearly the same whether it holds 2 messages or 100.  While the previous batch's arrivals are still under
-  // way the next one is taken only if at least min_take messages wait; the caller drops the threshold once they are done.
-  if (max(nready[0], nready[1]) < min_take && max(nready[0], nready[1]) > 0) return 0;
+  (void)min_take;
   if (nready[0] == 0 && nready[1] == 0) {
     unsigned fin = 0;
     if (lane == 0) fin = ld_acq(&C.g->done);
     if (!warp_uniform(fin)) return 0;
+    // (the rings are empty for good only if nothing arrived between the polls and the flag: look once more)
+    bool late = false;
+    if (lane < 2 && (dirs & (1 << lane))) { Hdr x; const unsigned t = S.head[lane]; late = entry_load(&P.ring[lane].e[t & P.ring[lane].mask], t + 1u, x); }
+    if (__any_sync(0xffffffffu, late)) return 0;
     if (lane == 0) {
       S.count = 0; S.dir = BWD; S.flags = BATCH_TERMINATE; S.n_upd = 0; S.upd_t = 0; S.eval = 0;
       if (S.n_acc > 0 && !C.eval) {                            // epoch-end flush of the leftover gradients
@@ -612,31 +624,41 @@ __device__ __noinline__ int form_batch(const Ctx& C, DevPPT& P, TileS& S, const 
   }
   const bool fwd_first = !(C.tune & 128) && nready[BWD] < 32 && nready[FWD] > nready[BWD];
   const int dir = (nready[BWD] == 0 || (fwd_first && nready[FWD] > 0)) ? FWD : BWD;
-  int take = min(nready[dir], P.BM);
-  Hdr h[NPL];
-  unsigned em[NPL];
+  const int cap = min(P.BM, FBM);
+  int take = min(nready[dir], cap);
+  Hdr* const out = S.hdr[S.fpb];
+  if (lane < take) out[lane] = dir == FWD ? hh[FWD] : hh[BWD];
+  if (nready[dir] == W && W < cap) {                             // the window was full: the entries behind it, straight into the batch
+    unsigned m[NPL];
 #pragma unroll
-  for (int j = 0; j < NPL; j++) {
-    h[j] = Hdr{0, 0, 0, 0, 0, 0, 0, 0};
-    if (lane + 32 * j < take) {
-      const int4* e = reinterpret_cast<const int4*>(&P.ring[dir].e[dir == FWD ? slot[FWD][j] : slot[BWD][j]]);
-      const int4 a = __ldcg(e), b = __ldcg(e + 1);
-      h[j].inst = a.x; h[j].seq = a.y; h[j].slot = a.z; h[j].it = a.w; h[j].u = b.x; h[j].port = b.y; h[j].rows = b.z; h[j].flags = b.w;
+    for (int j = 0; j < NPL; j++) {
+      const int idx = W + lane + 32 * j;
+      bool ready = false;
+      if (idx < cap) {
+        Hdr x;
+        const unsigned t = S.head[dir] + (unsigned)idx;
+        ready = entry_load(&P.ring[dir].e[t & P.ring[dir].mask], t + 1u, x);
+        if (ready) out[idx] = x;
+      }
+      m[j] = __ballot_sync(0xffffffffu, ready);
     }
+    take = min(W + leading(m), cap);
   }
-  const int eval0 = __shfl_sync(0xffffffffu, (int)((h[0].flags & HDR_EVAL) != 0), 0);
+  __syncwarp();
+  // the batch ends where training and forward-only messages meet
+  const int eval0 = (out[0].flags & HDR_EVAL) != 0;
+  {
+    unsigned em[NPL];
 #pragma unroll
-  for (int j = 0; j < NPL; j++) em[j] = __ballot_sync(0xffffffffu, lane + 32 * j < take && (int)((h[j].flags & HDR_EVAL) != 0) == eval0);
-  take = leading(em);
+    for (int j = 0; j < NPL; j++) em[j] = __ballot_sync(0xffffffffu, lane + 32 * j < take && (int)((out[lane + 32 * j].flags & HDR_EVAL) != 0) == eval0);
+    take = leading(em);
+  }
   bool upd = false;
   const bool grads = (dir == BWD || fused) && !eval0;          // a fused loss head turns every forward message into a gradient at once
   if (grads) {
     const int muf = node_muf(C, P);
     if (S.n_acc + take >= muf) { take = max(1, muf - S.n_acc); upd = true; }
   }
-#pragma unroll
-  for (int j = 0; j < NPL; j++) if (lane + 32 * j < take) S.hdr[S.fpb][lane + 32 * j] = h[j];
-  __syncwarp();
   if (lane == 0) {
     S.count = take; S.dir = dir; S.flags = upd ? BATCH_UPDATE : 0; S.eval = eval0;
     S.n_upd = upd ? S.n_acc + take : 0; S.upd_t = upd ? (int)S.n_updates + 1 : 0;
@@ -665,18 +687,28 @@ __device__ __noinline__ int form_batch_split(const Ctx& C, DevPPT& P, TileS& S, 
   const unsigned k0 = S.head[FWD], own_next = k0 * (unsigned)LT + (unsigned)t;
   const unsigned muf = (unsigned)node_muf(C, P);
   const unsigned long long done_grads = S.n_updates * (unsigned long long)muf, bnd = done_grads + muf;     // tickets below bnd belong to the next update
+  // one round trip: the ring's tail, the end of the epoch, and the first W own entries themselves
+  const int W = light ? 8 : 32;
   unsigned probe = 0;
-  if (lane == 0) probe = ld_rlx(rg.tail);
-  if (lane == 1) probe = ld_rlx(&rg.seq[own_next & rg.mask]) == own_next + 1u;
-  if (lane == 2) probe = ld_rlx(&C.g->done);
-  const unsigned tail = __shfl_sync(0xffffffffu, probe, 0), head_ready = __shfl_sync(0xffffffffu, probe, 1), fin0 = __shfl_sync(0xffffffffu, probe, 2);
+  if (lane == 30) probe = ld_rlx(rg.tail);
+  if (lane == 31) probe = ld_rlx(&C.g->done);
+  Hdr h0;
+  bool ready0 = false;
+  if (lane < W) {
+    const unsigned tk = (k0 + (unsigned)lane) * (unsigned)LT + (unsigned)t;
+    if (!training || tk < bnd) ready0 = entry_load(&rg.e[tk & rg.mask], tk + 1u, h0);
+  }
+  const unsigned m0 = __ballot_sync(0xffffffffu, ready0);
+  int nready = m0 == 0xffffffffu ? 32 : __ffs((int)~m0) - 1;
+  const unsigned tail = __shfl_sync(0xffffffffu, probe, 30), fin0 = __shfl_sync(0xffffffffu, probe, 31);
   const bool at_boundary = training && own_next >= bnd;
-  if (light && !fin0 && !(at_boundary ? tail >= bnd : head_ready != 0)) return 0;
+  if (light && !fin0 && !(at_boundary ? tail >= bnd : nready > 0)) return 0;
   if (leader && lane == 0 && tail - own_next < (1u << 30) && tail - own_next > S.qmax[FWD]) S.qmax[FWD] = tail - own_next;
   auto close_epoch = [&]() {                       // after `done`: the ring's tail is final
     unsigned fin_tail = 0;
     if (lane == 0) { fence_acq(); fin_tail = ld_rlx(rg.tail); }
     fin_tail = __shfl_sync(0xffffffffu, fin_tail, 0);
+    if (training && (long long)fin_tail - (long long)done_grads >= (long long)muf) return 0;      // (the tail read above was stale: a whole update is still due)
     if (lane == 0) {
       S.count = 0; S.dir = FWD; S.flags = BATCH_TERMINATE; S.n_upd = 0; S.upd_t = 0; S.eval = 0;
       const long long left = training ? (long long)fin_tail - (long long)done_grads : 0;
@@ -705,33 +737,36 @@ __device__ __noinline__ int form_batch_split(const Ctx& C, DevPPT& P, TileS& S, 
     if (!warp_uniform(fin)) return 0;
     return close_epoch();
   }
-  constexpr int NPL = FBM / 32;
-  unsigned slot[NPL], m[NPL];
-#pragma unroll
-  for (int j = 0; j < NPL; j++) {
-    const unsigned tk = (k0 + lane + 32 * j) * (unsigned)LT + (unsigned)t;
-    slot[j] = tk & rg.mask;
-    const bool ready = (!training || tk < bnd) && ld_rlx(&rg.seq[slot[j]]) == tk + 1u;
-    m[j] = __ballot_sync(0xffffffffu, ready);
-  }
-  fence_acq();
-  int nready = 0;
-#pragma unroll
-  for (int j = 0; j < NPL; j++) { if (m[j] == 0xffffffffu) nready += 32; else { nready += __ffs((int)~m[j]) - 1; break; } }
   if (nready == 0) {
     unsigned fin = 0;
     if (lane == 0) fin = ld_acq(&C.g->done);
     if (!warp_uniform(fin)) return 0;
     return close_epoch();
   }
-  const int take = min(nready, P.BM);
+  constexpr int NPL = FBM / 32;
+  const int cap = min(P.BM, FBM);
+  Hdr* const out = S.hdr[S.fpb];
+  if (lane < nready) out[lane] = h0;
+  if (nready == W && W < cap) {                                  // the window was full: the own entries behind it
+    unsigned m[NPL];
 #pragma unroll
-  for (int j = 0; j < NPL; j++)
-    if (lane + 32 * j < take) {
-      const int4* e = reinterpret_cast<const int4*>(&rg.e[slot[j]]);
-      const int4 a = __ldcg(e), b = __ldcg(e + 1);
-      S.hdr[S.fpb][lane + 32 * j] = Hdr{a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+    for (int j = 0; j < NPL; j++) {
+      const int idx = W + lane + 32 * j;
+      bool ready = false;
+      if (idx < cap) {
+        Hdr x;
+        const unsigned tk = (k0 + (unsigned)idx) * (unsigned)LT + (unsigned)t;
+        if (!training || tk < bnd) ready = entry_load(&rg.e[tk & rg.mask], tk + 1u, x);
+        if (ready) out[idx] = x;
+      }
+      m[j] = __ballot_sync(0xffffffffu, ready);
     }
+    int more = 0;
+#pragma unroll
+    for (int j = 0; j < NPL; j++) { if (m[j] == 0xffffffffu) more += 32; else { more += __ffs((int)~m[j]) - 1; break; } }
+    nready += more;
+  }
+  const int take = min(nready, cap);
   __syncwarp();
   if (lane == 0) {
     const int eval0 = (S.hdr[S.fpb][0].flags & HDR_EVAL) != 0;
@@ -1663,11 +1698,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
             if (lane == 0 && vm) tk = atomicAdd(P.ring[FWD].tail, (unsigned)__popc(vm));
             tk = __shfl_sync(0xffffffffu, tk, 0) + (unsigned)__popc(vm & ((1u << lane) - 1u));
             if (okm) {
-              const unsigned q = tk & P.ring[FWD].mask;
-              int4* d = reinterpret_cast<int4*>(&P.ring[FWD].e[q]);
-              d[0] = make_int4(inst, S.admit_seq, slot, 0);
-              d[1] = make_int4(u, 0, h.rows, h.flags);
-              st_rel(&P.ring[FWD].seq[q], tk + 1u);
+              entry_store(&P.ring[FWD].e[tk & P.ring[FWD].mask], inst, S.admit_seq, slot, 0, u, 0, h.rows, h.flags, tk + 1u);
             }
             if (lane == 0 && vm) atomicAdd(&S.node_msgs, (unsigned long long)__popc(vm));
           }

@@ -433,6 +433,38 @@ def test_stress_shape_without_updates_matches_oracle_on_tensor_cores_and_on_fma(
     e.close()
 
 
+@pytest.mark.parametrize("family,n,mak,lr,kind", [("mlp", 60, 4, 0.01, "momentum"), ("mlp", 60, 4, 0.001, "adam"), ("rnn", 90, 16, 0.01, "momentum"),
+                                                  ("rnn", 90, 16, 0.001, "adam"), ("tree", 40, 64, 0.005, "momentum"), ("tree", 40, 64, 0.001, "adam")])
+def test_asynchronous_flushes_with_momentum_and_adam_match_oracle(oracle_mod, family, n, mak, lr, kind):
+    """The update rules of the asynchronous path against the oracle where the schedule cannot matter: three epochs whose only
+    update is the flush at the end (the mean gradient of the whole set at the current parameters), so that the second and
+    third step use the moments and the step count the earlier ones left (every tile of a shared loss head keeps its own copy
+    of them)."""
+    import paper_1705_09786_b200 as amp
+    g, inst = _case(family, n)
+    p = wp.init_params(g)
+    opt = dict(kind=kind, momentum=0.8, beta1=0.85, beta2=0.99, eps=1e-6)
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst)
+    o.set_params(p)
+    o.set_optimizer(**opt)
+    e = amp.Engine(g)
+    e.load_instances(inst)
+    e.set_params(p)
+    e.set_optimizer(**opt)
+    for epoch in range(3):
+        _, oloss = o.run_epoch(mak=1, muf=1 << 30, lr=lr)
+        st, eloss = e.run_epoch(mak=mak, muf=1 << 30, lr=lr, deterministic=False, timeout_s=60)
+        np.testing.assert_allclose(eloss, oloss, rtol=2e-5, atol=4e-6)
+        ep, op = e.get_params(), o.get_params()
+        for k in op:
+            scale = np.abs(op[k]).max() + 1e-30
+            assert np.abs(ep[k] - op[k]).max() / scale <= 2e-4, (epoch, g.names[k[0]], k[1])
+    for i in g.ppt_nodes():
+        assert e.node_stats(i)["n_updates"] == 1
+    e.close()
+
+
 def test_tree_with_256_keys_in_flight(oracle_mod):
     """The tree workload with more keys than the benchmark uses (every instance of the set in flight at once)."""
     g, inst = _case("tree", 300)
