@@ -955,7 +955,7 @@ ampnet_status_t plan_run(ampnet_graph* g, int split, int mak, int det, int eval,
   g->d_keylog = X.keylog;
   const unsigned rcap = pow2_at_least(2ull * mak * (unsigned long long)std::max({D.maxT + 1, D.maxL, D.maxM + 1, 2}));
   X.retire_e = B.take<unsigned>(rcap);
-  X.retire_seq = C.take<unsigned>(rcap);
+  X.retire_seq = reinterpret_cast<unsigned*>(C.take<unsigned long long>(rcap));      // (the direct-delivery engine keeps 8-byte notices here)
   X.retire_mask = rcap - 1;
   X.order = nullptr; X.n_order = n_order;
   X.loss_out = B.take<float>((size_t)std::max<long long>(D.n, 1));

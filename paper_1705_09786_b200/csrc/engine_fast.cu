@@ -70,6 +70,17 @@ __device__ __forceinline__ bool entry_load(const Hdr* e, unsigned tag, Hdr& h) {
   h.it = (int)(b2 & 0xffffu); h.port = (int)((b2 >> 16) & 0xffu); h.flags = (int)(b2 >> 24);
   return a3 == tag && b3 == tag;
 }
+// Retire notices are one 8-byte word each: (ticket + 1) << 32 | key slot, stored with release and polled with acquire.
+__device__ __forceinline__ void retire_push(const Ctx& C, const int slot) {
+  const unsigned t = atomicAdd(&C.g->retire_tail, 1u);
+  const unsigned long long v = ((unsigned long long)(t + 1u) << 32) | (unsigned)slot;
+  asm volatile("st.release.gpu.global.u64 [%0], %1;" :: "l"(reinterpret_cast<unsigned long long*>(C.retire_seq) + (t & C.retire_mask)), "l"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long retire_poll(const Ctx& C, const unsigned h) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(reinterpret_cast<const unsigned long long*>(C.retire_seq) + (h & C.retire_mask)) : "memory");
+  return v;
+}
 __device__ __forceinline__ void red_add(float* p, float v) {
   asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(p), "f"(v) : "memory");
 }
@@ -519,9 +530,7 @@ __device__ __noinline__ void retire_arrive(const Ctx& C, int slot, int wgt) {
   const int old = atom_add_acq_rel(&C.outstanding[slot], -wgt);
   if (old < wgt) fail(C, ST_OVERFLOW, -30, slot);                // more source messages came home than were pumped
   if (old != wgt) return;
-  const unsigned t = atomicAdd(&C.g->retire_tail, 1u), s = t & C.retire_mask;
-  C.retire_e[s] = (unsigned)slot;
-  st_rel(&C.retire_seq[s], t + 1u);
+  retire_push(C, slot);
 }
 // One thread, after the barrier behind the deposits of its CTA: arrive at landing L of message h with weight wgt.
 __device__ __noinline__ void arrive(const Ctx& C, const int inst, const int seq, const int slot, const int flags, const int ibase, const Landing& L, int wgt,
@@ -543,9 +552,7 @@ __device__ __noinline__ void arrive(const Ctx& C, const int inst, const int seq,
     if (old < wgt) fail(C, ST_OVERFLOW, -30, slot);
     if (old != wgt) return;
     if (L.post) atomicAdd(node_msgs, (unsigned long long)L.post);
-    const unsigned t = atomicAdd(&C.g->retire_tail, 1u), s = t & C.retire_mask;
-    C.retire_e[s] = (unsigned)slot;
-    st_rel(&C.retire_seq[s], t + 1u);
+    retire_push(C, slot);
     return;
   }
   if (L.act != ACT_PUSH) return;
@@ -1574,11 +1581,19 @@ struct CtrlS {
   long long next, retired;
   int active;
   unsigned retire_head;
-  int admit_slot, admit_inst, admit_seq, admit_eval;
+  int admit_slot, admit_inst, admit_seq, admit_eval, admit_rows;
   int src_count[4];
   unsigned long long node_msgs;
   unsigned occ[OCC_SLOTS / 32];
   Landing dl[MAXD];
+  // kept on chip so that a retirement and the admission behind it wait for no load of the controller's own state
+  int slot_inst[OCC_SLOTS];           // instance in each key slot (slots beyond this live in device memory only)
+  int max_active;
+  double total_loss, inf_loss;
+  unsigned long long correct, n_pred, inf_instances, inf_correct, inf_pred;
+  unsigned src_tail[4];               // tickets handed out in the ring each direct source feeds (the controller is its only producer)
+  // the next instance to admit, looked up ahead of time
+  int pf_valid, pf_inst, pf_rows, pf_eval, pf_outstanding, pf_count[4];
 };
 
 // A source whose messages carry no payload of their own and feed a parameterised node directly (token ids, leaf ids,
@@ -1593,22 +1608,58 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
   IN_SMEM(&S);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const DevInst& I = C.inst;
-  if (tid == 0) { S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; S.node_msgs = 0; }
+  if (tid == 0) {
+    S.next = 0; S.retired = 0; S.active = 0; S.retire_head = 0; S.ok = 1; S.node_msgs = 0; S.max_active = 0; S.pf_valid = 0;
+    S.total_loss = S.inf_loss = 0.0; S.correct = S.n_pred = S.inf_instances = S.inf_correct = S.inf_pred = 0;
+  }
+  if (tid < 4) S.src_tail[tid] = 0;
   for (int i = tid; i < OCC_SLOTS / 32; i += FT) S.occ[i] = 0u;
+  for (int i = tid; i < min(C.mak, OCC_SLOTS); i += FT) S.slot_inst[i] = -1;
+  // every loss cell starts empty (predok = -1 marks "no loss evaluated at this key"); a retirement leaves its cells empty again
+  for (int li = 0; li < C.n_loss; li++) {
+    const DevNode& L = g_nodes[C.loss_nodes[li]];
+    const long long cnt = (long long)C.mak * C.IT * L.U_in;
+    for (long long k = tid; k < cnt; k += FT) { L.lossval[k] = 0.f; L.predok[k] = -1; }
+  }
+  __syncthreads();
+  // Look up the next instance of the order: what it pumps and what finishes it (thread 0, while nothing waits for it).
+  auto prefetch = [&]() {
+    S.pf_valid = 0;
+    if (S.next >= C.n_order) return;
+    const int inst = (int)(C.order ? C.order[S.next] : S.next);
+    int total = 0;
+    for (int s = 0; s < C.n_sources; s++) {
+      const DevNode& sn = g_nodes[C.src_nodes[s]];
+      int cnt = 1;
+      if (sn.fn == 2) cnt = (int)(I.offsets[inst + 1] - I.offsets[inst]);
+      else if (sn.fn == 4) cnt = (int)(I.leaf_off[inst + 1] - I.leaf_off[inst]);
+      S.pf_count[s] = cnt; total += cnt;
+    }
+    S.pf_eval = C.eval || (C.inference_only && C.inference_only[inst]);
+    if (S.pf_eval) {      // forward only: the instance is finished when every Loss / Sink has been reached
+      int exp = C.ends_per_instance;
+      if (C.ends_per_position) exp += C.ends_per_position * (int)(I.offsets[inst + 1] - I.offsets[inst]);
+      S.pf_outstanding = exp * JOIN_UNIT;
+    } else S.pf_outstanding = total * JOIN_UNIT;
+    S.pf_rows = (int)(I.offsets ? I.offsets[inst] : 0);
+    S.pf_inst = inst; S.pf_valid = 1;
+  };
+  if (tid == 0) prefetch();
   __syncthreads();
   unsigned idle = 0;
   for (;;) {
     // ---- retirements: sum the instance's loss cells in key order, free the slot ------------------------------
     if (warp == 0) {
       for (;;) {
-        unsigned h = 0, ready = 0;
-        if (lane == 0) { h = S.retire_head; ready = ld_acq(&C.retire_seq[h & C.retire_mask]) == h + 1u; }
+        unsigned h = 0, ready = 0, rs = 0;
+        if (lane == 0) { h = S.retire_head; const unsigned long long v = retire_poll(C, h); ready = (unsigned)(v >> 32) == h + 1u; rs = (unsigned)v; }
         h = warp_uniform(h);
         if (!warp_uniform(ready)) break;
-        const int slot = (int)__ldcg(&C.retire_e[h & C.retire_mask]);
+        const int slot = (int)warp_uniform(rs);
+        if ((unsigned)slot >= (unsigned)C.mak) { if (lane == 0) fail(C, ST_OVERFLOW, -33, slot); break; }
         __syncwarp();
         if (lane == 0) S.retire_head = h + 1u;
-        const int inst = C.slot_inst[slot];
+        const int inst = slot < OCC_SLOTS ? S.slot_inst[slot] : C.slot_inst[slot];
         double tot = 0.0; int okc = 0, np = 0;
         for (int li = 0; li < C.n_loss; li++) {
           const DevNode& L = g_nodes[C.loss_nodes[li]];
@@ -1616,7 +1667,8 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
           double dpart = 0.0;
           for (long long k = k0 + lane; k < k1; k += 32) {
             const int pk = __ldcg(&L.predok[k]);
-            if (pk >= 0) { dpart += (double)__ldcg(&L.lossval[k]); okc += pk; np += 1; }
+            const float lv = __ldcg(&L.lossval[k]);               // (both loads in flight together)
+            if (pk >= 0) { dpart += (double)lv; okc += pk; np += 1; L.lossval[k] = 0.f; L.predok[k] = -1; }
           }
           for (int o = 16; o; o >>= 1) dpart += __shfl_xor_sync(0xffffffffu, dpart, o);
           tot += dpart;
@@ -1624,10 +1676,10 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
         for (int o = 16; o; o >>= 1) { okc += __shfl_xor_sync(0xffffffffu, okc, o); np += __shfl_xor_sync(0xffffffffu, np, o); }
         if (lane == 0) {
           C.loss_out[inst] = (float)tot;
-          if (C.inference_only && C.inference_only[inst]) { C.g->inf_loss += tot; C.g->inf_instances += 1; C.g->inf_correct += okc; C.g->inf_pred += np; }
-          else { C.g->total_loss += tot; C.g->correct += okc; C.g->n_pred += np; }
+          if (C.inference_only && C.inference_only[inst]) { S.inf_loss += tot; S.inf_instances += 1; S.inf_correct += okc; S.inf_pred += np; }
+          else { S.total_loss += tot; S.correct += okc; S.n_pred += np; }
           C.slot_inst[slot] = -1;
-          if (slot < OCC_SLOTS) S.occ[slot >> 5] &= ~(1u << (slot & 31));
+          if (slot < OCC_SLOTS) { S.slot_inst[slot] = -1; S.occ[slot >> 5] &= ~(1u << (slot & 31)); }
           S.active--; S.retired++;
         }
         __syncwarp();
@@ -1638,7 +1690,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
     for (;;) {
       if (tid == 0) {
         S.admit_slot = -1;
-        if (S.active < C.mak && S.next < C.n_order) {
+        if (S.active < C.mak && S.pf_valid) {
           int slot = 0;                                                   // lowest free slot
           const int nw = (min(C.mak, OCC_SLOTS) + 31) >> 5;
           int w = 0;
@@ -1646,43 +1698,26 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
           if (w < nw) slot = w * 32 + __ffs(~S.occ[w]) - 1;
           else { slot = OCC_SLOTS; while (slot < C.mak && C.slot_inst[slot] >= 0) slot++; }
           if (slot < OCC_SLOTS) S.occ[slot >> 5] |= 1u << (slot & 31);
-          const int inst = (int)(C.order ? C.order[S.next] : S.next);
-          if (C.slot_inst[slot] >= 0) fail(C, ST_OVERFLOW, -32, slot);
-          S.admit_slot = slot; S.admit_inst = inst; S.admit_seq = (int)S.next;
+          const int inst = S.pf_inst;
+          if ((slot < OCC_SLOTS ? S.slot_inst[slot] : C.slot_inst[slot]) >= 0) fail(C, ST_OVERFLOW, -32, slot);
+          S.admit_slot = slot; S.admit_inst = inst; S.admit_seq = (int)S.next; S.admit_eval = S.pf_eval;
+          for (int s = 0; s < C.n_sources; s++) S.src_count[s] = S.pf_count[s];
           C.slot_inst[slot] = inst;
+          if (slot < OCC_SLOTS) S.slot_inst[slot] = inst;
           S.active++;
-          if (S.active > C.g->max_active) C.g->max_active = S.active;
-          int total = 0;
-          for (int s = 0; s < C.n_sources; s++) {
-            const DevNode& sn = g_nodes[C.src_nodes[s]];
-            int cnt = 1;
-            if (sn.fn == 2) cnt = (int)(I.offsets[inst + 1] - I.offsets[inst]);
-            else if (sn.fn == 4) cnt = (int)(I.leaf_off[inst + 1] - I.leaf_off[inst]);
-            S.src_count[s] = cnt; total += cnt;
-          }
-          S.admit_eval = C.eval || (C.inference_only && C.inference_only[inst]);
-          if (S.admit_eval) {      // forward only: the instance is finished when every Loss / Sink has been reached
-            int exp = C.ends_per_instance;
-            if (C.ends_per_position) exp += C.ends_per_position * (int)(I.offsets[inst + 1] - I.offsets[inst]);
-            C.outstanding[slot] = exp * JOIN_UNIT;
-          } else C.outstanding[slot] = total * JOIN_UNIT;
+          if (S.active > S.max_active) S.max_active = S.active;
+          C.outstanding[slot] = S.pf_outstanding;
+          S.admit_rows = S.pf_rows;
           S.next++;
         }
       }
       __syncthreads();
       const int slot = S.admit_slot;
       if (slot < 0) break;
-      // clear the slot's loss cells (predok = -1 marks "no loss evaluated at this key")
-      for (int li = 0; li < C.n_loss; li++) {
-        const DevNode& L = g_nodes[C.loss_nodes[li]];
-        const long long k0 = (long long)slot * C.IT * L.U_in, cnt = (long long)C.IT * L.U_in;
-        for (long long k = tid; k < cnt; k += FT) { L.lossval[k0 + k] = 0.f; L.predok[k0 + k] = -1; }
-      }
-      __threadfence();
-      __syncthreads();
-      // pump the source messages (Sec. 4: tokens / leaves, initial hidden state, dense row)
+      // pump the source messages (Sec. 4: tokens / leaves, initial hidden state, dense row); the stores above (the slot's
+      // bookkeeping, the emptied loss cells of its previous instance) are ordered before them by the entries' release
       const int inst = S.admit_inst;
-      Hdr h; h.inst = inst; h.seq = S.admit_seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = (int)(I.offsets ? I.offsets[inst] : 0); h.flags = S.admit_eval ? HDR_EVAL : 0;
+      Hdr h; h.inst = inst; h.seq = S.admit_seq; h.slot = slot; h.it = 0; h.u = 0; h.port = 0; h.rows = S.admit_rows; h.flags = S.admit_eval ? HDR_EVAL : 0;
       for (int s = 0; s < C.n_sources; s++) {
         const DevNode& sn = g_nodes[C.src_nodes[s]];
         const int cnt = S.src_count[s];
@@ -1695,7 +1730,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
             const bool okm = k < cnt && key_of(C, sn.succ_node[0], slot, 0, u, P.U) >= 0;
             const unsigned vm = __ballot_sync(0xffffffffu, okm);
             unsigned tk = 0;
-            if (lane == 0 && vm) tk = atomicAdd(P.ring[FWD].tail, (unsigned)__popc(vm));
+            if (lane == 0 && vm) tk = atomicAdd(&S.src_tail[s], (unsigned)__popc(vm));     // (shared memory: the only producer of this ring)
             tk = __shfl_sync(0xffffffffu, tk, 0) + (unsigned)__popc(vm & ((1u << lane) - 1u));
             if (okm) {
               entry_store(&P.ring[FWD].e[tk & P.ring[FWD].mask], inst, S.admit_seq, slot, 0, u, 0, h.rows, h.flags, tk + 1u);
@@ -1723,11 +1758,24 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
         }
       }
       __syncthreads();
+      if (tid == 0) {
+        for (int s = 0; s < C.n_sources; s++) {                 // the tickets handed out, for the tiles that read the ring's tail
+          const DevNode& sn = g_nodes[C.src_nodes[s]];
+          if (source_is_direct(sn)) *(volatile unsigned*)g_ppts[g_nodes[sn.succ_node[0]].ppt].ring[FWD].tail = S.src_tail[s];
+        }
+        prefetch();
+      }
+      __syncthreads();
     }
     // ---- termination / pacing ---------------------------------------------------------------------------------
     const bool finished = S.retired == C.n_order;
     if (finished) {
-      if (tid == 0) { C.g->rounds = 0; atomicAdd(&C.g->node_messages, S.node_msgs); __threadfence(); st_rel(&C.g->done, 1u); }
+      if (tid == 0) {
+        Globals& G = *C.g;
+        G.max_active = S.max_active; G.total_loss = S.total_loss; G.correct = S.correct; G.n_pred = S.n_pred;
+        G.inf_loss = S.inf_loss; G.inf_instances = S.inf_instances; G.inf_correct = S.inf_correct; G.inf_pred = S.inf_pred;
+        G.rounds = 0; atomicAdd(&G.node_messages, S.node_msgs); __threadfence(); st_rel(&G.done, 1u);
+      }
       break;
     }
     if (tid == 0) {
@@ -1738,7 +1786,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlS& S, const unsig
       }
       const unsigned hh = S.retire_head;
       unsigned spins = 0;
-      while (ld_acq(&C.retire_seq[hh & C.retire_mask]) != hh + 1u && spins < 64) { __nanosleep(50); spins++; }
+      while ((unsigned)(retire_poll(C, hh) >> 32) != hh + 1u && spins < 64) { __nanosleep(50); spins++; }
     }
     __syncthreads();
     if (!S.ok) break;
