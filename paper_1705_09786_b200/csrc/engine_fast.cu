@@ -930,40 +930,51 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
     // orders the issuing thread's view of the row (ordinary stores of other SMs, acquired through the ring) before the copy.
     const unsigned bar = smem_u32(&S.mbar);
     if (tid == 0 && bulk_ok) asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" :: "r"(bar), "r"((unsigned)(count * xwidth * 4)) : "memory");
-    if (tid < count) {
-      const Hdr h = S.hdr[pbn][tid];
+    // Two jobs per message, on different warps so that they run side by side: its key, staging copy and bookkeeping
+    // (message m on thread m), and its route (message m on thread m + 64, spread over two warps; a batch of more than 64
+    // messages wraps around, each thread then doing one job after the other).
+    auto stage_job = [&](const int m) {
+      const Hdr h = S.hdr[pbn][m];
       const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
-      S.key[tid] = key;
-      S.nd[pbn][tid] = 0; S.pre[pbn][tid] = 0;
-      if (key < 0) S.ok = 0;
-      if (key >= 0) {
-        if (!lookup) {
-          const float* x = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
-          S.rowptr[tid] = x;
-          if (bulk_ok) {
-            asm volatile("fence.proxy.async;" ::: "memory");
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         :: "r"(smem_u32(Xs + (size_t)tid * LX)), "l"(x), "r"((unsigned)(xwidth * 4)), "r"(bar) : "memory");
-          }
+      S.key[m] = key;
+      if (key < 0) { S.ok = 0; return; }
+      if (!lookup) {
+        const float* x = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+        S.rowptr[m] = x;
+        if (bulk_ok) {
+          asm volatile("fence.proxy.async;" ::: "memory");
+          asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                       :: "r"(smem_u32(Xs + (size_t)m * LX)), "l"(x), "r"((unsigned)(xwidth * 4)), "r"(bar) : "memory");
         }
-        if (lookup) {
-          const int id = C.inst.tokens[(long long)h.rows + h.u];
-          S.rowid[tid] = (unsigned)id < (unsigned)in ? id : -1;
-        }
-        if ((leader || split) && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
-        else if (leader && !S.eval && fwd_only) P.vcache[key] = max(S.version, (int)(S.wver_seen / (unsigned)P.TB));   // the version this forward pass uses (Sec. 3: staleness)
-        int pre = 0, nd = 0;
-        if (fused) {                                   // the label, fetched while the input rows are in flight
-          const DevInst& I = C.inst;
-          if (g_nodes[loss_node].type == LOSS_CE) S.rowid[tid] = I.labels_i[I.labels_per_node ? (long long)h.rows + h.u : h.inst];
-          else S.rowid[tid] = __float_as_int(I.labels_f[h.inst]);
-        }
-        if (fused) {                                   // the Loss and this node's own backward arrival, then the way back
-          if (!S.eval) nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][tid], pre);
-          pre += S.eval ? 1 : 2;
-        } else if (dir == FWD) nd = route_message(C, h, N.succ_node[0], N.succ_port[0], FWD, out, S.dl[pbn][tid], pre);
-        else nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][tid], pre);
-        S.nd[pbn][tid] = (unsigned char)nd; S.pre[pbn][tid] = (short)pre;
+      }
+      if (lookup) {
+        const int id = C.inst.tokens[(long long)h.rows + h.u];
+        S.rowid[m] = (unsigned)id < (unsigned)in ? id : -1;
+      }
+      if ((leader || split) && !S.eval && fused) atomicAdd(&S.stale_hist[0], 1ull);
+      else if (leader && !S.eval && fwd_only) P.vcache[key] = max(S.version, (int)(S.wver_seen / (unsigned)P.TB));   // the version this forward pass uses (Sec. 3: staleness)
+      if (fused) {                                     // the label, fetched while the input rows are in flight
+        const DevInst& I = C.inst;
+        if (g_nodes[loss_node].type == LOSS_CE) S.rowid[m] = I.labels_i[I.labels_per_node ? (long long)h.rows + h.u : h.inst];
+        else S.rowid[m] = __float_as_int(I.labels_f[h.inst]);
+      }
+    };
+    auto route_job = [&](const int m) {
+      const Hdr h = S.hdr[pbn][m];
+      int pre = 0, nd = 0;
+      if (fused) {                                     // the Loss and this node's own backward arrival, then the way back
+        if (!S.eval) nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][m], pre);
+        pre += S.eval ? 1 : 2;
+      } else if (dir == FWD) nd = route_message(C, h, N.succ_node[0], N.succ_port[0], FWD, out, S.dl[pbn][m], pre);
+      else nd = route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][m], pre);
+      S.nd[pbn][m] = (unsigned char)nd; S.pre[pbn][m] = (short)pre;
+    };
+    {
+      const int mr = tid >= 64 ? 2 * (tid & 31) + ((tid >> 5) & 1) : 64 + tid;        // message whose route this thread resolves
+#pragma unroll 1
+      for (int step = 0; step < 2; step++) {
+        if ((tid >= 64) == (step == 0)) { if (mr < count) route_job(mr); }
+        else if (tid < count) stage_job(tid);
       }
     }
     __syncwarp();
@@ -1422,22 +1433,32 @@ __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int ti
     TPHASE(0);
     if (!S.ok) return;
     const int count = S.count, flags = S.flags;
-    if (tid < count) {
-      const Hdr h = S.hdr[pbn][tid];
-      const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
-      S.key[tid] = key; S.nd[pbn][tid] = 0; S.pre[pbn][tid] = 0;
-      if (key < 0) S.ok = 0;
-      else {
-        S.rowptr[tid] = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
-        if (leader) {                                  // staleness: updates of this node between forward and backward (Sec. 3)
-          int st = S.version - ((flags & BATCH_UPDATE) ? 1 : 0) - P.vcache[key];
-          if (st < 0) st = 0;
-          atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
-          atomicMax(&S.max_stale, st);
+    // key and bookkeeping of message m on thread m, its route on thread m + 64 (two warps side by side; see tile_main)
+    {
+      const int mr = tid >= 64 ? 2 * (tid & 31) + ((tid >> 5) & 1) : 64 + tid;
+#pragma unroll 1
+      for (int step = 0; step < 2; step++) {
+        if ((tid >= 64) == (step == 0)) {
+          if (mr < count) {
+            int pre = 0;
+            S.nd[pbn][mr] = (unsigned char)route_message(C, S.hdr[pbn][mr], N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][mr], pre);
+            S.pre[pbn][mr] = (short)pre;
+          }
+        } else if (tid < count) {
+          const Hdr h = S.hdr[pbn][tid];
+          const long long key = key_of(C, P.node, h.slot, h.it, h.u, P.U);
+          S.key[tid] = key;
+          if (key < 0) S.ok = 0;
+          else {
+            S.rowptr[tid] = P.xcache ? P.xcache + key * (long long)P.xld : C.inst.dense + (long long)h.inst * C.inst.dense_dim;
+            if (leader) {                                  // staleness: updates of this node between forward and backward (Sec. 3)
+              int st = S.version - ((flags & BATCH_UPDATE) ? 1 : 0) - P.vcache[key];
+              if (st < 0) st = 0;
+              atomicAdd(&S.stale_hist[st > 63 ? 63 : st], 1ull);
+              atomicMax(&S.max_stale, st);
+            }
+          }
         }
-        int pre = 0;
-        S.nd[pbn][tid] = (unsigned char)route_message(C, h, N.pred_node[0], N.pred_port[0], BWD, in, S.dl[pbn][tid], pre);
-        S.pre[pbn][tid] = (short)pre;
       }
     }
     __syncwarp();
