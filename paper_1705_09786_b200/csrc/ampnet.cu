@@ -604,7 +604,7 @@ bool direct_candidate(ampnet_graph* g, const HostDataset& D, int det) {
 }
 
 // Tiles of the direct-delivery engine.  A Linear node is split by direction: forward row tiles of `rows` weight rows
-// (AMPNET_DIRECT_ROWS, default 8) and backward column tiles of `cols` input columns (AMPNET_DIRECT_COLS, default 16;
+// (AMPNET_DIRECT_ROWS, default 16) and backward column tiles of `cols` input columns (AMPNET_DIRECT_COLS, default 16;
 // 4, 8, 16 or 32), more per tile where the CTA budget, shared memory or the register-resident accumulators ask for it.
 // A node that feeds a Loss is one tile for both directions (the Loss needs the whole output row); a large embedding
 // table is dealt to four tiles by row id.
@@ -617,7 +617,7 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   size_t static_smem = 48 * 1024;
   ampnet_direct_static_smem(&static_smem);
   const size_t budget = (size_t)g->max_smem - static_smem - 1024;
-  int rows = 8, cols = 16;
+  int rows = 16, cols = 16;
   if (const char* e = getenv("AMPNET_DIRECT_ROWS")) rows = std::max(1, atoi(e));
   if (const char* e = getenv("AMPNET_DIRECT_COLS")) { const int c = atoi(e); if (c == 4 || c == 8 || c == 16 || c == 32) cols = c; }
   const int np = (int)g->ppts.size(), tile_budget = n_ctas - 1, max_units = ampnet_direct_max_units();
@@ -702,7 +702,7 @@ ampnet_status_t place_direct(ampnet_graph* g, int n_ctas, std::vector<Role>& rol
   // CTAs left over go to the loss heads: their tiles share the node's messages (every tree node, every list, passes
   // through that one node) and meet at its updates
   {
-    int used = 0, heads = 0, want = 4;
+    int used = 0, heads = 0, want = 8;
     if (const char* e = getenv("AMPNET_LOSS_TILES")) want = std::max(1, std::min(16, atoi(e)));
     for (int p = 0; p < np; p++) { used += g->ppts[p].T + g->ppts[p].TB; heads += fixed[p] && g->ppts[p].kind != LOOKUP; }
     for (int p = 0; p < np && heads > 0; p++) {
