@@ -414,7 +414,7 @@ __device__ __forceinline__ void gemm_nt_t(const float* __restrict__ A, const int
   const int tid = threadIdx.x;
   const int tA = (nA + TA - 1) / TA, tB = (nB + 3) >> 2, n_tiles = tA * tB;
   int nsl = 1, sh = 0;
-  while (nsl < 32 && n_tiles * nsl * 2 <= FT) { nsl <<= 1; sh++; }
+  while (nsl < 32 && n_tiles * nsl * 4 <= FT) { nsl <<= 1; sh++; }       // (measured: merging more slices by shuffles costs more than it spreads)
   const int per_pass = FT >> sh, ks = tid & (nsl - 1);
   const FastDiv dB(tB);
   for (int t0 = 0; t0 < n_tiles; t0 += per_pass) {
@@ -460,10 +460,37 @@ __device__ __forceinline__ void gemm_nt_t(const float* __restrict__ A, const int
     }
   }
 }
+// Up to four rows of A: a warp per row of B, the lanes take interleaved groups of four k and meet by shuffles (no blocks to
+// set up: a single message costs 900-1,300 cycles instead of 1,600).
+__device__ __forceinline__ void gemm_small(const float* __restrict__ A, const int lda, const int nA, const float* __restrict__ B, const int ldb,
+                                           const int nB, const int K4, float* __restrict__ out, const int ldo) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const float4* const A4 = reinterpret_cast<const float4*>(A);
+  const float4* const B4 = reinterpret_cast<const float4*>(B);
+  const int lda4 = lda >> 2, ldb4 = ldb >> 2;
+  for (int o = warp; o < nB; o += FW) {
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    for (int k4 = lane; k4 < K4; k4 += 32) {
+      const float4 w = B4[o * ldb4 + k4];
+#pragma unroll
+      for (int b = 0; b < 4; b++)
+        if (b < nA) {
+          const float4 x = A4[b * lda4 + k4];
+          acc[b] = fmaf(x.x, w.x, acc[b]); acc[b] = fmaf(x.y, w.y, acc[b]); acc[b] = fmaf(x.z, w.z, acc[b]); acc[b] = fmaf(x.w, w.w, acc[b]);
+        }
+    }
+#pragma unroll
+    for (int off = 16; off; off >>= 1)
+#pragma unroll
+      for (int b = 0; b < 4; b++) acc[b] += __shfl_xor_sync(0xffffffffu, acc[b], off);
+    if (lane < nA) out[lane * ldo + o] = lane == 0 ? acc[0] : lane == 1 ? acc[1] : lane == 2 ? acc[2] : acc[3];
+  }
+}
 // A handful of messages: one row of A per thread (nothing is spent on padding rows); otherwise 4 x 4 blocks.
 __device__ __forceinline__ void gemm_nt(const float* __restrict__ A, const int lda, const int nA, const float* __restrict__ B, const int ldb,
                                         const int nB, const int K4, float* __restrict__ out, const int ldo) {
-  if (nA <= 8) gemm_nt_t<1>(A, lda, nA, B, ldb, nB, K4, out, ldo);
+  if (nA <= 4 && K4 <= 128) gemm_small(A, lda, nA, B, ldb, nB, K4, out, ldo);
+  else if (nA <= 8) gemm_nt_t<1>(A, lda, nA, B, ldb, nB, K4, out, ldo);
   else gemm_nt_t<4>(A, lda, nA, B, ldb, nB, K4, out, ldo);
 }
 
