@@ -214,12 +214,13 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
       out[nout++] = pack_landing(C, d);
       pend = nullptr; pend_exp = 0; pend_slot = 0; post = 0; clear = clear2 = nullptr; phi_cnt = nullptr;
     };
+    Deliv d;
+    bool landed = false;
     switch (n.type) {
       case LINEAR: case LOOKUP: {
         DevPPT& Q = g_ppts[n.ppt];
         const long long key = key_of(C, f.node, h.slot, f.it, f.u, Q.U);
         if (key < 0) return nout;
-        Deliv d;
         if (f.dir == FWD) {
           if (!Q.xcache) { fail(C, ST_OVERFLOW, f.node, -10); return nout; }
           d.dst = Q.xcache + key * (long long)Q.xld;
@@ -233,32 +234,29 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
         d.expected = pend ? pend_exp : JOIN_UNIT;
         d.s0 = f.s0; d.w = f.w; d.act = ACT_PUSH; d.ppt = n.ppt; d.dir = f.dir; d.u = f.u; d.it = f.it; d.port = f.port;
         d.post = post + 1; d.node = f.node;
-        land(d);
+        landed = true;
       } break;
       case LOSS_CE: case LOSS_MSE: {
         pre++;
-        Deliv d;
         d.dst = nullptr; d.jcnt = nullptr; d.expected = 0; d.s0 = f.s0; d.w = f.w; d.act = ACT_LOSS; d.ppt = -1; d.dir = FWD;
         d.u = f.u; d.it = f.it; d.port = f.port; d.post = 0; d.node = f.node;
-        land(d);
+        landed = true;
       } break;
       case SOURCE: {                                        // a source message came home
         if (pend) { fail(C, ST_OVERFLOW, f.node, -14); return nout; }
-        Deliv d;
         d.dst = nullptr; d.jcnt = &C.outstanding[h.slot]; d.expected = 0; d.s0 = 0; d.w = 0; d.act = ACT_RETIRE; d.ppt = -1;
         d.dir = BWD; d.u = f.u; d.it = f.it; d.port = f.port; d.post = post; d.node = f.node;
         // a recorded origin may be cleared only when every tile has read it: the tiles' arrivals of this message meet at the
         // Phi's counter first, and the one that completes it retires the whole source message
         if (clear && phi_cnt) { d.jcnt = phi_cnt; d.expected = JOIN_UNIT; }
-        land(d);
+        landed = true;
       } break;
       case SINK:
         count();
         if (h.flags & HDR_EVAL) {
-          Deliv d;
-          d.dst = nullptr; d.jcnt = &C.outstanding[h.slot]; d.expected = 0; d.s0 = 0; d.w = 0; d.act = ACT_RETIRE; d.ppt = -1;
+            d.dst = nullptr; d.jcnt = &C.outstanding[h.slot]; d.expected = 0; d.s0 = 0; d.w = 0; d.act = ACT_RETIRE; d.ppt = -1;
           d.dir = FWD; d.u = f.u; d.it = f.it; d.port = f.port; d.post = post; d.node = f.node;
-          land(d);
+          landed = true;
         } else { f.null = 1; to_pred(0); }                   // answers with a zero gradient
         break;
       case COND:
@@ -333,12 +331,11 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
           if (key < 0) return nout;
           const DevNode& s = g_nodes[n.succ_node[0]];
           if ((unsigned)port >= (unsigned)n.fn_arg || !n.jalias || pend) { fail(C, ST_OVERFLOW, f.node, port); return nout; }
-          Deliv d;
-          d.dst = n.jbuf + key * n.jstride + port * n.in_dim;
+            d.dst = n.jbuf + key * n.jstride + port * n.in_dim;
           d.jcnt = &n.jcnt[key]; d.expected = n.fn_arg * JOIN_UNIT;
           d.s0 = f.s0; d.w = f.w; d.act = ACT_PUSH; d.ppt = s.ppt; d.dir = FWD; d.u = f.u; d.it = f.it; d.port = 0;
           d.post = 1; d.node = n.succ_node[0];
-          land(d);
+          landed = true;
         } else {
           count();
           for (int k = n.fn_arg - 1; k >= 0; k--) {
@@ -354,6 +351,7 @@ __device__ __noinline__ int route_message(const Ctx& C, const Hdr h, int start_n
         fail(C, ST_OVERFLOW, f.node, n.type);
         return nout;
     }
+    if (landed) land(d);                                 // (one copy of the code that packs a landing)
     if (!cont) {
       if (pend) { fail(C, ST_OVERFLOW, f.node, -13); return nout; }          // a sum that found no landing
       if (sp > 0) f = stack[--sp];
@@ -1400,7 +1398,6 @@ __device__ __noinline__ void tile_main(const Ctx& C, DevPPT& P, const int tile, 
 // cached input x.  Its columns of the input gradient dx = W^T dpre are complete sums: they are stored, not added, into
 // the slot they land in.  A[:, cols] += dpre x[cols]^T.  After the update (Sec. 3) the tile writes its columns to the
 // parameter array in device memory and counts itself in the node's version counter; the forward row tiles reload.
-constexpr int MAXU = 1;                 // accumulator units (four output rows x four columns) per thread
 
 __device__ __noinline__ void bwd_tile_main(const Ctx& C, DevPPT& P, const int tile, float* smem, TileS& S, const unsigned long long t0) {
   IN_SMEM(&P); IN_SMEM(smem); IN_SMEM(&S);
