@@ -58,12 +58,12 @@ enum { LSTM_LEAF = 1, LSTM_BRANCH = 2 };
 enum NodeType { SOURCE, LINEAR, LOOKUP, GRUCELL, LOSS_CE, LOSS_MSE, NPT_SUMROWS, COND, PHI, ISU, CONCAT, SPLIT,
                 BCAST, GROUP, UNGROUP, FLATMAP, SINK, NPT_LSTM, N_TYPES };
 enum Act { ACT_NONE, ACT_RELU, ACT_TANH, ACT_SIGMOID };
-enum { SRC_DENSE_ROW = 1, SRC_TOKENS, SRC_ZERO_STATE, SRC_TREE_LEAVES, SRC_GRAPH_NODES };
+enum { SRC_DENSE_ROW = 1, SRC_TOKENS, SRC_ZERO_STATE, SRC_TREE_LEAVES, SRC_GRAPH_NODES, SRC_TREE_LEAVES_GROUPED };
 enum { COND_SEQ_END = 1, COND_TREE_ROOT, COND_BY_U, COND_IT_LT, COND_ROUND_ROBIN };
 enum { ISU_U_INC = 1, ISU_TREE_PARENT, ISU_IT_INC };
 enum { CONCAT_BY_EDGE = 1, CONCAT_BY_STATE_PORT };
 enum { GROUP_EDGES_BY_TYPE = 1, GROUP_EDGES_BY_DST, GROUP_ALL_NODES };
-enum { UNGROUP_NODES = 1, UNGROUP_TYPE_EDGES };
+enum { UNGROUP_NODES = 1, UNGROUP_TYPE_EDGES, UNGROUP_LEAVES };
 enum { FLATMAP_OUT_EDGES = 1 };
 enum { LABEL_PER_INSTANCE = 1, LABEL_PER_TREE_NODE };
 enum { FLAG_SOURCE_ADJACENT = 1 };
@@ -728,11 +728,16 @@ struct Ungroup : Node {
   size_t cache_size() const override { return orig.size() + part.size(); }
   int row_u(const State& s, int i) const {
     const Structure& S = E->S(s);
+    if (fn == UNGROUP_LEAVES) return S.leaves[i];            // Sec. 6, grouped leaf operations: row i is the tree's i-th leaf
     return fn == UNGROUP_TYPE_EDGES ? S.type_edges[s.u][i] : i;
   }
   std::pair<int, int> inverse(const State& s) const {      // (group u, row)
     const Structure& S = E->S(s);
     if (fn == UNGROUP_TYPE_EDGES) return {S.etype[s.u], S.rank_type[s.u]};
+    if (fn == UNGROUP_LEAVES) {
+      for (size_t k = 0; k < S.leaves.size(); k++) if (S.leaves[k] == s.u) return {0, (int)k};
+      return {0, -1};
+    }
     return {0, s.u};
   }
   void forward(Msg& m, int) override {
@@ -931,6 +936,11 @@ struct Oracle {
           std::vector<real> ids(S.n_pos);
           for (int v = 0; v < S.n_pos; v++) ids[v] = (real)S.tokens[v];
           send(0, S.n_pos, 1, ids);
+        } break;
+        case SRC_TREE_LEAVES_GROUPED: {                      // one matrix message: the leaves' tokens in leaf order
+          std::vector<real> ids(S.leaves.size());
+          for (size_t k = 0; k < S.leaves.size(); k++) ids[k] = (real)S.tokens[S.leaves[k]];
+          send(0, (int)S.leaves.size(), 1, ids);
         } break;
         default: E.err = "Source: unknown fn";
       }

@@ -120,7 +120,7 @@ def ggnn_loss(g, P, inst, i, steps=4):
     return (y[0] - float(inst.labels_f[i])) ** 2
 
 
-LOSS_FNS = {"mlp": mlp_loss, "rnn": rnn_loss, "tree": tree_loss, "ggnn": ggnn_loss, "tree_lstm": tree_lstm_loss}
+LOSS_FNS = {"mlp": mlp_loss, "rnn": rnn_loss, "tree": tree_loss, "tree_grouped": tree_loss, "ggnn": ggnn_loss, "tree_lstm": tree_lstm_loss}
 
 
 def dataset_grad(g, params, inst):
@@ -144,6 +144,9 @@ def tiny_case(family, n=3, seed=0):
         inst = data.list_instances(n=n, max_len=4)
     elif family == "tree":
         g = ir.tree(vocab=12, emb=5, hidden=4, classes=3)
+        inst = data.tree_instances(n=n, min_leaves=2, max_leaves=5, vocab=12, classes=3)
+    elif family == "tree_grouped":
+        g = ir.tree(vocab=12, emb=5, hidden=4, classes=3, grouped_leaves=True)
         inst = data.tree_instances(n=n, min_leaves=2, max_leaves=5, vocab=12, classes=3)
     elif family == "tree_lstm":
         g = ir.tree_lstm(vocab=12, emb=5, hidden=4, classes=3)
@@ -175,7 +178,7 @@ def _logit_rows(g, P, inst, i):
         for t in inst.tokens[inst.offsets[i]:inst.offsets[i + 1]]:
             h = act(int(g.nodes[l1][3]), P[(l1, 0)] @ torch.cat([P[(look, 0)][int(t)], h]) + P[(l1, 1)])
         return [(P[(l2, 0)] @ h + P[(l2, 1)], int(inst.labels_i[i]))]
-    assert name == "tree"
+    assert name in ("tree", "tree_grouped")
     look, leaf, br, cls = (g.index(k) for k in ("lookup", "leaf_cell", "branch_cell", "classifier"))
     o = int(inst.offsets[i])
     rows = []

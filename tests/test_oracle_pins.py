@@ -39,6 +39,32 @@ def test_accumulators_equal_autograd_of_direct_formulation(oracle_mod, family):
     assert st.leftover_cache_entries == 0
 
 
+def test_grouped_leaves_give_the_gradients_and_message_count_of_the_recursion(oracle_mod):
+    """The tree IR with the leaf operations of a tree grouped into one matrix message (Sec. 6): the same losses and
+    gradients as the direct recursion over the tree (which knows nothing of the IR), the caches empty at the end, and
+    the node-message count that follows from the graph: Lookup, LeafCell and Ungroup take one forward message per tree
+    instead of two per leaf (3 - 2L), backward the Ungroup takes L and the other two one each instead of 2L (2 - L):
+    33L - 18 becomes 30L - 13."""
+    g, inst, p = H.tiny_case("tree_grouped", n=5)
+    o = make(oracle_mod, g, inst, p)
+    st, loss = o.run_epoch(mak=2, muf=BIG, lr=0.1, flush=False)
+    grads, losses = H.dataset_grad(g, p, inst)
+    np.testing.assert_allclose(loss, losses, rtol=1e-12, atol=1e-13)
+    for (node, which), gr in grads.items():
+        np.testing.assert_allclose(o.get_accum(node, which), gr, rtol=1e-9, atol=1e-12, err_msg=g.names[node])
+    L = (np.diff(inst.offsets) + 1) // 2
+    assert st.node_messages == int((30 * L - 13).sum()) and st.leftover_cache_entries == 0
+    # one flush of the whole set from the same start: the same step as with the ungrouped IR (a gradient is one payload row)
+    g0, _, _ = H.tiny_case("tree", n=5)
+    o0, o1 = make(oracle_mod, g0, inst, p), make(oracle_mod, g, inst, p)
+    o0.run_epoch(mak=2, muf=BIG, lr=0.1)
+    o1.run_epoch(mak=2, muf=BIG, lr=0.1)
+    p0, p1 = o0.get_params(), o1.get_params()
+    for k in p0:
+        np.testing.assert_allclose(p1[k], p0[k], rtol=1e-12, atol=1e-14)
+        assert o1.node_stats(k[0])["n_grads_applied"] == o0.node_stats(k[0])["n_grads_applied"]
+
+
 @pytest.mark.parametrize("family", FAMILIES)
 def test_accumulators_equal_finite_differences(oracle_mod, family):
     """Central differences of the independent loss; touches every parameter tensor."""

@@ -40,6 +40,7 @@ SRC_TOKENS = 2         # one message per token position u = 0..T-1 (payload = to
 SRC_ZERO_STATE = 3     # one message, zero payload of width out_dim (initial hidden state)
 SRC_TREE_LEAVES = 4    # one message per leaf u of the tree (payload = leaf token id)
 SRC_GRAPH_NODES = 5    # one message with N rows (payload = node type ids)
+SRC_TREE_LEAVES_GROUPED = 6   # one message with L rows: the tokens of the tree's leaves in leaf order (Sec. 6: grouped leaf operations)
 # COND.fn: successor index as a function of the state
 COND_SEQ_END = 1       # u < T ? 0 : 1          (T = number of tokens of the instance)
 COND_TREE_ROOT = 2     # u is the root ? 0 : 1
@@ -60,6 +61,7 @@ GROUP_ALL_NODES = 3       # u = node id -> key = 0,       member = u, count = N
 # UNGROUP.fn: state of row i of an incoming matrix message
 UNGROUP_NODES = 1         # row i -> u = i
 UNGROUP_TYPE_EDGES = 2    # u = type c, row i -> u = id of the i-th edge of type c
+UNGROUP_LEAVES = 3        # row i -> u = position of the tree's i-th leaf
 # FLATMAP.fn
 FLATMAP_OUT_EDGES = 1     # u = node v -> one message per out-edge e of v, u = e
 # LOSS.fn: where the label comes from
@@ -224,11 +226,14 @@ def tree_lstm(vocab=20000, emb=300, hidden=150, classes=5):
     return g
 
 
-def tree(vocab=20000, emb=300, hidden=150, classes=5):
+def tree(vocab=20000, emb=300, hidden=150, classes=5, grouped_leaves=False):
     """Binary tree RNN: Lookup -> LeafCell -> Phi <- BranchCell; Phi -> Bcast -> {Classifier -> Loss,
-    Cond(root ? Sink : Isu(parent) -> Concat(left,right) -> BranchCell)}.  33L-18 node-messages for L leaves."""
-    g = IRGraph("tree")
-    src = g.node("src_leaves", SOURCE, fn=SRC_TREE_LEAVES)
+    Cond(root ? Sink : Isu(parent) -> Concat(left,right) -> BranchCell)}.  33L-18 node-messages for L leaves.
+    grouped_leaves (Sec. 6: the leaf operations of a tree grouped into one call): the controller pumps one message whose
+    rows are the tokens of the tree's leaves, Lookup and LeafCell work on that matrix, and an Ungroup in front of the
+    Phi hands every leaf its row (backward: it collects the leaves' gradients into one matrix message)."""
+    g = IRGraph("tree_grouped" if grouped_leaves else "tree")
+    src = g.node("src_leaves", SOURCE, fn=SRC_TREE_LEAVES_GROUPED if grouped_leaves else SRC_TREE_LEAVES)
     look = g.node("lookup", LOOKUP, vocab, emb, flags=FLAG_SOURCE_ADJACENT)
     leaf = g.node("leaf_cell", LINEAR, emb, hidden, act=ACT_TANH)
     phi = g.node("phi", PHI, hidden, hidden)
@@ -242,7 +247,12 @@ def tree(vocab=20000, emb=300, hidden=150, classes=5):
     br = g.node("branch_cell", LINEAR, 2 * hidden, hidden, act=ACT_TANH)
     g.edge(src, look)
     g.edge(look, leaf)
-    g.edge(leaf, phi, 0, 0)
+    if grouped_leaves:
+        ung = g.node("ungroup_leaves", UNGROUP, hidden, hidden, fn=UNGROUP_LEAVES)
+        g.edge(leaf, ung)
+        g.edge(ung, phi, 0, 0)
+    else:
+        g.edge(leaf, phi, 0, 0)
     g.edge(br, phi, 0, 1)
     g.edge(phi, bc)
     g.edge(bc, cls, 0, 0)
