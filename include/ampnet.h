@@ -65,7 +65,8 @@ enum {
 enum { AMPNET_ACT_NONE = 0, AMPNET_ACT_RELU = 1, AMPNET_ACT_TANH = 2, AMPNET_ACT_SIGMOID = 3 };
 /* state functions; the message state is (inst, seq, slot, it, u, port)                                     */
 enum { AMPNET_SRC_DENSE_ROW = 1, AMPNET_SRC_TOKENS = 2, AMPNET_SRC_ZERO_STATE = 3, AMPNET_SRC_TREE_LEAVES = 4,
-       AMPNET_SRC_GRAPH_NODES = 5 };
+       AMPNET_SRC_GRAPH_NODES = 5,
+       AMPNET_SRC_TREE_LEAVES_GROUPED = 6 }; /* one message with L rows: the tokens of the tree's leaves in leaf order (Sec. 6) */
 enum { AMPNET_LSTM_LEAF = 1,   /* [pi, po, pu] (3H): c = s(pi) tanh(pu), h = s(po) tanh(c)                                   */
        AMPNET_LSTM_BRANCH = 2 }; /* [pi, pfL, pfR, po, pu] (5H), [cL; cR]: c = s(pi) tanh(pu) + s(pfL) cL + s(pfR) cR, h = s(po) tanh(c) */
 enum { AMPNET_COND_SEQ_END = 1,   /* u < #tokens ? 0 : 1        */
@@ -76,7 +77,8 @@ enum { AMPNET_COND_SEQ_END = 1,   /* u < #tokens ? 0 : 1        */
 enum { AMPNET_ISU_U_INC = 1, AMPNET_ISU_TREE_PARENT = 2, AMPNET_ISU_IT_INC = 3 };
 enum { AMPNET_CONCAT_BY_EDGE = 1, AMPNET_CONCAT_BY_STATE_PORT = 2 };
 enum { AMPNET_GROUP_EDGES_BY_TYPE = 1, AMPNET_GROUP_EDGES_BY_DST = 2, AMPNET_GROUP_ALL_NODES = 3 };
-enum { AMPNET_UNGROUP_NODES = 1, AMPNET_UNGROUP_TYPE_EDGES = 2 };
+enum { AMPNET_UNGROUP_NODES = 1, AMPNET_UNGROUP_TYPE_EDGES = 2,
+       AMPNET_UNGROUP_LEAVES = 3 };  /* row i -> u = position of the tree's i-th leaf */
 enum { AMPNET_FLATMAP_OUT_EDGES = 1 };
 enum { AMPNET_LABEL_PER_INSTANCE = 1, AMPNET_LABEL_PER_TREE_NODE = 2 };
 enum { AMPNET_FLAG_SOURCE_ADJACENT = 1 }; /* PPT fed directly by a SOURCE: no input gradient, retire instead */
@@ -116,6 +118,12 @@ ampnet_status_t ampnet_ir_tree_lstm(int32_t vocab, int32_t emb, int32_t hidden, 
 ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
                                ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
                                ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
+/* the tree model with the leaf operations of a tree grouped into one call (Sec. 6): the controller pumps one message whose
+ * rows are the leaves' tokens, LOOKUP and the leaf cell work on that matrix (at most 64 leaves per tree), an UNGROUP in
+ * front of the PHI hands every leaf its row and, backward, collects the leaves' gradients into one matrix message.   */
+ampnet_status_t ampnet_ir_tree_grouped(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
+                                       ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                                       ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);
 ampnet_status_t ampnet_ir_ggnn(int32_t n_node_types, int32_t hidden, int32_t steps, int32_t n_edge_types, int32_t readout,
                                ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
                                ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges);

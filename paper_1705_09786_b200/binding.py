@@ -13,7 +13,7 @@ EXPORTS = ["ampnet_graph_create", "ampnet_graph_destroy", "ampnet_load_instances
            "ampnet_param_count", "ampnet_get_params", "ampnet_set_params", "ampnet_get_node_stats",
            "ampnet_get_update_log", "ampnet_get_key_log", "ampnet_leftover_cache_entries", "ampnet_get_placement",
            "ampnet_last_error", "ampnet_set_optimizer", "ampnet_average_params", "ampnet_ir_rnn_replicated", "ampnet_run_epoch_mixed", "ampnet_param_device_ptr", "ampnet_run_epoch_static", "ampnet_get_phase_cycles", "ampnet_get_queue_occupancy", "ampnet_get_micro_batch_split", "ampnet_ir_mlp", "ampnet_ir_rnn",
-           "ampnet_ir_tree", "ampnet_ir_ggnn", "ampnet_ir_tree_lstm", "ampnet_measure_fma_peak"]
+           "ampnet_ir_tree", "ampnet_ir_tree_grouped", "ampnet_ir_ggnn", "ampnet_ir_tree_lstm", "ampnet_measure_fma_peak"]
 
 
 class InferenceStats(C.Structure):
@@ -110,6 +110,7 @@ def load_library():
     lib.ampnet_run_epoch_mixed.argtypes = [P, P, P, P, P, P]
     lib.ampnet_param_device_ptr.argtypes = [P, C.c_int32, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64)]
     lib.ampnet_ir_tree.argtypes = [I32] * 4 + tail
+    lib.ampnet_ir_tree_grouped.argtypes = [I32] * 4 + tail
     lib.ampnet_ir_tree_lstm.argtypes = [I32] * 4 + tail
     lib.ampnet_measure_fma_peak.argtypes = [C.c_int32, C.POINTER(C.c_double)]
     lib.ampnet_ir_ggnn.argtypes = [I32] * 5 + tail

@@ -250,7 +250,7 @@ ampnet_status_t build_topology(ampnet_graph* g) {
     ampnet_status_t st = AMPNET_OK;
     switch (h.type) {
       case SOURCE:
-        st = need(h.n_pred == 0 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 5, "SOURCE needs one successor and a valid fn");
+        st = need(h.n_pred == 0 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 6, "SOURCE needs one successor and a valid fn");
         if (st == AMPNET_OK) g->sources.push_back(i);
         break;
       case LINEAR:
@@ -287,7 +287,7 @@ ampnet_status_t build_topology(ampnet_graph* g) {
                   "SPLIT needs fn_arg successors of width in_dim / fn_arg");
         break;
       case GROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 3, "GROUP needs a valid fn"); break;
-      case UNGROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 2, "UNGROUP needs a valid fn"); break;
+      case UNGROUP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn >= 1 && h.fn <= 3, "UNGROUP needs a valid fn"); break;
       case FLATMAP: st = need(h.n_pred == 1 && h.n_succ == 1 && h.fn == 1, "FLATMAP needs a valid fn"); break;
       case NPT_SUMROWS: st = need(h.n_pred == 1 && h.n_succ == 1, "NPT_SUMROWS needs one predecessor and one successor"); break;
       case NPT_LSTM:
@@ -387,6 +387,7 @@ void infer_domains(ampnet_graph* g, const HostDataset& D) {
           if (h.fn == 2) o = Dom{D.maxT + 1, 1};
           else if (h.fn == 4) o = Dom{D.maxM, 1};
           else if (h.fn == 5) o = Dom{1, D.maxN};
+          else if (h.fn == 6) o = Dom{1, D.maxL};          // the leaves of a tree as the rows of one message
           else o = Dom{1, 1};
           break;
         case FLATMAP: o = Dom{D.maxD, 1}; break;
@@ -395,7 +396,7 @@ void infer_domains(ampnet_graph* g, const HostDataset& D) {
           else if (h.fn == 2) o = Dom{D.maxN, D.maxIn};
           else o = Dom{1, D.maxN};
           break;
-        case UNGROUP: o = h.fn == 2 ? Dom{D.maxD, 1} : Dom{D.maxN, 1}; break;
+        case UNGROUP: o = h.fn == 2 ? Dom{D.maxD, 1} : h.fn == 3 ? Dom{D.maxM, 1} : Dom{D.maxN, 1}; break;
         case NPT_SUMROWS: o = Dom{a.U, 1}; break;
         default: break;
       }
@@ -1298,7 +1299,7 @@ ampnet_status_t ampnet_load_instances(ampnet_graph_t* g, int32_t split, const am
   }
   for (int s : g->sources) {
     const int fn = g->hnodes[s].fn;
-    const int want = fn == 1 ? 0 : fn == 2 ? 1 : fn == 4 ? 2 : fn == 5 ? 3 : -1;
+    const int want = fn == 1 ? 0 : fn == 2 ? 1 : (fn == 4 || fn == 6) ? 2 : fn == 5 ? 3 : -1;
     if (want >= 0 && want != in->kind) return set_err(g, AMPNET_EINVAL, "instance kind %d does not match the graph's source (fn %d)", in->kind, fn);
     if (fn == 1 && g->hnodes[s].out_dim != in->dense_dim) return set_err(g, AMPNET_EINVAL, "dense_dim %d does not match the source width %d", in->dense_dim, g->hnodes[s].out_dim);
   }

@@ -599,7 +599,7 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
               if (!pool_offer(C, Q, c, lane)) { if (sp >= WALK_STACK) { fail(C, ST_OVERFLOW, f.node, sp); return; }
                                              if (lane == 0) stack[sp] = c; sp++; __syncwarp(); } }
             f.nparts = 1; f.part = 0;
-            int mu = n.fn == 2 ? I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i] : i;
+            int mu = n.fn == 2 ? I.type_list[I.type_off[(long long)f.inst * I.NT + f.u] + i] : n.fn == 3 ? I.leaf_ids[I.leaf_off[f.inst] + i] : i;
             f.p = f.p ? f.p + (size_t)i * f.ld : nullptr; f.rows = 1; f.u = mu;
             to_succ(f, n, 0);
             cont = true;
@@ -607,6 +607,14 @@ __device__ __noinline__ void walk(const Ctx& C, Frame f, Frame* stack, WalkAcc& 
             int gkey, row, expected;
             if (n.fn == 2) { const long long ebase = f.ebase; gkey = I.etype[ebase + f.u]; row = I.rank_type[ebase + f.u];
                              const long long* to = I.type_off + (long long)f.inst * I.NT + gkey; expected = (int)(to[1] - to[0]); }
+            else if (n.fn == 3) {                   // the leaf's rank among the leaves of its tree (their positions ascend)
+              const long long l0 = I.leaf_off[f.inst];
+              expected = (int)(I.leaf_off[f.inst + 1] - l0);
+              int lo = 0, hi = expected - 1;
+              while (lo < hi) { const int mid = (lo + hi) >> 1; if (I.leaf_ids[l0 + mid] < f.u) lo = mid + 1; else hi = mid; }
+              if (expected < 1 || I.leaf_ids[l0 + lo] != f.u) { fail(C, ST_OVERFLOW, f.node, f.u); return; }
+              gkey = 0; row = lo;
+            }
             else { gkey = 0; row = f.u; expected = (int)(I.offsets[f.inst + 1] - f.ibase); }
             long long key = key_of(C, f.node, f.slot, f.it, gkey, n.U_in);
             if (key < 0) return;
@@ -1363,8 +1371,10 @@ __device__ __noinline__ void load_batch_ctx(const Ctx& C, DevPPT& P, TileShared&
       const DevInst& I = C.inst;
       const long long base = I.offsets[h[j].inst];
       const float* g0 = P.gbuf + (size_t)key * P.rows_max * P.out_dim;
+      const DevNode& feeder = g_nodes[g_nodes[P.node].pred_node[0]];
+      const bool by_leaf = feeder.type == SOURCE && feeder.fn == 6;      // row r is the tree's r-th leaf
       for (int r = 0; r < rows[j]; r++) {
-        const int id = I.tokens[base + (I.kind == 3 ? r : h[j].u)];
+        const int id = I.tokens[base + (I.kind == 3 ? r : by_leaf ? I.leaf_ids[I.leaf_off[h[j].inst] + r] : h[j].u)];
         S.rowmsg[off + r] = i; S.rowptr[off + r] = g0 + (size_t)r * P.out_dim;
         S.rowid[off + r] = (unsigned)id < (unsigned)in ? id : -1;
       }
@@ -2323,6 +2333,7 @@ __device__ __noinline__ void controller_main(const Ctx& C, CtrlShared& S, const 
           case 3: f.dim = sn.out_dim; f.ld = sn.out_dim; break;
           case 4: f.u = I.leaf_ids[I.leaf_off[inst] + k]; break;
           case 5: f.rows = (int)(I.offsets[inst + 1] - I.offsets[inst]); break;
+          case 6: f.rows = (int)(I.leaf_off[inst + 1] - I.leaf_off[inst]); break;      // the tree's leaves as the rows of one message
         }
         walk(C, f, S.stack[warp], acc, &S.pool);
         __syncwarp();

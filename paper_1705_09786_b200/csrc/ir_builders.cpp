@@ -98,12 +98,12 @@ ampnet_status_t ampnet_ir_rnn_replicated(int32_t vocab, int32_t emb, int32_t hid
   return b.emit(nodes, cap_nodes, n_nodes, edges, cap_edges, n_edges);
 }
 
-ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
+static ampnet_status_t tree_ir(bool grouped, int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
                                ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
                                ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges) {
   if (vocab < 1 || emb < 1 || hidden < 1 || classes < 1) return AMPNET_EINVAL;
   Builder b;
-  int src = b.node(AMPNET_SOURCE, 0, 0, 0, AMPNET_SRC_TREE_LEAVES);
+  int src = b.node(AMPNET_SOURCE, 0, 0, 0, grouped ? AMPNET_SRC_TREE_LEAVES_GROUPED : AMPNET_SRC_TREE_LEAVES);
   int look = b.node(AMPNET_LOOKUP, vocab, emb, 0, 0, 0, AMPNET_FLAG_SOURCE_ADJACENT);
   int leaf = b.node(AMPNET_LINEAR, emb, hidden, AMPNET_ACT_TANH);
   int phi = b.node(AMPNET_PHI, hidden, hidden);
@@ -117,7 +117,11 @@ ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32
   int br = b.node(AMPNET_LINEAR, 2 * hidden, hidden, AMPNET_ACT_TANH);
   b.edge(src, look);
   b.edge(look, leaf);
-  b.edge(leaf, phi, 0, 0);
+  if (grouped) {                       // (the extra node comes last, so that the other nodes keep their indices)
+    int ung = b.node(AMPNET_UNGROUP, hidden, hidden, 0, AMPNET_UNGROUP_LEAVES);
+    b.edge(leaf, ung);
+    b.edge(ung, phi, 0, 0);
+  } else b.edge(leaf, phi, 0, 0);
   b.edge(br, phi, 0, 1);
   b.edge(phi, bc);
   b.edge(bc, cls, 0, 0);
@@ -128,6 +132,18 @@ ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32
   b.edge(isu, cat);
   b.edge(cat, br);
   return b.emit(nodes, cap_nodes, n_nodes, edges, cap_edges, n_edges);
+}
+
+ampnet_status_t ampnet_ir_tree(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
+                               ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                               ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges) {
+  return tree_ir(false, vocab, emb, hidden, classes, nodes, cap_nodes, n_nodes, edges, cap_edges, n_edges);
+}
+
+ampnet_status_t ampnet_ir_tree_grouped(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,
+                                       ampnet_node_desc_t* nodes, int32_t cap_nodes, int32_t* n_nodes,
+                                       ampnet_edge_desc_t* edges, int32_t cap_edges, int32_t* n_edges) {
+  return tree_ir(true, vocab, emb, hidden, classes, nodes, cap_nodes, n_nodes, edges, cap_edges, n_edges);
 }
 
 ampnet_status_t ampnet_ir_tree_lstm(int32_t vocab, int32_t emb, int32_t hidden, int32_t classes,

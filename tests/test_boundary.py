@@ -42,6 +42,7 @@ def test_enum_codes_agree_with_the_input_module():
              "CONCAT": ir.CONCAT, "SPLIT": ir.SPLIT, "BCAST": ir.BCAST, "GROUP": ir.GROUP, "UNGROUP": ir.UNGROUP,
              "FLATMAP": ir.FLATMAP, "SINK": ir.SINK, "NPT_LSTM": ir.NPT_LSTM, "LSTM_LEAF": ir.LSTM_LEAF, "LSTM_BRANCH": ir.LSTM_BRANCH, "ACT_TANH": ir.ACT_TANH, "ACT_SIGMOID": ir.ACT_SIGMOID,
              "SRC_GRAPH_NODES": ir.SRC_GRAPH_NODES, "SRC_TREE_LEAVES": ir.SRC_TREE_LEAVES,
+             "SRC_TREE_LEAVES_GROUPED": ir.SRC_TREE_LEAVES_GROUPED, "UNGROUP_LEAVES": ir.UNGROUP_LEAVES,
              "COND_IT_LT": ir.COND_IT_LT, "COND_BY_U": ir.COND_BY_U, "COND_ROUND_ROBIN": ir.COND_ROUND_ROBIN, "ISU_TREE_PARENT": ir.ISU_TREE_PARENT,
              "ISU_IT_INC": ir.ISU_IT_INC, "CONCAT_BY_STATE_PORT": ir.CONCAT_BY_STATE_PORT,
              "GROUP_ALL_NODES": ir.GROUP_ALL_NODES, "GROUP_EDGES_BY_DST": ir.GROUP_EDGES_BY_DST,
@@ -86,7 +87,8 @@ def test_library_ir_builders_emit_the_canonical_graphs(lib):
     import paper_1705_09786_b200 as amp
     from workloads import ir
     cases = [("mlp", ([784, 256, 256, 10],), ir.mlp()), ("mlp", ([5, 3],), ir.mlp((5, 3))),
-             ("rnn", (14, 128, 128, 10, ir.ACT_TANH), ir.rnn()), ("tree", (20000, 300, 150, 5), ir.tree()), ("tree_lstm", (20000, 300, 150, 5), ir.tree_lstm()),
+             ("rnn", (14, 128, 128, 10, ir.ACT_TANH), ir.rnn()), ("tree", (20000, 300, 150, 5), ir.tree()), ("tree_grouped", (20000, 300, 150, 5), ir.tree(grouped_leaves=True)),
+             ("tree_lstm", (20000, 300, 150, 5), ir.tree_lstm()),
              ("rnn_replicated", (14, 128, 128, 10, ir.ACT_TANH, 1), ir.rnn()),
              ("rnn_replicated", (14, 16, 16, 10, ir.ACT_TANH, 3), ir.rnn(14, 16, 16, 10, replicas=3)),
              ("ggnn", (15, 100, 4, 4, 100), ir.ggnn()), ("ggnn", (7, 8, 2, 3, 5), ir.ggnn(7, 8, 2, 3, 5))]

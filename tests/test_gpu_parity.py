@@ -465,6 +465,38 @@ def test_asynchronous_flushes_with_momentum_and_adam_match_oracle(oracle_mod, fa
     e.close()
 
 
+@pytest.mark.parametrize("n,mak,muf,lr", [(24, 1, 1, 0.002), (40, 64, 100, 0.05), (31, 6, 7, 0.01)])
+def test_tree_with_grouped_leaves_matches_oracle(oracle_mod, n, mak, muf, lr):
+    """The tree IR with the leaf operations of a tree grouped into one matrix message (Sec. 6): the deterministic schedule
+    against the oracle (routing, keys, update counts bit-exact), then an asynchronous epoch with exact accounting
+    (30L - 13 node messages per tree, one gradient per leaf at the embedding and the leaf cell) and, with no update before
+    the flush, the oracle's losses and parameters whatever the order of execution."""
+    import paper_1705_09786_b200 as amp
+    g = ir.tree(grouped_leaves=True)
+    inst = data.tree_instances(n=n)
+    p = wp.init_params(g)
+    r = parity.run_both(oracle_mod, g, inst, p, mak, muf, lr)
+    parity.assert_parity(g, *r)
+    e = r[3]
+    L = (np.diff(inst.offsets) + 1) // 2
+    e.set_params(p)
+    st, loss = e.run_epoch(mak=mak, muf=muf, lr=lr, deterministic=False, timeout_s=60)
+    assert st.node_messages == int((30 * L - 13).sum()) and e.leftover_cache_entries() == 0 and np.isfinite(loss).all()
+    for node, G in (("lookup", L.sum()), ("leaf_cell", L.sum()), ("branch_cell", (L - 1).sum()), ("classifier", (2 * L - 1).sum())):
+        assert e.node_stats(g.index(node))["n_grads_applied"] == G == e.update_log(g.index(node)).sum()
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst)
+    o.set_params(p)
+    _, oloss = o.run_epoch(mak=1, muf=1 << 30, lr=lr)
+    e.set_params(p)
+    st, eloss = e.run_epoch(mak=mak, muf=1 << 30, lr=lr, deterministic=False, timeout_s=60)
+    np.testing.assert_allclose(eloss, oloss, rtol=1e-5, atol=2e-6)
+    ep, op = e.get_params(), o.get_params()
+    for k in op:
+        assert np.abs(ep[k] - op[k]).max() / (np.abs(op[k]).max() + 1e-30) <= 1e-4, (g.names[k[0]], k[1])
+    e.close()
+
+
 def test_tree_with_256_keys_in_flight(oracle_mod):
     """The tree workload with more keys than the benchmark uses (every instance of the set in flight at once)."""
     g, inst = _case("tree", 300)
