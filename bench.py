@@ -31,6 +31,8 @@ WORKLOADS = {
     "rnn": (ir.rnn, data.list_instances, 20000, 16, 50, 0.05),
     "tree": (ir.tree, data.tree_instances, 8544, 64, 100, 0.05),
     "ggnn": (ir.ggnn, data.graph_instances, 130000, 128, 200, 0.01),
+    # the tree model with the leaf operations of a tree grouped into one matrix message (Sec. 6); runs on the interpreter engine
+    "tree_grouped": (lambda: ir.tree(grouped_leaves=True), data.tree_instances, 8544, 64, 100, 0.05),
     # the paper's sentiment model proper: binary Tree-LSTM (leaf and branch cells) on the same trees as "tree"
     "tree_lstm": (ir.tree_lstm, data.tree_instances, 8544, 64, 100, 0.05),
     # throughput stress: binary tree RNN, hidden 512, 64..512 leaves, bf16 messages with fp32 accumulators

@@ -42,7 +42,7 @@ def gradient_rows(graph, inst):
     if name == "rnn":
         T = int(np.diff(inst.offsets).sum())
         return {graph.index("lookup"): T, graph.index("linear1"): T, graph.index("linear2"): inst.n}
-    if name == "tree":
+    if name in ("tree", "tree_grouped"):                   # (grouping changes the messages, not the payload rows)
         L = (np.diff(inst.offsets) + 1) // 2
         return {graph.index("lookup"): int(L.sum()), graph.index("leaf_cell"): int(L.sum()),
                 graph.index("branch_cell"): int((L - 1).sum()), graph.index("classifier"): int((2 * L - 1).sum())}

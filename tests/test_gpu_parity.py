@@ -494,6 +494,15 @@ def test_tree_with_grouped_leaves_matches_oracle(oracle_mod, n, mak, muf, lr):
     ep, op = e.get_params(), o.get_params()
     for k in op:
         assert np.abs(ep[k] - op[k]).max() / (np.abs(op[k]).max() + 1e-30) <= 1e-4, (g.names[k[0]], k[1])
+    # forward only (evaluation split): losses and accuracy
+    o.load_instances(inst, split=1)
+    e.load_instances(inst, split=1)
+    o.set_params(p)
+    e.set_params(p)
+    oml, oacc, oloss = o.eval(split=1)
+    eml, eacc, eloss = e.eval(split=1, mak=16)
+    np.testing.assert_allclose(eloss, oloss, rtol=1e-5, atol=2e-6)
+    assert eacc == pytest.approx(oacc, abs=1e-12) and e.leftover_cache_entries() == 0
     e.close()
 
 
