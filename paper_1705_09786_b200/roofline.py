@@ -12,9 +12,9 @@ from workloads import ir   # integer codes of the IR format only
 SM_COUNT = 148             # B200: 2 dies x 74 SMs
 # dram__bytes_read.sum + dram__bytes_write.sum of the persistent kernel per instance, from the ncu captures summarised
 # under profiles/ (captured on a small case; traffic grows in proportion to the instances processed): the tree workload
-# on ampnet_engine_direct (600 trees: 14.15 + 15.80 MB), the graph workload on ampnet_engine (1,000 graphs), the stress
+# on ampnet_engine_direct (600 trees: 14.31 + 16.74 MB), the graph workload on ampnet_engine (1,000 graphs), the stress
 # configuration on ampnet_engine_direct (60 trees: 328.2 + 391.2 MB)
-MEASURED_DRAM_BYTES_PER_INSTANCE = {"tree": 49924.0, "ggnn": 858646.0, "stress": 11989589.0}
+MEASURED_DRAM_BYTES_PER_INSTANCE = {"tree": 51753.0, "ggnn": 858646.0, "stress": 11989589.0}
 FP32_LANES_PER_SM = 128
 
 
