@@ -506,6 +506,33 @@ def test_tree_with_grouped_leaves_matches_oracle(oracle_mod, n, mak, muf, lr):
     e.close()
 
 
+@pytest.mark.parametrize("k,mak", [(2, 16), (4, 64)])
+def test_replicated_linear_asynchronous_epoch_without_updates_matches_oracle(oracle_mod, k, mak):
+    """Replicas of Linear-1 (Sec. 5: round-robin Cond and a Phi around the copies) on the asynchronous path, where the
+    schedule cannot matter: which copy a token goes to follows from (instance + position), so with no update before the
+    flush every copy collects the same gradients in any order of execution."""
+    import paper_1705_09786_b200 as amp
+    g = ir.rnn(replicas=k)
+    inst = data.list_instances(n=150)
+    p = wp.init_params(g)
+    o = oracle_mod.Oracle(g)
+    o.load_instances(inst)
+    o.set_params(p)
+    _, oloss = o.run_epoch(mak=1, muf=1 << 30, lr=0.05)
+    e = amp.Engine(g)
+    e.load_instances(inst)
+    e.set_params(p)
+    st, eloss = e.run_epoch(mak=mak, muf=1 << 30, lr=0.05, deterministic=False, timeout_s=60)
+    np.testing.assert_allclose(eloss, oloss, rtol=1e-5, atol=2e-6)
+    ep, op = e.get_params(), o.get_params()
+    for key in op:
+        assert np.abs(ep[key] - op[key]).max() / (np.abs(op[key]).max() + 1e-30) <= 1e-4, (g.names[key[0]], key[1])
+    for i in g.ppt_nodes():
+        assert e.node_stats(i)["n_grads_applied"] == o.node_stats(i)["n_grads_applied"]
+    assert e.leftover_cache_entries() == 0
+    e.close()
+
+
 def test_tree_with_256_keys_in_flight(oracle_mod):
     """The tree workload with more keys than the benchmark uses (every instance of the set in flight at once)."""
     g, inst = _case("tree", 300)
