@@ -111,9 +111,21 @@ class ClockSampler(threading.Thread):
 
     def __init__(self, index):
         super().__init__(daemon=True)
-        self.index, self.samples, self.stop_flag = index, [], threading.Event()
+        self.index, self.samples, self.stop_flag, self.proc = index, [], threading.Event(), None
 
     def run(self):
+        # one nvidia-smi process that prints a line every 100 ms (starting a process per sample takes longer than that)
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i", str(self.index),
+                                          "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            for line in self.proc.stdout:
+                if self.stop_flag.is_set():
+                    break
+                if line.strip():
+                    self.samples.append([v.strip() for v in line.strip().split(",")])
+            return
+        except Exception:
+            self.proc = None
         while not self.stop_flag.is_set():
             try:
                 out = subprocess.run(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-i",
@@ -126,6 +138,9 @@ class ClockSampler(threading.Thread):
 
     def summary(self):
         self.stop_flag.set()
+        proc = getattr(self, "proc", None)
+        if proc is not None and proc.poll() is None:
+            proc.terminate()                                   # (the process this sampler started, nothing else)
         self.join(timeout=6)
         sm = [float(s[0]) for s in self.samples if s and s[0].replace(".", "").isdigit()]
         mx = [float(s[1]) for s in self.samples if len(s) > 1 and s[1].replace(".", "").isdigit()]
